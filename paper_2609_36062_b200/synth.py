@@ -1,0 +1,111 @@
+"""Seeded synthetic inputs shaped like the paper's prefill workloads.
+
+This module holds no arithmetic of the method: it only draws Q, K, V (and an upstream
+gradient dO) from a counter-based generator and rounds them to the storage dtype.  It is
+the single piece that both the CUDA path and the CPU oracle's tests read, so that the
+two see identical bytes.
+
+Recipe.  Every (tensor, batch·head) pair owns its own Philox stream keyed by
+(seed, tensor id, head index), so one head can be regenerated without the others.
+  * "scaled":     Q, K, V iid N(0,1)/sqrt(d)                         (fp32 small case)
+  * "normalised": Q, K iid N(0,1)/sqrt(d_k), then every row L2-normalised in fp32;
+                  V iid N(0,1)
+  * dO iid N(0,1)
+bf16 storage rounds the fp32 values once, to nearest even; the oracle widens exactly
+those rounded values to fp64.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+_TENSOR_ID = {"q": 0, "k": 1, "v": 2, "do": 3}
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    d: int            # VC dimension of the mask family member
+    batch: int
+    heads: int
+    T: int
+    d_k: int
+    d_v: int
+    chunk: int
+    dtype: str        # "f32" or "bf16"
+    recipe: str       # "scaled" or "normalised"
+    seed: int
+    backward: bool = False
+
+    @property
+    def bh(self) -> int:
+        return self.batch * self.heads
+
+    @property
+    def tokens(self) -> int:
+        return self.batch * self.T
+
+
+# The five benchmark configurations (index 0 is the small case an fp64 CPU check finishes in seconds).
+WORKLOADS = {
+    "small_d2":      Workload("small_d2", 2, 1, 1, 512, 64, 64, 64, "f32", "scaled", 0),
+    "small_d1":      Workload("small_d1", 1, 1, 1, 512, 64, 64, 64, "f32", "scaled", 0),
+    "t4k_d3":        Workload("t4k_d3", 3, 4, 8, 4096, 128, 128, 64, "bf16", "normalised", 1),
+    "t16k_d4":       Workload("t16k_d4", 4, 2, 16, 16384, 128, 128, 128, "bf16", "normalised", 2),
+    "t64k_d1":       Workload("t64k_d1", 1, 1, 16, 65536, 128, 128, 128, "bf16", "normalised", 3),
+    "t64k_d2":       Workload("t64k_d2", 2, 1, 16, 65536, 128, 128, 128, "bf16", "normalised", 3),
+    "t64k_d3":       Workload("t64k_d3", 3, 1, 16, 65536, 128, 128, 128, "bf16", "normalised", 3),
+    "t64k_d4":       Workload("t64k_d4", 4, 1, 16, 65536, 128, 128, 128, "bf16", "normalised", 3),
+    "t8k_d3_fwdbwd": Workload("t8k_d3_fwdbwd", 3, 8, 16, 8192, 128, 128, 64, "bf16", "normalised", 4, True),
+}
+
+
+def _stream(seed: int, tensor: str, head: int) -> np.random.Generator:
+    key = (int(seed) << 40) ^ (_TENSOR_ID[tensor] << 32) ^ int(head)
+    return np.random.Generator(np.random.Philox(key=key))
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """fp32 -> bf16 bit pattern (uint16), round to nearest even.  Inputs are finite."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    return ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_widen(b: np.ndarray) -> np.ndarray:
+    """bf16 bit pattern (uint16) -> the same value as fp32."""
+    return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def head_tensor(w: Workload, tensor: str, head: int, T: int | None = None) -> np.ndarray:
+    """fp32 values of one [T, dim] slice before storage rounding."""
+    T = w.T if T is None else T
+    dim = w.d_v if tensor in ("v", "do") else w.d_k
+    x = _stream(w.seed, tensor, head).standard_normal((T, dim), dtype=np.float32)
+    if tensor == "do":
+        return x
+    if w.recipe == "scaled":
+        return x * np.float32(1.0 / np.sqrt(dim))
+    if tensor in ("q", "k"):
+        x = x * np.float32(1.0 / np.sqrt(dim))
+        norm = np.sqrt(np.sum(x * x, axis=1, keepdims=True, dtype=np.float32))
+        return (x / norm).astype(np.float32)
+    return x
+
+
+def stored(w: Workload, tensor: str, head: int) -> np.ndarray:
+    """One head in its storage form: fp32 array, or uint16 array of bf16 bit patterns."""
+    x = head_tensor(w, tensor, head)
+    return x if w.dtype == "f32" else bf16_round(x)
+
+
+def as_float64(w: Workload, stored_head: np.ndarray) -> np.ndarray:
+    """The exact stored values widened to fp64 (what the oracle computes on)."""
+    if w.dtype == "f32":
+        return stored_head.astype(np.float64)
+    return bf16_widen(stored_head).astype(np.float64)
+
+
+def full_tensor(w: Workload, tensor: str) -> np.ndarray:
+    """All heads: shape [batch*heads, T, dim] in storage form."""
+    return np.stack([stored(w, tensor, h) for h in range(w.bh)])
