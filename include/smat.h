@@ -1,0 +1,152 @@
+/*
+ * smat.h — C boundary of the B200 chunkwise hard-routing SMat-Attention prefill.
+ *
+ * The library computes, for every (batch, head) independently,
+ *
+ *        O = (M^(d) ⊙ Q Kᵀ) V                                  [Sec. 2, augmented output with
+ *                                                                identity feature maps, no division]
+ *
+ * under the structured causal mask family M^(d) of Sec. 3 (block form, Eq. "blockform";
+ * point–hyperplane incidences over F_q^{d-1}, Eq. "Bcount", Eq. "Gdef"; positional
+ * assignment of profiles and types), without ever materialising M^(d): Algorithm 1
+ * (pool → tabulate → typed read ‖ chunk summaries → scan → per-chunk output) with the
+ * implicit incidence tabulation of Algorithm 2, and the matching backward pass of the
+ * chunking proof (Eq. "lr-adjoint", Eq. "local-adjoint", suffix scan).
+ *
+ * Conventions shared by all entry points
+ *   - Plain C linkage; no exceptions; the library keeps no global mutable state.
+ *   - Q, K are [batch, heads, T, d_k]; V, O, dO are [batch, heads, T, d_v]; dQ, dK like Q,
+ *     dV like V.  All are DEVICE pointers to contiguous row-major arrays (feature dimension
+ *     fastest) of the plan's dtype, 16-byte aligned.  Accumulation is fp32.
+ *   - The workspace is a DEVICE buffer owned by the caller, at least smat_workspace_bytes()
+ *     long and 256-byte aligned.  The library allocates no device memory, keeps no pointer
+ *     after a call returns, launches only on the stream it is given (a cudaStream_t passed
+ *     as void*; NULL is the default stream) and never synchronises it, except where stated.
+ *   - Every function returns a status code; argument errors are detected before any launch.
+ *   - Tokens are 0-based; token t < n is "distant", t >= n is "recent"; the paper's 1-based
+ *     recent index is i = t - n + 1.
+ */
+#ifndef SMAT_H_
+#define SMAT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct smat_plan smat_plan; /* opaque, host memory, immutable after creation */
+
+typedef enum {
+  SMAT_OK = 0,
+  SMAT_ERR_NULL = 1,           /* a required pointer is NULL */
+  SMAT_ERR_SHAPE = 2,          /* unsupported batch/heads/T/d_k/d_v/chunk combination */
+  SMAT_ERR_DTYPE = 3,          /* unknown dtype */
+  SMAT_ERR_GEOMETRY = 4,       /* d out of range, q not prime, q^(d-1) too large, T < 2*chunk with d >= 2 */
+  SMAT_ERR_WORKSPACE = 5,      /* workspace too small */
+  SMAT_ERR_ALIGN = 6,          /* a pointer is not aligned as required */
+  SMAT_ERR_ARCH = 7,           /* the current device is not compute capability 10.x */
+  SMAT_ERR_LAUNCH = 8,         /* a CUDA launch or runtime call failed */
+  SMAT_ERR_DEVICE_TIMEOUT = 9, /* a bounded device-side wait expired (read by smat_check_status) */
+  SMAT_ERR_UNSUPPORTED = 10    /* the request is valid but this build has no path for it */
+} smat_status;
+
+typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
+
+/* plan flags */
+#define SMAT_FLAG_SIMT_ONLY 1u      /* never use the tensor-core kernels (bf16 plans run the fp32-ALU path) */
+#define SMAT_FLAG_ALG2_TABULATION 2u /* tabulate with the direct double loop of Algorithm 2 instead of the staged sums */
+
+/* Sizes of the construction (Sec. 3, "construction of G" and "Scaling with sequence length"). */
+typedef struct {
+  int64_t T, c, n, m;  /* sequence length, chunk width, distant = c*floor(T/2c), recent = T - n */
+  int32_t d, q;        /* VC dimension; prime field size (0 when d = 1) */
+  int64_t P;           /* profile cells q^(d-1)            (1 when d = 1) */
+  int64_t A;           /* normalised directions (q^(d-1)-1)/(q-1) (1 when d = 1) */
+  int64_t B;           /* types = hyperplanes = q*A = cached subset states (1 when d = 1) */
+  int64_t nnzC;        /* nonzeros of the incidence matrix = B*q^(d-2) */
+  int32_t vc_conditions_met; /* P <= n and 2B <= m, the conditions of the positional construction */
+} smat_geometry;
+
+/*
+ * Create a plan for one problem shape.
+ *   batch, heads >= 1; T >= 1 and a multiple of `chunk`; d_k, d_v in {64, 128};
+ *   chunk in {16, 32, 64, 128}; d in [1, 8] is the VC dimension of the mask (d = 1: causal mask).
+ *   q_override = 0 takes the default field size, the smallest prime q with q^d >= n
+ *   (Sec. 3 asks for q = Θ(n^{1/d}); this constant reproduces the cache sizes the paper prints);
+ *   any other value must be a prime and is used as given (small test cases).
+ * On success *out owns host memory until smat_plan_destroy.  No device work is done.
+ */
+smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, int d_k, int d_v, int d, int chunk,
+                             int q_override, smat_dtype dtype, unsigned flags);
+void smat_plan_destroy(smat_plan* plan);
+
+smat_status smat_get_geometry(const smat_plan* plan, smat_geometry* out);
+
+/* Bytes of workspace smat_forward (for_backward = 0) or smat_backward (for_backward = 1) needs. 0 if plan is NULL. */
+size_t smat_workspace_bytes(const smat_plan* plan, int for_backward);
+
+/*
+ * Forward pass, Algorithm 1 steps 2-7 (step 1 is implicit: φ = q_i, ψ = k_j, Z_j = k_j v_jᵀ).
+ * Reads Q, K, V; writes O (plan dtype).  The profile table F, the type table U ("cached subset
+ * states") and the incoming chunk states S_in are left in the workspace as fp32 and can be read
+ * back with smat_debug_tables.  Asynchronous on `cuda_stream`.
+ */
+smat_status smat_forward(const smat_plan* plan, const void* Q, const void* K, const void* V, void* O, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward pass (chunking proof, "Backward Pass"): given dO = ∂L/∂O writes dQ, dK, dV (plan dtype).
+ * It rebuilds the forward tables it needs (S_in, F, U) inside the workspace, so it does not
+ * depend on an earlier smat_forward call.  Asynchronous on `cuda_stream`.
+ */
+smat_status smat_backward(const smat_plan* plan, const void* Q, const void* K, const void* V, const void* dO, void* dQ,
+                          void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Routing as the library's index code sees it (HOST output buffers, caller-allocated):
+ *   prof    [n * (d-1)]  base-q digits of (t mod P), least significant first      (Sec. 3, positional assignment)
+ *   type    [m]          (t - n + 1) mod B for t = n .. T-1
+ *   type_ab [B * d]      for every type h = dir*q + b: the direction a (d-1 entries), then b
+ * Any of the three may be NULL to skip it.  For d = 1 prof is empty, type is all zeros and
+ * type_ab holds the single entry 0.
+ */
+smat_status smat_routing_indices(const smat_plan* plan, int32_t* prof, int32_t* type, int32_t* type_ab);
+
+/*
+ * The mask M^(d) as the DEVICE index code evaluates it: mask is a DEVICE buffer of T*T bytes
+ * (row-major, 0/1).  Only for T <= 8192.  Asynchronous on `cuda_stream`.
+ */
+smat_status smat_debug_mask(const smat_plan* plan, uint8_t* mask, void* cuda_stream);
+
+/*
+ * Copies of the fp32 tables a finished forward (or backward) left in `workspace`, into DEVICE
+ * buffers (any may be NULL):
+ *   F   [batch*heads, P, d_k, d_v]     profile table        (Eq. "schedule")
+ *   U   [batch*heads, B, d_k, d_v]     type table           (Eq. "schedule", Algorithm 2)
+ *   Sin [batch*heads, T/chunk, d_k, d_v] incoming chunk states (Sec. 3.1, causal branch)
+ * For d = 1 there is no separate F/U: the single state U_0 = F_0 is carried by the scan, and
+ * F and U receive that state (the incoming state of the first recent chunk).
+ * Asynchronous on `cuda_stream`.
+ */
+smat_status smat_debug_tables(const smat_plan* plan, const void* workspace, float* F, float* U, float* Sin,
+                              void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and reads the device status word kept at the start of the
+ * workspace.  Returns SMAT_OK, SMAT_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel
+ * expired (the kernel then returned early and the outputs are invalid), or SMAT_ERR_LAUNCH
+ * if the stream reports a CUDA error.
+ */
+smat_status smat_check_status(const smat_plan* plan, const void* workspace, void* cuda_stream);
+
+/* Number of kernels the last smat_forward / smat_backward on this plan launched (host counter). */
+int smat_last_launch_count(const smat_plan* plan);
+
+const char* smat_status_string(smat_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SMAT_H_ */

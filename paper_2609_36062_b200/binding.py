@@ -1,0 +1,217 @@
+"""Thin ctypes binding of libsmat.so: argument marshalling only, same names as the C boundary.
+
+Every step of the path runs inside the library's CUDA kernels.  PyTorch is used for device
+memory and streams.  There is no CPU fallback: if the shared library is missing or the device
+is absent the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsmat.so")
+
+SMAT_F32, SMAT_BF16 = 0, 1
+FLAG_SIMT_ONLY = 1
+FLAG_ALG2_TABULATION = 2
+
+EXPORTS = [
+    "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
+    "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
+    "smat_last_launch_count", "smat_status_string",
+]
+
+
+class SmatError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: status {code} ({status_string(code)})")
+        self.code = code
+
+
+class _Geometry(ctypes.Structure):
+    _fields_ = [("T", ctypes.c_int64), ("c", ctypes.c_int64), ("n", ctypes.c_int64), ("m", ctypes.c_int64),
+                ("d", ctypes.c_int32), ("q", ctypes.c_int32), ("P", ctypes.c_int64), ("A", ctypes.c_int64),
+                ("B", ctypes.c_int64), ("nnzC", ctypes.c_int64), ("vc_conditions_met", ctypes.c_int32)]
+
+
+@dataclass(frozen=True)
+class Geometry:
+    T: int
+    c: int
+    n: int
+    m: int
+    d: int
+    q: int
+    P: int
+    A: int
+    B: int
+    nnzC: int
+    vc_conditions_met: bool
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libsmat.so (built in-tree by paper_2609_36062_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(f"{LIB_PATH} not found: build it with `python -m paper_2609_36062_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i, i64, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+    lib.smat_plan_create.argtypes = [ctypes.POINTER(vp), i, i, i64, i, i, i, i, i, i, ctypes.c_uint]
+    lib.smat_plan_create.restype = i
+    lib.smat_plan_destroy.argtypes = [vp]
+    lib.smat_plan_destroy.restype = None
+    lib.smat_get_geometry.argtypes = [vp, ctypes.POINTER(_Geometry)]
+    lib.smat_get_geometry.restype = i
+    lib.smat_workspace_bytes.argtypes = [vp, i]
+    lib.smat_workspace_bytes.restype = sz
+    lib.smat_forward.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.smat_forward.restype = i
+    lib.smat_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.smat_backward.restype = i
+    lib.smat_routing_indices.argtypes = [vp, vp, vp, vp]
+    lib.smat_routing_indices.restype = i
+    lib.smat_debug_mask.argtypes = [vp, vp, vp]
+    lib.smat_debug_mask.restype = i
+    lib.smat_debug_tables.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.smat_debug_tables.restype = i
+    lib.smat_check_status.argtypes = [vp, vp, vp]
+    lib.smat_check_status.restype = i
+    lib.smat_last_launch_count.argtypes = [vp]
+    lib.smat_last_launch_count.restype = i
+    lib.smat_status_string.argtypes = [i]
+    lib.smat_status_string.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().smat_status_string(int(code)).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise SmatError(code, what)
+
+
+def _ptr(t: torch.Tensor | None) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+_TORCH_DTYPE = {SMAT_F32: torch.float32, SMAT_BF16: torch.bfloat16}
+
+
+class SmatPlan:
+    """Owns one smat_plan and (optionally) a workspace tensor; mirrors the C entry points."""
+
+    def __init__(self, batch: int, heads: int, T: int, d_k: int, d_v: int, d: int, chunk: int, dtype="bf16",
+                 q_override: int = 0, flags: int = 0):
+        self.lib = load_library()
+        self.dtype_code = {"f32": SMAT_F32, "bf16": SMAT_BF16}[dtype] if isinstance(dtype, str) else int(dtype)
+        self.torch_dtype = _TORCH_DTYPE[self.dtype_code]
+        self.shape = (batch, heads, T, d_k, d_v)
+        handle = ctypes.c_void_p()
+        _check(self.lib.smat_plan_create(ctypes.byref(handle), batch, heads, T, d_k, d_v, d, chunk, q_override,
+                                         self.dtype_code, flags), "smat_plan_create")
+        self.handle = handle
+        self._ws = None
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            self.lib.smat_plan_destroy(self.handle)
+            self.handle = None
+
+    # -- queries ---------------------------------------------------------------------------
+    def geometry(self) -> Geometry:
+        g = _Geometry()
+        _check(self.lib.smat_get_geometry(self.handle, ctypes.byref(g)), "smat_get_geometry")
+        return Geometry(g.T, g.c, g.n, g.m, g.d, g.q, g.P, g.A, g.B, g.nnzC, bool(g.vc_conditions_met))
+
+    def workspace_bytes(self, for_backward: bool = False) -> int:
+        return int(self.lib.smat_workspace_bytes(self.handle, int(for_backward)))
+
+    def workspace(self, for_backward: bool = False, device="cuda") -> torch.Tensor:
+        need = self.workspace_bytes(for_backward)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=device)
+        return self._ws
+
+    def last_launch_count(self) -> int:
+        return int(self.lib.smat_last_launch_count(self.handle))
+
+    # -- the hot path ------------------------------------------------------------------------
+    def _check_tensor(self, t: torch.Tensor, last: int, name: str) -> None:
+        b, h, T, _, _ = self.shape
+        if not t.is_cuda:
+            raise ValueError(f"{name} must be a CUDA tensor")
+        if t.dtype != self.torch_dtype or tuple(t.shape) != (b, h, T, last) or not t.is_contiguous():
+            raise ValueError(f"{name}: expected contiguous {self.torch_dtype} of shape {(b, h, T, last)}, "
+                             f"got {t.dtype} {tuple(t.shape)}")
+
+    def forward(self, Q, K, V, O=None, workspace=None, stream=None):
+        _, _, _, dk, dv = self.shape
+        self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
+        if O is None:
+            O = torch.empty_like(V)
+        self._check_tensor(O, dv, "O")
+        ws = self.workspace(False, Q.device) if workspace is None else workspace
+        _check(self.lib.smat_forward(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(ws), ws.numel(),
+                                     _stream(stream)), "smat_forward")
+        return O
+
+    def backward(self, Q, K, V, dO, dQ=None, dK=None, dV=None, workspace=None, stream=None):
+        _, _, _, dk, dv = self.shape
+        self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
+        self._check_tensor(dO, dv, "dO")
+        dQ = torch.empty_like(Q) if dQ is None else dQ
+        dK = torch.empty_like(K) if dK is None else dK
+        dV = torch.empty_like(V) if dV is None else dV
+        ws = self.workspace(True, Q.device) if workspace is None else workspace
+        _check(self.lib.smat_backward(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(dQ), _ptr(dK), _ptr(dV),
+                                      _ptr(ws), ws.numel(), _stream(stream)), "smat_backward")
+        return dQ, dK, dV
+
+    # -- verification exports ------------------------------------------------------------------
+    def routing_indices(self):
+        g = self.geometry()
+        D = max(g.d - 1, 0)
+        prof = torch.zeros((g.n, D), dtype=torch.int32)
+        typ = torch.zeros(g.m, dtype=torch.int32)
+        ab = torch.zeros((g.B, g.d), dtype=torch.int32)
+        _check(self.lib.smat_routing_indices(self.handle, _ptr(prof) if prof.numel() else None, _ptr(typ), _ptr(ab)),
+               "smat_routing_indices")
+        return prof, typ, ab
+
+    def debug_mask(self, device="cuda", stream=None) -> torch.Tensor:
+        T = self.shape[2]
+        mask = torch.empty((T, T), dtype=torch.uint8, device=device)
+        _check(self.lib.smat_debug_mask(self.handle, _ptr(mask), _stream(stream)), "smat_debug_mask")
+        return mask
+
+    def debug_tables(self, workspace=None, stream=None):
+        b, h, T, dk, dv = self.shape
+        g = self.geometry()
+        ws = self._ws if workspace is None else workspace
+        F = torch.empty((b * h, g.P, dk, dv), dtype=torch.float32, device=ws.device)
+        U = torch.empty((b * h, g.B, dk, dv), dtype=torch.float32, device=ws.device)
+        Sin = torch.empty((b * h, T // g.c, dk, dv), dtype=torch.float32, device=ws.device)
+        _check(self.lib.smat_debug_tables(self.handle, _ptr(ws), _ptr(F), _ptr(U), _ptr(Sin), _stream(stream)),
+               "smat_debug_tables")
+        return F, U, Sin
+
+    def check_status(self, workspace=None, stream=None) -> None:
+        ws = self._ws if workspace is None else workspace
+        _check(self.lib.smat_check_status(self.handle, _ptr(ws), _stream(stream)), "smat_check_status")

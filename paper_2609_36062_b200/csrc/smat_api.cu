@@ -1,0 +1,425 @@
+// Host side of libsmat: plan construction (geometry of Sec. 3, workspace layout) and the C entry
+// points that sequence the kernels of Algorithm 1 and of the backward pass.
+#include <cuda_runtime.h>
+
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "../../include/smat.h"
+#include "smat_internal.h"
+
+struct smat_plan {
+  int batch, heads, bh;
+  int r, p;            // d_k, d_v
+  int64_t T, c, NC;    // tokens, chunk width, chunks
+  smat_dtype dtype;
+  unsigned flags;
+  SmatGeo geo;
+  int64_t rp;          // state entries
+  // workspace layout (byte offsets, 256-byte aligned)
+  size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_fwd_end;
+  size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
+  mutable int launches;
+};
+
+namespace {
+
+bool is_prime(int64_t v) {
+  if (v < 2) return false;
+  for (int64_t f = 2; f * f <= v; ++f)
+    if (v % f == 0) return false;
+  return true;
+}
+
+// q^e >= n without overflow
+bool pow_at_least(int64_t q, int e, int64_t n) {
+  int64_t acc = 1;
+  for (int i = 0; i < e; ++i) {
+    acc *= q;
+    if (acc >= n) return true;
+  }
+  return acc >= n;
+}
+
+size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
+
+smat_status build_geometry(SmatGeo* g, int64_t T, int64_t c, int d, int q_override) {
+  memset(g, 0, sizeof(*g));
+  g->T = T; g->c = c; g->d = d;
+  g->n = c * (T / (2 * c));  // Sec. 3.1: n = c*floor(T/2c), so no chunk crosses the block boundary
+  g->m = T - g->n;
+  if (d == 1) {              // Sec. 3: B = 1, H_0 = F_q^0, G all ones
+    g->dense_G = 1; g->q = 0; g->D = 0; g->P = 1; g->A = 1; g->B = 1; g->nnzC = 1;
+    for (int k = 0; k < SMAT_MAX_D; ++k) g->qpow[k] = 1;
+    return SMAT_OK;
+  }
+  if (g->n == 0) return SMAT_ERR_GEOMETRY;
+  int64_t q = q_override;
+  if (q == 0) {
+    q = 2;
+    while (!(is_prime(q) && pow_at_least(q, d, g->n))) ++q;
+  } else if (!is_prime(q)) {
+    return SMAT_ERR_GEOMETRY;
+  }
+  g->q = (int32_t)q; g->D = d - 1;
+  int64_t acc = 1;
+  for (int k = 0; k < SMAT_MAX_D; ++k) {
+    g->qpow[k] = acc;
+    if (k < g->D) {
+      if (acc > (int64_t)1 << 40) return SMAT_ERR_GEOMETRY;
+      acc *= q;
+    }
+  }
+  g->P = g->qpow[g->D];
+  g->A = (g->P - 1) / (q - 1);   // Eq. "Bcount"
+  g->B = q * g->A;
+  g->nnzC = g->B * g->qpow[g->D - 1];
+  if (g->P > 60000 || g->B > 60000) return SMAT_ERR_GEOMETRY;  // grid.y carries the state index
+  int64_t start = 0;
+  for (int lead = 0; lead < g->D; ++lead) {
+    g->dir_group_start[lead] = start;
+    start += g->qpow[g->D - 1 - lead];
+  }
+  return SMAT_OK;
+}
+
+SmatOperand operand(const void* ptr, int bf16, int64_t s_bh, int64_t s_g, int64_t s0, int64_t s1, int tok0 = 0,
+                    int tok1 = 0) {
+  SmatOperand o; o.ptr = ptr; o.bf16 = bf16; o.s_bh = s_bh; o.s_g = s_g; o.s0 = s0; o.s1 = s1;
+  o.tok0 = tok0; o.tok1 = tok1;
+  return o;
+}
+
+SmatGroupSpec group(const smat_plan* pl, int mode) {
+  SmatGroupSpec s; s.mode = mode; s.n = pl->geo.n; s.T = pl->T; s.c = pl->c;
+  s.period = mode == SMAT_GM_PROFILE ? pl->geo.P : pl->geo.B;
+  return s;
+}
+
+struct Ctx {
+  const smat_plan* pl;
+  cudaStream_t st;
+  char* ws;
+  cudaError_t err;
+  int launches;
+  float* f(size_t off) const { return reinterpret_cast<float*>(ws + off); }
+};
+
+#define SMAT_TRY(ctx, call)                         \
+  do {                                              \
+    if ((ctx).err == cudaSuccess) {                 \
+      (ctx).err = (call);                           \
+      ++(ctx).launches;                             \
+    }                                               \
+  } while (0)
+
+int64_t max_group_tokens(const smat_plan* pl, int mode) {
+  const SmatGeo& g = pl->geo;
+  if (mode == SMAT_GM_CHUNK) return pl->c;
+  if (mode == SMAT_GM_PROFILE) return (g.n + g.P - 1) / g.P;
+  return (g.m + g.B - 1) / g.B;
+}
+int64_t group_count(const smat_plan* pl, int mode) {
+  if (mode == SMAT_GM_CHUNK) return pl->NC;
+  return mode == SMAT_GM_PROFILE ? pl->geo.P : pl->geo.B;
+}
+
+// state[bh][g] (r x p, fp32) = Σ_{tokens of g} a_tᵀ b_t   with a: [T, r], b: [T, p]
+void outer_sum(Ctx& cx, int mode, const void* a, const void* b, float* state) {
+  const smat_plan* pl = cx.pl;
+  const int bf = pl->dtype == SMAT_BF16;
+  const int64_t G = group_count(pl, mode);
+  SmatGemmArgs g{};
+  g.A = operand(a, bf, pl->T * pl->r, 0, 1, pl->r, 0, 1);
+  g.B = operand(b, bf, pl->T * pl->p, 0, pl->p, 1, 1, 0);
+  g.C = operand(state, 0, G * pl->rp, pl->rp, pl->p, 1);
+  g.M = pl->r; g.N = pl->p; g.tokK = 1; g.grp = group(pl, mode);
+  SMAT_TRY(cx, smat_launch_gemm(g, pl->r, pl->p, G, pl->bh, cx.st));
+}
+
+// out[bh][t] (+)= x_t · state_g(t)  (transposed = 0: x: [T, r] contracts the first state index, out: [T, p];
+//                                     transposed = 1: x: [T, p] contracts the second state index, out: [T, r])
+// `out_final` (plan dtype) receives acc_in + product when non-null; otherwise the fp32 accumulator is updated.
+void state_read(Ctx& cx, int mode, const void* x, const float* state, int transposed, const float* acc_in,
+                float* acc_out, void* out_final) {
+  const smat_plan* pl = cx.pl;
+  const int bf = pl->dtype == SMAT_BF16;
+  const int64_t G = group_count(pl, mode);
+  const int kdim = transposed ? pl->p : pl->r, odim = transposed ? pl->r : pl->p;
+  SmatGemmArgs g{};
+  g.A = operand(x, bf, pl->T * kdim, 0, kdim, 1, 1, 0);
+  g.B = transposed ? operand(state, 0, G * pl->rp, pl->rp, 1, pl->p) : operand(state, 0, G * pl->rp, pl->rp, pl->p, 1);
+  g.Cin = operand(acc_in, 0, pl->T * odim, 0, odim, 1, 1, 0);
+  g.C = out_final ? operand(out_final, bf, pl->T * odim, 0, odim, 1, 1, 0)
+                  : operand(acc_out, 0, pl->T * odim, 0, odim, 1, 1, 0);
+  g.K = kdim; g.N = odim; g.tokM = 1; g.grp = group(pl, mode);
+  SMAT_TRY(cx, smat_launch_gemm(g, (int)max_group_tokens(pl, mode), odim, G, pl->bh, cx.st));
+}
+
+// tile[bh][chunk] (c x c, fp32) = tril(X_b Y_bᵀ), X, Y: [T, dim]
+void tril_scores(Ctx& cx, const void* x, const void* y, int dim, float* tile) {
+  const smat_plan* pl = cx.pl;
+  const int bf = pl->dtype == SMAT_BF16;
+  SmatGemmArgs g{};
+  g.A = operand(x, bf, pl->T * dim, 0, dim, 1, 1, 0);
+  g.B = operand(y, bf, pl->T * dim, 0, 1, dim, 0, 1);
+  g.C = operand(tile, 0, pl->NC * pl->c * pl->c, pl->c * pl->c, pl->c, 1);
+  g.K = dim; g.tokM = 1; g.tokN = 1; g.tril = 1; g.grp = group(pl, SMAT_GM_CHUNK);
+  SMAT_TRY(cx, smat_launch_gemm(g, (int)pl->c, (int)pl->c, pl->NC, pl->bh, cx.st));
+}
+
+// out[bh][t in chunk] = acc_in + tile_b(ᵀ) · Y_b     (tile c x c; Y: [T, dim])
+void tile_apply(Ctx& cx, const float* tile, int tile_transposed, const void* y, int dim, const float* acc_in,
+                float* acc_out, void* out_final) {
+  const smat_plan* pl = cx.pl;
+  const int bf = pl->dtype == SMAT_BF16;
+  const int64_t cc = pl->c * pl->c;
+  SmatGemmArgs g{};
+  g.A = tile_transposed ? operand(tile, 0, pl->NC * cc, cc, 1, pl->c) : operand(tile, 0, pl->NC * cc, cc, pl->c, 1);
+  g.B = operand(y, bf, pl->T * dim, 0, dim, 1, 1, 0);
+  g.Cin = operand(acc_in, 0, pl->T * dim, 0, dim, 1, 1, 0);
+  g.C = out_final ? operand(out_final, bf, pl->T * dim, 0, dim, 1, 1, 0)
+                  : operand(acc_out, 0, pl->T * dim, 0, dim, 1, 1, 0);
+  g.N = dim; g.tokM = 1; g.tokK = 1; g.grp = group(pl, SMAT_GM_CHUNK);
+  SMAT_TRY(cx, smat_launch_gemm(g, (int)pl->c, dim, pl->NC, pl->bh, cx.st));
+}
+
+void scan_states(Ctx& cx, float* S, int reverse) {
+  const smat_plan* pl = cx.pl;
+  const int64_t ncd = pl->geo.n / pl->c;
+  if (pl->geo.dense_G)  // d = 1: U_0 = F_0 is exactly the carry across the boundary, so the scan runs through
+    SMAT_TRY(cx, smat_launch_scan(S, pl->rp, pl->NC, pl->bh, 0, pl->NC, 0, 0, reverse, cx.st));
+  else
+    SMAT_TRY(cx, smat_launch_scan(S, pl->rp, pl->NC, pl->bh, 0, ncd, ncd, pl->NC, reverse, cx.st));
+}
+
+smat_status check_common(const smat_plan* pl, const void* ws, size_t ws_bytes, int for_backward) {
+  if (!pl || !ws) return SMAT_ERR_NULL;
+  if (ws_bytes < smat_workspace_bytes(pl, for_backward)) return SMAT_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(ws) & 255) return SMAT_ERR_ALIGN;
+  return SMAT_OK;
+}
+
+bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
+
+// Steps 2-3 and 5-6 of Algorithm 1: the tables S_in, F, U.
+void build_forward_tables(Ctx& cx, const void* K, const void* V) {
+  const smat_plan* pl = cx.pl;
+  if (!pl->geo.dense_G) {
+    outer_sum(cx, SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));                                         // step 2
+    SMAT_TRY(cx, smat_launch_tabulate_alg2(cx.f(pl->off_F), cx.f(pl->off_U), pl->geo, pl->rp, pl->bh, 0, cx.st));  // step 3
+  }
+  outer_sum(cx, SMAT_GM_CHUNK, K, V, cx.f(pl->off_sin));                                           // step 5
+  scan_states(cx, cx.f(pl->off_sin), 0);                                                           // step 6
+}
+
+}  // namespace
+
+extern "C" {
+
+smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, int d_k, int d_v, int d, int chunk,
+                             int q_override, smat_dtype dtype, unsigned flags) {
+  if (!out) return SMAT_ERR_NULL;
+  *out = nullptr;
+  if (dtype != SMAT_F32 && dtype != SMAT_BF16) return SMAT_ERR_DTYPE;
+  if (batch < 1 || heads < 1 || T < 1 || (int64_t)batch * heads > 65535) return SMAT_ERR_SHAPE;
+  if ((d_k != 64 && d_k != 128) || (d_v != 64 && d_v != 128)) return SMAT_ERR_SHAPE;
+  if (chunk != 16 && chunk != 32 && chunk != 64 && chunk != 128) return SMAT_ERR_SHAPE;
+  if (T % chunk != 0 || T / chunk > 65535) return SMAT_ERR_SHAPE;
+  if (d < 1 || d > SMAT_MAX_D || q_override < 0) return SMAT_ERR_GEOMETRY;
+  smat_plan* pl = new (std::nothrow) smat_plan();
+  if (!pl) return SMAT_ERR_LAUNCH;
+  pl->batch = batch; pl->heads = heads; pl->bh = batch * heads;
+  pl->r = d_k; pl->p = d_v; pl->T = T; pl->c = chunk; pl->NC = T / chunk;
+  pl->dtype = dtype; pl->flags = flags; pl->rp = (int64_t)d_k * d_v; pl->launches = 0;
+  smat_status s = build_geometry(&pl->geo, T, chunk, d, q_override);
+  if (s != SMAT_OK) { delete pl; return s; }
+  const SmatGeo& g = pl->geo;
+  if (!g.dense_G && (smat_tabulate_alg2_slab(g.B, pl->rp) < 1)) { delete pl; return SMAT_ERR_UNSUPPORTED; }
+  const size_t state = (size_t)pl->rp * sizeof(float);
+  const int wide = d_k > d_v ? d_k : d_v;
+  size_t off = 0;
+  pl->off_status = off; off = align_up(off + 256);
+  pl->off_sin = off;    off = align_up(off + (size_t)pl->bh * pl->NC * state);
+  pl->off_F = off;      off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.P * state));
+  pl->off_U = off;      off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.B * state));
+  pl->off_acc = off;    off = align_up(off + (size_t)pl->bh * T * wide * sizeof(float));
+  pl->off_tileA = off;  off = align_up(off + (size_t)pl->bh * T * chunk * sizeof(float));
+  pl->off_fwd_end = off;
+  pl->off_dbar = off;   off = align_up(off + (size_t)pl->bh * pl->NC * state);
+  pl->off_ubar = off;   off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.B * state));
+  pl->off_fbar = off;   off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.P * state));
+  pl->off_tileG = off;  off = align_up(off + (size_t)pl->bh * T * chunk * sizeof(float));
+  pl->off_bwd_end = off;
+  *out = pl;
+  return SMAT_OK;
+}
+
+void smat_plan_destroy(smat_plan* plan) { delete plan; }
+
+smat_status smat_get_geometry(const smat_plan* pl, smat_geometry* out) {
+  if (!pl || !out) return SMAT_ERR_NULL;
+  const SmatGeo& g = pl->geo;
+  out->T = g.T; out->c = g.c; out->n = g.n; out->m = g.m; out->d = g.d; out->q = g.q;
+  out->P = g.P; out->A = g.A; out->B = g.B; out->nnzC = g.nnzC;
+  out->vc_conditions_met = g.dense_G ? 1 : (g.P <= g.n && 2 * g.B <= g.m);
+  return SMAT_OK;
+}
+
+size_t smat_workspace_bytes(const smat_plan* pl, int for_backward) {
+  if (!pl) return 0;
+  return for_backward ? pl->off_bwd_end : pl->off_fwd_end;
+}
+
+smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, const void* V, void* O, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  if (!Q || !K || !V || !O) return SMAT_ERR_NULL;
+  smat_status s = check_common(pl, workspace, workspace_bytes, 0);
+  if (s != SMAT_OK) return s;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return SMAT_ERR_ALIGN;
+  Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
+  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  build_forward_tables(cx, K, V);
+  float* acc = cx.f(pl->off_acc);
+  float* tileA = cx.f(pl->off_tileA);
+  tril_scores(cx, Q, K, pl->r, tileA);                                     // within-chunk scores, Eq. "local"
+  state_read(cx, SMAT_GM_CHUNK, Q, cx.f(pl->off_sin), 0, nullptr, acc, nullptr);  // earlier chunks
+  if (!pl->geo.dense_G)                                                    // step 4: typed read, rows in place
+    state_read(cx, SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, acc, acc, nullptr);
+  tile_apply(cx, tileA, 0, V, pl->p, acc, nullptr, O);                     // step 7
+  pl->launches = cx.launches;
+  return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
+smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, const void* V, const void* dO, void* dQ,
+                          void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!Q || !K || !V || !dO || !dQ || !dK || !dV) return SMAT_ERR_NULL;
+  smat_status s = check_common(pl, workspace, workspace_bytes, 1);
+  if (s != SMAT_OK) return s;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(dO) || misaligned(dQ) || misaligned(dK) ||
+      misaligned(dV))
+    return SMAT_ERR_ALIGN;
+  Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
+  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  const bool lr = !pl->geo.dense_G;
+  build_forward_tables(cx, K, V);
+  float* sin = cx.f(pl->off_sin);
+  float* dbar = cx.f(pl->off_dbar);
+  float* acc = cx.f(pl->off_acc);
+  float* tileA = cx.f(pl->off_tileA);
+  float* tileG = cx.f(pl->off_tileG);
+  // S̄_in_b = Q_bᵀ dO_b, then D̄ = exclusive suffix scan (scan adjoint)
+  outer_sum(cx, SMAT_GM_CHUNK, Q, dO, dbar);
+  scan_states(cx, dbar, 1);
+  // long-range adjoints: Ū_h = Σ q dOᵀ over the type, F̄ = Cᵀ Ū   (Eq. "lr-adjoint")
+  if (lr) {
+    outer_sum(cx, SMAT_GM_TYPE, Q, dO, cx.f(pl->off_ubar));
+    SMAT_TRY(cx, smat_launch_tabulate_alg2(cx.f(pl->off_ubar), cx.f(pl->off_fbar), pl->geo, pl->rp, pl->bh, 1, cx.st));
+  }
+  tril_scores(cx, Q, K, pl->r, tileA);    // A = tril(Q Kᵀ)
+  tril_scores(cx, dO, V, pl->p, tileG);   // tril(dO Vᵀ)
+  // dQ = dO S_inᵀ + U_type dO (recent) + tril(dO Vᵀ) K                      (Eq. "local-adjoint", Eq. "lr-adjoint")
+  state_read(cx, SMAT_GM_CHUNK, dO, sin, 1, nullptr, acc, nullptr);
+  if (lr) state_read(cx, SMAT_GM_TYPE, dO, cx.f(pl->off_U), 1, acc, acc, nullptr);
+  tile_apply(cx, tileG, 0, K, pl->r, acc, nullptr, dQ);
+  // dK = tril(dO Vᵀ)ᵀ Q + F̄_prof v (distant) + D̄ v
+  tile_apply(cx, tileG, 1, Q, pl->r, nullptr, acc, nullptr);
+  if (lr) state_read(cx, SMAT_GM_PROFILE, V, cx.f(pl->off_fbar), 1, acc, acc, nullptr);
+  state_read(cx, SMAT_GM_CHUNK, V, dbar, 1, acc, nullptr, dK);
+  // dV = Aᵀ dO + F̄_profᵀ k (distant) + D̄ᵀ k
+  tile_apply(cx, tileA, 1, dO, pl->p, nullptr, acc, nullptr);
+  if (lr) state_read(cx, SMAT_GM_PROFILE, K, cx.f(pl->off_fbar), 0, acc, acc, nullptr);
+  state_read(cx, SMAT_GM_CHUNK, K, dbar, 0, acc, nullptr, dV);
+  pl->launches = cx.launches;
+  return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
+smat_status smat_routing_indices(const smat_plan* pl, int32_t* prof, int32_t* type, int32_t* type_ab) {
+  if (!pl) return SMAT_ERR_NULL;
+  const SmatGeo& g = pl->geo;
+  if (g.dense_G) {
+    if (type) for (int64_t i = 0; i < g.m; ++i) type[i] = 0;
+    if (type_ab) type_ab[0] = 0;
+    return SMAT_OK;
+  }
+  if (prof)
+    for (int64_t t = 0; t < g.n; ++t) {
+      int64_t v = smat_profile_of(g, t);
+      for (int k = 0; k < g.D; ++k) { prof[t * g.D + k] = (int32_t)(v % g.q); v /= g.q; }
+    }
+  if (type)
+    for (int64_t t = g.n; t < g.T; ++t) type[t - g.n] = (int32_t)smat_type_of(g, t);
+  if (type_ab)
+    for (int64_t h = 0; h < g.B; ++h) {
+      int32_t a[SMAT_MAX_DIM];
+      smat_direction(g, h / g.q, a);
+      for (int k = 0; k < g.D; ++k) type_ab[h * g.d + k] = a[k];
+      type_ab[h * g.d + g.D] = (int32_t)(h % g.q);
+    }
+  return SMAT_OK;
+}
+
+smat_status smat_debug_mask(const smat_plan* pl, uint8_t* mask, void* cuda_stream) {
+  if (!pl || !mask) return SMAT_ERR_NULL;
+  if (pl->T > 8192) return SMAT_ERR_SHAPE;
+  return smat_launch_mask(mask, pl->geo, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? SMAT_OK
+                                                                                                 : SMAT_ERR_LAUNCH;
+}
+
+smat_status smat_debug_tables(const smat_plan* pl, const void* workspace, float* F, float* U, float* Sin,
+                              void* cuda_stream) {
+  if (!pl || !workspace) return SMAT_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const char* ws = static_cast<const char*>(workspace);
+  const size_t state = (size_t)pl->rp * sizeof(float);
+  cudaError_t err = cudaSuccess;
+  if (Sin) err = cudaMemcpyAsync(Sin, ws + pl->off_sin, (size_t)pl->bh * pl->NC * state, cudaMemcpyDeviceToDevice, st);
+  if (pl->geo.dense_G) {
+    const int64_t first_recent = pl->geo.n / pl->c;
+    for (int t = 0; t < 2; ++t) {
+      float* dst = t ? U : F;
+      if (!dst || err != cudaSuccess) continue;
+      err = cudaMemcpy2DAsync(dst, state, ws + pl->off_sin + (size_t)first_recent * state, (size_t)pl->NC * state,
+                              state, pl->bh, cudaMemcpyDeviceToDevice, st);
+    }
+  } else {
+    if (F && err == cudaSuccess)
+      err = cudaMemcpyAsync(F, ws + pl->off_F, (size_t)pl->bh * pl->geo.P * state, cudaMemcpyDeviceToDevice, st);
+    if (U && err == cudaSuccess)
+      err = cudaMemcpyAsync(U, ws + pl->off_U, (size_t)pl->bh * pl->geo.B * state, cudaMemcpyDeviceToDevice, st);
+  }
+  return err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
+smat_status smat_check_status(const smat_plan* pl, const void* workspace, void* cuda_stream) {
+  if (!pl || !workspace) return SMAT_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, static_cast<const char*>(workspace) + pl->off_status, sizeof(int), cudaMemcpyDeviceToHost,
+                      st) != cudaSuccess)
+    return SMAT_ERR_LAUNCH;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  return word == 0 ? SMAT_OK : SMAT_ERR_DEVICE_TIMEOUT;
+}
+
+int smat_last_launch_count(const smat_plan* pl) { return pl ? pl->launches : 0; }
+
+const char* smat_status_string(smat_status s) {
+  switch (s) {
+    case SMAT_OK: return "ok";
+    case SMAT_ERR_NULL: return "null pointer";
+    case SMAT_ERR_SHAPE: return "unsupported shape";
+    case SMAT_ERR_DTYPE: return "unknown dtype";
+    case SMAT_ERR_GEOMETRY: return "invalid mask geometry";
+    case SMAT_ERR_WORKSPACE: return "workspace too small";
+    case SMAT_ERR_ALIGN: return "misaligned pointer";
+    case SMAT_ERR_ARCH: return "device is not sm_100";
+    case SMAT_ERR_LAUNCH: return "CUDA launch or runtime failure";
+    case SMAT_ERR_DEVICE_TIMEOUT: return "bounded device wait expired";
+    case SMAT_ERR_UNSUPPORTED: return "no kernel path for this request";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,74 @@
+// Internal declarations shared by the translation units of libsmat (not part of the C boundary).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "smat_geometry.h"
+
+// ---- token groups -----------------------------------------------------------------------------
+// A "group" is a set of tokens t0, t0+ts, t0+2ts, ... that one state belongs to:
+//   CHUNK   g = chunk index        tokens g*c .. g*c+c-1                          (Sec. 3.1, causal branch)
+//   PROFILE g = packed profile x   distant tokens t ≡ x (mod P), t < n            (Eq. "schedule", F_x)
+//   TYPE    g = type h             recent tokens with (t-n+1) ≡ h (mod B), t < T  (Eq. "schedule", U_h)
+enum SmatGroupMode { SMAT_GM_NONE = 0, SMAT_GM_CHUNK = 1, SMAT_GM_PROFILE = 2, SMAT_GM_TYPE = 3 };
+
+struct SmatGroupSpec {
+  int mode;
+  int64_t n, T, c, period;  // period = P (PROFILE) or B (TYPE)
+};
+
+SMAT_HD void smat_group_tokens(const SmatGroupSpec& s, int64_t g, int64_t* t0, int64_t* ts, int64_t* cnt) {
+  switch (s.mode) {
+    case SMAT_GM_CHUNK:
+      *t0 = g * s.c; *ts = 1; *cnt = s.c;
+      break;
+    case SMAT_GM_PROFILE:
+      *t0 = g; *ts = s.period; *cnt = g < s.n ? (s.n - g + s.period - 1) / s.period : 0;
+      break;
+    case SMAT_GM_TYPE: {
+      int64_t i0 = g ? g : s.period;  // paper's 1-based recent index of the first token of this type
+      int64_t m = s.T - s.n;
+      *t0 = s.n + i0 - 1; *ts = s.period; *cnt = i0 <= m ? (m - i0) / s.period + 1 : 0;
+      break;
+    }
+    default:
+      *t0 = 0; *ts = 1; *cnt = 0;
+  }
+}
+
+// ---- generic batched small GEMM on the fp32 ALUs ---------------------------------------------------
+// C(m,n) = [Cin(m,n) +] Σ_k A(m,k) B(k,n), optionally zeroed above the diagonal (n > m).
+// An operand element lives at  ptr + bh*s_bh + g*s_g + X0*s0 + X1*s1  where Xi is the logical
+// index itself or, when the operand's tok flag for that index is set, the token it maps to.
+struct SmatOperand {
+  const void* ptr;
+  int bf16;  // 0: float, 1: __nv_bfloat16
+  int64_t s_bh, s_g, s0, s1;
+  int tok0, tok1;  // 1: that logical index of this operand is a token position of the group
+};
+
+struct SmatGemmArgs {
+  SmatOperand A, B, C, Cin;  // Cin.ptr == nullptr: no addend.  Cin is always float.
+  int M, N, K;               // extents of the dimensions that are not token dimensions
+  int tokM, tokN, tokK;      // 1: that dimension runs over the group's tokens (extent = token count)
+  int tril;
+  int tilesN;                // number of 64-wide column tiles launched
+  SmatGroupSpec grp;
+};
+
+cudaError_t smat_launch_gemm(const SmatGemmArgs& a, int max_M, int max_N, int64_t groups, int bh, cudaStream_t st);
+
+// Exclusive scan of per-chunk states in place, over up to two independent chunk ranges; reverse = suffix scan.
+cudaError_t smat_launch_scan(float* S, int64_t state_elems, int64_t NC, int bh, int64_t lo0, int64_t hi0, int64_t lo1,
+                             int64_t hi1, int reverse, cudaStream_t st);
+
+// Algorithm 2 (direct form) and its transpose, one slab of state entries per CTA held in shared memory.
+// transpose = 0: out[h] = Σ_{x ∈ H_h} in[x]  (in: P states, out: B states)
+// transpose = 1: out[x] = Σ_{h ∋ x} in[h]   (in: B states, out: P states)
+cudaError_t smat_launch_tabulate_alg2(const float* in, float* out, const SmatGeo& geo, int64_t state_elems, int bh,
+                                      int transpose, cudaStream_t st);
+// Largest slab (entries) the direct tabulation can hold in shared memory; 0 if none fits.
+int smat_tabulate_alg2_slab(int64_t rows_in, int64_t state_elems);
+
+cudaError_t smat_launch_mask(uint8_t* mask, const SmatGeo& geo, cudaStream_t st);

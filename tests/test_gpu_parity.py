@@ -1,0 +1,181 @@
+"""GPU parity: the CUDA path (through the C boundary) against the fp64 dense-mask oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import chunkwise_ref as cw
+from oracle import smat_oracle as so
+from paper_2609_36062_b200 import binding, synth
+from tests.helpers import TOL, device_inputs, rel_err, sample_tokens, to_numpy64
+
+pytestmark = pytest.mark.gpu
+
+
+def _small(name, d, T, dk, dv, c, dtype, batch=1, heads=2, seed=11, recipe="scaled"):
+    return synth.Workload(name, d, batch, heads, T, dk, dv, c, dtype, recipe, seed)
+
+
+def _plan(w, q=0, flags=0):
+    return binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype, q_override=q, flags=flags)
+
+
+# ---- routing: the mask as the device index code evaluates it ---------------------------------------
+@pytest.mark.parametrize("T,c,d,q", [(512, 64, 1, 0), (512, 64, 2, 0), (1024, 32, 3, 0), (1024, 16, 4, 3),
+                                     (512, 16, 5, 2), (4096, 64, 3, 0), (2048, 64, 4, 0)])
+def test_device_mask_is_bit_exact(T, c, d, q):
+    plan = binding.SmatPlan(1, 1, T, 64, 64, d, c, "f32", q_override=q)
+    got = plan.debug_mask().cpu().numpy()
+    ref = so.dense_mask(T, c, d, q or None)
+    assert np.array_equal(got, ref)
+
+
+# ---- full dense comparison on small shapes ---------------------------------------------------------
+SMALL = [
+    # d, T, dk, dv, c, dtype, q
+    (1, 256, 64, 64, 32, "f32", 0),
+    (2, 512, 64, 64, 64, "f32", 0),
+    (2, 384, 64, 128, 16, "f32", 0),        # ragged: n = 192, mixed head dims
+    (3, 512, 128, 64, 32, "f32", 0),
+    (3, 768, 64, 64, 64, "bf16", 0),
+    (4, 1024, 64, 64, 16, "f32", 3),
+    (4, 512, 128, 128, 128, "bf16", 2),
+    (5, 512, 64, 64, 16, "f32", 2),
+    (3, 640, 128, 128, 128, "bf16", 0),     # T/c = 5: n = 256, m = 384
+]
+
+
+@pytest.mark.parametrize("d,T,dk,dv,c,dtype,q", SMALL)
+def test_forward_matches_dense_oracle(d, T, dk, dv, c, dtype, q):
+    w = _small("s", d, T, dk, dv, c, dtype)
+    host, dev = device_inputs(w)
+    plan = _plan(w, q)
+    O = plan.forward(dev["q"], dev["k"], dev["v"])
+    plan.check_status()
+    M = so.dense_mask(T, c, d, q or None)
+    geo = so.geometry(T, c, d, q or None)
+    F, U, Sin = plan.debug_tables()
+    for h in range(w.bh):
+        Q64, K64, V64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v"))
+        ref = so.forward_dense(Q64, K64, V64, M)
+        got = to_numpy64(O.reshape(w.bh, T, dv)[h])
+        assert rel_err(got, ref) <= TOL[dtype], (h, rel_err(got, ref))
+        if h == 0:   # intermediate tables against the chunkwise restatement (fp32 tables: tight bound)
+            _, tab = cw.forward(Q64, K64, V64, geo, return_tables=True)
+            ref_sin = tab["Sin"].copy()
+            if d == 1:   # the library carries U_0 = F_0 across the boundary inside the scan
+                ref_sin[geo.n // c:] += tab["U"][0]
+                assert rel_err(to_numpy64(U[0]), tab["U"]) <= 1e-5
+            assert rel_err(to_numpy64(Sin[0]), ref_sin) <= 1e-5
+            if d > 1:
+                assert rel_err(to_numpy64(F[0]), tab["F"]) <= 1e-5
+                assert rel_err(to_numpy64(U[0]), tab["U"]) <= 1e-5
+
+
+@pytest.mark.parametrize("d,T,dk,dv,c,dtype,q", SMALL)
+def test_backward_matches_dense_oracle(d, T, dk, dv, c, dtype, q):
+    w = _small("s", d, T, dk, dv, c, dtype, seed=12)
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    plan = _plan(w, q)
+    dQ, dK, dV = plan.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+    plan.check_status()
+    M = so.dense_mask(T, c, d, q or None)
+    for h in range(w.bh):
+        Q64, K64, V64, G64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v", "do"))
+        rq, rk, rv = so.backward_dense(Q64, K64, V64, G64, M)
+        for name, got, ref in (("dQ", dQ, rq), ("dK", dK, rk), ("dV", dV, rv)):
+            g = to_numpy64(got.reshape(w.bh, T, -1)[h])
+            assert rel_err(g, ref) <= TOL[dtype], (name, h, rel_err(g, ref))
+
+
+def test_chunk_size_invariance_on_device():
+    outs = []
+    for c in (16, 32, 64, 128):
+        w = _small("inv", 2, 512, 64, 64, c, "f32", seed=5)
+        host, dev = device_inputs(w)
+        outs.append(to_numpy64(_plan(w).forward(dev["q"], dev["k"], dev["v"])))
+    for o in outs[1:]:
+        assert rel_err(o, outs[0]) <= 2e-6
+
+
+def test_degenerate_shapes():
+    # T = 2c (one chunk per block), a single chunk with d = 1, and P > n (empty profile cells)
+    for (d, T, c, q) in [(2, 128, 64, 0), (1, 64, 64, 0), (3, 64, 16, 7)]:
+        w = _small("deg", d, T, 64, 64, c, "f32", heads=1)
+        host, dev = device_inputs(w, ("q", "k", "v", "do"))
+        plan = _plan(w, q)
+        O = plan.forward(dev["q"], dev["k"], dev["v"])
+        dQ, dK, dV = plan.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+        M = so.dense_mask(T, c, d, q or None)
+        Q64, K64, V64, G64 = (synth.as_float64(w, host[x][0]) for x in ("q", "k", "v", "do"))
+        assert rel_err(to_numpy64(O[0, 0]), so.forward_dense(Q64, K64, V64, M)) <= 1e-4
+        for got, ref in zip((dQ, dK, dV), so.backward_dense(Q64, K64, V64, G64, M)):
+            assert rel_err(to_numpy64(got[0, 0]), ref) <= 1e-4
+
+
+# ---- the benchmark configurations --------------------------------------------------------------------
+def test_config1_full_dense():
+    for name in ("small_d2", "small_d1"):
+        w = synth.WORKLOADS[name]
+        host, dev = device_inputs(w, ("q", "k", "v", "do"))
+        plan = _plan(w)
+        O = plan.forward(dev["q"], dev["k"], dev["v"])
+        dQ, dK, dV = plan.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+        plan.check_status()
+        M = so.dense_mask(w.T, w.chunk, w.d)
+        Q64, K64, V64, G64 = (synth.as_float64(w, host[x][0]) for x in ("q", "k", "v", "do"))
+        assert rel_err(to_numpy64(O[0, 0]), so.forward_dense(Q64, K64, V64, M)) <= 1e-4
+        for got, ref in zip((dQ, dK, dV), so.backward_dense(Q64, K64, V64, G64, M)):
+            assert rel_err(to_numpy64(got[0, 0]), ref) <= 1e-4
+
+
+def _check_sampled(w, heads_to_check, nrows, backward=False, dense_head=None):
+    tensors = ("q", "k", "v", "do") if backward else ("q", "k", "v")
+    host, dev = device_inputs(w, tensors)
+    plan = _plan(w)
+    geo = so.geometry(w.T, w.chunk, w.d)
+    O = plan.forward(dev["q"], dev["k"], dev["v"])
+    grads = plan.backward(dev["q"], dev["k"], dev["v"], dev["do"]) if backward else None
+    plan.check_status()
+    O = O.reshape(w.bh, w.T, w.d_v)
+    tol = TOL[w.dtype]
+    for h in heads_to_check:
+        Q64, K64, V64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v"))
+        rows = sample_tokens(geo, nrows, seed=100 + h)
+        ref = so.forward_rows(Q64, K64, V64, geo, rows)
+        got = to_numpy64(O[h][rows])
+        # normalise by the largest entry of the whole output, which the sampled rows at the end reach
+        assert rel_err(got, ref) <= tol, ("O", h, rel_err(got, ref))
+        if backward:
+            G64 = synth.as_float64(w, host["do"][h])
+            dQ, dK, dV = (g.reshape(w.bh, w.T, -1)[h] for g in grads)
+            rq = so.dq_rows(Q64, K64, V64, G64, geo, rows)
+            rk, rv = so.dkdv_cols(Q64, K64, V64, G64, geo, rows)
+            for name, g, r in (("dQ", dQ, rq), ("dK", dK, rk), ("dV", dV, rv)):
+                e = rel_err(to_numpy64(g[rows]), r)
+                assert e <= tol, (name, h, e)
+    if dense_head is not None:
+        h = dense_head
+        Q64, K64, V64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v"))
+        ref = so.forward_dense(Q64, K64, V64, so.dense_mask(w.T, w.chunk, w.d))
+        assert rel_err(to_numpy64(O[h]), ref) <= tol
+
+
+def test_config2_t4k_d3():
+    w = synth.WORKLOADS["t4k_d3"]
+    _check_sampled(w, heads_to_check=[0, 13, w.bh - 1], nrows=96, dense_head=5)
+
+
+def test_config3_t16k_d4():
+    w = synth.WORKLOADS["t16k_d4"]
+    _check_sampled(w, heads_to_check=[0, 17, w.bh - 1], nrows=96)
+
+
+@pytest.mark.parametrize("name", ["t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4"])
+def test_config4_t64k(name):
+    w = synth.WORKLOADS[name]
+    _check_sampled(w, heads_to_check=[0, w.bh - 1], nrows=64)
+
+
+def test_config5_t8k_d3_forward_backward():
+    w = synth.WORKLOADS["t8k_d3_fwdbwd"]
+    _check_sampled(w, heads_to_check=[0, 77, w.bh - 1], nrows=64, backward=True)

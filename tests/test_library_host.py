@@ -1,0 +1,97 @@
+"""CPU-side checks of the C boundary: the library loads, exports every declared symbol, validates its
+arguments, and its integer routing matches the oracle bit for bit.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import smat_oracle as so
+from paper_2609_36062_b200 import binding, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(smat_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    lib = binding.load_library()
+    declared = _declared_symbols()
+    assert declared, "no declarations found"
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert set(binding.EXPORTS) <= declared
+
+
+@pytest.mark.parametrize("name", list(synth.WORKLOADS))
+def test_plan_geometry_matches_the_oracle(name):
+    w = synth.WORKLOADS[name]
+    plan = binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype)
+    g = plan.geometry()
+    o = so.geometry(w.T, w.chunk, w.d)
+    assert (g.n, g.m, g.q, g.P, g.A, g.B, g.nnzC) == (o.n, o.m, o.q, o.P, o.A, o.B, o.nnzC)
+    assert g.vc_conditions_met == o.conditions_met
+    assert plan.workspace_bytes(True) >= plan.workspace_bytes(False) > 0
+
+
+@pytest.mark.parametrize("T,c,d,q", [(512, 64, 2, 0), (512, 64, 1, 0), (4096, 64, 3, 0), (2048, 32, 4, 0), (256, 16, 3, 5),
+                                     (256, 16, 4, 3), (512, 16, 5, 3), (16384, 128, 4, 0), (8192, 64, 3, 0)])
+def test_routing_indices_are_bit_exact(T, c, d, q):
+    plan = binding.SmatPlan(1, 1, T, 64, 64, d, c, "f32", q_override=q)
+    geo = so.geometry(T, c, d, q or None)
+    prof, typ, ab = plan.routing_indices()
+    o_prof, o_typ, o_ab = so.routing_tables(geo)
+    assert np.array_equal(prof.numpy(), o_prof.reshape(prof.shape))
+    assert np.array_equal(typ.numpy(), o_typ)
+    assert np.array_equal(ab.numpy(), o_ab)
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    lib = binding.load_library()
+    h = ctypes.c_void_p()
+    mk = lambda *a: lib.smat_plan_create(ctypes.byref(h), *a)
+    assert lib.smat_plan_create(None, 1, 1, 512, 64, 64, 2, 64, 0, 0, 0) == 1          # null
+    assert mk(1, 1, 512, 64, 64, 2, 64, 0, 7, 0) == 3                                   # dtype
+    assert mk(1, 1, 512, 48, 64, 2, 64, 0, 0, 0) == 2                                   # d_k
+    assert mk(1, 1, 500, 64, 64, 2, 64, 0, 0, 0) == 2                                   # T % chunk
+    assert mk(1, 1, 512, 64, 64, 2, 48, 0, 0, 0) == 2                                   # chunk
+    assert mk(1, 1, 512, 64, 64, 0, 64, 0, 0, 0) == 4                                   # d
+    assert mk(1, 1, 512, 64, 64, 9, 64, 0, 0, 0) == 4
+    assert mk(1, 1, 512, 64, 64, 2, 64, 15, 0, 0) == 4                                  # q not prime
+    assert mk(1, 1, 64, 64, 64, 2, 64, 0, 0, 0) == 4                                    # T < 2c with d >= 2
+    assert mk(1, 1, 64, 64, 64, 1, 64, 0, 0, 0) == 0                                    # ... but fine for d = 1
+    plan = h.value
+    # forward with null / short / misaligned buffers never launches
+    assert lib.smat_forward(plan, None, 256, 256, 256, 256, 1 << 40, None) == 1
+    assert lib.smat_forward(plan, 256, 256, 256, 256, None, 1 << 40, None) == 1
+    assert lib.smat_forward(plan, 256, 256, 256, 256, 256, 16, None) == 5
+    assert lib.smat_forward(plan, 256, 256, 256, 256, 264, 1 << 40, None) == 6
+    assert lib.smat_forward(plan, 260, 256, 256, 256, 256, 1 << 40, None) == 6
+    assert lib.smat_backward(plan, 256, 256, 256, None, 256, 256, 256, 256, 1 << 40, None) == 1
+    assert lib.smat_workspace_bytes(None, 0) == 0
+    lib.smat_plan_destroy(h)
+    assert binding.status_string(5) == "workspace too small"
+
+
+def test_binding_rejects_wrong_tensors():
+    import torch
+    plan = binding.SmatPlan(1, 1, 512, 64, 64, 2, 64, "f32")
+    x = torch.zeros(1, 1, 512, 64)
+    with pytest.raises(ValueError):
+        plan.forward(x, x, x)          # CPU tensors: no fallback
+
+
+def test_non_default_geometry_flags():
+    g = binding.SmatPlan(1, 1, 256, 64, 64, 4, 16, "f32").geometry()   # default q too large for this T
+    assert not g.vc_conditions_met
+    g = binding.SmatPlan(1, 1, 256, 64, 64, 4, 16, "f32", q_override=2).geometry()
+    assert g.vc_conditions_met and (g.P, g.B) == (8, 14)
