@@ -1,0 +1,396 @@
+#!/usr/bin/env python
+"""Benchmark of the chunkwise hard-routing SMat prefill on B200.
+
+One "step" is one pass of the whole hot path over one batch of seeded synthetic input:
+smat_forward for the forward workloads, smat_forward + smat_backward for the fwd+bwd workload.
+Prints ONE JSON line (rank 0).  `value` is prefill tokens/s with inputs resident in HBM; `e2e`
+is the same metric through the C-ABI call with pinned HOST buffers (H2D of Q, K, V and D2H of O —
+and of dQ, dK, dV — inside the timed region).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--no-sweep]
+    python bench.py --impl reference ...      # the fp64 CPU oracle on a bounded sample of the same workload
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the
+workload: (batch, head) pairs share no data, so there is no collective on the data path
+(weak scaling, `value` = N x tokens / max-over-ranks time).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2609_36062_b200 import roofline, synth  # noqa: E402
+
+DEFAULT_WORKLOAD = "t16k_d4"
+SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
+METRIC = "SMat prefill tokens/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(synth.WORKLOADS))
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short runs of the other workloads")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="plan flags (see include/smat.h)")
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------ oracle leg
+def oracle_sample(w: synth.Workload, budget_s: float, backward: bool):
+    """Times the fp64 dense-mask oracle, as it stands, on sampled rows of head 0 of the workload.
+
+    Returns (tokens/s extrapolated to the whole workload, threads used, description, rows done, seconds)."""
+    from oracle import smat_oracle as so
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    geo = so.geometry(w.T, w.chunk, w.d)
+    names = ("q", "k", "v", "do") if backward else ("q", "k", "v")
+    host = {x: synth.as_float64(w, synth.stored(w, x, 0)) for x in names}
+    rng = np.random.default_rng(0)
+    order = rng.permutation(w.T)
+    done, t0 = 0, time.perf_counter()
+    batch = 8
+    while True:
+        rows = order[done:done + batch]
+        if len(rows) == 0:
+            break
+        so.forward_rows(host["q"], host["k"], host["v"], geo, rows)
+        if backward:
+            so.dq_rows(host["q"], host["k"], host["v"], host["do"], geo, rows)
+            so.dkdv_cols(host["q"], host["k"], host["v"], host["do"], geo, rows)
+        done += len(rows)
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    # a token is done when its row is done in every head of its batch element
+    tokens_per_s = done / dt / w.heads
+    what = (f"{done} uniformly sampled rows of O" + (" and of dQ, dK, dV" if backward else "") +
+            f" of head 0 ({dt:.1f} s), scaled by 1/heads to whole tokens")
+    return tokens_per_s, threads, what, done, dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = synth.WORKLOADS[args.workload]
+    steps, warm = max(1, args.steps), max(0, args.warmup)
+    budget = min(6.0, 120.0 / (steps + warm))
+    for _ in range(warm):
+        oracle_sample(w, min(budget, 1.0), w.backward)
+    vals, secs, rows, threads, what = [], 0.0, 0, 1, ""
+    for _ in range(steps):
+        v, threads, what, r, dt = oracle_sample(w, budget, w.backward)
+        vals.append(v); secs += dt; rows += r
+    value = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": 1e3 * secs / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, 1),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                         "sample": f"each step: {what}"},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ helpers
+def workload_config(w: synth.Workload, n_gpus: int):
+    return {"workload": w.name, "d": w.d, "batch": w.batch, "heads": w.heads, "T": w.T, "d_k": w.d_k, "d_v": w.d_v,
+            "chunk": w.chunk, "pass": "fwd+bwd" if w.backward else "fwd", "input_dtype": w.dtype,
+            "replicas": n_gpus, "l2": "inputs and tables exceed the 126 MB L2; no flush"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def make_inputs(w: synth.Workload, torch):
+    """Pinned host tensors [batch, heads, T, dim] in the storage dtype."""
+    names = ("q", "k", "v", "do") if w.backward else ("q", "k", "v")
+    out = {}
+    for x in names:
+        arr = synth.full_tensor(w, x)
+        if w.dtype == "f32":
+            t = torch.from_numpy(arr)
+        else:
+            t = torch.from_numpy(arr.view(np.int16)).view(torch.bfloat16)
+        out[x] = t.reshape(w.batch, w.heads, w.T, -1).pin_memory()
+    return out
+
+
+class Runner:
+    def __init__(self, w: synth.Workload, torch, binding, flags=0):
+        self.w, self.torch = w, torch
+        self.plan = binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype, flags=flags)
+        self.host = make_inputs(w, torch)
+        self.dev = {k: v.cuda(non_blocking=True) for k, v in self.host.items()}
+        self.O = torch.empty_like(self.dev["v"])
+        self.ws = self.plan.workspace(for_backward=w.backward)
+        if w.backward:
+            self.dQ, self.dK, self.dV = (torch.empty_like(self.dev[x]) for x in ("q", "k", "v"))
+        self.host_out = {"o": torch.empty_like(self.host["v"]).pin_memory()}
+        if w.backward:
+            for nm, src in (("dq", "q"), ("dk", "k"), ("dv", "v")):
+                self.host_out[nm] = torch.empty_like(self.host[src]).pin_memory()
+        torch.cuda.synchronize()
+
+    def step(self):
+        d = self.dev
+        self.plan.forward(d["q"], d["k"], d["v"], self.O, self.ws)
+        n = self.plan.last_launch_count()
+        if self.w.backward:
+            self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws)
+            n += self.plan.last_launch_count()
+        return n
+
+    def step_e2e(self):
+        for k, v in self.host.items():
+            self.dev[k].copy_(v, non_blocking=True)
+        self.step()
+        self.host_out["o"].copy_(self.O, non_blocking=True)
+        if self.w.backward:
+            self.host_out["dq"].copy_(self.dQ, non_blocking=True)
+            self.host_out["dk"].copy_(self.dK, non_blocking=True)
+            self.host_out["dv"].copy_(self.dV, non_blocking=True)
+
+    def bytes_e2e(self):
+        h2d = sum(v.numel() * v.element_size() for v in self.host.values())
+        d2h = sum(v.numel() * v.element_size() for v in self.host_out.values())
+        return h2d, d2h
+
+    def time_steps(self, fn, steps, warmup, barrier=None):
+        torch = self.torch
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(steps):
+            fn()
+        end.record()
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        return start.elapsed_time(end) / 1e3   # seconds for `steps` steps
+
+    def stage_profile(self, steps):
+        """Average per-kernel durations (ms) over `steps` steps, CUDA events on the launching stream."""
+        self.plan.profile_enable(True)
+        acc, order = {}, []
+        for _ in range(steps):
+            d = self.dev
+            self.plan.forward(d["q"], d["k"], d["v"], self.O, self.ws)
+            recs = self.plan.profile_read()
+            if self.w.backward:
+                self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws)
+                recs += [("bwd:" + n if not n.startswith("bwd_") else n, t) for n, t in self.plan.profile_read()]
+            for n, t in recs:
+                if n not in acc:
+                    acc[n] = 0.0; order.append(n)
+                acc[n] += t
+        self.plan.profile_enable(False)
+        return [(n, acc[n] / steps) for n in order]
+
+
+def path_report(w, geo, seconds_per_step, peaks):
+    e = 4 if w.dtype == "f32" else 2
+    work = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo)
+    if w.backward:
+        work = work + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo)
+    work = work.scaled(w.bh)
+    t = roofline.roofline_times(work, peaks)
+    return {
+        "frac_2term": t["t_2term"] / seconds_per_step, "frac_3term": t["t_3term"] / seconds_per_step,
+        "roofline_ms_2term": 1e3 * t["t_2term"], "roofline_ms_3term": 1e3 * t["t_3term"],
+        "t_tensor_ms": 1e3 * t["t_tensor"], "t_alu_ms": 1e3 * t["t_alu"], "t_hbm_ms": 1e3 * t["t_hbm"],
+        "algorithmic": {"tensor_flop": work.flops, "alu_adds": work.adds, "hbm_bytes": work.bytes},
+        "peaks": peaks["source"],
+    }
+
+
+def dominant_kernel_report(w, geo, stages, peaks):
+    e = 4 if w.dtype == "f32" else 2
+    total = sum(t for _, t in stages)
+    name, ms = max(stages, key=lambda s: s[1])
+    base = name.split(":")[-1]
+    work = roofline.stage_work(base, w.T, w.chunk, w.d_k, w.d_v, e, geo).scaled(w.bh)
+    t = roofline.roofline_times(work, peaks, sustained=True)
+    bounds = {"hbm": t["t_hbm"], "alu": t["t_alu"], "tensor": t["t_tensor"]}
+    bound = max(bounds, key=bounds.get)
+    sec = ms / 1e3
+    if bound == "hbm":
+        achieved, peak, unit = work.bytes / sec / 1e9, peaks["hbm_gbs"], "GB/s"
+    elif bound == "alu":
+        achieved, peak, unit = work.adds / sec / 1e9, t["alu_peak_adds"] / 1e9, "Gadd/s"
+    else:
+        achieved, peak, unit = work.flops / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
+    return {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+            "frac": achieved / peak if peak else None, "traffic": None, "ms": ms, "share": ms / total if total else None,
+            "peak_source": peaks["source"] + (" (fp32 add peak nominal: 148 SM x 128 lanes x max clock)" if bound == "alu" else ""),
+            "kernels_ms": {n: round(t_, 4) for n, t_ in stages}}
+
+
+def run_native(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_36062_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the hot path")
+    torch.cuda.set_device(local)
+    build.build()
+    binding.load_library()
+    barrier = None
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        barrier = dist.barrier
+
+    peaks = roofline.load_peaks(ROOT)
+    w = synth.WORKLOADS[args.workload]
+    steps, warm = max(1, args.steps), max(3, args.warmup)
+    runner = Runner(w, torch, binding, args.flags)
+    g = runner.plan.geometry()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches = runner.step()
+    secs = runner.time_steps(runner.step, steps, warm, barrier)
+    clocks = sampler.stop()
+    secs_e2e = runner.time_steps(runner.step_e2e, max(2, steps // 4), 2, barrier) / max(2, steps // 4)
+    if world > 1:
+        tmax = torch.tensor([secs, secs_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        secs, secs_e2e = float(tmax[0]), float(tmax[1])
+    per_step = secs / steps
+    value = world * w.tokens / per_step
+    h2d, d2h = runner.bytes_e2e()
+
+    line = None
+    if rank == 0:
+        stages = runner.stage_profile(min(steps, 10))
+        line = {
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warm,
+            "ms_per_step": 1e3 * per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if w.dtype == "f32" else "bf16 in, f32 accumulate", "data": "synthetic",
+            "config": workload_config(w, world),
+            "e2e": {"value": world * w.tokens / secs_e2e, "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches * steps,
+            "clocks": clocks,
+            "roofline": dominant_kernel_report(w, g, stages, peaks),
+            "path_roofline": path_report(w, g, per_step, peaks),
+            "tables": {"profile_states_P": g.P, "cached_subset_states_B": g.B, "nnzC": g.nnzC, "q": g.q},
+        }
+    del runner
+    torch.cuda.empty_cache()
+
+    if rank == 0 and world == 1 and not args.no_sweep:
+        sweep = []
+        for name in SWEEP:
+            if name == args.workload:
+                continue
+            ws_ = synth.WORKLOADS[name]
+            r = Runner(ws_, torch, binding, args.flags)
+            gg = r.plan.geometry()
+            k = 5
+            s = r.time_steps(r.step, k, 3) / k
+            rep = path_report(ws_, gg, s, peaks)
+            sweep.append({"workload": name, "value": ws_.tokens / s, "unit": "tokens/s", "ms_per_step": 1e3 * s,
+                          "frac_2term": rep["frac_2term"], "frac_3term": rep["frac_3term"],
+                          "cached_subset_states_B": gg.B, "profile_states_P": gg.P})
+            del r
+            torch.cuda.empty_cache()
+        line["sweep"] = sweep
+
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            v, threads, what, _, _ = oracle_sample(w, 12.0, w.backward)
+            line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what}
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_native(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -141,6 +141,17 @@ smat_status smat_debug_tables(const smat_plan* plan, const void* workspace, floa
  */
 smat_status smat_check_status(const smat_plan* plan, const void* workspace, void* cuda_stream);
 
+/*
+ * Per-kernel timing for measurement (the paper has no counterpart; this serves the roofline report).
+ * While enabled, smat_forward / smat_backward record a CUDA event on the launching stream before
+ * and after every kernel they launch.  The events belong to the plan and to the device that was
+ * current when profiling was enabled; disable before destroying the context.
+ * smat_profile_read waits for the last recorded event, then fills up to max_stages kernel names
+ * (static strings) and durations in milliseconds, in launch order, and returns how many it filled.
+ */
+smat_status smat_profile_enable(smat_plan* plan, int enable);
+int smat_profile_read(const smat_plan* plan, const char** names, float* ms, int max_stages);
+
 /* Number of kernels the last smat_forward / smat_backward on this plan launched (host counter). */
 int smat_last_launch_count(const smat_plan* plan);
 

@@ -22,7 +22,7 @@ FLAG_ALG2_TABULATION = 2
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
-    "smat_last_launch_count", "smat_status_string",
+    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read",
 ]
 
 
@@ -87,6 +87,10 @@ def load_library() -> ctypes.CDLL:
     lib.smat_check_status.restype = i
     lib.smat_last_launch_count.argtypes = [vp]
     lib.smat_last_launch_count.restype = i
+    lib.smat_profile_enable.argtypes = [vp, i]
+    lib.smat_profile_enable.restype = i
+    lib.smat_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float), i]
+    lib.smat_profile_read.restype = i
     lib.smat_status_string.argtypes = [i]
     lib.smat_status_string.restype = ctypes.c_char_p
     _lib = lib
@@ -130,7 +134,7 @@ class SmatPlan:
         self._ws = None
 
     def __del__(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and self.lib is not None:
             self.lib.smat_plan_destroy(self.handle)
             self.handle = None
 
@@ -148,6 +152,16 @@ class SmatPlan:
         if self._ws is None or self._ws.numel() < need:
             self._ws = torch.empty(need, dtype=torch.uint8, device=device)
         return self._ws
+
+    def profile_enable(self, enable: bool = True) -> None:
+        _check(self.lib.smat_profile_enable(self.handle, int(enable)), "smat_profile_enable")
+
+    def profile_read(self, max_stages: int = 64):
+        """[(kernel name, milliseconds)] of the last forward/backward, in launch order."""
+        names = (ctypes.c_char_p * max_stages)()
+        ms = (ctypes.c_float * max_stages)()
+        count = self.lib.smat_profile_read(self.handle, names, ms, max_stages)
+        return [(names[k].decode(), float(ms[k])) for k in range(count)]
 
     def last_launch_count(self) -> int:
         return int(self.lib.smat_last_launch_count(self.handle))

@@ -9,6 +9,8 @@
 #include "../../include/smat.h"
 #include "smat_internal.h"
 
+#define SMAT_MAX_STAGES 40
+
 struct smat_plan {
   int batch, heads, bh;
   int r, p;            // d_k, d_v
@@ -21,7 +23,13 @@ struct smat_plan {
   size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_fwd_end;
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
   mutable int launches;
+  // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
+  mutable bool profiling;
+  mutable cudaEvent_t events[SMAT_MAX_STAGES + 1];
+  mutable const char* stage_names[SMAT_MAX_STAGES];
+  mutable int stages;
 };
+
 
 namespace {
 
@@ -106,10 +114,23 @@ struct Ctx {
   float* f(size_t off) const { return reinterpret_cast<float*>(ws + off); }
 };
 
-#define SMAT_TRY(ctx, call)                         \
+void mark_stage(const smat_plan* pl, cudaStream_t st, const char* name) {
+  if (!pl->profiling || pl->stages >= SMAT_MAX_STAGES) return;
+  if (pl->stages == 0) cudaEventRecord(pl->events[0], st);
+  pl->stage_names[pl->stages] = name;
+}
+void end_stage(const smat_plan* pl, cudaStream_t st) {
+  if (!pl->profiling || pl->stages >= SMAT_MAX_STAGES) return;
+  ++pl->stages;
+  cudaEventRecord(pl->events[pl->stages], st);
+}
+
+#define SMAT_TRY(ctx, name, call)                   \
   do {                                              \
     if ((ctx).err == cudaSuccess) {                 \
+      mark_stage((ctx).pl, (ctx).st, name);         \
       (ctx).err = (call);                           \
+      end_stage((ctx).pl, (ctx).st);                \
       ++(ctx).launches;                             \
     }                                               \
   } while (0)
@@ -126,7 +147,7 @@ int64_t group_count(const smat_plan* pl, int mode) {
 }
 
 // state[bh][g] (r x p, fp32) = Σ_{tokens of g} a_tᵀ b_t   with a: [T, r], b: [T, p]
-void outer_sum(Ctx& cx, int mode, const void* a, const void* b, float* state) {
+void outer_sum(Ctx& cx, const char* name, int mode, const void* a, const void* b, float* state) {
   const smat_plan* pl = cx.pl;
   const int bf = pl->dtype == SMAT_BF16;
   const int64_t G = group_count(pl, mode);
@@ -135,13 +156,13 @@ void outer_sum(Ctx& cx, int mode, const void* a, const void* b, float* state) {
   g.B = operand(b, bf, pl->T * pl->p, 0, pl->p, 1, 1, 0);
   g.C = operand(state, 0, G * pl->rp, pl->rp, pl->p, 1);
   g.M = pl->r; g.N = pl->p; g.tokK = 1; g.grp = group(pl, mode);
-  SMAT_TRY(cx, smat_launch_gemm(g, pl->r, pl->p, G, pl->bh, cx.st));
+  SMAT_TRY(cx, name, smat_launch_gemm(g, pl->r, pl->p, G, pl->bh, cx.st));
 }
 
 // out[bh][t] (+)= x_t · state_g(t)  (transposed = 0: x: [T, r] contracts the first state index, out: [T, p];
 //                                     transposed = 1: x: [T, p] contracts the second state index, out: [T, r])
 // `out_final` (plan dtype) receives acc_in + product when non-null; otherwise the fp32 accumulator is updated.
-void state_read(Ctx& cx, int mode, const void* x, const float* state, int transposed, const float* acc_in,
+void state_read(Ctx& cx, const char* name, int mode, const void* x, const float* state, int transposed, const float* acc_in,
                 float* acc_out, void* out_final) {
   const smat_plan* pl = cx.pl;
   const int bf = pl->dtype == SMAT_BF16;
@@ -154,11 +175,11 @@ void state_read(Ctx& cx, int mode, const void* x, const float* state, int transp
   g.C = out_final ? operand(out_final, bf, pl->T * odim, 0, odim, 1, 1, 0)
                   : operand(acc_out, 0, pl->T * odim, 0, odim, 1, 1, 0);
   g.K = kdim; g.N = odim; g.tokM = 1; g.grp = group(pl, mode);
-  SMAT_TRY(cx, smat_launch_gemm(g, (int)max_group_tokens(pl, mode), odim, G, pl->bh, cx.st));
+  SMAT_TRY(cx, name, smat_launch_gemm(g, (int)max_group_tokens(pl, mode), odim, G, pl->bh, cx.st));
 }
 
 // tile[bh][chunk] (c x c, fp32) = tril(X_b Y_bᵀ), X, Y: [T, dim]
-void tril_scores(Ctx& cx, const void* x, const void* y, int dim, float* tile) {
+void tril_scores(Ctx& cx, const char* name, const void* x, const void* y, int dim, float* tile) {
   const smat_plan* pl = cx.pl;
   const int bf = pl->dtype == SMAT_BF16;
   SmatGemmArgs g{};
@@ -166,11 +187,11 @@ void tril_scores(Ctx& cx, const void* x, const void* y, int dim, float* tile) {
   g.B = operand(y, bf, pl->T * dim, 0, 1, dim, 0, 1);
   g.C = operand(tile, 0, pl->NC * pl->c * pl->c, pl->c * pl->c, pl->c, 1);
   g.K = dim; g.tokM = 1; g.tokN = 1; g.tril = 1; g.grp = group(pl, SMAT_GM_CHUNK);
-  SMAT_TRY(cx, smat_launch_gemm(g, (int)pl->c, (int)pl->c, pl->NC, pl->bh, cx.st));
+  SMAT_TRY(cx, name, smat_launch_gemm(g, (int)pl->c, (int)pl->c, pl->NC, pl->bh, cx.st));
 }
 
 // out[bh][t in chunk] = acc_in + tile_b(ᵀ) · Y_b     (tile c x c; Y: [T, dim])
-void tile_apply(Ctx& cx, const float* tile, int tile_transposed, const void* y, int dim, const float* acc_in,
+void tile_apply(Ctx& cx, const char* name, const float* tile, int tile_transposed, const void* y, int dim, const float* acc_in,
                 float* acc_out, void* out_final) {
   const smat_plan* pl = cx.pl;
   const int bf = pl->dtype == SMAT_BF16;
@@ -182,16 +203,16 @@ void tile_apply(Ctx& cx, const float* tile, int tile_transposed, const void* y, 
   g.C = out_final ? operand(out_final, bf, pl->T * dim, 0, dim, 1, 1, 0)
                   : operand(acc_out, 0, pl->T * dim, 0, dim, 1, 1, 0);
   g.N = dim; g.tokM = 1; g.tokK = 1; g.grp = group(pl, SMAT_GM_CHUNK);
-  SMAT_TRY(cx, smat_launch_gemm(g, (int)pl->c, dim, pl->NC, pl->bh, cx.st));
+  SMAT_TRY(cx, name, smat_launch_gemm(g, (int)pl->c, dim, pl->NC, pl->bh, cx.st));
 }
 
-void scan_states(Ctx& cx, float* S, int reverse) {
+void scan_states(Ctx& cx, const char* name, float* S, int reverse) {
   const smat_plan* pl = cx.pl;
   const int64_t ncd = pl->geo.n / pl->c;
   if (pl->geo.dense_G)  // d = 1: U_0 = F_0 is exactly the carry across the boundary, so the scan runs through
-    SMAT_TRY(cx, smat_launch_scan(S, pl->rp, pl->NC, pl->bh, 0, pl->NC, 0, 0, reverse, cx.st));
+    SMAT_TRY(cx, name, smat_launch_scan(S, pl->rp, pl->NC, pl->bh, 0, pl->NC, 0, 0, reverse, cx.st));
   else
-    SMAT_TRY(cx, smat_launch_scan(S, pl->rp, pl->NC, pl->bh, 0, ncd, ncd, pl->NC, reverse, cx.st));
+    SMAT_TRY(cx, name, smat_launch_scan(S, pl->rp, pl->NC, pl->bh, 0, ncd, ncd, pl->NC, reverse, cx.st));
 }
 
 smat_status check_common(const smat_plan* pl, const void* ws, size_t ws_bytes, int for_backward) {
@@ -207,11 +228,11 @@ bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) !=
 void build_forward_tables(Ctx& cx, const void* K, const void* V) {
   const smat_plan* pl = cx.pl;
   if (!pl->geo.dense_G) {
-    outer_sum(cx, SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));                                         // step 2
-    SMAT_TRY(cx, smat_launch_tabulate_alg2(cx.f(pl->off_F), cx.f(pl->off_U), pl->geo, pl->rp, pl->bh, 0, cx.st));  // step 3
+    outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));                                         // step 2
+    SMAT_TRY(cx, "tabulate", smat_launch_tabulate_alg2(cx.f(pl->off_F), cx.f(pl->off_U), pl->geo, pl->rp, pl->bh, 0, cx.st));  // step 3
   }
-  outer_sum(cx, SMAT_GM_CHUNK, K, V, cx.f(pl->off_sin));                                           // step 5
-  scan_states(cx, cx.f(pl->off_sin), 0);                                                           // step 6
+  outer_sum(cx, "chunk_state", SMAT_GM_CHUNK, K, V, cx.f(pl->off_sin));                                           // step 5
+  scan_states(cx, "scan", cx.f(pl->off_sin), 0);                                                           // step 6
 }
 
 }  // namespace
@@ -233,6 +254,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->batch = batch; pl->heads = heads; pl->bh = batch * heads;
   pl->r = d_k; pl->p = d_v; pl->T = T; pl->c = chunk; pl->NC = T / chunk;
   pl->dtype = dtype; pl->flags = flags; pl->rp = (int64_t)d_k * d_v; pl->launches = 0;
+  pl->profiling = false; pl->stages = 0;
   smat_status s = build_geometry(&pl->geo, T, chunk, d, q_override);
   if (s != SMAT_OK) { delete pl; return s; }
   const SmatGeo& g = pl->geo;
@@ -256,7 +278,38 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   return SMAT_OK;
 }
 
-void smat_plan_destroy(smat_plan* plan) { delete plan; }
+void smat_plan_destroy(smat_plan* plan) {
+  if (plan && plan->profiling) smat_profile_enable(plan, 0);
+  delete plan;
+}
+
+smat_status smat_profile_enable(smat_plan* pl, int enable) {
+  if (!pl) return SMAT_ERR_NULL;
+  if ((enable != 0) == pl->profiling) return SMAT_OK;
+  if (enable) {
+    for (int i = 0; i <= SMAT_MAX_STAGES; ++i)
+      if (cudaEventCreate(&pl->events[i]) != cudaSuccess) return SMAT_ERR_LAUNCH;
+    pl->profiling = true;
+  } else {
+    for (int i = 0; i <= SMAT_MAX_STAGES; ++i) cudaEventDestroy(pl->events[i]);
+    pl->profiling = false;
+  }
+  pl->stages = 0;
+  return SMAT_OK;
+}
+
+int smat_profile_read(const smat_plan* pl, const char** names, float* ms, int max_stages) {
+  if (!pl || !pl->profiling || pl->stages == 0) return 0;
+  if (cudaEventSynchronize(pl->events[pl->stages]) != cudaSuccess) return 0;
+  int count = pl->stages < max_stages ? pl->stages : max_stages;
+  for (int i = 0; i < count; ++i) {
+    float t = 0.f;
+    cudaEventElapsedTime(&t, pl->events[i], pl->events[i + 1]);
+    if (ms) ms[i] = t;
+    if (names) names[i] = pl->stage_names[i];
+  }
+  return count;
+}
 
 smat_status smat_get_geometry(const smat_plan* pl, smat_geometry* out) {
   if (!pl || !out) return SMAT_ERR_NULL;
@@ -279,15 +332,16 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
   if (s != SMAT_OK) return s;
   if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return SMAT_ERR_ALIGN;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
+  pl->stages = 0;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   build_forward_tables(cx, K, V);
   float* acc = cx.f(pl->off_acc);
   float* tileA = cx.f(pl->off_tileA);
-  tril_scores(cx, Q, K, pl->r, tileA);                                     // within-chunk scores, Eq. "local"
-  state_read(cx, SMAT_GM_CHUNK, Q, cx.f(pl->off_sin), 0, nullptr, acc, nullptr);  // earlier chunks
+  tril_scores(cx, "scores", Q, K, pl->r, tileA);                           // within-chunk scores, Eq. "local"
+  state_read(cx, "read_chunk", SMAT_GM_CHUNK, Q, cx.f(pl->off_sin), 0, nullptr, acc, nullptr);  // earlier chunks
   if (!pl->geo.dense_G)                                                    // step 4: typed read, rows in place
-    state_read(cx, SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, acc, acc, nullptr);
-  tile_apply(cx, tileA, 0, V, pl->p, acc, nullptr, O);                     // step 7
+    state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, acc, acc, nullptr);
+  tile_apply(cx, "output", tileA, 0, V, pl->p, acc, nullptr, O);                     // step 7
   pl->launches = cx.launches;
   return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
 }
@@ -301,6 +355,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
       misaligned(dV))
     return SMAT_ERR_ALIGN;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
+  pl->stages = 0;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   const bool lr = !pl->geo.dense_G;
   build_forward_tables(cx, K, V);
@@ -310,27 +365,27 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
   float* tileA = cx.f(pl->off_tileA);
   float* tileG = cx.f(pl->off_tileG);
   // S̄_in_b = Q_bᵀ dO_b, then D̄ = exclusive suffix scan (scan adjoint)
-  outer_sum(cx, SMAT_GM_CHUNK, Q, dO, dbar);
-  scan_states(cx, dbar, 1);
+  outer_sum(cx, "bwd_chunk_state", SMAT_GM_CHUNK, Q, dO, dbar);
+  scan_states(cx, "bwd_scan", dbar, 1);
   // long-range adjoints: Ū_h = Σ q dOᵀ over the type, F̄ = Cᵀ Ū   (Eq. "lr-adjoint")
   if (lr) {
-    outer_sum(cx, SMAT_GM_TYPE, Q, dO, cx.f(pl->off_ubar));
-    SMAT_TRY(cx, smat_launch_tabulate_alg2(cx.f(pl->off_ubar), cx.f(pl->off_fbar), pl->geo, pl->rp, pl->bh, 1, cx.st));
+    outer_sum(cx, "bwd_pool_type", SMAT_GM_TYPE, Q, dO, cx.f(pl->off_ubar));
+    SMAT_TRY(cx, "bwd_tabulate_t", smat_launch_tabulate_alg2(cx.f(pl->off_ubar), cx.f(pl->off_fbar), pl->geo, pl->rp, pl->bh, 1, cx.st));
   }
-  tril_scores(cx, Q, K, pl->r, tileA);    // A = tril(Q Kᵀ)
-  tril_scores(cx, dO, V, pl->p, tileG);   // tril(dO Vᵀ)
+  tril_scores(cx, "bwd_scores_qk", Q, K, pl->r, tileA);    // A = tril(Q Kᵀ)
+  tril_scores(cx, "bwd_scores_gv", dO, V, pl->p, tileG);   // tril(dO Vᵀ)
   // dQ = dO S_inᵀ + U_type dO (recent) + tril(dO Vᵀ) K                      (Eq. "local-adjoint", Eq. "lr-adjoint")
-  state_read(cx, SMAT_GM_CHUNK, dO, sin, 1, nullptr, acc, nullptr);
-  if (lr) state_read(cx, SMAT_GM_TYPE, dO, cx.f(pl->off_U), 1, acc, acc, nullptr);
-  tile_apply(cx, tileG, 0, K, pl->r, acc, nullptr, dQ);
+  state_read(cx, "bwd_dq_chunk", SMAT_GM_CHUNK, dO, sin, 1, nullptr, acc, nullptr);
+  if (lr) state_read(cx, "bwd_dq_type", SMAT_GM_TYPE, dO, cx.f(pl->off_U), 1, acc, acc, nullptr);
+  tile_apply(cx, "bwd_dq_tile", tileG, 0, K, pl->r, acc, nullptr, dQ);
   // dK = tril(dO Vᵀ)ᵀ Q + F̄_prof v (distant) + D̄ v
-  tile_apply(cx, tileG, 1, Q, pl->r, nullptr, acc, nullptr);
-  if (lr) state_read(cx, SMAT_GM_PROFILE, V, cx.f(pl->off_fbar), 1, acc, acc, nullptr);
-  state_read(cx, SMAT_GM_CHUNK, V, dbar, 1, acc, nullptr, dK);
+  tile_apply(cx, "bwd_dk_tile", tileG, 1, Q, pl->r, nullptr, acc, nullptr);
+  if (lr) state_read(cx, "bwd_dk_profile", SMAT_GM_PROFILE, V, cx.f(pl->off_fbar), 1, acc, acc, nullptr);
+  state_read(cx, "bwd_dk_chunk", SMAT_GM_CHUNK, V, dbar, 1, acc, nullptr, dK);
   // dV = Aᵀ dO + F̄_profᵀ k (distant) + D̄ᵀ k
-  tile_apply(cx, tileA, 1, dO, pl->p, nullptr, acc, nullptr);
-  if (lr) state_read(cx, SMAT_GM_PROFILE, K, cx.f(pl->off_fbar), 0, acc, acc, nullptr);
-  state_read(cx, SMAT_GM_CHUNK, K, dbar, 0, acc, nullptr, dV);
+  tile_apply(cx, "bwd_dv_tile", tileA, 1, dO, pl->p, nullptr, acc, nullptr);
+  if (lr) state_read(cx, "bwd_dv_profile", SMAT_GM_PROFILE, K, cx.f(pl->off_fbar), 0, acc, acc, nullptr);
+  state_read(cx, "bwd_dv_chunk", SMAT_GM_CHUNK, K, dbar, 0, acc, nullptr, dV);
   pl->launches = cx.launches;
   return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
 }

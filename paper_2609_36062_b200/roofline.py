@@ -1,0 +1,102 @@
+"""Algorithmic work of the chunkwise SMat prefill and the roofline it implies.
+
+Counts are what the method itself has to do (Theorem 2's cost terms), per (batch, head), with
+r = d_k, p = d_v, e = bytes per input element, fp32 tables:
+
+  tensor flop (forward)  = T (c+1)(r+p)             within-chunk tril tiles (two products)
+                         + 2rp (T + T + n + m)      chunk summaries, carried-state read, pool, typed read
+  ALU adds   (forward)   = nnz(C) rp + (T/c) rp     Algorithm 2's state additions + the scan
+  HBM bytes  (forward)   = (2r + 2p) T e            Q, K, V in, O out
+                         + 2 P rp 4 + 2 B rp 4      profile table and type table, written once and read once
+                           (d = 1 has neither table)
+  backward               = T (c+1)(3r+2p) + 15 T rp flop, the same adds again (Cᵀ tabulation, suffix scan),
+                           (4r + 3p) T e bytes of tensors and 2 (2P + 2B) rp 4 bytes of tables
+                           (F, U rebuilt; Ū, F̄ written and read)
+
+Chunk-state traffic (T/c states written and read) depends on the implementation and is not counted.
+Peaks come from MEASURED_PEAKS.json when present (HBM copy GB/s, dense bf16 TFLOP/s, both measured on
+this machine's B200s), else from the stated fallback.  The fp32 add peak is nominal:
+148 SMs x 128 lanes x the maximum SM clock.
+"""
+from __future__ import annotations
+
+import json
+import os
+from dataclasses import dataclass
+
+FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0}
+
+
+def load_peaks(root: str) -> dict:
+    path = os.path.join(root, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            data = json.load(f)
+        data["source"] = "measured"
+        return data
+    data = dict(FALLBACK)
+    data["source"] = "fallback"
+    return data
+
+
+@dataclass
+class Work:
+    flops: float       # dense contraction flop
+    adds: float        # fp32 state additions on the plain ALUs
+    bytes: float       # HBM bytes
+
+    def __add__(self, o):
+        return Work(self.flops + o.flops, self.adds + o.adds, self.bytes + o.bytes)
+
+    def scaled(self, k):
+        return Work(self.flops * k, self.adds * k, self.bytes * k)
+
+
+def forward_work(T, c, r, p, e, geo) -> Work:
+    rp = r * p
+    lr = geo.d > 1
+    flops = T * (c + 1) * (r + p) + 2 * rp * (2 * T + (geo.n + geo.m if lr else 0))
+    adds = (geo.nnzC * rp if lr else 0) + (T // c) * rp
+    by = (2 * r + 2 * p) * T * e + (2 * (geo.P + geo.B) * rp * 4 if lr else 0)
+    return Work(flops, adds, by)
+
+
+def backward_work(T, c, r, p, e, geo) -> Work:
+    rp = r * p
+    lr = geo.d > 1
+    flops = T * (c + 1) * (3 * r + 2 * p) + (15 if lr else 10) * T * rp
+    adds = (geo.nnzC * rp if lr else 0) + (T // c) * rp
+    by = (4 * r + 3 * p) * T * e + (2 * (2 * geo.P + 2 * geo.B) * rp * 4 if lr else 0)
+    return Work(flops, adds, by)
+
+
+def roofline_times(work: Work, peaks: dict, sustained: bool = True) -> dict:
+    """Seconds each ceiling needs for `work`, and the two path rooflines (2-term: every operation charged
+    at the tensor peak against the HBM term; 3-term: table additions charged at the fp32 add peak)."""
+    tflops = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"] * 1e12
+    hbm = peaks["hbm_gbs"] * 1e9
+    alu = 148 * 128 * peaks.get("sm_max_mhz", 1965.0) * 1e6
+    t_tensor = work.flops / tflops
+    t_alu = work.adds / alu
+    t_hbm = work.bytes / hbm
+    t2 = max((work.flops + work.adds) / tflops, t_hbm)
+    t3 = max(t_tensor, t_alu, t_hbm)
+    return {"t_tensor": t_tensor, "t_alu": t_alu, "t_hbm": t_hbm, "t_2term": t2, "t_3term": t3, "alu_peak_adds": alu}
+
+
+# Per-kernel algorithmic traffic (bytes), adds and flop, keyed by the stage names the library reports.
+def stage_work(name: str, T, c, r, p, e, geo) -> Work:
+    rp, NC = r * p, T // c
+    n, m, P, B = geo.n, geo.m, geo.P, geo.B
+    st = 4 * rp
+    table = {
+        "pool":        Work(2 * n * rp, 0, n * (r + p) * e + P * st),
+        "tabulate":    Work(0, geo.nnzC * rp, (P + B) * st),
+        "chunk_state": Work(2 * T * rp, 0, T * (r + p) * e + NC * st),
+        "scan":        Work(0, NC * rp, 2 * NC * st),
+        "scores":      Work(T * (c + 1) * r, 0, 2 * T * r * e + T * c * 4),
+        "read_chunk":  Work(2 * T * rp, 0, T * r * e + NC * st + T * p * 4),
+        "read_type":   Work(2 * m * rp, 0, m * r * e + B * st + 2 * m * p * 4),
+        "output":      Work(T * (c + 1) * p, 0, T * c * 4 + T * p * e + T * p * 4 + T * p * e),
+    }
+    return table.get(name, Work(0, 0, 0))
