@@ -151,12 +151,7 @@ void outer_sum(Ctx& cx, const char* name, int mode, const void* a, const void* b
   const smat_plan* pl = cx.pl;
   const int bf = pl->dtype == SMAT_BF16;
   const int64_t G = group_count(pl, mode);
-  SmatGemmArgs g{};
-  g.A = operand(a, bf, pl->T * pl->r, 0, 1, pl->r, 0, 1);
-  g.B = operand(b, bf, pl->T * pl->p, 0, pl->p, 1, 1, 0);
-  g.C = operand(state, 0, G * pl->rp, pl->rp, pl->p, 1);
-  g.M = pl->r; g.N = pl->p; g.tokK = 1; g.grp = group(pl, mode);
-  SMAT_TRY(cx, name, smat_launch_gemm(g, pl->r, pl->p, G, pl->bh, cx.st));
+  SMAT_TRY(cx, name, smat_launch_pool(a, b, bf, state, group(pl, mode), pl->T, G, pl->bh, pl->r, pl->p, cx.st));
 }
 
 // out[bh][t] (+)= x_t · state_g(t)  (transposed = 0: x: [T, r] contracts the first state index, out: [T, p];
@@ -168,6 +163,11 @@ void state_read(Ctx& cx, const char* name, int mode, const void* x, const float*
   const int bf = pl->dtype == SMAT_BF16;
   const int64_t G = group_count(pl, mode);
   const int kdim = transposed ? pl->p : pl->r, odim = transposed ? pl->r : pl->p;
+  if (mode != SMAT_GM_CHUNK && !out_final) {  // a handful of tokens per state: stream the state once
+    SMAT_TRY(cx, name, smat_launch_state_read(x, bf, state, transposed, acc_in, acc_out, group(pl, mode), pl->T, G,
+                                              pl->bh, pl->r, pl->p, cx.st));
+    return;
+  }
   SmatGemmArgs g{};
   g.A = operand(x, bf, pl->T * kdim, 0, kdim, 1, 1, 0);
   g.B = transposed ? operand(state, 0, G * pl->rp, pl->rp, 1, pl->p) : operand(state, 0, G * pl->rp, pl->rp, pl->p, 1);
@@ -224,12 +224,22 @@ smat_status check_common(const smat_plan* pl, const void* ws, size_t ws_bytes, i
 
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
 
+// Step 3 of Algorithm 1 (transpose = 0) or F̄ = Cᵀ Ū (transpose = 1).
+void tabulate(Ctx& cx, const char* name, const float* in, float* out, int transpose) {
+  const smat_plan* pl = cx.pl;
+  if (in == out) return;  // d = 2: hyperplanes are single points, the type table is the profile table
+  if (!(pl->flags & SMAT_FLAG_ALG2_TABULATION) && smat_tabulate_staged_slab(pl->geo, pl->rp, transpose) >= 4)
+    SMAT_TRY(cx, name, smat_launch_tabulate_staged(in, out, pl->geo, pl->rp, pl->bh, transpose, cx.st));
+  else
+    SMAT_TRY(cx, name, smat_launch_tabulate_alg2(in, out, pl->geo, pl->rp, pl->bh, transpose, cx.st));
+}
+
 // Steps 2-3 and 5-6 of Algorithm 1: the tables S_in, F, U.
 void build_forward_tables(Ctx& cx, const void* K, const void* V) {
   const smat_plan* pl = cx.pl;
   if (!pl->geo.dense_G) {
     outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));                                         // step 2
-    SMAT_TRY(cx, "tabulate", smat_launch_tabulate_alg2(cx.f(pl->off_F), cx.f(pl->off_U), pl->geo, pl->rp, pl->bh, 0, cx.st));  // step 3
+    tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0);                                 // step 3
   }
   outer_sum(cx, "chunk_state", SMAT_GM_CHUNK, K, V, cx.f(pl->off_sin));                                           // step 5
   scan_states(cx, "scan", cx.f(pl->off_sin), 0);                                                           // step 6
@@ -264,13 +274,15 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   size_t off = 0;
   pl->off_status = off; off = align_up(off + 256);
   pl->off_sin = off;    off = align_up(off + (size_t)pl->bh * pl->NC * state);
-  pl->off_F = off;      off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.P * state));
+  // d = 2: C is the identity (U_h = F_h), so the two tables share storage unless Algorithm 2 is forced
+  const bool alias = g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION);
+  pl->off_F = off;      off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.P * state));
   pl->off_U = off;      off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.B * state));
   pl->off_acc = off;    off = align_up(off + (size_t)pl->bh * T * wide * sizeof(float));
   pl->off_tileA = off;  off = align_up(off + (size_t)pl->bh * T * chunk * sizeof(float));
   pl->off_fwd_end = off;
   pl->off_dbar = off;   off = align_up(off + (size_t)pl->bh * pl->NC * state);
-  pl->off_ubar = off;   off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.B * state));
+  pl->off_ubar = off;   off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.B * state));
   pl->off_fbar = off;   off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.P * state));
   pl->off_tileG = off;  off = align_up(off + (size_t)pl->bh * T * chunk * sizeof(float));
   pl->off_bwd_end = off;
@@ -370,7 +382,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
   // long-range adjoints: Ū_h = Σ q dOᵀ over the type, F̄ = Cᵀ Ū   (Eq. "lr-adjoint")
   if (lr) {
     outer_sum(cx, "bwd_pool_type", SMAT_GM_TYPE, Q, dO, cx.f(pl->off_ubar));
-    SMAT_TRY(cx, "bwd_tabulate_t", smat_launch_tabulate_alg2(cx.f(pl->off_ubar), cx.f(pl->off_fbar), pl->geo, pl->rp, pl->bh, 1, cx.st));
+    tabulate(cx, "bwd_tabulate_t", cx.f(pl->off_ubar), cx.f(pl->off_fbar), 1);
   }
   tril_scores(cx, "bwd_scores_qk", Q, K, pl->r, tileA);    // A = tril(Q Kᵀ)
   tril_scores(cx, "bwd_scores_gv", dO, V, pl->p, tileG);   // tril(dO Vᵀ)

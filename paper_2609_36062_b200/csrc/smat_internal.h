@@ -72,3 +72,17 @@ cudaError_t smat_launch_tabulate_alg2(const float* in, float* out, const SmatGeo
 int smat_tabulate_alg2_slab(int64_t rows_in, int64_t state_elems);
 
 cudaError_t smat_launch_mask(uint8_t* mask, const SmatGeo& geo, cudaStream_t st);
+
+// Pooling of outer products into one fp32 state per group: state[bh][g] = Σ_{tokens of g} a_tᵀ b_t.
+cudaError_t smat_launch_pool(const void* A, const void* Bm, int bf16, float* state, const SmatGroupSpec& grp,
+                             int64_t Tlen, int64_t groups, int bh, int r, int p, cudaStream_t st);
+
+// Routed read of per-group states: acc_out[t] = acc_in[t] + x_t · state[g(t)] for the tokens of every group.
+cudaError_t smat_launch_state_read(const void* X, int bf16, const float* state, int transposed, const float* acc_in,
+                                   float* acc_out, const SmatGroupSpec& grp, int64_t Tlen, int64_t groups, int bh,
+                                   int r, int p, cudaStream_t st);
+
+// Staged exact tabulation (same sums as Algorithm 2, one coordinate at a time). Slab = 0: not available.
+int smat_tabulate_staged_slab(const SmatGeo& geo, int64_t state_elems, int transpose);
+cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatGeo& geo, int64_t state_elems, int bh,
+                                        int transpose, cudaStream_t st);

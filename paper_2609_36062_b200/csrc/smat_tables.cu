@@ -1,0 +1,390 @@
+// Long-range branch on the plain ALUs and HBM: pooling of outer products into per-group states, the
+// tabulation U = C F (staged exact sums for d = 3, 4) and its transpose, and the routed reads of
+// per-group states by the few tokens that share them.  None of these is a dense contraction worth a
+// tensor-core tile: every state is touched by a handful of tokens, so they are shaped for HBM streaming.
+#include <cuda_bf16.h>
+
+#include "smat_internal.h"
+
+namespace {
+
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+__device__ __forceinline__ float4 add4(float4 a, const float4 b) {
+  a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+  return a;
+}
+__device__ __forceinline__ float4 fma4(float s, const float4 b, float4 a) {
+  a.x = fmaf(s, b.x, a.x); a.y = fmaf(s, b.y, a.y); a.z = fmaf(s, b.z, a.z); a.w = fmaf(s, b.w, a.w);
+  return a;
+}
+
+// ---- pooling: state[g] = Σ_{tokens of g} a_tᵀ b_t ------------------------------------------------------------
+// One CTA per (group, head).  Tokens are staged 32 at a time; every thread owns one float4 column
+// strip of the state and NS rows of it, so the 64 KB state is written once with 512-byte rows.
+template <int R, int PD, typename T>
+__global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ A, const T* __restrict__ Bm,
+                                                   float* __restrict__ state, SmatGroupSpec grp, int64_t Tlen,
+                                                   int64_t groups) {
+  constexpr int TK = 32;
+  constexpr int NJ4 = PD / 4;
+  constexpr int NG = 256 / NJ4;
+  constexpr int NS = R / NG;
+  __shared__ __align__(16) float As[TK][R];
+  __shared__ __align__(16) float Bs[TK][PD];
+  const int64_t g = blockIdx.x, bh = blockIdx.y;
+  int64_t t0, ts, cnt;
+  smat_group_tokens(grp, g, &t0, &ts, &cnt);
+  const int tid = threadIdx.x;
+  const int j4 = tid % NJ4, ig = tid / NJ4;
+  float4 acc[NS];
+#pragma unroll
+  for (int s = 0; s < NS; ++s) acc[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+  const T* Ab = A + bh * Tlen * R;
+  const T* Bb = Bm + bh * Tlen * PD;
+  for (int64_t k0 = 0; k0 < cnt; k0 += TK) {
+    const int kn = (int)((cnt - k0) < TK ? (cnt - k0) : TK);
+    for (int idx = tid; idx < kn * R; idx += 256) {
+      const int k = idx / R, i = idx % R;
+      As[k][i] = to_float(Ab[(t0 + (k0 + k) * ts) * R + i]);
+    }
+    for (int idx = tid; idx < kn * PD; idx += 256) {
+      const int k = idx / PD, j = idx % PD;
+      Bs[k][j] = to_float(Bb[(t0 + (k0 + k) * ts) * PD + j]);
+    }
+    __syncthreads();
+    for (int k = 0; k < kn; ++k) {
+      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[k][j4 * 4]);
+#pragma unroll
+      for (int s = 0; s < NS; ++s) acc[s] = fma4(As[k][ig + s * NG], b4, acc[s]);
+    }
+    __syncthreads();
+  }
+  float* out = state + (bh * groups + g) * (int64_t)(R * PD);
+#pragma unroll
+  for (int s = 0; s < NS; ++s) *reinterpret_cast<float4*>(out + (int64_t)(ig + s * NG) * PD + j4 * 4) = acc[s];
+}
+
+// ---- routed read: out[t] = acc_in[t] + x_t · state[g(t)] ------------------------------------------------------
+// One CTA per (group, head) streams the 64 KB state once for up to KT tokens at a time.
+// TRANS = 0: x_t has R entries and contracts the first state index (output PD wide).
+// TRANS = 1: x_t has PD entries and contracts the second state index (output R wide).
+template <int R, int PD, int TRANS, typename T>
+__global__ void __launch_bounds__(256) state_read_kernel(const T* __restrict__ X, const float* __restrict__ state,
+                                                         const float* acc_in, float* acc_out, SmatGroupSpec grp,
+                                                         int64_t Tlen, int64_t groups) {
+  constexpr int KT = 8;
+  constexpr int NJ4 = PD / 4;
+  constexpr int NG = 256 / NJ4;        // row groups (one or more per warp)
+  constexpr int RPG = R / NG;          // state rows per group
+  constexpr int XD = TRANS ? PD : R;   // length of x_t
+  constexpr int OD = TRANS ? R : PD;   // length of the output row
+  __shared__ __align__(16) float Xs[KT][XD];
+  __shared__ __align__(16) float red[TRANS ? 1 : NG][KT][TRANS ? R : PD];
+  const int64_t g = blockIdx.x, bh = blockIdx.y;
+  int64_t t0, ts, cnt;
+  smat_group_tokens(grp, g, &t0, &ts, &cnt);
+  if (cnt == 0) return;
+  const int tid = threadIdx.x;
+  const int j4 = tid % NJ4, ig = tid / NJ4;
+  const float4* S4 = reinterpret_cast<const float4*>(state + (bh * groups + g) * (int64_t)(R * PD));
+  const T* Xb = X + bh * Tlen * XD;
+  for (int64_t k0 = 0; k0 < cnt; k0 += KT) {
+    const int kn = (int)((cnt - k0) < KT ? (cnt - k0) : KT);
+    for (int idx = tid; idx < KT * XD; idx += 256) {
+      const int k = idx / XD, i = idx % XD;
+      Xs[k][i] = k < kn ? to_float(Xb[(t0 + (k0 + k) * ts) * XD + i]) : 0.f;
+    }
+    __syncthreads();
+    if (!TRANS) {
+      float4 acc[KT];
+#pragma unroll
+      for (int k = 0; k < KT; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+      for (int s = 0; s < RPG; ++s) {
+        const int i = ig * RPG + s;
+        const float4 u = __ldg(S4 + i * NJ4 + j4);
+#pragma unroll
+        for (int k = 0; k < KT; ++k) acc[k] = fma4(Xs[k][i], u, acc[k]);
+      }
+#pragma unroll
+      for (int k = 0; k < KT; ++k) *reinterpret_cast<float4*>(&red[ig][k][j4 * 4]) = acc[k];
+      __syncthreads();
+      for (int idx = tid; idx < kn * PD; idx += 256) {
+        const int k = idx / PD, j = idx % PD;
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < NG; ++w) v += red[w][k][j];
+        const int64_t off = (bh * Tlen + t0 + (k0 + k) * ts) * OD + j;
+        acc_out[off] = v + (acc_in ? acc_in[off] : 0.f);
+      }
+    } else {
+      // every lane holds 4 columns of row i; the row sum is a reduction across the NJ4 lanes of the group
+#pragma unroll 2
+      for (int s = 0; s < RPG; ++s) {
+        const int i = ig * RPG + s;
+        const float4 u = __ldg(S4 + i * NJ4 + j4);
+        float part[KT];
+#pragma unroll
+        for (int k = 0; k < KT; ++k) {
+          const float4 x4 = *reinterpret_cast<const float4*>(&Xs[k][j4 * 4]);
+          part[k] = u.x * x4.x + u.y * x4.y + u.z * x4.z + u.w * x4.w;
+        }
+#pragma unroll
+        for (int off = NJ4 / 2; off > 0; off >>= 1)
+#pragma unroll
+          for (int k = 0; k < KT; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], off);
+        if (j4 == 0)
+#pragma unroll
+          for (int k = 0; k < KT; ++k) red[0][k][i] = part[k];
+      }
+      __syncthreads();
+      for (int idx = tid; idx < kn * R; idx += 256) {
+        const int k = idx / R, i = idx % R;
+        const int64_t off = (bh * Tlen + t0 + (k0 + k) * ts) * OD + i;
+        acc_out[off] = red[0][k][i] + (acc_in ? acc_in[off] : 0.f);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ---- staged exact tabulation -------------------------------------------------------------------------------------
+// U_{a,b} = Σ_{x : aᵀx = b} F_x for every normalised direction a and offset b (Algorithm 2), evaluated
+// one coordinate at a time instead of one hyperplane at a time.  For D = d-1 = 3 and a = (1, a2, a3):
+//     W_{a3}[u, x2]   = Σ_{x3} F[u - a3 x3, x2, x3]          (q adds for each of q^2 entries, per a3)
+//     U_{a,b}         = Σ_{x2} W_{a3}[b - a2 x2, x2]         (q adds for each of q^2 (a2, b) pairs, per a3)
+// which costs 2 q^4 state additions for the q^2 directions of this group instead of q^5; directions with
+// a leading zero work on F summed over x1 (and x2).  The sums are the same real numbers as Algorithm 2's,
+// added in a different order.  Every state entry is an independent copy of this map, so a CTA owns a slab
+// of E consecutive entries, keeps F[:, slab] in shared memory and writes U[:, slab].
+// Layout in shared memory: point index major, E floats per point; a thread owns one float4 of an item.
+template <int D>
+__global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __restrict__ in, float* __restrict__ out,
+                                                              int q, int64_t P, int64_t Bn, int64_t state_elems,
+                                                              int E) {
+  extern __shared__ __align__(16) float4 smem4[];
+  const int L4 = E / 4;            // float4 lanes per item
+  const int IPP = 256 / L4;        // items per pass
+  const int tid = threadIdx.x;
+  const int l = tid % L4, it0 = tid / L4;
+  const int64_t bh = blockIdx.y;
+  const int64_t e0 = (int64_t)blockIdx.x * E;
+  const int qq = q * q;
+  float4* Fs = smem4;                                  // [P][L4]
+  const float4* src = reinterpret_cast<const float4*>(in + bh * P * state_elems + e0);
+  const int64_t row4 = state_elems / 4;
+  for (int64_t idx = tid; idx < P * L4; idx += 256) {
+    const int64_t x = idx / L4;
+    Fs[idx] = __ldg(src + x * row4 + (idx - x * L4));
+  }
+  __syncthreads();
+  float4* dst = reinterpret_cast<float4*>(out + bh * Bn * state_elems + e0);
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  if (D == 2) {
+    // a = (1, a2):  U[a2*q + b] = Σ_{x2} F[(b - a2 x2) mod q, x2]
+    for (int item = it0; item < qq; item += IPP) {
+      const int a2 = item / q, b = item - a2 * q;
+      float4 acc = zero;
+      int x1 = b;
+      for (int x2 = 0; x2 < q; ++x2) {
+        acc = add4(acc, Fs[(x1 + q * x2) * L4 + l]);
+        x1 -= a2;
+        if (x1 < 0) x1 += q;
+      }
+      dst[(int64_t)item * row4 + l] = acc;
+    }
+    // a = (0, 1):  U[q*q + b] = Σ_{x1} F[x1, b]
+    for (int b = it0; b < q; b += IPP) {
+      float4 acc = zero;
+      for (int x1 = 0; x1 < q; ++x1) acc = add4(acc, Fs[(x1 + q * b) * L4 + l]);
+      dst[(int64_t)(qq + b) * row4 + l] = acc;
+    }
+  } else {
+    float4* G2 = Fs + P * L4;          // [q*q][L4]   F summed over x1, indexed x2 + q*x3
+    float4* W = G2 + (int64_t)qq * L4;  // [2][q*q][L4] double-buffered W_{a3}, indexed u + q*x2
+    for (int item = it0; item < qq; item += IPP) {
+      float4 acc = zero;
+      const float4* p = Fs + (int64_t)item * q * L4 + l;
+      for (int x1 = 0; x1 < q; ++x1) acc = add4(acc, p[x1 * L4]);
+      G2[item * L4 + l] = acc;
+    }
+    __syncthreads();
+    // a = (0, 1, a3):  U[(q^2 + a3) q + b] = Σ_{x3} G2[(b - a3 x3) mod q, x3]
+    for (int item = it0; item < qq; item += IPP) {
+      const int a3 = item / q, b = item - a3 * q;
+      float4 acc = zero;
+      int x2 = b;
+      for (int x3 = 0; x3 < q; ++x3) {
+        acc = add4(acc, G2[(x2 + q * x3) * L4 + l]);
+        x2 -= a3;
+        if (x2 < 0) x2 += q;
+      }
+      dst[(int64_t)(qq * q + item) * row4 + l] = acc;
+    }
+    // a = (0, 0, 1):  U[(q^2 + q) q + b] = Σ_{x2} G2[x2, b]
+    for (int b = it0; b < q; b += IPP) {
+      float4 acc = zero;
+      for (int x2 = 0; x2 < q; ++x2) acc = add4(acc, G2[(x2 + q * b) * L4 + l]);
+      dst[(int64_t)((qq + q) * q + b) * row4 + l] = acc;
+    }
+    // a = (1, a2, a3)
+    for (int a3 = 0; a3 < q; ++a3) {
+      float4* Wc = W + (int64_t)(a3 & 1) * qq * L4;
+      for (int item = it0; item < qq; item += IPP) {       // item = u + q*x2
+        const int x2 = item / q, u = item - x2 * q;
+        float4 acc = zero;
+        int x1 = u;
+        const float4* p = Fs + (int64_t)(q * x2) * L4 + l;
+        for (int x3 = 0; x3 < q; ++x3) {
+          acc = add4(acc, p[(x1 + qq * x3) * L4]);
+          x1 -= a3;
+          if (x1 < 0) x1 += q;
+        }
+        Wc[item * L4 + l] = acc;
+      }
+      __syncthreads();
+      for (int item = it0; item < qq; item += IPP) {       // item = b + q*a2
+        const int a2 = item / q, b = item - a2 * q;
+        float4 acc = zero;
+        int u = b;
+        for (int x2 = 0; x2 < q; ++x2) {
+          acc = add4(acc, Wc[(u + q * x2) * L4 + l]);
+          u -= a2;
+          if (u < 0) u += q;
+        }
+        const int64_t h = (int64_t)(a2 + q * a3) * q + b;
+        dst[h * row4 + l] = acc;
+      }
+    }
+  }
+}
+
+// Transpose for D = 2:  F̄[x1, x2] = Σ_{a2} Ū[(1,a2), x1 + a2 x2] + Ū[(0,1), x2]
+__global__ void __launch_bounds__(256) tabulate_staged_t2_kernel(const float* __restrict__ in, float* __restrict__ out,
+                                                                 int q, int64_t P, int64_t Bn, int64_t state_elems,
+                                                                 int E) {
+  extern __shared__ __align__(16) float4 smem4[];
+  const int L4 = E / 4, IPP = 256 / L4;
+  const int tid = threadIdx.x;
+  const int l = tid % L4, it0 = tid / L4;
+  const int64_t bh = blockIdx.y;
+  const int64_t e0 = (int64_t)blockIdx.x * E;
+  const int qq = q * q;
+  float4* Us = smem4;  // [Bn][L4]
+  const float4* src = reinterpret_cast<const float4*>(in + bh * Bn * state_elems + e0);
+  const int64_t row4 = state_elems / 4;
+  for (int64_t idx = tid; idx < Bn * L4; idx += 256) {
+    const int64_t h = idx / L4;
+    Us[idx] = __ldg(src + h * row4 + (idx - h * L4));
+  }
+  __syncthreads();
+  float4* dst = reinterpret_cast<float4*>(out + bh * P * state_elems + e0);
+  for (int item = it0; item < qq; item += IPP) {  // item = x1 + q*x2
+    const int x2 = item / q, x1 = item - x2 * q;
+    float4 acc = Us[(qq + x2) * L4 + l];
+    int b = x1;
+    for (int a2 = 0; a2 < q; ++a2) {
+      acc = add4(acc, Us[(a2 * q + b) * L4 + l]);
+      b += x2;
+      if (b >= q) b -= q;
+    }
+    dst[(int64_t)item * row4 + l] = acc;
+  }
+}
+
+template <typename K>
+cudaError_t set_smem(K kernel, size_t bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace
+
+// ---- launchers ------------------------------------------------------------------------------------------------------
+template <typename T>
+static cudaError_t launch_pool_t(const void* A, const void* Bm, float* state, const SmatGroupSpec& grp, int64_t Tlen,
+                                 int64_t groups, int bh, int r, int p, cudaStream_t st) {
+  dim3 grid((unsigned)groups, (unsigned)bh);
+  const T* a = static_cast<const T*>(A);
+  const T* b = static_cast<const T*>(Bm);
+  if (r == 128 && p == 128) pool_kernel<128, 128, T><<<grid, 256, 0, st>>>(a, b, state, grp, Tlen, groups);
+  else if (r == 64 && p == 64) pool_kernel<64, 64, T><<<grid, 256, 0, st>>>(a, b, state, grp, Tlen, groups);
+  else if (r == 64 && p == 128) pool_kernel<64, 128, T><<<grid, 256, 0, st>>>(a, b, state, grp, Tlen, groups);
+  else pool_kernel<128, 64, T><<<grid, 256, 0, st>>>(a, b, state, grp, Tlen, groups);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_pool(const void* A, const void* Bm, int bf16, float* state, const SmatGroupSpec& grp,
+                             int64_t Tlen, int64_t groups, int bh, int r, int p, cudaStream_t st) {
+  return bf16 ? launch_pool_t<__nv_bfloat16>(A, Bm, state, grp, Tlen, groups, bh, r, p, st)
+              : launch_pool_t<float>(A, Bm, state, grp, Tlen, groups, bh, r, p, st);
+}
+
+template <int TRANS, typename T>
+static cudaError_t launch_read_t(const void* X, const float* state, const float* acc_in, float* acc_out,
+                                 const SmatGroupSpec& grp, int64_t Tlen, int64_t groups, int bh, int r, int p,
+                                 cudaStream_t st) {
+  dim3 grid((unsigned)groups, (unsigned)bh);
+  const T* x = static_cast<const T*>(X);
+  if (r == 128 && p == 128)
+    state_read_kernel<128, 128, TRANS, T><<<grid, 256, 0, st>>>(x, state, acc_in, acc_out, grp, Tlen, groups);
+  else if (r == 64 && p == 64)
+    state_read_kernel<64, 64, TRANS, T><<<grid, 256, 0, st>>>(x, state, acc_in, acc_out, grp, Tlen, groups);
+  else if (r == 64 && p == 128)
+    state_read_kernel<64, 128, TRANS, T><<<grid, 256, 0, st>>>(x, state, acc_in, acc_out, grp, Tlen, groups);
+  else
+    state_read_kernel<128, 64, TRANS, T><<<grid, 256, 0, st>>>(x, state, acc_in, acc_out, grp, Tlen, groups);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_state_read(const void* X, int bf16, const float* state, int transposed, const float* acc_in,
+                                   float* acc_out, const SmatGroupSpec& grp, int64_t Tlen, int64_t groups, int bh,
+                                   int r, int p, cudaStream_t st) {
+  if (transposed)
+    return bf16 ? launch_read_t<1, __nv_bfloat16>(X, state, acc_in, acc_out, grp, Tlen, groups, bh, r, p, st)
+                : launch_read_t<1, float>(X, state, acc_in, acc_out, grp, Tlen, groups, bh, r, p, st);
+  return bf16 ? launch_read_t<0, __nv_bfloat16>(X, state, acc_in, acc_out, grp, Tlen, groups, bh, r, p, st)
+              : launch_read_t<0, float>(X, state, acc_in, acc_out, grp, Tlen, groups, bh, r, p, st);
+}
+
+// Shared-memory floats per slab entry the staged kernels need.
+static int64_t staged_rows(const SmatGeo& geo, int transpose) {
+  const int64_t q = geo.q;
+  if (geo.D == 2) return transpose ? geo.B : geo.P;
+  if (geo.D == 3 && !transpose) return geo.P + 3 * q * q;
+  return 0;
+}
+
+int smat_tabulate_staged_slab(const SmatGeo& geo, int64_t state_elems, int transpose) {
+  const int64_t rows = staged_rows(geo, transpose);
+  if (rows == 0) return 0;
+  // prefer two resident CTAs per SM (about 110 KB each) with at least 16 entries, else the largest slab that fits
+  const int64_t two = 110 * 1024, one = 220 * 1024;
+  for (int E = 32; E >= 16; E >>= 1)
+    if (rows * E * 4 <= two && state_elems % E == 0) return E;
+  for (int E = 32; E >= 4; E >>= 1)
+    if (rows * E * 4 <= one && state_elems % E == 0) return E;
+  return 0;
+}
+
+cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatGeo& geo, int64_t state_elems, int bh,
+                                        int transpose, cudaStream_t st) {
+  const int E = smat_tabulate_staged_slab(geo, state_elems, transpose);
+  if (E < 4) return cudaErrorInvalidConfiguration;
+  const size_t smem = (size_t)staged_rows(geo, transpose) * E * sizeof(float);
+  dim3 grid((unsigned)(state_elems / E), (unsigned)bh);
+  cudaError_t err;
+  if (geo.D == 2 && transpose) {
+    if ((err = set_smem(tabulate_staged_t2_kernel, smem)) != cudaSuccess) return err;
+    tabulate_staged_t2_kernel<<<grid, 256, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+  } else if (geo.D == 2) {
+    if ((err = set_smem(tabulate_staged_kernel<2>, smem)) != cudaSuccess) return err;
+    tabulate_staged_kernel<2><<<grid, 256, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+  } else {
+    if ((err = set_smem(tabulate_staged_kernel<3>, smem)) != cudaSuccess) return err;
+    tabulate_staged_kernel<3><<<grid, 256, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+  }
+  return cudaGetLastError();
+}

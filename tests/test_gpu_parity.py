@@ -87,6 +87,27 @@ def test_backward_matches_dense_oracle(d, T, dk, dv, c, dtype, q):
             assert rel_err(g, ref) <= TOL[dtype], (name, h, rel_err(g, ref))
 
 
+@pytest.mark.parametrize("d,T,c,q", [(2, 512, 32, 0), (3, 1024, 32, 0), (3, 2048, 64, 13), (4, 1024, 16, 3), (4, 2048, 64, 5)])
+@pytest.mark.parametrize("flags", [0, binding.FLAG_ALG2_TABULATION])
+def test_tabulation_variants_match_algorithm2(d, T, c, q, flags):
+    """Both the staged sums and the direct double loop of Algorithm 2 must give the oracle's type table,
+    and the transposed tabulation of the backward pass its adjoint."""
+    w = _small("tab", d, T, 64, 64, c, "f32", heads=1, seed=21)
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    plan = _plan(w, q, flags)
+    geo = so.geometry(T, c, d, q or None)
+    plan.forward(dev["q"], dev["k"], dev["v"])
+    F, U, _ = plan.debug_tables()
+    Q64, K64, V64, G64 = (synth.as_float64(w, host[x][0]) for x in ("q", "k", "v", "do"))
+    _, tab = cw.forward(Q64, K64, V64, geo, return_tables=True)
+    assert rel_err(to_numpy64(F[0]), tab["F"]) <= 1e-5
+    assert rel_err(to_numpy64(U[0]), tab["U"]) <= 1e-5
+    dQ, dK, dV = plan.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+    M = so.dense_mask(T, c, d, q or None)
+    for got, ref in zip((dQ, dK, dV), so.backward_dense(Q64, K64, V64, G64, M)):
+        assert rel_err(to_numpy64(got[0, 0]), ref) <= 1e-4
+
+
 def test_chunk_size_invariance_on_device():
     outs = []
     for c in (16, 32, 64, 128):
