@@ -11,9 +11,19 @@ namespace {
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-__device__ __forceinline__ float4 add4(float4 a, const float4 b) {
-  a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-  return a;
+// two packed fp32x2 additions (one instruction per pair on sm_100)
+__device__ __forceinline__ float4 add4(const float4 a, const float4 b) {
+  const float2 lo = __fadd2_rn(make_float2(a.x, a.y), make_float2(b.x, b.y));
+  const float2 hi = __fadd2_rn(make_float2(a.z, a.w), make_float2(b.z, b.w));
+  return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+// 16-byte asynchronous copy global -> shared, bypassing registers
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"((unsigned)__cvta_generic_to_shared(smem)), "l"(gmem)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
 }
 __device__ __forceinline__ float4 fma4(float s, const float4 b, float4 a) {
   a.x = fmaf(s, b.x, a.x); a.y = fmaf(s, b.y, a.y); a.z = fmaf(s, b.z, a.z); a.w = fmaf(s, b.w, a.w);
@@ -161,12 +171,13 @@ __global__ void __launch_bounds__(256) state_read_kernel(const T* __restrict__ X
 // of E consecutive entries, keeps F[:, slab] in shared memory and writes U[:, slab].
 // Layout in shared memory: point index major, E floats per point; a thread owns one float4 of an item.
 template <int D>
-__global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __restrict__ in, float* __restrict__ out,
+__global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* __restrict__ in, float* __restrict__ out,
                                                               int q, int64_t P, int64_t Bn, int64_t state_elems,
                                                               int E) {
   extern __shared__ __align__(16) float4 smem4[];
-  const int L4 = E / 4;            // float4 lanes per item
-  const int IPP = 256 / L4;        // items per pass
+  const int L4 = E / 4;                 // float4 lanes per item
+  const int NT = blockDim.x;
+  const int IPP = NT / L4;              // items per pass
   const int tid = threadIdx.x;
   const int l = tid % L4, it0 = tid / L4;
   const int64_t bh = blockIdx.y;
@@ -175,10 +186,11 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
   float4* Fs = smem4;                                  // [P][L4]
   const float4* src = reinterpret_cast<const float4*>(in + bh * P * state_elems + e0);
   const int64_t row4 = state_elems / 4;
-  for (int64_t idx = tid; idx < P * L4; idx += 256) {
+  for (int64_t idx = tid; idx < P * L4; idx += NT) {
     const int64_t x = idx / L4;
-    Fs[idx] = __ldg(src + x * row4 + (idx - x * L4));
+    cp_async16(Fs + idx, src + x * row4 + (idx - x * L4));
   }
+  cp_async_wait_all();
   __syncthreads();
   float4* dst = reinterpret_cast<float4*>(out + bh * Bn * state_elems + e0);
   const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -189,6 +201,7 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
       const int a2 = item / q, b = item - a2 * q;
       float4 acc = zero;
       int x1 = b;
+#pragma unroll 4
       for (int x2 = 0; x2 < q; ++x2) {
         acc = add4(acc, Fs[(x1 + q * x2) * L4 + l]);
         x1 -= a2;
@@ -199,6 +212,7 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
     // a = (0, 1):  U[q*q + b] = Σ_{x1} F[x1, b]
     for (int b = it0; b < q; b += IPP) {
       float4 acc = zero;
+#pragma unroll 4
       for (int x1 = 0; x1 < q; ++x1) acc = add4(acc, Fs[(x1 + q * b) * L4 + l]);
       dst[(int64_t)(qq + b) * row4 + l] = acc;
     }
@@ -208,6 +222,7 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
     for (int item = it0; item < qq; item += IPP) {
       float4 acc = zero;
       const float4* p = Fs + (int64_t)item * q * L4 + l;
+#pragma unroll 4
       for (int x1 = 0; x1 < q; ++x1) acc = add4(acc, p[x1 * L4]);
       G2[item * L4 + l] = acc;
     }
@@ -217,6 +232,7 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
       const int a3 = item / q, b = item - a3 * q;
       float4 acc = zero;
       int x2 = b;
+#pragma unroll 4
       for (int x3 = 0; x3 < q; ++x3) {
         acc = add4(acc, G2[(x2 + q * x3) * L4 + l]);
         x2 -= a3;
@@ -227,6 +243,7 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
     // a = (0, 0, 1):  U[(q^2 + q) q + b] = Σ_{x2} G2[x2, b]
     for (int b = it0; b < q; b += IPP) {
       float4 acc = zero;
+#pragma unroll 4
       for (int x2 = 0; x2 < q; ++x2) acc = add4(acc, G2[(x2 + q * b) * L4 + l]);
       dst[(int64_t)((qq + q) * q + b) * row4 + l] = acc;
     }
@@ -238,6 +255,7 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
         float4 acc = zero;
         int x1 = u;
         const float4* p = Fs + (int64_t)(q * x2) * L4 + l;
+#pragma unroll 4
         for (int x3 = 0; x3 < q; ++x3) {
           acc = add4(acc, p[(x1 + qq * x3) * L4]);
           x1 -= a3;
@@ -250,6 +268,7 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
         const int a2 = item / q, b = item - a2 * q;
         float4 acc = zero;
         int u = b;
+#pragma unroll 4
         for (int x2 = 0; x2 < q; ++x2) {
           acc = add4(acc, Wc[(u + q * x2) * L4 + l]);
           u -= a2;
@@ -263,11 +282,11 @@ __global__ void __launch_bounds__(256) tabulate_staged_kernel(const float* __res
 }
 
 // Transpose for D = 2:  F̄[x1, x2] = Σ_{a2} Ū[(1,a2), x1 + a2 x2] + Ū[(0,1), x2]
-__global__ void __launch_bounds__(256) tabulate_staged_t2_kernel(const float* __restrict__ in, float* __restrict__ out,
+__global__ void __launch_bounds__(1024, 1) tabulate_staged_t2_kernel(const float* __restrict__ in, float* __restrict__ out,
                                                                  int q, int64_t P, int64_t Bn, int64_t state_elems,
                                                                  int E) {
   extern __shared__ __align__(16) float4 smem4[];
-  const int L4 = E / 4, IPP = 256 / L4;
+  const int L4 = E / 4, NT = blockDim.x, IPP = NT / L4;
   const int tid = threadIdx.x;
   const int l = tid % L4, it0 = tid / L4;
   const int64_t bh = blockIdx.y;
@@ -276,16 +295,18 @@ __global__ void __launch_bounds__(256) tabulate_staged_t2_kernel(const float* __
   float4* Us = smem4;  // [Bn][L4]
   const float4* src = reinterpret_cast<const float4*>(in + bh * Bn * state_elems + e0);
   const int64_t row4 = state_elems / 4;
-  for (int64_t idx = tid; idx < Bn * L4; idx += 256) {
+  for (int64_t idx = tid; idx < Bn * L4; idx += NT) {
     const int64_t h = idx / L4;
-    Us[idx] = __ldg(src + h * row4 + (idx - h * L4));
+    cp_async16(Us + idx, src + h * row4 + (idx - h * L4));
   }
+  cp_async_wait_all();
   __syncthreads();
   float4* dst = reinterpret_cast<float4*>(out + bh * P * state_elems + e0);
   for (int item = it0; item < qq; item += IPP) {  // item = x1 + q*x2
     const int x2 = item / q, x1 = item - x2 * q;
     float4 acc = Us[(qq + x2) * L4 + l];
     int b = x1;
+#pragma unroll 4
     for (int a2 = 0; a2 < q; ++a2) {
       acc = add4(acc, Us[(a2 * q + b) * L4 + l]);
       b += x2;
@@ -375,16 +396,21 @@ cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatG
   if (E < 4) return cudaErrorInvalidConfiguration;
   const size_t smem = (size_t)staged_rows(geo, transpose) * E * sizeof(float);
   dim3 grid((unsigned)(state_elems / E), (unsigned)bh);
+  // threads: one (item, float4 lane) unit each, q^2 items per stage, split evenly over as few passes as possible
+  const int64_t units = (int64_t)geo.q * geo.q * (E / 4);
+  const int64_t passes = (units + 1023) / 1024;
+  int nt = (int)(((units + passes - 1) / passes + 31) / 32 * 32);
+  if (nt < 128) nt = 128;
   cudaError_t err;
   if (geo.D == 2 && transpose) {
     if ((err = set_smem(tabulate_staged_t2_kernel, smem)) != cudaSuccess) return err;
-    tabulate_staged_t2_kernel<<<grid, 256, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+    tabulate_staged_t2_kernel<<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
   } else if (geo.D == 2) {
     if ((err = set_smem(tabulate_staged_kernel<2>, smem)) != cudaSuccess) return err;
-    tabulate_staged_kernel<2><<<grid, 256, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+    tabulate_staged_kernel<2><<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
   } else {
     if ((err = set_smem(tabulate_staged_kernel<3>, smem)) != cudaSuccess) return err;
-    tabulate_staged_kernel<3><<<grid, 256, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+    tabulate_staged_kernel<3><<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
   }
   return cudaGetLastError();
 }
