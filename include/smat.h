@@ -84,6 +84,10 @@ void smat_plan_destroy(smat_plan* plan);
 
 smat_status smat_get_geometry(const smat_plan* plan, smat_geometry* out);
 
+/* 1 when this plan runs its causal branch on the tcgen05 tensor-core kernels (bf16, d_k = d_v = 128, block
+ * boundary and recent length multiples of 128, SMAT_FLAG_SIMT_ONLY not set), 0 when it runs on the fp32 ALUs. */
+int smat_uses_tensor_cores(const smat_plan* plan);
+
 /* Bytes of workspace smat_forward (for_backward = 0) or smat_backward (for_backward = 1) needs. 0 if plan is NULL. */
 size_t smat_workspace_bytes(const smat_plan* plan, int for_backward);
 
@@ -128,6 +132,8 @@ smat_status smat_debug_mask(const smat_plan* plan, uint8_t* mask, void* cuda_str
  *   Sin [batch*heads, T/chunk, d_k, d_v] incoming chunk states (Sec. 3.1, causal branch)
  * For d = 1 there is no separate F/U: the single state U_0 = F_0 is carried by the scan, and
  * F and U receive that state (the incoming state of the first recent chunk).
+ * Plans that use the tensor-core kernels keep S_in as bf16 128-token tiles: for them Sin (and, for d = 1,
+ * F and U) must be NULL, otherwise SMAT_ERR_UNSUPPORTED is returned.
  * Asynchronous on `cuda_stream`.
  */
 smat_status smat_debug_tables(const smat_plan* plan, const void* workspace, float* F, float* U, float* Sin,

@@ -22,7 +22,7 @@ FLAG_ALG2_TABULATION = 2
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
-    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read",
+    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores",
 ]
 
 
@@ -87,6 +87,8 @@ def load_library() -> ctypes.CDLL:
     lib.smat_check_status.restype = i
     lib.smat_last_launch_count.argtypes = [vp]
     lib.smat_last_launch_count.restype = i
+    lib.smat_uses_tensor_cores.argtypes = [vp]
+    lib.smat_uses_tensor_cores.restype = i
     lib.smat_profile_enable.argtypes = [vp, i]
     lib.smat_profile_enable.restype = i
     lib.smat_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float), i]
@@ -143,6 +145,9 @@ class SmatPlan:
         g = _Geometry()
         _check(self.lib.smat_get_geometry(self.handle, ctypes.byref(g)), "smat_get_geometry")
         return Geometry(g.T, g.c, g.n, g.m, g.d, g.q, g.P, g.A, g.B, g.nnzC, bool(g.vc_conditions_met))
+
+    def uses_tensor_cores(self) -> bool:
+        return bool(self.lib.smat_uses_tensor_cores(self.handle))
 
     def workspace_bytes(self, for_backward: bool = False) -> int:
         return int(self.lib.smat_workspace_bytes(self.handle, int(for_backward)))
@@ -219,9 +224,13 @@ class SmatPlan:
         b, h, T, dk, dv = self.shape
         g = self.geometry()
         ws = self._ws if workspace is None else workspace
-        F = torch.empty((b * h, g.P, dk, dv), dtype=torch.float32, device=ws.device)
-        U = torch.empty((b * h, g.B, dk, dv), dtype=torch.float32, device=ws.device)
-        Sin = torch.empty((b * h, T // g.c, dk, dv), dtype=torch.float32, device=ws.device)
+        tc = self.uses_tensor_cores()
+        F = U = Sin = None
+        if not (tc and g.d == 1):
+            F = torch.empty((b * h, g.P, dk, dv), dtype=torch.float32, device=ws.device)
+            U = torch.empty((b * h, g.B, dk, dv), dtype=torch.float32, device=ws.device)
+        if not tc:
+            Sin = torch.empty((b * h, T // g.c, dk, dv), dtype=torch.float32, device=ws.device)
         _check(self.lib.smat_debug_tables(self.handle, _ptr(ws), _ptr(F), _ptr(U), _ptr(Sin), _stream(stream)),
                "smat_debug_tables")
         return F, U, Sin

@@ -22,6 +22,7 @@ struct smat_plan {
   // workspace layout (byte offsets, 256-byte aligned)
   size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_fwd_end;
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
+  bool tc;             // tensor-core kernels for the causal branch
   mutable int launches;
   // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
   mutable bool profiling;
@@ -268,6 +269,8 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   smat_status s = build_geometry(&pl->geo, T, chunk, d, q_override);
   if (s != SMAT_OK) { delete pl; return s; }
   const SmatGeo& g = pl->geo;
+  pl->tc = dtype == SMAT_BF16 && d_k == 128 && d_v == 128 && !(flags & SMAT_FLAG_SIMT_ONLY) && g.n % 128 == 0 &&
+           g.m % 128 == 0 && g.n >= 128 && smat_tc_available();
   if (!g.dense_G && (smat_tabulate_alg2_slab(g.B, pl->rp) < 1)) { delete pl; return SMAT_ERR_UNSUPPORTED; }
   const size_t state = (size_t)pl->rp * sizeof(float);
   const int wide = d_k > d_v ? d_k : d_v;
@@ -332,6 +335,8 @@ smat_status smat_get_geometry(const smat_plan* pl, smat_geometry* out) {
   return SMAT_OK;
 }
 
+int smat_uses_tensor_cores(const smat_plan* pl) { return pl && pl->tc ? 1 : 0; }
+
 size_t smat_workspace_bytes(const smat_plan* pl, int for_backward) {
   if (!pl) return 0;
   return for_backward ? pl->off_bwd_end : pl->off_fwd_end;
@@ -346,6 +351,23 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  if (pl->tc) {
+    int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
+    float* ylr = cx.f(pl->off_acc);
+    const bool lr = !pl->geo.dense_G;
+    if (lr) {
+      outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));                         // step 2
+      tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0);                         // step 3
+      state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);  // step 4
+    }
+    SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, pl->geo.n,
+                                                             lr ? 0 : 1, status, cx.st));   // steps 5-6
+    SMAT_TRY(cx, "chunk_output_tc", smat_launch_chunk_output_tc(Q, K, V, cx.ws + pl->off_sin, ylr,
+                                                                 lr ? pl->geo.n : pl->T, O, pl->T, pl->bh, status,
+                                                                 cx.st));                   // step 7
+    pl->launches = cx.launches;
+    return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+  }
   build_forward_tables(cx, K, V);
   float* acc = cx.f(pl->off_acc);
   float* tileA = cx.f(pl->off_tileA);
@@ -441,6 +463,7 @@ smat_status smat_debug_tables(const smat_plan* pl, const void* workspace, float*
   const char* ws = static_cast<const char*>(workspace);
   const size_t state = (size_t)pl->rp * sizeof(float);
   cudaError_t err = cudaSuccess;
+  if (pl->tc && (Sin || (pl->geo.dense_G && (F || U)))) return SMAT_ERR_UNSUPPORTED;  // tensor-core path keeps S_in as bf16 tiles
   if (Sin) err = cudaMemcpyAsync(Sin, ws + pl->off_sin, (size_t)pl->bh * pl->NC * state, cudaMemcpyDeviceToDevice, st);
   if (pl->geo.dense_G) {
     const int64_t first_recent = pl->geo.n / pl->c;

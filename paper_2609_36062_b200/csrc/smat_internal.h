@@ -86,3 +86,14 @@ cudaError_t smat_launch_state_read(const void* X, int bf16, const float* state, 
 int smat_tabulate_staged_slab(const SmatGeo& geo, int64_t state_elems, int transpose);
 cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatGeo& geo, int64_t state_elems, int bh,
                                         int transpose, cudaStream_t st);
+
+// Tensor-core kernels of the causal branch (bf16, d_k = d_v = 128, 128-token tiles; n and T - n multiples of 128).
+bool smat_tc_available();
+// S_in[bh][tile] (bf16 [128][128]) = exclusive prefix sum of K_bᵀ V_b over the tiles of each block;
+// through = 1 runs one scan over the whole sequence (d = 1), else the scan restarts at token n.
+cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf16, int64_t T, int bh, int64_t n,
+                                      int through, int* status, cudaStream_t st);
+// O_b = Q_b S_in[b] + tril(Q_b K_bᵀ) V_b (+ ylr rows for tokens >= n_lr).
+cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
+                                        const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,
+                                        cudaStream_t st);

@@ -1,0 +1,390 @@
+// Causal branch of Algorithm 1 on the 5th-generation tensor cores (bf16 inputs, d_k = d_v = 128,
+// 128-token tiles): tcgen05.mma with TMEM accumulators, operands staged by TMA into 128-byte-swizzled
+// shared memory.
+//
+//   chunk_scan_tc_kernel   : D_b = K_bᵀ V_b for the chunks of one block in order, with the exclusive
+//                            prefix sum carried in registers; emits S_in[b] as bf16        (steps 5-6)
+//   chunk_output_tc_kernel : O_b = Q_b S_in[b] + tril(Q_b K_bᵀ) V_b + Y_lr,b               (step 7, Eq. "local")
+//
+// The tile width is 128 tokens whatever chunk size the caller named: the result does not depend on the
+// chunk width once the block boundary n is fixed, and the launcher requires n and T - n to be multiples of 128.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "smat_internal.h"
+#include "smat_tc.cuh"
+
+namespace {
+
+using namespace tc;
+
+constexpr int TILE = 128;              // tokens per tile, and d_k = d_v
+constexpr int HALF = 64;               // columns per 128-byte swizzled row
+constexpr int BOX_BYTES = TILE * 128;  // one TMA box: 128 rows x 128 bytes = 16 KB
+
+// ---------------------------------------------------------------------------------------------------------------
+// chunk_scan_tc_kernel: one CTA per (head, block, 64-column half of the state).
+//   warp 4 lane 0 : TMA producer (K_b: two boxes, V_b[:, half]: one box) into a 3-stage ring
+//   warp 5 lane 0 : MMA issuer, D_b = K_bᵀ V_b[:, half]  (M = 128 features, N = 64, K = 128 tokens) into a 4-deep TMEM ring
+//   warps 0-3     : one TMEM lane (state row) per thread; keep the running sum in registers, write it as bf16
+//                   (the state *before* chunk b is S_in[b]), then add D_b
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int SCAN_STAGES = 3;
+constexpr int SCAN_DBUF = 4;
+constexpr int SCAN_STAGE_BYTES = 3 * BOX_BYTES;
+constexpr int SCAN_SMEM = SCAN_STAGES * SCAN_STAGE_BYTES + 1024 + 256;
+
+struct ScanParams {
+  int64_t T;        // tokens per head
+  int NC;           // tiles per head
+  int lo[2], hi[2]; // tile ranges of the (up to two) blocks
+  __nv_bfloat16* Sin;  // [bh][NC][128][128]
+  int* status;
+};
+
+__global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                            const __grid_constant__ CUtensorMap tmV,
+                                                            const ScanParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SCAN_STAGES * SCAN_STAGE_BYTES);
+  uint64_t* full = bars;                     // [SCAN_STAGES]
+  uint64_t* empty = bars + SCAN_STAGES;      // [SCAN_STAGES]
+  uint64_t* dfull = empty + SCAN_STAGES;     // [SCAN_DBUF]
+  uint64_t* dempty = dfull + SCAN_DBUF;      // [SCAN_DBUF]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(dempty + SCAN_DBUF);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int half = blockIdx.x & 1, blk = blockIdx.x >> 1;
+  const int bh = blockIdx.y;
+  const int lo = prm.lo[blk], hi = prm.hi[blk];
+  const WaitCtx wc{cta_abort, prm.status};
+
+  if (threadIdx.x == 0) {
+    *cta_abort = 0;
+    for (int s = 0; s < SCAN_STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    for (int s = 0; s < SCAN_DBUF; ++s) { mbar_init(dfull + s, 1); mbar_init(dempty + s, 4); }
+    fence_barrier_init();
+  }
+  if (warp == 4) tmem_alloc(tmem_slot, SCAN_DBUF * HALF);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4 && lane == 0) {
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+    for (int b = lo; b + 1 < hi; ++b) {  // the last tile's own sum is never read
+      const int it = b - lo, s = it % SCAN_STAGES;
+      if (it >= SCAN_STAGES && !mbar_wait(empty + s, ((it / SCAN_STAGES) - 1) & 1, wc)) break;
+      uint8_t* st = smem + s * SCAN_STAGE_BYTES;
+      const int row = (int)(bh * prm.T + (int64_t)b * TILE);
+      mbar_expect_tx(full + s, SCAN_STAGE_BYTES);
+      tma_load_2d(st, &tmK, 0, row, full + s);
+      tma_load_2d(st + BOX_BYTES, &tmK, HALF, row, full + s);
+      tma_load_2d(st + 2 * BOX_BYTES, &tmV, half * HALF, row, full + s);
+    }
+  } else if (warp == 5 && lane == 0) {
+    constexpr uint32_t idesc = make_idesc(TILE, HALF, 1, 1);
+    for (int b = lo; b + 1 < hi; ++b) {
+      const int it = b - lo, s = it % SCAN_STAGES, db = it % SCAN_DBUF;
+      if (!mbar_wait(full + s, (it / SCAN_STAGES) & 1, wc)) break;
+      if (it >= SCAN_DBUF && !mbar_wait(dempty + db, ((it / SCAN_DBUF) - 1) & 1, wc)) break;
+      fence_after_sync();
+      const uint32_t sK = smem_u32(smem + s * SCAN_STAGE_BYTES);
+      const uint32_t sV = sK + 2 * BOX_BYTES;
+      const uint64_t dA = make_desc(sK, BOX_BYTES, 1024);  // K_b as MN-major A: two 64-feature blocks 16 KB apart
+      const uint64_t dB = make_desc(sV, BOX_BYTES, 1024);
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk)  // 16 tokens per instruction = two 8-row groups = 2048 bytes
+        mma_bf16(tmem_base + db * HALF, dA + (uint64_t)(kk * 128), dB + (uint64_t)(kk * 128), idesc, kk != 0);
+      mma_commit(empty + s);
+      mma_commit(dfull + db);
+    }
+  } else if (warp < 4) {
+    const int row = warp * 32 + lane;  // state row i (TMEM lane)
+    float acc[HALF];
+#pragma unroll
+    for (int j = 0; j < HALF; ++j) acc[j] = 0.f;
+    for (int b = lo; b < hi; ++b) {
+      const int it = b - lo, db = it % SCAN_DBUF;
+      // S_in[b] = running sum before this tile
+      uint4* dst = reinterpret_cast<uint4*>(prm.Sin + (((int64_t)bh * prm.NC + b) * TILE + row) * TILE + half * HALF);
+#pragma unroll
+      for (int j8 = 0; j8 < HALF / 8; ++j8) {
+        uint4 pk;
+        pk.x = pack_bf16(acc[j8 * 8 + 0], acc[j8 * 8 + 1]);
+        pk.y = pack_bf16(acc[j8 * 8 + 2], acc[j8 * 8 + 3]);
+        pk.z = pack_bf16(acc[j8 * 8 + 4], acc[j8 * 8 + 5]);
+        pk.w = pack_bf16(acc[j8 * 8 + 6], acc[j8 * 8 + 7]);
+        dst[j8] = pk;
+      }
+      if (b + 1 == hi) break;  // every issued MMA has been consumed: nothing is in flight at teardown
+      if (!mbar_wait(dfull + db, (it / SCAN_DBUF) & 1, wc)) break;
+      fence_after_sync();
+      uint32_t v0[32], v1[32];
+      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + db * HALF;
+      tmem_ld32(taddr, v0);
+      tmem_ld32(taddr + 32, v1);
+      tmem_ld_wait();
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(dempty + db);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        acc[j] += __uint_as_float(v0[j]);
+        acc[32 + j] += __uint_as_float(v1[j]);
+      }
+    }
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after_sync();
+    tmem_dealloc(tmem_base, SCAN_DBUF * HALF);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// chunk_output_tc_kernel: one CTA per (tile, head, 64-column half of the output).
+//   warp 4 lane 0 : TMA loads (Q_b, K_b: two boxes each; V_b[:, half], S_in[b][:, half]: one box each), then the MMAs
+//        MMA1  Sc = Q_b K_bᵀ                 (M = N = 128 tokens, K = 128)            -> TMEM columns [0, 128)
+//        MMA2  Oh = Q_b S_in[b][:, half]     (M = 128, N = 64, K = 128)               -> TMEM columns [128, 192)
+//        MMA3  Oh += P V_b[:, half]          (P = tril(Sc) in bf16, written over K_b)
+//   warps 0-3     : one query row per thread: mask and round the scores into the swizzled K-major layout,
+//                   later read Oh, add the long-range term and store the output row
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int OUT_SMEM = 6 * BOX_BYTES + 1024 + 256;
+
+struct OutParams {
+  int64_t T;
+  int NC;
+  int64_t n_lr;          // rows t >= n_lr add ylr (T: none)
+  const float* ylr;      // [bh][T][128] fp32 long-range term (rows >= n_lr valid)
+  __nv_bfloat16* O;      // [bh][T][128]
+  int* status;
+};
+
+__global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+                                                              const __grid_constant__ CUtensorMap tmK,
+                                                              const __grid_constant__ CUtensorMap tmV,
+                                                              const __grid_constant__ CUtensorMap tmS,
+                                                              const OutParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;                    // 2 boxes (K-major, k-blocks 0 and 1)
+  uint8_t* sK = smem + 2 * BOX_BYTES;    // 2 boxes; reused for P
+  uint8_t* sV = smem + 4 * BOX_BYTES;    // 1 box (MN-major)
+  uint8_t* sS = smem + 5 * BOX_BYTES;    // 1 box (MN-major)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 6 * BOX_BYTES);
+  uint64_t* bar_qk = bars + 0;
+  uint64_t* bar_vs = bars + 1;
+  uint64_t* bar_sc = bars + 2;   // scores in TMEM
+  uint64_t* bar_p = bars + 3;    // P in shared memory (128 arrivals)
+  uint64_t* bar_o = bars + 4;    // output in TMEM
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int half = blockIdx.x & 1, b = blockIdx.x >> 1;
+  const int bh = blockIdx.y;
+  const int64_t row0 = (int64_t)bh * prm.T + (int64_t)b * TILE;
+  const WaitCtx wc{cta_abort, prm.status};
+
+  if (threadIdx.x == 0) {
+    *cta_abort = 0;
+    mbar_init(bar_qk, 1); mbar_init(bar_vs, 1); mbar_init(bar_sc, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+    fence_barrier_init();
+  }
+  if (warp == 4) tmem_alloc(tmem_slot, 256);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_sc = tmem_base, tmem_o = tmem_base + TILE;
+
+  if (warp == 4 && lane == 0) {
+    mbar_expect_tx(bar_qk, 4 * BOX_BYTES);
+    tma_load_2d(sQ, &tmQ, 0, (int)row0, bar_qk);
+    tma_load_2d(sQ + BOX_BYTES, &tmQ, HALF, (int)row0, bar_qk);
+    tma_load_2d(sK, &tmK, 0, (int)row0, bar_qk);
+    tma_load_2d(sK + BOX_BYTES, &tmK, HALF, (int)row0, bar_qk);
+    mbar_expect_tx(bar_vs, 2 * BOX_BYTES);
+    tma_load_2d(sV, &tmV, half * HALF, (int)row0, bar_vs);
+    tma_load_2d(sS, &tmS, half * HALF, (int)(((int64_t)bh * prm.NC + b) * TILE), bar_vs);
+
+    constexpr uint32_t idesc_sc = make_idesc(TILE, TILE, 0, 0);
+    constexpr uint32_t idesc_o = make_idesc(TILE, HALF, 0, 1);
+    bool ok = mbar_wait(bar_qk, 0, wc);
+    if (ok) {
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) {  // k-block kk/4 (16 KB apart), 32 bytes per 16 k-elements inside it
+        const uint64_t dA = make_desc(smem_u32(sQ) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = make_desc(smem_u32(sK) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        mma_bf16(tmem_sc, dA, dB, idesc_sc, kk != 0);
+      }
+      mma_commit(bar_sc);
+      ok = mbar_wait(bar_vs, 0, wc);
+    }
+    if (ok) {
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) {
+        const uint64_t dA = make_desc(smem_u32(sQ) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = make_desc(smem_u32(sS) + kk * 2048, BOX_BYTES, 1024);
+        mma_bf16(tmem_o, dA, dB, idesc_o, kk != 0);
+      }
+      ok = mbar_wait(bar_p, 0, wc);
+    }
+    if (ok) {
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) {
+        const uint64_t dA = make_desc(smem_u32(sK) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = make_desc(smem_u32(sV) + kk * 2048, BOX_BYTES, 1024);
+        mma_bf16(tmem_o, dA, dB, idesc_o, 1);
+      }
+      mma_commit(bar_o);
+    }
+  } else if (warp < 4) {
+    const int m = warp * 32 + lane;  // query row inside the tile = TMEM lane
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    if (mbar_wait(bar_sc, 0, wc)) {
+      fence_after_sync();
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_sc + lane_base + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {  // 16-byte chunk = 8 keys
+          uint32_t pk[4];
+#pragma unroll
+          for (int h2 = 0; h2 < 4; ++h2) {
+            const int k0 = cb * 32 + i * 8 + h2 * 2;
+            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
+            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            pk[h2] = pack_bf16(lo, hi);
+          }
+          const int j8 = cb * 4 + i;  // chunk index along the key dimension, 0..15
+          uint8_t* dst = sK + (j8 >> 3) * BOX_BYTES + m * 128 + (((j8 & 7) ^ (m & 7)) << 4);
+          *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
+      fence_proxy_async();
+      fence_before_sync();
+      mbar_arrive(bar_p);
+      if (mbar_wait(bar_o, 0, wc)) {
+        fence_after_sync();
+        const int64_t t = (int64_t)b * TILE + m;
+        const bool add_lr = t >= prm.n_lr;
+        const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+        uint4* dst = reinterpret_cast<uint4*>(prm.O + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+          uint32_t v[32];
+          tmem_ld32(tmem_o + lane_base + cb * 32, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i * 8 + e]);
+            if (add_lr) {
+              const float4 a = __ldg(y4 + cb * 8 + i * 2), c = __ldg(y4 + cb * 8 + i * 2 + 1);
+              f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
+              f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
+            }
+            dst[cb * 4 + i] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
+                                         pack_bf16(f[6], f[7]));
+          }
+        }
+      }
+    }
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after_sync();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
+// ---- host: tensor maps ----------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, 128] row-major, box = 64 columns x 128 rows, 128-byte swizzle
+bool make_map(CUtensorMap* map, const void* base, uint64_t rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)TILE, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)TILE * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)HALF, (cuuint32_t)TILE};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool smat_tc_available() { return encode_fn() != nullptr; }
+
+cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf16, int64_t T, int bh, int64_t n,
+                                      int through, int* status, cudaStream_t st) {
+  CUtensorMap tmK, tmV;
+  if (!make_map(&tmK, K, (uint64_t)bh * T) || !make_map(&tmV, V, (uint64_t)bh * T)) return cudaErrorInvalidValue;
+  ScanParams prm;
+  prm.T = T; prm.NC = (int)(T / TILE);
+  prm.Sin = static_cast<__nv_bfloat16*>(Sin_bf16);
+  prm.status = status;
+  int blocks;
+  if (through) {  // d = 1: the single state U_0 = F_0 is the carry across the boundary
+    blocks = 1; prm.lo[0] = 0; prm.hi[0] = prm.NC; prm.lo[1] = prm.hi[1] = 0;
+  } else {
+    blocks = 2; prm.lo[0] = 0; prm.hi[0] = (int)(n / TILE); prm.lo[1] = prm.hi[0]; prm.hi[1] = prm.NC;
+  }
+  cudaError_t err = cudaFuncSetAttribute(chunk_scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM);
+  if (err != cudaSuccess) return err;
+  dim3 grid((unsigned)(blocks * 2), (unsigned)bh);
+  chunk_scan_tc_kernel<<<grid, 192, SCAN_SMEM, st>>>(tmK, tmV, prm);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
+                                        const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,
+                                        cudaStream_t st) {
+  CUtensorMap tmQ, tmK, tmV, tmS;
+  const int NC = (int)(T / TILE);
+  if (!make_map(&tmQ, Q, (uint64_t)bh * T) || !make_map(&tmK, K, (uint64_t)bh * T) ||
+      !make_map(&tmV, V, (uint64_t)bh * T) || !make_map(&tmS, Sin_bf16, (uint64_t)bh * NC * TILE))
+    return cudaErrorInvalidValue;
+  OutParams prm;
+  prm.T = T; prm.NC = NC; prm.n_lr = n_lr; prm.ylr = ylr;
+  prm.O = static_cast<__nv_bfloat16*>(O);
+  prm.status = status;
+  cudaError_t err =
+      cudaFuncSetAttribute(chunk_output_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, OUT_SMEM);
+  if (err != cudaSuccess) return err;
+  dim3 grid((unsigned)(NC * 2), (unsigned)bh);
+  chunk_output_tc_kernel<<<grid, 160, OUT_SMEM, st>>>(tmQ, tmK, tmV, tmS, prm);
+  return cudaGetLastError();
+}
