@@ -281,6 +281,115 @@ __global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* _
   }
 }
 
+// ---- D = 3 with the whole q x q image of a sub-problem held in registers --------------------------------------------
+// For a fixed x2 (and one state entry) the sums W_{a3}[u, x2] = Σ_{x3} F[u - a3 x3, x2, x3] over all (a3, u) are
+// the finite Radon transform of the q x q image F[., x2, .]: q^2 inputs, q^2 outputs, q^3 additions.  A thread
+// loads one image into registers, forms every line sum with compile-time indices (no address arithmetic, no
+// shared-memory read per addition) and writes the q^2 results back over the image it read.  The second stage is
+// the same transform of the image W_{a3}[., .] for a fixed a3; its results again replace the image, which leaves
+// rows 0 .. q^3-1 of U in the slab, in order, ready for a coalesced copy out.
+template <int Q, int A>
+struct RadonSlope {
+  // line sums of slope A: out[u] = Σ_y img[y][(u - A y) mod Q], stored with stride `os`
+  static __device__ __forceinline__ void run(const float (&img)[Q][Q], float* out, int os) {
+#pragma unroll
+    for (int u = 0; u < Q; ++u) {
+      float sum = img[0][u];
+#pragma unroll
+      for (int y = 1; y < Q; ++y) sum += img[y][((u - A * y) % Q + Q) % Q];
+      out[u * os] = sum;
+    }
+  }
+};
+template <int Q>
+__device__ __forceinline__ void radon_dispatch(int a, const float (&img)[Q][Q], float* out, int os) {
+#define SMAT_SLOPE(k) \
+  case k:             \
+    if constexpr (k < Q) RadonSlope<Q, (k < Q ? k : 0)>::run(img, out, os); \
+    break;
+  switch (a) {
+    SMAT_SLOPE(0) SMAT_SLOPE(1) SMAT_SLOPE(2) SMAT_SLOPE(3) SMAT_SLOPE(4) SMAT_SLOPE(5) SMAT_SLOPE(6)
+    SMAT_SLOPE(7) SMAT_SLOPE(8) SMAT_SLOPE(9) SMAT_SLOPE(10) SMAT_SLOPE(11) SMAT_SLOPE(12)
+    default: break;
+  }
+#undef SMAT_SLOPE
+}
+
+// One in-place transform: image[y][x] at base[(x * sx + y * sy) * E], slope a results to base[(x * sx + a * sy) * E].
+template <int Q, int E>
+__device__ __noinline__ void radon_inplace(float* base, int sx, int sy) {
+  float img[Q][Q];
+#pragma unroll
+  for (int y = 0; y < Q; ++y)
+#pragma unroll
+    for (int x = 0; x < Q; ++x) img[y][x] = base[(x * sx + y * sy) * E];
+#pragma unroll 1
+  for (int a = 0; a < Q; ++a) radon_dispatch<Q>(a, img, base + a * sy * E, sx * E);
+}
+
+template <int Q, int E>
+__global__ void __launch_bounds__((Q * E + 31) / 32 * 32, Q <= 11 ? 2 : 1)
+    tabulate_radon3_kernel(const float* __restrict__ in, float* __restrict__ out, int P, int Bn, int64_t state_elems) {
+  extern __shared__ __align__(16) float4 smem4[];
+  constexpr int q = Q, qq = Q * Q;
+  constexpr int L4 = E / 4;
+  constexpr int log2L4 = E == 32 ? 3 : 2;
+  static_assert(E == 16 || E == 32, "slab width");
+  const int NT = blockDim.x;
+  const int IPP = NT >> log2L4;
+  const int tid = threadIdx.x;
+  const int l = tid & (L4 - 1), it0 = tid >> log2L4;
+  const int64_t bh = blockIdx.y;
+  const int64_t e0 = (int64_t)blockIdx.x * E;
+  float4* Fs = smem4;
+  const float4* src = reinterpret_cast<const float4*>(in + bh * P * state_elems + e0);
+  const int row4 = (int)(state_elems / 4);
+  for (int idx = tid; idx < P * L4; idx += NT) cp_async16(Fs + idx, src + (int64_t)(idx >> log2L4) * row4 + (idx & (L4 - 1)));
+  cp_async_wait_all();
+  __syncthreads();
+  float4* dst4 = reinterpret_cast<float4*>(out + bh * Bn * state_elems + e0);
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+  // directions with a leading zero work on G2[x2, x3] = Σ_{x1} F[x1, x2, x3]
+  float4* G2 = Fs + P * L4;
+  for (int item = it0; item < qq; item += IPP) {
+    float4 acc = zero;
+    const float4* p = Fs + item * q * L4 + l;
+#pragma unroll
+    for (int x1 = 0; x1 < q; ++x1) acc = add4(acc, p[x1 * L4]);
+    G2[item * L4 + l] = acc;
+  }
+  __syncthreads();
+  for (int item = it0; item < qq; item += IPP) {  // a = (0, 1, a3)
+    const int a3 = item / q, b = item - a3 * q;
+    float4 acc = zero;
+    int x2 = b;
+#pragma unroll
+    for (int x3 = 0; x3 < q; ++x3) {
+      acc = add4(acc, G2[(x2 + q * x3) * L4 + l]);
+      x2 -= a3;
+      if (x2 < 0) x2 += q;
+    }
+    dst4[(int64_t)(qq * q + item) * row4 + l] = acc;
+  }
+  for (int b = it0; b < q; b += IPP) {  // a = (0, 0, 1)
+    float4 acc = zero;
+#pragma unroll
+    for (int x2 = 0; x2 < q; ++x2) acc = add4(acc, G2[(x2 + q * b) * L4 + l]);
+    dst4[(int64_t)((qq + q) * q + b) * row4 + l] = acc;
+  }
+  // a = (1, a2, a3), stage 1: thread (x2, e) transforms the image F[., x2, .] in place
+  float* Ff = reinterpret_cast<float*>(Fs);
+  const int e = tid & (E - 1), it = tid >> (log2L4 + 2);
+  if (it < q) radon_inplace<Q, E>(Ff + (q * it) * E + e, 1, qq);  // image [x3][x1]; W_{a3}[u, x2] over F[u, x2, a3]
+  __syncthreads();
+  // stage 2: thread (a3, e) transforms the image W_{a3}[., .]:  U_{(1,a2,a3), b} = Σ_{x2} W_{a3}[b - a2 x2, x2];
+  // slot b + q a2 + q^2 a3 is row h = (a2 + q a3) q + b of U
+  if (it < q) radon_inplace<Q, E>(Ff + (qq * it) * E + e, 1, q);  // image [x2][u]
+  __syncthreads();
+  for (int idx = tid; idx < P * L4; idx += NT)  // rows 0 .. q^3-1 of U, 16-byte stores
+    dst4[(int64_t)(idx >> log2L4) * row4 + (idx & (L4 - 1))] = Fs[idx];
+}
+
 // Transpose for D = 2:  F̄[x1, x2] = Σ_{a2} Ū[(1,a2), x1 + a2 x2] + Ū[(0,1), x2]
 __global__ void __launch_bounds__(1024, 1) tabulate_staged_t2_kernel(const float* __restrict__ in, float* __restrict__ out,
                                                                  int q, int64_t P, int64_t Bn, int64_t state_elems,
@@ -371,10 +480,11 @@ cudaError_t smat_launch_state_read(const void* X, int bf16, const float* state, 
 }
 
 // Shared-memory floats per slab entry the staged kernels need.
+static bool radon3_q(int q) { return q == 5 || q == 7 || q == 11 || q == 13; }
 static int64_t staged_rows(const SmatGeo& geo, int transpose) {
   const int64_t q = geo.q;
   if (geo.D == 2) return transpose ? geo.B : geo.P;
-  if (geo.D == 3 && !transpose) return geo.P + 3 * q * q;
+  if (geo.D == 3 && !transpose) return radon3_q(geo.q) ? geo.P + q * q : geo.P + 3 * q * q;
   return 0;
 }
 
@@ -402,6 +512,18 @@ cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatG
   int nt = (int)(((units + passes - 1) / passes + 31) / 32 * 32);
   if (nt < 128) nt = 128;
   cudaError_t err;
+  if (geo.D == 3 && !transpose && radon3_q(geo.q)) {
+    const int nr = (int)(((int64_t)geo.q * E + 31) / 32 * 32);   // one thread per (image, entry)
+#define SMAT_RADON3(QV, EV)                                                                                \
+  if (geo.q == QV && E == EV) {                                                                            \
+    if ((err = set_smem(tabulate_radon3_kernel<QV, EV>, smem)) != cudaSuccess) return err;                 \
+    tabulate_radon3_kernel<QV, EV><<<grid, nr, smem, st>>>(in, out, (int)geo.P, (int)geo.B, state_elems);  \
+    return cudaGetLastError();                                                                             \
+  }
+    SMAT_RADON3(5, 32) SMAT_RADON3(7, 32) SMAT_RADON3(11, 16) SMAT_RADON3(13, 16)
+#undef SMAT_RADON3
+    return cudaErrorInvalidConfiguration;
+  }
   if (geo.D == 2 && transpose) {
     if ((err = set_smem(tabulate_staged_t2_kernel, smem)) != cudaSuccess) return err;
     tabulate_staged_t2_kernel<<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
