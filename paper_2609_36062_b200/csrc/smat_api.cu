@@ -166,7 +166,8 @@ void state_read(Ctx& cx, const char* name, int mode, const void* x, const float*
   const int kdim = transposed ? pl->p : pl->r, odim = transposed ? pl->r : pl->p;
   if (mode != SMAT_GM_CHUNK && !out_final) {  // a handful of tokens per state: stream the state once
     SMAT_TRY(cx, name, smat_launch_state_read(x, bf, state, transposed, acc_in, acc_out, group(pl, mode), pl->T, G,
-                                              pl->bh, pl->r, pl->p, cx.st));
+                                              pl->bh, pl->r, pl->p, reinterpret_cast<int*>(cx.ws + pl->off_status),
+                                              cx.st));
     return;
   }
   SmatGemmArgs g{};

@@ -80,7 +80,7 @@ cudaError_t smat_launch_pool(const void* A, const void* Bm, int bf16, float* sta
 // Routed read of per-group states: acc_out[t] = acc_in[t] + x_t · state[g(t)] for the tokens of every group.
 cudaError_t smat_launch_state_read(const void* X, int bf16, const float* state, int transposed, const float* acc_in,
                                    float* acc_out, const SmatGroupSpec& grp, int64_t Tlen, int64_t groups, int bh,
-                                   int r, int p, cudaStream_t st);
+                                   int r, int p, int* status, cudaStream_t st);
 
 // Staged exact tabulation (same sums as Algorithm 2, one coordinate at a time). Slab = 0: not available.
 int smat_tabulate_staged_slab(const SmatGeo& geo, int64_t state_elems, int transpose);

@@ -1,15 +1,11 @@
-// Long-range branch on the plain ALUs and HBM: pooling of outer products into per-group states, the
-// tabulation U = C F (staged exact sums for d = 3, 4) and its transpose, and the routed reads of
-// per-group states by the few tokens that share them.  None of these is a dense contraction worth a
-// tensor-core tile: every state is touched by a handful of tokens, so they are shaped for HBM streaming.
+// Long-range branch, tabulation U = C F (Algorithm 2) as staged exact sums for d = 3, 4, and its transpose.
+// The sums run on the plain fp32 ALUs: the incidence matrix is sparse (density 1/q) and every state entry is
+// an independent copy of the same integer-indexed map, so this is not a dense contraction.
 #include <cuda_bf16.h>
 
 #include "smat_internal.h"
 
 namespace {
-
-__device__ __forceinline__ float to_float(float v) { return v; }
-__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 
 // two packed fp32x2 additions (one instruction per pair on sm_100)
 __device__ __forceinline__ float4 add4(const float4 a, const float4 b) {
@@ -24,140 +20,6 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
 }
 __device__ __forceinline__ void cp_async_wait_all() {
   asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
-}
-__device__ __forceinline__ float4 fma4(float s, const float4 b, float4 a) {
-  a.x = fmaf(s, b.x, a.x); a.y = fmaf(s, b.y, a.y); a.z = fmaf(s, b.z, a.z); a.w = fmaf(s, b.w, a.w);
-  return a;
-}
-
-// ---- pooling: state[g] = Σ_{tokens of g} a_tᵀ b_t ------------------------------------------------------------
-// One CTA per (group, head).  Tokens are staged 32 at a time; every thread owns one float4 column
-// strip of the state and NS rows of it, so the 64 KB state is written once with 512-byte rows.
-template <int R, int PD, typename T>
-__global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ A, const T* __restrict__ Bm,
-                                                   float* __restrict__ state, SmatGroupSpec grp, int64_t Tlen,
-                                                   int64_t groups) {
-  constexpr int TK = 32;
-  constexpr int NJ4 = PD / 4;
-  constexpr int NG = 256 / NJ4;
-  constexpr int NS = R / NG;
-  __shared__ __align__(16) float As[TK][R];
-  __shared__ __align__(16) float Bs[TK][PD];
-  const int64_t g = blockIdx.x, bh = blockIdx.y;
-  int64_t t0, ts, cnt;
-  smat_group_tokens(grp, g, &t0, &ts, &cnt);
-  const int tid = threadIdx.x;
-  const int j4 = tid % NJ4, ig = tid / NJ4;
-  float4 acc[NS];
-#pragma unroll
-  for (int s = 0; s < NS; ++s) acc[s] = make_float4(0.f, 0.f, 0.f, 0.f);
-  const T* Ab = A + bh * Tlen * R;
-  const T* Bb = Bm + bh * Tlen * PD;
-  for (int64_t k0 = 0; k0 < cnt; k0 += TK) {
-    const int kn = (int)((cnt - k0) < TK ? (cnt - k0) : TK);
-    for (int idx = tid; idx < kn * R; idx += 256) {
-      const int k = idx / R, i = idx % R;
-      As[k][i] = to_float(Ab[(t0 + (k0 + k) * ts) * R + i]);
-    }
-    for (int idx = tid; idx < kn * PD; idx += 256) {
-      const int k = idx / PD, j = idx % PD;
-      Bs[k][j] = to_float(Bb[(t0 + (k0 + k) * ts) * PD + j]);
-    }
-    __syncthreads();
-    for (int k = 0; k < kn; ++k) {
-      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[k][j4 * 4]);
-#pragma unroll
-      for (int s = 0; s < NS; ++s) acc[s] = fma4(As[k][ig + s * NG], b4, acc[s]);
-    }
-    __syncthreads();
-  }
-  float* out = state + (bh * groups + g) * (int64_t)(R * PD);
-#pragma unroll
-  for (int s = 0; s < NS; ++s) *reinterpret_cast<float4*>(out + (int64_t)(ig + s * NG) * PD + j4 * 4) = acc[s];
-}
-
-// ---- routed read: out[t] = acc_in[t] + x_t · state[g(t)] ------------------------------------------------------
-// One CTA per (group, head) streams the 64 KB state once for up to KT tokens at a time.
-// TRANS = 0: x_t has R entries and contracts the first state index (output PD wide).
-// TRANS = 1: x_t has PD entries and contracts the second state index (output R wide).
-template <int R, int PD, int TRANS, typename T>
-__global__ void __launch_bounds__(256) state_read_kernel(const T* __restrict__ X, const float* __restrict__ state,
-                                                         const float* acc_in, float* acc_out, SmatGroupSpec grp,
-                                                         int64_t Tlen, int64_t groups) {
-  constexpr int KT = 8;
-  constexpr int NJ4 = PD / 4;
-  constexpr int NG = 256 / NJ4;        // row groups (one or more per warp)
-  constexpr int RPG = R / NG;          // state rows per group
-  constexpr int XD = TRANS ? PD : R;   // length of x_t
-  constexpr int OD = TRANS ? R : PD;   // length of the output row
-  __shared__ __align__(16) float Xs[KT][XD];
-  __shared__ __align__(16) float red[TRANS ? 1 : NG][KT][TRANS ? R : PD];
-  const int64_t g = blockIdx.x, bh = blockIdx.y;
-  int64_t t0, ts, cnt;
-  smat_group_tokens(grp, g, &t0, &ts, &cnt);
-  if (cnt == 0) return;
-  const int tid = threadIdx.x;
-  const int j4 = tid % NJ4, ig = tid / NJ4;
-  const float4* S4 = reinterpret_cast<const float4*>(state + (bh * groups + g) * (int64_t)(R * PD));
-  const T* Xb = X + bh * Tlen * XD;
-  for (int64_t k0 = 0; k0 < cnt; k0 += KT) {
-    const int kn = (int)((cnt - k0) < KT ? (cnt - k0) : KT);
-    for (int idx = tid; idx < KT * XD; idx += 256) {
-      const int k = idx / XD, i = idx % XD;
-      Xs[k][i] = k < kn ? to_float(Xb[(t0 + (k0 + k) * ts) * XD + i]) : 0.f;
-    }
-    __syncthreads();
-    if (!TRANS) {
-      float4 acc[KT];
-#pragma unroll
-      for (int k = 0; k < KT; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-      for (int s = 0; s < RPG; ++s) {
-        const int i = ig * RPG + s;
-        const float4 u = __ldg(S4 + i * NJ4 + j4);
-#pragma unroll
-        for (int k = 0; k < KT; ++k) acc[k] = fma4(Xs[k][i], u, acc[k]);
-      }
-#pragma unroll
-      for (int k = 0; k < KT; ++k) *reinterpret_cast<float4*>(&red[ig][k][j4 * 4]) = acc[k];
-      __syncthreads();
-      for (int idx = tid; idx < kn * PD; idx += 256) {
-        const int k = idx / PD, j = idx % PD;
-        float v = 0.f;
-#pragma unroll
-        for (int w = 0; w < NG; ++w) v += red[w][k][j];
-        const int64_t off = (bh * Tlen + t0 + (k0 + k) * ts) * OD + j;
-        acc_out[off] = v + (acc_in ? acc_in[off] : 0.f);
-      }
-    } else {
-      // every lane holds 4 columns of row i; the row sum is a reduction across the NJ4 lanes of the group
-#pragma unroll 2
-      for (int s = 0; s < RPG; ++s) {
-        const int i = ig * RPG + s;
-        const float4 u = __ldg(S4 + i * NJ4 + j4);
-        float part[KT];
-#pragma unroll
-        for (int k = 0; k < KT; ++k) {
-          const float4 x4 = *reinterpret_cast<const float4*>(&Xs[k][j4 * 4]);
-          part[k] = u.x * x4.x + u.y * x4.y + u.z * x4.z + u.w * x4.w;
-        }
-#pragma unroll
-        for (int off = NJ4 / 2; off > 0; off >>= 1)
-#pragma unroll
-          for (int k = 0; k < KT; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], off);
-        if (j4 == 0)
-#pragma unroll
-          for (int k = 0; k < KT; ++k) red[0][k][i] = part[k];
-      }
-      __syncthreads();
-      for (int idx = tid; idx < kn * R; idx += 256) {
-        const int k = idx / R, i = idx % R;
-        const int64_t off = (bh * Tlen + t0 + (k0 + k) * ts) * OD + i;
-        acc_out[off] = red[0][k][i] + (acc_in ? acc_in[off] : 0.f);
-      }
-    }
-    __syncthreads();
-  }
 }
 
 // ---- staged exact tabulation -------------------------------------------------------------------------------------
@@ -433,52 +295,6 @@ cudaError_t set_smem(K kernel, size_t bytes) {
 }  // namespace
 
 // ---- launchers ------------------------------------------------------------------------------------------------------
-template <typename T>
-static cudaError_t launch_pool_t(const void* A, const void* Bm, float* state, const SmatGroupSpec& grp, int64_t Tlen,
-                                 int64_t groups, int bh, int r, int p, cudaStream_t st) {
-  dim3 grid((unsigned)groups, (unsigned)bh);
-  const T* a = static_cast<const T*>(A);
-  const T* b = static_cast<const T*>(Bm);
-  if (r == 128 && p == 128) pool_kernel<128, 128, T><<<grid, 256, 0, st>>>(a, b, state, grp, Tlen, groups);
-  else if (r == 64 && p == 64) pool_kernel<64, 64, T><<<grid, 256, 0, st>>>(a, b, state, grp, Tlen, groups);
-  else if (r == 64 && p == 128) pool_kernel<64, 128, T><<<grid, 256, 0, st>>>(a, b, state, grp, Tlen, groups);
-  else pool_kernel<128, 64, T><<<grid, 256, 0, st>>>(a, b, state, grp, Tlen, groups);
-  return cudaGetLastError();
-}
-
-cudaError_t smat_launch_pool(const void* A, const void* Bm, int bf16, float* state, const SmatGroupSpec& grp,
-                             int64_t Tlen, int64_t groups, int bh, int r, int p, cudaStream_t st) {
-  return bf16 ? launch_pool_t<__nv_bfloat16>(A, Bm, state, grp, Tlen, groups, bh, r, p, st)
-              : launch_pool_t<float>(A, Bm, state, grp, Tlen, groups, bh, r, p, st);
-}
-
-template <int TRANS, typename T>
-static cudaError_t launch_read_t(const void* X, const float* state, const float* acc_in, float* acc_out,
-                                 const SmatGroupSpec& grp, int64_t Tlen, int64_t groups, int bh, int r, int p,
-                                 cudaStream_t st) {
-  dim3 grid((unsigned)groups, (unsigned)bh);
-  const T* x = static_cast<const T*>(X);
-  if (r == 128 && p == 128)
-    state_read_kernel<128, 128, TRANS, T><<<grid, 256, 0, st>>>(x, state, acc_in, acc_out, grp, Tlen, groups);
-  else if (r == 64 && p == 64)
-    state_read_kernel<64, 64, TRANS, T><<<grid, 256, 0, st>>>(x, state, acc_in, acc_out, grp, Tlen, groups);
-  else if (r == 64 && p == 128)
-    state_read_kernel<64, 128, TRANS, T><<<grid, 256, 0, st>>>(x, state, acc_in, acc_out, grp, Tlen, groups);
-  else
-    state_read_kernel<128, 64, TRANS, T><<<grid, 256, 0, st>>>(x, state, acc_in, acc_out, grp, Tlen, groups);
-  return cudaGetLastError();
-}
-
-cudaError_t smat_launch_state_read(const void* X, int bf16, const float* state, int transposed, const float* acc_in,
-                                   float* acc_out, const SmatGroupSpec& grp, int64_t Tlen, int64_t groups, int bh,
-                                   int r, int p, cudaStream_t st) {
-  if (transposed)
-    return bf16 ? launch_read_t<1, __nv_bfloat16>(X, state, acc_in, acc_out, grp, Tlen, groups, bh, r, p, st)
-                : launch_read_t<1, float>(X, state, acc_in, acc_out, grp, Tlen, groups, bh, r, p, st);
-  return bf16 ? launch_read_t<0, __nv_bfloat16>(X, state, acc_in, acc_out, grp, Tlen, groups, bh, r, p, st)
-              : launch_read_t<0, float>(X, state, acc_in, acc_out, grp, Tlen, groups, bh, r, p, st);
-}
-
 // Shared-memory floats per slab entry the staged kernels need.
 static bool radon3_q(int q) { return q == 5 || q == 7 || q == 11 || q == 13; }
 static int64_t staged_rows(const SmatGeo& geo, int transpose) {
