@@ -367,9 +367,12 @@ def run_native(args):
             k = 5
             s = r.time_steps(r.step, k, 3) / k
             rep = path_report(ws_, gg, s, peaks)
+            st_ = r.stage_profile(3)
             sweep.append({"workload": name, "value": ws_.tokens / s, "unit": "tokens/s", "ms_per_step": 1e3 * s,
                           "frac_2term": rep["frac_2term"], "frac_3term": rep["frac_3term"],
-                          "cached_subset_states_B": gg.B, "profile_states_P": gg.P})
+                          "roofline_ms_2term": rep["roofline_ms_2term"],
+                          "cached_subset_states_B": gg.B, "profile_states_P": gg.P,
+                          "kernels_ms": {n: round(t_, 4) for n, t_ in st_}})
             del r
             torch.cuda.empty_cache()
         line["sweep"] = sweep
