@@ -35,6 +35,10 @@ from paper_2609_36062_b200 import roofline, synth  # noqa: E402
 DEFAULT_WORKLOAD = "t16k_d4"
 SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
 METRIC = "SMat prefill tokens/s"
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu
+# capture summarised in profiles/forward_kernels_t16k_d4_h2.md: taken on the 2-head copy of the workload and
+# scaled by heads (every head owns its own tables, so traffic is proportional to the head count).
+NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate"): (174.49e6 + 144.24e6) * 32 / 2}
 
 
 def parse_args():
@@ -293,7 +297,9 @@ def dominant_kernel_report(w, geo, stages, peaks):
     else:
         achieved, peak, unit = work.flops / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
     return {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-            "frac": achieved / peak if peak else None, "traffic": None, "ms": ms, "share": ms / total if total else None,
+            "frac": achieved / peak if peak else None, "traffic": NCU_TRAFFIC_BYTES.get((w.name, base)),
+            "algorithmic_bytes": work.bytes, "algorithmic_adds": work.adds,
+            "ms": ms, "share": ms / total if total else None,
             "peak_source": peaks["source"] + (" (fp32 add peak nominal: 148 SM x 128 lanes x max clock)" if bound == "alu" else ""),
             "kernels_ms": {n: round(t_, 4) for n, t_ in stages}}
 
