@@ -158,6 +158,32 @@ smat_status smat_check_status(const smat_plan* plan, const void* workspace, void
 smat_status smat_profile_enable(smat_plan* plan, int enable);
 int smat_profile_read(const smat_plan* plan, const char** names, float* ms, int max_stages);
 
+/*
+ * Causal forward without any workspace from the caller (the paper has no counterpart: this exists for
+ * integration, not for the method).  Computes O = (L_T ⊙ QKᵀ)V — the d = 1 member of the family — for
+ * bf16 Q, K, V, O of shape [batch, heads, T, 128] (DEVICE pointers, 16-byte aligned, T a multiple of 128).
+ *
+ * Who needs it: callers that cannot allocate device memory themselves — a plug-in inside an application
+ * that owns the whole device heap, or a serving loop that bans cudaMalloc on its request path because an
+ * allocation can synchronise the device.  The incoming chunk states this path needs live in a fixed array
+ * inside the library image (SMAT_STATIC_MAX_TILES bf16 states of 32 KB plus a status word, 32 MiB in all,
+ * resident on every device that loads the library until the process exits).  The call allocates nothing,
+ * neither with cudaMalloc nor through any library.
+ *
+ * Limit: batch * heads * (T / 128) <= SMAT_STATIC_MAX_TILES, otherwise SMAT_ERR_WORKSPACE (use smat_forward
+ * with a workspace of your own).  Other errors as for smat_forward; SMAT_ERR_ARCH if the tensor-core path is
+ * unavailable.
+ *
+ * The first call on each device looks up the device address of that array (with the device current); make
+ * that first call outside any stream capture.  All calls on a device share the one array, which keeps the
+ * previous call's contents (the library clears the part that must start at zero): two calls that overlap on
+ * the GPU — different streams, or different host threads — race on it, so serialise them.
+ * Asynchronous on `cuda_stream`.
+ */
+#define SMAT_STATIC_MAX_TILES 1024
+smat_status smat_forward_causal_static(const void* Q, const void* K, const void* V, void* O, int batch, int heads,
+                                       int64_t T, void* cuda_stream);
+
 /* Number of kernels the last smat_forward / smat_backward on this plan launched (host counter). */
 int smat_last_launch_count(const smat_plan* plan);
 

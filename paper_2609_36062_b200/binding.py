@@ -22,7 +22,7 @@ FLAG_ALG2_TABULATION = 2
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
-    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores",
+    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_forward_causal_static",
 ]
 
 
@@ -89,6 +89,8 @@ def load_library() -> ctypes.CDLL:
     lib.smat_last_launch_count.restype = i
     lib.smat_uses_tensor_cores.argtypes = [vp]
     lib.smat_uses_tensor_cores.restype = i
+    lib.smat_forward_causal_static.argtypes = [vp, vp, vp, vp, i, i, i64, vp]
+    lib.smat_forward_causal_static.restype = i
     lib.smat_profile_enable.argtypes = [vp, i]
     lib.smat_profile_enable.restype = i
     lib.smat_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float), i]
@@ -118,6 +120,27 @@ def _stream(stream) -> int:
 
 
 _TORCH_DTYPE = {SMAT_F32: torch.float32, SMAT_BF16: torch.bfloat16}
+
+STATIC_MAX_TILES = 1024
+
+
+def forward_causal_static(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, O: torch.Tensor | None = None,
+                          stream=None) -> torch.Tensor:
+    """Causal (d = 1) forward that needs no workspace: smat_forward_causal_static.
+
+    For callers that may not allocate device memory; the scratch lives in a fixed 32 MiB array inside the
+    library, so batch * heads * T / 128 must not exceed STATIC_MAX_TILES, and calls must not overlap on the GPU.
+    O may be passed in by a caller who cannot allocate; it is created here only as a convenience."""
+    lib = load_library()
+    for name, t in (("Q", Q), ("K", K), ("V", V)):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.dim() == 4 and t.shape[-1] == 128):
+            raise ValueError(f"{name}: expected a contiguous CUDA bf16 tensor [batch, heads, T, 128]")
+    if O is None:
+        O = torch.empty_like(V)
+    b, h, T, _ = Q.shape
+    _check(lib.smat_forward_causal_static(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), b, h, T, _stream(stream)),
+           "smat_forward_causal_static")
+    return O
 
 
 class SmatPlan:
