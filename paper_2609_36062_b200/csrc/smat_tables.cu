@@ -150,47 +150,49 @@ __global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* _
 // shared-memory read per addition) and writes the q^2 results back over the image it read.  The second stage is
 // the same transform of the image W_{a3}[., .] for a fixed a3; its results again replace the image, which leaves
 // rows 0 .. q^3-1 of U in the slab, in order, ready for a coalesced copy out.
+// Line sums of slope A: out[v] = Σ_y img[y][(v - A y) mod Q], stored with stride `os`.
 template <int Q, int A>
 struct RadonSlope {
-  // line sums of slope A: out[u] = Σ_y img[y][(u - A y) mod Q], stored with stride `os`
   static __device__ __forceinline__ void run(const float (&img)[Q][Q], float* out, int os) {
+    float p[Q];  // the Q sums advance together, one image row at a time: Q independent additions per step
 #pragma unroll
-    for (int u = 0; u < Q; ++u) {
-      float sum = img[0][u];
+    for (int v = 0; v < Q; ++v) p[v] = img[0][v];
 #pragma unroll
-      for (int y = 1; y < Q; ++y) sum += img[y][((u - A * y) % Q + Q) % Q];
-      out[u * os] = sum;
-    }
+    for (int y = 1; y < Q; ++y)
+#pragma unroll
+      for (int v = 0; v < Q; ++v) p[v] += img[y][((v - A * y) % Q + Q) % Q];
+#pragma unroll
+    for (int v = 0; v < Q; ++v) out[v * os] = p[v];
   }
 };
-template <int Q>
-__device__ __forceinline__ void radon_dispatch(int a, const float (&img)[Q][Q], float* out, int os) {
-#define SMAT_SLOPE(k) \
-  case k:             \
-    if constexpr (k < Q) RadonSlope<Q, (k < Q ? k : 0)>::run(img, out, os); \
-    break;
-  switch (a) {
-    SMAT_SLOPE(0) SMAT_SLOPE(1) SMAT_SLOPE(2) SMAT_SLOPE(3) SMAT_SLOPE(4) SMAT_SLOPE(5) SMAT_SLOPE(6)
-    SMAT_SLOPE(7) SMAT_SLOPE(8) SMAT_SLOPE(9) SMAT_SLOPE(10) SMAT_SLOPE(11) SMAT_SLOPE(12)
-    default: break;
+
+// All Q slopes in turn.  The empty asm between two slopes keeps the compiler from interleaving their sums, which
+// would multiply the number of live partial sums (and spill the image).
+template <int Q, int A = 0>
+__device__ __forceinline__ void radon_all_slopes(const float (&img)[Q][Q], float* base, int slope_stride, int os) {
+  if constexpr (A < Q) {
+    RadonSlope<Q, A>::run(img, base + A * slope_stride, os);
+    asm volatile("" ::: "memory");
+    radon_all_slopes<Q, A + 1>(img, base, slope_stride, os);
   }
-#undef SMAT_SLOPE
 }
 
-// One in-place transform: image[y][x] at base[(x * sx + y * sy) * E], slope a results to base[(x * sx + a * sy) * E].
-template <int Q, int E>
-__device__ __noinline__ void radon_inplace(float* base, int sx, int sy) {
+// One in-place transform: image[y][x] at base[(x + y * SY) * E], slope a results to base[(x + a * SY) * E].
+// Kept out of line so that the two transforms of the kernel get their registers allocated independently.
+template <int Q, int E, int SY>
+__device__ __noinline__ void radon_inplace(float* base) {
   float img[Q][Q];
 #pragma unroll
   for (int y = 0; y < Q; ++y)
 #pragma unroll
-    for (int x = 0; x < Q; ++x) img[y][x] = base[(x * sx + y * sy) * E];
-#pragma unroll 1
-  for (int a = 0; a < Q; ++a) radon_dispatch<Q>(a, img, base + a * sy * E, sx * E);
+    for (int x = 0; x < Q; ++x) img[y][x] = base[(x + y * SY) * E];
+  radon_all_slopes<Q>(img, base, SY * E, E);
 }
 
+// Register budget: 168 keeps two 192-thread CTAs per SM (q <= 11); the 7-warp CTAs of q = 13 may take 224.
+// Larger fields do not fit a q x q image in the registers of one thread and use tabulate_staged_kernel.
 template <int Q, int E>
-__global__ void __launch_bounds__((Q * E + 31) / 32 * 32, Q <= 11 ? 2 : 1)
+__global__ void __maxnreg__(Q <= 11 ? 168 : 224)
     tabulate_radon3_kernel(const float* __restrict__ in, float* __restrict__ out, int P, int Bn, int64_t state_elems) {
   extern __shared__ __align__(16) float4 smem4[];
   constexpr int q = Q, qq = Q * Q;
@@ -242,11 +244,11 @@ __global__ void __launch_bounds__((Q * E + 31) / 32 * 32, Q <= 11 ? 2 : 1)
   // a = (1, a2, a3), stage 1: thread (x2, e) transforms the image F[., x2, .] in place
   float* Ff = reinterpret_cast<float*>(Fs);
   const int e = tid & (E - 1), it = tid >> (log2L4 + 2);
-  if (it < q) radon_inplace<Q, E>(Ff + (q * it) * E + e, 1, qq);  // image [x3][x1]; W_{a3}[u, x2] over F[u, x2, a3]
+  if (it < q) radon_inplace<Q, E, Q * Q>(Ff + (q * it) * E + e);  // image [x3][x1]; W_{a3}[u, x2] over F[u, x2, a3]
   __syncthreads();
   // stage 2: thread (a3, e) transforms the image W_{a3}[., .]:  U_{(1,a2,a3), b} = Σ_{x2} W_{a3}[b - a2 x2, x2];
   // slot b + q a2 + q^2 a3 is row h = (a2 + q a3) q + b of U
-  if (it < q) radon_inplace<Q, E>(Ff + (qq * it) * E + e, 1, q);  // image [x2][u]
+  if (it < q) radon_inplace<Q, E, Q>(Ff + (qq * it) * E + e);  // image [x2][u]
   __syncthreads();
   for (int idx = tid; idx < P * L4; idx += NT)  // rows 0 .. q^3-1 of U, 16-byte stores
     dst4[(int64_t)(idx >> log2L4) * row4 + (idx & (L4 - 1))] = Fs[idx];
@@ -296,7 +298,9 @@ cudaError_t set_smem(K kernel, size_t bytes) {
 
 // ---- launchers ------------------------------------------------------------------------------------------------------
 // Shared-memory floats per slab entry the staged kernels need.
-static bool radon3_q(int q) { return q == 5 || q == 7 || q == 11 || q == 13; }
+// slab width of the register-resident form for the field sizes it is compiled for (0: not available)
+static int radon3_slab(int q) { return q == 5 || q == 7 ? 32 : (q == 11 || q == 13 ? 16 : 0); }
+static bool radon3_q(int q) { return radon3_slab(q) != 0; }
 static int64_t staged_rows(const SmatGeo& geo, int transpose) {
   const int64_t q = geo.q;
   if (geo.D == 2) return transpose ? geo.B : geo.P;
@@ -307,6 +311,7 @@ static int64_t staged_rows(const SmatGeo& geo, int transpose) {
 int smat_tabulate_staged_slab(const SmatGeo& geo, int64_t state_elems, int transpose) {
   const int64_t rows = staged_rows(geo, transpose);
   if (rows == 0) return 0;
+  if (geo.D == 3 && !transpose && radon3_q(geo.q) && state_elems % 32 == 0) return radon3_slab(geo.q);
   // prefer two resident CTAs per SM (about 110 KB each) with at least 16 entries, else the largest slab that fits
   const int64_t two = 110 * 1024, one = 220 * 1024;
   for (int E = 32; E >= 16; E >>= 1)
@@ -329,9 +334,9 @@ cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatG
   if (nt < 128) nt = 128;
   cudaError_t err;
   if (geo.D == 3 && !transpose && radon3_q(geo.q)) {
-    const int nr = (int)(((int64_t)geo.q * E + 31) / 32 * 32);   // one thread per (image, entry)
 #define SMAT_RADON3(QV, EV)                                                                                \
   if (geo.q == QV && E == EV) {                                                                            \
+    const int nr = (QV * EV + 31) / 32 * 32; /* one thread per (image, entry) */                           \
     if ((err = set_smem(tabulate_radon3_kernel<QV, EV>, smem)) != cudaSuccess) return err;                 \
     tabulate_radon3_kernel<QV, EV><<<grid, nr, smem, st>>>(in, out, (int)geo.P, (int)geo.B, state_elems);  \
     return cudaGetLastError();                                                                             \
