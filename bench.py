@@ -38,7 +38,7 @@ METRIC = "SMat prefill tokens/s"
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu
 # capture summarised in profiles/forward_kernels_t16k_d4_h2.md: taken on the 2-head copy of the workload and
 # scaled by heads (every head owns its own tables, so traffic is proportional to the head count).
-NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate"): (174.49e6 + 144.24e6) * 32 / 2}
+NCU_TRAFFIC_BYTES = {}
 
 
 def parse_args():
@@ -264,15 +264,22 @@ class Runner:
         return [(n, acc[n] / steps) for n in order]
 
 
-def path_report(w, geo, seconds_per_step, peaks):
+def path_report(w, geo, seconds_per_step, peaks, u_bytes=4):
+    """Fractions against the path roofline.  The bytes are those of the design that ran: where the type table is
+    kept as bf16 (u_bytes = 2) its round trip is charged at 2 bytes per entry, and the fraction against the
+    roofline with fp32 tables is given beside it."""
     e = 4 if w.dtype == "f32" else 2
-    work = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo)
-    if w.backward:
-        work = work + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo)
-    work = work.scaled(w.bh)
+    def total(ub):
+        wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub)
+        if w.backward:
+            wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo)
+        return wk.scaled(w.bh)
+    work = total(u_bytes)
     t = roofline.roofline_times(work, peaks)
+    t32 = roofline.roofline_times(total(4), peaks)
     return {
         "frac_2term": t["t_2term"] / seconds_per_step, "frac_3term": t["t_3term"] / seconds_per_step,
+        "frac_2term_fp32_tables": t32["t_2term"] / seconds_per_step, "type_table_bytes_per_entry": u_bytes,
         "roofline_ms_2term": 1e3 * t["t_2term"], "roofline_ms_3term": 1e3 * t["t_3term"],
         "t_tensor_ms": 1e3 * t["t_tensor"], "t_alu_ms": 1e3 * t["t_alu"], "t_hbm_ms": 1e3 * t["t_hbm"],
         "algorithmic": {"tensor_flop": work.flops, "alu_adds": work.adds, "hbm_bytes": work.bytes},
@@ -280,12 +287,12 @@ def path_report(w, geo, seconds_per_step, peaks):
     }
 
 
-def dominant_kernel_report(w, geo, stages, peaks):
+def dominant_kernel_report(w, geo, stages, peaks, u_bytes=4):
     e = 4 if w.dtype == "f32" else 2
     total = sum(t for _, t in stages)
     name, ms = max(stages, key=lambda s: s[1])
     base = name.split(":")[-1]
-    work = roofline.stage_work(base, w.T, w.chunk, w.d_k, w.d_v, e, geo).scaled(w.bh)
+    work = roofline.stage_work(base, w.T, w.chunk, w.d_k, w.d_v, e, geo, u_bytes).scaled(w.bh)
     t = roofline.roofline_times(work, peaks, sustained=True)
     bounds = {"hbm": t["t_hbm"], "alu": t["t_alu"], "tensor": t["t_tensor"]}
     bound = max(bounds, key=bounds.get)
@@ -345,6 +352,7 @@ def run_native(args):
 
     line = None
     if rank == 0:
+        ub = runner.plan.type_table_element_bytes()
         stages = runner.stage_profile(min(steps, 10))
         line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warm,
@@ -355,8 +363,8 @@ def run_native(args):
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": launches * steps,
             "clocks": clocks,
-            "roofline": dominant_kernel_report(w, g, stages, peaks),
-            "path_roofline": path_report(w, g, per_step, peaks),
+            "roofline": dominant_kernel_report(w, g, stages, peaks, ub),
+            "path_roofline": path_report(w, g, per_step, peaks, ub),
             "tables": {"profile_states_P": g.P, "cached_subset_states_B": g.B, "nnzC": g.nnzC, "q": g.q},
         }
     del runner
@@ -372,10 +380,11 @@ def run_native(args):
             gg = r.plan.geometry()
             k = 5
             s = r.time_steps(r.step, k, 3) / k
-            rep = path_report(ws_, gg, s, peaks)
+            rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes())
             st_ = r.stage_profile(3)
             sweep.append({"workload": name, "value": ws_.tokens / s, "unit": "tokens/s", "ms_per_step": 1e3 * s,
                           "frac_2term": rep["frac_2term"], "frac_3term": rep["frac_3term"],
+                          "frac_2term_fp32_tables": rep["frac_2term_fp32_tables"],
                           "roofline_ms_2term": rep["roofline_ms_2term"],
                           "cached_subset_states_B": gg.B, "profile_states_P": gg.P,
                           "kernels_ms": {n: round(t_, 4) for n, t_ in st_}})

@@ -88,6 +88,11 @@ smat_status smat_get_geometry(const smat_plan* plan, smat_geometry* out);
  * boundary and recent length multiples of 128, SMAT_FLAG_SIMT_ONLY not set), 0 when it runs on the fp32 ALUs. */
 int smat_uses_tensor_cores(const smat_plan* plan);
 
+/* Bytes per element of the type table U as smat_forward keeps it: 4 (fp32), or 2 when the plan runs the typed read on
+ * the tensor cores (bf16 inputs, d >= 3): there U is only ever a bf16 MMA operand, so it is rounded once when the
+ * tabulation stores it and the table's HBM traffic halves.  smat_backward always builds fp32 tables. */
+int smat_type_table_element_bytes(const smat_plan* plan);
+
 /* Bytes of workspace smat_forward (for_backward = 0) or smat_backward (for_backward = 1) needs. 0 if plan is NULL. */
 size_t smat_workspace_bytes(const smat_plan* plan, int for_backward);
 

@@ -22,7 +22,7 @@ FLAG_ALG2_TABULATION = 2
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
-    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_forward_causal_static",
+    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
 ]
 
 
@@ -87,6 +87,8 @@ def load_library() -> ctypes.CDLL:
     lib.smat_check_status.restype = i
     lib.smat_last_launch_count.argtypes = [vp]
     lib.smat_last_launch_count.restype = i
+    lib.smat_type_table_element_bytes.argtypes = [vp]
+    lib.smat_type_table_element_bytes.restype = i
     lib.smat_uses_tensor_cores.argtypes = [vp]
     lib.smat_uses_tensor_cores.restype = i
     lib.smat_forward_causal_static.argtypes = [vp, vp, vp, vp, i, i, i64, vp]
@@ -171,6 +173,9 @@ class SmatPlan:
 
     def uses_tensor_cores(self) -> bool:
         return bool(self.lib.smat_uses_tensor_cores(self.handle))
+
+    def type_table_element_bytes(self) -> int:
+        return int(self.lib.smat_type_table_element_bytes(self.handle))
 
     def workspace_bytes(self, for_backward: bool = False) -> int:
         return int(self.lib.smat_workspace_bytes(self.handle, int(for_backward)))

@@ -23,7 +23,9 @@ struct smat_plan {
   size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_fwd_end;
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
   bool tc;             // tensor-core kernels for the causal branch
+  bool u_bf16;         // forward keeps the type table U in bf16 and reads it with the tensor-core typed read
   mutable int launches;
+  mutable bool last_was_forward;  // which call left its tables in the workspace
   // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
   mutable bool profiling;
   mutable cudaEvent_t events[SMAT_MAX_STAGES + 1];
@@ -227,11 +229,11 @@ smat_status check_common(const smat_plan* pl, const void* ws, size_t ws_bytes, i
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
 
 // Step 3 of Algorithm 1 (transpose = 0) or F̄ = Cᵀ Ū (transpose = 1).
-void tabulate(Ctx& cx, const char* name, const float* in, float* out, int transpose) {
+void tabulate(Ctx& cx, const char* name, const float* in, float* out, int transpose, int out_bf16 = 0) {
   const smat_plan* pl = cx.pl;
   if (in == out) return;  // d = 2: hyperplanes are single points, the type table is the profile table
   if (!(pl->flags & SMAT_FLAG_ALG2_TABULATION) && smat_tabulate_staged_slab(pl->geo, pl->rp, transpose) >= 4)
-    SMAT_TRY(cx, name, smat_launch_tabulate_staged(in, out, pl->geo, pl->rp, pl->bh, transpose, cx.st));
+    SMAT_TRY(cx, name, smat_launch_tabulate_staged(in, out, pl->geo, pl->rp, pl->bh, transpose, out_bf16, cx.st));
   else
     SMAT_TRY(cx, name, smat_launch_tabulate_alg2(in, out, pl->geo, pl->rp, pl->bh, transpose, cx.st));
 }
@@ -266,13 +268,16 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->batch = batch; pl->heads = heads; pl->bh = batch * heads;
   pl->r = d_k; pl->p = d_v; pl->T = T; pl->c = chunk; pl->NC = T / chunk;
   pl->dtype = dtype; pl->flags = flags; pl->rp = (int64_t)d_k * d_v; pl->launches = 0;
-  pl->profiling = false; pl->stages = 0;
+  pl->profiling = false; pl->stages = 0; pl->last_was_forward = true;
   smat_status s = build_geometry(&pl->geo, T, chunk, d, q_override);
   if (s != SMAT_OK) { delete pl; return s; }
   const SmatGeo& g = pl->geo;
   pl->tc = dtype == SMAT_BF16 && d_k == 128 && d_v == 128 && !(flags & SMAT_FLAG_SIMT_ONLY) && g.n % 128 == 0 &&
            g.m % 128 == 0 && g.n >= 128 && smat_tc_available();
   if (!g.dense_G && (smat_tabulate_alg2_slab(g.B, pl->rp) < 1)) { delete pl; return SMAT_ERR_UNSUPPORTED; }
+  // d >= 3 on the tensor-core path: U is only ever a bf16 MMA operand, so it is stored as bf16 (half the bytes)
+  pl->u_bf16 = pl->tc && g.D >= 2 && !(flags & SMAT_FLAG_ALG2_TABULATION) &&
+               smat_tabulate_staged_slab(g, pl->rp, 0) >= 4;
   const size_t state = (size_t)pl->rp * sizeof(float);
   const int wide = d_k > d_v ? d_k : d_v;
   size_t off = 0;
@@ -338,6 +343,8 @@ smat_status smat_get_geometry(const smat_plan* pl, smat_geometry* out) {
 
 int smat_uses_tensor_cores(const smat_plan* pl) { return pl && pl->tc ? 1 : 0; }
 
+int smat_type_table_element_bytes(const smat_plan* pl) { return pl && pl->u_bf16 ? 2 : 4; }
+
 size_t smat_workspace_bytes(const smat_plan* pl, int for_backward) {
   if (!pl) return 0;
   return for_backward ? pl->off_bwd_end : pl->off_fwd_end;
@@ -351,6 +358,7 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
   if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return SMAT_ERR_ALIGN;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
+  pl->last_was_forward = true;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   if (pl->tc) {
     int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
@@ -358,8 +366,12 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
     const bool lr = !pl->geo.dense_G;
     if (lr) {
       outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));                         // step 2
-      tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0);                         // step 3
-      state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);  // step 4
+      tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);              // step 3
+      if (pl->u_bf16)                                                                        // step 4
+        SMAT_TRY(cx, "read_type_tc", smat_launch_state_read_tc(Q, cx.ws + pl->off_U, ylr, pl->T, pl->geo.n,
+                                                               pl->geo.B, pl->bh, status, cx.st));
+      else
+        state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);
     }
     SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, pl->geo.n,
                                                              lr ? 0 : 1, status, cx.st));   // steps 5-6
@@ -391,6 +403,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
     return SMAT_ERR_ALIGN;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
+  pl->last_was_forward = false;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   const bool lr = !pl->geo.dense_G;
   build_forward_tables(cx, K, V);
@@ -477,8 +490,12 @@ smat_status smat_debug_tables(const smat_plan* pl, const void* workspace, float*
   } else {
     if (F && err == cudaSuccess)
       err = cudaMemcpyAsync(F, ws + pl->off_F, (size_t)pl->bh * pl->geo.P * state, cudaMemcpyDeviceToDevice, st);
-    if (U && err == cudaSuccess)
-      err = cudaMemcpyAsync(U, ws + pl->off_U, (size_t)pl->bh * pl->geo.B * state, cudaMemcpyDeviceToDevice, st);
+    if (U && err == cudaSuccess) {
+      if (pl->u_bf16 && pl->last_was_forward)  // the forward of this plan keeps U in bf16: widen on export
+        err = smat_launch_widen_bf16(ws + pl->off_U, U, (int64_t)pl->bh * pl->geo.B * pl->rp, st);
+      else
+        err = cudaMemcpyAsync(U, ws + pl->off_U, (size_t)pl->bh * pl->geo.B * state, cudaMemcpyDeviceToDevice, st);
+    }
   }
   return err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
 }

@@ -84,8 +84,9 @@ cudaError_t smat_launch_state_read(const void* X, int bf16, const float* state, 
 
 // Staged exact tabulation (same sums as Algorithm 2, one coordinate at a time). Slab = 0: not available.
 int smat_tabulate_staged_slab(const SmatGeo& geo, int64_t state_elems, int transpose);
-cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatGeo& geo, int64_t state_elems, int bh,
-                                        int transpose, cudaStream_t st);
+// out_bf16 = 1 writes the result table as bf16 (same layout, half the bytes) instead of fp32.
+cudaError_t smat_launch_tabulate_staged(const float* in, void* out, const SmatGeo& geo, int64_t state_elems, int bh,
+                                        int transpose, int out_bf16, cudaStream_t st);
 
 // Tensor-core kernels of the causal branch (bf16, d_k = d_v = 128, 128-token tiles; n and T - n multiples of 128).
 bool smat_tc_available();
@@ -97,3 +98,8 @@ cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf
 cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
                                         const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,
                                         cudaStream_t st);
+// Typed read on tensor cores: ylr[t] = q_tᵀ U_type(t) for recent tokens, U kept as bf16 [bh][B][128][128].
+cudaError_t smat_launch_state_read_tc(const void* Q, const void* U_bf16, float* ylr, int64_t T, int64_t n, int64_t B,
+                                      int bh, int* status, cudaStream_t st);
+// bf16 -> fp32 copy of a table (debug export).
+cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st);

@@ -13,6 +13,19 @@ __device__ __forceinline__ float4 add4(const float4 a, const float4 b) {
   const float2 hi = __fadd2_rn(make_float2(a.z, a.w), make_float2(b.z, b.w));
   return make_float4(lo.x, lo.y, hi.x, hi.y);
 }
+// One float4 of a result state, written as fp32 (16 bytes) or rounded to bf16 (8 bytes); `idx4` counts float4s.
+template <int BF16>
+__device__ __forceinline__ void store_out4(void* base, int64_t idx4, const float4 v) {
+  if (BF16) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(base)[idx4] = pk;
+  } else {
+    reinterpret_cast<float4*>(base)[idx4] = v;
+  }
+}
 // 16-byte asynchronous copy global -> shared, bypassing registers
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"((unsigned)__cvta_generic_to_shared(smem)), "l"(gmem)
@@ -32,8 +45,8 @@ __device__ __forceinline__ void cp_async_wait_all() {
 // added in a different order.  Every state entry is an independent copy of this map, so a CTA owns a slab
 // of E consecutive entries, keeps F[:, slab] in shared memory and writes U[:, slab].
 // Layout in shared memory: point index major, E floats per point; a thread owns one float4 of an item.
-template <int D>
-__global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* __restrict__ in, float* __restrict__ out,
+template <int D, int BF16>
+__global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* __restrict__ in, void* __restrict__ out,
                                                               int q, int64_t P, int64_t Bn, int64_t state_elems,
                                                               int E) {
   extern __shared__ __align__(16) float4 smem4[];
@@ -54,7 +67,7 @@ __global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* _
   }
   cp_async_wait_all();
   __syncthreads();
-  float4* dst = reinterpret_cast<float4*>(out + bh * Bn * state_elems + e0);
+  const int64_t out0 = (bh * Bn * state_elems + e0) / 4;  // first float4 of this CTA's slab in the result table
   const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
 
   if (D == 2) {
@@ -69,14 +82,14 @@ __global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* _
         x1 -= a2;
         if (x1 < 0) x1 += q;
       }
-      dst[(int64_t)item * row4 + l] = acc;
+      store_out4<BF16>(out, out0 + (int64_t)item * row4 + l, acc);
     }
     // a = (0, 1):  U[q*q + b] = Σ_{x1} F[x1, b]
     for (int b = it0; b < q; b += IPP) {
       float4 acc = zero;
 #pragma unroll 4
       for (int x1 = 0; x1 < q; ++x1) acc = add4(acc, Fs[(x1 + q * b) * L4 + l]);
-      dst[(int64_t)(qq + b) * row4 + l] = acc;
+      store_out4<BF16>(out, out0 + (int64_t)(qq + b) * row4 + l, acc);
     }
   } else {
     float4* G2 = Fs + P * L4;          // [q*q][L4]   F summed over x1, indexed x2 + q*x3
@@ -100,14 +113,14 @@ __global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* _
         x2 -= a3;
         if (x2 < 0) x2 += q;
       }
-      dst[(int64_t)(qq * q + item) * row4 + l] = acc;
+      store_out4<BF16>(out, out0 + (int64_t)(qq * q + item) * row4 + l, acc);
     }
     // a = (0, 0, 1):  U[(q^2 + q) q + b] = Σ_{x2} G2[x2, b]
     for (int b = it0; b < q; b += IPP) {
       float4 acc = zero;
 #pragma unroll 4
       for (int x2 = 0; x2 < q; ++x2) acc = add4(acc, G2[(x2 + q * b) * L4 + l]);
-      dst[(int64_t)((qq + q) * q + b) * row4 + l] = acc;
+      store_out4<BF16>(out, out0 + (int64_t)((qq + q) * q + b) * row4 + l, acc);
     }
     // a = (1, a2, a3)
     for (int a3 = 0; a3 < q; ++a3) {
@@ -137,7 +150,7 @@ __global__ void __launch_bounds__(1024, 1) tabulate_staged_kernel(const float* _
           if (u < 0) u += q;
         }
         const int64_t h = (int64_t)(a2 + q * a3) * q + b;
-        dst[h * row4 + l] = acc;
+        store_out4<BF16>(out, out0 + h * row4 + l, acc);
       }
     }
   }
@@ -191,9 +204,9 @@ __device__ __noinline__ void radon_inplace(float* base) {
 
 // Register budget: 168 keeps two 192-thread CTAs per SM (q <= 11); the 7-warp CTAs of q = 13 may take 224.
 // Larger fields do not fit a q x q image in the registers of one thread and use tabulate_staged_kernel.
-template <int Q, int E>
+template <int Q, int E, int BF16>
 __global__ void __maxnreg__(Q <= 11 ? 168 : 224)
-    tabulate_radon3_kernel(const float* __restrict__ in, float* __restrict__ out, int P, int Bn, int64_t state_elems) {
+    tabulate_radon3_kernel(const float* __restrict__ in, void* __restrict__ out, int P, int Bn, int64_t state_elems) {
   extern __shared__ __align__(16) float4 smem4[];
   constexpr int q = Q, qq = Q * Q;
   constexpr int L4 = E / 4;
@@ -211,7 +224,7 @@ __global__ void __maxnreg__(Q <= 11 ? 168 : 224)
   for (int idx = tid; idx < P * L4; idx += NT) cp_async16(Fs + idx, src + (int64_t)(idx >> log2L4) * row4 + (idx & (L4 - 1)));
   cp_async_wait_all();
   __syncthreads();
-  float4* dst4 = reinterpret_cast<float4*>(out + bh * Bn * state_elems + e0);
+  const int64_t out0 = (bh * Bn * state_elems + e0) / 4;  // first float4 of this CTA's slab in the result table
   const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
   // directions with a leading zero work on G2[x2, x3] = Σ_{x1} F[x1, x2, x3]
   float4* G2 = Fs + P * L4;
@@ -233,13 +246,13 @@ __global__ void __maxnreg__(Q <= 11 ? 168 : 224)
       x2 -= a3;
       if (x2 < 0) x2 += q;
     }
-    dst4[(int64_t)(qq * q + item) * row4 + l] = acc;
+    store_out4<BF16>(out, out0 + (int64_t)(qq * q + item) * row4 + l, acc);
   }
   for (int b = it0; b < q; b += IPP) {  // a = (0, 0, 1)
     float4 acc = zero;
 #pragma unroll
     for (int x2 = 0; x2 < q; ++x2) acc = add4(acc, G2[(x2 + q * b) * L4 + l]);
-    dst4[(int64_t)((qq + q) * q + b) * row4 + l] = acc;
+    store_out4<BF16>(out, out0 + (int64_t)((qq + q) * q + b) * row4 + l, acc);
   }
   // a = (1, a2, a3), stage 1: thread (x2, e) transforms the image F[., x2, .] in place
   float* Ff = reinterpret_cast<float*>(Fs);
@@ -251,7 +264,7 @@ __global__ void __maxnreg__(Q <= 11 ? 168 : 224)
   if (it < q) radon_inplace<Q, E, Q>(Ff + (qq * it) * E + e);  // image [x2][u]
   __syncthreads();
   for (int idx = tid; idx < P * L4; idx += NT)  // rows 0 .. q^3-1 of U, 16-byte stores
-    dst4[(int64_t)(idx >> log2L4) * row4 + (idx & (L4 - 1))] = Fs[idx];
+    store_out4<BF16>(out, out0 + (int64_t)(idx >> log2L4) * row4 + (idx & (L4 - 1)), Fs[idx]);
 }
 
 // Transpose for D = 2:  F̄[x1, x2] = Σ_{a2} Ū[(1,a2), x1 + a2 x2] + Ū[(0,1), x2]
@@ -296,6 +309,11 @@ cudaError_t set_smem(K kernel, size_t bytes) {
 
 }  // namespace
 
+__global__ void widen_bf16_kernel(const __nv_bfloat16* __restrict__ src, float* __restrict__ dst, int64_t count) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) dst[i] = __bfloat162float(src[i]);
+}
+
 // ---- launchers ------------------------------------------------------------------------------------------------------
 // Shared-memory floats per slab entry the staged kernels need.
 // slab width of the register-resident form for the field sizes it is compiled for (0: not available)
@@ -321,8 +339,9 @@ int smat_tabulate_staged_slab(const SmatGeo& geo, int64_t state_elems, int trans
   return 0;
 }
 
-cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatGeo& geo, int64_t state_elems, int bh,
-                                        int transpose, cudaStream_t st) {
+cudaError_t smat_launch_tabulate_staged(const float* in, void* out, const SmatGeo& geo, int64_t state_elems, int bh,
+                                        int transpose, int out_bf16, cudaStream_t st) {
+  if (out_bf16 && transpose) return cudaErrorInvalidValue;
   const int E = smat_tabulate_staged_slab(geo, state_elems, transpose);
   if (E < 4) return cudaErrorInvalidConfiguration;
   const size_t smem = (size_t)staged_rows(geo, transpose) * E * sizeof(float);
@@ -334,12 +353,17 @@ cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatG
   if (nt < 128) nt = 128;
   cudaError_t err;
   if (geo.D == 3 && !transpose && radon3_q(geo.q)) {
-#define SMAT_RADON3(QV, EV)                                                                                \
-  if (geo.q == QV && E == EV) {                                                                            \
-    const int nr = (QV * EV + 31) / 32 * 32; /* one thread per (image, entry) */                           \
-    if ((err = set_smem(tabulate_radon3_kernel<QV, EV>, smem)) != cudaSuccess) return err;                 \
-    tabulate_radon3_kernel<QV, EV><<<grid, nr, smem, st>>>(in, out, (int)geo.P, (int)geo.B, state_elems);  \
-    return cudaGetLastError();                                                                             \
+#define SMAT_RADON3(QV, EV)                                                                                      \
+  if (geo.q == QV && E == EV) {                                                                                  \
+    const int nr = (QV * EV + 31) / 32 * 32; /* one thread per (image, entry) */                                 \
+    if (out_bf16) {                                                                                              \
+      if ((err = set_smem(tabulate_radon3_kernel<QV, EV, 1>, smem)) != cudaSuccess) return err;                  \
+      tabulate_radon3_kernel<QV, EV, 1><<<grid, nr, smem, st>>>(in, out, (int)geo.P, (int)geo.B, state_elems);   \
+    } else {                                                                                                     \
+      if ((err = set_smem(tabulate_radon3_kernel<QV, EV, 0>, smem)) != cudaSuccess) return err;                  \
+      tabulate_radon3_kernel<QV, EV, 0><<<grid, nr, smem, st>>>(in, out, (int)geo.P, (int)geo.B, state_elems);   \
+    }                                                                                                            \
+    return cudaGetLastError();                                                                                   \
   }
     SMAT_RADON3(5, 32) SMAT_RADON3(7, 32) SMAT_RADON3(11, 16) SMAT_RADON3(13, 16)
 #undef SMAT_RADON3
@@ -347,13 +371,21 @@ cudaError_t smat_launch_tabulate_staged(const float* in, float* out, const SmatG
   }
   if (geo.D == 2 && transpose) {
     if ((err = set_smem(tabulate_staged_t2_kernel, smem)) != cudaSuccess) return err;
-    tabulate_staged_t2_kernel<<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
-  } else if (geo.D == 2) {
-    if ((err = set_smem(tabulate_staged_kernel<2>, smem)) != cudaSuccess) return err;
-    tabulate_staged_kernel<2><<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+    tabulate_staged_t2_kernel<<<grid, nt, smem, st>>>(in, static_cast<float*>(out), geo.q, geo.P, geo.B, state_elems, E);
   } else {
-    if ((err = set_smem(tabulate_staged_kernel<3>, smem)) != cudaSuccess) return err;
-    tabulate_staged_kernel<3><<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+#define SMAT_STAGED(DV, BV)                                                                         \
+  if (geo.D == DV && out_bf16 == BV) {                                                              \
+    if ((err = set_smem(tabulate_staged_kernel<DV, BV>, smem)) != cudaSuccess) return err;          \
+    tabulate_staged_kernel<DV, BV><<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E); \
   }
+    SMAT_STAGED(2, 0) SMAT_STAGED(2, 1) SMAT_STAGED(3, 0) SMAT_STAGED(3, 1)
+#undef SMAT_STAGED
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st) {
+  widen_bf16_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src_bf16), dst,
+                                                                     count);
   return cudaGetLastError();
 }

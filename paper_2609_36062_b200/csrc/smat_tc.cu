@@ -314,6 +314,136 @@ __global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_const
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// state_read_tc_kernel: typed read Y_lr[t] = q_tᵀ U_type(t) (Algorithm 1, step 4) for plans whose type table is
+// kept in bf16.  Persistent CTAs (three per SM), one (type, head) item at a time:
+//   warp 4 lane 0 : TMA load of the 128 x 128 bf16 state (two boxes, MN-major B operand), then the MMA
+//                   Y = Q_h U_h   (M = up to 128 queries of the type, N = 128, K = 128)
+//   warps 0-3     : gather the queries of the type (token stride B) into the swizzled K-major A tile with
+//                   cp.async, later read the rows of Y from TMEM and scatter them to their tokens
+// Types with more than 128 queries take several passes over the same state.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int READ_SMEM = 4 * BOX_BYTES + 1024 + 256;
+
+struct ReadParams {
+  int64_t T, n, B;       // tokens per head, first recent token, number of types
+  int64_t items;         // heads * B
+  const __nv_bfloat16* Q;
+  float* ylr;            // [bh][T][128]
+  int* status;
+};
+
+__device__ __forceinline__ void cp_async16_tc(uint32_t smem_addr, const void* gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gmem) : "memory");
+}
+
+__global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constant__ CUtensorMap tmU,
+                                                            const ReadParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = smem;                    // queries, K-major, two 64-column blocks
+  uint8_t* sB = smem + 2 * BOX_BYTES;    // state, MN-major, two 64-column blocks
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 4 * BOX_BYTES);
+  uint64_t* bar_u = bars + 0;   // state landed (TMA)
+  uint64_t* bar_a = bars + 1;   // queries landed (128 arrivals)
+  uint64_t* bar_d = bars + 2;   // product in TMEM
+  uint64_t* bar_e = bars + 3;   // TMEM read out (4 arrivals)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const WaitCtx wc{cta_abort, prm.status};
+
+  if (threadIdx.x == 0) {
+    *cta_abort = 0;
+    mbar_init(bar_u, 1); mbar_init(bar_a, 128); mbar_init(bar_d, 1); mbar_init(bar_e, 4);
+    fence_barrier_init();
+  }
+  if (warp == 4) tmem_alloc(tmem_slot, TILE);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_d = *tmem_slot;
+  const int64_t m_recent = prm.T - prm.n;
+  uint32_t n_item = 0, n_pass = 0;  // completed uses of bar_u and of bar_a / bar_d / bar_e
+  constexpr uint32_t idesc = make_idesc(TILE, TILE, 0, 1);
+
+  for (int64_t item = blockIdx.x; item < prm.items; item += gridDim.x) {
+    const int64_t bh = item / prm.B, h = item - bh * prm.B;
+    const int64_t i0 = h ? h : prm.B;                            // first recent index (1-based) of this type
+    const int64_t cnt = i0 <= m_recent ? (m_recent - i0) / prm.B + 1 : 0;
+    if (cnt == 0) continue;
+    const int64_t t_first = prm.n + i0 - 1;
+    bool ok = true;
+    if (warp == 4 && lane == 0) {
+      mbar_expect_tx(bar_u, 2 * BOX_BYTES);
+      const int row = (int)(item * TILE);
+      tma_load_2d(sB, &tmU, 0, row, bar_u);
+      tma_load_2d(sB + BOX_BYTES, &tmU, HALF, row, bar_u);
+    }
+    for (int64_t k0 = 0; k0 < cnt && ok; k0 += TILE, ++n_pass) {
+      const int kn = (int)((cnt - k0) < TILE ? (cnt - k0) : TILE);
+      if (warp < 4) {
+        const int tid = threadIdx.x;
+        const uint32_t a_base = smem_u32(sA);
+        for (int idx = tid; idx < kn * 16; idx += 128) {
+          const int m = idx >> 4, gc = idx & 15;
+          const __nv_bfloat16* src = prm.Q + ((bh * prm.T + t_first + (k0 + m) * prm.B) * TILE + gc * 8);
+          cp_async16_tc(a_base + (gc >> 3) * BOX_BYTES + m * 128 + (((gc & 7) ^ (m & 7)) << 4), src);
+        }
+        asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+        fence_proxy_async();
+        mbar_arrive(bar_a);
+        ok = mbar_wait(bar_d, n_pass & 1, wc);
+        if (ok) {
+          fence_after_sync();
+          const int m = warp * 32 + lane;
+          float4* dst = reinterpret_cast<float4*>(prm.ylr + (bh * prm.T + t_first + (k0 + m) * prm.B) * TILE);
+#pragma unroll
+          for (int cb = 0; cb < 4; ++cb) {
+            uint32_t v[32];
+            tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+            tmem_ld_wait();
+            if (m < kn) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                dst[cb * 8 + i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                              __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+            }
+          }
+          fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_e);
+        }
+      } else if (lane == 0) {
+        if (k0 == 0) ok = mbar_wait(bar_u, n_item & 1, wc);
+        if (ok) ok = mbar_wait(bar_a, n_pass & 1, wc);
+        if (ok && n_pass > 0) ok = mbar_wait(bar_e, (n_pass - 1) & 1, wc);  // previous product has been read out
+        if (ok) {
+          fence_after_sync();
+#pragma unroll
+          for (int kk = 0; kk < TILE / 16; ++kk) {
+            const uint64_t dA = make_desc(smem_u32(sA) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+            const uint64_t dB = make_desc(smem_u32(sB) + kk * 2048, BOX_BYTES, 1024);
+            mma_bf16(tmem_d, dA, dB, idesc, kk != 0);
+          }
+          mma_commit(bar_d);
+          // the operands may be overwritten (next pass or next item) only after the MMA has read them
+          ok = mbar_wait(bar_d, n_pass & 1, wc);
+        }
+      }
+      ok = (__shfl_sync(0xffffffffu, (int)ok, 0) != 0) && ok;  // lanes of a warp leave together
+    }
+    ++n_item;
+    if (!ok) break;
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after_sync();
+    tmem_dealloc(tmem_d, TILE);
+  }
+}
+
 // ---- host: tensor maps ----------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -386,5 +516,24 @@ cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void
   if (err != cudaSuccess) return err;
   dim3 grid((unsigned)(NC * 2), (unsigned)bh);
   chunk_output_tc_kernel<<<grid, 160, OUT_SMEM, st>>>(tmQ, tmK, tmV, tmS, prm);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_state_read_tc(const void* Q, const void* U_bf16, float* ylr, int64_t T, int64_t n, int64_t B,
+                                      int bh, int* status, cudaStream_t st) {
+  CUtensorMap tmU;
+  if (!make_map(&tmU, U_bf16, (uint64_t)bh * B * TILE)) return cudaErrorInvalidValue;
+  ReadParams prm;
+  prm.T = T; prm.n = n; prm.B = B; prm.items = (int64_t)bh * B;
+  prm.Q = static_cast<const __nv_bfloat16*>(Q);
+  prm.ylr = ylr;
+  prm.status = status;
+  cudaError_t err = cudaFuncSetAttribute(state_read_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, READ_SMEM);
+  if (err != cudaSuccess) return err;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int64_t grid = prm.items < 3LL * sms ? prm.items : 3LL * sms;
+  state_read_tc_kernel<<<(unsigned)grid, 160, READ_SMEM, st>>>(tmU, prm);
   return cudaGetLastError();
 }

@@ -7,8 +7,9 @@ r = d_k, p = d_v, e = bytes per input element, fp32 tables:
                          + 2rp (T + T + n + m)      chunk summaries, carried-state read, pool, typed read
   ALU adds   (forward)   = nnz(C) rp + (T/c) rp     Algorithm 2's state additions + the scan
   HBM bytes  (forward)   = (2r + 2p) T e            Q, K, V in, O out
-                         + 2 P rp 4 + 2 B rp 4      profile table and type table, written once and read once
-                           (d = 1 has neither table)
+                         + 2 P rp 4 + 2 B rp s_U    profile table and type table, written once and read once
+                           (d = 1 has neither table; s_U = 4, or 2 where the implementation stores U as bf16 —
+                           both variants are reported)
   backward               = T (c+1)(3r+2p) + 15 T rp flop, the same adds again (Cᵀ tabulation, suffix scan),
                            (4r + 3p) T e bytes of tensors and 2 (2P + 2B) rp 4 bytes of tables
                            (F, U rebuilt; Ū, F̄ written and read)
@@ -52,12 +53,13 @@ class Work:
         return Work(self.flops * k, self.adds * k, self.bytes * k)
 
 
-def forward_work(T, c, r, p, e, geo) -> Work:
+def forward_work(T, c, r, p, e, geo, u_bytes=4) -> Work:
+    """u_bytes: element size of the type table as the implementation keeps it (4, or 2 where it is stored as bf16)."""
     rp = r * p
     lr = geo.d > 1
     flops = T * (c + 1) * (r + p) + 2 * rp * (2 * T + (geo.n + geo.m if lr else 0))
     adds = (geo.nnzC * rp if lr else 0) + (T // c) * rp
-    by = (2 * r + 2 * p) * T * e + (2 * (geo.P + geo.B) * rp * 4 if lr else 0)
+    by = (2 * r + 2 * p) * T * e + (2 * geo.P * rp * 4 + 2 * geo.B * rp * u_bytes if lr else 0)
     return Work(flops, adds, by)
 
 
@@ -85,18 +87,23 @@ def roofline_times(work: Work, peaks: dict, sustained: bool = True) -> dict:
 
 
 # Per-kernel algorithmic traffic (bytes), adds and flop, keyed by the stage names the library reports.
-def stage_work(name: str, T, c, r, p, e, geo) -> Work:
+def stage_work(name: str, T, c, r, p, e, geo, u_bytes=4) -> Work:
     rp, NC = r * p, T // c
     n, m, P, B = geo.n, geo.m, geo.P, geo.B
     st = 4 * rp
+    su = u_bytes * rp
+    tc_tiles = T // 128
     table = {
         "pool":        Work(2 * n * rp, 0, n * (r + p) * e + P * st),
-        "tabulate":    Work(0, geo.nnzC * rp, (P + B) * st),
+        "tabulate":    Work(0, geo.nnzC * rp, P * st + B * su),
         "chunk_state": Work(2 * T * rp, 0, T * (r + p) * e + NC * st),
         "scan":        Work(0, NC * rp, 2 * NC * st),
         "scores":      Work(T * (c + 1) * r, 0, 2 * T * r * e + T * c * 4),
         "read_chunk":  Work(2 * T * rp, 0, T * r * e + NC * st + T * p * 4),
         "read_type":   Work(2 * m * rp, 0, m * r * e + B * st + 2 * m * p * 4),
+        "read_type_tc": Work(2 * m * rp, 0, m * r * e + B * su + m * p * 4),
+        "chunk_scan_tc": Work(2 * T * rp, tc_tiles * rp, T * (r + p) * e + tc_tiles * rp * 2),
+        "chunk_output_tc": Work(T * 129 * (r + p) + 2 * T * rp, 0, T * (2 * r + 2 * p) * e + tc_tiles * rp * 2 + m * p * 4),
         "output":      Work(T * (c + 1) * p, 0, T * c * 4 + T * p * e + T * p * 4 + T * p * e),
     }
     return table.get(name, Work(0, 0, 0))

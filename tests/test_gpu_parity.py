@@ -72,8 +72,10 @@ def test_forward_matches_dense_oracle(d, T, dk, dv, c, dtype, q):
                     assert rel_err(to_numpy64(U[0]), tab["U"]) <= 1e-5
                 assert rel_err(to_numpy64(Sin[0]), ref_sin) <= 1e-5
             if d > 1:
+                # tensor-core plans with d >= 3 keep U in bf16 (it is only ever a bf16 MMA operand): one rounding
+                u_tol = 8e-3 if (plan.uses_tensor_cores() and d >= 3) else 1e-5
                 assert rel_err(to_numpy64(F[0]), tab["F"]) <= 1e-5
-                assert rel_err(to_numpy64(U[0]), tab["U"]) <= 1e-5
+                assert rel_err(to_numpy64(U[0]), tab["U"]) <= u_tol
 
 
 @pytest.mark.parametrize("d,T,dk,dv,c,dtype,q", SMALL)
