@@ -89,8 +89,9 @@ smat_status smat_get_geometry(const smat_plan* plan, smat_geometry* out);
 int smat_uses_tensor_cores(const smat_plan* plan);
 
 /* Bytes per element of the type table U as smat_forward keeps it: 4 (fp32), or 2 when the plan runs the typed read on
- * the tensor cores (bf16 inputs, d >= 3): there U is only ever a bf16 MMA operand, so it is rounded once when the
- * tabulation stores it and the table's HBM traffic halves.  smat_backward always builds fp32 tables. */
+ * the tensor cores (bf16 inputs; d >= 3, or d = 2 with at least 12 tokens per profile): there U is only ever a bf16
+ * MMA operand, so it is rounded once when it is stored and the table's HBM traffic halves (for d = 2 the profile
+ * table is the type table and is kept in bf16 too).  smat_backward always builds fp32 tables. */
 int smat_type_table_element_bytes(const smat_plan* plan);
 
 /* Bytes of workspace smat_forward (for_backward = 0) or smat_backward (for_backward = 1) needs. 0 if plan is NULL. */

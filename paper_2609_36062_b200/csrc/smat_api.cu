@@ -24,6 +24,8 @@ struct smat_plan {
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
   bool tc;             // tensor-core kernels for the causal branch
   bool u_bf16;         // forward keeps the type table U in bf16 and reads it with the tensor-core typed read
+  bool pool_tc;        // forward pools the profile table on the tensor cores (enough tokens per profile)
+  bool f_bf16;         // d = 2 on that path: the profile table is the type table, kept in bf16
   mutable int launches;
   mutable bool last_was_forward;  // which call left its tables in the workspace
   // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
@@ -276,8 +278,10 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
            g.m % 128 == 0 && g.n >= 128 && smat_tc_available();
   if (!g.dense_G && (smat_tabulate_alg2_slab(g.B, pl->rp) < 1)) { delete pl; return SMAT_ERR_UNSUPPORTED; }
   // d >= 3 on the tensor-core path: U is only ever a bf16 MMA operand, so it is stored as bf16 (half the bytes)
-  pl->u_bf16 = pl->tc && g.D >= 2 && !(flags & SMAT_FLAG_ALG2_TABULATION) &&
-               smat_tabulate_staged_slab(g, pl->rp, 0) >= 4;
+  pl->pool_tc = pl->tc && !g.dense_G && g.n / g.P >= 12;
+  pl->f_bf16 = pl->pool_tc && g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION);
+  pl->u_bf16 = pl->f_bf16 || (pl->tc && g.D >= 2 && !(flags & SMAT_FLAG_ALG2_TABULATION) &&
+                              smat_tabulate_staged_slab(g, pl->rp, 0) >= 4);
   const size_t state = (size_t)pl->rp * sizeof(float);
   const int wide = d_k > d_v ? d_k : d_v;
   size_t off = 0;
@@ -365,7 +369,11 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
     float* ylr = cx.f(pl->off_acc);
     const bool lr = !pl->geo.dense_G;
     if (lr) {
-      outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));                         // step 2
+      if (pl->pool_tc)                                                                       // step 2
+        SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, pl->T, pl->geo.n, pl->geo.P,
+                                                    pl->bh, status, cx.st));
+      else
+        outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
       tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);              // step 3
       if (pl->u_bf16)                                                                        // step 4
         SMAT_TRY(cx, "read_type_tc", smat_launch_state_read_tc(Q, cx.ws + pl->off_U, ylr, pl->T, pl->geo.n,
@@ -488,8 +496,12 @@ smat_status smat_debug_tables(const smat_plan* pl, const void* workspace, float*
                               state, pl->bh, cudaMemcpyDeviceToDevice, st);
     }
   } else {
-    if (F && err == cudaSuccess)
-      err = cudaMemcpyAsync(F, ws + pl->off_F, (size_t)pl->bh * pl->geo.P * state, cudaMemcpyDeviceToDevice, st);
+    if (F && err == cudaSuccess) {
+      if (pl->f_bf16 && pl->last_was_forward)
+        err = smat_launch_widen_bf16(ws + pl->off_F, F, (int64_t)pl->bh * pl->geo.P * pl->rp, st);
+      else
+        err = cudaMemcpyAsync(F, ws + pl->off_F, (size_t)pl->bh * pl->geo.P * state, cudaMemcpyDeviceToDevice, st);
+    }
     if (U && err == cudaSuccess) {
       if (pl->u_bf16 && pl->last_was_forward)  // the forward of this plan keeps U in bf16: widen on export
         err = smat_launch_widen_bf16(ws + pl->off_U, U, (int64_t)pl->bh * pl->geo.B * pl->rp, st);

@@ -103,3 +103,6 @@ cudaError_t smat_launch_state_read_tc(const void* Q, const void* U_bf16, float* 
                                       int bh, int* status, cudaStream_t st);
 // bf16 -> fp32 copy of a table (debug export).
 cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st);
+// Pooling on tensor cores: F[bh][x] = Σ_{t ≡ x (mod P), t < n} k_t v_tᵀ, stored as fp32 or bf16.
+cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, int64_t T, int64_t n, int64_t P,
+                                int bh, int* status, cudaStream_t st);

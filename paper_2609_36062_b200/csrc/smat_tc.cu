@@ -444,6 +444,139 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// pool_tc_kernel: F_x = Σ_{t ≡ x (mod P), t < n} k_t v_tᵀ (Algorithm 1, step 2) for profiles shared by enough tokens to
+// fill tensor-core tiles (d = 2: ~170 tokens per profile, d = 3: 12-24).  Persistent CTAs, one (profile, head) item at
+// a time:
+//   warps 0-3     : gather the profile's K and V rows (token stride P) into swizzled MN-major tiles with cp.async
+//                   (rows up to the next multiple of 16 are zeroed), later write the 128 x 128 state from TMEM
+//   warp 4 lane 0 : MMA  F_x += K_xᵀ V_x  (M = N = 128 features, K = 16 tokens per instruction), TOK tokens per pass
+// OUT_BF16 = 1 stores the state as bf16 (d = 2, where the profile table is the type table and is only read as an MMA
+// operand), else fp32.
+// ---------------------------------------------------------------------------------------------------------------
+struct PoolParams {
+  int64_t T, n, P;
+  int64_t items;           // heads * P
+  const __nv_bfloat16* K;
+  const __nv_bfloat16* V;
+  void* F;                 // [bh][P][128][128] fp32 or bf16
+  int* status;
+};
+
+template <int TOK, int OUT_BF16>
+__global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
+  constexpr int OP_BYTES = 2 * TOK * 128;  // one operand: two 64-feature blocks of TOK rows x 128 bytes
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + OP_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * OP_BYTES);
+  uint64_t* bar_a = bars + 0;   // operands landed (128 arrivals)
+  uint64_t* bar_d = bars + 1;   // MMAs of the pass finished
+  uint64_t* bar_e = bars + 2;   // state read out of TMEM (4 arrivals)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const WaitCtx wc{cta_abort, prm.status};
+
+  if (threadIdx.x == 0) {
+    *cta_abort = 0;
+    mbar_init(bar_a, 128); mbar_init(bar_d, 1); mbar_init(bar_e, 4);
+    fence_barrier_init();
+  }
+  if (warp == 4) tmem_alloc(tmem_slot, TILE);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_d = *tmem_slot;
+  uint32_t n_pass = 0, n_item = 0;
+  constexpr uint32_t idesc = make_idesc(TILE, TILE, 1, 1);
+
+  for (int64_t item = blockIdx.x; item < prm.items; item += gridDim.x, ++n_item) {
+    const int64_t bh = item / prm.P, x = item - bh * prm.P;
+    const int64_t cnt = x < prm.n ? (prm.n - x + prm.P - 1) / prm.P : 0;
+    bool ok = true;
+    for (int64_t k0 = 0; k0 < cnt && ok; k0 += TOK, ++n_pass) {
+      const int kn = (int)((cnt - k0) < TOK ? (cnt - k0) : TOK);
+      const int kpad = (kn + 15) & ~15;
+      if (warp < 4) {
+        const int tid = threadIdx.x;
+        if (n_pass > 0) ok = mbar_wait(bar_d, (n_pass - 1) & 1, wc);  // previous pass has read the tiles
+        if (ok) {
+          const uint32_t a_base = smem_u32(sA), b_base = smem_u32(sB);
+          for (int idx = tid; idx < kpad * 32; idx += 128) {  // 16 chunks of K and 16 of V per token
+            const int k = idx >> 5, w = idx & 31, gc = w & 15;
+            const uint32_t dst = (w < 16 ? a_base : b_base) + (gc >> 3) * (TOK * 128) + k * 128 + (((gc & 7) ^ (k & 7)) << 4);
+            if (k < kn) {
+              const __nv_bfloat16* src = (w < 16 ? prm.K : prm.V) + ((bh * prm.T + x + (k0 + k) * prm.P) * TILE + gc * 8);
+              cp_async16_tc(dst, src);
+            } else {
+              asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
+            }
+          }
+          asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+          fence_proxy_async();
+          mbar_arrive(bar_a);
+        }
+      } else if (lane == 0) {
+        ok = mbar_wait(bar_a, n_pass & 1, wc);
+        if (ok && k0 == 0 && n_item > 0) ok = mbar_wait(bar_e, (n_item - 1) & 1, wc);  // previous state has been read out
+        if (ok) {
+          fence_after_sync();
+          const uint64_t dA = make_desc(smem_u32(sA), TOK * 128, 1024);
+          const uint64_t dB = make_desc(smem_u32(sB), TOK * 128, 1024);
+          for (int kk = 0; kk < kpad / 16; ++kk)
+            mma_bf16(tmem_d, dA + (uint64_t)(kk * 128), dB + (uint64_t)(kk * 128), idesc, (k0 | kk) != 0);
+          mma_commit(bar_d);
+        }
+      }
+      ok = (__shfl_sync(0xffffffffu, (int)ok, 0) != 0) && ok;
+    }
+    if (!ok) break;
+    if (warp < 4) {
+      const int i = warp * 32 + lane;  // state row = TMEM lane
+      if (cnt > 0) {
+        ok = mbar_wait(bar_d, (n_pass - 1) & 1, wc);
+        if (!ok) break;
+        fence_after_sync();
+      }
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        if (cnt > 0) {
+          tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0u;  // profile cell without tokens (P > n)
+        }
+        if (OUT_BF16) {
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(prm.F) + (item * TILE + i) * TILE + cb * 32);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4)
+            dst[q4] = make_uint4(pack_bf16(__uint_as_float(v[8 * q4]), __uint_as_float(v[8 * q4 + 1])),
+                                 pack_bf16(__uint_as_float(v[8 * q4 + 2]), __uint_as_float(v[8 * q4 + 3])),
+                                 pack_bf16(__uint_as_float(v[8 * q4 + 4]), __uint_as_float(v[8 * q4 + 5])),
+                                 pack_bf16(__uint_as_float(v[8 * q4 + 6]), __uint_as_float(v[8 * q4 + 7])));
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(prm.F) + (item * TILE + i) * TILE + cb * 32);
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4) dst[q4] = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+        }
+      }
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_e);
+    }
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after_sync();
+    tmem_dealloc(tmem_d, TILE);
+  }
+}
+
 // ---- host: tensor maps ----------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -536,4 +669,30 @@ cudaError_t smat_launch_state_read_tc(const void* Q, const void* U_bf16, float* 
   const int64_t grid = prm.items < 3LL * sms ? prm.items : 3LL * sms;
   state_read_tc_kernel<<<(unsigned)grid, 160, READ_SMEM, st>>>(tmU, prm);
   return cudaGetLastError();
+}
+
+template <int TOK, int OUT_BF16>
+static cudaError_t launch_pool_tc(const PoolParams& prm, cudaStream_t st) {
+  const int smem = 4 * TOK * 128 + 1024 + 256;
+  cudaError_t err = cudaFuncSetAttribute(pool_tc_kernel<TOK, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (err != cudaSuccess) return err;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int64_t grid = prm.items < 3LL * sms ? prm.items : 3LL * sms;
+  pool_tc_kernel<TOK, OUT_BF16><<<(unsigned)grid, 160, smem, st>>>(prm);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, int64_t T, int64_t n, int64_t P,
+                                int bh, int* status, cudaStream_t st) {
+  PoolParams prm;
+  prm.T = T; prm.n = n; prm.P = P; prm.items = (int64_t)bh * P;
+  prm.K = static_cast<const __nv_bfloat16*>(K);
+  prm.V = static_cast<const __nv_bfloat16*>(V);
+  prm.F = F;
+  prm.status = status;
+  const int64_t max_cnt = (n + P - 1) / P;
+  if (max_cnt <= 32) return out_bf16 ? launch_pool_tc<32, 1>(prm, st) : launch_pool_tc<32, 0>(prm, st);
+  return out_bf16 ? launch_pool_tc<128, 1>(prm, st) : launch_pool_tc<128, 0>(prm, st);
 }
