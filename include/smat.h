@@ -57,6 +57,8 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
 /* plan flags */
 #define SMAT_FLAG_SIMT_ONLY 1u      /* never use the tensor-core kernels (bf16 plans run the fp32-ALU path) */
 #define SMAT_FLAG_ALG2_TABULATION 2u /* tabulate with the direct double loop of Algorithm 2 instead of the staged sums */
+#define SMAT_FLAG_PER_TILE_STATES 4u /* tensor-core causal branch: store one incoming state per 128-token tile (scan, then
+                                        independent tiles) instead of one per segment of tiles (two-level form) */
 
 /* Sizes of the construction (Sec. 3, "construction of G" and "Scaling with sequence length"). */
 typedef struct {

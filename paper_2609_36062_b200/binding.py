@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsmat.so")
 SMAT_F32, SMAT_BF16 = 0, 1
 FLAG_SIMT_ONLY = 1
 FLAG_ALG2_TABULATION = 2
+FLAG_PER_TILE_STATES = 4
 
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",

@@ -381,11 +381,22 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
       else
         state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);
     }
-    SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, pl->geo.n,
-                                                             lr ? 0 : 1, status, cx.st));   // steps 5-6
-    SMAT_TRY(cx, "chunk_output_tc", smat_launch_chunk_output_tc(Q, K, V, cx.ws + pl->off_sin, ylr,
-                                                                 lr ? pl->geo.n : pl->T, O, pl->T, pl->bh, status,
-                                                                 cx.st));                   // step 7
+    const int64_t tiles0 = lr ? pl->geo.n / 128 : pl->T / 128, tiles1 = lr ? pl->geo.m / 128 : 0;
+    const int L = (pl->flags & SMAT_FLAG_PER_TILE_STATES) ? 1 : smat_segment_tiles(tiles0, tiles1, pl->bh);
+    if (L >= 2) {  // steps 5-7, two-level: segment totals, scan of the totals, fused per-segment output
+      float* seg = cx.f(pl->off_sin);
+      const int64_t nseg = pl->T / 128 / L, nseg0 = tiles0 / L;
+      SMAT_TRY(cx, "segment_state_tc", smat_launch_segment_state_tc(K, V, seg, pl->T, L, pl->bh, status, cx.st));
+      SMAT_TRY(cx, "segment_scan", smat_launch_scan(seg, pl->rp, nseg, pl->bh, 0, nseg0, nseg0, nseg, 0, cx.st));
+      SMAT_TRY(cx, "segment_output_tc", smat_launch_segment_output_tc(Q, K, V, seg, ylr, lr ? pl->geo.n : pl->T, O,
+                                                                       pl->T, L, pl->bh, status, cx.st));
+    } else {
+      SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, pl->geo.n,
+                                                               lr ? 0 : 1, status, cx.st));   // steps 5-6
+      SMAT_TRY(cx, "chunk_output_tc", smat_launch_chunk_output_tc(Q, K, V, cx.ws + pl->off_sin, ylr,
+                                                                   lr ? pl->geo.n : pl->T, O, pl->T, pl->bh, status,
+                                                                   cx.st));                   // step 7
+    }
     pl->launches = cx.launches;
     return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
   }

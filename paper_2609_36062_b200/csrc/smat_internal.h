@@ -106,3 +106,10 @@ cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t cou
 // Pooling on tensor cores: F[bh][x] = Σ_{t ≡ x (mod P), t < n} k_t v_tᵀ, stored as fp32 or bf16.
 cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, int64_t T, int64_t n, int64_t P,
                                 int bh, int* status, cudaStream_t st);
+// Two-level causal branch: segment totals, then (after an exclusive scan of the totals) per-segment fused output.
+int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh);
+cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* totals, int64_t T, int L, int bh,
+                                         int* status, cudaStream_t st);
+cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const void* V, const float* seg_in,
+                                          const float* ylr, int64_t n_lr, void* O, int64_t T, int L, int bh,
+                                          int* status, cudaStream_t st);

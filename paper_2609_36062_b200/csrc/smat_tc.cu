@@ -315,6 +315,306 @@ __global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_const
 }
 
 // ---------------------------------------------------------------------------------------------------------------
+// Two-level form of the causal branch.  Each block of the sequence is cut into segments of L tiles.
+//   segment_state_tc_kernel  : total[seg] = Σ_{tiles of the segment} K_bᵀ V_b, accumulated in TMEM (fp32), written once
+//   (scan_kernel turns the totals into the state entering each segment: exclusive prefix sum per block, fp32)
+//   segment_output_tc_kernel : one CTA per (segment, head, 64-column half) walks its L tiles with the running state
+//                              S in TMEM:  O_b = Q_b S + tril(Q_b K_bᵀ) V_b + Y_lr,b ;  S += K_bᵀ V_b
+// Against the per-tile form (chunk_scan + chunk_output) this writes and reads one fp32 state per segment instead of
+// one bf16 state per tile, at the price of reading K and V a second time.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int SEG_STATE_STAGES = 3;
+constexpr int SEG_STATE_SMEM = SEG_STATE_STAGES * 4 * BOX_BYTES + 1024 + 256;
+
+struct SegStateParams {
+  int64_t T;
+  int L, nseg;           // tiles per segment, segments per head
+  float* totals;         // [bh][nseg][128][128]
+  int* status;
+};
+
+__global__ void __launch_bounds__(192) segment_state_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                               const __grid_constant__ CUtensorMap tmV,
+                                                               const SegStateParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SEG_STATE_STAGES * 4 * BOX_BYTES);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + SEG_STATE_STAGES;
+  uint64_t* done = empty + SEG_STATE_STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int seg = blockIdx.x, bh = blockIdx.y;
+  const WaitCtx wc{cta_abort, prm.status};
+  if (threadIdx.x == 0) {
+    *cta_abort = 0;
+    for (int s = 0; s < SEG_STATE_STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    mbar_init(done, 1);
+    fence_barrier_init();
+  }
+  if (warp == 4) tmem_alloc(tmem_slot, TILE);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_d = *tmem_slot;
+  if (warp == 4 && lane == 0) {
+    for (int it = 0; it < prm.L; ++it) {
+      const int s = it % SEG_STATE_STAGES;
+      if (it >= SEG_STATE_STAGES && !mbar_wait(empty + s, ((it / SEG_STATE_STAGES) - 1) & 1, wc)) break;
+      uint8_t* st = smem + s * 4 * BOX_BYTES;
+      const int row = (int)((int64_t)bh * prm.T + ((int64_t)seg * prm.L + it) * TILE);
+      mbar_expect_tx(full + s, 4 * BOX_BYTES);
+      tma_load_2d(st, &tmK, 0, row, full + s);
+      tma_load_2d(st + BOX_BYTES, &tmK, HALF, row, full + s);
+      tma_load_2d(st + 2 * BOX_BYTES, &tmV, 0, row, full + s);
+      tma_load_2d(st + 3 * BOX_BYTES, &tmV, HALF, row, full + s);
+    }
+  } else if (warp == 5 && lane == 0) {
+    constexpr uint32_t idesc = make_idesc(TILE, TILE, 1, 1);
+    bool ok = true;
+    for (int it = 0; it < prm.L && ok; ++it) {
+      const int s = it % SEG_STATE_STAGES;
+      ok = mbar_wait(full + s, (it / SEG_STATE_STAGES) & 1, wc);
+      if (!ok) break;
+      fence_after_sync();
+      const uint32_t sK = smem_u32(smem + s * 4 * BOX_BYTES);
+      const uint64_t dA = make_desc(sK, BOX_BYTES, 1024);
+      const uint64_t dB = make_desc(sK + 2 * BOX_BYTES, BOX_BYTES, 1024);
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk)
+        mma_bf16(tmem_d, dA + (uint64_t)(kk * 128), dB + (uint64_t)(kk * 128), idesc, (it | kk) != 0);
+      mma_commit(empty + s);
+    }
+    if (ok) mma_commit(done);
+  } else if (warp < 4) {
+    if (mbar_wait(done, 0, wc)) {
+      fence_after_sync();
+      const int i = warp * 32 + lane;
+      uint4* dst = reinterpret_cast<uint4*>(prm.totals + (((int64_t)bh * prm.nseg + seg) * TILE + i) * TILE);
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4) dst[cb * 8 + q4] = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+      }
+    }
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after_sync();
+    tmem_dealloc(tmem_d, TILE);
+  }
+}
+
+// Shared memory of segment_output_tc_kernel: two stages of (Q: 2 boxes, K: 2 boxes, V half: 1 box), the bf16 copy
+// of the running state half (1 box), the rounded score tile P (2 boxes).
+constexpr int SEG_OUT_STAGE = 5 * BOX_BYTES;
+constexpr int SEG_OUT_SMEM = 2 * SEG_OUT_STAGE + 3 * BOX_BYTES + 1024 + 256;
+
+struct SegOutParams {
+  int64_t T;
+  int L, nseg;
+  const float* seg_in;   // [bh][nseg][128][128] state entering each segment
+  int64_t n_lr;
+  const float* ylr;
+  __nv_bfloat16* O;
+  int* status;
+};
+
+__global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+                                                                const __grid_constant__ CUtensorMap tmK,
+                                                                const __grid_constant__ CUtensorMap tmV,
+                                                                const SegOutParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sS = smem + 2 * SEG_OUT_STAGE;            // bf16 state half, MN-major (rows = state row i)
+  uint8_t* sP = sS + BOX_BYTES;                      // rounded scores, K-major, two 64-key blocks
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + 2 * BOX_BYTES);
+  uint64_t* full = bars;          // [2] tile operands landed
+  uint64_t* empty = bars + 2;     // [2] tile operands consumed
+  uint64_t* bar_s = bars + 4;     // state half converted (128 arrivals)
+  uint64_t* bar_sc = bars + 5;    // scores in TMEM
+  uint64_t* bar_p = bars + 6;     // P written (128 arrivals)
+  uint64_t* bar_o = bars + 7;     // output in TMEM and state updated
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int half = blockIdx.x & 1, seg = blockIdx.x >> 1, bh = blockIdx.y;
+  const WaitCtx wc{cta_abort, prm.status};
+  if (threadIdx.x == 0) {
+    *cta_abort = 0;
+    mbar_init(full, 1); mbar_init(full + 1, 1); mbar_init(empty, 1); mbar_init(empty + 1, 1);
+    mbar_init(bar_s, 128); mbar_init(bar_sc, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+    fence_barrier_init();
+  }
+  if (warp == 4) tmem_alloc(tmem_slot, 256);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s = tmem_base, tmem_sc = tmem_base + HALF, tmem_o = tmem_base + HALF + TILE;
+  const int64_t tile0 = (int64_t)seg * prm.L;
+
+  if (warp == 4 && lane == 0) {
+    for (int it = 0; it < prm.L; ++it) {
+      const int s = it & 1;
+      if (it >= 2 && !mbar_wait(empty + s, ((it >> 1) - 1) & 1, wc)) break;
+      uint8_t* st = smem + s * SEG_OUT_STAGE;
+      const int row = (int)((int64_t)bh * prm.T + (tile0 + it) * TILE);
+      mbar_expect_tx(full + s, SEG_OUT_STAGE);
+      tma_load_2d(st, &tmQ, 0, row, full + s);
+      tma_load_2d(st + BOX_BYTES, &tmQ, HALF, row, full + s);
+      tma_load_2d(st + 2 * BOX_BYTES, &tmK, 0, row, full + s);
+      tma_load_2d(st + 3 * BOX_BYTES, &tmK, HALF, row, full + s);
+      tma_load_2d(st + 4 * BOX_BYTES, &tmV, half * HALF, row, full + s);
+    }
+  } else if (warp == 5 && lane == 0) {
+    constexpr uint32_t idesc_sc = make_idesc(TILE, TILE, 0, 0);
+    constexpr uint32_t idesc_o = make_idesc(TILE, HALF, 0, 1);
+    constexpr uint32_t idesc_s = make_idesc(TILE, HALF, 1, 1);
+    for (int it = 0; it < prm.L; ++it) {
+      const int s = it & 1;
+      const uint32_t sQ = smem_u32(smem + s * SEG_OUT_STAGE);
+      const uint32_t sK = sQ + 2 * BOX_BYTES, sV = sQ + 4 * BOX_BYTES;
+      if (!mbar_wait(full + s, (it >> 1) & 1, wc)) break;
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) {   // scores Sc = Q Kᵀ
+        const uint64_t dA = make_desc(sQ + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = make_desc(sK + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        mma_bf16(tmem_sc, dA, dB, idesc_sc, kk != 0);
+      }
+      mma_commit(bar_sc);
+      if (!mbar_wait(bar_s, it & 1, wc)) break;  // bf16 copy of the state is in shared memory, O of the last tile read out
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) {   // O = Q S
+        const uint64_t dA = make_desc(sQ + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = make_desc(smem_u32(sS) + kk * 2048, BOX_BYTES, 1024);
+        mma_bf16(tmem_o, dA, dB, idesc_o, kk != 0);
+      }
+      if (!mbar_wait(bar_p, it & 1, wc)) break;
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) {   // O += P V
+        const uint64_t dA = make_desc(smem_u32(sP) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = make_desc(sV + kk * 2048, BOX_BYTES, 1024);
+        mma_bf16(tmem_o, dA, dB, idesc_o, 1);
+      }
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) {   // S += Kᵀ V
+        const uint64_t dA = make_desc(sK + kk * 2048, BOX_BYTES, 1024);
+        const uint64_t dB = make_desc(sV + kk * 2048, BOX_BYTES, 1024);
+        mma_bf16(tmem_s, dA, dB, idesc_s, 1);
+      }
+      mma_commit(bar_o);
+      mma_commit(empty + s);
+    }
+  } else if (warp < 4) {
+    const int m = warp * 32 + lane;  // TMEM lane: state row i, and query row of the tile
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    bool ok = true;
+    for (int it = 0; it < prm.L && ok; ++it) {
+      // --- bf16 copy of the state half entering this tile ---
+      uint32_t v0[32], v1[32];
+      if (it == 0) {  // state entering the segment: global fp32 -> TMEM (accumulator) and shared memory
+        const uint4* src = reinterpret_cast<const uint4*>(prm.seg_in + (((int64_t)bh * prm.nseg + seg) * TILE + m) * TILE + half * HALF);
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4) {
+          const uint4 a = __ldg(src + q4), b = __ldg(src + 8 + q4);
+          v0[4 * q4] = a.x; v0[4 * q4 + 1] = a.y; v0[4 * q4 + 2] = a.z; v0[4 * q4 + 3] = a.w;
+          v1[4 * q4] = b.x; v1[4 * q4 + 1] = b.y; v1[4 * q4 + 2] = b.z; v1[4 * q4 + 3] = b.w;
+        }
+        tmem_st32(tmem_s + lane_base, v0);
+        tmem_st32(tmem_s + lane_base + 32, v1);
+        tmem_st_wait();
+      } else {
+        tmem_ld32(tmem_s + lane_base, v0);
+        tmem_ld32(tmem_s + lane_base + 32, v1);
+        tmem_ld_wait();
+      }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {  // eight 16-byte chunks = 64 columns of row m
+        const uint32_t* v = c < 4 ? v0 : v1;
+        const int o = (c & 3) * 8;
+        const uint4 pk = make_uint4(pack_bf16(__uint_as_float(v[o]), __uint_as_float(v[o + 1])),
+                                    pack_bf16(__uint_as_float(v[o + 2]), __uint_as_float(v[o + 3])),
+                                    pack_bf16(__uint_as_float(v[o + 4]), __uint_as_float(v[o + 5])),
+                                    pack_bf16(__uint_as_float(v[o + 6]), __uint_as_float(v[o + 7])));
+        *reinterpret_cast<uint4*>(sS + m * 128 + ((c ^ (m & 7)) << 4)) = pk;
+      }
+      fence_proxy_async();
+      fence_before_sync();
+      mbar_arrive(bar_s);
+      // --- scores -> masked bf16 P ---
+      ok = mbar_wait(bar_sc, it & 1, wc);
+      if (!ok) break;
+      fence_after_sync();
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_sc + lane_base + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int h2 = 0; h2 < 4; ++h2) {
+            const int k0 = cb * 32 + i * 8 + h2 * 2;
+            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
+            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            pk[h2] = pack_bf16(lo, hi);
+          }
+          const int j8 = cb * 4 + i;
+          *reinterpret_cast<uint4*>(sP + (j8 >> 3) * BOX_BYTES + m * 128 + (((j8 & 7) ^ (m & 7)) << 4)) =
+              make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
+      fence_proxy_async();
+      fence_before_sync();
+      mbar_arrive(bar_p);
+      // --- output rows ---
+      ok = mbar_wait(bar_o, it & 1, wc);
+      if (!ok) break;
+      fence_after_sync();
+      const int64_t t = (tile0 + it) * TILE + m;
+      const bool add_lr = t >= prm.n_lr;
+      const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+      uint4* dst = reinterpret_cast<uint4*>(prm.O + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+#pragma unroll
+      for (int cb = 0; cb < 2; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_o + lane_base + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float f[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i * 8 + e]);
+          if (add_lr) {
+            const float4 a = __ldg(y4 + cb * 8 + i * 2), c = __ldg(y4 + cb * 8 + i * 2 + 1);
+            f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
+            f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
+          }
+          dst[cb * 4 + i] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
+                                       pack_bf16(f[6], f[7]));
+        }
+      }
+    }
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after_sync();
+    tmem_dealloc(tmem_base, 256);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
 // state_read_tc_kernel: typed read Y_lr[t] = q_tᵀ U_type(t) (Algorithm 1, step 4) for plans whose type table is
 // kept in bf16.  Persistent CTAs (three per SM), one (type, head) item at a time:
 //   warp 4 lane 0 : TMA load of the 128 x 128 bf16 state (two boxes, MN-major B operand), then the MMA
@@ -695,4 +995,47 @@ cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_b
   const int64_t max_cnt = (n + P - 1) / P;
   if (max_cnt <= 32) return out_bf16 ? launch_pool_tc<32, 1>(prm, st) : launch_pool_tc<32, 0>(prm, st);
   return out_bf16 ? launch_pool_tc<128, 1>(prm, st) : launch_pool_tc<128, 0>(prm, st);
+}
+
+// Largest segment length (tiles) that divides every block and still leaves enough CTAs to fill the machine.
+int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh) {
+  for (int L = 8; L >= 2; L >>= 1) {
+    if (tiles_block0 % L || (tiles_block1 && tiles_block1 % L)) continue;
+    const int64_t ctas = (tiles_block0 + tiles_block1) / L * 2 * bh;
+    if (ctas >= 296 || L == 2) return L;
+  }
+  return 1;
+}
+
+cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* totals, int64_t T, int L, int bh,
+                                         int* status, cudaStream_t st) {
+  CUtensorMap tmK, tmV;
+  if (!make_map(&tmK, K, (uint64_t)bh * T) || !make_map(&tmV, V, (uint64_t)bh * T)) return cudaErrorInvalidValue;
+  SegStateParams prm;
+  prm.T = T; prm.L = L; prm.nseg = (int)(T / TILE / L); prm.totals = totals; prm.status = status;
+  cudaError_t err =
+      cudaFuncSetAttribute(segment_state_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_STATE_SMEM);
+  if (err != cudaSuccess) return err;
+  dim3 grid((unsigned)prm.nseg, (unsigned)bh);
+  segment_state_tc_kernel<<<grid, 192, SEG_STATE_SMEM, st>>>(tmK, tmV, prm);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const void* V, const float* seg_in,
+                                          const float* ylr, int64_t n_lr, void* O, int64_t T, int L, int bh,
+                                          int* status, cudaStream_t st) {
+  CUtensorMap tmQ, tmK, tmV;
+  if (!make_map(&tmQ, Q, (uint64_t)bh * T) || !make_map(&tmK, K, (uint64_t)bh * T) ||
+      !make_map(&tmV, V, (uint64_t)bh * T))
+    return cudaErrorInvalidValue;
+  SegOutParams prm;
+  prm.T = T; prm.L = L; prm.nseg = (int)(T / TILE / L); prm.seg_in = seg_in; prm.n_lr = n_lr; prm.ylr = ylr;
+  prm.O = static_cast<__nv_bfloat16*>(O);
+  prm.status = status;
+  cudaError_t err =
+      cudaFuncSetAttribute(segment_output_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_OUT_SMEM);
+  if (err != cudaSuccess) return err;
+  dim3 grid((unsigned)(prm.nseg * 2), (unsigned)bh);
+  segment_output_tc_kernel<<<grid, 192, SEG_OUT_SMEM, st>>>(tmQ, tmK, tmV, prm);
+  return cudaGetLastError();
 }

@@ -131,6 +131,25 @@ def test_tensor_core_and_alu_paths_agree():
     assert rel_err(a, b) <= 1e-2
 
 
+@pytest.mark.parametrize("d,T,q", [(1, 4096, 0), (3, 4096, 0), (2, 2560, 0), (4, 8192, 0)])
+def test_two_level_and_per_tile_causal_branches_agree(d, T, q):
+    """Segment form (one fp32 state per segment of tiles) against the per-tile form, and both against the oracle."""
+    w = _small("seg", d, T, 128, 128, 128, "bf16", heads=3, seed=51, recipe="normalised")
+    host, dev = device_inputs(w)
+    seg_plan, tile_plan = _plan(w, q), _plan(w, q, flags=binding.FLAG_PER_TILE_STATES)
+    a = seg_plan.forward(dev["q"], dev["k"], dev["v"])
+    seg_plan.check_status()
+    b = tile_plan.forward(dev["q"], dev["k"], dev["v"])
+    tile_plan.check_status()
+    geo = so.geometry(T, 128, d, q or None)
+    rows = sample_tokens(geo, 64, seed=3)
+    Q64, K64, V64 = (synth.as_float64(w, host[x][1]) for x in ("q", "k", "v"))
+    ref = so.forward_rows(Q64, K64, V64, geo, rows)
+    for out in (a, b):
+        assert rel_err(to_numpy64(out[0, 1][rows]), ref) <= TOL["bf16"]
+    assert rel_err(to_numpy64(a), to_numpy64(b)) <= 1e-2
+
+
 def test_chunk_size_invariance_on_device():
     outs = []
     for c in (16, 32, 64, 128):
