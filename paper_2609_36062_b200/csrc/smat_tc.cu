@@ -425,10 +425,11 @@ struct SegOutParams {
   int* status;
 };
 
-__global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+__global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                 const __grid_constant__ CUtensorMap tmK,
                                                                 const __grid_constant__ CUtensorMap tmV,
                                                                 const SegOutParams prm) {
+  // warps 0-3: state conversion and output rows; warps 4-7: scores -> P; warp 8: TMA producer; warp 9: MMA issuer
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sS = smem + 2 * SEG_OUT_STAGE;            // bf16 state half, MN-major (rows = state row i)
@@ -451,15 +452,16 @@ __global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_con
     mbar_init(bar_s, 128); mbar_init(bar_sc, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
     fence_barrier_init();
   }
-  if (warp == 4) tmem_alloc(tmem_slot, 256);
+  if (warp == 8) tmem_alloc(tmem_slot, 512);
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_sc = tmem_base + HALF, tmem_o = tmem_base + HALF + TILE;
+  // columns: running state half [0,64), scores [64,192), two output buffers [192,256) and [256,320)
+  const uint32_t tmem_s = tmem_base, tmem_sc = tmem_base + HALF, tmem_o0 = tmem_base + HALF + TILE;
   const int64_t tile0 = (int64_t)seg * prm.L;
 
-  if (warp == 4 && lane == 0) {
+  if (warp == 8 && lane == 0) {
     for (int it = 0; it < prm.L; ++it) {
       const int s = it & 1;
       if (it >= 2 && !mbar_wait(empty + s, ((it >> 1) - 1) & 1, wc)) break;
@@ -472,7 +474,7 @@ __global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_con
       tma_load_2d(st + 3 * BOX_BYTES, &tmK, HALF, row, full + s);
       tma_load_2d(st + 4 * BOX_BYTES, &tmV, half * HALF, row, full + s);
     }
-  } else if (warp == 5 && lane == 0) {
+  } else if (warp == 9 && lane == 0) {
     constexpr uint32_t idesc_sc = make_idesc(TILE, TILE, 0, 0);
     constexpr uint32_t idesc_o = make_idesc(TILE, HALF, 0, 1);
     constexpr uint32_t idesc_s = make_idesc(TILE, HALF, 1, 1);
@@ -480,16 +482,17 @@ __global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_con
       const int s = it & 1;
       const uint32_t sQ = smem_u32(smem + s * SEG_OUT_STAGE);
       const uint32_t sK = sQ + 2 * BOX_BYTES, sV = sQ + 4 * BOX_BYTES;
+      const uint32_t tmem_o = tmem_o0 + (it & 1) * HALF;
       if (!mbar_wait(full + s, (it >> 1) & 1, wc)) break;
       fence_after_sync();
 #pragma unroll
-      for (int kk = 0; kk < TILE / 16; ++kk) {   // scores Sc = Q Kᵀ
+      for (int kk = 0; kk < TILE / 16; ++kk) {   // scores Sc = Q Kᵀ (the score buffer was read out before bar_p of the last tile)
         const uint64_t dA = make_desc(sQ + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
         const uint64_t dB = make_desc(sK + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
         mma_bf16(tmem_sc, dA, dB, idesc_sc, kk != 0);
       }
       mma_commit(bar_sc);
-      if (!mbar_wait(bar_s, it & 1, wc)) break;  // bf16 copy of the state is in shared memory, O of the last tile read out
+      if (!mbar_wait(bar_s, it & 1, wc)) break;  // bf16 copy of the state is in shared memory
       fence_after_sync();
 #pragma unroll
       for (int kk = 0; kk < TILE / 16; ++kk) {   // O = Q S
@@ -517,28 +520,10 @@ __global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_con
   } else if (warp < 4) {
     const int m = warp * 32 + lane;  // TMEM lane: state row i, and query row of the tile
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-    bool ok = true;
-    for (int it = 0; it < prm.L && ok; ++it) {
-      // --- bf16 copy of the state half entering this tile ---
-      uint32_t v0[32], v1[32];
-      if (it == 0) {  // state entering the segment: global fp32 -> TMEM (accumulator) and shared memory
-        const uint4* src = reinterpret_cast<const uint4*>(prm.seg_in + (((int64_t)bh * prm.nseg + seg) * TILE + m) * TILE + half * HALF);
+    // writes the bf16 copy of this thread's state row (64 columns held in v0, v1) into the swizzled B tile
+    auto publish_state = [&](const uint32_t (&v0)[32], const uint32_t (&v1)[32]) {
 #pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4) {
-          const uint4 a = __ldg(src + q4), b = __ldg(src + 8 + q4);
-          v0[4 * q4] = a.x; v0[4 * q4 + 1] = a.y; v0[4 * q4 + 2] = a.z; v0[4 * q4 + 3] = a.w;
-          v1[4 * q4] = b.x; v1[4 * q4 + 1] = b.y; v1[4 * q4 + 2] = b.z; v1[4 * q4 + 3] = b.w;
-        }
-        tmem_st32(tmem_s + lane_base, v0);
-        tmem_st32(tmem_s + lane_base + 32, v1);
-        tmem_st_wait();
-      } else {
-        tmem_ld32(tmem_s + lane_base, v0);
-        tmem_ld32(tmem_s + lane_base + 32, v1);
-        tmem_ld_wait();
-      }
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {  // eight 16-byte chunks = 64 columns of row m
+      for (int c = 0; c < 8; ++c) {
         const uint32_t* v = c < 4 ? v0 : v1;
         const int o = (c & 3) * 8;
         const uint4 pk = make_uint4(pack_bf16(__uint_as_float(v[o]), __uint_as_float(v[o + 1])),
@@ -550,41 +535,41 @@ __global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_con
       fence_proxy_async();
       fence_before_sync();
       mbar_arrive(bar_s);
-      // --- scores -> masked bf16 P ---
-      ok = mbar_wait(bar_sc, it & 1, wc);
-      if (!ok) break;
-      fence_after_sync();
+    };
+    {  // state entering the segment: global fp32 -> TMEM (accumulator) and shared memory
+      uint32_t v0[32], v1[32];
+      const uint4* src = reinterpret_cast<const uint4*>(prm.seg_in + (((int64_t)bh * prm.nseg + seg) * TILE + m) * TILE + half * HALF);
 #pragma unroll
-      for (int cb = 0; cb < 4; ++cb) {
-        uint32_t v[32];
-        tmem_ld32(tmem_sc + lane_base + cb * 32, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint32_t pk[4];
-#pragma unroll
-          for (int h2 = 0; h2 < 4; ++h2) {
-            const int k0 = cb * 32 + i * 8 + h2 * 2;
-            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
-            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
-            pk[h2] = pack_bf16(lo, hi);
-          }
-          const int j8 = cb * 4 + i;
-          *reinterpret_cast<uint4*>(sP + (j8 >> 3) * BOX_BYTES + m * 128 + (((j8 & 7) ^ (m & 7)) << 4)) =
-              make_uint4(pk[0], pk[1], pk[2], pk[3]);
-        }
+      for (int q4 = 0; q4 < 8; ++q4) {
+        const uint4 a = __ldg(src + q4), b = __ldg(src + 8 + q4);
+        v0[4 * q4] = a.x; v0[4 * q4 + 1] = a.y; v0[4 * q4 + 2] = a.z; v0[4 * q4 + 3] = a.w;
+        v1[4 * q4] = b.x; v1[4 * q4 + 1] = b.y; v1[4 * q4 + 2] = b.z; v1[4 * q4 + 3] = b.w;
       }
-      fence_proxy_async();
-      fence_before_sync();
-      mbar_arrive(bar_p);
-      // --- output rows ---
-      ok = mbar_wait(bar_o, it & 1, wc);
-      if (!ok) break;
-      fence_after_sync();
+      tmem_st32(tmem_s + lane_base, v0);
+      tmem_st32(tmem_s + lane_base + 32, v1);
+      tmem_st_wait();
+      publish_state(v0, v1);
+    }
+    for (int it = 0; it < prm.L; ++it) {
       const int64_t t = (tile0 + it) * TILE + m;
       const bool add_lr = t >= prm.n_lr;
-      const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+      float4 y[16];  // long-range term of this row, fetched before the wait
+      if (add_lr) {
+        const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) y[i] = __ldg(y4 + i);
+      }
+      if (!mbar_wait(bar_o, it & 1, wc)) break;
+      fence_after_sync();
+      if (it + 1 < prm.L) {  // the state now includes this tile: publish it for the next one first (critical path)
+        uint32_t v0[32], v1[32];
+        tmem_ld32(tmem_s + lane_base, v0);
+        tmem_ld32(tmem_s + lane_base + 32, v1);
+        tmem_ld_wait();
+        publish_state(v0, v1);
+      }
       uint4* dst = reinterpret_cast<uint4*>(prm.O + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+      const uint32_t tmem_o = tmem_o0 + (it & 1) * HALF;
 #pragma unroll
       for (int cb = 0; cb < 2; ++cb) {
         uint32_t v[32];
@@ -596,7 +581,7 @@ __global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_con
 #pragma unroll
           for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i * 8 + e]);
           if (add_lr) {
-            const float4 a = __ldg(y4 + cb * 8 + i * 2), c = __ldg(y4 + cb * 8 + i * 2 + 1);
+            const float4 a = y[cb * 8 + i * 2], c = y[cb * 8 + i * 2 + 1];
             f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
             f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
           }
@@ -605,12 +590,46 @@ __global__ void __launch_bounds__(192) segment_output_tc_kernel(const __grid_con
         }
       }
     }
+  } else if (warp < 8) {
+    const int m = (warp - 4) * 32 + lane;  // query row of the tile = TMEM lane
+    const uint32_t lane_base = (uint32_t)((warp - 4) * 32) << 16;
+    for (int it = 0; it < prm.L; ++it) {
+      if (!mbar_wait(bar_sc, it & 1, wc)) break;
+      fence_after_sync();
+      uint4 pk[16];  // the masked, rounded score row: sixteen 16-byte chunks of 8 keys
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_sc + lane_base + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint32_t w[4];
+#pragma unroll
+          for (int h2 = 0; h2 < 4; ++h2) {
+            const int k0 = cb * 32 + i * 8 + h2 * 2;
+            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
+            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            w[h2] = pack_bf16(lo, hi);
+          }
+          pk[cb * 4 + i] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      // P of the previous tile must have been consumed (its MMA is covered by bar_o of that tile)
+      if (it > 0 && !mbar_wait(bar_o, (it - 1) & 1, wc)) break;
+#pragma unroll
+      for (int j8 = 0; j8 < 16; ++j8)
+        *reinterpret_cast<uint4*>(sP + (j8 >> 3) * BOX_BYTES + m * 128 + (((j8 & 7) ^ (m & 7)) << 4)) = pk[j8];
+      fence_proxy_async();
+      fence_before_sync();
+      mbar_arrive(bar_p);
+    }
   }
   fence_before_sync();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 8) {
     fence_after_sync();
-    tmem_dealloc(tmem_base, 256);
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -1036,6 +1055,6 @@ cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const vo
       cudaFuncSetAttribute(segment_output_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_OUT_SMEM);
   if (err != cudaSuccess) return err;
   dim3 grid((unsigned)(prm.nseg * 2), (unsigned)bh);
-  segment_output_tc_kernel<<<grid, 192, SEG_OUT_SMEM, st>>>(tmQ, tmK, tmV, prm);
+  segment_output_tc_kernel<<<grid, 320, SEG_OUT_SMEM, st>>>(tmQ, tmK, tmV, prm);
   return cudaGetLastError();
 }
