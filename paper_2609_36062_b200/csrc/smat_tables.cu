@@ -351,6 +351,8 @@ cudaError_t smat_launch_tabulate_staged(const float* in, void* out, const SmatGe
   const int64_t passes = (units + 1023) / 1024;
   int nt = (int)(((units + passes - 1) / passes + 31) / 32 * 32);
   if (nt < 128) nt = 128;
+  // d = 3 has no barrier between its sums: small CTAs, several per SM, overlap one CTA's slab load with another's sums
+  if (geo.D == 2 && nt > 256) nt = 256;
   cudaError_t err;
   if (geo.D == 3 && !transpose && radon3_q(geo.q)) {
 #define SMAT_RADON3(QV, EV)                                                                                      \

@@ -1018,7 +1018,7 @@ cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_b
 
 // Largest segment length (tiles) that divides every block and still leaves enough CTAs to fill the machine.
 int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh) {
-  for (int L = 8; L >= 2; L >>= 1) {
+  for (int L = 16; L >= 2; L >>= 1) {
     if (tiles_block0 % L || (tiles_block1 && tiles_block1 % L)) continue;
     const int64_t ctas = (tiles_block0 + tiles_block1) / L * 2 * bh;
     if (ctas >= 296 || L == 2) return L;
