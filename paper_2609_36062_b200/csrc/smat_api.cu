@@ -370,14 +370,15 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
     const bool lr = !pl->geo.dense_G;
     if (lr) {
       if (pl->pool_tc)                                                                       // step 2
-        SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, pl->T, pl->geo.n, pl->geo.P,
-                                                    pl->bh, status, cx.st));
+        SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, group(pl, SMAT_GM_PROFILE),
+                                                    pl->geo.P, max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh,
+                                                    status, cx.st));
       else
         outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
       tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);              // step 3
       if (pl->u_bf16)                                                                        // step 4
-        SMAT_TRY(cx, "read_type_tc", smat_launch_state_read_tc(Q, cx.ws + pl->off_U, ylr, pl->T, pl->geo.n,
-                                                               pl->geo.B, pl->bh, status, cx.st));
+        SMAT_TRY(cx, "read_type_tc", smat_launch_state_read_tc(Q, cx.ws + pl->off_U, ylr, 0, group(pl, SMAT_GM_TYPE),
+                                                               pl->geo.B, pl->T, pl->bh, status, cx.st));
       else
         state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);
     }
@@ -392,7 +393,7 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
                                                                        pl->T, L, pl->bh, status, cx.st));
     } else {
       SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, pl->geo.n,
-                                                               lr ? 0 : 1, status, cx.st));   // steps 5-6
+                                                               lr ? 0 : 1, 0, status, cx.st));   // steps 5-6
       SMAT_TRY(cx, "chunk_output_tc", smat_launch_chunk_output_tc(Q, K, V, cx.ws + pl->off_sin, ylr,
                                                                    lr ? pl->geo.n : pl->T, O, pl->T, pl->bh, status,
                                                                    cx.st));                   // step 7
@@ -425,6 +426,72 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
   pl->last_was_forward = false;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   const bool lr = !pl->geo.dense_G;
+  if (pl->tc) {
+    // Tensor-core backward.  Forward tables are rebuilt as in smat_forward (U in bf16 where the plan keeps it so);
+    // the per-tile states S_in and D̄ are bf16 tiles; the long-range contributions go through one fp32 buffer
+    // that each within-chunk adjoint adds to its rows.
+    int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
+    float* lrbuf = cx.f(pl->off_acc);
+    const SmatGroupSpec types = group(pl, SMAT_GM_TYPE), profs = group(pl, SMAT_GM_PROFILE);
+    const int64_t n = pl->geo.n;
+    const bool fbar_bf16 = pl->u_bf16 && pl->geo.D <= 2;  // F̄ readable by the tensor-core read (d = 2, 3)
+    if (lr) {
+      if (pl->pool_tc)
+        SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, profs, pl->geo.P,
+                                                    max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh, status,
+                                                    cx.st));
+      else
+        outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
+      tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
+      // Ū_h = Σ q dOᵀ over the type (Eq. "lr-adjoint"), then F̄ = Cᵀ Ū
+      const bool ubar_tc = pl->geo.m / pl->geo.B >= 12;
+      const bool ubar_bf16 = ubar_tc && pl->geo.D == 1 && fbar_bf16;  // d = 2: F̄ is Ū itself
+      if (ubar_tc)
+        SMAT_TRY(cx, "bwd_pool_type_tc", smat_launch_pool_tc(Q, dO, cx.ws + pl->off_ubar, ubar_bf16, types, pl->geo.B,
+                                                             max_group_tokens(pl, SMAT_GM_TYPE), pl->T, pl->bh,
+                                                             status, cx.st));
+      else
+        outer_sum(cx, "bwd_pool_type", SMAT_GM_TYPE, Q, dO, cx.f(pl->off_ubar));
+      const bool fbar_is_bf16 = pl->geo.D == 1 ? ubar_bf16 : fbar_bf16;
+      tabulate(cx, "bwd_tabulate_t", cx.f(pl->off_ubar), cx.f(pl->off_fbar), 1, pl->geo.D == 2 && fbar_bf16);
+      // per-tile states
+      SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 0, 0, status, cx.st));
+      SMAT_TRY(cx, "bwd_chunk_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 0, 1, status, cx.st));
+      // dQ: recent rows add U_type dO
+      if (pl->u_bf16)
+        SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, lrbuf, 1, types, pl->geo.B,
+                                                                 pl->T, pl->bh, status, cx.st));
+      else
+        state_read(cx, "bwd_dq_type", SMAT_GM_TYPE, dO, cx.f(pl->off_U), 1, nullptr, lrbuf, nullptr);
+      SMAT_TRY(cx, "bwd_dq_tile_tc", smat_launch_chunk_adjoint_tc(0, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
+                                                                  lrbuf, n, pl->T, dQ, pl->T, pl->bh, status, cx.st));
+      // dK: distant rows add F̄_prof v
+      if (fbar_is_bf16)
+        SMAT_TRY(cx, "bwd_dk_profile_tc", smat_launch_state_read_tc(V, cx.ws + pl->off_fbar, lrbuf, 1, profs, pl->geo.P,
+                                                                    pl->T, pl->bh, status, cx.st));
+      else
+        state_read(cx, "bwd_dk_profile", SMAT_GM_PROFILE, V, cx.f(pl->off_fbar), 1, nullptr, lrbuf, nullptr);
+      SMAT_TRY(cx, "bwd_dk_tile_tc", smat_launch_chunk_adjoint_tc(1, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
+                                                                  lrbuf, 0, n, dK, pl->T, pl->bh, status, cx.st));
+      // dV: distant rows add F̄_profᵀ k
+      if (fbar_is_bf16)
+        SMAT_TRY(cx, "bwd_dv_profile_tc", smat_launch_state_read_tc(K, cx.ws + pl->off_fbar, lrbuf, 0, profs, pl->geo.P,
+                                                                    pl->T, pl->bh, status, cx.st));
+      else
+        state_read(cx, "bwd_dv_profile", SMAT_GM_PROFILE, K, cx.f(pl->off_fbar), 0, nullptr, lrbuf, nullptr);
+      SMAT_TRY(cx, "bwd_dv_tile_tc", smat_launch_chunk_adjoint_tc(2, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
+                                                                  lrbuf, 0, n, dV, pl->T, pl->bh, status, cx.st));
+    } else {
+      SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 1, 0, status, cx.st));
+      SMAT_TRY(cx, "bwd_chunk_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 1, 1, status, cx.st));
+      for (int which = 0; which < 3; ++which)
+        SMAT_TRY(cx, which == 0 ? "bwd_dq_tile_tc" : (which == 1 ? "bwd_dk_tile_tc" : "bwd_dv_tile_tc"),
+                 smat_launch_chunk_adjoint_tc(which, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar, lrbuf, 0, 0,
+                                              which == 0 ? dQ : (which == 1 ? dK : dV), pl->T, pl->bh, status, cx.st));
+    }
+    pl->launches = cx.launches;
+    return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+  }
   build_forward_tables(cx, K, V);
   float* sin = cx.f(pl->off_sin);
   float* dbar = cx.f(pl->off_dbar);

@@ -92,20 +92,28 @@ cudaError_t smat_launch_tabulate_staged(const float* in, void* out, const SmatGe
 bool smat_tc_available();
 // S_in[bh][tile] (bf16 [128][128]) = exclusive prefix sum of K_bᵀ V_b over the tiles of each block;
 // through = 1 runs one scan over the whole sequence (d = 1), else the scan restarts at token n.
+// reverse = 1 gives exclusive suffix sums instead (the scan adjoint, with K, V replaced by Q, dO).
 cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf16, int64_t T, int bh, int64_t n,
-                                      int through, int* status, cudaStream_t st);
+                                      int through, int reverse, int* status, cudaStream_t st);
+// Within-chunk adjoints on tensor cores (which = 0: dQ, 1: dK, 2: dV), see tile_product_tc_kernel.
+cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K, const void* V, const void* dO,
+                                         const void* Sin_bf16, const void* Dbar_bf16, const float* addend,
+                                         int64_t add_lo, int64_t add_hi, void* Out, int64_t T, int bh, int* status,
+                                         cudaStream_t st);
 // O_b = Q_b S_in[b] + tril(Q_b K_bᵀ) V_b (+ ylr rows for tokens >= n_lr).
 cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
                                         const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,
                                         cudaStream_t st);
 // Typed read on tensor cores: ylr[t] = q_tᵀ U_type(t) for recent tokens, U kept as bf16 [bh][B][128][128].
-cudaError_t smat_launch_state_read_tc(const void* Q, const void* U_bf16, float* ylr, int64_t T, int64_t n, int64_t B,
-                                      int bh, int* status, cudaStream_t st);
+// (transposed = 1 contracts the second state index instead: out[t] = state · x_t; grp selects types or profiles)
+cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, int transposed,
+                                      const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh, int* status,
+                                      cudaStream_t st);
 // bf16 -> fp32 copy of a table (debug export).
 cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st);
 // Pooling on tensor cores: F[bh][x] = Σ_{t ≡ x (mod P), t < n} k_t v_tᵀ, stored as fp32 or bf16.
-cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, int64_t T, int64_t n, int64_t P,
-                                int bh, int* status, cudaStream_t st);
+cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, const SmatGroupSpec& grp,
+                                int64_t groups, int64_t max_tokens, int64_t T, int bh, int* status, cudaStream_t st);
 // Two-level causal branch: segment totals, then (after an exclusive scan of the totals) per-segment fused output.
 int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh);
 cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* totals, int64_t T, int L, int bh,

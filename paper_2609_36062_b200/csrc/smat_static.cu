@@ -66,7 +66,7 @@ extern "C" smat_status smat_forward_causal_static(const void* Q, const void* K, 
   // writes every S_in tile of this problem before the output kernel reads it.
   if (cudaMemsetAsync(status, 0, STATIC_STATUS_BYTES, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
   const int bh = batch * heads;
-  if (smat_launch_chunk_scan_tc(K, V, sin, T, bh, 0, /*through=*/1, status, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  if (smat_launch_chunk_scan_tc(K, V, sin, T, bh, 0, /*through=*/1, /*reverse=*/0, status, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
   if (smat_launch_chunk_output_tc(Q, K, V, sin, nullptr, /*n_lr=*/T, O, T, bh, status, st) != cudaSuccess)
     return SMAT_ERR_LAUNCH;
   return SMAT_OK;

@@ -268,7 +268,8 @@ __global__ void __maxnreg__(Q <= 11 ? 168 : 224)
 }
 
 // Transpose for D = 2:  F̄[x1, x2] = Σ_{a2} Ū[(1,a2), x1 + a2 x2] + Ū[(0,1), x2]
-__global__ void __launch_bounds__(1024, 1) tabulate_staged_t2_kernel(const float* __restrict__ in, float* __restrict__ out,
+template <int BF16>
+__global__ void __launch_bounds__(1024, 1) tabulate_staged_t2_kernel(const float* __restrict__ in, void* __restrict__ out,
                                                                  int q, int64_t P, int64_t Bn, int64_t state_elems,
                                                                  int E) {
   extern __shared__ __align__(16) float4 smem4[];
@@ -287,7 +288,7 @@ __global__ void __launch_bounds__(1024, 1) tabulate_staged_t2_kernel(const float
   }
   cp_async_wait_all();
   __syncthreads();
-  float4* dst = reinterpret_cast<float4*>(out + bh * P * state_elems + e0);
+  const int64_t out0 = (bh * P * state_elems + e0) / 4;
   for (int item = it0; item < qq; item += IPP) {  // item = x1 + q*x2
     const int x2 = item / q, x1 = item - x2 * q;
     float4 acc = Us[(qq + x2) * L4 + l];
@@ -298,7 +299,7 @@ __global__ void __launch_bounds__(1024, 1) tabulate_staged_t2_kernel(const float
       b += x2;
       if (b >= q) b -= q;
     }
-    dst[(int64_t)item * row4 + l] = acc;
+    store_out4<BF16>(out, out0 + (int64_t)item * row4 + l, acc);
   }
 }
 
@@ -341,7 +342,7 @@ int smat_tabulate_staged_slab(const SmatGeo& geo, int64_t state_elems, int trans
 
 cudaError_t smat_launch_tabulate_staged(const float* in, void* out, const SmatGeo& geo, int64_t state_elems, int bh,
                                         int transpose, int out_bf16, cudaStream_t st) {
-  if (out_bf16 && transpose) return cudaErrorInvalidValue;
+  if (out_bf16 && transpose && geo.D != 2) return cudaErrorInvalidValue;
   const int E = smat_tabulate_staged_slab(geo, state_elems, transpose);
   if (E < 4) return cudaErrorInvalidConfiguration;
   const size_t smem = (size_t)staged_rows(geo, transpose) * E * sizeof(float);
@@ -372,8 +373,13 @@ cudaError_t smat_launch_tabulate_staged(const float* in, void* out, const SmatGe
     return cudaErrorInvalidConfiguration;
   }
   if (geo.D == 2 && transpose) {
-    if ((err = set_smem(tabulate_staged_t2_kernel, smem)) != cudaSuccess) return err;
-    tabulate_staged_t2_kernel<<<grid, nt, smem, st>>>(in, static_cast<float*>(out), geo.q, geo.P, geo.B, state_elems, E);
+    if (out_bf16) {
+      if ((err = set_smem(tabulate_staged_t2_kernel<1>, smem)) != cudaSuccess) return err;
+      tabulate_staged_t2_kernel<1><<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+    } else {
+      if ((err = set_smem(tabulate_staged_t2_kernel<0>, smem)) != cudaSuccess) return err;
+      tabulate_staged_t2_kernel<0><<<grid, nt, smem, st>>>(in, out, geo.q, geo.P, geo.B, state_elems, E);
+    }
   } else {
 #define SMAT_STAGED(DV, BV)                                                                         \
   if (geo.D == DV && out_bf16 == BV) {                                                              \

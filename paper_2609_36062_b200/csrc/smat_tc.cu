@@ -4,7 +4,8 @@
 //
 //   chunk_scan_tc_kernel   : D_b = K_bᵀ V_b for the chunks of one block in order, with the exclusive
 //                            prefix sum carried in registers; emits S_in[b] as bf16        (steps 5-6)
-//   chunk_output_tc_kernel : O_b = Q_b S_in[b] + tril(Q_b K_bᵀ) V_b + Y_lr,b               (step 7, Eq. "local")
+//   tile_product_tc_kernel : O_b = Q_b S_in[b] + tril(Q_b K_bᵀ) V_b + Y_lr,b (step 7, Eq. "local") and the three
+//                            within-chunk adjoints of the backward pass (Eq. "local-adjoint")
 //
 // The tile width is 128 tokens whatever chunk size the caller named: the result does not depend on the
 // chunk width once the block boundary n is fixed, and the launcher requires n and T - n to be multiples of 128.
@@ -39,6 +40,7 @@ struct ScanParams {
   int64_t T;        // tokens per head
   int NC;           // tiles per head
   int lo[2], hi[2]; // tile ranges of the (up to two) blocks
+  int reverse;      // 0: exclusive prefix sums (S_in); 1: exclusive suffix sums (the scan adjoint D̄)
   __nv_bfloat16* Sin;  // [bh][NC][128][128]
   int* status;
 };
@@ -77,8 +79,8 @@ __global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constan
   if (warp == 4 && lane == 0) {
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
-    for (int b = lo; b + 1 < hi; ++b) {  // the last tile's own sum is never read
-      const int it = b - lo, s = it % SCAN_STAGES;
+    for (int it = 0; it + 1 < hi - lo; ++it) {  // the last visited tile's own sum is never read
+      const int b = prm.reverse ? hi - 1 - it : lo + it, s = it % SCAN_STAGES;
       if (it >= SCAN_STAGES && !mbar_wait(empty + s, ((it / SCAN_STAGES) - 1) & 1, wc)) break;
       uint8_t* st = smem + s * SCAN_STAGE_BYTES;
       const int row = (int)(bh * prm.T + (int64_t)b * TILE);
@@ -89,8 +91,8 @@ __global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constan
     }
   } else if (warp == 5 && lane == 0) {
     constexpr uint32_t idesc = make_idesc(TILE, HALF, 1, 1);
-    for (int b = lo; b + 1 < hi; ++b) {
-      const int it = b - lo, s = it % SCAN_STAGES, db = it % SCAN_DBUF;
+    for (int it = 0; it + 1 < hi - lo; ++it) {
+      const int s = it % SCAN_STAGES, db = it % SCAN_DBUF;
       if (!mbar_wait(full + s, (it / SCAN_STAGES) & 1, wc)) break;
       if (it >= SCAN_DBUF && !mbar_wait(dempty + db, ((it / SCAN_DBUF) - 1) & 1, wc)) break;
       fence_after_sync();
@@ -109,9 +111,9 @@ __global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constan
     float acc[HALF];
 #pragma unroll
     for (int j = 0; j < HALF; ++j) acc[j] = 0.f;
-    for (int b = lo; b < hi; ++b) {
-      const int it = b - lo, db = it % SCAN_DBUF;
-      // S_in[b] = running sum before this tile
+    for (int it = 0; it < hi - lo; ++it) {
+      const int b = prm.reverse ? hi - 1 - it : lo + it, db = it % SCAN_DBUF;
+      // state[b] = running sum before this tile (in visiting order)
       uint4* dst = reinterpret_cast<uint4*>(prm.Sin + (((int64_t)bh * prm.NC + b) * TILE + row) * TILE + half * HALF);
 #pragma unroll
       for (int j8 = 0; j8 < HALF / 8; ++j8) {
@@ -122,7 +124,7 @@ __global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constan
         pk.w = pack_bf16(acc[j8 * 8 + 6], acc[j8 * 8 + 7]);
         dst[j8] = pk;
       }
-      if (b + 1 == hi) break;  // every issued MMA has been consumed: nothing is in flight at teardown
+      if (it + 1 == hi - lo) break;  // every issued MMA has been consumed: nothing is in flight at teardown
       if (!mbar_wait(dfull + db, (it / SCAN_DBUF) & 1, wc)) break;
       fence_after_sync();
       uint32_t v0[32], v1[32];
@@ -149,41 +151,54 @@ __global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// chunk_output_tc_kernel: one CTA per (tile, head, 64-column half of the output).
-//   warp 4 lane 0 : TMA loads (Q_b, K_b: two boxes each; V_b[:, half], S_in[b][:, half]: one box each), then the MMAs
-//        MMA1  Sc = Q_b K_bᵀ                 (M = N = 128 tokens, K = 128)            -> TMEM columns [0, 128)
-//        MMA2  Oh = Q_b S_in[b][:, half]     (M = 128, N = 64, K = 128)               -> TMEM columns [128, 192)
-//        MMA3  Oh += P V_b[:, half]          (P = tril(Sc) in bf16, written over K_b)
-//   warps 0-3     : one query row per thread: mask and round the scores into the swizzled K-major layout,
-//                   later read Oh, add the long-range term and store the output row
+// tile_product_tc_kernel: one CTA per (tile, head, 64-column half of the output) computes
+//
+//        Out_b = X · P3_b  +  P4_b · St_b  (+ addend rows),      X = tril(P1_b P2_bᵀ) or its transpose,
+//
+// which is the forward tile (Eq. "local") and each of the three within-chunk adjoints (Eq. "local-adjoint")
+// together with the broadcast of the scanned state adjoint:
+//        O_b  = tril(Q Kᵀ)   V  + Q  S_in      P1 = Q,  P2 = K, P3 = V,  P4 = Q  (= P1), St = S_in   as [k = i][n = j]
+//        dQ_b = tril(dO Vᵀ)  K  + dO S_inᵀ     P1 = dO, P2 = V, P3 = K,  P4 = dO (= P1), St = S_inᵀ: K-major rows i
+//        dK_b = tril(dO Vᵀ)ᵀ Q  + V  D̄ᵀ        P1 = dO, P2 = V, P3 = Q,  P4 = V  (= P2), St = D̄ᵀ  : K-major rows i
+//        dV_b = tril(Q Kᵀ)ᵀ  dO + K  D̄         P1 = Q,  P2 = K, P3 = dO, P4 = K  (= P2), St = D̄    as [k = i][n = j]
+// All operands are the natural row-major tiles; transposes are expressed through the operand-major bits of the MMA.
+//   warp 4 lane 0 : TMA loads (P1, P2: two boxes each; P3[:, half]; state half), then
+//        MMA1  Sc = P1 P2ᵀ                                     -> TMEM columns [0, 128)
+//        MMA2  Oh = P4 · St half          (M = 128, N = 64)    -> TMEM columns [128, 192)
+//        MMA3  Oh += X(ᵀ) · P3[:, half]   (X = masked, rounded Sc, written over the score operand that P4 is not)
+//   warps 0-3     : one tile row per thread: mask and round the scores into the swizzled layout, later read Oh,
+//                   add the long-range rows and store
 // ---------------------------------------------------------------------------------------------------------------
 constexpr int OUT_SMEM = 6 * BOX_BYTES + 1024 + 256;
 
-struct OutParams {
+struct TileParams {
   int64_t T;
   int NC;
-  int64_t n_lr;          // rows t >= n_lr add ylr (T: none)
-  const float* ylr;      // [bh][T][128] fp32 long-range term (rows >= n_lr valid)
-  __nv_bfloat16* O;      // [bh][T][128]
+  int64_t add_lo, add_hi;  // rows add_lo <= t < add_hi of every head add `addend`
+  const float* addend;     // [bh][T][128] fp32
+  __nv_bfloat16* Out;      // [bh][T][128]
   int* status;
 };
 
-__global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
-                                                              const __grid_constant__ CUtensorMap tmK,
-                                                              const __grid_constant__ CUtensorMap tmV,
-                                                              const __grid_constant__ CUtensorMap tmS,
-                                                              const OutParams prm) {
+template <bool P4_IS_P1, bool XT, bool ST_KMAJOR>
+__global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_constant__ CUtensorMap tm1,
+                                                              const __grid_constant__ CUtensorMap tm2,
+                                                              const __grid_constant__ CUtensorMap tm3,
+                                                              const __grid_constant__ CUtensorMap tmSt,
+                                                              const TileParams prm) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;                    // 2 boxes (K-major, k-blocks 0 and 1)
-  uint8_t* sK = smem + 2 * BOX_BYTES;    // 2 boxes; reused for P
-  uint8_t* sV = smem + 4 * BOX_BYTES;    // 1 box (MN-major)
-  uint8_t* sS = smem + 5 * BOX_BYTES;    // 1 box (MN-major)
+  uint8_t* s1 = smem;                    // P1: 2 boxes (K-major, k-blocks 0 and 1)
+  uint8_t* s2 = smem + 2 * BOX_BYTES;    // P2: 2 boxes
+  uint8_t* s3 = smem + 4 * BOX_BYTES;    // P3 half: 1 box (MN-major B)
+  uint8_t* sS = smem + 5 * BOX_BYTES;    // state half: 1 box
+  uint8_t* s4 = P4_IS_P1 ? s1 : s2;      // A operand of the state product
+  uint8_t* sX = P4_IS_P1 ? s2 : s1;      // the masked scores replace the other score operand
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 6 * BOX_BYTES);
   uint64_t* bar_qk = bars + 0;
   uint64_t* bar_vs = bars + 1;
   uint64_t* bar_sc = bars + 2;   // scores in TMEM
-  uint64_t* bar_p = bars + 3;    // P in shared memory (128 arrivals)
+  uint64_t* bar_p = bars + 3;    // X in shared memory (128 arrivals)
   uint64_t* bar_o = bars + 4;    // output in TMEM
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -208,23 +223,30 @@ __global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_const
 
   if (warp == 4 && lane == 0) {
     mbar_expect_tx(bar_qk, 4 * BOX_BYTES);
-    tma_load_2d(sQ, &tmQ, 0, (int)row0, bar_qk);
-    tma_load_2d(sQ + BOX_BYTES, &tmQ, HALF, (int)row0, bar_qk);
-    tma_load_2d(sK, &tmK, 0, (int)row0, bar_qk);
-    tma_load_2d(sK + BOX_BYTES, &tmK, HALF, (int)row0, bar_qk);
+    tma_load_2d(s1, &tm1, 0, (int)row0, bar_qk);
+    tma_load_2d(s1 + BOX_BYTES, &tm1, HALF, (int)row0, bar_qk);
+    tma_load_2d(s2, &tm2, 0, (int)row0, bar_qk);
+    tma_load_2d(s2 + BOX_BYTES, &tm2, HALF, (int)row0, bar_qk);
     mbar_expect_tx(bar_vs, 2 * BOX_BYTES);
-    tma_load_2d(sV, &tmV, half * HALF, (int)row0, bar_vs);
-    tma_load_2d(sS, &tmS, half * HALF, (int)(((int64_t)bh * prm.NC + b) * TILE), bar_vs);
+    tma_load_2d(s3, &tm3, half * HALF, (int)row0, bar_vs);
+    const int srow = (int)(((int64_t)bh * prm.NC + b) * TILE);
+    if (ST_KMAJOR) {  // rows half*64 .. +63 of the state (the output columns), all 128 columns: two 64 x 64 boxes
+      tma_load_2d(sS, &tmSt, 0, srow + half * HALF, bar_vs);
+      tma_load_2d(sS + BOX_BYTES / 2, &tmSt, HALF, srow + half * HALF, bar_vs);
+    } else {          // columns half*64 .. +63 of the state, all 128 rows
+      tma_load_2d(sS, &tmSt, half * HALF, srow, bar_vs);
+    }
 
     constexpr uint32_t idesc_sc = make_idesc(TILE, TILE, 0, 0);
-    constexpr uint32_t idesc_o = make_idesc(TILE, HALF, 0, 1);
+    constexpr uint32_t idesc_st = make_idesc(TILE, HALF, 0, ST_KMAJOR ? 0 : 1);
+    constexpr uint32_t idesc_x = make_idesc(TILE, HALF, XT ? 1 : 0, 1);
     bool ok = mbar_wait(bar_qk, 0, wc);
     if (ok) {
       fence_after_sync();
 #pragma unroll
       for (int kk = 0; kk < TILE / 16; ++kk) {  // k-block kk/4 (16 KB apart), 32 bytes per 16 k-elements inside it
-        const uint64_t dA = make_desc(smem_u32(sQ) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-        const uint64_t dB = make_desc(smem_u32(sK) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dA = make_desc(smem_u32(s1) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = make_desc(smem_u32(s2) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
         mma_bf16(tmem_sc, dA, dB, idesc_sc, kk != 0);
       }
       mma_commit(bar_sc);
@@ -234,9 +256,10 @@ __global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_const
       fence_after_sync();
 #pragma unroll
       for (int kk = 0; kk < TILE / 16; ++kk) {
-        const uint64_t dA = make_desc(smem_u32(sQ) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-        const uint64_t dB = make_desc(smem_u32(sS) + kk * 2048, BOX_BYTES, 1024);
-        mma_bf16(tmem_o, dA, dB, idesc_o, kk != 0);
+        const uint64_t dA = make_desc(smem_u32(s4) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = ST_KMAJOR ? make_desc(smem_u32(sS) + (kk >> 2) * (BOX_BYTES / 2) + (kk & 3) * 32, 16, 1024)
+                                      : make_desc(smem_u32(sS) + kk * 2048, BOX_BYTES, 1024);
+        mma_bf16(tmem_o, dA, dB, idesc_st, kk != 0);
       }
       ok = mbar_wait(bar_p, 0, wc);
     }
@@ -244,14 +267,17 @@ __global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_const
       fence_after_sync();
 #pragma unroll
       for (int kk = 0; kk < TILE / 16; ++kk) {
-        const uint64_t dA = make_desc(smem_u32(sK) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-        const uint64_t dB = make_desc(smem_u32(sV) + kk * 2048, BOX_BYTES, 1024);
-        mma_bf16(tmem_o, dA, dB, idesc_o, 1);
+        // X is stored [row m][key k], two 64-key blocks.  As it is: K-major A (reduce over keys).  Transposed:
+        // MN-major A (rows = reduction index m, 64-key blocks 16 KB apart, 16 rows = 2048 bytes per step).
+        const uint64_t dA = XT ? make_desc(smem_u32(sX) + kk * 2048, BOX_BYTES, 1024)
+                               : make_desc(smem_u32(sX) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = make_desc(smem_u32(s3) + kk * 2048, BOX_BYTES, 1024);
+        mma_bf16(tmem_o, dA, dB, idesc_x, 1);
       }
       mma_commit(bar_o);
     }
   } else if (warp < 4) {
-    const int m = warp * 32 + lane;  // query row inside the tile = TMEM lane
+    const int m = warp * 32 + lane;  // row inside the tile = TMEM lane
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     if (mbar_wait(bar_sc, 0, wc)) {
       fence_after_sync();
@@ -271,7 +297,7 @@ __global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_const
             pk[h2] = pack_bf16(lo, hi);
           }
           const int j8 = cb * 4 + i;  // chunk index along the key dimension, 0..15
-          uint8_t* dst = sK + (j8 >> 3) * BOX_BYTES + m * 128 + (((j8 & 7) ^ (m & 7)) << 4);
+          uint8_t* dst = sX + (j8 >> 3) * BOX_BYTES + m * 128 + (((j8 & 7) ^ (m & 7)) << 4);
           *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
       }
@@ -281,9 +307,9 @@ __global__ void __launch_bounds__(160) chunk_output_tc_kernel(const __grid_const
       if (mbar_wait(bar_o, 0, wc)) {
         fence_after_sync();
         const int64_t t = (int64_t)b * TILE + m;
-        const bool add_lr = t >= prm.n_lr;
-        const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
-        uint4* dst = reinterpret_cast<uint4*>(prm.O + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+        const bool add_lr = t >= prm.add_lo && t < prm.add_hi;
+        const float4* y4 = reinterpret_cast<const float4*>(prm.addend + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+        uint4* dst = reinterpret_cast<uint4*>(prm.Out + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
 #pragma unroll
         for (int cb = 0; cb < 2; ++cb) {
           uint32_t v[32];
@@ -645,10 +671,12 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
 constexpr int READ_SMEM = 4 * BOX_BYTES + 1024 + 256;
 
 struct ReadParams {
-  int64_t T, n, B;       // tokens per head, first recent token, number of types
-  int64_t items;         // heads * B
-  const __nv_bfloat16* Q;
-  float* ylr;            // [bh][T][128]
+  int64_t T;             // tokens per head
+  SmatGroupSpec grp;     // which tokens share a state: types (recent tokens) or profiles (distant tokens)
+  int64_t groups;        // states per head
+  int64_t items;         // heads * groups
+  const __nv_bfloat16* X;  // [bh][T][128] rows contracted against the state
+  float* out;            // [bh][T][128]
   int* status;
 };
 
@@ -656,6 +684,9 @@ __device__ __forceinline__ void cp_async16_tc(uint32_t smem_addr, const void* gm
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gmem) : "memory");
 }
 
+// TRANS = 0: out[t][j] = Σ_i x_t[i] St[i][j]  (state as MN-major B);  TRANS = 1: out[t][i] = Σ_j x_t[j] St[i][j]
+// (the same two boxes read as a K-major B).
+template <int TRANS>
 __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constant__ CUtensorMap tmU,
                                                             const ReadParams prm) {
   extern __shared__ uint8_t smem_raw[];
@@ -682,16 +713,14 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_d = *tmem_slot;
-  const int64_t m_recent = prm.T - prm.n;
   uint32_t n_item = 0, n_pass = 0;  // completed uses of bar_u and of bar_a / bar_d / bar_e
-  constexpr uint32_t idesc = make_idesc(TILE, TILE, 0, 1);
+  constexpr uint32_t idesc = make_idesc(TILE, TILE, 0, TRANS ? 0 : 1);
 
   for (int64_t item = blockIdx.x; item < prm.items; item += gridDim.x) {
-    const int64_t bh = item / prm.B, h = item - bh * prm.B;
-    const int64_t i0 = h ? h : prm.B;                            // first recent index (1-based) of this type
-    const int64_t cnt = i0 <= m_recent ? (m_recent - i0) / prm.B + 1 : 0;
+    const int64_t bh = item / prm.groups, h = item - bh * prm.groups;
+    int64_t t_first, t_stride, cnt;
+    smat_group_tokens(prm.grp, h, &t_first, &t_stride, &cnt);
     if (cnt == 0) continue;
-    const int64_t t_first = prm.n + i0 - 1;
     bool ok = true;
     if (warp == 4 && lane == 0) {
       mbar_expect_tx(bar_u, 2 * BOX_BYTES);
@@ -706,7 +735,7 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
         const uint32_t a_base = smem_u32(sA);
         for (int idx = tid; idx < kn * 16; idx += 128) {
           const int m = idx >> 4, gc = idx & 15;
-          const __nv_bfloat16* src = prm.Q + ((bh * prm.T + t_first + (k0 + m) * prm.B) * TILE + gc * 8);
+          const __nv_bfloat16* src = prm.X + ((bh * prm.T + t_first + (k0 + m) * t_stride) * TILE + gc * 8);
           cp_async16_tc(a_base + (gc >> 3) * BOX_BYTES + m * 128 + (((gc & 7) ^ (m & 7)) << 4), src);
         }
         asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
@@ -716,7 +745,7 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
         if (ok) {
           fence_after_sync();
           const int m = warp * 32 + lane;
-          float4* dst = reinterpret_cast<float4*>(prm.ylr + (bh * prm.T + t_first + (k0 + m) * prm.B) * TILE);
+          float4* dst = reinterpret_cast<float4*>(prm.out + (bh * prm.T + t_first + (k0 + m) * t_stride) * TILE);
 #pragma unroll
           for (int cb = 0; cb < 4; ++cb) {
             uint32_t v[32];
@@ -742,7 +771,8 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
 #pragma unroll
           for (int kk = 0; kk < TILE / 16; ++kk) {
             const uint64_t dA = make_desc(smem_u32(sA) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-            const uint64_t dB = make_desc(smem_u32(sB) + kk * 2048, BOX_BYTES, 1024);
+            const uint64_t dB = TRANS ? make_desc(smem_u32(sB) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024)
+                                      : make_desc(smem_u32(sB) + kk * 2048, BOX_BYTES, 1024);
             mma_bf16(tmem_d, dA, dB, idesc, kk != 0);
           }
           mma_commit(bar_d);
@@ -774,11 +804,13 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
 // operand), else fp32.
 // ---------------------------------------------------------------------------------------------------------------
 struct PoolParams {
-  int64_t T, n, P;
-  int64_t items;           // heads * P
-  const __nv_bfloat16* K;
-  const __nv_bfloat16* V;
-  void* F;                 // [bh][P][128][128] fp32 or bf16
+  int64_t T;
+  SmatGroupSpec grp;       // profiles (F = Σ k vᵀ over distant tokens) or types (Ū = Σ q dOᵀ over recent tokens)
+  int64_t groups;          // states per head
+  int64_t items;           // heads * groups
+  const __nv_bfloat16* K;  // rows giving the first state index
+  const __nv_bfloat16* V;  // rows giving the second state index
+  void* F;                 // [bh][groups][128][128] fp32 or bf16
   int* status;
 };
 
@@ -812,8 +844,9 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
   constexpr uint32_t idesc = make_idesc(TILE, TILE, 1, 1);
 
   for (int64_t item = blockIdx.x; item < prm.items; item += gridDim.x, ++n_item) {
-    const int64_t bh = item / prm.P, x = item - bh * prm.P;
-    const int64_t cnt = x < prm.n ? (prm.n - x + prm.P - 1) / prm.P : 0;
+    const int64_t bh = item / prm.groups, g = item - bh * prm.groups;
+    int64_t t_first, t_stride, cnt;
+    smat_group_tokens(prm.grp, g, &t_first, &t_stride, &cnt);
     bool ok = true;
     for (int64_t k0 = 0; k0 < cnt && ok; k0 += TOK, ++n_pass) {
       const int kn = (int)((cnt - k0) < TOK ? (cnt - k0) : TOK);
@@ -827,7 +860,7 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
             const int k = idx >> 5, w = idx & 31, gc = w & 15;
             const uint32_t dst = (w < 16 ? a_base : b_base) + (gc >> 3) * (TOK * 128) + k * 128 + (((gc & 7) ^ (k & 7)) << 4);
             if (k < kn) {
-              const __nv_bfloat16* src = (w < 16 ? prm.K : prm.V) + ((bh * prm.T + x + (k0 + k) * prm.P) * TILE + gc * 8);
+              const __nv_bfloat16* src = (w < 16 ? prm.K : prm.V) + ((bh * prm.T + t_first + (k0 + k) * t_stride) * TILE + gc * 8);
               cp_async16_tc(dst, src);
             } else {
               asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
@@ -913,13 +946,13 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 matrix [rows, 128] row-major, box = 64 columns x 128 rows, 128-byte swizzle
-bool make_map(CUtensorMap* map, const void* base, uint64_t rows) {
+// bf16 matrix [rows, 128] row-major, box = 64 columns x box_rows rows, 128-byte swizzle
+bool make_map(CUtensorMap* map, const void* base, uint64_t rows, int box_rows = TILE) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)TILE, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)TILE * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)HALF, (cuuint32_t)TILE};
+  const cuuint32_t box[2] = {(cuuint32_t)HALF, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -931,13 +964,14 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t rows) {
 bool smat_tc_available() { return encode_fn() != nullptr; }
 
 cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf16, int64_t T, int bh, int64_t n,
-                                      int through, int* status, cudaStream_t st) {
+                                      int through, int reverse, int* status, cudaStream_t st) {
   CUtensorMap tmK, tmV;
   if (!make_map(&tmK, K, (uint64_t)bh * T) || !make_map(&tmV, V, (uint64_t)bh * T)) return cudaErrorInvalidValue;
   ScanParams prm;
   prm.T = T; prm.NC = (int)(T / TILE);
   prm.Sin = static_cast<__nv_bfloat16*>(Sin_bf16);
   prm.status = status;
+  prm.reverse = reverse;
   int blocks;
   if (through) {  // d = 1: the single state U_0 = F_0 is the carry across the boundary
     blocks = 1; prm.lo[0] = 0; prm.hi[0] = prm.NC; prm.lo[1] = prm.hi[1] = 0;
@@ -951,42 +985,70 @@ cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf
   return cudaGetLastError();
 }
 
-cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
-                                        const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,
-                                        cudaStream_t st) {
-  CUtensorMap tmQ, tmK, tmV, tmS;
+template <bool P4_IS_P1, bool XT, bool ST_KMAJOR>
+static cudaError_t launch_tile_product(const void* P1, const void* P2, const void* P3, const void* St_bf16,
+                                       const float* addend, int64_t add_lo, int64_t add_hi, void* Out, int64_t T,
+                                       int bh, int* status, cudaStream_t st) {
+  CUtensorMap tm1, tm2, tm3, tmS;
   const int NC = (int)(T / TILE);
-  if (!make_map(&tmQ, Q, (uint64_t)bh * T) || !make_map(&tmK, K, (uint64_t)bh * T) ||
-      !make_map(&tmV, V, (uint64_t)bh * T) || !make_map(&tmS, Sin_bf16, (uint64_t)bh * NC * TILE))
+  if (!make_map(&tm1, P1, (uint64_t)bh * T) || !make_map(&tm2, P2, (uint64_t)bh * T) ||
+      !make_map(&tm3, P3, (uint64_t)bh * T) || !make_map(&tmS, St_bf16, (uint64_t)bh * NC * TILE, ST_KMAJOR ? HALF : TILE))
     return cudaErrorInvalidValue;
-  OutParams prm;
-  prm.T = T; prm.NC = NC; prm.n_lr = n_lr; prm.ylr = ylr;
-  prm.O = static_cast<__nv_bfloat16*>(O);
+  TileParams prm;
+  prm.T = T; prm.NC = NC; prm.add_lo = add_lo; prm.add_hi = add_hi; prm.addend = addend;
+  prm.Out = static_cast<__nv_bfloat16*>(Out);
   prm.status = status;
-  cudaError_t err =
-      cudaFuncSetAttribute(chunk_output_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, OUT_SMEM);
+  cudaError_t err = cudaFuncSetAttribute(tile_product_tc_kernel<P4_IS_P1, XT, ST_KMAJOR>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, OUT_SMEM);
   if (err != cudaSuccess) return err;
   dim3 grid((unsigned)(NC * 2), (unsigned)bh);
-  chunk_output_tc_kernel<<<grid, 160, OUT_SMEM, st>>>(tmQ, tmK, tmV, tmS, prm);
+  tile_product_tc_kernel<P4_IS_P1, XT, ST_KMAJOR><<<grid, 160, OUT_SMEM, st>>>(tm1, tm2, tm3, tmS, prm);
   return cudaGetLastError();
 }
 
-cudaError_t smat_launch_state_read_tc(const void* Q, const void* U_bf16, float* ylr, int64_t T, int64_t n, int64_t B,
-                                      int bh, int* status, cudaStream_t st) {
+cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
+                                        const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,
+                                        cudaStream_t st) {
+  return launch_tile_product<true, false, false>(Q, K, V, Sin_bf16, ylr, n_lr, T, O, T, bh, status, st);
+}
+
+// The three within-chunk adjoints (which = 0: dQ, 1: dK, 2: dV).  Sin / Dbar are the per-tile bf16 states
+// (incoming state, scanned state adjoint); addend rows [add_lo, add_hi) carry the long-range contribution.
+cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K, const void* V, const void* dO,
+                                         const void* Sin_bf16, const void* Dbar_bf16, const float* addend,
+                                         int64_t add_lo, int64_t add_hi, void* Out, int64_t T, int bh, int* status,
+                                         cudaStream_t st) {
+  if (which == 0)
+    return launch_tile_product<true, false, true>(dO, V, K, Sin_bf16, addend, add_lo, add_hi, Out, T, bh, status, st);
+  if (which == 1)
+    return launch_tile_product<false, true, true>(dO, V, Q, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st);
+  return launch_tile_product<false, true, false>(Q, K, dO, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st);
+}
+
+cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, int transposed,
+                                      const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh, int* status,
+                                      cudaStream_t st) {
   CUtensorMap tmU;
-  if (!make_map(&tmU, U_bf16, (uint64_t)bh * B * TILE)) return cudaErrorInvalidValue;
+  if (!make_map(&tmU, state_bf16, (uint64_t)bh * groups * TILE)) return cudaErrorInvalidValue;
   ReadParams prm;
-  prm.T = T; prm.n = n; prm.B = B; prm.items = (int64_t)bh * B;
-  prm.Q = static_cast<const __nv_bfloat16*>(Q);
-  prm.ylr = ylr;
+  prm.T = T; prm.grp = grp; prm.groups = groups; prm.items = (int64_t)bh * groups;
+  prm.X = static_cast<const __nv_bfloat16*>(X);
+  prm.out = out;
   prm.status = status;
-  cudaError_t err = cudaFuncSetAttribute(state_read_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, READ_SMEM);
-  if (err != cudaSuccess) return err;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int64_t grid = prm.items < 3LL * sms ? prm.items : 3LL * sms;
-  state_read_tc_kernel<<<(unsigned)grid, 160, READ_SMEM, st>>>(tmU, prm);
+  cudaError_t err;
+  if (transposed) {
+    err = cudaFuncSetAttribute(state_read_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, READ_SMEM);
+    if (err != cudaSuccess) return err;
+    state_read_tc_kernel<1><<<(unsigned)grid, 160, READ_SMEM, st>>>(tmU, prm);
+  } else {
+    err = cudaFuncSetAttribute(state_read_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, READ_SMEM);
+    if (err != cudaSuccess) return err;
+    state_read_tc_kernel<0><<<(unsigned)grid, 160, READ_SMEM, st>>>(tmU, prm);
+  }
   return cudaGetLastError();
 }
 
@@ -1003,16 +1065,15 @@ static cudaError_t launch_pool_tc(const PoolParams& prm, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, int64_t T, int64_t n, int64_t P,
-                                int bh, int* status, cudaStream_t st) {
+cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, const SmatGroupSpec& grp,
+                                int64_t groups, int64_t max_tokens, int64_t T, int bh, int* status, cudaStream_t st) {
   PoolParams prm;
-  prm.T = T; prm.n = n; prm.P = P; prm.items = (int64_t)bh * P;
+  prm.T = T; prm.grp = grp; prm.groups = groups; prm.items = (int64_t)bh * groups;
   prm.K = static_cast<const __nv_bfloat16*>(K);
   prm.V = static_cast<const __nv_bfloat16*>(V);
   prm.F = F;
   prm.status = status;
-  const int64_t max_cnt = (n + P - 1) / P;
-  if (max_cnt <= 32) return out_bf16 ? launch_pool_tc<32, 1>(prm, st) : launch_pool_tc<32, 0>(prm, st);
+  if (max_tokens <= 32) return out_bf16 ? launch_pool_tc<32, 1>(prm, st) : launch_pool_tc<32, 0>(prm, st);
   return out_bf16 ? launch_pool_tc<128, 1>(prm, st) : launch_pool_tc<128, 0>(prm, st);
 }
 

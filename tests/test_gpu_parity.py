@@ -150,6 +150,27 @@ def test_two_level_and_per_tile_causal_branches_agree(d, T, q):
     assert rel_err(to_numpy64(a), to_numpy64(b)) <= 1e-2
 
 
+@pytest.mark.parametrize("d,T,q", [(1, 2048, 0), (2, 4096, 0), (3, 4096, 0), (3, 2560, 0), (4, 4096, 0), (2, 1024, 0)])
+def test_tensor_core_backward_matches_oracle_and_alu_path(d, T, q):
+    """smat_backward on the tcgen05 path against sampled oracle gradients and against the fp32-ALU path."""
+    w = _small("tcb", d, T, 128, 128, 128, "bf16", heads=2, seed=61, recipe="normalised")
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    tc_plan, alu_plan = _plan(w, q), _plan(w, q, flags=binding.FLAG_SIMT_ONLY)
+    assert tc_plan.uses_tensor_cores()
+    got = tc_plan.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+    tc_plan.check_status()
+    ref_alu = alu_plan.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+    geo = so.geometry(T, 128, d, q or None)
+    rows = sample_tokens(geo, 48, seed=9)
+    Q64, K64, V64, G64 = (synth.as_float64(w, host[x][1]) for x in ("q", "k", "v", "do"))
+    rq = so.dq_rows(Q64, K64, V64, G64, geo, rows)
+    rk, rv = so.dkdv_cols(Q64, K64, V64, G64, geo, rows)
+    for name, g, a, r in (("dQ", got[0], ref_alu[0], rq), ("dK", got[1], ref_alu[1], rk), ("dV", got[2], ref_alu[2], rv)):
+        e = rel_err(to_numpy64(g[0, 1][rows]), r)
+        assert e <= TOL["bf16"], (name, e)
+        assert rel_err(to_numpy64(g), to_numpy64(a)) <= 2e-2, name
+
+
 def test_chunk_size_invariance_on_device():
     outs = []
     for c in (16, 32, 64, 128):
