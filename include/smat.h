@@ -57,6 +57,9 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
 /* plan flags */
 #define SMAT_FLAG_SIMT_ONLY 1u      /* never use the tensor-core kernels (bf16 plans run the fp32-ALU path) */
 #define SMAT_FLAG_ALG2_TABULATION 2u /* tabulate with the direct double loop of Algorithm 2 instead of the staged sums */
+#define SMAT_FLAG_KEEP_FORWARD_TABLES 8u /* smat_backward does not rebuild the profile and type tables F, U: the caller
+                                            promises that `workspace` still holds what smat_forward wrote for the same
+                                            K, V with this plan (no other call on that workspace in between) */
 #define SMAT_FLAG_PER_TILE_STATES 4u /* tensor-core causal branch: store one incoming state per 128-token tile (scan, then
                                         independent tiles) instead of one per segment of tiles (two-level form) */
 
@@ -111,7 +114,9 @@ smat_status smat_forward(const smat_plan* plan, const void* Q, const void* K, co
 /*
  * Backward pass (chunking proof, "Backward Pass"): given dO = ∂L/∂O writes dQ, dK, dV (plan dtype).
  * It rebuilds the forward tables it needs (S_in, F, U) inside the workspace, so it does not
- * depend on an earlier smat_forward call.  Asynchronous on `cuda_stream`.
+ * depend on an earlier smat_forward call — unless the plan was created with SMAT_FLAG_KEEP_FORWARD_TABLES
+ * (tensor-core plans only), in which case F and U are taken from the workspace as the preceding smat_forward
+ * left them.  Asynchronous on `cuda_stream`.
  */
 smat_status smat_backward(const smat_plan* plan, const void* Q, const void* K, const void* V, const void* dO, void* dQ,
                           void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream);

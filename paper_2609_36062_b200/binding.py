@@ -19,6 +19,7 @@ SMAT_F32, SMAT_BF16 = 0, 1
 FLAG_SIMT_ONLY = 1
 FLAG_ALG2_TABULATION = 2
 FLAG_PER_TILE_STATES = 4
+FLAG_KEEP_FORWARD_TABLES = 8
 
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",

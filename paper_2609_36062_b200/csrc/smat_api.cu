@@ -423,7 +423,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
     return SMAT_ERR_ALIGN;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
-  pl->last_was_forward = false;
+  pl->last_was_forward = (pl->tc && (pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES)) ? pl->last_was_forward : false;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   const bool lr = !pl->geo.dense_G;
   if (pl->tc) {
@@ -436,13 +436,15 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
     const int64_t n = pl->geo.n;
     const bool fbar_bf16 = pl->u_bf16 && pl->geo.D <= 2;  // F̄ readable by the tensor-core read (d = 2, 3)
     if (lr) {
-      if (pl->pool_tc)
-        SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, profs, pl->geo.P,
-                                                    max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh, status,
-                                                    cx.st));
-      else
-        outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
-      tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
+      if (!(pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES)) {
+        if (pl->pool_tc)
+          SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, profs, pl->geo.P,
+                                                      max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh, status,
+                                                      cx.st));
+        else
+          outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
+        tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
+      }
       // Ū_h = Σ q dOᵀ over the type (Eq. "lr-adjoint"), then F̄ = Cᵀ Ū
       const bool ubar_tc = pl->geo.m / pl->geo.B >= 12;
       const bool ubar_bf16 = ubar_tc && pl->geo.D == 1 && fbar_bf16;  // d = 2: F̄ is Ū itself

@@ -819,9 +819,12 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
   constexpr int OP_BYTES = 2 * TOK * 128;  // one operand: two 64-feature blocks of TOK rows x 128 bytes
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  constexpr int STAGE_LD = TILE + 4;                                     // floats per staging row (padded)
+  constexpr int STAGE_BYTES = OUT_BF16 ? 0 : TILE * STAGE_LD * 4;
   uint8_t* sA = smem;
   uint8_t* sB = smem + OP_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * OP_BYTES);
+  float* stage = reinterpret_cast<float*>(smem + 2 * OP_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * OP_BYTES + STAGE_BYTES);
   uint64_t* bar_a = bars + 0;   // operands landed (128 arrivals)
   uint64_t* bar_d = bars + 1;   // MMAs of the pass finished
   uint64_t* bar_e = bars + 2;   // state read out of TMEM (4 arrivals)
@@ -887,15 +890,15 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
     if (!ok) break;
     if (warp < 4) {
       const int i = warp * 32 + lane;  // state row = TMEM lane
-      if (cnt > 0) {
-        ok = mbar_wait(bar_d, (n_pass - 1) & 1, wc);
-        if (!ok) break;
-        fence_after_sync();
-      }
+      bool ok_e = true;
+      if (cnt > 0) ok_e = mbar_wait(bar_d, (n_pass - 1) & 1, wc);
+      ok_e = __all_sync(0xffffffffu, ok_e);
+      if (!ok_e && OUT_BF16) break;
+      if (ok_e) fence_after_sync();
 #pragma unroll
       for (int cb = 0; cb < 4; ++cb) {
         uint32_t v[32];
-        if (cnt > 0) {
+        if (cnt > 0 && ok_e) {
           tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
           tmem_ld_wait();
         } else {
@@ -910,11 +913,24 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
                                  pack_bf16(__uint_as_float(v[8 * q4 + 2]), __uint_as_float(v[8 * q4 + 3])),
                                  pack_bf16(__uint_as_float(v[8 * q4 + 4]), __uint_as_float(v[8 * q4 + 5])),
                                  pack_bf16(__uint_as_float(v[8 * q4 + 6]), __uint_as_float(v[8 * q4 + 7])));
-        } else {
-          uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(prm.F) + (item * TILE + i) * TILE + cb * 32);
+        } else {  // fp32 state: through a padded staging tile so that the global writes are whole 512-byte rows
+          uint4* srow = reinterpret_cast<uint4*>(stage + i * STAGE_LD + cb * 32);
 #pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) dst[q4] = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+          for (int q4 = 0; q4 < 8; ++q4) srow[q4] = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
         }
+      }
+      if (!OUT_BF16) {
+        fence_before_sync();
+        const bool bad = bar_or_128(!ok_e);  // the four epilogue warps meet here and agree on giving up
+        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.F) + item * (int64_t)(TILE * TILE));
+        const int tid = threadIdx.x;
+#pragma unroll 4
+        for (int it = 0; it < TILE * TILE / 4 / 128; ++it) {
+          const int idx = it * 128 + tid, r = idx >> 5, c4 = idx & 31;
+          dst[idx] = *reinterpret_cast<const float4*>(stage + r * STAGE_LD + c4 * 4);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");  // staging tile free again
+        if (bad) break;
       }
       fence_before_sync();
       __syncwarp();
@@ -1054,13 +1070,14 @@ cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, flo
 
 template <int TOK, int OUT_BF16>
 static cudaError_t launch_pool_tc(const PoolParams& prm, cudaStream_t st) {
-  const int smem = 4 * TOK * 128 + 1024 + 256;
+  const int smem = 4 * TOK * 128 + (OUT_BF16 ? 0 : TILE * (TILE + 4) * 4) + 1024 + 256;
   cudaError_t err = cudaFuncSetAttribute(pool_tc_kernel<TOK, OUT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (err != cudaSuccess) return err;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int64_t grid = prm.items < 3LL * sms ? prm.items : 3LL * sms;
+  const int per_sm = smem <= 72 * 1024 ? 3 : (smem <= 110 * 1024 ? 2 : 1);
+  const int64_t grid = prm.items < (int64_t)per_sm * sms ? prm.items : (int64_t)per_sm * sms;
   pool_tc_kernel<TOK, OUT_BF16><<<(unsigned)grid, 160, smem, st>>>(prm);
   return cudaGetLastError();
 }

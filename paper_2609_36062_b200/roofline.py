@@ -63,12 +63,18 @@ def forward_work(T, c, r, p, e, geo, u_bytes=4) -> Work:
     return Work(flops, adds, by)
 
 
-def backward_work(T, c, r, p, e, geo) -> Work:
+def backward_work(T, c, r, p, e, geo, u_bytes=4, fbar_bytes=4, keep_forward_tables=False) -> Work:
+    """Tables of the backward pass: Ū (fp32) and F̄ written and read once each, U read once; F and U rebuilt
+    first (F written and read, U written) unless the forward's tables are kept in the workspace."""
     rp = r * p
     lr = geo.d > 1
-    flops = T * (c + 1) * (3 * r + 2 * p) + (15 if lr else 10) * T * rp
-    adds = (geo.nnzC * rp if lr else 0) + (T // c) * rp
-    by = (4 * r + 3 * p) * T * e + (2 * (2 * geo.P + 2 * geo.B) * rp * 4 if lr else 0)
+    rebuilt = 0 if keep_forward_tables else 2
+    flops = T * (c + 1) * (3 * r + 2 * p) + ((15 - (0 if rebuilt else 3)) if lr else 10) * T * rp
+    adds = (geo.nnzC * rp * (2 if rebuilt else 1) if lr else 0) + 2 * (T // c) * rp
+    tables = (rebuilt * geo.P * 4 + (rebuilt // 2) * geo.B * u_bytes   # F written + read, U written
+              + geo.B * u_bytes                                        # U read by the dQ typed read
+              + 2 * geo.B * 4 + 2 * geo.P * fbar_bytes) * rp           # Ū, F̄ written and read
+    by = (4 * r + 3 * p) * T * e + (tables if lr else 0)
     return Work(flops, adds, by)
 
 

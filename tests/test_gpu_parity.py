@@ -171,6 +171,20 @@ def test_tensor_core_backward_matches_oracle_and_alu_path(d, T, q):
         assert rel_err(to_numpy64(g), to_numpy64(a)) <= 2e-2, name
 
 
+def test_backward_with_kept_forward_tables_matches_rebuilding_them():
+    w = _small("keep", 3, 4096, 128, 128, 128, "bf16", heads=2, seed=71, recipe="normalised")
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    keep, rebuild = _plan(w, flags=binding.FLAG_KEEP_FORWARD_TABLES), _plan(w)
+    ws = keep.workspace(for_backward=True)
+    keep.forward(dev["q"], dev["k"], dev["v"], workspace=ws)
+    a = keep.backward(dev["q"], dev["k"], dev["v"], dev["do"], workspace=ws)
+    keep.check_status(ws)
+    b = rebuild.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+    assert keep.last_launch_count() < rebuild.last_launch_count()
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
 def test_chunk_size_invariance_on_device():
     outs = []
     for c in (16, 32, 64, 128):
