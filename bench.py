@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-from paper_2609_36062_b200 import roofline, synth  # noqa: E402
+from paper_2609_36062_b200 import replicas, roofline, synth  # noqa: E402
 
 DEFAULT_WORKLOAD = "t16k_d4"
 SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
@@ -346,10 +346,7 @@ def run_native(args):
     secs = runner.time_steps(runner.step, steps, warm, barrier)
     clocks = sampler.stop()
     secs_e2e = runner.time_steps(runner.step_e2e, max(2, steps // 4), 2, barrier) / max(2, steps // 4)
-    if world > 1:
-        tmax = torch.tensor([secs, secs_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        secs, secs_e2e = float(tmax[0]), float(tmax[1])
+    secs, secs_e2e = replicas.max_over_ranks([secs, secs_e2e], device="cuda")
     per_step = secs / steps
     value = world * w.tokens / per_step
     h2d, d2h = runner.bytes_e2e()
