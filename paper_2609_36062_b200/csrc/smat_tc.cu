@@ -344,7 +344,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
 // Two-level form of the causal branch.  Each block of the sequence is cut into segments of L tiles.
 //   segment_state_tc_kernel  : total[seg] = Σ_{tiles of the segment} K_bᵀ V_b, accumulated in TMEM (fp32), written once
 //   (scan_kernel turns the totals into the state entering each segment: exclusive prefix sum per block, fp32)
-//   segment_output_tc_kernel : one CTA per (segment, head, 64-column half) walks its L tiles with the running state
+//   segment_output_tc_kernel : one CTA per (segment, head) walks its L tiles with the running state
 //                              S in TMEM:  O_b = Q_b S + tril(Q_b K_bᵀ) V_b + Y_lr,b ;  S += K_bᵀ V_b
 // Against the per-tile form (chunk_scan + chunk_output) this writes and reads one fp32 state per segment instead of
 // one bf16 state per tile, at the price of reading K and V a second time.
@@ -436,10 +436,10 @@ __global__ void __launch_bounds__(192) segment_state_tc_kernel(const __grid_cons
   }
 }
 
-// Shared memory of segment_output_tc_kernel: two stages of (Q: 2 boxes, K: 2 boxes, V half: 1 box), the bf16 copy
-// of the running state half (1 box), the rounded score tile P (2 boxes).
-constexpr int SEG_OUT_STAGE = 5 * BOX_BYTES;
-constexpr int SEG_OUT_SMEM = 2 * SEG_OUT_STAGE + 3 * BOX_BYTES + 1024 + 256;
+// Shared memory of segment_output_tc_kernel: two stages of (Q, K, V: two boxes each) and one 32 KB tile that holds the
+// bf16 copy of the running state while O = Q S is formed and the rounded score tile P afterwards.
+constexpr int SEG_OUT_STAGE = 6 * BOX_BYTES;
+constexpr int SEG_OUT_SMEM = 2 * SEG_OUT_STAGE + 2 * BOX_BYTES + 1024 + 256;
 
 struct SegOutParams {
   int64_t T;
@@ -451,31 +451,35 @@ struct SegOutParams {
   int* status;
 };
 
+// One CTA per (segment, head), all 128 output columns.
+//   warps 0-7 : two warpgroups, each owning one 64-column half of every TMEM tile (state, scores, output)
+//   warp 8    : TMA producer (two stages);   warp 9 : MMA issuer
+// TMEM columns: running state S [0,128), scores [128,256), two output accumulators [256,384) and [384,512).
+// Per tile:  Sc = Q Kᵀ ;  O = Q S_bf16 ;  O += tril(Sc)_bf16 V ;  S += Kᵀ V.
 __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                 const __grid_constant__ CUtensorMap tmK,
                                                                 const __grid_constant__ CUtensorMap tmV,
                                                                 const SegOutParams prm) {
-  // warps 0-3: state conversion and output rows; warps 4-7: scores -> P; warp 8: TMA producer; warp 9: MMA issuer
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sS = smem + 2 * SEG_OUT_STAGE;            // bf16 state half, MN-major (rows = state row i)
-  uint8_t* sP = sS + BOX_BYTES;                      // rounded scores, K-major, two 64-key blocks
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + 2 * BOX_BYTES);
+  uint8_t* sSP = smem + 2 * SEG_OUT_STAGE;           // 128 x 128 bf16, two 64-column blocks: S_bf16, then P
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sSP + 2 * BOX_BYTES);
   uint64_t* full = bars;          // [2] tile operands landed
   uint64_t* empty = bars + 2;     // [2] tile operands consumed
-  uint64_t* bar_s = bars + 4;     // state half converted (128 arrivals)
+  uint64_t* bar_s = bars + 4;     // bf16 state written (256 arrivals)
   uint64_t* bar_sc = bars + 5;    // scores in TMEM
-  uint64_t* bar_p = bars + 6;     // P written (128 arrivals)
-  uint64_t* bar_o = bars + 7;     // output in TMEM and state updated
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  uint64_t* bar_qs = bars + 6;    // O = Q S finished: the shared tile may take P
+  uint64_t* bar_p = bars + 7;     // P written (256 arrivals)
+  uint64_t* bar_o = bars + 8;     // output in TMEM and state updated
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int half = blockIdx.x & 1, seg = blockIdx.x >> 1, bh = blockIdx.y;
+  const int seg = blockIdx.x, bh = blockIdx.y;
   const WaitCtx wc{cta_abort, prm.status};
   if (threadIdx.x == 0) {
     *cta_abort = 0;
     mbar_init(full, 1); mbar_init(full + 1, 1); mbar_init(empty, 1); mbar_init(empty + 1, 1);
-    mbar_init(bar_s, 128); mbar_init(bar_sc, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+    mbar_init(bar_s, 256); mbar_init(bar_sc, 1); mbar_init(bar_qs, 1); mbar_init(bar_p, 256); mbar_init(bar_o, 1);
     fence_barrier_init();
   }
   if (warp == 8) tmem_alloc(tmem_slot, 512);
@@ -483,8 +487,7 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // columns: running state half [0,64), scores [64,192), two output buffers [192,256) and [256,320)
-  const uint32_t tmem_s = tmem_base, tmem_sc = tmem_base + HALF, tmem_o0 = tmem_base + HALF + TILE;
+  const uint32_t tmem_s = tmem_base, tmem_sc = tmem_base + TILE, tmem_o0 = tmem_base + 2 * TILE;
   const int64_t tile0 = (int64_t)seg * prm.L;
 
   if (warp == 8 && lane == 0) {
@@ -498,39 +501,42 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
       tma_load_2d(st + BOX_BYTES, &tmQ, HALF, row, full + s);
       tma_load_2d(st + 2 * BOX_BYTES, &tmK, 0, row, full + s);
       tma_load_2d(st + 3 * BOX_BYTES, &tmK, HALF, row, full + s);
-      tma_load_2d(st + 4 * BOX_BYTES, &tmV, half * HALF, row, full + s);
+      tma_load_2d(st + 4 * BOX_BYTES, &tmV, 0, row, full + s);
+      tma_load_2d(st + 5 * BOX_BYTES, &tmV, HALF, row, full + s);
     }
   } else if (warp == 9 && lane == 0) {
-    constexpr uint32_t idesc_sc = make_idesc(TILE, TILE, 0, 0);
-    constexpr uint32_t idesc_o = make_idesc(TILE, HALF, 0, 1);
-    constexpr uint32_t idesc_s = make_idesc(TILE, HALF, 1, 1);
+    constexpr uint32_t idesc_sc = make_idesc(TILE, TILE, 0, 0);   // Q Kᵀ: both K-major
+    constexpr uint32_t idesc_o = make_idesc(TILE, TILE, 0, 1);    // A K-major (Q or P), B MN-major (S or V)
+    constexpr uint32_t idesc_s = make_idesc(TILE, TILE, 1, 1);    // Kᵀ V: both MN-major
+    const uint32_t aSP = smem_u32(sSP);
     for (int it = 0; it < prm.L; ++it) {
       const int s = it & 1;
       const uint32_t sQ = smem_u32(smem + s * SEG_OUT_STAGE);
       const uint32_t sK = sQ + 2 * BOX_BYTES, sV = sQ + 4 * BOX_BYTES;
-      const uint32_t tmem_o = tmem_o0 + (it & 1) * HALF;
+      const uint32_t tmem_o = tmem_o0 + (it & 1) * TILE;
       if (!mbar_wait(full + s, (it >> 1) & 1, wc)) break;
       fence_after_sync();
 #pragma unroll
-      for (int kk = 0; kk < TILE / 16; ++kk) {   // scores Sc = Q Kᵀ (the score buffer was read out before bar_p of the last tile)
+      for (int kk = 0; kk < TILE / 16; ++kk) {   // Sc = Q Kᵀ (the score tile was read out before bar_p of the last tile)
         const uint64_t dA = make_desc(sQ + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
         const uint64_t dB = make_desc(sK + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
         mma_bf16(tmem_sc, dA, dB, idesc_sc, kk != 0);
       }
       mma_commit(bar_sc);
-      if (!mbar_wait(bar_s, it & 1, wc)) break;  // bf16 copy of the state is in shared memory
+      if (!mbar_wait(bar_s, it & 1, wc)) break;  // bf16 state in the shared tile; output buffer of tile it-2 read out
       fence_after_sync();
 #pragma unroll
       for (int kk = 0; kk < TILE / 16; ++kk) {   // O = Q S
         const uint64_t dA = make_desc(sQ + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-        const uint64_t dB = make_desc(smem_u32(sS) + kk * 2048, BOX_BYTES, 1024);
+        const uint64_t dB = make_desc(aSP + kk * 2048, BOX_BYTES, 1024);
         mma_bf16(tmem_o, dA, dB, idesc_o, kk != 0);
       }
+      mma_commit(bar_qs);
       if (!mbar_wait(bar_p, it & 1, wc)) break;
       fence_after_sync();
 #pragma unroll
       for (int kk = 0; kk < TILE / 16; ++kk) {   // O += P V
-        const uint64_t dA = make_desc(smem_u32(sP) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dA = make_desc(aSP + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
         const uint64_t dB = make_desc(sV + kk * 2048, BOX_BYTES, 1024);
         mma_bf16(tmem_o, dA, dB, idesc_o, 1);
       }
@@ -543,45 +549,77 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
       mma_commit(bar_o);
       mma_commit(empty + s);
     }
-  } else if (warp < 4) {
-    const int m = warp * 32 + lane;  // TMEM lane: state row i, and query row of the tile
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-    // writes the bf16 copy of this thread's state row (64 columns held in v0, v1) into the swizzled B tile
+  } else if (warp < 8) {
+    const int wg = warp >> 2;                        // column half owned by this warpgroup
+    const int m = (warp & 3) * 32 + lane;            // TMEM lane: state row i / query row of the tile
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t col0 = wg * HALF;
+    uint8_t* my_tile = sSP + wg * BOX_BYTES + m * 128;  // this thread's 128-byte row in its 64-column block
+    // bf16 copy of this thread's 64 state columns (v0, v1) into the shared tile
     auto publish_state = [&](const uint32_t (&v0)[32], const uint32_t (&v1)[32]) {
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         const uint32_t* v = c < 4 ? v0 : v1;
         const int o = (c & 3) * 8;
-        const uint4 pk = make_uint4(pack_bf16(__uint_as_float(v[o]), __uint_as_float(v[o + 1])),
-                                    pack_bf16(__uint_as_float(v[o + 2]), __uint_as_float(v[o + 3])),
-                                    pack_bf16(__uint_as_float(v[o + 4]), __uint_as_float(v[o + 5])),
-                                    pack_bf16(__uint_as_float(v[o + 6]), __uint_as_float(v[o + 7])));
-        *reinterpret_cast<uint4*>(sS + m * 128 + ((c ^ (m & 7)) << 4)) = pk;
+        *reinterpret_cast<uint4*>(my_tile + ((c ^ (m & 7)) << 4)) =
+            make_uint4(pack_bf16(__uint_as_float(v[o]), __uint_as_float(v[o + 1])),
+                       pack_bf16(__uint_as_float(v[o + 2]), __uint_as_float(v[o + 3])),
+                       pack_bf16(__uint_as_float(v[o + 4]), __uint_as_float(v[o + 5])),
+                       pack_bf16(__uint_as_float(v[o + 6]), __uint_as_float(v[o + 7])));
       }
       fence_proxy_async();
       fence_before_sync();
       mbar_arrive(bar_s);
     };
-    {  // state entering the segment: global fp32 -> TMEM (accumulator) and shared memory
+    {  // state entering the segment: global fp32 -> TMEM (accumulator) and the shared tile
       uint32_t v0[32], v1[32];
-      const uint4* src = reinterpret_cast<const uint4*>(prm.seg_in + (((int64_t)bh * prm.nseg + seg) * TILE + m) * TILE + half * HALF);
+      const uint4* src = reinterpret_cast<const uint4*>(prm.seg_in + (((int64_t)bh * prm.nseg + seg) * TILE + m) * TILE + col0);
 #pragma unroll
       for (int q4 = 0; q4 < 8; ++q4) {
         const uint4 a = __ldg(src + q4), b = __ldg(src + 8 + q4);
         v0[4 * q4] = a.x; v0[4 * q4 + 1] = a.y; v0[4 * q4 + 2] = a.z; v0[4 * q4 + 3] = a.w;
         v1[4 * q4] = b.x; v1[4 * q4 + 1] = b.y; v1[4 * q4 + 2] = b.z; v1[4 * q4 + 3] = b.w;
       }
-      tmem_st32(tmem_s + lane_base, v0);
-      tmem_st32(tmem_s + lane_base + 32, v1);
+      tmem_st32(tmem_s + lane_base + col0, v0);
+      tmem_st32(tmem_s + lane_base + col0 + 32, v1);
       tmem_st_wait();
       publish_state(v0, v1);
     }
     for (int it = 0; it < prm.L; ++it) {
+      // --- scores of this tile -> masked bf16 P (registers), stored once O = Q S has consumed the shared tile ---
+      if (!mbar_wait(bar_sc, it & 1, wc)) break;
+      fence_after_sync();
+      uint4 pk[8];
+#pragma unroll
+      for (int cb = 0; cb < 2; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_sc + lane_base + col0 + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint32_t w[4];
+#pragma unroll
+          for (int h2 = 0; h2 < 4; ++h2) {
+            const int k0 = (int)col0 + cb * 32 + i * 8 + h2 * 2;
+            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
+            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            w[h2] = pack_bf16(lo, hi);
+          }
+          pk[cb * 4 + i] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      if (!mbar_wait(bar_qs, it & 1, wc)) break;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(my_tile + ((c ^ (m & 7)) << 4)) = pk[c];
+      fence_proxy_async();
+      fence_before_sync();
+      mbar_arrive(bar_p);
+      // --- long-range rows of this tile, fetched while the MMAs run ---
       const int64_t t = (tile0 + it) * TILE + m;
       const bool add_lr = t >= prm.n_lr;
-      float4 y[16];  // long-range term of this row, fetched before the wait
+      float4 y[16];
       if (add_lr) {
-        const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+        const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + col0);
 #pragma unroll
         for (int i = 0; i < 16; ++i) y[i] = __ldg(y4 + i);
       }
@@ -589,17 +627,17 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
       fence_after_sync();
       if (it + 1 < prm.L) {  // the state now includes this tile: publish it for the next one first (critical path)
         uint32_t v0[32], v1[32];
-        tmem_ld32(tmem_s + lane_base, v0);
-        tmem_ld32(tmem_s + lane_base + 32, v1);
+        tmem_ld32(tmem_s + lane_base + col0, v0);
+        tmem_ld32(tmem_s + lane_base + col0 + 32, v1);
         tmem_ld_wait();
         publish_state(v0, v1);
       }
-      uint4* dst = reinterpret_cast<uint4*>(prm.O + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
-      const uint32_t tmem_o = tmem_o0 + (it & 1) * HALF;
+      uint4* dst = reinterpret_cast<uint4*>(prm.O + ((int64_t)bh * prm.T + t) * TILE + col0);
+      const uint32_t tmem_o = tmem_o0 + (it & 1) * TILE;
 #pragma unroll
       for (int cb = 0; cb < 2; ++cb) {
         uint32_t v[32];
-        tmem_ld32(tmem_o + lane_base + cb * 32, v);
+        tmem_ld32(tmem_o + lane_base + col0 + cb * 32, v);
         tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -615,40 +653,6 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
                                        pack_bf16(f[6], f[7]));
         }
       }
-    }
-  } else if (warp < 8) {
-    const int m = (warp - 4) * 32 + lane;  // query row of the tile = TMEM lane
-    const uint32_t lane_base = (uint32_t)((warp - 4) * 32) << 16;
-    for (int it = 0; it < prm.L; ++it) {
-      if (!mbar_wait(bar_sc, it & 1, wc)) break;
-      fence_after_sync();
-      uint4 pk[16];  // the masked, rounded score row: sixteen 16-byte chunks of 8 keys
-#pragma unroll
-      for (int cb = 0; cb < 4; ++cb) {
-        uint32_t v[32];
-        tmem_ld32(tmem_sc + lane_base + cb * 32, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint32_t w[4];
-#pragma unroll
-          for (int h2 = 0; h2 < 4; ++h2) {
-            const int k0 = cb * 32 + i * 8 + h2 * 2;
-            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
-            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
-            w[h2] = pack_bf16(lo, hi);
-          }
-          pk[cb * 4 + i] = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-      }
-      // P of the previous tile must have been consumed (its MMA is covered by bar_o of that tile)
-      if (it > 0 && !mbar_wait(bar_o, (it - 1) & 1, wc)) break;
-#pragma unroll
-      for (int j8 = 0; j8 < 16; ++j8)
-        *reinterpret_cast<uint4*>(sP + (j8 >> 3) * BOX_BYTES + m * 128 + (((j8 & 7) ^ (m & 7)) << 4)) = pk[j8];
-      fence_proxy_async();
-      fence_before_sync();
-      mbar_arrive(bar_p);
     }
   }
   fence_before_sync();
@@ -1098,7 +1102,7 @@ cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_b
 int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh) {
   for (int L = 16; L >= 2; L >>= 1) {
     if (tiles_block0 % L || (tiles_block1 && tiles_block1 % L)) continue;
-    const int64_t ctas = (tiles_block0 + tiles_block1) / L * 2 * bh;
+    const int64_t ctas = (tiles_block0 + tiles_block1) / L * bh;
     if (ctas >= 296 || L == 2) return L;
   }
   return 1;
@@ -1132,7 +1136,7 @@ cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const vo
   cudaError_t err =
       cudaFuncSetAttribute(segment_output_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_OUT_SMEM);
   if (err != cudaSuccess) return err;
-  dim3 grid((unsigned)(prm.nseg * 2), (unsigned)bh);
+  dim3 grid((unsigned)prm.nseg, (unsigned)bh);
   segment_output_tc_kernel<<<grid, 320, SEG_OUT_SMEM, st>>>(tmQ, tmK, tmV, prm);
   return cudaGetLastError();
 }
