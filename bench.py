@@ -267,23 +267,26 @@ class Runner:
         return [(n, acc[n] / steps) for n in order]
 
 
-def path_report(w, geo, seconds_per_step, peaks, u_bytes=4):
-    """Fractions against the path roofline.  The bytes are those of the design that ran: where the type table is
-    kept as bf16 (u_bytes = 2) its round trip is charged at 2 bytes per entry, and the fraction against the
-    roofline with fp32 tables is given beside it."""
+def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4):
+    """Fractions against the path roofline.  The bytes are those of the design that ran: where a table is kept as
+    bf16 its round trip is charged at 2 bytes per entry, and the fraction against the roofline with fp32 tables is
+    given beside it."""
     e = 4 if w.dtype == "f32" else 2
-    def total(ub):
-        wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub)
-        if w.backward:  # bench.py's fwd+bwd step keeps the forward's tables; F̄ is bf16 where U is (d <= 3)
-            fb = 2 if (ub == 2 and geo.d <= 3) else 4
-            wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub, fb, keep_forward_tables=True)
+    def total(ub, fb):
+        wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub, fb)
+        if w.backward:  # bench.py's fwd+bwd step keeps the forward's tables; the adjoint tables follow the forward's
+            fbar = 2 if (fb == 2 or (ub == 2 and geo.d <= 3)) else 4
+            ubar = 2 if (fb == 2 and geo.d >= 3) or (ub == 2 and geo.d == 2) else 4
+            wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub, fbar, keep_forward_tables=True,
+                                             f_bytes=fb, ubar_bytes=ubar)
         return wk.scaled(w.bh)
-    work = total(u_bytes)
+    work = total(u_bytes, f_bytes)
     t = roofline.roofline_times(work, peaks)
-    t32 = roofline.roofline_times(total(4), peaks)
+    t32 = roofline.roofline_times(total(4, 4), peaks)
     return {
         "frac_2term": t["t_2term"] / seconds_per_step, "frac_3term": t["t_3term"] / seconds_per_step,
         "frac_2term_fp32_tables": t32["t_2term"] / seconds_per_step, "type_table_bytes_per_entry": u_bytes,
+        "profile_table_bytes_per_entry": f_bytes,
         "roofline_ms_2term": 1e3 * t["t_2term"], "roofline_ms_3term": 1e3 * t["t_3term"],
         "t_tensor_ms": 1e3 * t["t_tensor"], "t_alu_ms": 1e3 * t["t_alu"], "t_hbm_ms": 1e3 * t["t_hbm"],
         "algorithmic": {"tensor_flop": work.flops, "alu_adds": work.adds, "hbm_bytes": work.bytes},
@@ -291,27 +294,26 @@ def path_report(w, geo, seconds_per_step, peaks, u_bytes=4):
     }
 
 
-def dominant_kernel_report(w, geo, stages, peaks, u_bytes=4):
+def dominant_kernel_report(w, geo, stages, peaks, u_bytes=4, f_bytes=4):
+    """Roofline of the stage that takes the longest.  Its bound is the slower of its bytes at the HBM peak and its
+    operations (contraction flop plus Algorithm 2's additions, one flop each) at the tensor peak."""
     e = 4 if w.dtype == "f32" else 2
     total = sum(t for _, t in stages)
     name, ms = max(stages, key=lambda s: s[1])
     base = name.split(":")[-1]
-    work = roofline.stage_work(base, w.T, w.chunk, w.d_k, w.d_v, e, geo, u_bytes).scaled(w.bh)
+    work = roofline.stage_work(base, w.T, w.chunk, w.d_k, w.d_v, e, geo, u_bytes, f_bytes).scaled(w.bh)
     t = roofline.roofline_times(work, peaks, sustained=True)
-    bounds = {"hbm": t["t_hbm"], "alu": t["t_alu"], "tensor": t["t_tensor"]}
-    bound = max(bounds, key=bounds.get)
+    ops = work.flops + work.adds
+    t_ops = ops / (peaks["bf16_tflops_sustained"] * 1e12)
     sec = ms / 1e3
-    if bound == "hbm":
-        achieved, peak, unit = work.bytes / sec / 1e9, peaks["hbm_gbs"], "GB/s"
-    elif bound == "alu":
-        achieved, peak, unit = work.adds / sec / 1e9, t["alu_peak_adds"] / 1e9, "Gadd/s"
+    if t["t_hbm"] >= t_ops:
+        bound, achieved, peak, unit = "hbm", work.bytes / sec / 1e9, peaks["hbm_gbs"], "GB/s"
     else:
-        achieved, peak, unit = work.flops / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
+        bound, achieved, peak, unit = "tensor", ops / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
     return {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
             "frac": achieved / peak if peak else None, "traffic": NCU_TRAFFIC_BYTES.get((w.name, base)),
-            "algorithmic_bytes": work.bytes, "algorithmic_adds": work.adds,
-            "ms": ms, "share": ms / total if total else None,
-            "peak_source": peaks["source"] + (" (fp32 add peak nominal: 148 SM x 128 lanes x max clock)" if bound == "alu" else ""),
+            "algorithmic_bytes": work.bytes, "algorithmic_ops": ops,
+            "ms": ms, "share": ms / total if total else None, "peak_source": peaks["source"],
             "kernels_ms": {n: round(t_, 4) for n, t_ in stages}}
 
 
@@ -353,7 +355,7 @@ def run_native(args):
 
     line = None
     if rank == 0:
-        ub = runner.plan.type_table_element_bytes()
+        ub, fb = runner.plan.type_table_element_bytes(), runner.plan.profile_table_element_bytes()
         stages = runner.stage_profile(min(steps, 10))
         line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warm,
@@ -364,8 +366,8 @@ def run_native(args):
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": launches * steps,
             "clocks": clocks,
-            "roofline": dominant_kernel_report(w, g, stages, peaks, ub),
-            "path_roofline": path_report(w, g, per_step, peaks, ub),
+            "roofline": dominant_kernel_report(w, g, stages, peaks, ub, fb),
+            "path_roofline": path_report(w, g, per_step, peaks, ub, fb),
             "tables": {"profile_states_P": g.P, "cached_subset_states_B": g.B, "nnzC": g.nnzC, "q": g.q},
         }
     del runner
@@ -381,7 +383,7 @@ def run_native(args):
             gg = r.plan.geometry()
             k = 5
             s = r.time_steps(r.step, k, 3) / k
-            rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes())
+            rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes(), r.plan.profile_table_element_bytes())
             st_ = r.stage_profile(3)
             sweep.append({"workload": name, "value": ws_.tokens / s, "unit": "tokens/s", "ms_per_step": 1e3 * s,
                           "frac_2term": rep["frac_2term"], "frac_3term": rep["frac_3term"],

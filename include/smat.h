@@ -63,6 +63,10 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
 #define SMAT_FLAG_PER_TILE_STATES 4u /* tensor-core causal branch: store one incoming state per 128-token tile (scan, then
                                         independent tiles) instead of one per segment of tiles (two-level form) */
 
+#define SMAT_FLAG_ALU_TABULATION 16u /* d = 3, 4 on the tensor-core path: keep the profile table in fp32 and tabulate
+                                        with staged sums on the fp32 ALUs instead of the Radon stages on the tensor cores
+                                        (which keep F, U and the stage intermediate in bf16) */
+
 /* Sizes of the construction (Sec. 3, "construction of G" and "Scaling with sequence length"). */
 typedef struct {
   int64_t T, c, n, m;  /* sequence length, chunk width, distant = c*floor(T/2c), recent = T - n */
@@ -96,8 +100,14 @@ int smat_uses_tensor_cores(const smat_plan* plan);
 /* Bytes per element of the type table U as smat_forward keeps it: 4 (fp32), or 2 when the plan runs the typed read on
  * the tensor cores (bf16 inputs; d >= 3, or d = 2 with at least 12 tokens per profile): there U is only ever a bf16
  * MMA operand, so it is rounded once when it is stored and the table's HBM traffic halves (for d = 2 the profile
- * table is the type table and is kept in bf16 too).  smat_backward always builds fp32 tables. */
+ * table is the type table and is kept in bf16 too). */
 int smat_type_table_element_bytes(const smat_plan* plan);
+
+/* Bytes per element of the profile table F as smat_forward keeps it: 2 for d = 2 on the tensor-core path and for
+ * d = 3, 4 when the tabulation (Algorithm 2) runs as Radon stages on the tensor cores — F, the stage intermediate and
+ * U are then bf16 MMA operands, sums are taken in fp32 — else 4.  On those plans smat_backward keeps the adjoint
+ * tables (the per-type sums of q dOᵀ and their transposed tabulation) in bf16 as well. */
+int smat_profile_table_element_bytes(const smat_plan* plan);
 
 /* Bytes of workspace smat_forward (for_backward = 0) or smat_backward (for_backward = 1) needs. 0 if plan is NULL. */
 size_t smat_workspace_bytes(const smat_plan* plan, int for_backward);

@@ -20,11 +20,13 @@ FLAG_SIMT_ONLY = 1
 FLAG_ALG2_TABULATION = 2
 FLAG_PER_TILE_STATES = 4
 FLAG_KEEP_FORWARD_TABLES = 8
+FLAG_ALU_TABULATION = 16
 
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
     "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
+    "smat_profile_table_element_bytes",
 ]
 
 
@@ -91,6 +93,8 @@ def load_library() -> ctypes.CDLL:
     lib.smat_last_launch_count.restype = i
     lib.smat_type_table_element_bytes.argtypes = [vp]
     lib.smat_type_table_element_bytes.restype = i
+    lib.smat_profile_table_element_bytes.argtypes = [vp]
+    lib.smat_profile_table_element_bytes.restype = i
     lib.smat_uses_tensor_cores.argtypes = [vp]
     lib.smat_uses_tensor_cores.restype = i
     lib.smat_forward_causal_static.argtypes = [vp, vp, vp, vp, i, i, i64, vp]
@@ -178,6 +182,9 @@ class SmatPlan:
 
     def type_table_element_bytes(self) -> int:
         return int(self.lib.smat_type_table_element_bytes(self.handle))
+
+    def profile_table_element_bytes(self) -> int:
+        return int(self.lib.smat_profile_table_element_bytes(self.handle))
 
     def workspace_bytes(self, for_backward: bool = False) -> int:
         return int(self.lib.smat_workspace_bytes(self.handle, int(for_backward)))

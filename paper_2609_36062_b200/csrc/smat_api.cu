@@ -20,12 +20,13 @@ struct smat_plan {
   SmatGeo geo;
   int64_t rp;          // state entries
   // workspace layout (byte offsets, 256-byte aligned)
-  size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_fwd_end;
+  size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_W, off_fwd_end;
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
   bool tc;             // tensor-core kernels for the causal branch
   bool u_bf16;         // forward keeps the type table U in bf16 and reads it with the tensor-core typed read
   bool pool_tc;        // forward pools the profile table on the tensor cores (enough tokens per profile)
-  bool f_bf16;         // d = 2 on that path: the profile table is the type table, kept in bf16
+  bool f_bf16;         // the profile table is kept in bf16 (d = 2: it is the type table; tab_tc: it is an MMA operand)
+  bool tab_tc;         // d = 3, 4: tabulation and its transpose on the tensor cores (bf16 tables, resident Radon matrix)
   mutable int launches;
   mutable bool last_was_forward;  // which call left its tables in the workspace
   // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
@@ -240,6 +241,15 @@ void tabulate(Ctx& cx, const char* name, const float* in, float* out, int transp
     SMAT_TRY(cx, name, smat_launch_tabulate_alg2(in, out, pl->geo, pl->rp, pl->bh, transpose, cx.st));
 }
 
+// The same two operations for plans whose tables are bf16: Radon stages on the tensor cores (one launch for d = 3, two for d = 4).
+void tabulate_tc(Ctx& cx, const char* name, const void* in, void* out, int transpose) {
+  const smat_plan* pl = cx.pl;
+  int launches = 1;
+  SMAT_TRY(cx, name, smat_launch_tabulate_tc(in, out, cx.ws + pl->off_W, pl->geo, pl->rp, pl->bh, transpose,
+                                             reinterpret_cast<int*>(cx.ws + pl->off_status), cx.st, &launches));
+  cx.launches += launches - 1;
+}
+
 // Steps 2-3 and 5-6 of Algorithm 1: the tables S_in, F, U.
 void build_forward_tables(Ctx& cx, const void* K, const void* V) {
   const smat_plan* pl = cx.pl;
@@ -278,8 +288,10 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
            g.m % 128 == 0 && g.n >= 128 && smat_tc_available();
   if (!g.dense_G && (smat_tabulate_alg2_slab(g.B, pl->rp) < 1)) { delete pl; return SMAT_ERR_UNSUPPORTED; }
   // d >= 3 on the tensor-core path: U is only ever a bf16 MMA operand, so it is stored as bf16 (half the bytes)
-  pl->pool_tc = pl->tc && !g.dense_G && g.n / g.P >= 12;
-  pl->f_bf16 = pl->pool_tc && g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION);
+  pl->tab_tc = pl->tc && !g.dense_G && !(flags & (SMAT_FLAG_ALG2_TABULATION | SMAT_FLAG_ALU_TABULATION)) &&
+               smat_tabulate_tc_supported(g, pl->rp);
+  pl->pool_tc = pl->tc && !g.dense_G && (g.n / g.P >= 12 || pl->tab_tc);
+  pl->f_bf16 = pl->pool_tc && ((g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION)) || pl->tab_tc);
   pl->u_bf16 = pl->f_bf16 || (pl->tc && g.D >= 2 && !(flags & SMAT_FLAG_ALG2_TABULATION) &&
                               smat_tabulate_staged_slab(g, pl->rp, 0) >= 4);
   const size_t state = (size_t)pl->rp * sizeof(float);
@@ -293,6 +305,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->off_U = off;      off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.B * state));
   pl->off_acc = off;    off = align_up(off + (size_t)pl->bh * T * wide * sizeof(float));
   pl->off_tileA = off;  off = align_up(off + (size_t)pl->bh * T * chunk * sizeof(float));
+  pl->off_W = off;      off = align_up(off + (pl->tab_tc ? (size_t)pl->bh * smat_tabulate_tc_scratch_rows(g) * pl->rp * 2 : 0));
   pl->off_fwd_end = off;
   pl->off_dbar = off;   off = align_up(off + (size_t)pl->bh * pl->NC * state);
   pl->off_ubar = off;   off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.B * state));
@@ -349,6 +362,8 @@ int smat_uses_tensor_cores(const smat_plan* pl) { return pl && pl->tc ? 1 : 0; }
 
 int smat_type_table_element_bytes(const smat_plan* pl) { return pl && pl->u_bf16 ? 2 : 4; }
 
+int smat_profile_table_element_bytes(const smat_plan* pl) { return pl && pl->f_bf16 ? 2 : 4; }
+
 size_t smat_workspace_bytes(const smat_plan* pl, int for_backward) {
   if (!pl) return 0;
   return for_backward ? pl->off_bwd_end : pl->off_fwd_end;
@@ -375,7 +390,10 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
                                                     status, cx.st));
       else
         outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
-      tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);              // step 3
+      if (pl->tab_tc)                                                                        // step 3
+        tabulate_tc(cx, "tabulate_tc", cx.ws + pl->off_F, cx.ws + pl->off_U, 0);
+      else
+        tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
       if (pl->u_bf16)                                                                        // step 4
         SMAT_TRY(cx, "read_type_tc", smat_launch_state_read_tc(Q, cx.ws + pl->off_U, ylr, 0, group(pl, SMAT_GM_TYPE),
                                                                pl->geo.B, pl->T, pl->bh, status, cx.st));
@@ -443,19 +461,25 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
                                                       cx.st));
         else
           outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
-        tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
+        if (pl->tab_tc)
+          tabulate_tc(cx, "tabulate_tc", cx.ws + pl->off_F, cx.ws + pl->off_U, 0);
+        else
+          tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
       }
       // Ū_h = Σ q dOᵀ over the type (Eq. "lr-adjoint"), then F̄ = Cᵀ Ū
-      const bool ubar_tc = pl->geo.m / pl->geo.B >= 12;
-      const bool ubar_bf16 = ubar_tc && pl->geo.D == 1 && fbar_bf16;  // d = 2: F̄ is Ū itself
+      const bool ubar_tc = pl->tab_tc || pl->geo.m / pl->geo.B >= 12;
+      const bool ubar_bf16 = ubar_tc && ((pl->geo.D == 1 && fbar_bf16) || pl->tab_tc);  // d = 2: F̄ is Ū itself
       if (ubar_tc)
         SMAT_TRY(cx, "bwd_pool_type_tc", smat_launch_pool_tc(Q, dO, cx.ws + pl->off_ubar, ubar_bf16, types, pl->geo.B,
                                                              max_group_tokens(pl, SMAT_GM_TYPE), pl->T, pl->bh,
                                                              status, cx.st));
       else
         outer_sum(cx, "bwd_pool_type", SMAT_GM_TYPE, Q, dO, cx.f(pl->off_ubar));
-      const bool fbar_is_bf16 = pl->geo.D == 1 ? ubar_bf16 : fbar_bf16;
-      tabulate(cx, "bwd_tabulate_t", cx.f(pl->off_ubar), cx.f(pl->off_fbar), 1, pl->geo.D == 2 && fbar_bf16);
+      const bool fbar_is_bf16 = pl->tab_tc || (pl->geo.D == 1 ? ubar_bf16 : fbar_bf16);
+      if (pl->tab_tc)
+        tabulate_tc(cx, "bwd_tabulate_t_tc", cx.ws + pl->off_ubar, cx.ws + pl->off_fbar, 1);
+      else
+        tabulate(cx, "bwd_tabulate_t", cx.f(pl->off_ubar), cx.f(pl->off_fbar), 1, pl->geo.D == 2 && fbar_bf16);
       // per-tile states
       SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 0, 0, status, cx.st));
       SMAT_TRY(cx, "bwd_chunk_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 0, 1, status, cx.st));

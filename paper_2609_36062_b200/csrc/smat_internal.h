@@ -110,6 +110,11 @@ cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, flo
                                       const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh, int* status,
                                       cudaStream_t st);
 // bf16 -> fp32 copy of a table (debug export).
+// Tabulation on the tensor cores (bf16 tables; d = 3, 4 with a prime small enough for a resident Radon matrix).
+int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems);
+int64_t smat_tabulate_tc_scratch_rows(const SmatGeo& geo);
+cudaError_t smat_launch_tabulate_tc(const void* in, void* out, void* scratch, const SmatGeo& geo, int64_t state_elems,
+                                    int bh, int transpose, int* status, cudaStream_t st, int* launches);
 cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st);
 // Pooling on tensor cores: F[bh][x] = Σ_{t ≡ x (mod P), t < n} k_t v_tᵀ, stored as fp32 or bf16.
 cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, const SmatGroupSpec& grp,

@@ -7,9 +7,9 @@ r = d_k, p = d_v, e = bytes per input element, fp32 tables:
                          + 2rp (T + T + n + m)      chunk summaries, carried-state read, pool, typed read
   ALU adds   (forward)   = nnz(C) rp + (T/c) rp     Algorithm 2's state additions + the scan
   HBM bytes  (forward)   = (2r + 2p) T e            Q, K, V in, O out
-                         + 2 P rp 4 + 2 B rp s_U    profile table and type table, written once and read once
-                           (d = 1 has neither table; s_U = 4, or 2 where the implementation stores U as bf16 —
-                           both variants are reported)
+                         + 2 P rp s_F + 2 B rp s_U  profile table and type table, written once and read once
+                           (d = 1 has neither table; s = 4, or 2 where the implementation stores the table as
+                           bf16 — the fraction against fp32 tables is reported beside the design's own)
   backward               = T (c+1)(3r+2p) + 15 T rp flop, the same adds again (Cᵀ tabulation, suffix scan),
                            (4r + 3p) T e bytes of tensors and 2 (2P + 2B) rp 4 bytes of tables
                            (F, U rebuilt; Ū, F̄ written and read)
@@ -53,17 +53,19 @@ class Work:
         return Work(self.flops * k, self.adds * k, self.bytes * k)
 
 
-def forward_work(T, c, r, p, e, geo, u_bytes=4) -> Work:
-    """u_bytes: element size of the type table as the implementation keeps it (4, or 2 where it is stored as bf16)."""
+def forward_work(T, c, r, p, e, geo, u_bytes=4, f_bytes=4) -> Work:
+    """u_bytes, f_bytes: element sizes of the type and profile tables as the implementation keeps them (4, or 2
+    where a table is stored as bf16)."""
     rp = r * p
     lr = geo.d > 1
     flops = T * (c + 1) * (r + p) + 2 * rp * (2 * T + (geo.n + geo.m if lr else 0))
     adds = (geo.nnzC * rp if lr else 0) + (T // c) * rp
-    by = (2 * r + 2 * p) * T * e + (2 * geo.P * rp * 4 + 2 * geo.B * rp * u_bytes if lr else 0)
+    by = (2 * r + 2 * p) * T * e + (2 * geo.P * rp * f_bytes + 2 * geo.B * rp * u_bytes if lr else 0)
     return Work(flops, adds, by)
 
 
-def backward_work(T, c, r, p, e, geo, u_bytes=4, fbar_bytes=4, keep_forward_tables=False) -> Work:
+def backward_work(T, c, r, p, e, geo, u_bytes=4, fbar_bytes=4, keep_forward_tables=False, f_bytes=4,
+                  ubar_bytes=4) -> Work:
     """Tables of the backward pass: Ū (fp32) and F̄ written and read once each, U read once; F and U rebuilt
     first (F written and read, U written) unless the forward's tables are kept in the workspace."""
     rp = r * p
@@ -71,9 +73,9 @@ def backward_work(T, c, r, p, e, geo, u_bytes=4, fbar_bytes=4, keep_forward_tabl
     rebuilt = 0 if keep_forward_tables else 2
     flops = T * (c + 1) * (3 * r + 2 * p) + ((15 - (0 if rebuilt else 3)) if lr else 10) * T * rp
     adds = (geo.nnzC * rp * (2 if rebuilt else 1) if lr else 0) + 2 * (T // c) * rp
-    tables = (rebuilt * geo.P * 4 + (rebuilt // 2) * geo.B * u_bytes   # F written + read, U written
+    tables = (rebuilt * geo.P * f_bytes + (rebuilt // 2) * geo.B * u_bytes   # F written + read, U written
               + geo.B * u_bytes                                        # U read by the dQ typed read
-              + 2 * geo.B * 4 + 2 * geo.P * fbar_bytes) * rp           # Ū, F̄ written and read
+              + 2 * geo.B * ubar_bytes + 2 * geo.P * fbar_bytes) * rp  # Ū, F̄ written and read
     by = (4 * r + 3 * p) * T * e + (tables if lr else 0)
     return Work(flops, adds, by)
 
@@ -93,15 +95,23 @@ def roofline_times(work: Work, peaks: dict, sustained: bool = True) -> dict:
 
 
 # Per-kernel algorithmic traffic (bytes), adds and flop, keyed by the stage names the library reports.
-def stage_work(name: str, T, c, r, p, e, geo, u_bytes=4) -> Work:
+def stage_work(name: str, T, c, r, p, e, geo, u_bytes=4, f_bytes=4) -> Work:
+    """What one forward stage has to do at the least: its contraction flop, Algorithm 2's additions where it
+    tabulates, and the bytes of its inputs and outputs (scratch the stage exchanges with itself is not counted)."""
     rp, NC = r * p, T // c
     n, m, P, B = geo.n, geo.m, geo.P, geo.B
     st = 4 * rp
     su = u_bytes * rp
+    sf = f_bytes * rp
     tc_tiles = T // 128
     table = {
         "pool":        Work(2 * n * rp, 0, n * (r + p) * e + P * st),
+        "pool_tc":     Work(2 * n * rp, 0, n * (r + p) * e + P * sf),
         "tabulate":    Work(0, geo.nnzC * rp, P * st + B * su),
+        "tabulate_tc": Work(0, geo.nnzC * rp, P * sf + B * su),
+        "segment_state_tc": Work(2 * T * rp, 0, T * (r + p) * e),
+        "segment_scan": Work(0, 0, 0),
+        "segment_output_tc": Work(T * 129 * (r + p) + 4 * T * rp, 0, T * (2 * r + 2 * p) * e + m * p * 4),
         "chunk_state": Work(2 * T * rp, 0, T * (r + p) * e + NC * st),
         "scan":        Work(0, NC * rp, 2 * NC * st),
         "scores":      Work(T * (c + 1) * r, 0, 2 * T * r * e + T * c * 4),
