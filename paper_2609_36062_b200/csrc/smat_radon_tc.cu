@@ -11,17 +11,20 @@
 // These are the sums of Algorithm 2 taken one coordinate pair at a time (same real numbers, different order).
 // The transposes run the same stages backwards with Rᵀ.  R is small (q <= 23) and fixed, the images are
 // independent across the r p state entries, so each stage is a product of a resident 0/1 matrix with a stream
-// of images: dense enough for the tensor cores (q of every q^2... entries of a row are nonzero, but the
-// 5th-generation tensor cores add 60 times faster than the fp32 pipes), and bound by the image traffic.
+// of images: dense enough for the tensor cores (q of every q^2 entries of a row are nonzero, and the
+// 5th-generation tensor cores multiply-add about 60 times faster than the fp32 pipes add), bound by the image
+// traffic.
 //
-// radon_tc_kernel, persistent, one CTA per SM:
-//   every thread   : builds its part of R (N_part output indices x K_pad input indices, K-major, 128-byte swizzle)
-//                    and the row tables once
-//   warps 4-7      : producers; gather the image rows (64 input indices x 128 state entries per ring slot, MN-major
-//                    A operand) with cp.async, up to LA slots in flight
-//   warp 8 lane 0  : MMA issuer, D[128 entries, N_part] += A_slot * R_slotᵀ, accumulators double-buffered in TMEM
-//   warps 0-3      : epilogue, one state entry (TMEM lane) per thread: round to bf16, transpose 32 output rows at a
-//                    time through a staging tile, store whole 256-byte rows
+// radon_tc_kernel, persistent, one CTA per SM.  An item is one image restricted to 128 consecutive state entries;
+// a CTA owns `mt` tiles of 128 output indices (its part of R) and applies them to every item it is given:
+//   every thread   : builds the CTA's part of R (128 mt output indices x K_pad input indices, K-major, 128-byte
+//                    swizzle) and the row tables once
+//   warps 8-15     : producers; each gathers the image rows of one ring slot at a time (64 input indices x 128 state
+//                    entries, MN-major B operand) with cp.async, so up to eight slots are in flight
+//   warp 16 lane 0 : MMA issuer, D_t[128 outputs, 128 entries] += R_t,slot * B_slot for each tile t; up to four
+//                    accumulator sets in flight in TMEM
+//   warps 0-7      : epilogue, one output index (TMEM lane) per thread: round 32 entries at a time to bf16 and store
+//                    them as 64 contiguous bytes of the output row
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -35,7 +38,12 @@ using namespace tc;
 
 constexpr int SLOT_ROWS = 64;                     // input indices per ring slot (four K-steps of 16)
 constexpr int SLOT_BYTES = SLOT_ROWS * 256;       // two 64-entry blocks of 64 rows x 128 bytes
-constexpr int STAGE_BYTES = 2 * 32 * 128 * 2;    // epilogue staging: two tiles of 32 output rows x 128 entries, bf16
+constexpr int TILE_ROWS = 128;                    // output indices per tile (MMA M)
+constexpr int EPI_WARPS = 8;
+constexpr int PROD_WARPS = 8;
+constexpr int MMA_WARP = EPI_WARPS + PROD_WARPS;
+constexpr int RADON_THREADS = 32 * (MMA_WARP + 1);
+constexpr int MAX_ACC = 4;                        // accumulator sets in flight: min(4, 512 / (128 mt))
 constexpr int ROW_INVALID = -1;
 constexpr int ROW_VERT = 1 << 30;                 // flag: row of the extra ("vertical") class
 
@@ -52,7 +60,7 @@ struct RadonSide {
 struct RadonParams {
   int32_t q, transpose;
   int32_t k_pad;                   // input indices rounded up to 16
-  int32_t n_part, parts;           // output indices per CTA (multiple of 32, <= 256) and CTAs sharing an image
+  int32_t mt, parts;               // tiles of 128 output indices per CTA; CTAs sharing an image
   int32_t ring;                    // ring slots
   int32_t images;
   int32_t slabs_per_head;          // rp / 128
@@ -63,6 +71,13 @@ struct RadonParams {
   __nv_bfloat16* dst;
   int* status;
 };
+
+// Lane 0 polls the barrier and the warp follows.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, const WaitCtx& w) {
+  bool ok = true;
+  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, w);
+  return __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+}
 
 __device__ __forceinline__ int side_row(const RadonSide& s, int idx, int q) {
   if (idx >= s.count) return ROW_INVALID;
@@ -76,31 +91,28 @@ __device__ __forceinline__ bool radon_entry(int q, int transpose, int n, int k) 
   return a < q ? (lo + a * hi) % q == u : hi == u;
 }
 
-__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* gmem) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gmem) : "memory");
-}
-__device__ __forceinline__ void st_zero16(uint32_t smem_addr) {
-  asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr), "r"(0u) : "memory");
+// 16-byte copy that reads `bytes` (16 or 0) from global memory and fills the rest with zeros
+__device__ __forceinline__ void cp_async16_zfill(uint32_t smem_addr, const void* gmem, int bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gmem), "r"(bytes) : "memory");
 }
 
-template <int LA>
-__global__ void __launch_bounds__(288, 1) radon_tc_kernel(const RadonParams prm) {
+__global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const RadonParams prm) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int q = prm.q;
   const int kgroups = (prm.k_pad + SLOT_ROWS - 1) / SLOT_ROWS;
-  const int r_bytes = prm.n_part * kgroups * 128;             // R part: kgroups blocks of n_part rows x 128 bytes
+  const int n_cta = prm.mt * TILE_ROWS;                         // output indices of this CTA
+  const int r_bytes = n_cta * kgroups * 128;                    // R part: [tile][64-index block][128 rows][128 bytes]
   uint8_t* sR = smem;
-  uint8_t* sRing = smem + r_bytes;                            // r_bytes is a multiple of 1024 (n_part % 32 == 0)
-  __nv_bfloat16* stage = reinterpret_cast<__nv_bfloat16*>(sRing + prm.ring * SLOT_BYTES);   // two [32][128] tiles
-  int32_t* in_tab = reinterpret_cast<int32_t*>(sRing + prm.ring * SLOT_BYTES + STAGE_BYTES);   // [kgroups*64]
-  int32_t* out_tab = in_tab + kgroups * SLOT_ROWS;                                 // [n_part]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_tab + prm.n_part);
-  uint64_t* full = bars;                    // [ring] slot filled (128 arrivals)
+  uint8_t* sRing = smem + r_bytes;
+  int32_t* in_tab = reinterpret_cast<int32_t*>(sRing + prm.ring * SLOT_BYTES);   // [kgroups*64]
+  int32_t* out_tab = in_tab + kgroups * SLOT_ROWS;                                 // [n_cta]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_tab + n_cta);
+  uint64_t* full = bars;                    // [ring] slot filled (one arrival, from the warp that filled it)
   uint64_t* empty = bars + prm.ring;        // [ring] slot consumed by the MMAs
-  uint64_t* acc_full = empty + prm.ring;    // [2] accumulator complete
-  uint64_t* acc_empty = acc_full + 2;       // [2] accumulator read out (4 arrivals)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* acc_full = empty + prm.ring;    // [MAX_ACC] accumulator set complete
+  uint64_t* acc_empty = acc_full + MAX_ACC; // [MAX_ACC] accumulator set read out (one arrival per epilogue warp)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + MAX_ACC);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const WaitCtx wc{cta_abort, prm.status};
@@ -108,15 +120,15 @@ __global__ void __launch_bounds__(288, 1) radon_tc_kernel(const RadonParams prm)
 
   if (threadIdx.x == 0) {
     *cta_abort = 0;
-    for (int s = 0; s < prm.ring; ++s) { mbar_init(full + s, 128); mbar_init(empty + s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 4); }
+    for (int s = 0; s < prm.ring; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    for (int b = 0; b < MAX_ACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, EPI_WARPS); }
     fence_barrier_init();
   }
-  if (warp == 8) tmem_alloc(tmem_slot, 512);
+  if (warp == MMA_WARP) tmem_alloc(tmem_slot, 512);
   // R part, 16 bytes (8 input indices) per store
-  for (int c = threadIdx.x; c < prm.n_part * kgroups * 8; c += blockDim.x) {
-    const int n = c % prm.n_part, kc = c / prm.n_part;       // kc: chunk of 8 input indices
-    const int nidx = part * prm.n_part + n;
+  for (int c = threadIdx.x; c < n_cta * kgroups * 8; c += blockDim.x) {
+    const int n = c % n_cta, kc = c / n_cta;                   // kc: chunk of 8 input indices
+    const int nidx = part * n_cta + n;
     uint32_t w[4] = {0u, 0u, 0u, 0u};
     if (nidx < prm.out.count) {
 #pragma unroll
@@ -125,11 +137,12 @@ __global__ void __launch_bounds__(288, 1) radon_tc_kernel(const RadonParams prm)
         if (k < prm.in.count && radon_entry(q, prm.transpose, nidx, k)) w[e >> 1] |= 0x3F80u << ((e & 1) * 16);  // bf16 1.0
       }
     }
-    uint8_t* dst = sR + (kc >> 3) * (prm.n_part * 128) + n * 128 + (((kc & 7) ^ (n & 7)) << 4);
+    const int t = n >> 7, row = n & 127;
+    uint8_t* dst = sR + ((t * kgroups + (kc >> 3)) * TILE_ROWS + row) * 128 + (((kc & 7) ^ (row & 7)) << 4);
     *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
   }
   for (int k = threadIdx.x; k < kgroups * SLOT_ROWS; k += blockDim.x) in_tab[k] = side_row(prm.in, k, q);
-  for (int n = threadIdx.x; n < prm.n_part; n += blockDim.x) out_tab[n] = side_row(prm.out, part * prm.n_part + n, q);
+  for (int n = threadIdx.x; n < n_cta; n += blockDim.x) out_tab[n] = side_row(prm.out, part * n_cta + n, q);
   for (int c = threadIdx.x; c < prm.ring * SLOT_BYTES / 16; c += blockDim.x)
     reinterpret_cast<uint4*>(sRing)[c] = make_uint4(0u, 0u, 0u, 0u);   // stale rows must never hold NaN patterns
   fence_proxy_async();
@@ -137,124 +150,118 @@ __global__ void __launch_bounds__(288, 1) radon_tc_kernel(const RadonParams prm)
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  const uint32_t acc_cols = prm.mt * 128;                       // TMEM columns of one accumulator set
+  const uint32_t nacc = min(MAX_ACC, 512 / (int)acc_cols);
 
   // items of this CTA: same part always; slab fastest, image slowest
-  const int64_t first = blockIdx.x / prm.parts, step = gridDim.x / prm.parts;
-  const int64_t total = prm.slabs * prm.images;
+  const uint32_t first = blockIdx.x / prm.parts, step = gridDim.x / prm.parts;
+  const uint32_t slabs = (uint32_t)prm.slabs, total = slabs * (uint32_t)prm.images;   // < 2^31 (checked by the launcher)
 
-  if (warp >= 4 && warp < 8) {
-    // ---- producers --------------------------------------------------------------------------------------------
-    const int tid = threadIdx.x - 128;
-    const int j = tid & 15, r0 = tid >> 4;                    // 16-byte piece of a 256-byte row; first row of eight
-    const uint32_t ring_base = smem_u32(sRing);
-    uint32_t gc = 0;                                          // groups issued
-    uint32_t done = 0;                                        // groups published
+  if (warp >= EPI_WARPS && warp < MMA_WARP) {
+    // ---- producers: warp pw fills the slots of the groups with (group counter) % active == pw, one group in flight each ----
+    // A warp must never be two uses of a slot ahead of the consumer (its wait names a phase parity), hence no more
+    // active producer warps than ring slots.
+    const int pw = warp - EPI_WARPS;
+    const uint32_t active = min(PROD_WARPS, prm.ring);
+    const int j = lane & 15, rl = lane >> 4;                  // 16-byte piece of a 256-byte row; row parity
+    const uint32_t ring_base = smem_u32(sRing) + (j >> 3) * (SLOT_ROWS * 128);
+    uint32_t gc = 0;                                          // groups of this CTA so far
     bool ok = true;
-    for (int64_t it = first; it < total && ok; it += step) {
-      const int img = (int)(it / prm.slabs);
-      const int64_t slab = it - (int64_t)img * prm.slabs;
-      const int64_t head = slab / prm.slabs_per_head;
-      const int e0 = (int)(slab - head * prm.slabs_per_head) * 128;
-      const __nv_bfloat16* base = prm.src + head * prm.in.rows_per_head * prm.rp + e0 + j * 8;
-      const int reg_off = img * prm.in.s_img, vert_off = prm.in.v0 + img * prm.in.sv_img;
-      const bool vert = img >= prm.in.vert_from;
-      for (int g = 0; g < kgroups && ok; ++g, ++gc) {
+    for (uint32_t it = first; it < total && ok; it += step) {
+      const uint32_t img = it / slabs, slab = it - img * slabs;
+      const uint32_t head = slab / (uint32_t)prm.slabs_per_head;
+      const int e0 = (int)(slab - head * (uint32_t)prm.slabs_per_head) * 128;
+      const __nv_bfloat16* base = prm.src + (int64_t)head * prm.in.rows_per_head * prm.rp + e0 + j * 8;
+      const int reg_off = (int)img * prm.in.s_img, vert_off = prm.in.v0 + (int)img * prm.in.sv_img;
+      const bool vert = (int)img >= prm.in.vert_from;
+      for (int g = 0; g < kgroups; ++g, ++gc) {
+        if ((int)(gc % active) != pw) continue;
         const int slot = gc % prm.ring;
-        if (gc >= (uint32_t)prm.ring) ok = mbar_wait(empty + slot, ((gc / prm.ring) - 1) & 1, wc);
+        if (gc >= (uint32_t)prm.ring) ok = mbar_wait_warp(empty + slot, ((gc / prm.ring) - 1) & 1, wc);
         if (!ok) break;
-        const uint32_t sbase = ring_base + slot * SLOT_BYTES + (j >> 3) * (SLOT_ROWS * 128);
+        const uint32_t sbase = ring_base + slot * SLOT_BYTES;
         const int rows = min(SLOT_ROWS, prm.k_pad - g * SLOT_ROWS);
+        const int32_t* tab = in_tab + g * SLOT_ROWS;
+        for (int i0 = 0; i0 < rows / 2; i0 += 8) {              // rows is a multiple of 16
+          int t[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int r = r0 + 8 * i;
-          if (r < rows) {
-            const int t = in_tab[g * SLOT_ROWS + r];
-            const uint32_t dst = sbase + r * 128 + (((j & 7) ^ (r & 7)) << 4);
-            if (t == ROW_INVALID || ((t & ROW_VERT) && !vert)) {
-              st_zero16(dst);
-            } else {
-              const int row = (t & ROW_VERT) ? vert_off + (t & ~ROW_VERT) : reg_off + t;
-              cp_async16(dst, base + (int64_t)row * prm.rp);
-            }
+          for (int u = 0; u < 8; ++u) t[u] = tab[rl + 2 * (i0 + u)];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int r = rl + 2 * (i0 + u);
+            const bool valid = t[u] >= 0 && (!(t[u] & ROW_VERT) || vert);
+            const int row = valid ? (t[u] & (ROW_VERT - 1)) + ((t[u] & ROW_VERT) ? vert_off : reg_off) : 0;
+            cp_async16_zfill(sbase + r * 128 + (((j & 7) ^ (r & 7)) << 4), base + (int64_t)row * prm.rp, valid ? 16 : 0);
           }
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        if (gc >= (uint32_t)LA) {
-          asm volatile("cp.async.wait_group %0;" ::"n"(LA) : "memory");
-          fence_proxy_async();
-          mbar_arrive(full + (done % prm.ring));
-          ++done;
-        }
+        asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full + slot);
       }
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    fence_proxy_async();
-    for (; done < gc; ++done) mbar_arrive(full + (done % prm.ring));
-  } else if (warp == 8 && lane == 0) {
+  } else if (warp == MMA_WARP && lane == 0) {
     // ---- MMA issuer -------------------------------------------------------------------------------------------
-    const uint32_t idesc = make_idesc(128, prm.n_part, 1, 0);   // A MN-major (image rows), B K-major (R)
+    constexpr uint32_t idesc = make_idesc(TILE_ROWS, 128, 0, 1);   // A K-major (R), B MN-major (image rows)
     const uint32_t aR = smem_u32(sR), aRing = smem_u32(sRing);
     uint32_t gc = 0, n_item = 0;
     bool ok = true;
-    for (int64_t it = first; it < total && ok; it += step, ++n_item) {
-      const uint32_t buf = n_item & 1;
-      if (n_item >= 2) ok = mbar_wait(acc_empty + buf, ((n_item >> 1) - 1) & 1, wc);
+    for (uint32_t it = first; it < total && ok; it += step, ++n_item) {
+      const uint32_t buf = n_item % nacc;
+      if (n_item >= nacc) ok = mbar_wait(acc_empty + buf, ((n_item / nacc) - 1) & 1, wc);
       if (!ok) break;
       fence_after_sync();
-      const uint32_t tmem_d = tmem_base + buf * 256;
+      const uint32_t tmem_d = tmem_base + buf * acc_cols;
       for (int g = 0; g < kgroups && ok; ++g, ++gc) {
         const int slot = gc % prm.ring;
         ok = mbar_wait(full + slot, (gc / prm.ring) & 1, wc);
         if (!ok) break;
         fence_after_sync();
         const int steps = min(4, (prm.k_pad - g * SLOT_ROWS) / 16);
-        for (int kk = 0; kk < steps; ++kk) {
-          const uint64_t dA = make_desc(aRing + slot * SLOT_BYTES + kk * 2048, SLOT_ROWS * 128, 1024);
-          const uint64_t dB = make_desc(aR + g * (prm.n_part * 128) + kk * 32, 16, 1024);
-          mma_bf16(tmem_d, dA, dB, idesc, (g | kk) != 0);
-        }
+        for (int t = 0; t < prm.mt; ++t)
+          for (int kk = 0; kk < steps; ++kk) {
+            const uint64_t dA = make_desc(aR + (t * kgroups + g) * (TILE_ROWS * 128) + kk * 32, 16, 1024);
+            const uint64_t dB = make_desc(aRing + slot * SLOT_BYTES + kk * 2048, SLOT_ROWS * 128, 1024);
+            mma_bf16(tmem_d + t * 128, dA, dB, idesc, (g | kk) != 0);
+          }
         mma_commit(empty + slot);
       }
       if (ok) mma_commit(acc_full + buf);
     }
-  } else if (warp < 4) {
+  } else if (warp < EPI_WARPS) {
     // ---- epilogue ---------------------------------------------------------------------------------------------
-    // 32 output indices at a time: every thread drops its entry's 32 values into a [32][128] bf16 staging tile,
-    // then the 128 threads write the tile out as whole 256-byte rows (16 bytes per thread and store).
-    const int tid = threadIdx.x;
-    const int e = tid;                                           // state entry of the slab = TMEM lane
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-    uint32_t n_item = 0, n_chunk = 0;
-    for (int64_t it = first; it < total; it += step, ++n_item) {
-      const uint32_t buf = n_item & 1;
-      const int img = (int)(it / prm.slabs);
-      const int64_t slab = it - (int64_t)img * prm.slabs;
-      const int64_t head = slab / prm.slabs_per_head;
-      const int e0 = (int)(slab - head * prm.slabs_per_head) * 128;
-      __nv_bfloat16* base = prm.dst + head * prm.out.rows_per_head * prm.rp + e0 + (tid & 15) * 8;
-      const int reg_off = img * prm.out.s_img, vert_off = prm.out.v0 + img * prm.out.sv_img;
-      const bool vert = img >= prm.out.vert_from;
-      const bool ok = mbar_wait(acc_full + buf, (n_item >> 1) & 1, wc);
-      if (bar_or_128(!ok)) break;                                // the four warps give up together
+    // Units of work per item: (tile, 32-entry column chunk); warp w takes the units of parity w / 4 in its lane
+    // quarter w % 4.
+    const int qd = warp & 3, half = warp >> 2;
+    const int orow = qd * 32 + lane;                            // output index inside a tile = TMEM lane
+    const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+    uint32_t n_item = 0;
+    for (uint32_t it = first; it < total; it += step, ++n_item) {
+      const uint32_t buf = n_item % nacc;
+      const uint32_t img = it / slabs, slab = it - img * slabs;
+      const uint32_t head = slab / (uint32_t)prm.slabs_per_head;
+      const int e0 = (int)(slab - head * (uint32_t)prm.slabs_per_head) * 128;
+      __nv_bfloat16* base = prm.dst + (int64_t)head * prm.out.rows_per_head * prm.rp + e0;
+      const int reg_off = (int)img * prm.out.s_img, vert_off = prm.out.v0 + (int)img * prm.out.sv_img;
+      const bool vert = (int)img >= prm.out.vert_from;
+      if (!mbar_wait_warp(acc_full + buf, (n_item / nacc) & 1, wc)) break;
       fence_after_sync();
-      for (int cb = 0; cb < prm.n_part / 32; ++cb, ++n_chunk) {
-        if (part * prm.n_part + cb * 32 >= prm.out.count) break;   // uniform: nothing valid from here on
+      for (int unit = half; unit < prm.mt * 4; unit += 2) {
+        const int t = unit >> 2, cb = unit & 3;
+        if (part * n_cta + t * TILE_ROWS >= prm.out.count) break;   // uniform: the tile holds no output index
         uint32_t v[32];
-        tmem_ld32(tmem_base + lane_base + buf * 256 + cb * 32, v);
+        tmem_ld32(tmem_base + lane_base + buf * acc_cols + t * 128 + cb * 32, v);
         tmem_ld_wait();
-        __nv_bfloat16* tile = stage + (n_chunk & 1) * (32 * 128);
+        const int tv = out_tab[t * TILE_ROWS + orow];
+        if (tv == ROW_INVALID || ((tv & ROW_VERT) && !vert)) continue;
+        const int row = (tv & ROW_VERT) ? vert_off + (tv & ~ROW_VERT) : reg_off + tv;
+        uint4* dst = reinterpret_cast<uint4*>(base + (int64_t)row * prm.rp + cb * 32);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) tile[i * 128 + e] = __float2bfloat16_rn(__uint_as_float(v[i]));
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-#pragma unroll
-        for (int x = 0; x < 4; ++x) {
-          const int i = (tid >> 4) + 8 * x;
-          const int t = out_tab[cb * 32 + i];
-          if (t == ROW_INVALID || ((t & ROW_VERT) && !vert)) continue;
-          const int row = (t & ROW_VERT) ? vert_off + (t & ~ROW_VERT) : reg_off + t;
-          *reinterpret_cast<uint4*>(base + (int64_t)row * prm.rp) =
-              *reinterpret_cast<const uint4*>(tile + i * 128 + (tid & 15) * 8);
-        }
+        for (int q4 = 0; q4 < 4; ++q4)
+          dst[q4] = make_uint4(pack_bf16(__uint_as_float(v[8 * q4]), __uint_as_float(v[8 * q4 + 1])),
+                               pack_bf16(__uint_as_float(v[8 * q4 + 2]), __uint_as_float(v[8 * q4 + 3])),
+                               pack_bf16(__uint_as_float(v[8 * q4 + 4]), __uint_as_float(v[8 * q4 + 5])),
+                               pack_bf16(__uint_as_float(v[8 * q4 + 6]), __uint_as_float(v[8 * q4 + 7])));
       }
       fence_before_sync();
       __syncwarp();
@@ -263,35 +270,34 @@ __global__ void __launch_bounds__(288, 1) radon_tc_kernel(const RadonParams prm)
   }
   fence_before_sync();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == MMA_WARP) {
     fence_after_sync();
     tmem_dealloc(tmem_base, 512);
   }
 }
 
 struct RadonShape {
-  int k_pad, kgroups, n_part, parts, ring, smem;
+  int k_pad, kgroups, mt, parts, ring, smem;
 };
 
-// Splits the output indices over `parts` CTAs so that the resident part of R and a ring of at least four slots fit
-// in shared memory.  Returns false when q is too large for this kernel.
+// Splits the output indices into tiles of 128 and the tiles over CTAs: two tiles per CTA when the resident part of R
+// then still leaves a ring of six slots, else one.  Returns false when q is too large for this kernel.
 bool radon_shape(int count_in, int count_out, RadonShape* s) {
   const int budget = 227 * 1024 - 1024 - 512;
   s->k_pad = (count_in + 15) & ~15;
   s->kgroups = (s->k_pad + SLOT_ROWS - 1) / SLOT_ROWS;
-  for (int parts = 1; parts <= 6; ++parts) {
-    const int per = (count_out + parts - 1) / parts;
-    const int n_part = (per + 31) & ~31;
-    if (n_part > 256) continue;
-    const int r_bytes = n_part * s->kgroups * 128;
-    const int tables = (s->kgroups * SLOT_ROWS + n_part) * 4;
-    const int left = budget - r_bytes - tables - STAGE_BYTES;
-    if (left < 4 * SLOT_BYTES) continue;
+  const int tiles = (count_out + TILE_ROWS - 1) / TILE_ROWS;
+  for (int mt = (tiles >= 2 ? 2 : 1); mt >= 1; --mt) {
+    const int r_bytes = mt * TILE_ROWS * s->kgroups * 128;
+    const int tables = (s->kgroups * SLOT_ROWS + mt * TILE_ROWS) * 4;
+    const int left = budget - r_bytes - tables;
+    const int need = mt == 2 ? 6 : 4;
+    if (left < need * SLOT_BYTES) continue;
     int ring = left / SLOT_BYTES;
     if (ring > 8) ring = 8;
-    s->n_part = n_part; s->parts = parts; s->ring = ring;
-    s->smem = r_bytes + ring * SLOT_BYTES + STAGE_BYTES + tables + 512 + 1024;
-    return true;
+    s->mt = mt; s->parts = (tiles + mt - 1) / mt; s->ring = ring;
+    s->smem = r_bytes + ring * SLOT_BYTES + tables + 512 + 1024;
+    return s->parts <= 8;
   }
   return false;
 }
@@ -307,9 +313,10 @@ RadonSide side(int count, int s_lo, int s_hi, int s_img, int64_t rows_per_head, 
 cudaError_t launch_radon(int q, int transpose, int images, const RadonSide& in, const RadonSide& out, const void* src,
                          void* dst, int64_t rp, int bh, int* status, cudaStream_t st) {
   RadonShape sh;
-  if (!radon_shape(in.count, out.count, &sh) || rp % 128) return cudaErrorInvalidValue;
+  if (!radon_shape(in.count, out.count, &sh) || rp % 128 || (int64_t)bh * (rp / 128) * images >= (1LL << 31))
+    return cudaErrorInvalidValue;
   RadonParams prm;
-  prm.q = q; prm.transpose = transpose; prm.k_pad = sh.k_pad; prm.n_part = sh.n_part; prm.parts = sh.parts;
+  prm.q = q; prm.transpose = transpose; prm.k_pad = sh.k_pad; prm.mt = sh.mt; prm.parts = sh.parts;
   prm.ring = sh.ring; prm.images = images; prm.slabs_per_head = (int)(rp / 128); prm.slabs = (int64_t)bh * (rp / 128);
   prm.rp = rp; prm.in = in; prm.out = out;
   prm.src = static_cast<const __nv_bfloat16*>(src);
@@ -321,16 +328,9 @@ cudaError_t launch_radon(int q, int transpose, int images, const RadonSide& in, 
   int64_t ctas = (int64_t)(sms / sh.parts) * sh.parts;
   const int64_t items = prm.slabs * images * sh.parts;
   if (items < ctas) ctas = items;
-  cudaError_t err;
-  if (sh.ring >= 6) {
-    err = cudaFuncSetAttribute(radon_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.smem);
-    if (err != cudaSuccess) return err;
-    radon_tc_kernel<4><<<(unsigned)ctas, 288, sh.smem, st>>>(prm);
-  } else {
-    err = cudaFuncSetAttribute(radon_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.smem);
-    if (err != cudaSuccess) return err;
-    radon_tc_kernel<2><<<(unsigned)ctas, 288, sh.smem, st>>>(prm);
-  }
+  cudaError_t err = cudaFuncSetAttribute(radon_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.smem);
+  if (err != cudaSuccess) return err;
+  radon_tc_kernel<<<(unsigned)ctas, RADON_THREADS, sh.smem, st>>>(prm);
   return cudaGetLastError();
 }
 
