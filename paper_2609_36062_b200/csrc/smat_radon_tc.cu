@@ -16,15 +16,15 @@
 // traffic.
 //
 // radon_tc_kernel, persistent, one CTA per SM.  An item is one image restricted to 128 consecutive state entries;
-// a CTA owns `mt` tiles of 128 output indices (its part of R) and applies them to every item it is given:
-//   every thread   : builds the CTA's part of R (128 mt output indices x K_pad input indices, K-major, 128-byte
-//                    swizzle) and the row tables once
+// a CTA owns up to 128 output indices (its part of R; the output indices are split evenly over `parts` CTAs that
+// then share every image) and applies them to every item it is given:
+//   warps 0-3      : build the CTA's part of R once and move it to tensor memory (lane = output index, one column
+//                    per two operand rows), where the MMAs read it as their A operand
 //   warp 16 lane 0 : TMA producer; a ring slot holds `sps` lines (fixed hi, all lo) of the image x 128 state entries
 //                    (MN-major B operand, two boxes of 64 entries); the extra class travels in a slot of its own
-//   warp 17 lane 0 : MMA issuer, D_t[128 outputs, 128 entries] += R_t,slot * B_slot for each tile t; up to four
-//                    accumulator sets in flight in TMEM
-//   warps 0-15     : epilogue, one output index (TMEM lane) per thread: round 32 entries at a time to bf16 and store
-//                    them as 64 contiguous bytes of the output row
+//   warp 17 lane 0 : MMA issuer, D[128 outputs, 128 entries] += R_slot * B_slot; up to four accumulators in flight
+//   warps 0-15     : epilogue, one output index (TMEM lane) per thread and one 32-entry column chunk per warp:
+//                    round to bf16 and store 64 contiguous bytes of the output row as two 32-byte sectors
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -41,7 +41,7 @@ constexpr int EPI_WARPS = 16;
 constexpr int PROD_WARP = EPI_WARPS;
 constexpr int MMA_WARP = EPI_WARPS + 1;
 constexpr int RADON_THREADS = 32 * (MMA_WARP + 1);
-constexpr int MAX_ACC = 4;                        // accumulator sets in flight: min(4, 512 / (128 mt))
+constexpr int MAX_ACC = 4;                        // accumulators in flight: what the R columns leave of 512, at most 4
 constexpr int ROW_INVALID = -1;
 constexpr int ROW_VERT = 1 << 30;                 // flag: row of the extra ("vertical") class
 
@@ -59,7 +59,7 @@ struct RadonParams {
   int32_t q, transpose;
   int32_t sps, sr;                 // lines (hi values) per ring slot; rows of a slot = sps*q rounded up to 16
   int32_t nreg, nslots;            // slots of regular lines per image; plus one when the input has the extra class
-  int32_t mt, parts;               // tiles of 128 output indices per CTA; CTAs sharing an image
+  int32_t parts, rows_pp;          // CTAs sharing an image, and output indices per CTA (<= 128)
   int32_t ring;                    // ring slots
   int32_t images;
   int32_t slabs_per_head;          // rp / 128
@@ -83,22 +83,38 @@ __device__ __forceinline__ int side_row(const RadonSide& s, int idx, int q) {
   const int lo = idx % q, hi = idx / q;
   return hi < q ? lo * s.s_lo + hi * s.s_hi : (ROW_VERT | lo * s.sv_lo);
 }
-// 1 when output index n and input index k are incident
-__device__ __forceinline__ bool radon_entry(int q, int transpose, int n, int k) {
-  const int o = transpose ? k : n, pt = transpose ? n : k;
-  const int u = o % q, a = o / q, lo = pt % q, hi = pt / q;
-  return a < q ? (lo + a * hi) % q == u : hi == u;
+
+// Row of the streamed operand that holds input index (lo, line): slot line / sps, then the line's q rows.
+__device__ __forceinline__ int operand_row(const RadonParams& p, int line, int lo) {
+  if (line >= p.q) return p.nreg * p.sr + lo;                 // extra class: a slot of its own
+  const int slot = line / p.sps;
+  return slot * p.sr + (line - slot * p.sps) * p.q + lo;
 }
 
-// Input index (lo + q*hi, hi == q for the extra class) held by row k of the streamed operand, or -1 for padding.
-// Slot s < nreg holds the lines hi = s*sps .. s*sps + sps - 1, q rows each; slot nreg holds the extra class.
-__device__ __forceinline__ int input_index(const RadonParams& p, int k) {
-  const int slot = k / p.sr, r = k - slot * p.sr, q = p.q;
-  if (slot < p.nreg) {
-    const int hi = slot * p.sps + r / q;
-    return (r < p.sps * q && hi < q) ? (r % q) + q * hi : -1;
+// Marks in `row` (one bf16 per operand row, zeroed by the caller) the input indices incident with output index n.
+// Forward: n = (u, a); a < q meets every line hi in lo = u - a hi, a = q (extra class) meets the whole line u.
+// Transposed: n = point (lo, hi); it lies on one offset u = lo + a hi of every slope a, and on offset hi of the extra class.
+__device__ __forceinline__ void mark_incident(const RadonParams& p, int n, __nv_bfloat16* row) {
+  const int q = p.q, x = n % q, y = n / q;
+  const __nv_bfloat16 one = __float2bfloat16(1.0f);
+  if (!p.transpose) {
+    if (y < q) {
+      int lo = x;                                               // u - a*hi for hi = 0, 1, ...
+      for (int hi = 0; hi < q; ++hi) {
+        row[operand_row(p, hi, lo)] = one;
+        lo -= y; if (lo < 0) lo += q;
+      }
+    } else {
+      for (int lo = 0; lo < q; ++lo) row[operand_row(p, x, lo)] = one;
+    }
+  } else {
+    int u = x;                                                  // lo + a*hi for a = 0, 1, ...
+    for (int a = 0; a < q; ++a) {
+      row[operand_row(p, a, u)] = one;
+      u += y; if (u >= q) u -= q;
+    }
+    if (p.in.count > q * q) row[operand_row(p, q, y)] = one;
   }
-  return r < q ? q * q + r : -1;
 }
 
 // box of 64 state entries x q rows x sps lines (regular map) or 64 x q rows (extra-class map)
@@ -124,31 +140,38 @@ __device__ __forceinline__ void st_global_v8(void* dst, const uint32_t (&w)[8]) 
                : "memory");
 }
 
-// The MMAs of one ring slot: STEPS K-steps of 16 operand rows for each of MT tiles.  Fully unrolled so that the lone
-// issuing thread spends a handful of instructions per MMA.
-template <int STEPS, int MT>
-__device__ __forceinline__ void issue_slot(uint32_t tmem_d, uint64_t dA, uint64_t dA_tile, uint64_t dB, uint32_t idesc,
-                                           bool first) {
-#pragma unroll
-  for (int kk = 0; kk < STEPS; ++kk) {
-    const uint64_t a = dA + (uint64_t)((kk >> 2) * (TILE_ROWS * 128 >> 4) + (kk & 3) * 2);
-    const uint64_t b = dB + (uint64_t)(kk * 128);
-    mma_bf16(tmem_d, a, b, idesc, !(first && kk == 0));
-    if (MT == 2) mma_bf16(tmem_d + 128, a + dA_tile, b, idesc, !(first && kk == 0));
-  }
+// D[tmem_d] (+)= A[tmem_a] * B[desc_b]: A (128 x 16, bf16) read from tensor memory, B from shared memory.
+__device__ __forceinline__ void mma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
-template <int MT>
-__device__ __forceinline__ void issue_slot_steps(int steps, uint32_t tmem_d, uint64_t dA, uint64_t dA_tile, uint64_t dB,
-                                                 uint32_t idesc, bool first) {
+
+// The MMAs of one ring slot: STEPS K-steps of 16 operand rows.  Fully unrolled so that the lone issuing thread spends
+// a handful of instructions per MMA.  A K-step reads 8 columns of R (two bf16 per column) and 16 rows of the slot.
+template <int STEPS>
+__device__ __forceinline__ void issue_slot(uint32_t tmem_d, uint32_t tmem_a, uint64_t dB, uint32_t idesc, bool first) {
+#pragma unroll
+  for (int kk = 0; kk < STEPS; ++kk)
+    mma_bf16_ta(tmem_d, tmem_a + kk * 8, dB + (uint64_t)(kk * 128), idesc, !(first && kk == 0));
+}
+__device__ __forceinline__ void issue_slot_steps(int steps, uint32_t tmem_d, uint32_t tmem_a, uint64_t dB, uint32_t idesc,
+                                                 bool first) {
   switch (steps) {
-    case 1: issue_slot<1, MT>(tmem_d, dA, dA_tile, dB, idesc, first); break;
-    case 2: issue_slot<2, MT>(tmem_d, dA, dA_tile, dB, idesc, first); break;
-    case 3: issue_slot<3, MT>(tmem_d, dA, dA_tile, dB, idesc, first); break;
-    case 4: issue_slot<4, MT>(tmem_d, dA, dA_tile, dB, idesc, first); break;
-    case 5: issue_slot<5, MT>(tmem_d, dA, dA_tile, dB, idesc, first); break;
-    case 6: issue_slot<6, MT>(tmem_d, dA, dA_tile, dB, idesc, first); break;
-    case 7: issue_slot<7, MT>(tmem_d, dA, dA_tile, dB, idesc, first); break;
-    default: issue_slot<8, MT>(tmem_d, dA, dA_tile, dB, idesc, first); break;
+    case 1: issue_slot<1>(tmem_d, tmem_a, dB, idesc, first); break;
+    case 2: issue_slot<2>(tmem_d, tmem_a, dB, idesc, first); break;
+    case 3: issue_slot<3>(tmem_d, tmem_a, dB, idesc, first); break;
+    case 4: issue_slot<4>(tmem_d, tmem_a, dB, idesc, first); break;
+    case 5: issue_slot<5>(tmem_d, tmem_a, dB, idesc, first); break;
+    case 6: issue_slot<6>(tmem_d, tmem_a, dB, idesc, first); break;
+    case 7: issue_slot<7>(tmem_d, tmem_a, dB, idesc, first); break;
+    default: issue_slot<8>(tmem_d, tmem_a, dB, idesc, first); break;
   }
 }
 
@@ -159,18 +182,14 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int q = prm.q;
   const int slot_bytes = prm.sr * 256;                          // two 64-entry blocks of sr rows x 128 bytes
-  const int kb2 = (prm.sr + 63) / 64;                           // 64-row blocks of R per slot
-  const int kblocks = prm.nslots * kb2;                         // and per tile
-  const int n_cta = prm.mt * TILE_ROWS;                         // output indices of this CTA
-  const int r_bytes = n_cta * kblocks * 128;                    // R part: [tile][64-index block][128 rows][128 bytes]
-  uint8_t* sR = smem;
-  uint8_t* sRing = smem + r_bytes;
-  int32_t* out_tab = reinterpret_cast<int32_t*>(sRing + prm.ring * slot_bytes);    // [n_cta]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_tab + n_cta);
+  const int kt = prm.nslots * prm.sr;                           // operand rows per image
+  uint8_t* sRing = smem;
+  int32_t* out_tab = reinterpret_cast<int32_t*>(sRing + prm.ring * slot_bytes);    // [128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_tab + TILE_ROWS);
   uint64_t* full = bars;                    // [ring] slot filled (TMA bytes)
   uint64_t* empty = bars + prm.ring;        // [ring] slot consumed by the MMAs
-  uint64_t* acc_full = empty + prm.ring;    // [MAX_ACC] accumulator set complete
-  uint64_t* acc_empty = acc_full + MAX_ACC; // [MAX_ACC] accumulator set read out (one arrival per epilogue warp)
+  uint64_t* acc_full = empty + prm.ring;    // [MAX_ACC] accumulator complete
+  uint64_t* acc_empty = acc_full + MAX_ACC; // [MAX_ACC] accumulator read out (one arrival per epilogue warp)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + MAX_ACC);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -186,34 +205,40 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     prefetch_tmap(&tm_vert);
   }
   if (warp == MMA_WARP) tmem_alloc(tmem_slot, 512);
-  // R part, 16 bytes (8 rows of the streamed operand) per store; per tile one run of kb2 blocks for every slot
-  for (int c = threadIdx.x; c < n_cta * kblocks * 8; c += blockDim.x) {
-    const int n = c % n_cta, kc = c / n_cta;                   // kc: chunk of 8 operand rows, counted in blocks of 64
-    const int g = kc / (kb2 * 8), r0 = (kc - g * kb2 * 8) * 8; // slot and first row inside it
-    const int nidx = part * n_cta + n;
-    uint32_t w[4] = {0u, 0u, 0u, 0u};
-    if (nidx < prm.out.count) {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const int idx = r0 + e < prm.sr ? input_index(prm, g * prm.sr + r0 + e) : -1;
-        if (idx >= 0 && idx < prm.in.count && radon_entry(q, prm.transpose, nidx, idx))
-          w[e >> 1] |= 0x3F80u << ((e & 1) * 16);              // bf16 1.0
-      }
-    }
-    const int t = n >> 7, row = n & 127;
-    uint8_t* dst = sR + ((t * kblocks + (kc >> 3)) * TILE_ROWS + row) * 128 + (((kc & 7) ^ (row & 7)) << 4);
-    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-  }
-  for (int n = threadIdx.x; n < n_cta; n += blockDim.x) out_tab[n] = side_row(prm.out, part * n_cta + n, q);
+  // This CTA's part of R, built row by row in the (still unused) ring and moved to tensor memory: lane = output
+  // index, one column per two operand rows.  The launcher guarantees ring * slot_bytes >= 128 * kt * 2.
+  __nv_bfloat16* scratch = reinterpret_cast<__nv_bfloat16*>(sRing);
   for (int c = threadIdx.x; c < prm.ring * slot_bytes / 16; c += blockDim.x)
-    reinterpret_cast<uint4*>(sRing)[c] = make_uint4(0u, 0u, 0u, 0u);   // rows no box writes must never hold NaN patterns
-  fence_proxy_async();
+    reinterpret_cast<uint4*>(sRing)[c] = make_uint4(0u, 0u, 0u, 0u);
+  for (int n = threadIdx.x; n < TILE_ROWS; n += blockDim.x)
+    out_tab[n] = n < prm.rows_pp ? side_row(prm.out, part * prm.rows_pp + n, q) : ROW_INVALID;
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t acc_cols = prm.mt * 128;                       // TMEM columns of one accumulator set
-  const uint32_t nacc = min(MAX_ACC, 512 / (int)acc_cols);
+  const uint32_t r_cols = (uint32_t)((kt / 2 + 31) & ~31);       // columns taken by R
+  const uint32_t nacc = min(MAX_ACC, (int)((512 - r_cols) / 128));
+  if (warp < 4) {
+    const int n = warp * 32 + lane;
+    __nv_bfloat16* row = scratch + (size_t)n * kt;
+    if (n < prm.rows_pp && part * prm.rows_pp + n < prm.out.count) mark_incident(prm, part * prm.rows_pp + n, row);
+    __syncwarp();
+    const uint32_t* roww = reinterpret_cast<const uint32_t*>(row);
+    for (int c0 = 0; c0 < (int)r_cols; c0 += 32) {
+      uint32_t v[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = (c0 + i) * 2 < kt ? roww[c0 + i] : 0u;
+      tmem_st32(tmem_base + ((uint32_t)(warp * 32) << 16) + c0, v);
+    }
+    tmem_st_wait();
+  }
+  __syncthreads();
+  // rows no box writes must never hold NaN patterns: the ones just written are 0 or 1, which is fine
+  fence_proxy_async();
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_acc = tmem_base + r_cols;
 
   // items of this CTA: same part always; slab fastest, image slowest
   const uint32_t first = blockIdx.x / prm.parts, step = gridDim.x / prm.parts;
@@ -257,30 +282,26 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     }
   } else if (warp == MMA_WARP && lane == 0) {
     // ---- MMA issuer -------------------------------------------------------------------------------------------
-    constexpr uint32_t idesc = make_idesc(TILE_ROWS, 128, 0, 1);   // A K-major (R), B MN-major (image rows)
-    const uint64_t dA0 = make_desc(smem_u32(sR), 16, 1024);
+    constexpr uint32_t idesc = make_idesc(TILE_ROWS, 128, 0, 1);   // A from tensor memory (R), B MN-major (image rows)
     const uint64_t dB0 = make_desc(smem_u32(sRing), prm.sr * 128, 1024);
     const uint32_t slot16 = (uint32_t)slot_bytes >> 4;            // descriptor address units are 16 bytes
-    const uint32_t tile16 = (uint32_t)kblocks * (TILE_ROWS * 128 >> 4);
-    const uint32_t slotA16 = (uint32_t)kb2 * (TILE_ROWS * 128 >> 4);
-    const int steps = prm.sr / 16, nslots = prm.nslots, mt = prm.mt;
+    const uint32_t slot_cols = (uint32_t)prm.sr / 2;              // columns of R per slot
+    const int steps = prm.sr / 16, nslots = prm.nslots;
     const uint32_t ring = (uint32_t)prm.ring;
     uint32_t slot = 0, par = 0;                                   // ring position and the parity its full barrier shows
-    uint32_t buf = 0, apar = 0, n_item = 0;                       // accumulator set; parity of its empty barrier's phase to wait for
+    uint32_t buf = 0, apar = 0, n_item = 0;                       // accumulator; parity of its empty barrier's phase to wait for
     bool ok = true;
     for (uint32_t it = first; it < total && ok; it += step, ++n_item) {
       if (n_item >= nacc) ok = mbar_wait(acc_empty + buf, apar, wc);
       if (!ok) break;
       fence_after_sync();
-      const uint32_t tmem_d = tmem_base + buf * acc_cols;
-      uint64_t dA = dA0;
-      for (int g = 0; g < nslots && ok; ++g, dA += slotA16) {
+      const uint32_t tmem_d = tmem_acc + buf * 128;
+      uint32_t tmem_a = tmem_base;
+      for (int g = 0; g < nslots && ok; ++g, tmem_a += slot_cols) {
         ok = mbar_wait(full + slot, par, wc);
         if (!ok) break;
         fence_after_sync();
-        const uint64_t dB = dB0 + (uint64_t)(slot * slot16);
-        if (mt == 2) issue_slot_steps<2>(steps, tmem_d, dA, tile16, dB, idesc, g == 0);
-        else issue_slot_steps<1>(steps, tmem_d, dA, tile16, dB, idesc, g == 0);
+        issue_slot_steps(steps, tmem_d, tmem_a, dB0 + (uint64_t)(slot * slot16), idesc, g == 0);
         mma_commit(empty + slot);
         if (++slot == ring) { slot = 0; par ^= 1; }
       }
@@ -289,44 +310,45 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     }
   } else if (warp < EPI_WARPS) {
     // ---- epilogue ---------------------------------------------------------------------------------------------
-    // Units of work per item: (tile, 32-entry column chunk); warp w takes every fourth unit, starting at w / 4, in
-    // its lane quarter w % 4.
-    const int qd = warp & 3, sub = warp >> 2;
-    const int orow = qd * 32 + lane;                            // output index inside a tile = TMEM lane
+    // Warp w reads lane quarter w % 4 (32 output indices) and the 32-entry column chunk w / 4 of every item.
+    const int qd = warp & 3, cb = warp >> 2;
+    const int orow = qd * 32 + lane;                            // output index of this CTA = TMEM lane
     const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
-    uint32_t n_item = 0;
-    for (uint32_t it = first; it < total; it += step, ++n_item) {
-      const uint32_t buf = n_item % nacc;
-      const uint32_t img = it / slabs, slab = it - img * slabs;
-      const uint32_t head = slab / (uint32_t)prm.slabs_per_head;
-      const int e0 = (int)(slab - head * (uint32_t)prm.slabs_per_head) * 128;
-      __nv_bfloat16* base = prm.dst + (int64_t)head * prm.out.rows_per_head * prm.rp + e0;
-      const int reg_off = (int)img * prm.out.s_img, vert_off = prm.out.v0 + (int)img * prm.out.sv_img;
-      const bool vert = (int)img >= prm.out.vert_from;
-      if (!mbar_wait_warp(acc_full + buf, (n_item / nacc) & 1, wc)) break;
+    const int tv = out_tab[orow];
+    const bool active = qd * 32 < prm.rows_pp;                  // warp-uniform: some output index in these lanes
+    const uint32_t sph = (uint32_t)prm.slabs_per_head;
+    uint32_t buf = 0, apar = 0;
+    uint32_t img = first / slabs, slab = first - img * slabs;
+    for (uint32_t it = first; it < total; it += step) {
+      const uint32_t head = slab / sph;
+      const int e0 = (int)(slab - head * sph) * 128;
+      if (!mbar_wait_warp(acc_full + buf, apar, wc)) break;
       fence_after_sync();
-      for (int unit = sub; unit < prm.mt * 4; unit += 4) {
-        const int t = unit >> 2, cb = unit & 3;
-        if (part * n_cta + t * TILE_ROWS + qd * 32 >= prm.out.count) break;   // warp-uniform: no output index in these lanes
+      if (active) {
         uint32_t v[32];
-        tmem_ld32(tmem_base + lane_base + buf * acc_cols + t * 128 + cb * 32, v);
+        tmem_ld32(tmem_acc + lane_base + buf * 128 + cb * 32, v);
         tmem_ld_wait();
-        const int tv = out_tab[t * TILE_ROWS + orow];
-        if (tv == ROW_INVALID || ((tv & ROW_VERT) && !vert)) continue;
-        const int row = (tv & ROW_VERT) ? vert_off + (tv & ~ROW_VERT) : reg_off + tv;
-        __nv_bfloat16* dst = base + (int64_t)row * prm.rp + cb * 32;
+        const bool vert = (int)img >= prm.out.vert_from;
+        if (tv != ROW_INVALID && (!(tv & ROW_VERT) || vert)) {
+          const int row = (tv & ROW_VERT) ? prm.out.v0 + (int)img * prm.out.sv_img + (tv & ~ROW_VERT)
+                                          : (int)img * prm.out.s_img + tv;
+          __nv_bfloat16* dst = prm.dst + ((int64_t)head * prm.out.rows_per_head + row) * prm.rp + e0 + cb * 32;
 #pragma unroll
-        for (int h8 = 0; h8 < 2; ++h8) {   // two whole 32-byte sectors per thread
-          uint32_t w[8];
+          for (int h8 = 0; h8 < 2; ++h8) {   // two whole 32-byte sectors per thread
+            uint32_t w[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            w[i] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * i]), __uint_as_float(v[16 * h8 + 2 * i + 1]));
-          st_global_v8(dst + 16 * h8, w);
+            for (int i = 0; i < 8; ++i)
+              w[i] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * i]), __uint_as_float(v[16 * h8 + 2 * i + 1]));
+            st_global_v8(dst + 16 * h8, w);
+          }
         }
       }
       fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty + buf);
+      if (++buf == nacc) { buf = 0; apar ^= 1; }
+      slab += step;
+      while (slab >= slabs) { slab -= slabs; ++img; }
     }
   }
   fence_before_sync();
@@ -338,40 +360,35 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
 }
 
 struct RadonShape {
-  int sps, sr, nreg, nslots, mt, parts, ring, smem;
+  int sps, sr, nreg, nslots, parts, rows_pp, ring, smem;
 };
 
-// Ring slots of `sps` lines (sps*q rows, rounded up to 16) and the split of the output indices into tiles of 128 and
-// of the tiles over CTAs (two tiles per CTA when the resident part of R then still leaves a ring of three slots,
-// else one), chosen for the least MMA work.  Returns false when q is too large for this kernel.
+// Ring slots of `sps` lines (sps*q rows, rounded up to 16), chosen for the least MMA work; the output indices are
+// split evenly over `parts` CTAs of at most 128 each.  R (128 lanes x one column per two operand rows) and at least
+// two accumulators of 128 columns must fit the 512 columns of tensor memory, and the ring must be able to hold the
+// scratch copy of R while it is built.  Returns false when q is too large for this kernel.
 bool radon_shape(int q, int in_has_extra, int count_out, RadonShape* s) {
-  const int budget = 227 * 1024 - 1024 - 512;
+  const int budget = 227 * 1024 - 1024 - 512 - TILE_ROWS * 4;
   if (q < 2 || q > 64) return false;
-  const int tiles = (count_out + TILE_ROWS - 1) / TILE_ROWS;
+  const int parts = (count_out + TILE_ROWS - 1) / TILE_ROWS;
+  if (parts > 8) return false;
   int best = 1 << 30;
   for (int sps = 1; sps <= q; ++sps) {
     const int sr = (sps * q + 15) & ~15;
     if (sr > 128) break;
     const int nreg = (q + sps - 1) / sps, nslots = nreg + (in_has_extra ? 1 : 0);
-    const int kblocks = nslots * ((sr + 63) / 64);   // R keeps a run of 64-row blocks per slot
+    const int r_cols = (nslots * sr / 2 + 31) & ~31;
+    if (r_cols + 2 * 128 > 512) continue;
     const int slot_bytes = sr * 256;
-    for (int mt = (tiles >= 2 ? 2 : 1); mt >= 1; --mt) {
-      const int r_bytes = mt * TILE_ROWS * kblocks * 128;
-      const int tables = mt * TILE_ROWS * 4;
-      const int left = budget - r_bytes - tables;
-      if (left < 3 * slot_bytes) continue;
-      int ring = left / slot_bytes;
-      if (ring > 8) ring = 8;
-      const int parts = (tiles + mt - 1) / mt;
-      if (parts > 8) continue;
-      // MMA work per image (operand rows, plus a charge per slot for its hand-over), times the CTAs that repeat it
-      const int cost = nslots * (sr + 48) * parts;
-      if (cost < best) {
-        best = cost;
-        s->sps = sps; s->sr = sr; s->nreg = nreg; s->nslots = nslots; s->mt = mt; s->parts = parts; s->ring = ring;
-        s->smem = r_bytes + ring * slot_bytes + tables + 512 + 1024;
-      }
-      break;   // the largest feasible mt for this sps
+    int ring = budget / slot_bytes;
+    if (ring > 8) ring = 8;
+    if (ring < 3 || ring < nslots) continue;
+    const int cost = nslots * (sr + 48);   // operand rows per image, plus a charge per slot for its hand-over
+    if (cost < best) {
+      best = cost;
+      s->sps = sps; s->sr = sr; s->nreg = nreg; s->nslots = nslots; s->parts = parts;
+      s->rows_pp = (count_out + parts - 1) / parts; s->ring = ring;
+      s->smem = ring * slot_bytes + TILE_ROWS * 4 + 512 + 1024;
     }
   }
   return best != (1 << 30);
@@ -428,7 +445,7 @@ cudaError_t launch_radon(int q, int transpose, int images, const RadonSide& in, 
     return cudaErrorInvalidValue;
   RadonParams prm;
   prm.q = q; prm.transpose = transpose; prm.sps = sh.sps; prm.sr = sh.sr; prm.nreg = sh.nreg; prm.nslots = sh.nslots;
-  prm.mt = sh.mt; prm.parts = sh.parts;
+  prm.parts = sh.parts; prm.rows_pp = sh.rows_pp;
   prm.ring = sh.ring; prm.images = images; prm.slabs_per_head = (int)(rp / 128); prm.slabs = (int64_t)bh * (rp / 128);
   prm.rp = rp; prm.in = in; prm.out = out;
   prm.src = static_cast<const __nv_bfloat16*>(src);
