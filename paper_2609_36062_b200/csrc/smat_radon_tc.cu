@@ -133,13 +133,6 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
-// 32-byte store (a whole sector per thread)
-__device__ __forceinline__ void st_global_v8(void* dst, const uint32_t (&w)[8]) {
-  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
-               "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
-               : "memory");
-}
-
 // D[tmem_d] (+)= A[tmem_a] * B[desc_b]: A (128 x 16, bf16) read from tensor memory, B from shared memory.
 __device__ __forceinline__ void mma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
                                             uint32_t accumulate) {
@@ -339,7 +332,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
 #pragma unroll
             for (int i = 0; i < 8; ++i)
               w[i] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * i]), __uint_as_float(v[16 * h8 + 2 * i + 1]));
-            st_global_v8(dst + 16 * h8, w);
+            st_global_v8(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
           }
         }
       }

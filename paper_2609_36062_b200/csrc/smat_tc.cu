@@ -116,13 +116,11 @@ __global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constan
       // state[b] = running sum before this tile (in visiting order)
       uint4* dst = reinterpret_cast<uint4*>(prm.Sin + (((int64_t)bh * prm.NC + b) * TILE + row) * TILE + half * HALF);
 #pragma unroll
-      for (int j8 = 0; j8 < HALF / 8; ++j8) {
-        uint4 pk;
-        pk.x = pack_bf16(acc[j8 * 8 + 0], acc[j8 * 8 + 1]);
-        pk.y = pack_bf16(acc[j8 * 8 + 2], acc[j8 * 8 + 3]);
-        pk.z = pack_bf16(acc[j8 * 8 + 4], acc[j8 * 8 + 5]);
-        pk.w = pack_bf16(acc[j8 * 8 + 6], acc[j8 * 8 + 7]);
-        dst[j8] = pk;
+      for (int j16 = 0; j16 < HALF / 16; ++j16) {   // whole 32-byte sectors
+        uint32_t w[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) w[e] = pack_bf16(acc[j16 * 16 + 2 * e], acc[j16 * 16 + 2 * e + 1]);
+        st_global_v8(dst + 2 * j16, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
       }
       if (it + 1 == hi - lo) break;  // every issued MMA has been consumed: nothing is in flight at teardown
       if (!mbar_wait(dfull + db, (it / SCAN_DBUF) & 1, wc)) break;
@@ -315,6 +313,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
           uint32_t v[32];
           tmem_ld32(tmem_o + lane_base + cb * 32, v);
           tmem_ld_wait();
+          uint32_t w[16];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             float f[8];
@@ -325,9 +324,13 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
               f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
               f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
             }
-            dst[cb * 4 + i] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
-                                         pack_bf16(f[6], f[7]));
+            w[4 * i] = pack_bf16(f[0], f[1]); w[4 * i + 1] = pack_bf16(f[2], f[3]);
+            w[4 * i + 2] = pack_bf16(f[4], f[5]); w[4 * i + 3] = pack_bf16(f[6], f[7]);
           }
+#pragma unroll
+          for (int h8 = 0; h8 < 2; ++h8)   // whole 32-byte sectors
+            st_global_v8(dst + cb * 4 + 2 * h8, w[8 * h8], w[8 * h8 + 1], w[8 * h8 + 2], w[8 * h8 + 3], w[8 * h8 + 4],
+                         w[8 * h8 + 5], w[8 * h8 + 6], w[8 * h8 + 7]);
         }
       }
     }
@@ -424,7 +427,9 @@ __global__ void __launch_bounds__(192) segment_state_tc_kernel(const __grid_cons
         tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
         tmem_ld_wait();
 #pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4) dst[cb * 8 + q4] = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+        for (int q8 = 0; q8 < 4; ++q8)   // whole 32-byte sectors
+          st_global_v8(dst + cb * 8 + 2 * q8, v[8 * q8], v[8 * q8 + 1], v[8 * q8 + 2], v[8 * q8 + 3], v[8 * q8 + 4], v[8 * q8 + 5],
+                       v[8 * q8 + 6], v[8 * q8 + 7]);
       }
     }
   }
@@ -639,6 +644,7 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
         uint32_t v[32];
         tmem_ld32(tmem_o + lane_base + col0 + cb * 32, v);
         tmem_ld_wait();
+        uint32_t w[16];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           float f[8];
@@ -649,9 +655,13 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
             f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
             f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
           }
-          dst[cb * 4 + i] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
-                                       pack_bf16(f[6], f[7]));
+          w[4 * i] = pack_bf16(f[0], f[1]); w[4 * i + 1] = pack_bf16(f[2], f[3]);
+          w[4 * i + 2] = pack_bf16(f[4], f[5]); w[4 * i + 3] = pack_bf16(f[6], f[7]);
         }
+#pragma unroll
+        for (int h8 = 0; h8 < 2; ++h8)   // whole 32-byte sectors
+          st_global_v8(dst + cb * 4 + 2 * h8, w[8 * h8], w[8 * h8 + 1], w[8 * h8 + 2], w[8 * h8 + 3], w[8 * h8 + 4],
+                       w[8 * h8 + 5], w[8 * h8 + 6], w[8 * h8 + 7]);
       }
     }
   }
@@ -757,9 +767,9 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
             tmem_ld_wait();
             if (m < kn) {
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
-                dst[cb * 8 + i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                              __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+              for (int i = 0; i < 4; ++i)   // whole 32-byte sectors
+                st_global_v8(dst + cb * 8 + 2 * i, v[8 * i], v[8 * i + 1], v[8 * i + 2], v[8 * i + 3], v[8 * i + 4],
+                             v[8 * i + 5], v[8 * i + 6], v[8 * i + 7]);
             }
           }
           fence_before_sync();
@@ -910,13 +920,15 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
           for (int j = 0; j < 32; ++j) v[j] = 0u;  // profile cell without tokens (P > n)
         }
         if (OUT_BF16) {
-          uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(prm.F) + (item * TILE + i) * TILE + cb * 32);
+          __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(prm.F) + (item * TILE + i) * TILE + cb * 32;
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4)
-            dst[q4] = make_uint4(pack_bf16(__uint_as_float(v[8 * q4]), __uint_as_float(v[8 * q4 + 1])),
-                                 pack_bf16(__uint_as_float(v[8 * q4 + 2]), __uint_as_float(v[8 * q4 + 3])),
-                                 pack_bf16(__uint_as_float(v[8 * q4 + 4]), __uint_as_float(v[8 * q4 + 5])),
-                                 pack_bf16(__uint_as_float(v[8 * q4 + 6]), __uint_as_float(v[8 * q4 + 7])));
+          for (int h8 = 0; h8 < 2; ++h8) {  // whole 32-byte sectors
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              w[e] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * e]), __uint_as_float(v[16 * h8 + 2 * e + 1]));
+            st_global_v8(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+          }
         } else {  // fp32 state: through a padded staging tile so that the global writes are whole 512-byte rows
           uint4* srow = reinterpret_cast<uint4*>(stage + i * STAGE_LD + cb * 32);
 #pragma unroll
