@@ -1092,7 +1092,8 @@ static cudaError_t launch_pool_tc(const PoolParams& prm, cudaStream_t st) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int per_sm = smem <= 72 * 1024 ? 3 : (smem <= 110 * 1024 ? 2 : 1);
+  // each CTA holds 128 columns of tensor memory, so at most four fit an SM
+  const int per_sm = smem <= 54 * 1024 ? 4 : (smem <= 72 * 1024 ? 3 : (smem <= 110 * 1024 ? 2 : 1));
   const int64_t grid = prm.items < (int64_t)per_sm * sms ? prm.items : (int64_t)per_sm * sms;
   pool_tc_kernel<TOK, OUT_BF16><<<(unsigned)grid, 160, smem, st>>>(prm);
   return cudaGetLastError();
