@@ -35,10 +35,11 @@ from paper_2609_36062_b200 import replicas, roofline, synth  # noqa: E402
 DEFAULT_WORKLOAD = "t16k_d4"
 SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
 METRIC = "SMat prefill tokens/s"
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu
-# capture summarised in profiles/forward_kernels_t16k_d4_h2.md: taken on the 2-head copy of the workload and
-# scaled by heads (every head owns its own tables, so traffic is proportional to the head count).
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant stage per step — the tabulation, two
+# launches of radon_tc_kernel — from the ncu capture summarised in profiles/radon_tc_kernel_t16k_d4_h2.md: taken on
+# the 2-head copy of the workload (280.6 MB) and scaled by heads (every head owns its tables).  At 2 heads about half
+# of the stage intermediate W is served by L2; with W fully in DRAM, as at 32 heads, the figure would be 5.97e9.
+NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate_tc"): 280.6e6 * 16}
 
 
 def parse_args():
@@ -138,7 +139,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -148,6 +149,13 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
+
+    def wait_ready(self, timeout_s: float = 3.0):
+        """Blocks until nvidia-smi has delivered its first sample, so that the timed region is covered."""
+        t0 = time.perf_counter()
+        while self.proc and not self.lines and time.perf_counter() - t0 < timeout_s:
+            time.sleep(0.01)
+        self.idle = len(self.lines)   # samples taken before any work was queued
 
     def stop(self):
         if not self.proc:
@@ -159,7 +167,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for ln in self.lines[getattr(self, "idle", 0):]:
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 7:
                 continue
@@ -344,6 +352,7 @@ def run_native(args):
 
     sampler = ClockSampler(local)
     sampler.start()
+    sampler.wait_ready()
     launches = runner.step()
     secs = runner.time_steps(runner.step, steps, warm, barrier)
     clocks = sampler.stop()
