@@ -513,44 +513,47 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
     constexpr uint32_t idesc_sc = make_idesc(TILE, TILE, 0, 0);   // Q Kᵀ: both K-major
     constexpr uint32_t idesc_o = make_idesc(TILE, TILE, 0, 1);    // A K-major (Q or P), B MN-major (S or V)
     constexpr uint32_t idesc_s = make_idesc(TILE, TILE, 1, 1);    // Kᵀ V: both MN-major
-    const uint32_t aSP = smem_u32(sSP);
+    // Descriptors are built once; inside the loops only constants are added (16-byte units): this lone thread pays
+    // the full latency of every instruction it issues.
+    constexpr uint32_t BOX16 = BOX_BYTES >> 4;
+    const uint64_t dSP_k = make_desc(smem_u32(sSP), 16, 1024);           // shared tile read K-major (P)
+    const uint64_t dSP_mn = make_desc(smem_u32(sSP), BOX_BYTES, 1024);   // and MN-major (S)
+    uint64_t dQ_k[2], dK_k[2], dK_mn[2], dV_mn[2];
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      const uint32_t sQ = smem_u32(smem + s * SEG_OUT_STAGE);
+      dQ_k[s] = make_desc(sQ, 16, 1024);
+      dK_k[s] = make_desc(sQ + 2 * BOX_BYTES, 16, 1024);
+      dK_mn[s] = make_desc(sQ + 2 * BOX_BYTES, BOX_BYTES, 1024);
+      dV_mn[s] = make_desc(sQ + 4 * BOX_BYTES, BOX_BYTES, 1024);
+    }
     for (int it = 0; it < prm.L; ++it) {
       const int s = it & 1;
-      const uint32_t sQ = smem_u32(smem + s * SEG_OUT_STAGE);
-      const uint32_t sK = sQ + 2 * BOX_BYTES, sV = sQ + 4 * BOX_BYTES;
+      const uint64_t qk = s ? dQ_k[1] : dQ_k[0], kk_ = s ? dK_k[1] : dK_k[0];
+      const uint64_t kmn = s ? dK_mn[1] : dK_mn[0], vmn = s ? dV_mn[1] : dV_mn[0];
       const uint32_t tmem_o = tmem_o0 + (it & 1) * TILE;
       if (!mbar_wait(full + s, (it >> 1) & 1, wc)) break;
       fence_after_sync();
 #pragma unroll
       for (int kk = 0; kk < TILE / 16; ++kk) {   // Sc = Q Kᵀ (the score tile was read out before bar_p of the last tile)
-        const uint64_t dA = make_desc(sQ + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-        const uint64_t dB = make_desc(sK + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-        mma_bf16(tmem_sc, dA, dB, idesc_sc, kk != 0);
+        const uint64_t off = (uint64_t)((kk >> 2) * BOX16 + (kk & 3) * 2);
+        mma_bf16(tmem_sc, qk + off, kk_ + off, idesc_sc, kk != 0);
       }
       mma_commit(bar_sc);
       if (!mbar_wait(bar_s, it & 1, wc)) break;  // bf16 state in the shared tile; output buffer of tile it-2 read out
       fence_after_sync();
 #pragma unroll
-      for (int kk = 0; kk < TILE / 16; ++kk) {   // O = Q S
-        const uint64_t dA = make_desc(sQ + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-        const uint64_t dB = make_desc(aSP + kk * 2048, BOX_BYTES, 1024);
-        mma_bf16(tmem_o, dA, dB, idesc_o, kk != 0);
-      }
+      for (int kk = 0; kk < TILE / 16; ++kk)     // O = Q S
+        mma_bf16(tmem_o, qk + (uint64_t)((kk >> 2) * BOX16 + (kk & 3) * 2), dSP_mn + (uint64_t)(kk * 128), idesc_o, kk != 0);
       mma_commit(bar_qs);
       if (!mbar_wait(bar_p, it & 1, wc)) break;
       fence_after_sync();
 #pragma unroll
-      for (int kk = 0; kk < TILE / 16; ++kk) {   // O += P V
-        const uint64_t dA = make_desc(aSP + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-        const uint64_t dB = make_desc(sV + kk * 2048, BOX_BYTES, 1024);
-        mma_bf16(tmem_o, dA, dB, idesc_o, 1);
-      }
+      for (int kk = 0; kk < TILE / 16; ++kk)     // O += P V
+        mma_bf16(tmem_o, dSP_k + (uint64_t)((kk >> 2) * BOX16 + (kk & 3) * 2), vmn + (uint64_t)(kk * 128), idesc_o, 1);
 #pragma unroll
-      for (int kk = 0; kk < TILE / 16; ++kk) {   // S += Kᵀ V
-        const uint64_t dA = make_desc(sK + kk * 2048, BOX_BYTES, 1024);
-        const uint64_t dB = make_desc(sV + kk * 2048, BOX_BYTES, 1024);
-        mma_bf16(tmem_s, dA, dB, idesc_s, 1);
-      }
+      for (int kk = 0; kk < TILE / 16; ++kk)     // S += Kᵀ V
+        mma_bf16(tmem_s, kmn + (uint64_t)(kk * 128), vmn + (uint64_t)(kk * 128), idesc_s, 1);
       mma_commit(bar_o);
       mma_commit(empty + s);
     }
