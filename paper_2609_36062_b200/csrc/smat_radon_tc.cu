@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   int32_t* out_tab = reinterpret_cast<int32_t*>(sRing + prm.ring * slot_bytes);    // [128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(out_tab + TILE_ROWS);
   uint64_t* full = bars;                    // [ring] slot filled (TMA bytes)
-  uint64_t* empty = bars + prm.ring;        // [ring] slot consumed by the MMAs
+  uint64_t* empty = bars + prm.ring;        // [ring] slot consumed by the MMAs (arrival from the epilogue, once the item is complete)
   uint64_t* acc_full = empty + prm.ring;    // [MAX_ACC] accumulator complete
   uint64_t* acc_empty = acc_full + MAX_ACC; // [MAX_ACC] accumulator read out (one arrival per epilogue warp)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + MAX_ACC);
@@ -295,10 +295,10 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
         if (!ok) break;
         fence_after_sync();
         issue_slot_steps(steps, tmem_d, tmem_a, dB0 + (uint64_t)(slot * slot16), idesc, g == 0);
-        mma_commit(empty + slot);
+        if (nslots == 1) mma_commit(empty + slot);   // one slot per item: free it directly (measured faster there)
         if (++slot == ring) { slot = 0; par ^= 1; }
       }
-      if (ok) mma_commit(acc_full + buf);
+      if (ok) mma_commit(acc_full + buf);   // with several slots per item the epilogue frees them when it sees this one
       if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
     }
   } else if (warp < EPI_WARPS) {
@@ -310,13 +310,20 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     const int tv = out_tab[orow];
     const bool active = qd * 32 < prm.rows_pp;                  // warp-uniform: some output index in these lanes
     const uint32_t sph = (uint32_t)prm.slabs_per_head;
-    uint32_t buf = 0, apar = 0;
+    uint32_t buf = 0, apar = 0, eslot = 0;
     uint32_t img = first / slabs, slab = first - img * slabs;
     for (uint32_t it = first; it < total; it += step) {
       const uint32_t head = slab / sph;
       const int e0 = (int)(slab - head * sph) * 128;
       if (!mbar_wait_warp(acc_full + buf, apar, wc)) break;
       fence_after_sync();
+      if (warp == 0 && prm.nslots > 1) {   // every MMA of the item has completed: its ring slots are free (a commit per slot would cost the
+                         // issuing thread more than the MMAs of the slot)
+        for (int g = 0; g < prm.nslots; ++g) {
+          if (lane == 0) mbar_arrive(empty + eslot);
+          if (++eslot == (uint32_t)prm.ring) eslot = 0;
+        }
+      }
       if (active) {
         uint32_t v[32];
         tmem_ld32(tmem_acc + lane_base + buf * 128 + cb * 32, v);
@@ -375,7 +382,8 @@ bool radon_shape(int q, int in_has_extra, int count_out, RadonShape* s) {
     const int slot_bytes = sr * 256;
     int ring = budget / slot_bytes;
     if (ring > 8) ring = 8;
-    if (ring < 3 || ring < nslots) continue;
+    if (ring < 3 || ring < nslots || (nslots > 1 && ring < 2 * nslots)) continue;   // several slots per item are freed
+                                                                                    // together: room for two items
     const int cost = nslots * (sr + 48);   // operand rows per image, plus a charge per slot for its hand-over
     if (cost < best) {
       best = cost;
