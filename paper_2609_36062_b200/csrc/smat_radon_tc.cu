@@ -22,7 +22,8 @@
 //                    per two operand rows), where the MMAs read it as their A operand
 //   warp 16 lane 0 : TMA producer; a ring slot holds `sps` lines (fixed hi, all lo) of the image x 128 state entries
 //                    (MN-major B operand, two boxes of 64 entries); the extra class travels in a slot of its own
-//   warp 17 lane 0 : MMA issuer, D[128 outputs, 128 entries] += R_slot * B_slot; up to four accumulators in flight
+//   warps 17, 18 (lane 0) : MMA issuers, alternating items: D[128 outputs, 128 entries] += R_slot * B_slot; up to
+//                    four accumulators in flight
 //   warps 0-15     : epilogue, one output index (TMEM lane) per thread and one 32-entry column chunk per warp:
 //                    round to bf16 and store 64 contiguous bytes of the output row as two 32-byte sectors
 #include <cuda.h>
@@ -40,7 +41,8 @@ constexpr int TILE_ROWS = 128;                    // output indices per tile (MM
 constexpr int EPI_WARPS = 16;
 constexpr int PROD_WARP = EPI_WARPS;
 constexpr int MMA_WARP = EPI_WARPS + 1;
-constexpr int RADON_THREADS = 32 * (MMA_WARP + 1);
+constexpr int MMA_WARPS = 2;                      // issuing threads; they take the items alternately
+constexpr int RADON_THREADS = 32 * (MMA_WARP + MMA_WARPS);
 constexpr int MAX_ACC = 4;                        // accumulators in flight: what the R columns leave of 512, at most 4
 constexpr int ROW_INVALID = -1;
 constexpr int ROW_VERT = 1 << 30;                 // flag: row of the extra ("vertical") class
@@ -273,8 +275,10 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
       slab += step;
       while (slab >= slabs) { slab -= slabs; ++img; }
     }
-  } else if (warp == MMA_WARP && lane == 0) {
-    // ---- MMA issuer -------------------------------------------------------------------------------------------
+  } else if (warp >= MMA_WARP && lane == 0) {
+    // ---- MMA issuers: the two threads take the items alternately, so that the issue latency of one item (waits,
+    // MMAs, commits: more than the tensor pipe needs for it) overlaps with the other thread's item ----------------
+    const uint32_t me = (uint32_t)(warp - MMA_WARP);
     constexpr uint32_t idesc = make_idesc(TILE_ROWS, 128, 0, 1);   // A from tensor memory (R), B MN-major (image rows)
     const uint64_t dB0 = make_desc(smem_u32(sRing), prm.sr * 128, 1024);
     const uint32_t slot16 = (uint32_t)slot_bytes >> 4;            // descriptor address units are 16 bytes
@@ -284,22 +288,47 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     uint32_t slot = 0, par = 0;                                   // ring position and the parity its full barrier shows
     uint32_t buf = 0, apar = 0, n_item = 0;                       // accumulator; parity of its empty barrier's phase to wait for
     bool ok = true;
-    for (uint32_t it = first; it < total && ok; it += step, ++n_item) {
-      if (n_item >= nacc) ok = mbar_wait(acc_empty + buf, apar, wc);
-      if (!ok) break;
-      fence_after_sync();
-      const uint32_t tmem_d = tmem_acc + buf * 128;
-      uint32_t tmem_a = tmem_base;
-      for (int g = 0; g < nslots && ok; ++g, tmem_a += slot_cols) {
+    if (nslots == 1) {
+      // One slot per item (q <= 11): a single thread, and the leanest loop: every instruction here is on the
+      // critical path of the stage.
+      for (uint32_t it = first; me == 0 && it < total && ok; it += step, ++n_item) {
+        if (n_item >= nacc) ok = mbar_wait(acc_empty + buf, apar, wc);
+        if (!ok) break;
         ok = mbar_wait(full + slot, par, wc);
         if (!ok) break;
         fence_after_sync();
-        issue_slot_steps(steps, tmem_d, tmem_a, dB0 + (uint64_t)(slot * slot16), idesc, g == 0);
-        if (nslots == 1) mma_commit(empty + slot);   // one slot per item: free it directly (measured faster there)
+        issue_slot_steps(steps, tmem_acc + buf * 128, tmem_base, dB0 + (uint64_t)(slot * slot16), idesc, true);
+        mma_commit(empty + slot);
+        mma_commit(acc_full + buf);
         if (++slot == ring) { slot = 0; par ^= 1; }
+        if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
       }
-      if (ok) mma_commit(acc_full + buf);   // with several slots per item the epilogue frees them when it sees this one
-      if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
+    } else {
+      uint32_t turn = 0;
+      for (uint32_t it = first; it < total && ok; it += step, ++n_item) {
+        const bool mine = turn == me;
+        if (++turn == MMA_WARPS) turn = 0;
+        if (!mine) {   // the other thread's item: step the counters over it
+          for (int g = 0; g < nslots; ++g)
+            if (++slot == ring) { slot = 0; par ^= 1; }
+          if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
+          continue;
+        }
+        if (n_item >= nacc) ok = mbar_wait(acc_empty + buf, apar, wc);
+        if (!ok) break;
+        fence_after_sync();
+        const uint32_t tmem_d = tmem_acc + buf * 128;
+        uint32_t tmem_a = tmem_base;
+        for (int g = 0; g < nslots && ok; ++g, tmem_a += slot_cols) {
+          ok = mbar_wait(full + slot, par, wc);
+          if (!ok) break;
+          fence_after_sync();
+          issue_slot_steps(steps, tmem_d, tmem_a, dB0 + (uint64_t)(slot * slot16), idesc, g == 0);
+          if (++slot == ring) { slot = 0; par ^= 1; }
+        }
+        if (ok) mma_commit(acc_full + buf);   // the only commit of the item: the epilogue frees its slots when it sees it
+        if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
+      }
     }
   } else if (warp < EPI_WARPS) {
     // ---- epilogue ---------------------------------------------------------------------------------------------
