@@ -831,6 +831,29 @@ struct PoolParams {
   int* status;
 };
 
+// One pass of pool_tc_kernel: up to TOK tokens of one (group, head) item.  Every role walks the same sequence.
+template <int TOK>
+struct PoolPass {
+  const PoolParams* pp;
+  int64_t item, stride;          // current item; items advance by the grid size
+  int64_t bh, t_first, t_stride, cnt, k0;
+  __device__ PoolPass(const PoolParams& p, int64_t first, int64_t stride_) : pp(&p), item(first), stride(stride_) { load(); }
+  __device__ void load() {
+    k0 = 0;
+    if (item < pp->items) {
+      bh = item / pp->groups;
+      smat_group_tokens(pp->grp, item - bh * pp->groups, &t_first, &t_stride, &cnt);
+    }
+  }
+  __device__ bool valid() const { return item < pp->items; }
+  __device__ bool first() const { return k0 == 0; }
+  __device__ bool last() const { return k0 + TOK >= cnt; }
+  __device__ int tokens() const { const int64_t left = cnt - k0; return (int)(left < TOK ? (left > 0 ? left : 0) : TOK); }
+  __device__ void next() {
+    if (last()) { item += stride; load(); } else k0 += TOK;
+  }
+};
+
 template <int TOK, int OUT_BF16>
 __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
   constexpr int OP_BYTES = 2 * TOK * 128;  // one operand: two 64-feature blocks of TOK rows x 128 bytes
@@ -860,100 +883,109 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_d = *tmem_slot;
-  uint32_t n_pass = 0, n_item = 0;
   constexpr uint32_t idesc = make_idesc(TILE, TILE, 1, 1);
+  PoolPass<TOK> cur(prm, blockIdx.x, gridDim.x);
 
-  for (int64_t item = blockIdx.x; item < prm.items; item += gridDim.x, ++n_item) {
-    const int64_t bh = item / prm.groups, g = item - bh * prm.groups;
-    int64_t t_first, t_stride, cnt;
-    smat_group_tokens(prm.grp, g, &t_first, &t_stride, &cnt);
-    bool ok = true;
-    for (int64_t k0 = 0; k0 < cnt && ok; k0 += TOK, ++n_pass) {
-      const int kn = (int)((cnt - k0) < TOK ? (cnt - k0) : TOK);
-      const int kpad = (kn + 15) & ~15;
-      if (warp < 4) {
-        const int tid = threadIdx.x;
-        if (n_pass > 0) ok = mbar_wait(bar_d, (n_pass - 1) & 1, wc);  // previous pass has read the tiles
-        if (ok) {
-          const uint32_t a_base = smem_u32(sA), b_base = smem_u32(sB);
-          for (int idx = tid; idx < kpad * 32; idx += 128) {  // 16 chunks of K and 16 of V per token
-            const int k = idx >> 5, w = idx & 31, gc = w & 15;
-            const uint32_t dst = (w < 16 ? a_base : b_base) + (gc >> 3) * (TOK * 128) + k * 128 + (((gc & 7) ^ (k & 7)) << 4);
-            if (k < kn) {
-              const __nv_bfloat16* src = (w < 16 ? prm.K : prm.V) + ((bh * prm.T + t_first + (k0 + k) * t_stride) * TILE + gc * 8);
-              cp_async16_tc(dst, src);
-            } else {
-              asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
-            }
-          }
-          asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
-          fence_proxy_async();
-          mbar_arrive(bar_a);
-        }
-      } else if (lane == 0) {
-        ok = mbar_wait(bar_a, n_pass & 1, wc);
-        if (ok && k0 == 0 && n_item > 0) ok = mbar_wait(bar_e, (n_item - 1) & 1, wc);  // previous state has been read out
-        if (ok) {
-          fence_after_sync();
-          const uint64_t dA = make_desc(smem_u32(sA), TOK * 128, 1024);
-          const uint64_t dB = make_desc(smem_u32(sB), TOK * 128, 1024);
-          for (int kk = 0; kk < kpad / 16; ++kk)
-            mma_bf16(tmem_d, dA + (uint64_t)(kk * 128), dB + (uint64_t)(kk * 128), idesc, (k0 | kk) != 0);
-          mma_commit(bar_d);
-        }
-      }
-      ok = (__shfl_sync(0xffffffffu, (int)ok, 0) != 0) && ok;
-    }
-    if (!ok) break;
-    if (warp < 4) {
-      const int i = warp * 32 + lane;  // state row = TMEM lane
-      bool ok_e = true;
-      if (cnt > 0) ok_e = mbar_wait(bar_d, (n_pass - 1) & 1, wc);
-      ok_e = __all_sync(0xffffffffu, ok_e);
-      if (!ok_e && OUT_BF16) break;
-      if (ok_e) fence_after_sync();
-#pragma unroll
-      for (int cb = 0; cb < 4; ++cb) {
-        uint32_t v[32];
-        if (cnt > 0 && ok_e) {
-          tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
-          tmem_ld_wait();
+  if (warp < 4) {
+    const int tid = threadIdx.x;
+    const int i = warp * 32 + lane;  // state row = TMEM lane
+    const uint32_t a_base = smem_u32(sA), b_base = smem_u32(sB);
+    // 16 chunks of K and 16 of V per token; rows up to the next multiple of 16 are zeroed (a group without tokens
+    // still gets one all-zero pass, so that its state is written as zeros by the same path)
+    auto gather = [&](const PoolPass<TOK>& ps) {
+      const int kn = ps.tokens();
+      const int kpad = kn ? (kn + 15) & ~15 : 16;
+      for (int idx = tid; idx < kpad * 32; idx += 128) {
+        const int k = idx >> 5, w = idx & 31, gc = w & 15;
+        const uint32_t dst = (w < 16 ? a_base : b_base) + (gc >> 3) * (TOK * 128) + k * 128 + (((gc & 7) ^ (k & 7)) << 4);
+        if (k < kn) {
+          const __nv_bfloat16* src = (w < 16 ? prm.K : prm.V) + ((ps.bh * prm.T + ps.t_first + (ps.k0 + k) * ps.t_stride) * TILE + gc * 8);
+          cp_async16_tc(dst, src);
         } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = 0u;  // profile cell without tokens (P > n)
+          asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
         }
-        if (OUT_BF16) {
-          __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(prm.F) + (item * TILE + i) * TILE + cb * 32;
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    uint32_t n_pass = 0;
+    if (cur.valid()) gather(cur);
+    while (cur.valid()) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      fence_proxy_async();
+      mbar_arrive(bar_a);                                    // pass published
+      PoolPass<TOK> nxt = cur;
+      nxt.next();
+      bool ok = mbar_wait(bar_d, n_pass & 1, wc);            // its MMAs have read the tiles (and, on the last pass, the state is complete)
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok && nxt.valid()) gather(nxt);                    // the next tokens travel while the state is written out
+      if (cur.last()) {
+        if (!ok && OUT_BF16) break;
+        if (ok) fence_after_sync();
+        const int64_t item = cur.item;
 #pragma unroll
-          for (int h8 = 0; h8 < 2; ++h8) {  // whole 32-byte sectors
-            uint32_t w[8];
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t v[32];
+          if (ok) {
+            tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+            tmem_ld_wait();
+          } else {
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-              w[e] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * e]), __uint_as_float(v[16 * h8 + 2 * e + 1]));
-            st_global_v8(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+            for (int j = 0; j < 32; ++j) v[j] = 0u;
           }
-        } else {  // fp32 state: through a padded staging tile so that the global writes are whole 512-byte rows
-          uint4* srow = reinterpret_cast<uint4*>(stage + i * STAGE_LD + cb * 32);
+          if (OUT_BF16) {
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(prm.F) + (item * TILE + i) * TILE + cb * 32;
 #pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) srow[q4] = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+            for (int h8 = 0; h8 < 2; ++h8) {  // whole 32-byte sectors
+              uint32_t w[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e)
+                w[e] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * e]), __uint_as_float(v[16 * h8 + 2 * e + 1]));
+              st_global_v8(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+            }
+          } else {  // fp32 state: through a padded staging tile so that the global writes are whole 512-byte rows
+            uint4* srow = reinterpret_cast<uint4*>(stage + i * STAGE_LD + cb * 32);
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) srow[q4] = make_uint4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+          }
         }
-      }
-      if (!OUT_BF16) {
-        fence_before_sync();
-        const bool bad = bar_or_128(!ok_e);  // the four epilogue warps meet here and agree on giving up
-        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.F) + item * (int64_t)(TILE * TILE));
-        const int tid = threadIdx.x;
+        if (!OUT_BF16) {
+          fence_before_sync();
+          const bool bad = bar_or_128(!ok);  // the four epilogue warps meet here and agree on giving up
+          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.F) + item * (int64_t)(TILE * TILE));
 #pragma unroll 4
-        for (int it = 0; it < TILE * TILE / 4 / 128; ++it) {
-          const int idx = it * 128 + tid, r = idx >> 5, c4 = idx & 31;
-          dst[idx] = *reinterpret_cast<const float4*>(stage + r * STAGE_LD + c4 * 4);
+          for (int it = 0; it < TILE * TILE / 4 / 128; ++it) {
+            const int idx = it * 128 + tid, r = idx >> 5, c4 = idx & 31;
+            dst[idx] = *reinterpret_cast<const float4*>(stage + r * STAGE_LD + c4 * 4);
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");  // staging tile free again
+          if (bad) break;
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");  // staging tile free again
-        if (bad) break;
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_e);
+      } else if (!ok) {
+        break;
       }
-      fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_e);
+      cur = nxt;
+      ++n_pass;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else if (lane == 0) {
+    uint32_t n_pass = 0, n_item = 0;
+    bool ok = true;
+    for (; cur.valid() && ok; cur.next(), ++n_pass) {
+      ok = mbar_wait(bar_a, n_pass & 1, wc);
+      if (ok && cur.first() && n_item > 0) ok = mbar_wait(bar_e, (n_item - 1) & 1, wc);  // previous state has been read out
+      if (!ok) break;
+      fence_after_sync();
+      const int kn = cur.tokens();
+      const int kpad = kn ? (kn + 15) & ~15 : 16;
+      const uint64_t dA = make_desc(smem_u32(sA), TOK * 128, 1024);
+      const uint64_t dB = make_desc(smem_u32(sB), TOK * 128, 1024);
+      for (int kk = 0; kk < kpad / 16; ++kk)
+        mma_bf16(tmem_d, dA + (uint64_t)(kk * 128), dB + (uint64_t)(kk * 128), idesc, !(cur.first() && kk == 0));
+      mma_commit(bar_d);
+      if (cur.last()) ++n_item;
     }
   }
   fence_before_sync();
