@@ -703,6 +703,30 @@ __device__ __forceinline__ void cp_async16_tc(uint32_t smem_addr, const void* gm
 
 // TRANS = 0: out[t][j] = Σ_i x_t[i] St[i][j]  (state as MN-major B);  TRANS = 1: out[t][i] = Σ_j x_t[j] St[i][j]
 // (the same two boxes read as a K-major B).
+// One pass of state_read_tc_kernel: up to 128 tokens of one (state, head) item; states without tokens are skipped.
+// Every role walks the same sequence.
+struct ReadPass {
+  const ReadParams* pp;
+  int64_t item, stride;
+  int64_t bh, t_first, t_stride, cnt, k0;
+  __device__ ReadPass(const ReadParams& p, int64_t first, int64_t stride_) : pp(&p), item(first), stride(stride_) { load(); }
+  __device__ void load() {
+    k0 = 0;
+    for (; item < pp->items; item += stride) {
+      bh = item / pp->groups;
+      smat_group_tokens(pp->grp, item - bh * pp->groups, &t_first, &t_stride, &cnt);
+      if (cnt > 0) break;
+    }
+  }
+  __device__ bool valid() const { return item < pp->items; }
+  __device__ bool first() const { return k0 == 0; }
+  __device__ bool last() const { return k0 + TILE >= cnt; }
+  __device__ int tokens() const { const int64_t left = cnt - k0; return (int)(left < TILE ? left : TILE); }
+  __device__ void next() {
+    if (last()) { item += stride; load(); } else k0 += TILE;
+  }
+};
+
 template <int TRANS>
 __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constant__ CUtensorMap tmU,
                                                             const ReadParams prm) {
@@ -730,77 +754,89 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_d = *tmem_slot;
-  uint32_t n_item = 0, n_pass = 0;  // completed uses of bar_u and of bar_a / bar_d / bar_e
   constexpr uint32_t idesc = make_idesc(TILE, TILE, 0, TRANS ? 0 : 1);
+  ReadPass cur(prm, blockIdx.x, gridDim.x);
 
-  for (int64_t item = blockIdx.x; item < prm.items; item += gridDim.x) {
-    const int64_t bh = item / prm.groups, h = item - bh * prm.groups;
-    int64_t t_first, t_stride, cnt;
-    smat_group_tokens(prm.grp, h, &t_first, &t_stride, &cnt);
-    if (cnt == 0) continue;
-    bool ok = true;
-    if (warp == 4 && lane == 0) {
+  if (warp < 4) {
+    const int tid = threadIdx.x;
+    const uint32_t a_base = smem_u32(sA);
+    auto gather = [&](const ReadPass& ps) {
+      const int kn = ps.tokens();
+      for (int idx = tid; idx < kn * 16; idx += 128) {
+        const int m = idx >> 4, gc = idx & 15;
+        const __nv_bfloat16* src = prm.X + ((ps.bh * prm.T + ps.t_first + (ps.k0 + m) * ps.t_stride) * TILE + gc * 8);
+        cp_async16_tc(a_base + (gc >> 3) * BOX_BYTES + m * 128 + (((gc & 7) ^ (m & 7)) << 4), src);
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    uint32_t n_pass = 0;
+    if (cur.valid()) gather(cur);
+    while (cur.valid()) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      fence_proxy_async();
+      mbar_arrive(bar_a);
+      ReadPass nxt = cur;
+      nxt.next();
+      bool ok = mbar_wait(bar_d, n_pass & 1, wc);            // the MMAs have read the query tile; the product is in TMEM
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      if (nxt.valid()) gather(nxt);                          // the next queries travel while this product is written out
+      fence_after_sync();
+      const int m = warp * 32 + lane, kn = cur.tokens();
+      float4* dst = reinterpret_cast<float4*>(prm.out + (cur.bh * prm.T + cur.t_first + (cur.k0 + m) * cur.t_stride) * TILE);
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+        tmem_ld_wait();
+        if (m < kn) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i)   // whole 32-byte sectors
+            st_global_v8(dst + cb * 8 + 2 * i, v[8 * i], v[8 * i + 1], v[8 * i + 2], v[8 * i + 3], v[8 * i + 4],
+                         v[8 * i + 5], v[8 * i + 6], v[8 * i + 7]);
+        }
+      }
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_e);
+      cur = nxt;
+      ++n_pass;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else if (lane == 0) {
+    auto load_state = [&](int64_t item) {
       mbar_expect_tx(bar_u, 2 * BOX_BYTES);
       const int row = (int)(item * TILE);
       tma_load_2d(sB, &tmU, 0, row, bar_u);
       tma_load_2d(sB + BOX_BYTES, &tmU, HALF, row, bar_u);
-    }
-    for (int64_t k0 = 0; k0 < cnt && ok; k0 += TILE, ++n_pass) {
-      const int kn = (int)((cnt - k0) < TILE ? (cnt - k0) : TILE);
-      if (warp < 4) {
-        const int tid = threadIdx.x;
-        const uint32_t a_base = smem_u32(sA);
-        for (int idx = tid; idx < kn * 16; idx += 128) {
-          const int m = idx >> 4, gc = idx & 15;
-          const __nv_bfloat16* src = prm.X + ((bh * prm.T + t_first + (k0 + m) * t_stride) * TILE + gc * 8);
-          cp_async16_tc(a_base + (gc >> 3) * BOX_BYTES + m * 128 + (((gc & 7) ^ (m & 7)) << 4), src);
-        }
-        asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
-        fence_proxy_async();
-        mbar_arrive(bar_a);
-        ok = mbar_wait(bar_d, n_pass & 1, wc);
-        if (ok) {
-          fence_after_sync();
-          const int m = warp * 32 + lane;
-          float4* dst = reinterpret_cast<float4*>(prm.out + (bh * prm.T + t_first + (k0 + m) * t_stride) * TILE);
+    };
+    uint32_t n_item = 0, n_pass = 0;  // completed uses of bar_u and of bar_a / bar_d / bar_e
+    bool ok = true;
+    if (cur.valid()) load_state(cur.item);
+    while (cur.valid() && ok) {
+      if (cur.first()) ok = mbar_wait(bar_u, n_item & 1, wc);
+      if (ok) ok = mbar_wait(bar_a, n_pass & 1, wc);
+      if (ok && n_pass > 0) ok = mbar_wait(bar_e, (n_pass - 1) & 1, wc);  // previous product has been read out
+      if (!ok) break;
+      fence_after_sync();
 #pragma unroll
-          for (int cb = 0; cb < 4; ++cb) {
-            uint32_t v[32];
-            tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
-            tmem_ld_wait();
-            if (m < kn) {
-#pragma unroll
-              for (int i = 0; i < 4; ++i)   // whole 32-byte sectors
-                st_global_v8(dst + cb * 8 + 2 * i, v[8 * i], v[8 * i + 1], v[8 * i + 2], v[8 * i + 3], v[8 * i + 4],
-                             v[8 * i + 5], v[8 * i + 6], v[8 * i + 7]);
-            }
-          }
-          fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_e);
-        }
-      } else if (lane == 0) {
-        if (k0 == 0) ok = mbar_wait(bar_u, n_item & 1, wc);
-        if (ok) ok = mbar_wait(bar_a, n_pass & 1, wc);
-        if (ok && n_pass > 0) ok = mbar_wait(bar_e, (n_pass - 1) & 1, wc);  // previous product has been read out
-        if (ok) {
-          fence_after_sync();
-#pragma unroll
-          for (int kk = 0; kk < TILE / 16; ++kk) {
-            const uint64_t dA = make_desc(smem_u32(sA) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
-            const uint64_t dB = TRANS ? make_desc(smem_u32(sB) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024)
-                                      : make_desc(smem_u32(sB) + kk * 2048, BOX_BYTES, 1024);
-            mma_bf16(tmem_d, dA, dB, idesc, kk != 0);
-          }
-          mma_commit(bar_d);
-          // the operands may be overwritten (next pass or next item) only after the MMA has read them
-          ok = mbar_wait(bar_d, n_pass & 1, wc);
-        }
+      for (int kk = 0; kk < TILE / 16; ++kk) {
+        const uint64_t dA = make_desc(smem_u32(sA) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+        const uint64_t dB = TRANS ? make_desc(smem_u32(sB) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024)
+                                  : make_desc(smem_u32(sB) + kk * 2048, BOX_BYTES, 1024);
+        mma_bf16(tmem_d, dA, dB, idesc, kk != 0);
       }
-      ok = (__shfl_sync(0xffffffffu, (int)ok, 0) != 0) && ok;  // lanes of a warp leave together
+      mma_commit(bar_d);
+      // the state tile may be overwritten (next item) only after the MMAs have read it
+      ok = mbar_wait(bar_d, n_pass & 1, wc);
+      const bool was_last = cur.last();
+      cur.next();
+      ++n_pass;
+      if (was_last) {
+        ++n_item;
+        if (ok && cur.valid()) load_state(cur.item);          // travels while the product is written out
+      }
     }
-    ++n_item;
-    if (!ok) break;
   }
   fence_before_sync();
   __syncthreads();
