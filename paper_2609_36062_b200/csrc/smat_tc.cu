@@ -457,11 +457,14 @@ struct SegOutParams {
 };
 
 // One CTA per (segment, head), all 128 output columns.
-//   warps 0-7 : two warpgroups, each owning one 64-column half of every TMEM tile (state, scores, output)
-//   warp 8    : TMA producer (two stages);   warp 9 : MMA issuer
+//   warps 0-15 : each owns 32 rows x 32 columns of every TMEM tile (state, scores, output)
+//   warp 16    : TMA producer (two stages);   warp 17 : MMA issuer
 // TMEM columns: running state S [0,128), scores [128,256), two output accumulators [256,384) and [384,512).
 // Per tile:  Sc = Q Kᵀ ;  O = Q S_bf16 ;  O += tril(Sc)_bf16 V ;  S += Kᵀ V.
-__global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+constexpr int SEG_EPI_WARPS = 16;
+constexpr int SEG_OUT_THREADS = 32 * (SEG_EPI_WARPS + 2);
+
+__global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                 const __grid_constant__ CUtensorMap tmK,
                                                                 const __grid_constant__ CUtensorMap tmV,
                                                                 const SegOutParams prm) {
@@ -471,10 +474,10 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
   uint64_t* bars = reinterpret_cast<uint64_t*>(sSP + 2 * BOX_BYTES);
   uint64_t* full = bars;          // [2] tile operands landed
   uint64_t* empty = bars + 2;     // [2] tile operands consumed
-  uint64_t* bar_s = bars + 4;     // bf16 state written (256 arrivals)
+  uint64_t* bar_s = bars + 4;     // bf16 state written (one arrival per warp)
   uint64_t* bar_sc = bars + 5;    // scores in TMEM
   uint64_t* bar_qs = bars + 6;    // O = Q S finished: the shared tile may take P
-  uint64_t* bar_p = bars + 7;     // P written (256 arrivals)
+  uint64_t* bar_p = bars + 7;     // P written (one arrival per warp)
   uint64_t* bar_o = bars + 8;     // output in TMEM and state updated
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -484,10 +487,11 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
   if (threadIdx.x == 0) {
     *cta_abort = 0;
     mbar_init(full, 1); mbar_init(full + 1, 1); mbar_init(empty, 1); mbar_init(empty + 1, 1);
-    mbar_init(bar_s, 256); mbar_init(bar_sc, 1); mbar_init(bar_qs, 1); mbar_init(bar_p, 256); mbar_init(bar_o, 1);
+    mbar_init(bar_s, SEG_EPI_WARPS); mbar_init(bar_sc, 1); mbar_init(bar_qs, 1); mbar_init(bar_p, SEG_EPI_WARPS);
+    mbar_init(bar_o, 1);
     fence_barrier_init();
   }
-  if (warp == 8) tmem_alloc(tmem_slot, 512);
+  if (warp == SEG_EPI_WARPS) tmem_alloc(tmem_slot, 512);
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
@@ -495,7 +499,7 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
   const uint32_t tmem_s = tmem_base, tmem_sc = tmem_base + TILE, tmem_o0 = tmem_base + 2 * TILE;
   const int64_t tile0 = (int64_t)seg * prm.L;
 
-  if (warp == 8 && lane == 0) {
+  if (warp == SEG_EPI_WARPS && lane == 0) {
     for (int it = 0; it < prm.L; ++it) {
       const int s = it & 1;
       if (it >= 2 && !mbar_wait(empty + s, ((it >> 1) - 1) & 1, wc)) break;
@@ -509,7 +513,7 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
       tma_load_2d(st + 4 * BOX_BYTES, &tmV, 0, row, full + s);
       tma_load_2d(st + 5 * BOX_BYTES, &tmV, HALF, row, full + s);
     }
-  } else if (warp == 9 && lane == 0) {
+  } else if (warp == SEG_EPI_WARPS + 1 && lane == 0) {
     constexpr uint32_t idesc_sc = make_idesc(TILE, TILE, 0, 0);   // Q Kᵀ: both K-major
     constexpr uint32_t idesc_o = make_idesc(TILE, TILE, 0, 1);    // A K-major (Q or P), B MN-major (S or V)
     constexpr uint32_t idesc_s = make_idesc(TILE, TILE, 1, 1);    // Kᵀ V: both MN-major
@@ -557,120 +561,121 @@ __global__ void __launch_bounds__(320) segment_output_tc_kernel(const __grid_con
       mma_commit(bar_o);
       mma_commit(empty + s);
     }
-  } else if (warp < 8) {
-    const int wg = warp >> 2;                        // column half owned by this warpgroup
+  } else if (warp < SEG_EPI_WARPS) {
+    // Sixteen warps: warp w owns the lane quarter w % 4 (32 rows) and the column quarter w / 4 (32 columns) of every
+    // TMEM tile.  The per-tile work of these threads (convert, store, publish, write out) is the critical path of
+    // the kernel, so it is spread as widely as the TMEM lane rule allows.
+    const int cq = warp >> 2;                        // column quarter
     const int m = (warp & 3) * 32 + lane;            // TMEM lane: state row i / query row of the tile
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t col0 = wg * HALF;
-    uint8_t* my_tile = sSP + wg * BOX_BYTES + m * 128;  // this thread's 128-byte row in its 64-column block
-    // bf16 copy of this thread's 64 state columns (v0, v1) into the shared tile
-    auto publish_state = [&](const uint32_t (&v0)[32], const uint32_t (&v1)[32]) {
+    const uint32_t col0 = cq * 32;
+    // this thread's 64 bytes (four 16-byte chunks) of its row in the 64-column block that holds its columns
+    uint8_t* my_tile = sSP + (cq >> 1) * BOX_BYTES + m * 128;
+    const int ch0 = (cq & 1) * 4;
+    auto store_row = [&](const uint4 (&pk)[4]) {
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const uint32_t* v = c < 4 ? v0 : v1;
-        const int o = (c & 3) * 8;
-        *reinterpret_cast<uint4*>(my_tile + ((c ^ (m & 7)) << 4)) =
-            make_uint4(pack_bf16(__uint_as_float(v[o]), __uint_as_float(v[o + 1])),
-                       pack_bf16(__uint_as_float(v[o + 2]), __uint_as_float(v[o + 3])),
-                       pack_bf16(__uint_as_float(v[o + 4]), __uint_as_float(v[o + 5])),
-                       pack_bf16(__uint_as_float(v[o + 6]), __uint_as_float(v[o + 7])));
-      }
+      for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(my_tile + (((ch0 + c) ^ (m & 7)) << 4)) = pk[c];
+    };
+    // bf16 copy of this thread's 32 state columns into the shared tile
+    auto publish_state = [&](const uint32_t (&v)[32]) {
+      uint4 pk[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        pk[c] = make_uint4(pack_bf16(__uint_as_float(v[8 * c]), __uint_as_float(v[8 * c + 1])),
+                           pack_bf16(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
+                           pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
+                           pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
+      store_row(pk);
       fence_proxy_async();
       fence_before_sync();
-      mbar_arrive(bar_s);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_s);   // one arrival per warp: 512 arrivals on one barrier serialise
     };
     {  // state entering the segment: global fp32 -> TMEM (accumulator) and the shared tile
-      uint32_t v0[32], v1[32];
+      uint32_t v[32];
       const uint4* src = reinterpret_cast<const uint4*>(prm.seg_in + (((int64_t)bh * prm.nseg + seg) * TILE + m) * TILE + col0);
 #pragma unroll
       for (int q4 = 0; q4 < 8; ++q4) {
-        const uint4 a = __ldg(src + q4), b = __ldg(src + 8 + q4);
-        v0[4 * q4] = a.x; v0[4 * q4 + 1] = a.y; v0[4 * q4 + 2] = a.z; v0[4 * q4 + 3] = a.w;
-        v1[4 * q4] = b.x; v1[4 * q4 + 1] = b.y; v1[4 * q4 + 2] = b.z; v1[4 * q4 + 3] = b.w;
+        const uint4 a = __ldg(src + q4);
+        v[4 * q4] = a.x; v[4 * q4 + 1] = a.y; v[4 * q4 + 2] = a.z; v[4 * q4 + 3] = a.w;
       }
-      tmem_st32(tmem_s + lane_base + col0, v0);
-      tmem_st32(tmem_s + lane_base + col0 + 32, v1);
+      tmem_st32(tmem_s + lane_base + col0, v);
       tmem_st_wait();
-      publish_state(v0, v1);
+      publish_state(v);
     }
     for (int it = 0; it < prm.L; ++it) {
       // --- scores of this tile -> masked bf16 P (registers), stored once O = Q S has consumed the shared tile ---
       if (!mbar_wait(bar_sc, it & 1, wc)) break;
       fence_after_sync();
-      uint4 pk[8];
-#pragma unroll
-      for (int cb = 0; cb < 2; ++cb) {
+      uint4 pk[4];
+      {
         uint32_t v[32];
-        tmem_ld32(tmem_sc + lane_base + col0 + cb * 32, v);
+        tmem_ld32(tmem_sc + lane_base + col0, v);
         tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           uint32_t w[4];
 #pragma unroll
           for (int h2 = 0; h2 < 4; ++h2) {
-            const int k0 = (int)col0 + cb * 32 + i * 8 + h2 * 2;
+            const int k0 = (int)col0 + i * 8 + h2 * 2;
             const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
             const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
             w[h2] = pack_bf16(lo, hi);
           }
-          pk[cb * 4 + i] = make_uint4(w[0], w[1], w[2], w[3]);
+          pk[i] = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
       if (!mbar_wait(bar_qs, it & 1, wc)) break;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(my_tile + ((c ^ (m & 7)) << 4)) = pk[c];
+      store_row(pk);
       fence_proxy_async();
       fence_before_sync();
-      mbar_arrive(bar_p);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p);
       // --- long-range rows of this tile, fetched while the MMAs run ---
       const int64_t t = (tile0 + it) * TILE + m;
       const bool add_lr = t >= prm.n_lr;
-      float4 y[16];
+      float4 y[8];
       if (add_lr) {
         const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + col0);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) y[i] = __ldg(y4 + i);
+        for (int i = 0; i < 8; ++i) y[i] = __ldg(y4 + i);
       }
       if (!mbar_wait(bar_o, it & 1, wc)) break;
       fence_after_sync();
       if (it + 1 < prm.L) {  // the state now includes this tile: publish it for the next one first (critical path)
-        uint32_t v0[32], v1[32];
-        tmem_ld32(tmem_s + lane_base + col0, v0);
-        tmem_ld32(tmem_s + lane_base + col0 + 32, v1);
-        tmem_ld_wait();
-        publish_state(v0, v1);
-      }
-      uint4* dst = reinterpret_cast<uint4*>(prm.O + ((int64_t)bh * prm.T + t) * TILE + col0);
-      const uint32_t tmem_o = tmem_o0 + (it & 1) * TILE;
-#pragma unroll
-      for (int cb = 0; cb < 2; ++cb) {
         uint32_t v[32];
-        tmem_ld32(tmem_o + lane_base + col0 + cb * 32, v);
+        tmem_ld32(tmem_s + lane_base + col0, v);
         tmem_ld_wait();
-        uint32_t w[16];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          float f[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i * 8 + e]);
-          if (add_lr) {
-            const float4 a = y[cb * 8 + i * 2], c = y[cb * 8 + i * 2 + 1];
-            f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
-            f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
-          }
-          w[4 * i] = pack_bf16(f[0], f[1]); w[4 * i + 1] = pack_bf16(f[2], f[3]);
-          w[4 * i + 2] = pack_bf16(f[4], f[5]); w[4 * i + 3] = pack_bf16(f[6], f[7]);
-        }
-#pragma unroll
-        for (int h8 = 0; h8 < 2; ++h8)   // whole 32-byte sectors
-          st_global_v8(dst + cb * 4 + 2 * h8, w[8 * h8], w[8 * h8 + 1], w[8 * h8 + 2], w[8 * h8 + 3], w[8 * h8 + 4],
-                       w[8 * h8 + 5], w[8 * h8 + 6], w[8 * h8 + 7]);
+        publish_state(v);
       }
+      __nv_bfloat16* dst = prm.O + ((int64_t)bh * prm.T + t) * TILE + col0;
+      const uint32_t tmem_o = tmem_o0 + (it & 1) * TILE;
+      uint32_t v[32];
+      tmem_ld32(tmem_o + lane_base + col0, v);
+      tmem_ld_wait();
+      uint32_t w[16];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float f[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i * 8 + e]);
+        if (add_lr) {
+          const float4 a = y[i * 2], c = y[i * 2 + 1];
+          f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
+          f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
+        }
+        w[4 * i] = pack_bf16(f[0], f[1]); w[4 * i + 1] = pack_bf16(f[2], f[3]);
+        w[4 * i + 2] = pack_bf16(f[4], f[5]); w[4 * i + 3] = pack_bf16(f[6], f[7]);
+      }
+#pragma unroll
+      for (int h8 = 0; h8 < 2; ++h8)   // whole 32-byte sectors
+        st_global_v8(dst + 16 * h8, w[8 * h8], w[8 * h8 + 1], w[8 * h8 + 2], w[8 * h8 + 3], w[8 * h8 + 4],
+                     w[8 * h8 + 5], w[8 * h8 + 6], w[8 * h8 + 7]);
     }
   }
   fence_before_sync();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == SEG_EPI_WARPS) {
     fence_after_sync();
     tmem_dealloc(tmem_base, 512);
   }
@@ -1221,6 +1226,6 @@ cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const vo
       cudaFuncSetAttribute(segment_output_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_OUT_SMEM);
   if (err != cudaSuccess) return err;
   dim3 grid((unsigned)prm.nseg, (unsigned)bh);
-  segment_output_tc_kernel<<<grid, 320, SEG_OUT_SMEM, st>>>(tmQ, tmK, tmV, prm);
+  segment_output_tc_kernel<<<grid, SEG_OUT_THREADS, SEG_OUT_SMEM, st>>>(tmQ, tmK, tmV, prm);
   return cudaGetLastError();
 }
