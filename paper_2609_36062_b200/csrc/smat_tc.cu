@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
   uint64_t* bar_qk = bars + 0;
   uint64_t* bar_vs = bars + 1;
   uint64_t* bar_sc = bars + 2;   // scores in TMEM
-  uint64_t* bar_p = bars + 3;    // X in shared memory (128 arrivals)
+  uint64_t* bar_p = bars + 3;    // X in shared memory (one arrival per warp)
   uint64_t* bar_o = bars + 4;    // output in TMEM
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
 
   if (threadIdx.x == 0) {
     *cta_abort = 0;
-    mbar_init(bar_qk, 1); mbar_init(bar_vs, 1); mbar_init(bar_sc, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+    mbar_init(bar_qk, 1); mbar_init(bar_vs, 1); mbar_init(bar_sc, 1); mbar_init(bar_p, 4); mbar_init(bar_o, 1);
     fence_barrier_init();
   }
   if (warp == 4) tmem_alloc(tmem_slot, 256);
@@ -301,7 +301,8 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
       }
       fence_proxy_async();
       fence_before_sync();
-      mbar_arrive(bar_p);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p);   // one arrival per warp
       if (mbar_wait(bar_o, 0, wc)) {
         fence_after_sync();
         const int64_t t = (int64_t)b * TILE + m;
@@ -741,7 +742,7 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
   uint8_t* sB = smem + 2 * BOX_BYTES;    // state, MN-major, two 64-column blocks
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 4 * BOX_BYTES);
   uint64_t* bar_u = bars + 0;   // state landed (TMA)
-  uint64_t* bar_a = bars + 1;   // queries landed (128 arrivals)
+  uint64_t* bar_a = bars + 1;   // queries landed (one arrival per warp)
   uint64_t* bar_d = bars + 2;   // product in TMEM
   uint64_t* bar_e = bars + 3;   // TMEM read out (4 arrivals)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
@@ -751,7 +752,7 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
 
   if (threadIdx.x == 0) {
     *cta_abort = 0;
-    mbar_init(bar_u, 1); mbar_init(bar_a, 128); mbar_init(bar_d, 1); mbar_init(bar_e, 4);
+    mbar_init(bar_u, 1); mbar_init(bar_a, 4); mbar_init(bar_d, 1); mbar_init(bar_e, 4);
     fence_barrier_init();
   }
   if (warp == 4) tmem_alloc(tmem_slot, TILE);
@@ -779,7 +780,8 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
     while (cur.valid()) {
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       fence_proxy_async();
-      mbar_arrive(bar_a);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_a);   // one arrival per warp
       ReadPass nxt = cur;
       nxt.next();
       bool ok = mbar_wait(bar_d, n_pass & 1, wc);            // the MMAs have read the query tile; the product is in TMEM
@@ -906,7 +908,7 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
   uint8_t* sB = smem + OP_BYTES;
   float* stage = reinterpret_cast<float*>(smem + 2 * OP_BYTES);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * OP_BYTES + STAGE_BYTES);
-  uint64_t* bar_a = bars + 0;   // operands landed (128 arrivals)
+  uint64_t* bar_a = bars + 0;   // operands landed (one arrival per warp)
   uint64_t* bar_d = bars + 1;   // MMAs of the pass finished
   uint64_t* bar_e = bars + 2;   // state read out of TMEM (4 arrivals)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3);
@@ -916,7 +918,7 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
 
   if (threadIdx.x == 0) {
     *cta_abort = 0;
-    mbar_init(bar_a, 128); mbar_init(bar_d, 1); mbar_init(bar_e, 4);
+    mbar_init(bar_a, 4); mbar_init(bar_d, 1); mbar_init(bar_e, 4);
     fence_barrier_init();
   }
   if (warp == 4) tmem_alloc(tmem_slot, TILE);
@@ -953,7 +955,8 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
     while (cur.valid()) {
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       fence_proxy_async();
-      mbar_arrive(bar_a);                                    // pass published
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_a);                     // pass published (one arrival per warp)
       PoolPass<TOK> nxt = cur;
       nxt.next();
       bool ok = mbar_wait(bar_d, n_pass & 1, wc);            // its MMAs have read the tiles (and, on the last pass, the state is complete)
