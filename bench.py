@@ -37,9 +37,9 @@ SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
 METRIC = "SMat prefill tokens/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant stage per step — the tabulation, two
 # launches of radon_tc_kernel — from the ncu capture summarised in profiles/radon_tc_kernel_t16k_d4_h2.md: taken on
-# the 2-head copy of the workload (279.6 MB) and scaled by heads (every head owns its tables).  At 2 heads about half
+# the 2-head copy of the workload (281.0 MB) and scaled by heads (every head owns its tables).  At 2 heads about half
 # of the stage intermediate W is served by L2; with W fully in DRAM, as at 32 heads, the figure would be 5.97e9.
-NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate_tc"): 279.6e6 * 16}
+NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate_tc"): 281.0e6 * 16}
 
 
 def parse_args():
