@@ -394,14 +394,19 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
         tabulate_tc(cx, "tabulate_tc", cx.ws + pl->off_F, cx.ws + pl->off_U, 0);
       else
         tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
-      if (pl->u_bf16)                                                                        // step 4
-        SMAT_TRY(cx, "read_type_tc", smat_launch_state_read_tc(Q, cx.ws + pl->off_U, ylr, 0, group(pl, SMAT_GM_TYPE),
-                                                               pl->geo.B, pl->T, pl->bh, status, cx.st));
+    }
+    // The two-level causal branch takes the long-range rows as bf16 (half the bytes for the typed read to write and
+    // for the output kernel to fetch); plans whose type table is fp32 use the per-tile form.
+    const int64_t tiles0 = lr ? pl->geo.n / 128 : pl->T / 128, tiles1 = lr ? pl->geo.m / 128 : 0;
+    const int L = ((pl->flags & SMAT_FLAG_PER_TILE_STATES) || (lr && !pl->u_bf16)) ? 1 : smat_segment_tiles(tiles0, tiles1, pl->bh);
+    if (lr) {                                                                                // step 4
+      if (pl->u_bf16)
+        SMAT_TRY(cx, "read_type_tc", smat_launch_state_read_tc(Q, cx.ws + pl->off_U, ylr, L >= 2 ? ylr : nullptr, 0,
+                                                               group(pl, SMAT_GM_TYPE), pl->geo.B, pl->T, pl->bh, status,
+                                                               cx.st));
       else
         state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);
     }
-    const int64_t tiles0 = lr ? pl->geo.n / 128 : pl->T / 128, tiles1 = lr ? pl->geo.m / 128 : 0;
-    const int L = (pl->flags & SMAT_FLAG_PER_TILE_STATES) ? 1 : smat_segment_tiles(tiles0, tiles1, pl->bh);
     if (L >= 2) {  // steps 5-7, two-level: segment totals, scan of the totals, fused per-segment output
       float* seg = cx.f(pl->off_sin);
       const int64_t nseg = pl->T / 128 / L, nseg0 = tiles0 / L;
@@ -485,7 +490,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
       SMAT_TRY(cx, "bwd_chunk_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 0, 1, status, cx.st));
       // dQ: recent rows add U_type dO
       if (pl->u_bf16)
-        SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, lrbuf, 1, types, pl->geo.B,
+        SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, lrbuf, nullptr, 1, types, pl->geo.B,
                                                                  pl->T, pl->bh, status, cx.st));
       else
         state_read(cx, "bwd_dq_type", SMAT_GM_TYPE, dO, cx.f(pl->off_U), 1, nullptr, lrbuf, nullptr);
@@ -493,7 +498,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
                                                                   lrbuf, n, pl->T, dQ, pl->T, pl->bh, status, cx.st));
       // dK: distant rows add F̄_prof v
       if (fbar_is_bf16)
-        SMAT_TRY(cx, "bwd_dk_profile_tc", smat_launch_state_read_tc(V, cx.ws + pl->off_fbar, lrbuf, 1, profs, pl->geo.P,
+        SMAT_TRY(cx, "bwd_dk_profile_tc", smat_launch_state_read_tc(V, cx.ws + pl->off_fbar, lrbuf, nullptr, 1, profs, pl->geo.P,
                                                                     pl->T, pl->bh, status, cx.st));
       else
         state_read(cx, "bwd_dk_profile", SMAT_GM_PROFILE, V, cx.f(pl->off_fbar), 1, nullptr, lrbuf, nullptr);
@@ -501,7 +506,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
                                                                   lrbuf, 0, n, dK, pl->T, pl->bh, status, cx.st));
       // dV: distant rows add F̄_profᵀ k
       if (fbar_is_bf16)
-        SMAT_TRY(cx, "bwd_dv_profile_tc", smat_launch_state_read_tc(K, cx.ws + pl->off_fbar, lrbuf, 0, profs, pl->geo.P,
+        SMAT_TRY(cx, "bwd_dv_profile_tc", smat_launch_state_read_tc(K, cx.ws + pl->off_fbar, lrbuf, nullptr, 0, profs, pl->geo.P,
                                                                     pl->T, pl->bh, status, cx.st));
       else
         state_read(cx, "bwd_dv_profile", SMAT_GM_PROFILE, K, cx.f(pl->off_fbar), 0, nullptr, lrbuf, nullptr);

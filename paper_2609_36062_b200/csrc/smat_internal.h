@@ -106,7 +106,8 @@ cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void
                                         cudaStream_t st);
 // Typed read on tensor cores: ylr[t] = q_tᵀ U_type(t) for recent tokens, U kept as bf16 [bh][B][128][128].
 // (transposed = 1 contracts the second state index instead: out[t] = state · x_t; grp selects types or profiles)
-cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, int transposed,
+// (the rows go to `out` as fp32, or to `out_bf16` when that is non-null)
+cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, void* out_bf16, int transposed,
                                       const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh, int* status,
                                       cudaStream_t st);
 // bf16 -> fp32 copy of a table (debug export).
@@ -124,5 +125,5 @@ int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh);
 cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* totals, int64_t T, int L, int bh,
                                          int* status, cudaStream_t st);
 cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const void* V, const float* seg_in,
-                                          const float* ylr, int64_t n_lr, void* O, int64_t T, int L, int bh,
+                                          const void* ylr_bf16, int64_t n_lr, void* O, int64_t T, int L, int bh,
                                           int* status, cudaStream_t st);

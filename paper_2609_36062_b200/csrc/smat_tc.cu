@@ -452,7 +452,7 @@ struct SegOutParams {
   int L, nseg;
   const float* seg_in;   // [bh][nseg][128][128] state entering each segment
   int64_t n_lr;
-  const float* ylr;
+  const __nv_bfloat16* ylr;   // [bh][T][128] long-range rows, bf16 (rows t >= n_lr are added)
   __nv_bfloat16* O;
   int* status;
 };
@@ -635,11 +635,11 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
       // --- long-range rows of this tile, fetched while the MMAs run ---
       const int64_t t = (tile0 + it) * TILE + m;
       const bool add_lr = t >= prm.n_lr;
-      float4 y[8];
+      uint4 y[4];                                    // 32 bf16 values
       if (add_lr) {
-        const float4* y4 = reinterpret_cast<const float4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + col0);
+        const uint4* y4 = reinterpret_cast<const uint4*>(prm.ylr + ((int64_t)bh * prm.T + t) * TILE + col0);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) y[i] = __ldg(y4 + i);
+        for (int i = 0; i < 4; ++i) y[i] = __ldg(y4 + i);
       }
       if (!mbar_wait(bar_o, it & 1, wc)) break;
       fence_after_sync();
@@ -661,9 +661,12 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
 #pragma unroll
         for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i * 8 + e]);
         if (add_lr) {
-          const float4 a = y[i * 2], c = y[i * 2 + 1];
-          f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
-          f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
+          const uint32_t yy[4] = {y[i].x, y[i].y, y[i].z, y[i].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            f[2 * e] += __uint_as_float(yy[e] << 16);
+            f[2 * e + 1] += __uint_as_float(yy[e] & 0xffff0000u);
+          }
         }
         w[4 * i] = pack_bf16(f[0], f[1]); w[4 * i + 1] = pack_bf16(f[2], f[3]);
         w[4 * i + 2] = pack_bf16(f[4], f[5]); w[4 * i + 3] = pack_bf16(f[6], f[7]);
@@ -699,7 +702,8 @@ struct ReadParams {
   int64_t groups;        // states per head
   int64_t items;         // heads * groups
   const __nv_bfloat16* X;  // [bh][T][128] rows contracted against the state
-  float* out;            // [bh][T][128]
+  float* out;            // [bh][T][128] fp32 rows, or
+  __nv_bfloat16* out_bf16;  // bf16 rows (when non-null)
   int* status;
 };
 
@@ -790,17 +794,30 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
       if (nxt.valid()) gather(nxt);                          // the next queries travel while this product is written out
       fence_after_sync();
       const int m = warp * 32 + lane, kn = cur.tokens();
-      float4* dst = reinterpret_cast<float4*>(prm.out + (cur.bh * prm.T + cur.t_first + (cur.k0 + m) * cur.t_stride) * TILE);
+      const int64_t row = (cur.bh * prm.T + cur.t_first + (cur.k0 + m) * cur.t_stride) * TILE;
+      float4* dst = reinterpret_cast<float4*>(prm.out + row);
+      __nv_bfloat16* dst16 = prm.out_bf16 + row;
 #pragma unroll
       for (int cb = 0; cb < 4; ++cb) {
         uint32_t v[32];
         tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
         tmem_ld_wait();
         if (m < kn) {
+          if (prm.out_bf16) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i)   // whole 32-byte sectors
-            st_global_v8(dst + cb * 8 + 2 * i, v[8 * i], v[8 * i + 1], v[8 * i + 2], v[8 * i + 3], v[8 * i + 4],
-                         v[8 * i + 5], v[8 * i + 6], v[8 * i + 7]);
+            for (int h8 = 0; h8 < 2; ++h8) {
+              uint32_t w[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e)
+                w[e] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * e]), __uint_as_float(v[16 * h8 + 2 * e + 1]));
+              st_global_v8(dst16 + cb * 32 + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)   // whole 32-byte sectors
+              st_global_v8(dst + cb * 8 + 2 * i, v[8 * i], v[8 * i + 1], v[8 * i + 2], v[8 * i + 3], v[8 * i + 4],
+                           v[8 * i + 5], v[8 * i + 6], v[8 * i + 7]);
+          }
         }
       }
       fence_before_sync();
@@ -1136,7 +1153,7 @@ cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K
   return launch_tile_product<false, true, false>(Q, K, dO, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st);
 }
 
-cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, int transposed,
+cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, void* out_bf16, int transposed,
                                       const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh, int* status,
                                       cudaStream_t st) {
   CUtensorMap tmU;
@@ -1145,6 +1162,7 @@ cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, flo
   prm.T = T; prm.grp = grp; prm.groups = groups; prm.items = (int64_t)bh * groups;
   prm.X = static_cast<const __nv_bfloat16*>(X);
   prm.out = out;
+  prm.out_bf16 = static_cast<__nv_bfloat16*>(out_bf16);
   prm.status = status;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
@@ -1215,14 +1233,14 @@ cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* to
 }
 
 cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const void* V, const float* seg_in,
-                                          const float* ylr, int64_t n_lr, void* O, int64_t T, int L, int bh,
+                                          const void* ylr_bf16, int64_t n_lr, void* O, int64_t T, int L, int bh,
                                           int* status, cudaStream_t st) {
   CUtensorMap tmQ, tmK, tmV;
   if (!make_map(&tmQ, Q, (uint64_t)bh * T) || !make_map(&tmK, K, (uint64_t)bh * T) ||
       !make_map(&tmV, V, (uint64_t)bh * T))
     return cudaErrorInvalidValue;
   SegOutParams prm;
-  prm.T = T; prm.L = L; prm.nseg = (int)(T / TILE / L); prm.seg_in = seg_in; prm.n_lr = n_lr; prm.ylr = ylr;
+  prm.T = T; prm.L = L; prm.nseg = (int)(T / TILE / L); prm.seg_in = seg_in; prm.n_lr = n_lr; prm.ylr = static_cast<const __nv_bfloat16*>(ylr_bf16);
   prm.O = static_cast<__nv_bfloat16*>(O);
   prm.status = status;
   cudaError_t err =
