@@ -111,13 +111,13 @@ def stage_work(name: str, T, c, r, p, e, geo, u_bytes=4, f_bytes=4) -> Work:
         "tabulate_tc": Work(0, geo.nnzC * rp, P * sf + B * su),
         "segment_state_tc": Work(2 * T * rp, 0, T * (r + p) * e),
         "segment_scan": Work(0, 0, 0),
-        "segment_output_tc": Work(T * 129 * (r + p) + 4 * T * rp, 0, T * (2 * r + 2 * p) * e + m * p * 4),
+        "segment_output_tc": Work(T * 129 * (r + p) + 4 * T * rp, 0, T * (2 * r + 2 * p) * e + m * p * 2),
         "chunk_state": Work(2 * T * rp, 0, T * (r + p) * e + NC * st),
         "scan":        Work(0, NC * rp, 2 * NC * st),
         "scores":      Work(T * (c + 1) * r, 0, 2 * T * r * e + T * c * 4),
         "read_chunk":  Work(2 * T * rp, 0, T * r * e + NC * st + T * p * 4),
         "read_type":   Work(2 * m * rp, 0, m * r * e + B * st + 2 * m * p * 4),
-        "read_type_tc": Work(2 * m * rp, 0, m * r * e + B * su + m * p * 4),
+        "read_type_tc": Work(2 * m * rp, 0, m * r * e + B * su + m * p * 2),
         "chunk_scan_tc": Work(2 * T * rp, tc_tiles * rp, T * (r + p) * e + tc_tiles * rp * 2),
         "chunk_output_tc": Work(T * 129 * (r + p) + 2 * T * rp, 0, T * (2 * r + 2 * p) * e + tc_tiles * rp * 2 + m * p * 4),
         "output":      Work(T * (c + 1) * p, 0, T * c * 4 + T * p * e + T * p * 4 + T * p * e),
