@@ -207,6 +207,28 @@ int smat_profile_read(const smat_plan* plan, const char** names, float* ms, int 
 smat_status smat_forward_causal_static(const void* Q, const void* K, const void* V, void* O, int batch, int heads,
                                        int64_t T, void* cuda_stream);
 
+/* ---- Cached decoding of the recent block (Sec. "Memory-efficient decoding", Theorem "Streaming decoding") ----
+ * The plan fixes T and with it the boundary n.  After the distant block (tokens 0 .. n-1) the decoder keeps B type
+ * states U_h and one running state S per (batch, head); each recent token t = n, n+1, ... then costs O(d_k d_v):
+ *     S_t = S_{t-1} + k_t v_t^T   (S_{n-1} = 0),      o_t = q_t^T (U_type(t) + S_t),     type(t) = (t - n + 1) mod B.
+ * o_t equals row t of smat_forward's O (no normaliser, like the rest of the library).
+ *
+ * cache: device memory owned by the caller, 256-byte aligned, smat_decode_cache_bytes(plan) bytes:
+ *        the type table [B*H][B][d_k][d_v] in the element type smat_type_table_element_bytes reports (fp32 for d = 1),
+ *        then S [B*H][d_k][d_v] in fp32.
+ * smat_decode_begin : K [B,H,T,d_k], V [B,H,T,d_v] device pointers of which rows 0 .. n-1 of every head are read;
+ *        pools and tabulates them (steps 2-3 of Algorithm 1, through `workspace` as smat_forward would), stores the
+ *        type table in the cache and zeroes S.  workspace: as for smat_forward (for_backward = 0).
+ * smat_decode_step  : q, k [B,H,d_k], v [B,H,d_v] device rows of token t for every (batch, head) in the plan's dtype,
+ *        o [B,H,d_v] device output in the same dtype.  Steps must be issued for t = n, n+1, ... in order, on one
+ *        stream (S is updated in place).  n <= t < T, else SMAT_ERR_SHAPE.
+ * Both launch on the given stream and return without synchronising; errors as for smat_forward. */
+size_t smat_decode_cache_bytes(const smat_plan* plan);
+smat_status smat_decode_begin(const smat_plan* plan, const void* K, const void* V, void* cache, size_t cache_bytes,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+smat_status smat_decode_step(const smat_plan* plan, const void* q, const void* k, const void* v, int64_t t, void* o,
+                             void* cache, size_t cache_bytes, void* cuda_stream);
+
 /* Number of kernels the last smat_forward / smat_backward on this plan launched (host counter). */
 int smat_last_launch_count(const smat_plan* plan);
 

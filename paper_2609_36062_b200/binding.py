@@ -26,7 +26,7 @@ EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
     "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
-    "smat_profile_table_element_bytes",
+    "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step",
 ]
 
 
@@ -93,6 +93,12 @@ def load_library() -> ctypes.CDLL:
     lib.smat_last_launch_count.restype = i
     lib.smat_type_table_element_bytes.argtypes = [vp]
     lib.smat_type_table_element_bytes.restype = i
+    lib.smat_decode_cache_bytes.argtypes = [vp]
+    lib.smat_decode_cache_bytes.restype = ctypes.c_size_t
+    lib.smat_decode_begin.argtypes = [vp, vp, vp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
+    lib.smat_decode_begin.restype = i
+    lib.smat_decode_step.argtypes = [vp, vp, vp, vp, i64, vp, vp, ctypes.c_size_t, vp]
+    lib.smat_decode_step.restype = i
     lib.smat_profile_table_element_bytes.argtypes = [vp]
     lib.smat_profile_table_element_bytes.restype = i
     lib.smat_uses_tensor_cores.argtypes = [vp]
@@ -239,6 +245,28 @@ class SmatPlan:
         _check(self.lib.smat_backward(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(dQ), _ptr(dK), _ptr(dV),
                                       _ptr(ws), ws.numel(), _stream(stream)), "smat_backward")
         return dQ, dK, dV
+
+    # -- cached decoding -----------------------------------------------------------------------
+    def decode_cache(self, device="cuda") -> torch.Tensor:
+        return torch.empty(int(self.lib.smat_decode_cache_bytes(self.handle)), dtype=torch.uint8, device=device)
+
+    def decode_begin(self, K, V, cache, workspace=None, stream=None) -> None:
+        _, _, _, dk, dv = self.shape
+        self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
+        ws = self.workspace(False, K.device) if workspace is None else workspace
+        self._ws = ws
+        _check(self.lib.smat_decode_begin(self.handle, _ptr(K), _ptr(V), _ptr(cache), cache.numel(), _ptr(ws), ws.numel(),
+                                          _stream(stream)), "smat_decode_begin")
+
+    def decode_step(self, q, k, v, t: int, cache, o=None, stream=None):
+        b, h, _, dk, dv = self.shape
+        for name, x, dim in (("q", q, dk), ("k", k, dk), ("v", v, dv)):
+            if not (x.is_cuda and x.is_contiguous() and x.dtype == self.torch_dtype and tuple(x.shape) == (b, h, dim)):
+                raise ValueError(f"{name}: expected a contiguous CUDA tensor [{b}, {h}, {dim}] of the plan's dtype")
+        o = torch.empty_like(v) if o is None else o
+        _check(self.lib.smat_decode_step(self.handle, _ptr(q), _ptr(k), _ptr(v), int(t), _ptr(o), _ptr(cache), cache.numel(),
+                                         _stream(stream)), "smat_decode_step")
+        return o
 
     # -- verification exports ------------------------------------------------------------------
     def routing_indices(self):

@@ -261,6 +261,37 @@ void build_forward_tables(Ctx& cx, const void* K, const void* V) {
   scan_states(cx, "scan", cx.f(pl->off_sin), 0);                                                           // step 6
 }
 
+// Steps 2-3 of Algorithm 1 alone, as the plan's forward runs them: the type table U ends in the workspace at the
+// returned offset (d = 1: the single state U_0 = F_0, fp32).
+size_t build_type_table(Ctx& cx, const void* K, const void* V) {
+  const smat_plan* pl = cx.pl;
+  if (pl->geo.dense_G) {
+    outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_sin));
+    return pl->off_sin;
+  }
+  if (pl->tc) {
+    int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
+    if (pl->pool_tc)
+      SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, group(pl, SMAT_GM_PROFILE),
+                                                  pl->geo.P, max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh,
+                                                  status, cx.st));
+    else
+      outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
+    if (pl->tab_tc)
+      tabulate_tc(cx, "tabulate_tc", cx.ws + pl->off_F, cx.ws + pl->off_U, 0);
+    else
+      tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
+  } else {
+    outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
+    tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0);
+  }
+  return pl->off_U;
+}
+
+size_t decode_table_bytes(const smat_plan* pl) {
+  return align_up((size_t)pl->bh * pl->geo.B * pl->rp * (pl->u_bf16 ? 2 : 4));
+}
+
 }  // namespace
 
 extern "C" {
@@ -633,6 +664,47 @@ smat_status smat_check_status(const smat_plan* pl, const void* workspace, void* 
 }
 
 int smat_last_launch_count(const smat_plan* pl) { return pl ? pl->launches : 0; }
+
+size_t smat_decode_cache_bytes(const smat_plan* pl) {
+  if (!pl) return 0;
+  return decode_table_bytes(pl) + (size_t)pl->bh * pl->rp * sizeof(float);
+}
+
+smat_status smat_decode_begin(const smat_plan* pl, const void* K, const void* V, void* cache, size_t cache_bytes,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!K || !V || !cache) return SMAT_ERR_NULL;
+  smat_status s = check_common(pl, workspace, workspace_bytes, 0);
+  if (s != SMAT_OK) return s;
+  if (cache_bytes < smat_decode_cache_bytes(pl)) return SMAT_ERR_WORKSPACE;
+  if (misaligned(K) || misaligned(V) || (reinterpret_cast<uintptr_t>(cache) & 255)) return SMAT_ERR_ALIGN;
+  Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
+  pl->stages = 0;
+  pl->last_was_forward = false;
+  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  const size_t off = build_type_table(cx, K, V);
+  const size_t tbytes = (size_t)pl->bh * pl->geo.B * pl->rp * (pl->u_bf16 ? 2 : 4);
+  if (cx.err == cudaSuccess)
+    cx.err = cudaMemcpyAsync(cache, cx.ws + off, tbytes, cudaMemcpyDeviceToDevice, cx.st);
+  if (cx.err == cudaSuccess)
+    cx.err = cudaMemsetAsync(static_cast<char*>(cache) + decode_table_bytes(pl), 0, (size_t)pl->bh * pl->rp * sizeof(float),
+                             cx.st);
+  pl->launches = cx.launches;
+  return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
+smat_status smat_decode_step(const smat_plan* pl, const void* q, const void* k, const void* v, int64_t t, void* o,
+                             void* cache, size_t cache_bytes, void* cuda_stream) {
+  if (!pl || !q || !k || !v || !o || !cache) return SMAT_ERR_NULL;
+  if (cache_bytes < smat_decode_cache_bytes(pl)) return SMAT_ERR_WORKSPACE;
+  if (t < pl->geo.n || t >= pl->T) return SMAT_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(cache) & 255) return SMAT_ERR_ALIGN;
+  float* S = reinterpret_cast<float*>(static_cast<char*>(cache) + decode_table_bytes(pl));
+  const cudaError_t err = smat_launch_decode_step(q, k, v, o, S, cache, pl->u_bf16 ? 1 : 0, pl->dtype == SMAT_BF16 ? 1 : 0,
+                                                  smat_type_of(pl->geo, t), pl->geo.B, pl->r, pl->p, pl->bh,
+                                                  static_cast<cudaStream_t>(cuda_stream));
+  pl->launches = 1;
+  return err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
 
 const char* smat_status_string(smat_status s) {
   switch (s) {

@@ -110,6 +110,10 @@ cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void
 cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, void* out_bf16, int transposed,
                                       const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh, int* status,
                                       cudaStream_t st);
+// One step of cached decoding: S += k vᵀ, o = qᵀ (U_type + S) for every head (fp32 running state).
+cudaError_t smat_launch_decode_step(const void* q, const void* k, const void* v, void* o, float* S, const void* U,
+                                    int u_bf16, int in_bf16, int64_t type, int64_t types, int r, int p, int bh,
+                                    cudaStream_t st);
 // bf16 -> fp32 copy of a table (debug export).
 // Tabulation on the tensor cores (bf16 tables; d = 3, 4 with a prime small enough for a resident Radon matrix).
 int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems);
