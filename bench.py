@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--no-sweep", action="store_true", help="skip the short runs of the other workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="plan flags (see include/smat.h)")
+    ap.add_argument("--decode-only", action="store_true",
+                    help="only the cached-decoding measurement, on --workload (a decode_* workload); prints its JSON object")
     return ap.parse_args()
 
 
@@ -371,6 +373,38 @@ def dominant_kernel_report(w, geo, stages, peaks, u_bytes=4, f_bytes=4):
             "kernels_ms": {n: round(t_, 4) for n, t_ in stages}}
 
 
+def decode_report(torch, binding, peaks, steps=64, name="decode_t2k_d3"):
+    """Cached decoding (one token per sequence and step): steps/s, tokens/s and the fraction of the HBM peak of the
+    step kernel, whose algorithmic bytes per head are the running state read and written (fp32) and one type state."""
+    w = synth.WORKLOADS[name]
+    plan = binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype)
+    g = plan.geometry()
+    host = make_inputs(w, torch)
+    K, V = host["k"].cuda(), host["v"].cuda()
+    cache = plan.decode_cache()
+    plan.decode_begin(K, V, cache)
+    rows = {x: [host[x][:, :, t].contiguous().cuda() for t in range(g.n, g.n + 8)] for x in ("q", "k", "v")}
+    o = torch.empty_like(rows["v"][0])
+    def run(count, t0):
+        for i in range(count):
+            plan.decode_step(rows["q"][i % 8], rows["k"][i % 8], rows["v"][i % 8], t0 + i, cache, o)
+    run(8, g.n)
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    run(steps, g.n + 8)
+    end.record()
+    torch.cuda.synchronize()
+    plan.check_status()
+    sec = start.elapsed_time(end) / 1e3 / steps
+    state = w.d_k * w.d_v
+    by = w.bh * state * (4 + 4 + plan.type_table_element_bytes())
+    return {"workload": w.name, "batch": w.batch, "heads": w.heads, "type_states_B": g.B, "us_per_step": 1e6 * sec,
+            "value": w.batch / sec, "unit": "tokens/s", "cache_bytes": int(cache.numel()),
+            "roofline": {"bound": "hbm", "achieved": by / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": by / sec / 1e9 / peaks["hbm_gbs"], "algorithmic_bytes": by, "traffic": None}}
+
+
 def run_native(args):
     import torch
     import torch.distributed as dist
@@ -391,6 +425,11 @@ def run_native(args):
         barrier = dist.barrier
 
     peaks = roofline.load_peaks(ROOT)
+    if args.decode_only:
+        if rank == 0:
+            name = args.workload if args.workload.startswith("decode") else "decode_t2k_d3"
+            print(json.dumps(decode_report(torch, binding, peaks, max(8, args.steps), name)))
+        return
     w = synth.WORKLOADS[args.workload]
     steps, warm = max(1, args.steps), max(3, args.warmup)
     runner = Runner(w, torch, binding, args.flags)
@@ -449,6 +488,7 @@ def run_native(args):
             del r
             torch.cuda.empty_cache()
         line["sweep"] = sweep
+        line["decode"] = decode_report(torch, binding, peaks)
 
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:

@@ -65,6 +65,10 @@ WORKLOADS = {
     "t64k_d1_h4":    Workload("t64k_d1_h4", 1, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t64k_d2_h4":    Workload("t64k_d2_h4", 2, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t8k_d3_fwdbwd": Workload("t8k_d3_fwdbwd", 3, 8, 16, 8192, 128, 128, 64, "bf16", "normalised", 4, True),
+    # cached decoding: 128 sequences of 16 heads, 2 K horizon (132 type states + one running state per head; the
+    # running states alone, 134 MB, exceed L2)
+    "decode_t2k_d3": Workload("decode_t2k_d3", 3, 128, 16, 2048, 128, 128, 64, "bf16", "normalised", 5),
+    "decode_t2k_d3_b32": Workload("decode_t2k_d3_b32", 3, 32, 16, 2048, 128, 128, 64, "bf16", "normalised", 5),
 }
 
 
