@@ -27,6 +27,7 @@ struct smat_plan {
   bool pool_tc;        // forward pools the profile table on the tensor cores (enough tokens per profile)
   bool f_bf16;         // the profile table is kept in bf16 (d = 2: it is the type table; tab_tc: it is an MMA operand)
   bool tab_tc;         // d = 3, 4: tabulation and its transpose on the tensor cores (bf16 tables, resident Radon matrix)
+  bool tab_d3_bf16;    // d = 3 with a prime too large for that kernel: bf16 profile table, sums on the fp32 ALUs
   mutable int launches;
   mutable bool last_was_forward;  // which call left its tables in the workspace
   // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
@@ -279,6 +280,9 @@ size_t build_type_table(Ctx& cx, const void* K, const void* V) {
       outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
     if (pl->tab_tc)
       tabulate_tc(cx, "tabulate_tc", cx.ws + pl->off_F, cx.ws + pl->off_U, 0);
+    else if (pl->tab_d3_bf16)
+      SMAT_TRY(cx, "tabulate_bf16", smat_launch_tabulate_d3_bf16(cx.ws + pl->off_F, cx.ws + pl->off_U, pl->geo, pl->rp,
+                                                                  pl->bh, cx.st));
     else
       tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
   } else {
@@ -321,8 +325,11 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   // d >= 3 on the tensor-core path: U is only ever a bf16 MMA operand, so it is stored as bf16 (half the bytes)
   pl->tab_tc = pl->tc && !g.dense_G && !(flags & (SMAT_FLAG_ALG2_TABULATION | SMAT_FLAG_ALU_TABULATION)) &&
                smat_tabulate_tc_supported(g, pl->rp);
-  pl->pool_tc = pl->tc && !g.dense_G && (g.n / g.P >= 12 || pl->tab_tc);
-  pl->f_bf16 = pl->pool_tc && ((g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION)) || pl->tab_tc);
+  pl->tab_d3_bf16 = pl->tc && g.D == 2 && !pl->tab_tc &&
+                    !(flags & (SMAT_FLAG_ALG2_TABULATION | SMAT_FLAG_ALU_TABULATION)) &&
+                    smat_tabulate_d3_bf16_slab(g, pl->rp) > 0;
+  pl->pool_tc = pl->tc && !g.dense_G && (g.n / g.P >= 12 || pl->tab_tc || pl->tab_d3_bf16);
+  pl->f_bf16 = pl->pool_tc && ((g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION)) || pl->tab_tc || pl->tab_d3_bf16);
   pl->u_bf16 = pl->f_bf16 || (pl->tc && g.D >= 2 && !(flags & SMAT_FLAG_ALG2_TABULATION) &&
                               smat_tabulate_staged_slab(g, pl->rp, 0) >= 4);
   const size_t state = (size_t)pl->rp * sizeof(float);
@@ -414,18 +421,7 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
     int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
     float* ylr = cx.f(pl->off_acc);
     const bool lr = !pl->geo.dense_G;
-    if (lr) {
-      if (pl->pool_tc)                                                                       // step 2
-        SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, group(pl, SMAT_GM_PROFILE),
-                                                    pl->geo.P, max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh,
-                                                    status, cx.st));
-      else
-        outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
-      if (pl->tab_tc)                                                                        // step 3
-        tabulate_tc(cx, "tabulate_tc", cx.ws + pl->off_F, cx.ws + pl->off_U, 0);
-      else
-        tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
-    }
+    if (lr) build_type_table(cx, K, V);                                                      // steps 2-3
     // The two-level causal branch takes the long-range rows as bf16 (half the bytes for the typed read to write and
     // for the output kernel to fetch); plans whose type table is fp32 use the per-tile form.
     const int64_t tiles0 = lr ? pl->geo.n / 128 : pl->T / 128, tiles1 = lr ? pl->geo.m / 128 : 0;
@@ -490,18 +486,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
     const int64_t n = pl->geo.n;
     const bool fbar_bf16 = pl->u_bf16 && pl->geo.D <= 2;  // F̄ readable by the tensor-core read (d = 2, 3)
     if (lr) {
-      if (!(pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES)) {
-        if (pl->pool_tc)
-          SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, profs, pl->geo.P,
-                                                      max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh, status,
-                                                      cx.st));
-        else
-          outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
-        if (pl->tab_tc)
-          tabulate_tc(cx, "tabulate_tc", cx.ws + pl->off_F, cx.ws + pl->off_U, 0);
-        else
-          tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0, pl->u_bf16);
-      }
+      if (!(pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES)) build_type_table(cx, K, V);
       // Ū_h = Σ q dOᵀ over the type (Eq. "lr-adjoint"), then F̄ = Cᵀ Ū
       const bool ubar_tc = pl->tab_tc || pl->geo.m / pl->geo.B >= 12;
       const bool ubar_bf16 = ubar_tc && ((pl->geo.D == 1 && fbar_bf16) || pl->tab_tc);  // d = 2: F̄ is Ū itself

@@ -114,6 +114,10 @@ cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, flo
 cudaError_t smat_launch_decode_step(const void* q, const void* k, const void* v, void* o, float* S, const void* U,
                                     int u_bf16, int in_bf16, int64_t type, int64_t types, int r, int p, int bh,
                                     cudaStream_t st);
+// d = 3 tabulation from a bf16 profile table on the fp32 ALUs (primes too large for the resident-matrix kernel).
+int smat_tabulate_d3_bf16_slab(const SmatGeo& geo, int64_t state_elems);
+cudaError_t smat_launch_tabulate_d3_bf16(const void* in, void* out, const SmatGeo& geo, int64_t state_elems, int bh,
+                                         cudaStream_t st);
 // bf16 -> fp32 copy of a table (debug export).
 // Tabulation on the tensor cores (bf16 tables; d = 3, 4 with a prime small enough for a resident Radon matrix).
 int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems);

@@ -392,6 +392,87 @@ cudaError_t smat_launch_tabulate_staged(const float* in, void* out, const SmatGe
   return cudaGetLastError();
 }
 
+// ---- d = 3 with bf16 tables and a prime too large for the resident-matrix kernel --------------------------------
+// U = R F (the two-dimensional Radon sums of Algorithm 2 for d = 3) from a bf16 profile table: the slab F[:, e0 .. e0+E)
+// sits in shared memory as bf16, a thread owns 8 entries of one output row and adds in fp32.  Against the fp32 form
+// this halves the shared-memory bytes per addition, which is what bounds these sums.
+__global__ void __launch_bounds__(256) tabulate_d3_bf16_kernel(const __nv_bfloat16* __restrict__ in,
+                                                               __nv_bfloat16* __restrict__ out, int q, int64_t P,
+                                                               int64_t Bn, int64_t state_elems, int E) {
+  extern __shared__ __align__(16) uint4 smem8[];            // [P][E / 8]: 8 bf16 per element
+  const int L8 = E / 8, NT = blockDim.x, tid = threadIdx.x;
+  const int l = tid % L8, it0 = tid / L8, IPP = NT / L8;
+  const int64_t bh = blockIdx.y, e0 = (int64_t)blockIdx.x * E;
+  const int qq = q * q;
+  const uint4* src = reinterpret_cast<const uint4*>(in + (bh * P) * state_elems + e0);
+  const int64_t row8 = state_elems / 8;
+  for (int64_t idx = tid; idx < P * L8; idx += NT) {
+    const int64_t x = idx / L8;
+    cp_async16(smem8 + idx, src + x * row8 + (idx - x * L8));
+  }
+  cp_async_wait_all();
+  __syncthreads();
+  uint4* dst = reinterpret_cast<uint4*>(out + (bh * Bn) * state_elems + e0);
+  auto add8 = [](float (&acc)[8], const uint4 w) {
+    const uint32_t v[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 s = __fadd2_rn(make_float2(acc[2 * i], acc[2 * i + 1]),
+                                  make_float2(__uint_as_float(v[i] << 16), __uint_as_float(v[i] & 0xffff0000u)));
+      acc[2 * i] = s.x; acc[2 * i + 1] = s.y;
+    }
+  };
+  auto store8 = [&](int64_t row, const float (&acc)[8]) {
+    uint4 w;
+    const __nv_bfloat162 a = __floats2bfloat162_rn(acc[0], acc[1]), b = __floats2bfloat162_rn(acc[2], acc[3]),
+                         c = __floats2bfloat162_rn(acc[4], acc[5]), d = __floats2bfloat162_rn(acc[6], acc[7]);
+    w.x = *reinterpret_cast<const uint32_t*>(&a); w.y = *reinterpret_cast<const uint32_t*>(&b);
+    w.z = *reinterpret_cast<const uint32_t*>(&c); w.w = *reinterpret_cast<const uint32_t*>(&d);
+    dst[row * row8 + l] = w;
+  };
+  // a = (1, a2):  U[a2*q + b] = Σ_{x2} F[(b - a2 x2) mod q, x2]
+  for (int item = it0; item < qq; item += IPP) {
+    const int a2 = item / q, b = item - a2 * q;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    int x1 = b;
+#pragma unroll 4
+    for (int x2 = 0; x2 < q; ++x2) {
+      add8(acc, smem8[(x1 + q * x2) * L8 + l]);
+      x1 -= a2;
+      if (x1 < 0) x1 += q;
+    }
+    store8(item, acc);
+  }
+  // a = (0, 1):  U[q*q + b] = Σ_{x1} F[x1, b]
+  for (int b = it0; b < q; b += IPP) {
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+    for (int x1 = 0; x1 < q; ++x1) add8(acc, smem8[(x1 + q * b) * L8 + l]);
+    store8(qq + b, acc);
+  }
+}
+
+// Entries per CTA slab of tabulate_d3_bf16_kernel (two CTAs per SM), or 0 when the geometry is not covered.
+int smat_tabulate_d3_bf16_slab(const SmatGeo& geo, int64_t state_elems) {
+  if (geo.D != 2) return 0;
+  for (int E = 32; E >= 8; E >>= 1)
+    if (geo.P * E * 2 <= 110 * 1024 && state_elems % E == 0) return E;
+  return 0;
+}
+
+cudaError_t smat_launch_tabulate_d3_bf16(const void* in, void* out, const SmatGeo& geo, int64_t state_elems, int bh,
+                                         cudaStream_t st) {
+  const int E = smat_tabulate_d3_bf16_slab(geo, state_elems);
+  if (!E) return cudaErrorInvalidConfiguration;
+  const size_t smem = (size_t)geo.P * E * 2;
+  cudaError_t err = set_smem(tabulate_d3_bf16_kernel, smem);
+  if (err != cudaSuccess) return err;
+  dim3 grid((unsigned)(state_elems / E), (unsigned)bh);
+  tabulate_d3_bf16_kernel<<<grid, 256, smem, st>>>(static_cast<const __nv_bfloat16*>(in), static_cast<__nv_bfloat16*>(out),
+                                                   geo.q, geo.P, geo.B, state_elems, E);
+  return cudaGetLastError();
+}
+
 cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st) {
   widen_bf16_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src_bf16), dst,
                                                                      count);

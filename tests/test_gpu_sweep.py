@@ -11,7 +11,8 @@ pytestmark = pytest.mark.gpu
 # d, T, chunk, q (0 = the default rule)
 CASES = [
     (3, 1024, 128, 2), (3, 1536, 128, 3), (3, 2048, 64, 5), (3, 2304, 128, 7), (3, 2560, 128, 11), (3, 3072, 128, 19),
-    (3, 2048, 128, 23),                     # q = 23: outside the resident-matrix kernel, staged sums on the ALUs
+    (3, 2048, 128, 23),                     # q = 23: outside the resident-matrix kernel, bf16 tables summed on the ALUs
+    (3, 4096, 128, 37),                     # q = 37, the prime of the 64 K configuration with d = 3
     (4, 1024, 128, 2), (4, 1280, 128, 3), (4, 2048, 32, 13), (4, 1792, 128, 19), (4, 2048, 128, 0),
     (2, 1792, 128, 0), (2, 3072, 64, 29), (1, 1792, 128, 0),
 ]
