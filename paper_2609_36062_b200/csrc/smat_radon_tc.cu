@@ -24,8 +24,17 @@
 //                    (MN-major B operand, two boxes of 64 entries); the extra class travels in a slot of its own
 //   warps 17, 18 (lane 0) : MMA issuers, alternating items: D[128 outputs, 128 entries] += R_slot * B_slot; up to
 //                    four accumulators in flight
-//   warps 0-15     : epilogue, one output index (TMEM lane) per thread and one 32-entry column chunk per warp:
-//                    round to bf16 and store 64 contiguous bytes of the output row as two 32-byte sectors
+//   warps 0-15     : epilogue in two groups of 8 warps that alternate items; one output index (TMEM lane) per
+//                    thread and one 64-entry column half per warp: round to bf16 and store 128 contiguous bytes of
+//                    the output row as 32-byte sectors
+//   warps 19, 20   : q = 11 only.  q^2 + q = 132 output indices are one tile of 128 and 4 left over, all of the extra
+//                    class (the sum of one line's q rows): these warps add them up from the ring slot itself, so
+//                    that one CTA covers an image instead of two CTAs loading it twice
+// d = 4 with q <= 11: both stages in ONE launch, slab by slab.  Stage 2 of a slab needs stage 1 of every image of the
+// same slab and nothing else, so a CTA keeps the slab's W rows in a private exchange buffer (q^3 + q^2 rows of 128
+// entries, rewritten for every slab, stored and loaded with the L2 evict-last priority while F and U stream with
+// evict-first) and the full-size W table is never built.  The storing warps make the slab's rows visible (memory
+// fence, proxy fence) and arrive on a barrier the producer waits on before the first stage-2 load.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -42,7 +51,10 @@ constexpr int EPI_WARPS = 16;
 constexpr int PROD_WARP = EPI_WARPS;
 constexpr int MMA_WARP = EPI_WARPS + 1;
 constexpr int MMA_WARPS = 2;                      // issuing threads; they take the items alternately
-constexpr int RADON_THREADS = 32 * (MMA_WARP + MMA_WARPS);
+constexpr int ALU_WARP = MMA_WARP + MMA_WARPS;    // first of the warps that sum the leftover extra-class rows
+constexpr int ALU_WARPS = 2;
+constexpr int ALU_MAX_ROWS = 8;
+constexpr int RADON_THREADS = 32 * (ALU_WARP + ALU_WARPS);
 constexpr int MAX_ACC = 4;                        // accumulators in flight: what the R columns leave of 512, at most 4
 constexpr int ROW_INVALID = -1;
 constexpr int ROW_VERT = 1 << 30;                 // flag: row of the extra ("vertical") class
@@ -57,20 +69,63 @@ struct RadonSide {
   int64_t rows_per_head;
 };
 
+// One stage: input and output index spaces, and where the rows live.  A "private" table is the exchange buffer of the
+// two-stage kernel: [CTA][rows_per_head][128 entries], one slab per CTA, rewritten for every slab so that it stays in L2.
+struct RadonPhase {
+  RadonSide in, out;
+  int32_t images;
+  int32_t src_private, dst_private;
+  int32_t src_heads;               // extent of the source maps' last coordinate: one past it reads zeros
+  int64_t dst_pitch;               // entries per row of dst
+  __nv_bfloat16* dst;
+};
+
 struct RadonParams {
   int32_t q, transpose;
   int32_t sps, sr;                 // lines (hi values) per ring slot; rows of a slot = sps*q rounded up to 16
   int32_t nreg, nslots;            // slots of regular lines per image; plus one when the input has the extra class
   int32_t parts, rows_pp;          // CTAs sharing an image, and output indices per CTA (<= 128)
+  int32_t alu_rows;                // output indices parts*rows_pp .. (all of the extra class) summed on the ALUs by the
+                                   // last part, straight from the ring slot; 0: every index goes through the MMAs
   int32_t ring;                    // ring slots
-  int32_t images;
+  int32_t nph;                     // 1, or 2: both stages of the d = 4 tabulation, slab by slab
   int32_t slabs_per_head;          // rp / 128
   int64_t slabs;                   // heads * slabs_per_head
-  int64_t rp;
-  RadonSide in, out;
-  const __nv_bfloat16* src;
-  __nv_bfloat16* dst;
+  RadonPhase ph[2];
   int* status;
+};
+
+// The items of one CTA, in the order every role walks them.  One phase: item = (slab, image) with the slab index
+// fastest over the whole grid.  Two phases: slab by slab, the images of phase 0 and then those of phase 1, whose input
+// is what phase 0 wrote for the same slab.
+struct ItemIter {
+  uint32_t slab, img, ph, left;    // the current item, and the items left including it
+  uint32_t step, slabs, nph, im0, im1;
+  __device__ __forceinline__ ItemIter(const RadonParams& p, uint32_t first, uint32_t step_) {
+    step = step_; slabs = (uint32_t)p.slabs; nph = (uint32_t)p.nph;
+    im0 = (uint32_t)p.ph[0].images; im1 = nph > 1 ? (uint32_t)p.ph[1].images : 0u;
+    ph = 0;
+    if (nph == 1) {
+      const uint32_t total = slabs * im0;                       // < 2^31 (checked by the launcher)
+      left = first < total ? (total - 1 - first) / step + 1 : 0;
+      img = first / slabs; slab = first - img * slabs;
+    } else {
+      left = first < slabs ? ((slabs - 1 - first) / step + 1) * (im0 + im1) : 0;
+      img = 0; slab = first;
+    }
+  }
+  __device__ __forceinline__ void next() {
+    --left;
+    if (nph == 1) {
+      slab += step;
+      while (slab >= slabs) { slab -= slabs; ++img; }
+    } else if (++img == (ph ? im1 : im0)) {
+      img = 0;
+      if (ph == 0) ph = 1; else { ph = 0; slab += step; }
+    }
+  }
+  // last item of phase 0 of a slab: phase 1 may start once its output is visible
+  __device__ __forceinline__ bool closes_phase0() const { return nph > 1 && ph == 0 && img + 1 == im0; }
 };
 
 // Lane 0 polls the barrier and the warp follows.
@@ -115,24 +170,47 @@ __device__ __forceinline__ void mark_incident(const RadonParams& p, int n, __nv_
       row[operand_row(p, a, u)] = one;
       u += y; if (u >= q) u -= q;
     }
-    if (p.in.count > q * q) row[operand_row(p, q, y)] = one;
+    if (p.ph[0].in.count > q * q) row[operand_row(p, q, y)] = one;
   }
 }
 
 // box of 64 state entries x q rows x sps lines (regular map) or 64 x q rows (extra-class map)
 __device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
-                                            int c4, uint64_t* bar) {
+                                            int c4, uint64_t* bar, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar))
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar)), "l"(pol)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
-                                            uint64_t* bar) {
+                                            uint64_t* bar, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar)), "l"(pol)
       : "memory");
+}
+
+// L2 eviction policies: the exchange rows of the two-stage kernel should stay in the cache (they are rewritten for
+// every slab, and written back to memory only when evicted), the tables streaming past them should leave it first.
+enum { POLICY_NORMAL = 0, POLICY_FIRST = 1, POLICY_LAST = 2 };
+__device__ __forceinline__ uint64_t l2_policy(int kind) {
+  uint64_t p;
+  if (kind == POLICY_FIRST) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  else if (kind == POLICY_LAST) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void st_global_v8_hint(void* dst, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
+                                                  uint32_t w4, uint32_t w5, uint32_t w6, uint32_t w7, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8}, %9;" ::"l"(dst), "r"(w0),
+               "r"(w1), "r"(w2), "r"(w3), "r"(w4), "r"(w5), "r"(w6), "r"(w7), "l"(pol)
+               : "memory");
+}
+__device__ __forceinline__ void st_global_v4_hint(void* dst, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
+                                                  uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(dst), "r"(w0), "r"(w1), "r"(w2),
+               "r"(w3), "l"(pol)
+               : "memory");
 }
 
 // D[tmem_d] (+)= A[tmem_a] * B[desc_b]: A (128 x 16, bf16) read from tensor memory, B from shared memory.
@@ -170,8 +248,10 @@ __device__ __forceinline__ void issue_slot_steps(int steps, uint32_t tmem_d, uin
   }
 }
 
-__global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid_constant__ CUtensorMap tm_reg,
-                                                                    const __grid_constant__ CUtensorMap tm_vert,
+__global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid_constant__ CUtensorMap tm_reg0,
+                                                                    const __grid_constant__ CUtensorMap tm_vert0,
+                                                                    const __grid_constant__ CUtensorMap tm_reg1,
+                                                                    const __grid_constant__ CUtensorMap tm_vert1,
                                                                     const RadonParams prm) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -179,25 +259,29 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   const int slot_bytes = prm.sr * 256;                          // two 64-entry blocks of sr rows x 128 bytes
   const int kt = prm.nslots * prm.sr;                           // operand rows per image
   uint8_t* sRing = smem;
-  int32_t* out_tab = reinterpret_cast<int32_t*>(sRing + prm.ring * slot_bytes);    // [128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_tab + TILE_ROWS);
+  int32_t* out_tab = reinterpret_cast<int32_t*>(sRing + prm.ring * slot_bytes);    // [2][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_tab + 2 * TILE_ROWS);
   uint64_t* full = bars;                    // [ring] slot filled (TMA bytes)
   uint64_t* empty = bars + prm.ring;        // [ring] slot consumed by the MMAs (arrival from the epilogue, once the item is complete)
   uint64_t* acc_full = empty + prm.ring;    // [MAX_ACC] accumulator complete
   uint64_t* acc_empty = acc_full + MAX_ACC; // [MAX_ACC] accumulator read out (one arrival per epilogue warp)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + MAX_ACC);
+  uint64_t* w_ready = acc_empty + MAX_ACC;  // phase 0 of the current slab written out (one arrival per storing warp)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(w_ready + 1);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const WaitCtx wc{cta_abort, prm.status};
   const int part = blockIdx.x % prm.parts;
+  const bool alu_here = prm.alu_rows > 0 && part == prm.parts - 1;
 
   if (threadIdx.x == 0) {
     *cta_abort = 0;
-    for (int s = 0; s < prm.ring; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
-    for (int b = 0; b < MAX_ACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, EPI_WARPS); }
+    for (int s = 0; s < prm.ring; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, alu_here ? 1 + ALU_WARPS : 1); }
+    for (int b = 0; b < MAX_ACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, EPI_WARPS / 2); }
+    mbar_init(w_ready, alu_here ? EPI_WARPS + ALU_WARPS : EPI_WARPS);
     fence_barrier_init();
-    prefetch_tmap(&tm_reg);
-    prefetch_tmap(&tm_vert);
+    prefetch_tmap(&tm_reg0);
+    prefetch_tmap(&tm_vert0);
+    if (prm.nph > 1) { prefetch_tmap(&tm_reg1); prefetch_tmap(&tm_vert1); }
   }
   if (warp == MMA_WARP) tmem_alloc(tmem_slot, 512);
   // This CTA's part of R, built row by row in the (still unused) ring and moved to tensor memory: lane = output
@@ -206,7 +290,8 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   for (int c = threadIdx.x; c < prm.ring * slot_bytes / 16; c += blockDim.x)
     reinterpret_cast<uint4*>(sRing)[c] = make_uint4(0u, 0u, 0u, 0u);
   for (int n = threadIdx.x; n < TILE_ROWS; n += blockDim.x)
-    out_tab[n] = n < prm.rows_pp ? side_row(prm.out, part * prm.rows_pp + n, q) : ROW_INVALID;
+    for (int h = 0; h < prm.nph; ++h)
+      out_tab[h * TILE_ROWS + n] = n < prm.rows_pp ? side_row(prm.ph[h].out, part * prm.rows_pp + n, q) : ROW_INVALID;
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
@@ -216,7 +301,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   if (warp < 4) {
     const int n = warp * 32 + lane;
     __nv_bfloat16* row = scratch + (size_t)n * kt;
-    if (n < prm.rows_pp && part * prm.rows_pp + n < prm.out.count) mark_incident(prm, part * prm.rows_pp + n, row);
+    if (n < prm.rows_pp && part * prm.rows_pp + n < prm.ph[0].out.count) mark_incident(prm, part * prm.rows_pp + n, row);
     __syncwarp();
     const uint32_t* roww = reinterpret_cast<const uint32_t*>(row);
     for (int c0 = 0; c0 < (int)r_cols; c0 += 32) {
@@ -235,49 +320,62 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   fence_after_sync();
   const uint32_t tmem_acc = tmem_base + r_cols;
 
-  // items of this CTA: same part always; slab fastest, image slowest
+  // per phase: streaming tables, or the exchange rows (two-stage kernel only)
+  const uint64_t pol_src0 = l2_policy(prm.nph > 1 ? (prm.ph[0].src_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
+  const uint64_t pol_src1 = l2_policy(prm.nph > 1 ? (prm.ph[1].src_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
+  const uint64_t pol_dst0 = l2_policy(prm.nph > 1 ? (prm.ph[0].dst_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
+  const uint64_t pol_dst1 = l2_policy(prm.nph > 1 ? (prm.ph[1].dst_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
+  // items of this CTA: same part always
   const uint32_t first = blockIdx.x / prm.parts, step = gridDim.x / prm.parts;
-  const uint32_t slabs = (uint32_t)prm.slabs, total = slabs * (uint32_t)prm.images;   // < 2^31 (checked by the launcher)
+  const uint32_t sph = (uint32_t)prm.slabs_per_head;
 
   if (warp == PROD_WARP && lane == 0) {
     // ---- TMA producer -----------------------------------------------------------------------------------------
     // The two single-thread roles keep running slot / parity counters: a lone thread pays the full latency of every
     // instruction, so divisions by the ring size inside the loop would show in the kernel time.
     uint32_t slot = 0, par = 0;                               // ring position; parity of the empty barrier's phase to wait for
+    uint32_t wpar = 0;                                        // parity of w_ready for the current slab
     bool first_lap = true, ok = true;
     const uint32_t reg_bytes = 2u * 128u * (uint32_t)(q * prm.sps), vert_bytes = 2u * 128u * (uint32_t)q;
-    const int heads = (int)(prm.slabs / prm.slabs_per_head);
-    const uint32_t sph = (uint32_t)prm.slabs_per_head;
-    uint32_t img = first / slabs, slab = first - img * slabs;
-    for (uint32_t it = first; it < total && ok; it += step) {
-      const uint32_t head = slab / sph;
-      const int e0 = (int)(slab - head * sph) * 128;
+    for (ItemIter it(prm, first, step); it.left && ok; it.next()) {
+      const RadonPhase& ph = prm.ph[it.ph];
+      const CUtensorMap* tm_reg = it.ph ? &tm_reg1 : &tm_reg0;
+      const CUtensorMap* tm_vert = it.ph ? &tm_vert1 : &tm_vert0;
+      const uint32_t head = it.slab / sph;
+      const int e0 = ph.src_private ? 0 : (int)(it.slab - head * sph) * 128;
+      const int hc = ph.src_private ? (int)blockIdx.x : (int)head;
+      const uint64_t pol = it.ph ? pol_src1 : pol_src0;
+      if (it.ph == 1 && it.img == 0) {   // this slab's phase 0 output is complete and visible to the copy engine
+        ok = mbar_wait(w_ready, wpar, wc);
+        wpar ^= 1;
+        fence_proxy_async_all();
+        if (!ok) break;
+      }
       for (int g = 0; g < prm.nslots; ++g) {
         if (!first_lap) ok = mbar_wait(empty + slot, par, wc);
         if (!ok) break;
         uint8_t* dst = sRing + slot * slot_bytes;
         if (g < prm.nreg) {   // lines hi = g*sps ..; lines past q - 1 are out of bounds and arrive as zeros
           mbar_expect_tx(full + slot, reg_bytes);
-          tma_load_5d(dst, &tm_reg, e0, 0, g * prm.sps, (int)img, (int)head, full + slot);
-          tma_load_5d(dst + prm.sr * 128, &tm_reg, e0 + 64, 0, g * prm.sps, (int)img, (int)head, full + slot);
+          tma_load_5d(dst, tm_reg, e0, 0, g * prm.sps, (int)it.img, hc, full + slot, pol);
+          tma_load_5d(dst + prm.sr * 128, tm_reg, e0 + 64, 0, g * prm.sps, (int)it.img, hc, full + slot, pol);
         } else {              // extra class; an image without it reads past the last head: zeros
-          const int h = (int)img >= prm.in.vert_from ? (int)head : heads;
-          const int ci = (int)img * prm.in.sv_img;   // 0 when every image shares the rows
+          const int h = (int)it.img >= ph.in.vert_from ? hc : ph.src_heads;
+          const int ci = (int)it.img * ph.in.sv_img;   // 0 when every image shares the rows
           mbar_expect_tx(full + slot, vert_bytes);
-          tma_load_4d(dst, &tm_vert, e0, 0, ci, h, full + slot);
-          tma_load_4d(dst + prm.sr * 128, &tm_vert, e0 + 64, 0, ci, h, full + slot);
+          tma_load_4d(dst, tm_vert, e0, 0, ci, h, full + slot, pol);
+          tma_load_4d(dst + prm.sr * 128, tm_vert, e0 + 64, 0, ci, h, full + slot, pol);
         }
         if (++slot == (uint32_t)prm.ring) {
           slot = 0;
           if (first_lap) { first_lap = false; par = 0; } else par ^= 1;
         }
       }
-      slab += step;
-      while (slab >= slabs) { slab -= slabs; ++img; }
     }
-  } else if (warp >= MMA_WARP && lane == 0) {
+  } else if (warp >= MMA_WARP && warp < ALU_WARP && lane == 0) {
     // ---- MMA issuers: the two threads take the items alternately, so that the issue latency of one item (waits,
-    // MMAs, commits: more than the tensor pipe needs for it) overlaps with the other thread's item ----------------
+    // MMAs, commits: more than the tensor pipe needs for it) overlaps with the other thread's item.  Both phases
+    // share R and the slot layout, so the issuers only count items. ---------------------------------------------
     const uint32_t me = (uint32_t)(warp - MMA_WARP);
     constexpr uint32_t idesc = make_idesc(TILE_ROWS, 128, 0, 1);   // A from tensor memory (R), B MN-major (image rows)
     const uint64_t dB0 = make_desc(smem_u32(sRing), prm.sr * 128, 1024);
@@ -285,13 +383,14 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     const uint32_t slot_cols = (uint32_t)prm.sr / 2;              // columns of R per slot
     const int steps = prm.sr / 16, nslots = prm.nslots;
     const uint32_t ring = (uint32_t)prm.ring;
+    const uint32_t items = ItemIter(prm, first, step).left;
     uint32_t slot = 0, par = 0;                                   // ring position and the parity its full barrier shows
-    uint32_t buf = 0, apar = 0, n_item = 0;                       // accumulator; parity of its empty barrier's phase to wait for
+    uint32_t buf = 0, apar = 0;                                   // accumulator; parity of its empty barrier's phase to wait for
     bool ok = true;
     if (nslots == 1) {
       // One slot per item (q <= 11): a single thread, and the leanest loop: every instruction here is on the
       // critical path of the stage.
-      for (uint32_t it = first; me == 0 && it < total && ok; it += step, ++n_item) {
+      for (uint32_t n_item = 0; me == 0 && n_item < items && ok; ++n_item) {
         if (n_item >= nacc) ok = mbar_wait(acc_empty + buf, apar, wc);
         if (!ok) break;
         ok = mbar_wait(full + slot, par, wc);
@@ -305,7 +404,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
       }
     } else {
       uint32_t turn = 0;
-      for (uint32_t it = first; it < total && ok; it += step, ++n_item) {
+      for (uint32_t n_item = 0; n_item < items && ok; ++n_item) {
         const bool mine = turn == me;
         if (++turn == MMA_WARPS) turn = 0;
         if (!mine) {   // the other thread's item: step the counters over it
@@ -330,54 +429,125 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
         if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
       }
     }
+  } else if (warp >= ALU_WARP) {
+    // ---- leftover rows on the ALUs ----------------------------------------------------------------------------
+    // q*q + q output indices rarely fill whole tiles of 128.  When only a few are left over, and they belong to the
+    // extra class (index q*q + u = the sum of line u's q rows), these warps add the rows up from the slot itself
+    // instead of a second, nearly empty tile paying for every MMA again.  A task is one leftover index and 8 state
+    // entries (one 16-byte chunk of the swizzled slot); 16 neighbouring tasks store 256 contiguous bytes.
+    if (alu_here) {
+      const int tid_a = (warp - ALU_WARP) * 32 + lane, tasks = prm.alu_rows * 16;
+      const uint32_t ring = (uint32_t)prm.ring;
+      uint32_t slot = 0, par = 0;
+      for (ItemIter it(prm, first, step); it.left; it.next()) {
+        const RadonPhase& ph = prm.ph[it.ph];
+        const uint32_t head = it.slab / sph;
+        const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
+        const int64_t hrow = (int64_t)(ph.dst_private ? blockIdx.x : head) * ph.out.rows_per_head;
+        if (!mbar_wait_warp(full + slot, par, wc)) break;
+        if ((int)it.img >= ph.out.vert_from) {
+          const uint8_t* sl = sRing + slot * slot_bytes;
+          for (int task = tid_a; task < tasks; task += 32 * ALU_WARPS) {
+            const int u = prm.parts * prm.rows_pp + (task >> 4) - q * q, ch = task & 15;
+            const uint8_t* blk = sl + (ch >> 3) * prm.sr * 128;
+            float acc[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+            for (int lo = 0; lo < q; ++lo) {
+              const int r = u * q + lo;                           // operand row of (line u, lo): one slot holds every line
+              const uint4 w = *reinterpret_cast<const uint4*>(blk + r * 128 + (((ch & 7) ^ (r & 7)) << 4));
+              acc[0] += __uint_as_float(w.x << 16); acc[1] += __uint_as_float(w.x & 0xffff0000u);
+              acc[2] += __uint_as_float(w.y << 16); acc[3] += __uint_as_float(w.y & 0xffff0000u);
+              acc[4] += __uint_as_float(w.z << 16); acc[5] += __uint_as_float(w.z & 0xffff0000u);
+              acc[6] += __uint_as_float(w.w << 16); acc[7] += __uint_as_float(w.w & 0xffff0000u);
+            }
+            const int row = ph.out.v0 + (int)it.img * ph.out.sv_img + u * ph.out.sv_lo;
+            __nv_bfloat16* dst = ph.dst + (hrow + row) * ph.dst_pitch + e0 + ch * 8;
+            st_global_v4_hint(dst, pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                              pack_bf16(acc[6], acc[7]), it.ph ? pol_dst1 : pol_dst0);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty + slot);
+        if (it.closes_phase0()) {   // what this warp stored for the slab is ordered before the copy engine's reads
+          __threadfence();
+          fence_proxy_async_all();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(w_ready);
+        }
+        if (++slot == ring) { slot = 0; par ^= 1; }
+      }
+    }
   } else if (warp < EPI_WARPS) {
     // ---- epilogue ---------------------------------------------------------------------------------------------
-    // Warp w reads lane quarter w % 4 (32 output indices) and the 32-entry column chunk w / 4 of every item.
-    const int qd = warp & 3, cb = warp >> 2;
+    // The store port of an SM (32 bytes a cycle) needs about as long for an item's output tile as the MMAs do, so it
+    // must never wait for the epilogue: two groups of 8 warps take the items alternately, and one group reads and
+    // packs its accumulator while the other group's stores drain.  Warp w of a group reads lane quarter w % 4 (32
+    // output indices) and the 64-entry column half (w / 4) % 2: every thread stores one whole 128-byte line.
+    const int qd = warp & 3, grp = warp >> 3, ch = (warp >> 2) & 1;
     const int orow = qd * 32 + lane;                            // output index of this CTA = TMEM lane
     const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
-    const int tv = out_tab[orow];
+    const int tv0 = out_tab[orow], tv1 = prm.nph > 1 ? out_tab[TILE_ROWS + orow] : ROW_INVALID;
     const bool active = qd * 32 < prm.rows_pp;                  // warp-uniform: some output index in these lanes
-    const uint32_t sph = (uint32_t)prm.slabs_per_head;
-    uint32_t buf = 0, apar = 0, eslot = 0;
-    uint32_t img = first / slabs, slab = first - img * slabs;
-    for (uint32_t it = first; it < total; it += step) {
-      const uint32_t head = slab / sph;
-      const int e0 = (int)(slab - head * sph) * 128;
-      if (!mbar_wait_warp(acc_full + buf, apar, wc)) break;
-      fence_after_sync();
-      if (warp == 0 && prm.nslots > 1) {   // every MMA of the item has completed: its ring slots are free (a commit per slot would cost the
-                         // issuing thread more than the MMAs of the slot)
-        for (int g = 0; g < prm.nslots; ++g) {
-          if (lane == 0) mbar_arrive(empty + eslot);
-          if (++eslot == (uint32_t)prm.ring) eslot = 0;
+    const uint32_t ring = (uint32_t)prm.ring;
+    uint32_t buf = 0, apar = 0, eslot = 0, turn = 0;
+    for (ItemIter it(prm, first, step); it.left; it.next()) {
+      const bool mine = turn == (uint32_t)grp;
+      turn ^= 1u;
+      if (mine) {
+        const RadonPhase& ph = prm.ph[it.ph];
+        const uint32_t head = it.slab / sph;
+        const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
+        const int64_t hrow = (int64_t)(ph.dst_private ? blockIdx.x : head) * ph.out.rows_per_head;
+        const int tv = it.ph ? tv1 : tv0;
+        const uint64_t pol = it.ph ? pol_dst1 : pol_dst0;
+        if (!mbar_wait_warp(acc_full + buf, apar, wc)) break;
+        fence_after_sync();
+        if ((warp & 7) == 0 && prm.nslots > 1 && lane == 0) {   // every MMA of the item has completed: its ring slots are
+          uint32_t sl = eslot;                                  // free (a commit per slot would cost the issuing thread
+          for (int g = 0; g < prm.nslots; ++g) {                // more than the MMAs of the slot)
+            mbar_arrive(empty + sl);
+            if (++sl == ring) sl = 0;
+          }
         }
-      }
-      if (active) {
-        uint32_t v[32];
-        tmem_ld32(tmem_acc + lane_base + buf * 128 + cb * 32, v);
-        tmem_ld_wait();
-        const bool vert = (int)img >= prm.out.vert_from;
-        if (tv != ROW_INVALID && (!(tv & ROW_VERT) || vert)) {
-          const int row = (tv & ROW_VERT) ? prm.out.v0 + (int)img * prm.out.sv_img + (tv & ~ROW_VERT)
-                                          : (int)img * prm.out.s_img + tv;
-          __nv_bfloat16* dst = prm.dst + ((int64_t)head * prm.out.rows_per_head + row) * prm.rp + e0 + cb * 32;
+        const bool vert = (int)it.img >= ph.out.vert_from;
+        const bool store = active && tv != ROW_INVALID && (!(tv & ROW_VERT) || vert);
+        const int row = (tv & ROW_VERT) ? ph.out.v0 + (int)it.img * ph.out.sv_img + (tv & ~ROW_VERT)
+                                        : (int)it.img * ph.out.s_img + tv;
+        __nv_bfloat16* dst = ph.dst + (hrow + row) * ph.dst_pitch + e0 + ch * 64;
 #pragma unroll
-          for (int h8 = 0; h8 < 2; ++h8) {   // two whole 32-byte sectors per thread
-            uint32_t w[8];
+        for (int jj = 0; jj < 2; ++jj) {
+          uint32_t v[32];
+          if (active) {
+            tmem_ld32(tmem_acc + lane_base + buf * 128 + ch * 64 + jj * 32, v);
+            tmem_ld_wait();
+          }
+          if (jj == 1) {   // the accumulator is in registers: the MMAs may have it back before the stores are out
+            fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty + buf);
+          }
+          if (store) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              w[i] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * i]), __uint_as_float(v[16 * h8 + 2 * i + 1]));
-            st_global_v8(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+            for (int h8 = 0; h8 < 2; ++h8) {   // whole 32-byte sectors
+              uint32_t w[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                w[i] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * i]), __uint_as_float(v[16 * h8 + 2 * i + 1]));
+              st_global_v8_hint(dst + jj * 32 + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7], pol);
+            }
           }
         }
       }
-      fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty + buf);
+      if (it.closes_phase0()) {   // as for the ALU warps: the slab's phase 0 rows (this warp's last ones were stored for
+        __threadfence();          // this item or the one before) before the copy engine reads them
+        fence_proxy_async_all();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(w_ready);
+      }
+      eslot += (uint32_t)prm.nslots;
+      if (eslot >= ring) eslot -= ring;
       if (++buf == nacc) { buf = 0; apar ^= 1; }
-      slab += step;
-      while (slab >= slabs) { slab -= slabs; ++img; }
     }
   }
   fence_before_sync();
@@ -389,15 +559,15 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
 }
 
 struct RadonShape {
-  int sps, sr, nreg, nslots, parts, rows_pp, ring, smem;
+  int sps, sr, nreg, nslots, parts, rows_pp, alu_rows, ring, smem;
 };
 
 // Ring slots of `sps` lines (sps*q rows, rounded up to 16), chosen for the least MMA work; the output indices are
 // split evenly over `parts` CTAs of at most 128 each.  R (128 lanes x one column per two operand rows) and at least
 // two accumulators of 128 columns must fit the 512 columns of tensor memory, and the ring must be able to hold the
 // scratch copy of R while it is built.  Returns false when q is too large for this kernel.
-bool radon_shape(int q, int in_has_extra, int count_out, RadonShape* s) {
-  const int budget = 227 * 1024 - 1024 - 512 - TILE_ROWS * 4;
+bool radon_shape(int q, int transpose, int in_has_extra, int count_out, RadonShape* s) {
+  const int budget = 227 * 1024 - 1024 - 512 - TILE_ROWS * 8;
   if (q < 2 || q > 64) return false;
   const int parts = (count_out + TILE_ROWS - 1) / TILE_ROWS;
   if (parts > 8) return false;
@@ -417,11 +587,19 @@ bool radon_shape(int q, int in_has_extra, int count_out, RadonShape* s) {
     if (cost < best) {
       best = cost;
       s->sps = sps; s->sr = sr; s->nreg = nreg; s->nslots = nslots; s->parts = parts;
-      s->rows_pp = (count_out + parts - 1) / parts; s->ring = ring;
-      s->smem = ring * slot_bytes + TILE_ROWS * 4 + 512 + 1024;
+      s->rows_pp = (count_out + parts - 1) / parts; s->alu_rows = 0; s->ring = ring;
+      s->smem = ring * slot_bytes + TILE_ROWS * 8 + 512 + 1024;
     }
   }
-  return best != (1 << 30);
+  if (best == (1 << 30)) return false;
+  // A few indices past the last full tile, all of the extra class, with every line in one slot: full tiles for the
+  // MMAs and the rest on the ALUs (q = 11: 132 = 128 + 4 indices, one CTA per image instead of two).
+  const int left = count_out % TILE_ROWS, whole = count_out - left;
+  if (!transpose && !in_has_extra && s->nslots == 1 && s->sps >= q && whole > 0 && left > 0 && left <= ALU_MAX_ROWS &&
+      whole >= q * q) {
+    s->parts = whole / TILE_ROWS; s->rows_pp = TILE_ROWS; s->alu_rows = left;
+  }
+  return true;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -467,49 +645,90 @@ RadonSide side(int count, int s_lo, int s_hi, int s_img, int64_t rows_per_head, 
   return s;
 }
 
-cudaError_t launch_radon(int q, int transpose, int images, const RadonSide& in, const RadonSide& out, const void* src,
-                         void* dst, int64_t rp, int bh, int* status, cudaStream_t st) {
+// One stage as the host states it; src / dst are whole tables [bh][rows_per_head][rp], or the private exchange buffer.
+struct StageSpec {
+  RadonSide in, out;
+  int images;
+  const void* src;
+  void* dst;
+  bool src_private, dst_private;
+};
+
+StageSpec stage(const RadonSide& in, const RadonSide& out, int images, const void* src, void* dst, bool src_private = false,
+                bool dst_private = false) {
+  StageSpec s;
+  s.in = in; s.out = out; s.images = images; s.src = src; s.dst = dst; s.src_private = src_private; s.dst_private = dst_private;
+  return s;
+}
+
+// nph = 1: one stage over the whole tables.  nph = 2: both stages in one launch, which must share R (the same
+// direction, the same index counts) and exchange their rows through the private buffer.
+cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int64_t rp, int bh, int* status,
+                         cudaStream_t st) {
   RadonShape sh;
-  const int in_has_extra = in.count > q * q;
-  if (!radon_shape(q, in_has_extra, out.count, &sh) || rp % 128 || (int64_t)bh * (rp / 128) * images >= (1LL << 31))
+  const int in_has_extra = sp[0].in.count > q * q;
+  int max_images = sp[0].images;
+  if (nph == 2 && sp[1].images > max_images) max_images = sp[1].images;
+  if (!radon_shape(q, transpose, in_has_extra, sp[0].out.count, &sh) || rp % 128 ||
+      (int64_t)bh * (rp / 128) * max_images * 2 >= (1LL << 31))
+    return cudaErrorInvalidValue;
+  if (nph == 2 && (sh.parts != 1 || sp[1].in.count != sp[0].in.count || sp[1].out.count != sp[0].out.count))
     return cudaErrorInvalidValue;
   RadonParams prm;
   prm.q = q; prm.transpose = transpose; prm.sps = sh.sps; prm.sr = sh.sr; prm.nreg = sh.nreg; prm.nslots = sh.nslots;
-  prm.parts = sh.parts; prm.rows_pp = sh.rows_pp;
-  prm.ring = sh.ring; prm.images = images; prm.slabs_per_head = (int)(rp / 128); prm.slabs = (int64_t)bh * (rp / 128);
-  prm.rp = rp; prm.in = in; prm.out = out;
-  prm.src = static_cast<const __nv_bfloat16*>(src);
-  prm.dst = static_cast<__nv_bfloat16*>(dst);
+  prm.parts = sh.parts; prm.rows_pp = sh.rows_pp; prm.alu_rows = sh.alu_rows;
+  prm.ring = sh.ring; prm.nph = nph; prm.slabs_per_head = (int)(rp / 128); prm.slabs = (int64_t)bh * (rp / 128);
   prm.status = status;
-  // regular lines: (entry, lo, hi, image, head); a size-one dimension keeps its stride valid
-  CUtensorMap tm_reg, tm_vert;
-  {
-    const int64_t sizes[4] = {q, q, images, bh};
-    const int64_t strides[4] = {in.s_lo, in.s_hi, images > 1 ? in.s_img : in.rows_per_head, in.rows_per_head};
-    const int box[4] = {q, sh.sps, 1, 1};
-    if (!radon_map(&tm_reg, src, rp, 5, sizes, strides, box)) return cudaErrorInvalidValue;
-  }
-  if (in_has_extra) {   // extra class: (entry, lo, image, head), rows v0 + image*sv_img + lo*sv_lo
-    const bool per_image = in.sv_img != 0;
-    const int64_t sizes[3] = {q, per_image ? images : 1, bh};
-    const int64_t strides[3] = {in.sv_lo, per_image ? in.sv_img : in.rows_per_head, in.rows_per_head};
-    const int box[3] = {q, 1, 1};
-    if (!radon_map(&tm_vert, static_cast<const __nv_bfloat16*>(src) + (int64_t)in.v0 * rp, rp, 4, sizes, strides, box))
-      return cudaErrorInvalidValue;
-    prm.in.sv_img = per_image ? 1 : 0;   // the kernel passes image * sv_img as the coordinate
-  } else {
-    tm_vert = tm_reg;
-  }
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   int64_t ctas = (int64_t)(sms / sh.parts) * sh.parts;
-  const int64_t items = prm.slabs * images * sh.parts;
+  const int64_t items = nph == 1 ? prm.slabs * sp[0].images * sh.parts : prm.slabs;
   if (items < ctas) ctas = items;
+  CUtensorMap tm_reg[2], tm_vert[2];
+  for (int i = 0; i < nph; ++i) {
+    RadonPhase& ph = prm.ph[i];
+    const RadonSide& in = sp[i].in;
+    const int images = sp[i].images;
+    const int64_t src_rp = sp[i].src_private ? 128 : rp, src_heads = sp[i].src_private ? ctas : bh;
+    ph.in = in; ph.out = sp[i].out; ph.images = images;
+    ph.src_private = sp[i].src_private; ph.dst_private = sp[i].dst_private;
+    ph.src_heads = (int)src_heads;
+    ph.dst_pitch = sp[i].dst_private ? 128 : rp;
+    ph.dst = static_cast<__nv_bfloat16*>(sp[i].dst);
+    {   // regular lines: (entry, lo, hi, image, head); a size-one dimension keeps its stride valid
+      const int64_t sizes[4] = {q, q, images, src_heads};
+      const int64_t strides[4] = {in.s_lo, in.s_hi, images > 1 ? in.s_img : in.rows_per_head, in.rows_per_head};
+      const int box[4] = {q, sh.sps, 1, 1};
+      if (!radon_map(&tm_reg[i], sp[i].src, src_rp, 5, sizes, strides, box)) return cudaErrorInvalidValue;
+    }
+    if (in_has_extra) {   // extra class: (entry, lo, image, head), rows v0 + image*sv_img + lo*sv_lo
+      const bool per_image = in.sv_img != 0;
+      const int64_t sizes[3] = {q, per_image ? images : 1, src_heads};
+      const int64_t strides[3] = {in.sv_lo, per_image ? in.sv_img : in.rows_per_head, in.rows_per_head};
+      const int box[3] = {q, 1, 1};
+      if (!radon_map(&tm_vert[i], static_cast<const __nv_bfloat16*>(sp[i].src) + (int64_t)in.v0 * src_rp, src_rp, 4, sizes,
+                     strides, box))
+        return cudaErrorInvalidValue;
+      ph.in.sv_img = per_image ? 1 : 0;   // the kernel passes image * sv_img as the coordinate
+    } else {
+      tm_vert[i] = tm_reg[i];
+    }
+  }
+  if (nph == 1) { prm.ph[1] = prm.ph[0]; tm_reg[1] = tm_reg[0]; tm_vert[1] = tm_vert[0]; }
   cudaError_t err = cudaFuncSetAttribute(radon_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.smem);
   if (err != cudaSuccess) return err;
-  radon_tc_kernel<<<(unsigned)ctas, RADON_THREADS, sh.smem, st>>>(tm_reg, tm_vert, prm);
+  radon_tc_kernel<<<(unsigned)ctas, RADON_THREADS, sh.smem, st>>>(tm_reg[0], tm_vert[0], tm_reg[1], tm_vert[1], prm);
   return cudaGetLastError();
+}
+
+// The two stages of d = 4 run as one launch when a CTA's exchange rows (q^3 + q^2 rows of 128 entries), times the
+// CTAs of the grid, stay well inside the L2 cache, and one CTA covers every output index of an image.
+bool radon_two_stage_fits(int q, int transpose) {
+  RadonShape sh;
+  const int qq = q * q;
+  if (!radon_shape(q, transpose, transpose ? 1 : 0, transpose ? qq : qq + q, &sh) || sh.parts != 1) return false;
+  return ((int64_t)qq * q + qq) * 256 * 148 <= (64LL << 20);
 }
 
 }  // namespace
@@ -520,7 +739,7 @@ int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems) {
   if (state_elems % 128) return 0;
   const int qq = geo.q * geo.q;
   RadonShape a, b;
-  return radon_encode_fn() && radon_shape(geo.q, 0, qq + geo.q, &a) && radon_shape(geo.q, 1, qq, &b) ? 1 : 0;
+  return radon_encode_fn() && radon_shape(geo.q, 0, 0, qq + geo.q, &a) && radon_shape(geo.q, 1, 1, qq, &b) ? 1 : 0;
 }
 
 // Rows (of state_elems bf16 each, per head) of the intermediate table the d = 4 stages exchange.
@@ -537,9 +756,9 @@ cudaError_t smat_launch_tabulate_tc(const void* in, void* out, void* scratch, co
   if (geo.D == 2) {
     const RadonSide pts = side(qq, 1, q, 0, geo.P);
     const RadonSide typ = side(qq + q, 1, q, 0, geo.B, qq, 1, 0, 0);
+    const StageSpec sp = transpose ? stage(typ, pts, 1, in, out) : stage(pts, typ, 1, in, out);
     *launches = 1;
-    return transpose ? launch_radon(q, 1, 1, typ, pts, in, out, state_elems, bh, status, st)
-                     : launch_radon(q, 0, 1, pts, typ, in, out, state_elems, bh, status, st);
+    return launch_radon(q, transpose, 1, &sp, state_elems, bh, status, st);
   }
   if (geo.D != 3) return cudaErrorInvalidValue;
   const int64_t wrows = smat_tabulate_tc_scratch_rows(geo);
@@ -547,14 +766,21 @@ cudaError_t smat_launch_tabulate_tc(const void* in, void* out, void* scratch, co
   const RadonSide w1_side = side(qq + q, 1, qq, q, wrows, qqq, q, 1, 0);    // (u, a3) -> W[a3][x2][u]; extra class -> G[x3][x2]
   const RadonSide w2_side = side(qq, 1, q, qq, wrows);                      // image a3 (image q: G), points (u, x2)
   const RadonSide u_side = side(qq + q, 1, q, qq, geo.B, qqq + qq, 1, 0, q);
-  cudaError_t err;
-  *launches = 2;
+  const bool fused = radon_two_stage_fits(q, transpose);
+  StageSpec sp[2];
   if (!transpose) {
-    err = launch_radon(q, 0, q, f_side, w1_side, in, scratch, state_elems, bh, status, st);
-    if (err != cudaSuccess) return err;
-    return launch_radon(q, 0, q + 1, w2_side, u_side, scratch, out, state_elems, bh, status, st);
+    sp[0] = stage(f_side, w1_side, q, in, scratch, false, fused);
+    sp[1] = stage(w2_side, u_side, q + 1, scratch, out, fused, false);
+  } else {
+    sp[0] = stage(u_side, w2_side, q + 1, in, scratch, false, fused);
+    sp[1] = stage(w1_side, f_side, q, scratch, out, fused, false);
   }
-  err = launch_radon(q, 1, q + 1, u_side, w2_side, in, scratch, state_elems, bh, status, st);
+  if (fused) {
+    *launches = 1;
+    return launch_radon(q, transpose, 2, sp, state_elems, bh, status, st);
+  }
+  *launches = 2;
+  cudaError_t err = launch_radon(q, transpose, 1, &sp[0], state_elems, bh, status, st);
   if (err != cudaSuccess) return err;
-  return launch_radon(q, 1, q, w1_side, f_side, scratch, out, state_elems, bh, status, st);
+  return launch_radon(q, transpose, 1, &sp[1], state_elems, bh, status, st);
 }

@@ -59,6 +59,7 @@ WORKLOADS = {
     "t64k_d4":       Workload("t64k_d4", 4, 1, 16, 65536, 128, 128, 128, "bf16", "normalised", 3),
     # reduced-head copies of two workloads, small enough to profile kernel by kernel (tables still exceed L2)
     "t16k_d4_h2":    Workload("t16k_d4_h2", 4, 1, 2, 16384, 128, 128, 128, "bf16", "normalised", 2),
+    "t16k_d4_h8":    Workload("t16k_d4_h8", 4, 1, 8, 16384, 128, 128, 128, "bf16", "normalised", 2),
     "t64k_d4_h1":    Workload("t64k_d4_h1", 4, 1, 1, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t64k_d3_h2":    Workload("t64k_d3_h2", 3, 1, 2, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t8k_d3_h8":     Workload("t8k_d3_h8", 3, 1, 8, 8192, 128, 128, 64, "bf16", "normalised", 4),
