@@ -343,7 +343,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->off_U = off;      off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.B * state));
   pl->off_acc = off;    off = align_up(off + (size_t)pl->bh * T * wide * sizeof(float));
   pl->off_tileA = off;  off = align_up(off + (size_t)pl->bh * T * chunk * sizeof(float));
-  pl->off_W = off;      off = align_up(off + (pl->tab_tc ? (size_t)pl->bh * smat_tabulate_tc_scratch_rows(g) * pl->rp * 2 : 0));
+  pl->off_W = off;      off = align_up(off + (pl->tab_tc ? (size_t)smat_tabulate_tc_scratch_elems(g, pl->rp, pl->bh) * 2 : 0));
   pl->off_fwd_end = off;
   pl->off_dbar = off;   off = align_up(off + (size_t)pl->bh * pl->NC * state);
   pl->off_ubar = off;   off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.B * state));

@@ -122,6 +122,7 @@ cudaError_t smat_launch_tabulate_d3_bf16(const void* in, void* out, const SmatGe
 // Tabulation on the tensor cores (bf16 tables; d = 3, 4 with a prime small enough for a resident Radon matrix).
 int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems);
 int64_t smat_tabulate_tc_scratch_rows(const SmatGeo& geo);
+int64_t smat_tabulate_tc_scratch_elems(const SmatGeo& geo, int64_t state_elems, int bh);
 cudaError_t smat_launch_tabulate_tc(const void* in, void* out, void* scratch, const SmatGeo& geo, int64_t state_elems,
                                     int bh, int transpose, int* status, cudaStream_t st, int* launches);
 cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st);

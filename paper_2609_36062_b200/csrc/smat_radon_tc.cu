@@ -747,8 +747,24 @@ int64_t smat_tabulate_tc_scratch_rows(const SmatGeo& geo) {
   return geo.D == 3 ? (int64_t)geo.q * geo.q * geo.q + (int64_t)geo.q * geo.q : 0;
 }
 
+// bf16 elements of the scratch table smat_launch_tabulate_tc needs: the whole intermediate table W, or, when both
+// directions run their two stages in one launch, one slab of it (128 entries per row) per CTA.
+int64_t smat_tabulate_tc_scratch_elems(const SmatGeo& geo, int64_t state_elems, int bh) {
+  const int64_t rows = smat_tabulate_tc_scratch_rows(geo);
+  if (rows == 0) return 0;
+  if (radon_two_stage_fits(geo.q, 0) && radon_two_stage_fits(geo.q, 1)) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int64_t ctas = (int64_t)bh * (state_elems / 128);
+    if (ctas > sms) ctas = sms;
+    return ctas * rows * 128;
+  }
+  return (int64_t)bh * rows * state_elems;
+}
+
 // transpose = 0: in = F [bh][P][rp] bf16, out = U [bh][B][rp] bf16.  transpose = 1: in = Ū [bh][B][rp], out = F̄ [bh][P][rp].
-// scratch: [bh][smat_tabulate_tc_scratch_rows][rp] bf16 (d = 4 only).  One launch for d = 3, two for d = 4.
+// scratch: smat_tabulate_tc_scratch_elems bf16 (d = 4 only).  One launch for d = 3; one or two for d = 4.
 cudaError_t smat_launch_tabulate_tc(const void* in, void* out, void* scratch, const SmatGeo& geo, int64_t state_elems,
                                     int bh, int transpose, int* status, cudaStream_t st, int* launches) {
   const int q = geo.q, qq = q * q, qqq = qq * q;
