@@ -35,11 +35,11 @@ from paper_2609_36062_b200 import replicas, roofline, synth  # noqa: E402
 DEFAULT_WORKLOAD = "t16k_d4"
 SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
 METRIC = "SMat prefill tokens/s"
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant stage per step — the tabulation, two
-# launches of radon_tc_kernel — from the ncu capture summarised in profiles/radon_tc_kernel_t16k_d4_h2.md: taken on
-# the 2-head copy of the workload (281.0 MB) and scaled by heads (every head owns its tables).  At 2 heads about half
-# of the stage intermediate W is served by L2; with W fully in DRAM, as at 32 heads, the figure would be 5.97e9.
-NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate_tc"): 281.0e6 * 16}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant stage per step — the tabulation, one
+# launch of radon_tc_kernel — from the ncu capture summarised in profiles/radon_tc_kernel_t16k_d4_h8.md: taken on the
+# 8-head copy of the workload (352.5 MB read + 559.8 MB written) and scaled by heads (every head owns its tables; the
+# per-CTA exchange buffer, the only shared footprint, is the same 55 MB at 8 and at 32 heads).
+NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate_tc"): 912.3e6 * 4}
 
 
 def parse_args():

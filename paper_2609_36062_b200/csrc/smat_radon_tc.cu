@@ -24,9 +24,8 @@
 //                    (MN-major B operand, two boxes of 64 entries); the extra class travels in a slot of its own
 //   warps 17, 18 (lane 0) : MMA issuers, alternating items: D[128 outputs, 128 entries] += R_slot * B_slot; up to
 //                    four accumulators in flight
-//   warps 0-15     : epilogue in two groups of 8 warps that alternate items; one output index (TMEM lane) per
-//                    thread and one 64-entry column half per warp: round to bf16 and store 128 contiguous bytes of
-//                    the output row as 32-byte sectors
+//   warps 0-15     : epilogue, one output index (TMEM lane) per thread and one 32-entry column chunk per warp:
+//                    round to bf16 and store 64 contiguous bytes of the output row as two 32-byte sectors
 //   warps 19, 20   : q = 11 only.  q^2 + q = 132 output indices are one tile of 128 and 4 left over, all of the extra
 //                    class (the sum of one line's q rows): these warps add them up from the ring slot itself, so
 //                    that one CTA covers an image instead of two CTAs loading it twice
@@ -276,7 +275,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   if (threadIdx.x == 0) {
     *cta_abort = 0;
     for (int s = 0; s < prm.ring; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, alu_here ? 1 + ALU_WARPS : 1); }
-    for (int b = 0; b < MAX_ACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, EPI_WARPS / 2); }
+    for (int b = 0; b < MAX_ACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, EPI_WARPS); }
     mbar_init(w_ready, alu_here ? EPI_WARPS + ALU_WARPS : EPI_WARPS);
     fence_barrier_init();
     prefetch_tmap(&tm_reg0);
@@ -480,73 +479,56 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     }
   } else if (warp < EPI_WARPS) {
     // ---- epilogue ---------------------------------------------------------------------------------------------
-    // The store port of an SM (32 bytes a cycle) needs about as long for an item's output tile as the MMAs do, so it
-    // must never wait for the epilogue: two groups of 8 warps take the items alternately, and one group reads and
-    // packs its accumulator while the other group's stores drain.  Warp w of a group reads lane quarter w % 4 (32
-    // output indices) and the 64-entry column half (w / 4) % 2: every thread stores one whole 128-byte line.
-    const int qd = warp & 3, grp = warp >> 3, ch = (warp >> 2) & 1;
+    // Warp w reads lane quarter w % 4 (32 output indices) and the 32-entry column chunk w / 4 of every item.
+    const int qd = warp & 3, cb = warp >> 2;
     const int orow = qd * 32 + lane;                            // output index of this CTA = TMEM lane
     const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
     const int tv0 = out_tab[orow], tv1 = prm.nph > 1 ? out_tab[TILE_ROWS + orow] : ROW_INVALID;
     const bool active = qd * 32 < prm.rows_pp;                  // warp-uniform: some output index in these lanes
-    const uint32_t ring = (uint32_t)prm.ring;
-    uint32_t buf = 0, apar = 0, eslot = 0, turn = 0;
+    uint32_t buf = 0, apar = 0, eslot = 0;
     for (ItemIter it(prm, first, step); it.left; it.next()) {
-      const bool mine = turn == (uint32_t)grp;
-      turn ^= 1u;
-      if (mine) {
-        const RadonPhase& ph = prm.ph[it.ph];
-        const uint32_t head = it.slab / sph;
-        const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
-        const int64_t hrow = (int64_t)(ph.dst_private ? blockIdx.x : head) * ph.out.rows_per_head;
-        const int tv = it.ph ? tv1 : tv0;
-        const uint64_t pol = it.ph ? pol_dst1 : pol_dst0;
-        if (!mbar_wait_warp(acc_full + buf, apar, wc)) break;
-        fence_after_sync();
-        if ((warp & 7) == 0 && prm.nslots > 1 && lane == 0) {   // every MMA of the item has completed: its ring slots are
-          uint32_t sl = eslot;                                  // free (a commit per slot would cost the issuing thread
-          for (int g = 0; g < prm.nslots; ++g) {                // more than the MMAs of the slot)
-            mbar_arrive(empty + sl);
-            if (++sl == ring) sl = 0;
-          }
+      const RadonPhase& ph = prm.ph[it.ph];
+      const uint32_t head = it.slab / sph;
+      const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
+      const int64_t hrow = (int64_t)(ph.dst_private ? blockIdx.x : head) * ph.out.rows_per_head;
+      const int tv = it.ph ? tv1 : tv0;
+      if (!mbar_wait_warp(acc_full + buf, apar, wc)) break;
+      fence_after_sync();
+      if (warp == 0 && prm.nslots > 1) {   // every MMA of the item has completed: its ring slots are free (a commit per slot would cost the
+                         // issuing thread more than the MMAs of the slot)
+        for (int g = 0; g < prm.nslots; ++g) {
+          if (lane == 0) mbar_arrive(empty + eslot);
+          if (++eslot == (uint32_t)prm.ring) eslot = 0;
         }
+      }
+      if (active) {
+        uint32_t v[32];
+        tmem_ld32(tmem_acc + lane_base + buf * 128 + cb * 32, v);
+        tmem_ld_wait();
         const bool vert = (int)it.img >= ph.out.vert_from;
-        const bool store = active && tv != ROW_INVALID && (!(tv & ROW_VERT) || vert);
-        const int row = (tv & ROW_VERT) ? ph.out.v0 + (int)it.img * ph.out.sv_img + (tv & ~ROW_VERT)
-                                        : (int)it.img * ph.out.s_img + tv;
-        __nv_bfloat16* dst = ph.dst + (hrow + row) * ph.dst_pitch + e0 + ch * 64;
+        if (tv != ROW_INVALID && (!(tv & ROW_VERT) || vert)) {
+          const int row = (tv & ROW_VERT) ? ph.out.v0 + (int)it.img * ph.out.sv_img + (tv & ~ROW_VERT)
+                                          : (int)it.img * ph.out.s_img + tv;
+          __nv_bfloat16* dst = ph.dst + (hrow + row) * ph.dst_pitch + e0 + cb * 32;
 #pragma unroll
-        for (int jj = 0; jj < 2; ++jj) {
-          uint32_t v[32];
-          if (active) {
-            tmem_ld32(tmem_acc + lane_base + buf * 128 + ch * 64 + jj * 32, v);
-            tmem_ld_wait();
-          }
-          if (jj == 1) {   // the accumulator is in registers: the MMAs may have it back before the stores are out
-            fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty + buf);
-          }
-          if (store) {
+          for (int h8 = 0; h8 < 2; ++h8) {   // two whole 32-byte sectors per thread
+            uint32_t w[8];
 #pragma unroll
-            for (int h8 = 0; h8 < 2; ++h8) {   // whole 32-byte sectors
-              uint32_t w[8];
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                w[i] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * i]), __uint_as_float(v[16 * h8 + 2 * i + 1]));
-              st_global_v8_hint(dst + jj * 32 + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7], pol);
-            }
+            for (int i = 0; i < 8; ++i)
+              w[i] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * i]), __uint_as_float(v[16 * h8 + 2 * i + 1]));
+            st_global_v8_hint(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7], it.ph ? pol_dst1 : pol_dst0);
           }
         }
       }
-      if (it.closes_phase0()) {   // as for the ALU warps: the slab's phase 0 rows (this warp's last ones were stored for
-        __threadfence();          // this item or the one before) before the copy engine reads them
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty + buf);
+      if (it.closes_phase0()) {   // as for the ALU warps: the slab's phase 0 rows before the copy engine reads them
+        __threadfence();
         fence_proxy_async_all();
         __syncwarp();
         if (lane == 0) mbar_arrive(w_ready);
       }
-      eslot += (uint32_t)prm.nslots;
-      if (eslot >= ring) eslot -= ring;
       if (++buf == nacc) { buf = 0; apar ^= 1; }
     }
   }
