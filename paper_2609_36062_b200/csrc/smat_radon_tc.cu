@@ -38,6 +38,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
+
 #include "smat_internal.h"
 #include "smat_tc.cuh"
 
@@ -87,6 +89,8 @@ struct RadonParams {
   int32_t alu_rows;                // output indices parts*rows_pp .. (all of the extra class) summed on the ALUs by the
                                    // last part, straight from the ring slot; 0: every index goes through the MMAs
   int32_t ring;                    // ring slots
+  int32_t tma_out;                 // the output tile leaves through the item's own ring slot and TMA stores (q = 11)
+  int32_t mini_bytes;              // tma_out: per slot, room for the extra-class rows of the tile (two halves)
   int32_t nph;                     // 1, or 2: both stages of the d = 4 tabulation, slab by slab
   int32_t slabs_per_head;          // rp / 128
   int64_t slabs;                   // heads * slabs_per_head
@@ -212,6 +216,26 @@ __device__ __forceinline__ void st_global_v4_hint(void* dst, uint32_t w0, uint32
                : "memory");
 }
 
+// Tile stores: shared memory (box layout, 128-byte swizzle) -> global, as one bulk group per item.
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, const void* smem_src, int c0, int c1, int c2, int c3,
+                                             int c4, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4, %5, %6}], [%1], %7;"
+      ::"l"(map), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(pol)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void* smem_src, int c0, int c1, int c2, int c3,
+                                             uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4, %5}], [%1], %6;"
+      ::"l"(map), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // D[tmem_d] (+)= A[tmem_a] * B[desc_b]: A (128 x 16, bf16) read from tensor memory, B from shared memory.
 __device__ __forceinline__ void mma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
                                             uint32_t accumulate) {
@@ -251,6 +275,10 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
                                                                     const __grid_constant__ CUtensorMap tm_vert0,
                                                                     const __grid_constant__ CUtensorMap tm_reg1,
                                                                     const __grid_constant__ CUtensorMap tm_vert1,
+                                                                    const __grid_constant__ CUtensorMap tm_oreg0,
+                                                                    const __grid_constant__ CUtensorMap tm_overt0,
+                                                                    const __grid_constant__ CUtensorMap tm_oreg1,
+                                                                    const __grid_constant__ CUtensorMap tm_overt1,
                                                                     const RadonParams prm) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -258,25 +286,35 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   const int slot_bytes = prm.sr * 256;                          // two 64-entry blocks of sr rows x 128 bytes
   const int kt = prm.nslots * prm.sr;                           // operand rows per image
   uint8_t* sRing = smem;
-  int32_t* out_tab = reinterpret_cast<int32_t*>(sRing + prm.ring * slot_bytes);    // [2][128]
+  uint8_t* sMini = sRing + prm.ring * slot_bytes;                                  // [ring] extra-class rows (tma_out)
+  int32_t* out_tab = reinterpret_cast<int32_t*>(sMini + prm.ring * prm.mini_bytes);  // [2][128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(out_tab + 2 * TILE_ROWS);
   uint64_t* full = bars;                    // [ring] slot filled (TMA bytes)
   uint64_t* empty = bars + prm.ring;        // [ring] slot consumed by the MMAs (arrival from the epilogue, once the item is complete)
   uint64_t* acc_full = empty + prm.ring;    // [MAX_ACC] accumulator complete
   uint64_t* acc_empty = acc_full + MAX_ACC; // [MAX_ACC] accumulator read out (one arrival per epilogue warp)
   uint64_t* w_ready = acc_empty + MAX_ACC;  // phase 0 of the current slab written out (one arrival per storing warp)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(w_ready + 1);
+  uint64_t* staged = w_ready + 1;           // [ring] tma_out: the item's tile is complete in its slot (one arrival per epilogue warp)
+  uint64_t* alu_done = staged + prm.ring;   // [ring] tma_out: the ALU warps have read the slot and written their rows
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(alu_done + prm.ring);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const WaitCtx wc{cta_abort, prm.status};
   const int part = blockIdx.x % prm.parts;
   const bool alu_here = prm.alu_rows > 0 && part == prm.parts - 1;
+  const bool tma_out = prm.tma_out != 0;
 
   if (threadIdx.x == 0) {
     *cta_abort = 0;
-    for (int s = 0; s < prm.ring; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, alu_here ? 1 + ALU_WARPS : 1); }
+    for (int s = 0; s < prm.ring; ++s) {
+      mbar_init(full + s, 1);
+      mbar_init(empty + s, tma_out ? 1 : (alu_here ? 1 + ALU_WARPS : 1));   // tma_out: the storing thread frees the slot
+      mbar_init(alu_done + s, ALU_WARPS);
+      mbar_init(staged + s, EPI_WARPS);
+    }
     for (int b = 0; b < MAX_ACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, EPI_WARPS); }
-    mbar_init(w_ready, alu_here ? EPI_WARPS + ALU_WARPS : EPI_WARPS);
+    mbar_init(w_ready, tma_out ? 1 : (alu_here ? EPI_WARPS + ALU_WARPS : EPI_WARPS));
+
     fence_barrier_init();
     prefetch_tmap(&tm_reg0);
     prefetch_tmap(&tm_vert0);
@@ -286,7 +324,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   // This CTA's part of R, built row by row in the (still unused) ring and moved to tensor memory: lane = output
   // index, one column per two operand rows.  The launcher guarantees ring * slot_bytes >= 128 * kt * 2.
   __nv_bfloat16* scratch = reinterpret_cast<__nv_bfloat16*>(sRing);
-  for (int c = threadIdx.x; c < prm.ring * slot_bytes / 16; c += blockDim.x)
+  for (int c = threadIdx.x; c < prm.ring * (slot_bytes + prm.mini_bytes) / 16; c += blockDim.x)
     reinterpret_cast<uint4*>(sRing)[c] = make_uint4(0u, 0u, 0u, 0u);
   for (int n = threadIdx.x; n < TILE_ROWS; n += blockDim.x)
     for (int h = 0; h < prm.nph; ++h)
@@ -376,6 +414,49 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     // MMAs, commits: more than the tensor pipe needs for it) overlaps with the other thread's item.  Both phases
     // share R and the slot layout, so the issuers only count items. ---------------------------------------------
     const uint32_t me = (uint32_t)(warp - MMA_WARP);
+    if (tma_out && me == 1) {
+      // ---- storing thread (the second issuing thread has no items when every item is one slot): one bulk group
+      // of tile stores per item; a slot goes back to the producer when the stores of its item have read it --------
+      const uint32_t ring = (uint32_t)prm.ring;
+      uint32_t slot = 0, par = 0, prev_slot = 0;
+      bool have_prev = false;
+      for (ItemIter it(prm, first, step); it.left; it.next()) {
+        const RadonPhase& ph = prm.ph[it.ph];
+        const CUtensorMap* oreg = it.ph ? &tm_oreg1 : &tm_oreg0;
+        const CUtensorMap* overt = it.ph ? &tm_overt1 : &tm_overt0;
+        const uint32_t head = it.slab / sph;
+        const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
+        const int hc = ph.dst_private ? (int)blockIdx.x : (int)head;
+        const uint64_t pol = it.ph ? pol_dst1 : pol_dst0;
+        if (!mbar_wait(staged + slot, par, wc)) break;
+        const uint8_t* tile = sRing + slot * slot_bytes;
+        tma_store_5d(oreg, tile, e0, 0, 0, (int)it.img, hc, pol);
+        tma_store_5d(oreg, tile + prm.sr * 128, e0 + 64, 0, 0, (int)it.img, hc, pol);
+        if (ph.out.count > q * q && (int)it.img >= ph.out.vert_from) {
+          const uint8_t* mini = sMini + slot * prm.mini_bytes;
+          const int ci = ph.out.sv_img != 0 ? (int)it.img : 0;   // the map's image stride is sv_img rows
+          tma_store_4d(overt, mini, e0, 0, ci, hc, pol);
+          tma_store_4d(overt, mini + prm.mini_bytes / 2, e0 + 64, 0, ci, hc, pol);
+        }
+        bulk_commit();
+        if (have_prev) {
+          bulk_wait_read<1>();
+          mbar_arrive(empty + prev_slot);
+        }
+        if (it.closes_phase0()) {   // the slab's stage-1 rows are in memory before the producer loads them back
+          bulk_wait_all();
+          fence_proxy_async_all();
+          mbar_arrive(empty + slot);
+          mbar_arrive(w_ready);
+          have_prev = false;
+        } else {
+          prev_slot = slot;
+          have_prev = true;
+        }
+        if (++slot == ring) { slot = 0; par ^= 1; }
+      }
+      bulk_wait_all();
+    }
     constexpr uint32_t idesc = make_idesc(TILE_ROWS, 128, 0, 1);   // A from tensor memory (R), B MN-major (image rows)
     const uint64_t dB0 = make_desc(smem_u32(sRing), prm.sr * 128, 1024);
     const uint32_t slot16 = (uint32_t)slot_bytes >> 4;            // descriptor address units are 16 bytes
@@ -396,7 +477,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
         if (!ok) break;
         fence_after_sync();
         issue_slot_steps(steps, tmem_acc + buf * 128, tmem_base, dB0 + (uint64_t)(slot * slot16), idesc, true);
-        mma_commit(empty + slot);
+        if (!tma_out) mma_commit(empty + slot);   // tma_out: the storing thread frees the slot once the tile has left it
         mma_commit(acc_full + buf);
         if (++slot == ring) { slot = 0; par ^= 1; }
         if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
@@ -460,11 +541,25 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
               acc[4] += __uint_as_float(w.z << 16); acc[5] += __uint_as_float(w.z & 0xffff0000u);
               acc[6] += __uint_as_float(w.w << 16); acc[7] += __uint_as_float(w.w & 0xffff0000u);
             }
-            const int row = ph.out.v0 + (int)it.img * ph.out.sv_img + u * ph.out.sv_lo;
-            __nv_bfloat16* dst = ph.dst + (hrow + row) * ph.dst_pitch + e0 + ch * 8;
-            st_global_v4_hint(dst, pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
-                              pack_bf16(acc[6], acc[7]), it.ph ? pol_dst1 : pol_dst0);
+            if (tma_out) {   // into the slot's extra-class rows, from where the storing thread sends them with the tile
+              uint8_t* mrow = sMini + slot * prm.mini_bytes + (ch >> 3) * (prm.mini_bytes / 2) + u * 128;
+              *reinterpret_cast<uint4*>(mrow + (((ch & 7) ^ (u & 7)) << 4)) =
+                  make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                             pack_bf16(acc[6], acc[7]));
+            } else {
+              const int row = ph.out.v0 + (int)it.img * ph.out.sv_img + u * ph.out.sv_lo;
+              __nv_bfloat16* dst = ph.dst + (hrow + row) * ph.dst_pitch + e0 + ch * 8;
+              st_global_v4_hint(dst, pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                                pack_bf16(acc[6], acc[7]), it.ph ? pol_dst1 : pol_dst0);
+            }
           }
+        }
+        if (tma_out) {
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(alu_done + slot);
+          if (++slot == ring) { slot = 0; par ^= 1; }
+          continue;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty + slot);
@@ -485,7 +580,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
     const int tv0 = out_tab[orow], tv1 = prm.nph > 1 ? out_tab[TILE_ROWS + orow] : ROW_INVALID;
     const bool active = qd * 32 < prm.rows_pp;                  // warp-uniform: some output index in these lanes
-    uint32_t buf = 0, apar = 0, eslot = 0;
+    uint32_t buf = 0, apar = 0, eslot = 0, epar = 0;
     for (ItemIter it(prm, first, step); it.left; it.next()) {
       const RadonPhase& ph = prm.ph[it.ph];
       const uint32_t head = it.slab / sph;
@@ -494,6 +589,37 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
       const int tv = it.ph ? tv1 : tv0;
       if (!mbar_wait_warp(acc_full + buf, apar, wc)) break;
       fence_after_sync();
+      if (tma_out) {
+        // The tile leaves through the item's own slot (the MMAs are done with it): every thread writes its 64 bytes
+        // in the box layout of a TMA tile — regular indices into the slot (row = index), extra-class indices into
+        // the slot's extra rows — and the storing thread sends the tile off.  The LSU sees 4 wavefronts per warp
+        // store instead of 32, and the bulk of the traffic bypasses it.
+        uint32_t v[32];
+        tmem_ld32(tmem_acc + lane_base + buf * 128 + cb * 32, v);
+        tmem_ld_wait();
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty + buf);             // the accumulator is in registers
+        if (alu_here && !mbar_wait_warp(alu_done + eslot, epar, wc)) break;   // the ALU warps have read the image
+        if (tv != ROW_INVALID) {
+          const int idx = orow < q * q ? orow : orow - q * q;     // row of the tile / of the extra rows
+          uint8_t* trow = (orow < q * q ? sRing + eslot * slot_bytes + (cb >> 1) * prm.sr * 128
+                                        : sMini + eslot * prm.mini_bytes + (cb >> 1) * (prm.mini_bytes / 2)) + idx * 128;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            *reinterpret_cast<uint4*>(trow + ((((cb & 1) * 4 + j) ^ (idx & 7)) << 4)) =
+                make_uint4(pack_bf16(__uint_as_float(v[8 * j]), __uint_as_float(v[8 * j + 1])),
+                           pack_bf16(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3])),
+                           pack_bf16(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5])),
+                           pack_bf16(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7])));
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(staged + eslot);
+        if (++eslot == (uint32_t)prm.ring) { eslot = 0; epar ^= 1; }
+        if (++buf == nacc) { buf = 0; apar ^= 1; }
+        continue;
+      }
       if (warp == 0 && prm.nslots > 1) {   // every MMA of the item has completed: its ring slots are free (a commit per slot would cost the
                          // issuing thread more than the MMAs of the slot)
         for (int g = 0; g < prm.nslots; ++g) {
@@ -661,13 +787,26 @@ cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int
   prm.parts = sh.parts; prm.rows_pp = sh.rows_pp; prm.alu_rows = sh.alu_rows;
   prm.ring = sh.ring; prm.nph = nph; prm.slabs_per_head = (int)(rp / 128); prm.slabs = (int64_t)bh * (rp / 128);
   prm.status = status;
+  // One slot per item, as large as an output tile, one CTA per image (q = 11, forward): the tile is stored by TMA
+  // from the item's own slot; every slot gets room for the q extra-class rows of its tile (two 64-entry halves).
+  int smem = sh.smem;
+  prm.tma_out = 0; prm.mini_bytes = 0;
+  if (!transpose && sh.nslots == 1 && sh.sr == TILE_ROWS && sh.parts == 1 && !getenv("SMAT_NO_TMA_OUT")) {
+    const int mini = 2 * ((q + 7) & ~7) * 128, slot = sh.sr * 256;
+    int ring = (227 * 1024 - 1024 - 512 - TILE_ROWS * 8) / (slot + mini);
+    if (ring > sh.ring) ring = sh.ring;
+    if (ring >= 4) {
+      prm.tma_out = 1; prm.mini_bytes = mini; prm.ring = ring;
+      smem = ring * (slot + mini) + TILE_ROWS * 8 + 512 + 1024;
+    }
+  }
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   int64_t ctas = (int64_t)(sms / sh.parts) * sh.parts;
   const int64_t items = nph == 1 ? prm.slabs * sp[0].images * sh.parts : prm.slabs;
   if (items < ctas) ctas = items;
-  CUtensorMap tm_reg[2], tm_vert[2];
+  CUtensorMap tm_reg[2], tm_vert[2], tm_oreg[2], tm_overt[2];
   for (int i = 0; i < nph; ++i) {
     RadonPhase& ph = prm.ph[i];
     const RadonSide& in = sp[i].in;
@@ -696,11 +835,32 @@ cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int
     } else {
       tm_vert[i] = tm_reg[i];
     }
+    tm_oreg[i] = tm_reg[i]; tm_overt[i] = tm_reg[i];
+    if (prm.tma_out) {   // the same two shapes over the output rows: boxes of q lines, and of the extra class
+      const RadonSide& out = sp[i].out;
+      const int64_t dst_rp = sp[i].dst_private ? 128 : rp, dst_heads = sp[i].dst_private ? ctas : bh;
+      const int64_t sizes[4] = {q, q, images, dst_heads};
+      const int64_t strides[4] = {out.s_lo, out.s_hi, images > 1 ? out.s_img : out.rows_per_head, out.rows_per_head};
+      const int box[4] = {q, q, 1, 1};
+      if (!radon_map(&tm_oreg[i], sp[i].dst, dst_rp, 5, sizes, strides, box)) return cudaErrorInvalidValue;
+      if (out.count > q * q) {
+        const bool per_image = out.sv_img != 0;
+        const int64_t vsizes[3] = {q, per_image ? images : 1, dst_heads};
+        const int64_t vstrides[3] = {out.sv_lo, per_image ? out.sv_img : out.rows_per_head, out.rows_per_head};
+        const int vbox[3] = {q, 1, 1};
+        if (!radon_map(&tm_overt[i], static_cast<__nv_bfloat16*>(sp[i].dst) + (int64_t)out.v0 * dst_rp, dst_rp, 4, vsizes,
+                       vstrides, vbox))
+          return cudaErrorInvalidValue;
+      }
+    }
   }
-  if (nph == 1) { prm.ph[1] = prm.ph[0]; tm_reg[1] = tm_reg[0]; tm_vert[1] = tm_vert[0]; }
-  cudaError_t err = cudaFuncSetAttribute(radon_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.smem);
+  if (nph == 1) {
+    prm.ph[1] = prm.ph[0]; tm_reg[1] = tm_reg[0]; tm_vert[1] = tm_vert[0]; tm_oreg[1] = tm_oreg[0]; tm_overt[1] = tm_overt[0];
+  }
+  cudaError_t err = cudaFuncSetAttribute(radon_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (err != cudaSuccess) return err;
-  radon_tc_kernel<<<(unsigned)ctas, RADON_THREADS, sh.smem, st>>>(tm_reg[0], tm_vert[0], tm_reg[1], tm_vert[1], prm);
+  radon_tc_kernel<<<(unsigned)ctas, RADON_THREADS, smem, st>>>(tm_reg[0], tm_vert[0], tm_reg[1], tm_vert[1], tm_oreg[0],
+                                                              tm_overt[0], tm_oreg[1], tm_overt[1], prm);
   return cudaGetLastError();
 }
 
