@@ -104,8 +104,8 @@ struct RadonParams {
 struct ItemIter {
   uint32_t slab, img, ph, left;    // the current item, and the items left including it
   uint32_t step, slabs, nph, im0, im1;
-  __device__ __forceinline__ ItemIter(const RadonParams& p, uint32_t first, uint32_t step_) {
-    step = step_; slabs = (uint32_t)p.slabs; nph = (uint32_t)p.nph;
+  __device__ __forceinline__ ItemIter(const RadonParams& p, uint32_t first, uint32_t step_, uint32_t nph_) {
+    step = step_; slabs = (uint32_t)p.slabs; nph = nph_;
     im0 = (uint32_t)p.ph[0].images; im1 = nph > 1 ? (uint32_t)p.ph[1].images : 0u;
     ph = 0;
     if (nph == 1) {
@@ -193,6 +193,21 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            int c4, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
+      : "memory");
+}
+
 // L2 eviction policies: the exchange rows of the two-stage kernel should stay in the cache (they are rewritten for
 // every slab, and written back to memory only when evicted), the tables streaming past them should leave it first.
 enum { POLICY_NORMAL = 0, POLICY_FIRST = 1, POLICY_LAST = 2 };
@@ -271,6 +286,9 @@ __device__ __forceinline__ void issue_slot_steps(int steps, uint32_t tmem_d, uin
   }
 }
 
+// FEAT = false is the plain instantiation (one stage per launch, every index through the MMAs, direct stores, no cache
+// hints): the single-thread roles pay for every instruction, and the prime-specific paths would cost the others time.
+template <bool FEAT>
 __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid_constant__ CUtensorMap tm_reg0,
                                                                     const __grid_constant__ CUtensorMap tm_vert0,
                                                                     const __grid_constant__ CUtensorMap tm_reg1,
@@ -301,8 +319,9 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const WaitCtx wc{cta_abort, prm.status};
   const int part = blockIdx.x % prm.parts;
-  const bool alu_here = prm.alu_rows > 0 && part == prm.parts - 1;
-  const bool tma_out = prm.tma_out != 0;
+  const bool alu_here = FEAT && prm.alu_rows > 0 && part == prm.parts - 1;
+  const bool tma_out = FEAT && prm.tma_out != 0;
+  const uint32_t nph = FEAT ? (uint32_t)prm.nph : 1u;
 
   if (threadIdx.x == 0) {
     *cta_abort = 0;
@@ -318,7 +337,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     fence_barrier_init();
     prefetch_tmap(&tm_reg0);
     prefetch_tmap(&tm_vert0);
-    if (prm.nph > 1) { prefetch_tmap(&tm_reg1); prefetch_tmap(&tm_vert1); }
+    if (nph > 1) { prefetch_tmap(&tm_reg1); prefetch_tmap(&tm_vert1); }
   }
   if (warp == MMA_WARP) tmem_alloc(tmem_slot, 512);
   // This CTA's part of R, built row by row in the (still unused) ring and moved to tensor memory: lane = output
@@ -327,7 +346,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   for (int c = threadIdx.x; c < prm.ring * (slot_bytes + prm.mini_bytes) / 16; c += blockDim.x)
     reinterpret_cast<uint4*>(sRing)[c] = make_uint4(0u, 0u, 0u, 0u);
   for (int n = threadIdx.x; n < TILE_ROWS; n += blockDim.x)
-    for (int h = 0; h < prm.nph; ++h)
+    for (int h = 0; h < (int)nph; ++h)
       out_tab[h * TILE_ROWS + n] = n < prm.rows_pp ? side_row(prm.ph[h].out, part * prm.rows_pp + n, q) : ROW_INVALID;
   fence_before_sync();
   __syncthreads();
@@ -358,10 +377,10 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   const uint32_t tmem_acc = tmem_base + r_cols;
 
   // per phase: streaming tables, or the exchange rows (two-stage kernel only)
-  const uint64_t pol_src0 = l2_policy(prm.nph > 1 ? (prm.ph[0].src_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
-  const uint64_t pol_src1 = l2_policy(prm.nph > 1 ? (prm.ph[1].src_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
-  const uint64_t pol_dst0 = l2_policy(prm.nph > 1 ? (prm.ph[0].dst_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
-  const uint64_t pol_dst1 = l2_policy(prm.nph > 1 ? (prm.ph[1].dst_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
+  const uint64_t pol_src0 = l2_policy(nph > 1 ? (prm.ph[0].src_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
+  const uint64_t pol_src1 = l2_policy(nph > 1 ? (prm.ph[1].src_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
+  const uint64_t pol_dst0 = l2_policy(nph > 1 ? (prm.ph[0].dst_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
+  const uint64_t pol_dst1 = l2_policy(nph > 1 ? (prm.ph[1].dst_private ? POLICY_LAST : POLICY_FIRST) : POLICY_NORMAL);
   // items of this CTA: same part always
   const uint32_t first = blockIdx.x / prm.parts, step = gridDim.x / prm.parts;
   const uint32_t sph = (uint32_t)prm.slabs_per_head;
@@ -374,10 +393,10 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     uint32_t wpar = 0;                                        // parity of w_ready for the current slab
     bool first_lap = true, ok = true;
     const uint32_t reg_bytes = 2u * 128u * (uint32_t)(q * prm.sps), vert_bytes = 2u * 128u * (uint32_t)q;
-    for (ItemIter it(prm, first, step); it.left && ok; it.next()) {
-      const RadonPhase& ph = prm.ph[it.ph];
-      const CUtensorMap* tm_reg = it.ph ? &tm_reg1 : &tm_reg0;
-      const CUtensorMap* tm_vert = it.ph ? &tm_vert1 : &tm_vert0;
+    for (ItemIter it(prm, first, step, nph); it.left && ok; it.next()) {
+      const RadonPhase& ph = FEAT ? prm.ph[it.ph] : prm.ph[0];
+      const CUtensorMap* tm_reg = FEAT && it.ph ? &tm_reg1 : &tm_reg0;
+      const CUtensorMap* tm_vert = FEAT && it.ph ? &tm_vert1 : &tm_vert0;
       const uint32_t head = it.slab / sph;
       const int e0 = ph.src_private ? 0 : (int)(it.slab - head * sph) * 128;
       const int hc = ph.src_private ? (int)blockIdx.x : (int)head;
@@ -394,14 +413,24 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
         uint8_t* dst = sRing + slot * slot_bytes;
         if (g < prm.nreg) {   // lines hi = g*sps ..; lines past q - 1 are out of bounds and arrive as zeros
           mbar_expect_tx(full + slot, reg_bytes);
-          tma_load_5d(dst, tm_reg, e0, 0, g * prm.sps, (int)it.img, hc, full + slot, pol);
-          tma_load_5d(dst + prm.sr * 128, tm_reg, e0 + 64, 0, g * prm.sps, (int)it.img, hc, full + slot, pol);
+          if (FEAT) {
+            tma_load_5d(dst, tm_reg, e0, 0, g * prm.sps, (int)it.img, hc, full + slot, pol);
+            tma_load_5d(dst + prm.sr * 128, tm_reg, e0 + 64, 0, g * prm.sps, (int)it.img, hc, full + slot, pol);
+          } else {
+            tma_load_5d(dst, tm_reg, e0, 0, g * prm.sps, (int)it.img, hc, full + slot);
+            tma_load_5d(dst + prm.sr * 128, tm_reg, e0 + 64, 0, g * prm.sps, (int)it.img, hc, full + slot);
+          }
         } else {              // extra class; an image without it reads past the last head: zeros
           const int h = (int)it.img >= ph.in.vert_from ? hc : ph.src_heads;
           const int ci = (int)it.img * ph.in.sv_img;   // 0 when every image shares the rows
           mbar_expect_tx(full + slot, vert_bytes);
-          tma_load_4d(dst, tm_vert, e0, 0, ci, h, full + slot, pol);
-          tma_load_4d(dst + prm.sr * 128, tm_vert, e0 + 64, 0, ci, h, full + slot, pol);
+          if (FEAT) {
+            tma_load_4d(dst, tm_vert, e0, 0, ci, h, full + slot, pol);
+            tma_load_4d(dst + prm.sr * 128, tm_vert, e0 + 64, 0, ci, h, full + slot, pol);
+          } else {
+            tma_load_4d(dst, tm_vert, e0, 0, ci, h, full + slot);
+            tma_load_4d(dst + prm.sr * 128, tm_vert, e0 + 64, 0, ci, h, full + slot);
+          }
         }
         if (++slot == (uint32_t)prm.ring) {
           slot = 0;
@@ -420,8 +449,8 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
       const uint32_t ring = (uint32_t)prm.ring;
       uint32_t slot = 0, par = 0, prev_slot = 0;
       bool have_prev = false;
-      for (ItemIter it(prm, first, step); it.left; it.next()) {
-        const RadonPhase& ph = prm.ph[it.ph];
+      for (ItemIter it(prm, first, step, nph); it.left; it.next()) {
+        const RadonPhase& ph = FEAT ? prm.ph[it.ph] : prm.ph[0];
         const CUtensorMap* oreg = it.ph ? &tm_oreg1 : &tm_oreg0;
         const CUtensorMap* overt = it.ph ? &tm_overt1 : &tm_overt0;
         const uint32_t head = it.slab / sph;
@@ -463,7 +492,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     const uint32_t slot_cols = (uint32_t)prm.sr / 2;              // columns of R per slot
     const int steps = prm.sr / 16, nslots = prm.nslots;
     const uint32_t ring = (uint32_t)prm.ring;
-    const uint32_t items = ItemIter(prm, first, step).left;
+    const uint32_t items = ItemIter(prm, first, step, nph).left;
     uint32_t slot = 0, par = 0;                                   // ring position and the parity its full barrier shows
     uint32_t buf = 0, apar = 0;                                   // accumulator; parity of its empty barrier's phase to wait for
     bool ok = true;
@@ -509,7 +538,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
         if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
       }
     }
-  } else if (warp >= ALU_WARP) {
+  } else if (FEAT && warp >= ALU_WARP) {
     // ---- leftover rows on the ALUs ----------------------------------------------------------------------------
     // q*q + q output indices rarely fill whole tiles of 128.  When only a few are left over, and they belong to the
     // extra class (index q*q + u = the sum of line u's q rows), these warps add the rows up from the slot itself
@@ -519,8 +548,8 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
       const int tid_a = (warp - ALU_WARP) * 32 + lane, tasks = prm.alu_rows * 16;
       const uint32_t ring = (uint32_t)prm.ring;
       uint32_t slot = 0, par = 0;
-      for (ItemIter it(prm, first, step); it.left; it.next()) {
-        const RadonPhase& ph = prm.ph[it.ph];
+      for (ItemIter it(prm, first, step, nph); it.left; it.next()) {
+        const RadonPhase& ph = FEAT ? prm.ph[it.ph] : prm.ph[0];
         const uint32_t head = it.slab / sph;
         const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
         const int64_t hrow = (int64_t)(ph.dst_private ? blockIdx.x : head) * ph.out.rows_per_head;
@@ -578,11 +607,11 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     const int qd = warp & 3, cb = warp >> 2;
     const int orow = qd * 32 + lane;                            // output index of this CTA = TMEM lane
     const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
-    const int tv0 = out_tab[orow], tv1 = prm.nph > 1 ? out_tab[TILE_ROWS + orow] : ROW_INVALID;
+    const int tv0 = out_tab[orow], tv1 = nph > 1 ? out_tab[TILE_ROWS + orow] : ROW_INVALID;
     const bool active = qd * 32 < prm.rows_pp;                  // warp-uniform: some output index in these lanes
     uint32_t buf = 0, apar = 0, eslot = 0, epar = 0;
-    for (ItemIter it(prm, first, step); it.left; it.next()) {
-      const RadonPhase& ph = prm.ph[it.ph];
+    for (ItemIter it(prm, first, step, nph); it.left; it.next()) {
+      const RadonPhase& ph = FEAT ? prm.ph[it.ph] : prm.ph[0];
       const uint32_t head = it.slab / sph;
       const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
       const int64_t hrow = (int64_t)(ph.dst_private ? blockIdx.x : head) * ph.out.rows_per_head;
@@ -642,7 +671,10 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
 #pragma unroll
             for (int i = 0; i < 8; ++i)
               w[i] = pack_bf16(__uint_as_float(v[16 * h8 + 2 * i]), __uint_as_float(v[16 * h8 + 2 * i + 1]));
-            st_global_v8_hint(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7], it.ph ? pol_dst1 : pol_dst0);
+            if (FEAT)
+              st_global_v8_hint(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7], it.ph ? pol_dst1 : pol_dst0);
+            else
+              st_global_v8(dst + 16 * h8, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
           }
         }
       }
@@ -857,10 +889,13 @@ cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int
   if (nph == 1) {
     prm.ph[1] = prm.ph[0]; tm_reg[1] = tm_reg[0]; tm_vert[1] = tm_vert[0]; tm_oreg[1] = tm_oreg[0]; tm_overt[1] = tm_overt[0];
   }
-  cudaError_t err = cudaFuncSetAttribute(radon_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const bool feat = nph > 1 || prm.alu_rows > 0 || prm.tma_out;
+  auto kernel = feat ? radon_tc_kernel<true> : radon_tc_kernel<false>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (err != cudaSuccess) return err;
-  radon_tc_kernel<<<(unsigned)ctas, RADON_THREADS, smem, st>>>(tm_reg[0], tm_vert[0], tm_reg[1], tm_vert[1], tm_oreg[0],
-                                                              tm_overt[0], tm_oreg[1], tm_overt[1], prm);
+  // the plain instantiation has no use for the two ALU warps
+  kernel<<<(unsigned)ctas, feat ? RADON_THREADS : 32 * ALU_WARP, smem, st>>>(tm_reg[0], tm_vert[0], tm_reg[1], tm_vert[1],
+                                                                            tm_oreg[0], tm_overt[0], tm_oreg[1], tm_overt[1], prm);
   return cudaGetLastError();
 }
 
