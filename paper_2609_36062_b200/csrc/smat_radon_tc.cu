@@ -34,6 +34,11 @@
 // entries, rewritten for every slab, stored and loaded with the L2 evict-last priority while F and U stream with
 // evict-first) and the full-size W table is never built.  The storing warps make the slab's rows visible (memory
 // fence, proxy fence) and arrive on a barrier the producer waits on before the first stage-2 load.
+// q = 11 also sends its output tiles off by TMA: the epilogue writes the rounded tile into the item's own ring slot
+// (as large as a tile, and dead once the MMAs have read it) in the box layout, and lane 0 of warp 18 issues the tile
+// stores and frees the slot; the bulk of the stores bypasses the LSU.
+// The kernel exists twice: radon_tc_kernel<false> without any of the prime-specific paths (q = 13, 17, 19 and
+// everything with one stage per launch and no leftover rows), radon_tc_kernel<true> with them.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
