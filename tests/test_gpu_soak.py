@@ -29,14 +29,16 @@ def test_repeated_forward_passes_leave_the_status_clean(d, batch, heads, T, dv, 
     assert torch.equal(out, first)
 
 
-def test_repeated_backward_passes_leave_the_status_clean():
-    w = synth.Workload("soak", 3, 2, 8, 4096, 128, 128, 64, "bf16", "normalised", 311)
+# d = 3 (q = 13, transposed Radon stage with three slots per image) and d = 4 (q = 11, both transposed stages in one launch)
+@pytest.mark.parametrize("d,batch,heads,T,c,passes", [(3, 2, 8, 4096, 64, 100), (4, 1, 4, 16384, 128, 40)])
+def test_repeated_backward_passes_leave_the_status_clean(d, batch, heads, T, c, passes):
+    w = synth.Workload("soak", d, batch, heads, T, 128, 128, c, "bf16", "normalised", 311)
     _, dev = device_inputs(w, ("q", "k", "v", "do"))
     plan = binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype)
     plan.forward(dev["q"], dev["k"], dev["v"])
     first = [g.clone() for g in plan.backward(dev["q"], dev["k"], dev["v"], dev["do"])]
     plan.check_status()
-    for i in range(100):
+    for i in range(passes):
         plan.forward(dev["q"], dev["k"], dev["v"])
         plan.check_status()
         grads = plan.backward(dev["q"], dev["k"], dev["v"], dev["do"])
