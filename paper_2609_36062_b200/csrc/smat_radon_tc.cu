@@ -496,6 +496,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     const uint32_t slot16 = (uint32_t)slot_bytes >> 4;            // descriptor address units are 16 bytes
     const uint32_t slot_cols = (uint32_t)prm.sr / 2;              // columns of R per slot
     const int steps = prm.sr / 16, nslots = prm.nslots;
+    const int steps_last = ((q - (prm.nreg - 1) * prm.sps) * q + 15) / 16, steps_extra = (q + 15) / 16;
     const uint32_t ring = (uint32_t)prm.ring;
     const uint32_t items = ItemIter(prm, first, step, nph).left;
     uint32_t slot = 0, par = 0;                                   // ring position and the parity its full barrier shows
@@ -536,7 +537,10 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
           ok = mbar_wait(full + slot, par, wc);
           if (!ok) break;
           fence_after_sync();
-          issue_slot_steps(steps, tmem_d, tmem_a, dB0 + (uint64_t)(slot * slot16), idesc, g == 0);
+          // the last slot of regular lines and the slot of the extra class hold fewer rows than a full slot: R has
+          // only zeros for the rest, so their K-steps are left out
+          const int st = g + 1 < prm.nreg ? steps : (g < prm.nreg ? steps_last : steps_extra);
+          issue_slot_steps(st, tmem_d, tmem_a, dB0 + (uint64_t)(slot * slot16), idesc, g == 0);
           if (++slot == ring) { slot = 0; par ^= 1; }
         }
         if (ok) mma_commit(acc_full + buf);   // the only commit of the item: the epilogue frees its slots when it sees it
