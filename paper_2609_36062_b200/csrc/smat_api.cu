@@ -436,11 +436,13 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
     }
     if (L >= 2) {  // steps 5-7, two-level: segment totals, scan of the totals, fused per-segment output
       float* seg = cx.f(pl->off_sin);
-      const int64_t nseg = pl->T / 128 / L, nseg0 = tiles0 / L;
-      SMAT_TRY(cx, "segment_state_tc", smat_launch_segment_state_tc(K, V, seg, pl->T, L, pl->bh, status, cx.st));
+      int nseg0 = 0, nseg1 = 0;
+      smat_segment_counts(tiles0, tiles1, pl->bh, L, &nseg0, &nseg1);
+      const int64_t nseg = nseg0 + nseg1;
+      SMAT_TRY(cx, "segment_state_tc", smat_launch_segment_state_tc(K, V, seg, tiles0, tiles1, nseg0, nseg1, pl->bh, status, cx.st));
       SMAT_TRY(cx, "segment_scan", smat_launch_scan(seg, pl->rp, nseg, pl->bh, 0, nseg0, nseg0, nseg, 0, cx.st));
       SMAT_TRY(cx, "segment_output_tc", smat_launch_segment_output_tc(Q, K, V, seg, ylr, lr ? pl->geo.n : pl->T, O,
-                                                                       pl->T, L, pl->bh, status, cx.st));
+                                                                       tiles0, tiles1, nseg0, nseg1, pl->bh, status, cx.st));
     } else {
       SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, pl->geo.n,
                                                                lr ? 0 : 1, 0, status, cx.st));   // steps 5-6

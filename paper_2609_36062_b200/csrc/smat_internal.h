@@ -131,8 +131,9 @@ cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_b
                                 int64_t groups, int64_t max_tokens, int64_t T, int bh, int* status, cudaStream_t st);
 // Two-level causal branch: segment totals, then (after an exclusive scan of the totals) per-segment fused output.
 int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh);
-cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* totals, int64_t T, int L, int bh,
-                                         int* status, cudaStream_t st);
+void smat_segment_counts(int64_t tiles0, int64_t tiles1, int bh, int L, int* nseg0, int* nseg1);
+cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* totals, int64_t tiles0, int64_t tiles1,
+                                         int nseg0, int nseg1, int bh, int* status, cudaStream_t st);
 cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const void* V, const float* seg_in,
-                                          const void* ylr_bf16, int64_t n_lr, void* O, int64_t T, int L, int bh,
-                                          int* status, cudaStream_t st);
+                                          const void* ylr_bf16, int64_t n_lr, void* O, int64_t tiles0, int64_t tiles1,
+                                          int nseg0, int nseg1, int bh, int* status, cudaStream_t st);

@@ -356,9 +356,28 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
 constexpr int SEG_STATE_STAGES = 3;
 constexpr int SEG_STATE_SMEM = SEG_STATE_STAGES * 4 * BOX_BYTES + 1024 + 256;
 
+// Segments of the two-level causal branch: block 0 (tiles0 tiles) is cut into nseg0 segments, block 1 into
+// nseg - nseg0, as evenly as whole tiles allow (lengths differ by at most one tile), so that the segment count can
+// be matched to the number of SMs.  Segment `seg` covers tiles [*tile0, *tile0 + *count).
+struct SegCut {
+  int nseg0, nseg;
+  int64_t tiles0, tiles1;
+};
+__device__ __forceinline__ void seg_range(const SegCut& c, int seg, int64_t* tile0, int* count) {
+  if (seg < c.nseg0) {
+    const int64_t a = (int64_t)seg * c.tiles0 / c.nseg0, b = (int64_t)(seg + 1) * c.tiles0 / c.nseg0;
+    *tile0 = a; *count = (int)(b - a);
+  } else {
+    const int s = seg - c.nseg0, n1 = c.nseg - c.nseg0;
+    const int64_t a = (int64_t)s * c.tiles1 / n1, b = (int64_t)(s + 1) * c.tiles1 / n1;
+    *tile0 = c.tiles0 + a; *count = (int)(b - a);
+  }
+}
+
 struct SegStateParams {
   int64_t T;
-  int L, nseg;           // tiles per segment, segments per head
+  SegCut cut;
+  int nseg;              // segments per head
   float* totals;         // [bh][nseg][128][128]
   int* status;
 };
@@ -376,6 +395,9 @@ __global__ void __launch_bounds__(192) segment_state_tc_kernel(const __grid_cons
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int seg = blockIdx.x, bh = blockIdx.y;
+  int64_t tile0;
+  int Lc;
+  seg_range(prm.cut, seg, &tile0, &Lc);
   const WaitCtx wc{cta_abort, prm.status};
   if (threadIdx.x == 0) {
     *cta_abort = 0;
@@ -389,11 +411,11 @@ __global__ void __launch_bounds__(192) segment_state_tc_kernel(const __grid_cons
   fence_after_sync();
   const uint32_t tmem_d = *tmem_slot;
   if (warp == 4 && lane == 0) {
-    for (int it = 0; it < prm.L; ++it) {
+    for (int it = 0; it < Lc; ++it) {
       const int s = it % SEG_STATE_STAGES;
       if (it >= SEG_STATE_STAGES && !mbar_wait(empty + s, ((it / SEG_STATE_STAGES) - 1) & 1, wc)) break;
       uint8_t* st = smem + s * 4 * BOX_BYTES;
-      const int row = (int)((int64_t)bh * prm.T + ((int64_t)seg * prm.L + it) * TILE);
+      const int row = (int)((int64_t)bh * prm.T + (tile0 + it) * TILE);
       mbar_expect_tx(full + s, 4 * BOX_BYTES);
       tma_load_2d(st, &tmK, 0, row, full + s);
       tma_load_2d(st + BOX_BYTES, &tmK, HALF, row, full + s);
@@ -403,7 +425,7 @@ __global__ void __launch_bounds__(192) segment_state_tc_kernel(const __grid_cons
   } else if (warp == 5 && lane == 0) {
     constexpr uint32_t idesc = make_idesc(TILE, TILE, 1, 1);
     bool ok = true;
-    for (int it = 0; it < prm.L && ok; ++it) {
+    for (int it = 0; it < Lc && ok; ++it) {
       const int s = it % SEG_STATE_STAGES;
       ok = mbar_wait(full + s, (it / SEG_STATE_STAGES) & 1, wc);
       if (!ok) break;
@@ -449,7 +471,8 @@ constexpr int SEG_OUT_SMEM = 2 * SEG_OUT_STAGE + 2 * BOX_BYTES + 1024 + 256;
 
 struct SegOutParams {
   int64_t T;
-  int L, nseg;
+  SegCut cut;
+  int nseg;
   const float* seg_in;   // [bh][nseg][128][128] state entering each segment
   int64_t n_lr;
   const __nv_bfloat16* ylr;   // [bh][T][128] long-range rows, bf16 (rows t >= n_lr are added)
@@ -484,6 +507,9 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int seg = blockIdx.x, bh = blockIdx.y;
+  int64_t tile0;
+  int Lc;
+  seg_range(prm.cut, seg, &tile0, &Lc);
   const WaitCtx wc{cta_abort, prm.status};
   if (threadIdx.x == 0) {
     *cta_abort = 0;
@@ -498,10 +524,9 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_sc = tmem_base + TILE, tmem_o0 = tmem_base + 2 * TILE;
-  const int64_t tile0 = (int64_t)seg * prm.L;
 
   if (warp == SEG_EPI_WARPS && lane == 0) {
-    for (int it = 0; it < prm.L; ++it) {
+    for (int it = 0; it < Lc; ++it) {
       const int s = it & 1;
       if (it >= 2 && !mbar_wait(empty + s, ((it >> 1) - 1) & 1, wc)) break;
       uint8_t* st = smem + s * SEG_OUT_STAGE;
@@ -532,7 +557,7 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
       dK_mn[s] = make_desc(sQ + 2 * BOX_BYTES, BOX_BYTES, 1024);
       dV_mn[s] = make_desc(sQ + 4 * BOX_BYTES, BOX_BYTES, 1024);
     }
-    for (int it = 0; it < prm.L; ++it) {
+    for (int it = 0; it < Lc; ++it) {
       const int s = it & 1;
       const uint64_t qk = s ? dQ_k[1] : dQ_k[0], kk_ = s ? dK_k[1] : dK_k[0];
       const uint64_t kmn = s ? dK_mn[1] : dK_mn[0], vmn = s ? dV_mn[1] : dV_mn[0];
@@ -604,7 +629,7 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
       tmem_st_wait();
       publish_state(v);
     }
-    for (int it = 0; it < prm.L; ++it) {
+    for (int it = 0; it < Lc; ++it) {
       // --- scores of this tile -> masked bf16 P (registers), stored once O = Q S has consumed the shared tile ---
       if (!mbar_wait(bar_sc, it & 1, wc)) break;
       fence_after_sync();
@@ -643,7 +668,7 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
       }
       if (!mbar_wait(bar_o, it & 1, wc)) break;
       fence_after_sync();
-      if (it + 1 < prm.L) {  // the state now includes this tile: publish it for the next one first (critical path)
+      if (it + 1 < Lc) {  // the state now includes this tile: publish it for the next one first (critical path)
         uint32_t v[32];
         tmem_ld32(tmem_s + lane_base + col0, v);
         tmem_ld_wait();
@@ -1218,12 +1243,48 @@ int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh) {
   return 1;
 }
 
-cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* totals, int64_t T, int L, int bh,
-                                         int* status, cudaStream_t st) {
+// Segment counts of the two blocks.  The output kernel runs one CTA per SM and a CTA walks its segment tile by tile,
+// so the launch takes ceil(segments * heads / SMs) rounds of the longest segment: the counts are chosen to fill the
+// last round (t64k with 16 heads: 37 segments of 13 or 14 tiles = 4 full rounds, where 32 segments of 16 tiles leave
+// the fourth round half empty).  A segment costs about two and a half tiles besides its tiles (its state goes to memory
+// and back, the pipeline fills), at most 16 tiles long and at least 2 on average.  L is the power-of-two length the
+// fixed rule picks, kept unless the estimate improves on it by a few percent.
+void smat_segment_counts(int64_t tiles0, int64_t tiles1, int bh, int L, int* nseg0, int* nseg1) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const double overhead = 2.5;
+  auto cost = [&](int64_t n0, int64_t n1) {
+    const int64_t l0 = (tiles0 + n0 - 1) / n0, l1 = n1 ? (tiles1 + n1 - 1) / n1 : 0;
+    const int64_t lmax = l0 > l1 ? l0 : l1;
+    const int64_t rounds = ((n0 + n1) * bh + sms - 1) / sms;
+    return (double)rounds * ((double)lmax + overhead);
+  };
+  int64_t best0 = tiles0 / L, best1 = tiles1 / L;
+  double best = cost(best0, best1) * 0.96;
+  const int64_t max0 = tiles0 / 2 > 0 ? tiles0 / 2 : 1, max1 = tiles1 / 2;
+  for (int64_t n0 = 1; n0 <= max0 && n0 <= 512; ++n0) {
+    if ((tiles0 + n0 - 1) / n0 > 16) continue;
+    // block 1 gets the count that gives it the same longest segment, or one more segment
+    const int64_t l0 = (tiles0 + n0 - 1) / n0;
+    for (int64_t n1 = tiles1 ? (tiles1 + l0 - 1) / l0 : 0, k = 0; k < 2; ++k, ++n1) {
+      if (tiles1 && (n1 < 1 || n1 > max1 || (tiles1 + n1 - 1) / n1 > 16)) continue;
+      if (!tiles1 && k) break;
+      const double c = cost(n0, n1);
+      if (c < best) { best = c; best0 = n0; best1 = n1; }
+    }
+  }
+  *nseg0 = (int)best0; *nseg1 = (int)best1;
+}
+
+cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* totals, int64_t tiles0, int64_t tiles1,
+                                         int nseg0, int nseg1, int bh, int* status, cudaStream_t st) {
+  const int64_t T = (tiles0 + tiles1) * TILE;
   CUtensorMap tmK, tmV;
   if (!make_map(&tmK, K, (uint64_t)bh * T) || !make_map(&tmV, V, (uint64_t)bh * T)) return cudaErrorInvalidValue;
   SegStateParams prm;
-  prm.T = T; prm.L = L; prm.nseg = (int)(T / TILE / L); prm.totals = totals; prm.status = status;
+  prm.T = T; prm.nseg = nseg0 + nseg1; prm.totals = totals; prm.status = status;
+  prm.cut.nseg0 = nseg0; prm.cut.nseg = nseg0 + nseg1; prm.cut.tiles0 = tiles0; prm.cut.tiles1 = tiles1;
   cudaError_t err =
       cudaFuncSetAttribute(segment_state_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_STATE_SMEM);
   if (err != cudaSuccess) return err;
@@ -1233,14 +1294,16 @@ cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* to
 }
 
 cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const void* V, const float* seg_in,
-                                          const void* ylr_bf16, int64_t n_lr, void* O, int64_t T, int L, int bh,
-                                          int* status, cudaStream_t st) {
+                                          const void* ylr_bf16, int64_t n_lr, void* O, int64_t tiles0, int64_t tiles1,
+                                          int nseg0, int nseg1, int bh, int* status, cudaStream_t st) {
+  const int64_t T = (tiles0 + tiles1) * TILE;
   CUtensorMap tmQ, tmK, tmV;
   if (!make_map(&tmQ, Q, (uint64_t)bh * T) || !make_map(&tmK, K, (uint64_t)bh * T) ||
       !make_map(&tmV, V, (uint64_t)bh * T))
     return cudaErrorInvalidValue;
   SegOutParams prm;
-  prm.T = T; prm.L = L; prm.nseg = (int)(T / TILE / L); prm.seg_in = seg_in; prm.n_lr = n_lr; prm.ylr = static_cast<const __nv_bfloat16*>(ylr_bf16);
+  prm.T = T; prm.nseg = nseg0 + nseg1; prm.seg_in = seg_in; prm.n_lr = n_lr; prm.ylr = static_cast<const __nv_bfloat16*>(ylr_bf16);
+  prm.cut.nseg0 = nseg0; prm.cut.nseg = nseg0 + nseg1; prm.cut.tiles0 = tiles0; prm.cut.tiles1 = tiles1;
   prm.O = static_cast<__nv_bfloat16*>(O);
   prm.status = status;
   cudaError_t err =
