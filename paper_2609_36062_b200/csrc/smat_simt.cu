@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(256) gemm_grouped_kernel(const SmatGemmArgs a)
 
 // ---- scan --------------------------------------------------------------------------------------
 // Each thread owns four consecutive state entries and walks the chunks of its range in order.
-// Loads are issued eight chunks ahead of the dependent additions.
+// Loads are issued sixteen chunks ahead of the dependent additions.
 __global__ void __launch_bounds__(256) scan_kernel(float* S, int64_t state_elems, int64_t NC, int64_t lo0, int64_t hi0,
                                                    int64_t lo1, int64_t hi1, int reverse) {
   const int64_t e4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -122,7 +122,7 @@ __global__ void __launch_bounds__(256) scan_kernel(float* S, int64_t state_elems
   float4* base = reinterpret_cast<float4*>(S + bh * NC * state_elems) + e4;
   const int64_t stride4 = state_elems / 4;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  constexpr int AHEAD = 8;
+  constexpr int AHEAD = 16;
   for (int64_t s = 0; s < hi - lo; s += AHEAD) {
     float4 v[AHEAD];
 #pragma unroll
