@@ -395,6 +395,8 @@ __global__ void __launch_bounds__(192) segment_state_tc_kernel(const __grid_cons
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int seg = blockIdx.x, bh = blockIdx.y;
+  // The scan is exclusive: nobody reads the total of a block's last segment (the scan loads it after its last store).
+  if (seg == prm.cut.nseg0 - 1 || seg == prm.cut.nseg - 1) return;
   int64_t tile0;
   int Lc;
   seg_range(prm.cut, seg, &tile0, &Lc);
