@@ -43,8 +43,6 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
-#include <cstdlib>
-
 #include "smat_internal.h"
 #include "smat_tc.cuh"
 
@@ -95,7 +93,9 @@ struct RadonParams {
                                    // last part, straight from the ring slot; 0: every index goes through the MMAs
   int32_t ring;                    // ring slots
   int32_t tma_out;                 // the output tile leaves through the item's own ring slot and TMA stores (q = 11)
-  int32_t mini_bytes;              // tma_out: per slot, room for the extra-class rows of the tile (two halves)
+  int32_t mini_bytes;              // tma_out: per slot, room for the extra-class rows of the tile (two halves); 0: the
+                                   // extra-class rows of a part sit in the tile itself, after its regular lines
+  int32_t lines_pp;                // tma_out: regular lines per tile (the store box; lines past q - 1 are clipped)
   int32_t nph;                     // 1, or 2: both stages of the d = 4 tabulation, slab by slab
   int32_t slabs_per_head;          // rp / 128
   int64_t slabs;                   // heads * slabs_per_head
@@ -317,7 +317,8 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   uint64_t* acc_full = empty + prm.ring;    // [MAX_ACC] accumulator complete
   uint64_t* acc_empty = acc_full + MAX_ACC; // [MAX_ACC] accumulator read out (one arrival per epilogue warp)
   uint64_t* w_ready = acc_empty + MAX_ACC;  // phase 0 of the current slab written out (one arrival per storing warp)
-  uint64_t* staged = w_ready + 1;           // [ring] tma_out: the item's tile is complete in its slot (one arrival per epilogue warp)
+  uint64_t* staged = w_ready + 1;           // [ring] tma_out: an item's tile is complete in its first slot (one arrival per
+                                            // epilogue warp); indexed by the item count modulo the ring size
   uint64_t* alu_done = staged + prm.ring;   // [ring] tma_out: the ALU warps have read the slot and written their rows
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(alu_done + prm.ring);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -325,7 +326,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   const WaitCtx wc{cta_abort, prm.status};
   const int part = blockIdx.x % prm.parts;
   const bool alu_here = FEAT && prm.alu_rows > 0 && part == prm.parts - 1;
-  const bool tma_out = FEAT && prm.tma_out != 0;
+  const bool tma_out = prm.tma_out != 0;
   const uint32_t nph = FEAT ? (uint32_t)prm.nph : 1u;
 
   if (threadIdx.x == 0) {
@@ -390,6 +391,64 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
   const uint32_t first = blockIdx.x / prm.parts, step = gridDim.x / prm.parts;
   const uint32_t sph = (uint32_t)prm.slabs_per_head;
 
+  // ---- storing thread (tma_out): one bulk group of tile stores per item; the item's first slot, which holds the tile,
+  // goes back to the producer when the stores have read it.  Lane 0 of the second MMA warp when every item is one
+  // slot (that warp has no items then), else lane 0 of warp 19.
+  auto store_role = [&]() {
+    const uint32_t ring = (uint32_t)prm.ring;
+    uint32_t slot = 0, prev_slot = 0;
+    uint32_t sidx = 0, spar = 0;                                // the item's "staged" barrier (items mod ring) and its parity
+    bool have_prev = false;
+    const int hi0 = part * prm.lines_pp;                        // first regular line of this CTA's tiles
+    const int xrow0 = q * q - part * prm.rows_pp;               // tile row of the first extra-class index
+    for (ItemIter it(prm, first, step, nph); it.left; it.next()) {
+      const RadonPhase& ph = FEAT ? prm.ph[it.ph] : prm.ph[0];
+      const CUtensorMap* oreg = FEAT && it.ph ? &tm_oreg1 : &tm_oreg0;
+      const CUtensorMap* overt = FEAT && it.ph ? &tm_overt1 : &tm_overt0;
+      const uint32_t head = it.slab / sph;
+      const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
+      const int hc = ph.dst_private ? (int)blockIdx.x : (int)head;
+      const uint64_t pol = it.ph ? pol_dst1 : pol_dst0;
+      if (!mbar_wait(staged + sidx, spar, wc)) break;
+      if (++sidx == ring) { sidx = 0; spar ^= 1; }
+      const uint8_t* tile = sRing + slot * slot_bytes;
+      if (hi0 < q) {
+        tma_store_5d(oreg, tile, e0, 0, hi0, (int)it.img, hc, pol);
+        tma_store_5d(oreg, tile + prm.sr * 128, e0 + 64, 0, hi0, (int)it.img, hc, pol);
+      }
+      if (ph.out.count > q * q && xrow0 < prm.rows_pp && (int)it.img >= ph.out.vert_from) {
+        const int ci = ph.out.sv_img != 0 ? (int)it.img : 0;   // the map's image stride is sv_img rows
+        if (prm.mini_bytes) {
+          const uint8_t* mini = sMini + slot * prm.mini_bytes;
+          tma_store_4d(overt, mini, e0, 0, ci, hc, pol);
+          tma_store_4d(overt, mini + prm.mini_bytes / 2, e0 + 64, 0, ci, hc, pol);
+        } else {
+          tma_store_4d(overt, tile + xrow0 * 128, e0, 0, ci, hc, pol);
+          tma_store_4d(overt, tile + prm.sr * 128 + xrow0 * 128, e0 + 64, 0, ci, hc, pol);
+        }
+      }
+      bulk_commit();
+      if (have_prev) {
+        bulk_wait_read<1>();
+        mbar_arrive(empty + prev_slot);
+      }
+      if (it.closes_phase0()) {   // the slab's stage-1 rows are in memory before the producer loads them back
+        bulk_wait_all();
+        fence_proxy_async_all();
+        mbar_arrive(empty + slot);
+        mbar_arrive(w_ready);
+        have_prev = false;
+      } else {
+        prev_slot = slot;
+        have_prev = true;
+      }
+      slot += (uint32_t)prm.nslots;
+      if (slot >= ring) slot -= ring;
+    }
+    if (have_prev) { bulk_wait_read<0>(); mbar_arrive(empty + prev_slot); }
+    bulk_wait_all();
+  };
+
   if (warp == PROD_WARP && lane == 0) {
     // ---- TMA producer -----------------------------------------------------------------------------------------
     // The two single-thread roles keep running slot / parity counters: a lone thread pays the full latency of every
@@ -448,49 +507,7 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     // MMAs, commits: more than the tensor pipe needs for it) overlaps with the other thread's item.  Both phases
     // share R and the slot layout, so the issuers only count items. ---------------------------------------------
     const uint32_t me = (uint32_t)(warp - MMA_WARP);
-    if (tma_out && me == 1) {
-      // ---- storing thread (the second issuing thread has no items when every item is one slot): one bulk group
-      // of tile stores per item; a slot goes back to the producer when the stores of its item have read it --------
-      const uint32_t ring = (uint32_t)prm.ring;
-      uint32_t slot = 0, par = 0, prev_slot = 0;
-      bool have_prev = false;
-      for (ItemIter it(prm, first, step, nph); it.left; it.next()) {
-        const RadonPhase& ph = FEAT ? prm.ph[it.ph] : prm.ph[0];
-        const CUtensorMap* oreg = it.ph ? &tm_oreg1 : &tm_oreg0;
-        const CUtensorMap* overt = it.ph ? &tm_overt1 : &tm_overt0;
-        const uint32_t head = it.slab / sph;
-        const int e0 = ph.dst_private ? 0 : (int)(it.slab - head * sph) * 128;
-        const int hc = ph.dst_private ? (int)blockIdx.x : (int)head;
-        const uint64_t pol = it.ph ? pol_dst1 : pol_dst0;
-        if (!mbar_wait(staged + slot, par, wc)) break;
-        const uint8_t* tile = sRing + slot * slot_bytes;
-        tma_store_5d(oreg, tile, e0, 0, 0, (int)it.img, hc, pol);
-        tma_store_5d(oreg, tile + prm.sr * 128, e0 + 64, 0, 0, (int)it.img, hc, pol);
-        if (ph.out.count > q * q && (int)it.img >= ph.out.vert_from) {
-          const uint8_t* mini = sMini + slot * prm.mini_bytes;
-          const int ci = ph.out.sv_img != 0 ? (int)it.img : 0;   // the map's image stride is sv_img rows
-          tma_store_4d(overt, mini, e0, 0, ci, hc, pol);
-          tma_store_4d(overt, mini + prm.mini_bytes / 2, e0 + 64, 0, ci, hc, pol);
-        }
-        bulk_commit();
-        if (have_prev) {
-          bulk_wait_read<1>();
-          mbar_arrive(empty + prev_slot);
-        }
-        if (it.closes_phase0()) {   // the slab's stage-1 rows are in memory before the producer loads them back
-          bulk_wait_all();
-          fence_proxy_async_all();
-          mbar_arrive(empty + slot);
-          mbar_arrive(w_ready);
-          have_prev = false;
-        } else {
-          prev_slot = slot;
-          have_prev = true;
-        }
-        if (++slot == ring) { slot = 0; par ^= 1; }
-      }
-      bulk_wait_all();
-    }
+    if (tma_out && me == 1 && prm.nslots == 1) store_role();
     constexpr uint32_t idesc = make_idesc(TILE_ROWS, 128, 0, 1);   // A from tensor memory (R), B MN-major (image rows)
     const uint64_t dB0 = make_desc(smem_u32(sRing), prm.sr * 128, 1024);
     const uint32_t slot16 = (uint32_t)slot_bytes >> 4;            // descriptor address units are 16 bytes
@@ -547,6 +564,8 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
         if (++buf == nacc) { buf = 0; if (n_item >= nacc) apar ^= 1; }
       }
     }
+  } else if (tma_out && prm.nslots > 1 && warp == ALU_WARP) {
+    if (lane == 0) store_role();
   } else if (FEAT && warp >= ALU_WARP) {
     // ---- leftover rows on the ALUs ----------------------------------------------------------------------------
     // q*q + q output indices rarely fill whole tiles of 128.  When only a few are left over, and they belong to the
@@ -618,7 +637,11 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
     const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
     const int tv0 = out_tab[orow], tv1 = nph > 1 ? out_tab[TILE_ROWS + orow] : ROW_INVALID;
     const bool active = qd * 32 < prm.rows_pp;                  // warp-uniform: some output index in these lanes
-    uint32_t buf = 0, apar = 0, eslot = 0, epar = 0;
+    uint32_t buf = 0, apar = 0, eslot = 0, epar = 0, sidx = 0;
+    // tma_out: where this thread's 64 bytes go inside the slot (or inside the slot's extra rows)
+    const bool st_mini = prm.mini_bytes != 0 && part * prm.rows_pp + orow >= q * q;
+    const int st_idx = st_mini ? part * prm.rows_pp + orow - q * q : orow;
+    const int st_off = (cb >> 1) * (st_mini ? prm.mini_bytes / 2 : prm.sr * 128) + st_idx * 128;
     for (ItemIter it(prm, first, step, nph); it.left; it.next()) {
       const RadonPhase& ph = FEAT ? prm.ph[it.ph] : prm.ph[0];
       const uint32_t head = it.slab / sph;
@@ -639,10 +662,19 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
         __syncwarp();
         if (lane == 0) mbar_arrive(acc_empty + buf);             // the accumulator is in registers
         if (alu_here && !mbar_wait_warp(alu_done + eslot, epar, wc)) break;   // the ALU warps have read the image
+        if (prm.nslots > 1) {                                     // the item's other slots are free already
+          if (warp == 0 && lane == 0)
+            for (int g = 1; g < prm.nslots; ++g) {
+              uint32_t sl = eslot + g; if (sl >= (uint32_t)prm.ring) sl -= (uint32_t)prm.ring;
+              mbar_arrive(empty + sl);
+            }
+          __syncwarp();
+        }
         if (tv != ROW_INVALID) {
-          const int idx = orow < q * q ? orow : orow - q * q;     // row of the tile / of the extra rows
-          uint8_t* trow = (orow < q * q ? sRing + eslot * slot_bytes + (cb >> 1) * prm.sr * 128
-                                        : sMini + eslot * prm.mini_bytes + (cb >> 1) * (prm.mini_bytes / 2)) + idx * 128;
+          // regular indices and, without extra rows of their own, the extra-class indices of the part: tile row =
+          // TMEM lane; with extra rows per slot (q = 11) the extra-class indices go there
+          const int idx = st_idx;
+          uint8_t* trow = (st_mini ? sMini + eslot * prm.mini_bytes : sRing + eslot * slot_bytes) + st_off;
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             *reinterpret_cast<uint4*>(trow + ((((cb & 1) * 4 + j) ^ (idx & 7)) << 4)) =
@@ -653,8 +685,10 @@ __global__ void __launch_bounds__(RADON_THREADS, 1) radon_tc_kernel(const __grid
         }
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(staged + eslot);
-        if (++eslot == (uint32_t)prm.ring) { eslot = 0; epar ^= 1; }
+        if (lane == 0) mbar_arrive(staged + sidx);   // one barrier per item in flight: at most `ring` of them
+        if (++sidx == (uint32_t)prm.ring) sidx = 0;
+        eslot += (uint32_t)prm.nslots;
+        if (eslot >= (uint32_t)prm.ring) { eslot -= (uint32_t)prm.ring; epar ^= 1; }
         if (++buf == nacc) { buf = 0; apar ^= 1; }
         continue;
       }
@@ -741,6 +775,10 @@ bool radon_shape(int q, int transpose, int in_has_extra, int count_out, RadonSha
     }
   }
   if (best == (1 << 30)) return false;
+  {   // whole lines per part where they fit: a part's tile can then leave as one box of lines
+    const int lines = count_out / q, lpp = (lines + s->parts - 1) / s->parts;
+    if (count_out % q == 0 && lpp * q <= TILE_ROWS) s->rows_pp = lpp * q;
+  }
   // A few indices past the last full tile, all of the extra class, with every line in one slot: full tiles for the
   // MMAs and the rest on the ALUs (q = 11: 132 = 128 + 4 indices, one CTA per image instead of two).
   const int left = count_out % TILE_ROWS, whole = count_out - left;
@@ -832,7 +870,10 @@ cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int
   // from the item's own slot; every slot gets room for the q extra-class rows of its tile (two 64-entry halves).
   int smem = sh.smem;
   prm.tma_out = 0; prm.mini_bytes = 0;
-  if (!transpose && sh.nslots == 1 && sh.sr == TILE_ROWS && sh.parts == 1 && !getenv("SMAT_NO_TMA_OUT")) {
+  prm.lines_pp = sh.rows_pp / q < q ? sh.rows_pp / q : q;
+  // (Tiles of whole lines could leave the same way for q = 13, 17 — the kernel handles several slots per item and
+  // several parts — but there the tile stores were measured 1.6 to 2 times slower than the direct stores.)
+  if (!transpose && sh.nslots == 1 && sh.sr == TILE_ROWS && sh.parts == 1) {
     const int mini = 2 * ((q + 7) & ~7) * 128, slot = sh.sr * 256;
     int ring = (227 * 1024 - 1024 - 512 - TILE_ROWS * 8) / (slot + mini);
     if (ring > sh.ring) ring = sh.ring;
@@ -882,7 +923,7 @@ cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int
       const int64_t dst_rp = sp[i].dst_private ? 128 : rp, dst_heads = sp[i].dst_private ? ctas : bh;
       const int64_t sizes[4] = {q, q, images, dst_heads};
       const int64_t strides[4] = {out.s_lo, out.s_hi, images > 1 ? out.s_img : out.rows_per_head, out.rows_per_head};
-      const int box[4] = {q, q, 1, 1};
+      const int box[4] = {q, prm.lines_pp, 1, 1};
       if (!radon_map(&tm_oreg[i], sp[i].dst, dst_rp, 5, sizes, strides, box)) return cudaErrorInvalidValue;
       if (out.count > q * q) {
         const bool per_image = out.sv_img != 0;
@@ -898,12 +939,12 @@ cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int
   if (nph == 1) {
     prm.ph[1] = prm.ph[0]; tm_reg[1] = tm_reg[0]; tm_vert[1] = tm_vert[0]; tm_oreg[1] = tm_oreg[0]; tm_overt[1] = tm_overt[0];
   }
-  const bool feat = nph > 1 || prm.alu_rows > 0 || prm.tma_out;
+  const bool feat = nph > 1 || prm.alu_rows > 0;
   auto kernel = feat ? radon_tc_kernel<true> : radon_tc_kernel<false>;
   cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (err != cudaSuccess) return err;
   // the plain instantiation has no use for the two ALU warps
-  kernel<<<(unsigned)ctas, feat ? RADON_THREADS : 32 * ALU_WARP, smem, st>>>(tm_reg[0], tm_vert[0], tm_reg[1], tm_vert[1],
+  kernel<<<(unsigned)ctas, feat ? RADON_THREADS : 32 * (ALU_WARP + (prm.tma_out ? 1 : 0)), smem, st>>>(tm_reg[0], tm_vert[0], tm_reg[1], tm_vert[1],
                                                                             tm_oreg[0], tm_overt[0], tm_oreg[1], tm_overt[1], prm);
   return cudaGetLastError();
 }
