@@ -37,9 +37,9 @@ SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
 METRIC = "SMat prefill tokens/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant stage per step — the tabulation, one
 # launch of radon_tc_kernel — from the ncu capture summarised in profiles/radon_tc_kernel_t16k_d4_h8.md: taken on the
-# 8-head copy of the workload (351.4 MB read + 530.2 MB written) and scaled by heads (every head owns its tables; the
+# 8-head copy of the workload (351.3 MB read + 530.1 MB written) and scaled by heads (every head owns its tables; the
 # per-CTA exchange buffer, the only shared footprint, is the same 55 MB at 8 and at 32 heads).
-NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate_tc"): 881.6e6 * 4}
+NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate_tc"): 881.4e6 * 4}
 
 
 def parse_args():
