@@ -16,8 +16,8 @@
 // traffic.
 //
 // radon_tc_kernel, persistent, one CTA per SM.  An item is one image restricted to 128 consecutive state entries;
-// a CTA owns up to 128 output indices (its part of R; the output indices are split evenly over `parts` CTAs that
-// then share every image) and applies them to every item it is given:
+// a CTA owns up to 128 output indices (its part of R; the output indices are split over `parts` CTAs, in whole
+// lines where these fit, that then share every image) and applies them to every item it is given:
 //   warps 0-3      : build the CTA's part of R once and move it to tensor memory (lane = output index, one column
 //                    per two operand rows), where the MMAs read it as their A operand
 //   warp 16 lane 0 : TMA producer; a ring slot holds `sps` lines (fixed hi, all lo) of the image x 128 state entries
@@ -37,8 +37,10 @@
 // q = 11 also sends its output tiles off by TMA: the epilogue writes the rounded tile into the item's own ring slot
 // (as large as a tile, and dead once the MMAs have read it) in the box layout, and lane 0 of warp 18 issues the tile
 // stores and frees the slot; the bulk of the stores bypasses the LSU.
-// The kernel exists twice: radon_tc_kernel<false> without any of the prime-specific paths (q = 13, 17, 19 and
-// everything with one stage per launch and no leftover rows), radon_tc_kernel<true> with them.
+// The kernel exists twice: radon_tc_kernel<false> for one stage per launch with every index through the MMAs (q = 13,
+// 17, 19 and the small primes), without cache hints, phase tables or ALU warps; radon_tc_kernel<true> with them.
+// (The tile-store path is written for several slots per item and several parts and is compiled into both, but the
+// launcher switches it on for q = 11 only: it was measured slower than the direct stores for q = 13 and 17.)
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
