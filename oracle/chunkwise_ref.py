@@ -1,8 +1,8 @@
 """Chunkwise fp64 CPU restatement of the SMat forward and backward algorithms.  TEST INFRASTRUCTURE ONLY.
 
-This is NOT the oracle (that is smat_oracle.py, the dense definition).  It takes the
-steps of Algorithm 1 (forward), Algorithm 2 (implicit incidence tabulation) and the
-adjoint equations of the chunking proof in the paper's order and notation, in float64,
+This is NOT the oracle (that is smat_oracle.py, the dense definition).  It evaluates the
+quantities of Algorithm 1 (forward), Algorithm 2 (implicit incidence tabulation) and the
+adjoint equations of the chunking proof with the paper's notation, in float64,
 one head at a time.  It is checked against the dense oracle in the CPU tests and then
 serves two purposes: an independent formula for the same numbers, and a way to look
 at the intermediate tables (F, U, D, S_in and their adjoints) when a GPU kernel is wrong.
@@ -31,31 +31,35 @@ def _chunks(geo):
     return out
 
 
+def _point_digits(geo):
+    """All points of F_q^D as an integer array [P, D]; row v holds the little-endian base-q digits of v."""
+    v = np.arange(geo.P, dtype=np.int64)
+    return np.stack([(v // geo.q ** ell) % geo.q for ell in range(geo.D)], axis=1)
+
+
 def tabulate(F, geo):
-    """Algorithm 2: U_{a,b} = Σ_{x : aᵀx = b} F_x, one state addition per nonzero of C."""
+    """Algorithm 2: U_{a,b} = Σ_{x : aᵀx = b} F_x.  For one direction a the offsets aᵀx split the points into q
+    classes; every class is summed into the state of its hyperplane."""
     if geo.dense_G:
-        return F.copy()                                   # line 1: U_0 <- F_0
+        return F.copy()                                   # one point, one hyperplane
     U = np.zeros((geo.B,) + F.shape[1:], dtype=np.float64)
-    dirs = so.directions(geo.q, geo.D)
-    for ai, a in enumerate(dirs):
-        for v in range(geo.P):
-            x = so.prof(v, geo)
-            b = sum(al * xl for al, xl in zip(a, x)) % geo.q      # finite-field arithmetic
-            U[ai * geo.q + b] += F[v]                             # ordinary state addition
+    pts = _point_digits(geo)
+    for ai, a in enumerate(so.directions(geo.q, geo.D)):
+        offset = (pts @ np.asarray(a, dtype=np.int64)) % geo.q
+        for b in range(geo.q):
+            U[ai * geo.q + b] = F[offset == b].sum(axis=0)
     return U
 
 
 def tabulate_transpose(Ubar, geo):
-    """F̄ = Cᵀ Ū: every point lies on one hyperplane per direction (Eq. lr-adjoint)."""
+    """F̄ = Cᵀ Ū: a point receives, from every direction, the state of the one hyperplane through it (Eq. lr-adjoint)."""
     if geo.dense_G:
         return Ubar.copy()
     Fbar = np.zeros((geo.P,) + Ubar.shape[1:], dtype=np.float64)
-    dirs = so.directions(geo.q, geo.D)
-    for v in range(geo.P):
-        x = so.prof(v, geo)
-        for ai, a in enumerate(dirs):
-            b = sum(al * xl for al, xl in zip(a, x)) % geo.q
-            Fbar[v] += Ubar[ai * geo.q + b]
+    pts = _point_digits(geo)
+    for ai, a in enumerate(so.directions(geo.q, geo.D)):
+        offset = (pts @ np.asarray(a, dtype=np.int64)) % geo.q
+        Fbar += Ubar[ai * geo.q + offset]
     return Fbar
 
 
@@ -68,31 +72,32 @@ def _profile(t, geo):
 
 
 def forward(Q, K, V, geo, return_tables=False):
-    """Algorithm 1, steps 1-7, without the final division."""
+    """Algorithm 1 without the final division: pooled profile states, tabulated type states, typed read, chunk
+    summaries and their exclusive scan per block, per-chunk output."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     T, r = Q.shape
     p = V.shape[1]
     n = geo.n
-    # step 2: pool the distant states by profile
+    # profile table: distant states pooled by profile cell (Eq. schedule)
     F = np.zeros((geo.P, r, p))
     for t in range(n):
         F[_profile(t, geo)] += np.outer(K[t], V[t])
-    # step 3: tabulate
+    # type table
     U = tabulate(F, geo)
-    # step 4: typed read, rows scattered back in chronological order
+    # typed read, rows back in chronological order
     Ylr = np.zeros((T, p))
     for t in range(n, T):
         Ylr[t] = Q[t] @ U[_type(t, geo)]
-    # step 5: chunk summaries;  step 6: exclusive scan inside each block
+    # chunk summaries and their exclusive scan inside each block (the state restarts at n)
     ch = _chunks(geo)
     Dsum = np.stack([K[s:e].T @ V[s:e] for s, e, _ in ch]) if ch else np.zeros((0, r, p))
     Sin = np.zeros_like(Dsum)
     for b, (s, e, lo) in enumerate(ch):
         if s != lo:
             Sin[b] = Sin[b - 1] + Dsum[b - 1]
-    # step 7: per-chunk output
+    # per-chunk output (Eq. local plus the long-range rows)
     O = np.zeros((T, p))
     for b, (s, e, lo) in enumerate(ch):
         A = np.tril(Q[s:e] @ K[s:e].T)

@@ -17,7 +17,7 @@ What follows which passage of the paper
 * output without feature map / normaliser: O = (M ⊙ QKᵀ)V   -> Eq. (augmented-attention-output)
   with φ = ψ = identity and the division left out
 
-Readings taken where the paper is silent (all listed in the design notes):
+Readings taken where the paper is silent:
   R1  q = smallest prime with q^d >= n   (the paper only says q = Θ(n^{1/d}); this rule
       reproduces the decode-cache sizes printed in the end-to-end cost table)
   R2  prof digits are little-endian: x_1 is the least significant base-q digit of t mod q^{d-1}

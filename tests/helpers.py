@@ -36,10 +36,17 @@ def rel_err(got: np.ndarray, ref: np.ndarray) -> float:
 
 def sample_tokens(geo, count: int, seed: int) -> list[int]:
     """Token indices that always include both ends, both sides of the block boundary and of chunk
-    edges, and one query of each of the first types; the rest are drawn at random."""
+    edges, and one query of each of the first 64 types (types 0..63, each at a different one of its
+    occurrences so that the samples spread over the recent block); the rest are drawn at random."""
     T, n, c = geo.T, geo.n, geo.c
     fixed = {0, 1, c - 1, c, n - 1, n, n + 1, n + c - 1, n + c, T - 1, T - c, T - c - 1, n // 2, n + (T - n) // 2}
-    fixed |= {n + i for i in range(min(16, T - n))}
+    B, m = geo.B, T - n
+    for h in range(min(64, B)):
+        first = h if h >= 1 else B                   # 1-based recent index of the type's first query
+        if first > m:
+            continue
+        occurrences = (m - first) // B + 1
+        fixed.add(n + first - 1 + (h % occurrences) * B)
     fixed = {t for t in fixed if 0 <= t < T}
     g = np.random.default_rng(seed)
     extra = g.choice(T, size=max(0, count - len(fixed)), replace=False).tolist() if count > len(fixed) else []

@@ -154,3 +154,36 @@ def test_witness_set_is_shattered_on_every_workload(name):
 
 def d_of(geo):
     return geo.d
+
+
+# ---- set_is_shattered itself: cases where the answer must be False ------------------------------------
+def test_shattering_check_rejects_sets_that_are_not_shattered():
+    # a hand-made set system: three columns, rows realise 7 of the 8 patterns
+    rows = [r for r in itertools.product([0, 1], repeat=3) if r != (1, 0, 1)]
+    table = np.array(rows, dtype=np.uint8)
+    assert not so.set_is_shattered(lambda t: table[t], [0, 1, 2], range(len(rows)))
+    assert so.set_is_shattered(lambda t: table[t], [0, 1], range(len(rows)))
+    full = np.array(list(itertools.product([0, 1], repeat=3)), dtype=np.uint8)
+    assert so.set_is_shattered(lambda t: full[t], [0, 1, 2], range(8))
+    assert not so.set_is_shattered(lambda t: full[t], [0, 1, 2], range(7))      # one pattern's row withheld
+
+
+@pytest.mark.parametrize("T,c,d,q", [(256, 4, 3, 5), (512, 64, 2, None), (1024, 16, 4, 3)])
+def test_witness_set_needs_both_sides_of_tau_and_cannot_grow(T, c, d, q):
+    """Lower-bound proof of Theorem 1: the last witness column n+τ separates recent rows before τ from rows after it.
+    With only the first B recent rows (every type once, all before τ = B+1) that column is never set, so the witness
+    set is NOT shattered; with 2B rows it is; and no set of d+1 columns is shattered by any rows (VC = d)."""
+    geo = so.geometry(T, c, d, q)
+    assert geo.conditions_met
+    D, n, B = geo.D, geo.n, geo.B
+    cols = [geo.q ** ell for ell in range(D)] + [n + B]
+    row = lambda t: so.mask_row(t, geo)
+    assert so.set_is_shattered(row, cols, range(n, n + 2 * B))
+    assert not so.set_is_shattered(row, cols, range(n, n + B))          # no row lies on the far side of τ
+    assert not so.set_is_shattered(row, cols, range(n + B, n + 2 * B))  # ... nor any on the near side
+    assert so.set_is_shattered(row, cols[:-1], range(n, n + B))         # the D profile columns alone need one side
+    # d+1 columns: the witness set plus any further column is not shattered by the whole mask (upper bound VC <= d)
+    for extra in (0, geo.q + 1, n - 1, n, n + 2 * B - 1, T - 1):
+        if extra in cols:
+            continue
+        assert not so.set_is_shattered(row, cols + [extra], range(T)), extra
