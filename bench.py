@@ -36,9 +36,9 @@ DEFAULT_WORKLOAD = "t16k_d4"
 SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
 METRIC = "SMat prefill tokens/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant stage per step — the tabulation, one
-# launch of radon_tc_kernel — from the ncu capture summarised in profiles/radon_tc_kernel_t16k_d4_h8.md: taken on the
-# 8-head copy of the workload (351.3 MB read + 530.1 MB written) and scaled by heads (every head owns its tables; the
-# per-CTA exchange buffer, the only shared footprint, is the same 55 MB at 8 and at 32 heads).
+# launch of radon_tc_kernel — from an ncu capture of the 8-head copy of the workload (351.3 MB read + 530.1 MB
+# written), scaled by heads (every head owns its tables; the per-CTA exchange buffer, the only shared footprint,
+# is the same 55 MB at 8 and at 32 heads).
 NCU_TRAFFIC_BYTES = {("t16k_d4", "tabulate_tc"): 881.4e6 * 4}
 
 
@@ -304,6 +304,32 @@ class Runner:
             barrier()
         return start.elapsed_time(end) / 1e3   # seconds for `steps` steps
 
+    def time_each(self, fn, steps, warmup):
+        """Per-step durations (seconds) from one CUDA event pair per step, after `warmup` untimed steps."""
+        torch = self.torch
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        evs[0].record()
+        for i in range(steps):
+            fn()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        return [evs[i].elapsed_time(evs[i + 1]) / 1e3 for i in range(steps)]
+
+    def time_sustained(self, fn, seconds_per_step, index, min_seconds=1.2):
+        """The same step back to back for at least `min_seconds` (long enough for the board power limit to act),
+        with the clocks sampled during the region."""
+        torch = self.torch
+        steps = max(20, int(min_seconds / max(seconds_per_step, 1e-6)) + 1)
+        sampler = ClockSampler(index)
+        sampler.start()
+        sampler.wait_ready()
+        total = self.time_steps(fn, steps, 3)
+        clocks = sampler.stop()
+        return {"steps": steps, "seconds": total, "ms_per_step": 1e3 * total / steps, "clocks": clocks}
+
     def stage_profile(self, steps):
         """Average per-kernel durations (ms) over `steps` steps, CUDA events on the launching stream."""
         self.plan.profile_enable(True)
@@ -314,7 +340,7 @@ class Runner:
             recs = self.plan.profile_read()
             if self.w.backward:
                 self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws)
-                recs += [("bwd:" + n if not n.startswith("bwd_") else n, t) for n, t in self.plan.profile_read()]
+                recs += [(n if n.startswith("bwd_") else "bwd_" + n, t) for n, t in self.plan.profile_read()]
             for n, t in recs:
                 if n not in acc:
                     acc[n] = 0.0; order.append(n)
@@ -345,6 +371,7 @@ def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4):
         "profile_table_bytes_per_entry": f_bytes,
         "roofline_ms_2term": 1e3 * t["t_2term"], "roofline_ms_3term": 1e3 * t["t_3term"],
         "t_tensor_ms": 1e3 * t["t_tensor"], "t_alu_ms": 1e3 * t["t_alu"], "t_hbm_ms": 1e3 * t["t_hbm"],
+        "alu_peak_adds_per_s": t["alu_peak_adds"], "alu_peak_source": t["alu_peak_source"],
         "algorithmic": {"tensor_flop": work.flops, "alu_adds": work.adds, "hbm_bytes": work.bytes},
         "peaks": peaks["source"],
     }
@@ -356,7 +383,7 @@ def dominant_kernel_report(w, geo, stages, peaks, u_bytes=4, f_bytes=4):
     e = 4 if w.dtype == "f32" else 2
     total = sum(t for _, t in stages)
     name, ms = max(stages, key=lambda s: s[1])
-    base = name.split(":")[-1]
+    base = name
     work = roofline.stage_work(base, w.T, w.chunk, w.d_k, w.d_v, e, geo, u_bytes, f_bytes).scaled(w.bh)
     t = roofline.roofline_times(work, peaks, sustained=True)
     ops = work.flops + work.adds
@@ -425,6 +452,10 @@ def run_native(args):
         barrier = dist.barrier
 
     peaks = roofline.load_peaks(ROOT)
+    if rank == 0:   # fp32 add rate of the plain ALUs, measured here (scalar and two-lane adds; the faster one counts)
+        rates = {"scalar": binding.measure_fadd_rate(False), "packed": binding.measure_fadd_rate(True)}
+        peaks["fadd_adds_per_s"] = max(rates.values())
+        peaks["fadd_rates"] = rates
     if args.decode_only:
         if rank == 0:
             name = args.workload if args.workload.startswith("decode") else "decode_t2k_d3"
@@ -441,9 +472,11 @@ def run_native(args):
     launches = runner.step()
     secs = runner.time_steps(runner.step, steps, warm, barrier)
     clocks = sampler.stop()
+    each = runner.time_each(runner.step, max(15, steps), 5)
     secs_e2e = runner.time_e2e(max(4, steps // 2), 2, barrier)
     secs, secs_e2e = replicas.max_over_ranks([secs, secs_e2e], device="cuda")
     per_step = secs / steps
+    sustained = runner.time_sustained(runner.step, per_step, local) if rank == 0 else None
     value = world * w.tokens / per_step
     h2d, d2h = runner.bytes_e2e()
 
@@ -453,7 +486,8 @@ def run_native(args):
         stages = runner.stage_profile(min(steps, 10))
         line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warm,
-            "ms_per_step": 1e3 * per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": 1e3 * per_step, "ms_per_step_median": 1e3 * float(np.median(each)),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if w.dtype == "f32" else "bf16 in, f32 accumulate", "data": "synthetic",
             "config": workload_config(w, world),
             "e2e": {"value": world * w.tokens / secs_e2e, "unit": "tokens/s", "h2d_bytes_per_step": h2d,
@@ -463,6 +497,9 @@ def run_native(args):
             "roofline": dominant_kernel_report(w, g, stages, peaks, ub, fb),
             "path_roofline": path_report(w, g, per_step, peaks, ub, fb),
             "tables": {"profile_states_P": g.P, "cached_subset_states_B": g.B, "nnzC": g.nnzC, "q": g.q},
+            "sustained": dict(sustained, value=world * w.tokens * sustained["steps"] / sustained["seconds"],
+                              unit="tokens/s"),
+            "fadd_rates_adds_per_s": peaks.get("fadd_rates"),
         }
     del runner
     torch.cuda.empty_cache()
@@ -475,11 +512,13 @@ def run_native(args):
             ws_ = synth.WORKLOADS[name]
             r = Runner(ws_, torch, binding, args.flags)
             gg = r.plan.geometry()
-            k = 5
-            s = r.time_steps(r.step, k, 3) / k
+            each_ = r.time_each(r.step, 15, 5)
+            s = float(np.median(each_))
             rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes(), r.plan.profile_table_element_bytes())
             st_ = r.stage_profile(3)
             sweep.append({"workload": name, "value": ws_.tokens / s, "unit": "tokens/s", "ms_per_step": 1e3 * s,
+                          "timing": "median of 15 steps after 5 warm-ups, one CUDA event pair per step",
+                          "ms_min": 1e3 * min(each_), "ms_max": 1e3 * max(each_),
                           "frac_2term": rep["frac_2term"], "frac_3term": rep["frac_3term"],
                           "frac_2term_fp32_tables": rep["frac_2term_fp32_tables"],
                           "roofline_ms_2term": rep["roofline_ms_2term"],

@@ -14,7 +14,8 @@
  * chunking proof (Eq. "lr-adjoint", Eq. "local-adjoint", suffix scan).
  *
  * Conventions shared by all entry points
- *   - Plain C linkage; no exceptions; the library keeps no global mutable state.
+ *   - Plain C linkage; no exceptions; the library keeps no global mutable state, with one exception that is
+ *     stated where it applies: the fixed device array (and its cached address) behind smat_forward_causal_static.
  *   - Q, K are [batch, heads, T, d_k]; V, O, dO are [batch, heads, T, d_v]; dQ, dK like Q,
  *     dV like V.  All are DEVICE pointers to contiguous row-major arrays (feature dimension
  *     fastest) of the plan's dtype, 16-byte aligned.  Accumulation is fp32.
@@ -85,7 +86,9 @@ typedef struct {
  *   q_override = 0 takes the default field size, the smallest prime q with q^d >= n
  *   (Sec. 3 asks for q = Θ(n^{1/d}); this constant reproduces the cache sizes the paper prints);
  *   any other value must be a prime and is used as given (small test cases).
- * On success *out owns host memory until smat_plan_destroy.  No device work is done.
+ * On success *out owns host memory until smat_plan_destroy.  No device work is done and no device is queried: the
+ * kernels a plan uses follow from the shape and the flags alone.  Calls that launch return SMAT_ERR_ARCH when the
+ * current device is not compute capability 10.x (the library holds sm_100a code only).
  */
 smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, int d_k, int d_v, int d, int chunk,
                              int q_override, smat_dtype dtype, unsigned flags);
@@ -94,7 +97,8 @@ void smat_plan_destroy(smat_plan* plan);
 smat_status smat_get_geometry(const smat_plan* plan, smat_geometry* out);
 
 /* 1 when this plan runs its causal branch on the tcgen05 tensor-core kernels (bf16, d_k = d_v = 128, block
- * boundary and recent length multiples of 128, SMAT_FLAG_SIMT_ONLY not set), 0 when it runs on the fp32 ALUs. */
+ * boundary and recent length multiples of 128, SMAT_FLAG_SIMT_ONLY not set), 0 when it runs on the fp32 ALUs.
+ * A property of the shape, not of the device. */
 int smat_uses_tensor_cores(const smat_plan* plan);
 
 /* Bytes per element of the type table U as smat_forward keeps it: 4 (fp32), or 2 when the plan runs the typed read on
@@ -109,14 +113,18 @@ int smat_type_table_element_bytes(const smat_plan* plan);
  * tables (the per-type sums of q dOᵀ and their transposed tabulation) in bf16 as well. */
 int smat_profile_table_element_bytes(const smat_plan* plan);
 
-/* Bytes of workspace smat_forward (for_backward = 0) or smat_backward (for_backward = 1) needs. 0 if plan is NULL. */
+/* Bytes of workspace smat_forward (for_backward = 0) or smat_backward (for_backward = 1) needs. 0 if plan is NULL.
+ * Every region is sized for the element type the plan stores in it (bf16 tables on tensor-core plans), and the
+ * score-tile buffers of the fp32-ALU path are reserved only for plans that run on it. */
 size_t smat_workspace_bytes(const smat_plan* plan, int for_backward);
 
 /*
  * Forward pass, Algorithm 1 steps 2-7 (step 1 is implicit: φ = q_i, ψ = k_j, Z_j = k_j v_jᵀ).
- * Reads Q, K, V; writes O (plan dtype).  The profile table F, the type table U ("cached subset
- * states") and the incoming chunk states S_in are left in the workspace as fp32 and can be read
- * back with smat_debug_tables.  Asynchronous on `cuda_stream`.
+ * Reads Q, K, V; writes O (plan dtype).  The profile table F and the type table U ("cached subset
+ * states") are left in the workspace in the element type the plan keeps them in (fp32, or bf16: see
+ * smat_profile_table_element_bytes / smat_type_table_element_bytes), the incoming states S_in as fp32 per
+ * chunk (fp32-ALU plans) or as bf16 per 128-token tile (tensor-core plans with SMAT_FLAG_PER_TILE_STATES);
+ * smat_debug_tables reads them back widened to fp32.  Asynchronous on `cuda_stream`.
  */
 smat_status smat_forward(const smat_plan* plan, const void* Q, const void* K, const void* V, void* O, void* workspace,
                          size_t workspace_bytes, void* cuda_stream);
@@ -148,15 +156,17 @@ smat_status smat_routing_indices(const smat_plan* plan, int32_t* prof, int32_t* 
 smat_status smat_debug_mask(const smat_plan* plan, uint8_t* mask, void* cuda_stream);
 
 /*
- * Copies of the fp32 tables a finished forward (or backward) left in `workspace`, into DEVICE
+ * Copies, widened to fp32, of the tables a finished forward (or backward) left in `workspace`, into DEVICE
  * buffers (any may be NULL):
  *   F   [batch*heads, P, d_k, d_v]     profile table        (Eq. "schedule")
  *   U   [batch*heads, B, d_k, d_v]     type table           (Eq. "schedule", Algorithm 2)
- *   Sin [batch*heads, T/chunk, d_k, d_v] incoming chunk states (Sec. 3.1, causal branch)
+ *   Sin [batch*heads, T/w, d_k, d_v]   incoming states of the causal branch (Sec. 3.1), one per chunk (w = chunk) on
+ *                                      fp32-ALU plans, one per 128-token tile (w = 128) on tensor-core plans
  * For d = 1 there is no separate F/U: the single state U_0 = F_0 is carried by the scan, and
- * F and U receive that state (the incoming state of the first recent chunk).
- * Plans that use the tensor-core kernels keep S_in as bf16 128-token tiles: for them Sin (and, for d = 1,
- * F and U) must be NULL, otherwise SMAT_ERR_UNSUPPORTED is returned.
+ * F and U receive that state (the incoming state of the first recent chunk or tile).
+ * Tensor-core plans have per-tile states only after a forward of a plan created with SMAT_FLAG_PER_TILE_STATES, or
+ * after smat_backward; the two-level form keeps one state per segment of tiles, which is no per-chunk table: there
+ * Sin (and, for d = 1, F and U) must be NULL, otherwise SMAT_ERR_UNSUPPORTED is returned.
  * Asynchronous on `cuda_stream`.
  */
 smat_status smat_debug_tables(const smat_plan* plan, const void* workspace, float* F, float* U, float* Sin,
@@ -206,6 +216,32 @@ int smat_profile_read(const smat_plan* plan, const char** names, float* ms, int 
 #define SMAT_STATIC_MAX_TILES 1024
 smat_status smat_forward_causal_static(const void* Q, const void* K, const void* V, void* O, int batch, int heads,
                                        int64_t T, void* cuda_stream);
+
+/*
+ * Status of the last smat_forward_causal_static on the current device (the paper has no counterpart).  That call has
+ * no workspace whose status word smat_check_status could read, so this reads the word kept in the static array:
+ * synchronises `cuda_stream`, returns SMAT_OK, SMAT_ERR_DEVICE_TIMEOUT if a bounded wait inside its kernels ran out
+ * (O is then invalid), or SMAT_ERR_LAUNCH if the stream reports a CUDA error.  Allocates nothing.
+ */
+smat_status smat_static_check_status(void* cuda_stream);
+
+/*
+ * Failure-path probe (the paper has no counterpart).  Launches a one-warp kernel in which one thread waits, with the
+ * same bounded wait every kernel of the library uses, on a barrier that nobody arrives on; after `limit_cycles` SM
+ * clock cycles (1 .. 2e9) the wait gives up, sets the status word at the start of `workspace` (DEVICE, 256-byte
+ * aligned, at least 256 bytes) and the kernel returns normally.  smat_check_status on that workspace then reports
+ * SMAT_ERR_DEVICE_TIMEOUT; the next smat_forward / smat_backward clears the word again.  Nothing faults or hangs.
+ */
+smat_status smat_debug_timeout_probe(void* workspace, int64_t limit_cycles, void* cuda_stream);
+
+/*
+ * Measured fp32 add rate of the plain ALUs of the current device (the paper has no counterpart; this is the ceiling
+ * the state additions of Algorithm 2 are charged against in the roofline report).  Runs independent register add
+ * chains on every SM, scalar adds (packed = 0) or two-lane adds (packed = 1), times them with CUDA events on
+ * `cuda_stream`, synchronises, and writes additions per second to *adds_per_second (HOST).  `scratch` is a DEVICE
+ * buffer of at least 4 bytes.
+ */
+smat_status smat_measure_fadd_rate(void* scratch, int packed, double* adds_per_second, void* cuda_stream);
 
 /* ---- Cached decoding of the recent block (Sec. "Memory-efficient decoding", Theorem "Streaming decoding") ----
  * The plan fixes T and with it the boundary n.  After the distant block (tokens 0 .. n-1) the decoder keeps B type

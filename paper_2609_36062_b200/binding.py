@@ -27,6 +27,7 @@ EXPORTS = [
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
     "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
     "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step",
+    "smat_static_check_status", "smat_debug_timeout_probe", "smat_measure_fadd_rate",
 ]
 
 
@@ -105,6 +106,12 @@ def load_library() -> ctypes.CDLL:
     lib.smat_uses_tensor_cores.restype = i
     lib.smat_forward_causal_static.argtypes = [vp, vp, vp, vp, i, i, i64, vp]
     lib.smat_forward_causal_static.restype = i
+    lib.smat_static_check_status.argtypes = [vp]
+    lib.smat_static_check_status.restype = i
+    lib.smat_debug_timeout_probe.argtypes = [vp, i64, vp]
+    lib.smat_debug_timeout_probe.restype = i
+    lib.smat_measure_fadd_rate.argtypes = [vp, i, ctypes.POINTER(ctypes.c_double), vp]
+    lib.smat_measure_fadd_rate.restype = i
     lib.smat_profile_enable.argtypes = [vp, i]
     lib.smat_profile_enable.restype = i
     lib.smat_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float), i]
@@ -157,6 +164,26 @@ def forward_causal_static(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, O: 
     return O
 
 
+def static_check_status(stream=None) -> None:
+    """Raises if the last forward_causal_static on this device hit a bounded-wait expiry (smat_static_check_status)."""
+    _check(load_library().smat_static_check_status(_stream(stream)), "smat_static_check_status")
+
+
+def debug_timeout_probe(workspace: torch.Tensor, limit_cycles: int = 2_000_000, stream=None) -> None:
+    """smat_debug_timeout_probe: a wait that is meant to run out sets the status word of `workspace`."""
+    _check(load_library().smat_debug_timeout_probe(_ptr(workspace), int(limit_cycles), _stream(stream)),
+           "smat_debug_timeout_probe")
+
+
+def measure_fadd_rate(packed: bool = False, stream=None) -> float:
+    """fp32 additions per second of the plain ALUs, measured (smat_measure_fadd_rate)."""
+    scratch = torch.zeros(64, dtype=torch.float32, device="cuda")
+    out = ctypes.c_double(0.0)
+    _check(load_library().smat_measure_fadd_rate(_ptr(scratch), int(packed), ctypes.byref(out), _stream(stream)),
+           "smat_measure_fadd_rate")
+    return float(out.value)
+
+
 class SmatPlan:
     """Owns one smat_plan and (optionally) a workspace tensor; mirrors the C entry points."""
 
@@ -166,6 +193,7 @@ class SmatPlan:
         self.dtype_code = {"f32": SMAT_F32, "bf16": SMAT_BF16}[dtype] if isinstance(dtype, str) else int(dtype)
         self.torch_dtype = _TORCH_DTYPE[self.dtype_code]
         self.shape = (batch, heads, T, d_k, d_v)
+        self.flags = int(flags)
         handle = ctypes.c_void_p()
         _check(self.lib.smat_plan_create(ctypes.byref(handle), batch, heads, T, d_k, d_v, d, chunk, q_override,
                                          self.dtype_code, flags), "smat_plan_create")
@@ -290,12 +318,13 @@ class SmatPlan:
         g = self.geometry()
         ws = self._ws if workspace is None else workspace
         tc = self.uses_tensor_cores()
+        tiles = tc and bool(self.flags & FLAG_PER_TILE_STATES)   # per-tile states exist on tensor-core plans only then
         F = U = Sin = None
-        if not (tc and g.d == 1):
+        if not (tc and g.d == 1 and not tiles):
             F = torch.empty((b * h, g.P, dk, dv), dtype=torch.float32, device=ws.device)
             U = torch.empty((b * h, g.B, dk, dv), dtype=torch.float32, device=ws.device)
-        if not tc:
-            Sin = torch.empty((b * h, T // g.c, dk, dv), dtype=torch.float32, device=ws.device)
+        if not tc or tiles:
+            Sin = torch.empty((b * h, T // (128 if tc else g.c), dk, dv), dtype=torch.float32, device=ws.device)
         _check(self.lib.smat_debug_tables(self.handle, _ptr(ws), _ptr(F), _ptr(U), _ptr(Sin), _stream(stream)),
                "smat_debug_tables")
         return F, U, Sin

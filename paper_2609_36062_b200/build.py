@@ -21,7 +21,8 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     stamp = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(HERE, "csrc", "*.h")) + glob.glob(os.path.join(HERE, "..", "include", "*.h"))
+    deps = (sources() + glob.glob(os.path.join(HERE, "csrc", "*.h")) + glob.glob(os.path.join(HERE, "csrc", "*.cuh")) +
+            glob.glob(os.path.join(HERE, "csrc", "*.inc")) + glob.glob(os.path.join(HERE, "..", "include", "*.h")))
     return any(os.path.getmtime(f) > stamp for f in deps)
 
 

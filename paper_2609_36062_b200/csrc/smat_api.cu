@@ -28,8 +28,11 @@ struct smat_plan {
   bool f_bf16;         // the profile table is kept in bf16 (d = 2: it is the type table; tab_tc: it is an MMA operand)
   bool tab_tc;         // d = 3, 4: tabulation and its transpose on the tensor cores (bf16 tables, resident Radon matrix)
   bool tab_d3_bf16;    // d = 3 with a prime too large for that kernel: bf16 profile table, sums on the fp32 ALUs
+  bool ubar_tc;        // backward pools the per-type adjoint states on the tensor cores
+  bool ubar_bf16;      // ... and keeps them in bf16
+  bool fbar_bf16;      // the per-profile adjoint states (transposed tabulation) are kept in bf16
   mutable int launches;
-  mutable bool last_was_forward;  // which call left its tables in the workspace
+  mutable bool tile_states;       // the last call left one bf16 incoming state per 128-token tile at off_sin
   // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
   mutable bool profiling;
   mutable cudaEvent_t events[SMAT_MAX_STAGES + 1];
@@ -232,6 +235,13 @@ smat_status check_common(const smat_plan* pl, const void* ws, size_t ws_bytes, i
 
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
 
+// Every kernel of the library is sm_100a code: a call that would launch on another device reports it instead.
+bool device_ok() {
+  const bool ok = smat_tc_available();
+  if (!ok) cudaGetLastError();  // a missing driver or device leaves a sticky-looking error code behind: clear it
+  return ok;
+}
+
 // Step 3 of Algorithm 1 (transpose = 0) or F̄ = Cᵀ Ū (transpose = 1).
 void tabulate(Ctx& cx, const char* name, const float* in, float* out, int transpose, int out_bf16 = 0) {
   const smat_plan* pl = cx.pl;
@@ -315,12 +325,14 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->batch = batch; pl->heads = heads; pl->bh = batch * heads;
   pl->r = d_k; pl->p = d_v; pl->T = T; pl->c = chunk; pl->NC = T / chunk;
   pl->dtype = dtype; pl->flags = flags; pl->rp = (int64_t)d_k * d_v; pl->launches = 0;
-  pl->profiling = false; pl->stages = 0; pl->last_was_forward = true;
+  pl->profiling = false; pl->stages = 0; pl->tile_states = false;
   smat_status s = build_geometry(&pl->geo, T, chunk, d, q_override);
   if (s != SMAT_OK) { delete pl; return s; }
   const SmatGeo& g = pl->geo;
+  // Which kernels a plan uses depends on the shape alone (no device work here); whether the current device can run
+  // them is checked by the calls that launch.
   pl->tc = dtype == SMAT_BF16 && d_k == 128 && d_v == 128 && !(flags & SMAT_FLAG_SIMT_ONLY) && g.n % 128 == 0 &&
-           g.m % 128 == 0 && g.n >= 128 && smat_tc_available();
+           g.m % 128 == 0 && g.n >= 128;
   if (!g.dense_G && (smat_tabulate_alg2_slab(g.B, pl->rp) < 1)) { delete pl; return SMAT_ERR_UNSUPPORTED; }
   // d >= 3 on the tensor-core path: U is only ever a bf16 MMA operand, so it is stored as bf16 (half the bytes)
   pl->tab_tc = pl->tc && !g.dense_G && !(flags & (SMAT_FLAG_ALG2_TABULATION | SMAT_FLAG_ALU_TABULATION)) &&
@@ -332,23 +344,35 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->f_bf16 = pl->pool_tc && ((g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION)) || pl->tab_tc || pl->tab_d3_bf16);
   pl->u_bf16 = pl->f_bf16 || (pl->tc && g.D >= 2 && !(flags & SMAT_FLAG_ALG2_TABULATION) &&
                               smat_tabulate_staged_slab(g, pl->rp, 0) >= 4);
-  const size_t state = (size_t)pl->rp * sizeof(float);
+  // adjoint tables of the backward pass
+  // F̄ readable by the tensor-core routed read: d = 2 (it is Ū), d = 3 when the staged transposed sums can write bf16
+  const bool fbar_by_read = pl->u_bf16 && (g.D == 1 || (g.D == 2 && !(flags & SMAT_FLAG_ALG2_TABULATION) &&
+                                                        smat_tabulate_staged_slab(g, pl->rp, 1) >= 4));
+  pl->ubar_tc = pl->tc && !g.dense_G && (pl->tab_tc || g.m / g.B >= 12);
+  pl->ubar_bf16 = pl->ubar_tc && ((g.D == 1 && fbar_by_read) || pl->tab_tc);   // d = 2: F̄ is Ū itself
+  pl->fbar_bf16 = pl->tc && !g.dense_G && (pl->tab_tc || (g.D == 1 ? pl->ubar_bf16 : fbar_by_read));
+  // Workspace regions, each sized for the element type the plan stores there.  Tensor-core plans keep the causal
+  // states per 128-token tile in bf16 (or, in the two-level form, fewer fp32 segment states in the same region) and
+  // have no score-tile buffers; the fp32-ALU plans keep one fp32 state per chunk and two fp32 score-tile buffers.
+  const size_t entries = (size_t)pl->rp;
   const int wide = d_k > d_v ? d_k : d_v;
+  const size_t causal = pl->tc ? (size_t)pl->bh * (T / 128) * entries * 2 : (size_t)pl->bh * pl->NC * entries * 4;
+  const size_t tiles = pl->tc ? 0 : (size_t)pl->bh * T * chunk * sizeof(float);
   size_t off = 0;
   pl->off_status = off; off = align_up(off + 256);
-  pl->off_sin = off;    off = align_up(off + (size_t)pl->bh * pl->NC * state);
+  pl->off_sin = off;    off = align_up(off + causal);
   // d = 2: C is the identity (U_h = F_h), so the two tables share storage unless Algorithm 2 is forced
   const bool alias = g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION);
-  pl->off_F = off;      off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.P * state));
-  pl->off_U = off;      off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.B * state));
+  pl->off_F = off;      off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.P * entries * (pl->f_bf16 ? 2 : 4)));
+  pl->off_U = off;      off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.B * entries * (pl->u_bf16 ? 2 : 4)));
   pl->off_acc = off;    off = align_up(off + (size_t)pl->bh * T * wide * sizeof(float));
-  pl->off_tileA = off;  off = align_up(off + (size_t)pl->bh * T * chunk * sizeof(float));
+  pl->off_tileA = off;  off = align_up(off + tiles);
   pl->off_W = off;      off = align_up(off + (pl->tab_tc ? (size_t)smat_tabulate_tc_scratch_elems(g, pl->rp, pl->bh) * 2 : 0));
   pl->off_fwd_end = off;
-  pl->off_dbar = off;   off = align_up(off + (size_t)pl->bh * pl->NC * state);
-  pl->off_ubar = off;   off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.B * state));
-  pl->off_fbar = off;   off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.P * state));
-  pl->off_tileG = off;  off = align_up(off + (size_t)pl->bh * T * chunk * sizeof(float));
+  pl->off_dbar = off;   off = align_up(off + causal);
+  pl->off_ubar = off;   off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.B * entries * (pl->ubar_bf16 ? 2 : 4)));
+  pl->off_fbar = off;   off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.P * entries * (pl->fbar_bf16 ? 2 : 4)));
+  pl->off_tileG = off;  off = align_up(off + tiles);
   pl->off_bwd_end = off;
   *out = pl;
   return SMAT_OK;
@@ -413,9 +437,9 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
   smat_status s = check_common(pl, workspace, workspace_bytes, 0);
   if (s != SMAT_OK) return s;
   if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
-  pl->last_was_forward = true;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   if (pl->tc) {
     int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
@@ -434,6 +458,7 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
       else
         state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);
     }
+    pl->tile_states = L < 2;
     if (L >= 2) {  // steps 5-7, two-level: segment totals, scan of the totals, fused per-segment output
       float* seg = cx.f(pl->off_sin);
       int nseg0 = 0, nseg1 = 0;
@@ -473,9 +498,9 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
   if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(dO) || misaligned(dQ) || misaligned(dK) ||
       misaligned(dV))
     return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
-  pl->last_was_forward = (pl->tc && (pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES)) ? pl->last_was_forward : false;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   const bool lr = !pl->geo.dense_G;
   if (pl->tc) {
@@ -484,28 +509,27 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
     // that each within-chunk adjoint adds to its rows.
     int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
     float* lrbuf = cx.f(pl->off_acc);
+    pl->tile_states = true;
     const SmatGroupSpec types = group(pl, SMAT_GM_TYPE), profs = group(pl, SMAT_GM_PROFILE);
     const int64_t n = pl->geo.n;
-    const bool fbar_bf16 = pl->u_bf16 && pl->geo.D <= 2;  // F̄ readable by the tensor-core read (d = 2, 3)
     if (lr) {
       if (!(pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES)) build_type_table(cx, K, V);
       // Ū_h = Σ q dOᵀ over the type (Eq. "lr-adjoint"), then F̄ = Cᵀ Ū
-      const bool ubar_tc = pl->tab_tc || pl->geo.m / pl->geo.B >= 12;
-      const bool ubar_bf16 = ubar_tc && ((pl->geo.D == 1 && fbar_bf16) || pl->tab_tc);  // d = 2: F̄ is Ū itself
+      const bool ubar_tc = pl->ubar_tc, ubar_bf16 = pl->ubar_bf16;
       if (ubar_tc)
         SMAT_TRY(cx, "bwd_pool_type_tc", smat_launch_pool_tc(Q, dO, cx.ws + pl->off_ubar, ubar_bf16, types, pl->geo.B,
                                                              max_group_tokens(pl, SMAT_GM_TYPE), pl->T, pl->bh,
                                                              status, cx.st));
       else
         outer_sum(cx, "bwd_pool_type", SMAT_GM_TYPE, Q, dO, cx.f(pl->off_ubar));
-      const bool fbar_is_bf16 = pl->tab_tc || (pl->geo.D == 1 ? ubar_bf16 : fbar_bf16);
+      const bool fbar_is_bf16 = pl->fbar_bf16;
       if (pl->tab_tc)
         tabulate_tc(cx, "bwd_tabulate_t_tc", cx.ws + pl->off_ubar, cx.ws + pl->off_fbar, 1);
       else
-        tabulate(cx, "bwd_tabulate_t", cx.f(pl->off_ubar), cx.f(pl->off_fbar), 1, pl->geo.D == 2 && fbar_bf16);
+        tabulate(cx, "bwd_tabulate_t", cx.f(pl->off_ubar), cx.f(pl->off_fbar), 1, pl->geo.D == 2 && pl->fbar_bf16);
       // per-tile states
-      SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 0, 0, status, cx.st));
-      SMAT_TRY(cx, "bwd_chunk_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 0, 1, status, cx.st));
+      SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 0, 0, status, cx.st));
+      SMAT_TRY(cx, "bwd_suffix_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 0, 1, status, cx.st));
       // dQ: recent rows add U_type dO
       if (pl->u_bf16)
         SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, lrbuf, nullptr, 1, types, pl->geo.B,
@@ -531,8 +555,8 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
       SMAT_TRY(cx, "bwd_dv_tile_tc", smat_launch_chunk_adjoint_tc(2, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
                                                                   lrbuf, 0, n, dV, pl->T, pl->bh, status, cx.st));
     } else {
-      SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 1, 0, status, cx.st));
-      SMAT_TRY(cx, "bwd_chunk_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 1, 1, status, cx.st));
+      SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 1, 0, status, cx.st));
+      SMAT_TRY(cx, "bwd_suffix_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 1, 1, status, cx.st));
       for (int which = 0; which < 3; ++which)
         SMAT_TRY(cx, which == 0 ? "bwd_dq_tile_tc" : (which == 1 ? "bwd_dk_tile_tc" : "bwd_dv_tile_tc"),
                  smat_launch_chunk_adjoint_tc(which, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar, lrbuf, 0, 0,
@@ -601,6 +625,7 @@ smat_status smat_routing_indices(const smat_plan* pl, int32_t* prof, int32_t* ty
 smat_status smat_debug_mask(const smat_plan* pl, uint8_t* mask, void* cuda_stream) {
   if (!pl || !mask) return SMAT_ERR_NULL;
   if (pl->T > 8192) return SMAT_ERR_SHAPE;
+  if (!device_ok()) return SMAT_ERR_ARCH;
   return smat_launch_mask(mask, pl->geo, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? SMAT_OK
                                                                                                  : SMAT_ERR_LAUNCH;
 }
@@ -612,8 +637,25 @@ smat_status smat_debug_tables(const smat_plan* pl, const void* workspace, float*
   const char* ws = static_cast<const char*>(workspace);
   const size_t state = (size_t)pl->rp * sizeof(float);
   cudaError_t err = cudaSuccess;
-  if (pl->tc && (Sin || (pl->geo.dense_G && (F || U)))) return SMAT_ERR_UNSUPPORTED;  // tensor-core path keeps S_in as bf16 tiles
-  if (Sin) err = cudaMemcpyAsync(Sin, ws + pl->off_sin, (size_t)pl->bh * pl->NC * state, cudaMemcpyDeviceToDevice, st);
+  if (pl->tc) {
+    // Tensor-core plans: incoming states exist per 128-token tile (bf16) after a per-tile forward or a backward; the
+    // two-level form keeps only one state per segment of tiles, which is no per-chunk table.
+    const bool want_states = Sin || (pl->geo.dense_G && (F || U));
+    if (want_states && !pl->tile_states) return SMAT_ERR_UNSUPPORTED;
+    const int64_t tiles = pl->T / 128;
+    if (Sin) err = smat_launch_widen_bf16(ws + pl->off_sin, Sin, (int64_t)pl->bh * tiles * pl->rp, st);
+    if (pl->geo.dense_G) {  // d = 1: the state entering the first recent tile is U_0 = F_0
+      for (int t = 0; t < 2; ++t) {
+        float* dst = t ? U : F;
+        for (int h = 0; dst && h < pl->bh && err == cudaSuccess; ++h)
+          err = smat_launch_widen_bf16(ws + pl->off_sin + ((size_t)h * tiles + pl->geo.n / 128) * pl->rp * 2,
+                                       dst + (size_t)h * pl->rp, pl->rp, st);
+      }
+      return err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+    }
+  } else if (Sin) {
+    err = cudaMemcpyAsync(Sin, ws + pl->off_sin, (size_t)pl->bh * pl->NC * state, cudaMemcpyDeviceToDevice, st);
+  }
   if (pl->geo.dense_G) {
     const int64_t first_recent = pl->geo.n / pl->c;
     for (int t = 0; t < 2; ++t) {
@@ -624,13 +666,13 @@ smat_status smat_debug_tables(const smat_plan* pl, const void* workspace, float*
     }
   } else {
     if (F && err == cudaSuccess) {
-      if (pl->f_bf16 && pl->last_was_forward)
+      if (pl->f_bf16)
         err = smat_launch_widen_bf16(ws + pl->off_F, F, (int64_t)pl->bh * pl->geo.P * pl->rp, st);
       else
         err = cudaMemcpyAsync(F, ws + pl->off_F, (size_t)pl->bh * pl->geo.P * state, cudaMemcpyDeviceToDevice, st);
     }
     if (U && err == cudaSuccess) {
-      if (pl->u_bf16 && pl->last_was_forward)  // the forward of this plan keeps U in bf16: widen on export
+      if (pl->u_bf16)  // this plan keeps U in bf16: widen on export
         err = smat_launch_widen_bf16(ws + pl->off_U, U, (int64_t)pl->bh * pl->geo.B * pl->rp, st);
       else
         err = cudaMemcpyAsync(U, ws + pl->off_U, (size_t)pl->bh * pl->geo.B * state, cudaMemcpyDeviceToDevice, st);
@@ -664,9 +706,9 @@ smat_status smat_decode_begin(const smat_plan* pl, const void* K, const void* V,
   if (s != SMAT_OK) return s;
   if (cache_bytes < smat_decode_cache_bytes(pl)) return SMAT_ERR_WORKSPACE;
   if (misaligned(K) || misaligned(V) || (reinterpret_cast<uintptr_t>(cache) & 255)) return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
-  pl->last_was_forward = false;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   const size_t off = build_type_table(cx, K, V);
   const size_t tbytes = (size_t)pl->bh * pl->geo.B * pl->rp * (pl->u_bf16 ? 2 : 4);
@@ -685,6 +727,7 @@ smat_status smat_decode_step(const smat_plan* pl, const void* q, const void* k, 
   if (cache_bytes < smat_decode_cache_bytes(pl)) return SMAT_ERR_WORKSPACE;
   if (t < pl->geo.n || t >= pl->T) return SMAT_ERR_SHAPE;
   if (reinterpret_cast<uintptr_t>(cache) & 255) return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
   float* S = reinterpret_cast<float*>(static_cast<char*>(cache) + decode_table_bytes(pl));
   const cudaError_t err = smat_launch_decode_step(q, k, v, o, S, cache, pl->u_bf16 ? 1 : 0, pl->dtype == SMAT_BF16 ? 1 : 0,
                                                   smat_type_of(pl->geo, t), pl->geo.B, pl->r, pl->p, pl->bh,

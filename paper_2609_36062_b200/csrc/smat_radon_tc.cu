@@ -62,6 +62,7 @@ constexpr int ALU_WARPS = 2;
 constexpr int ALU_MAX_ROWS = 8;
 constexpr int RADON_THREADS = 32 * (ALU_WARP + ALU_WARPS);
 constexpr int MAX_ACC = 4;                        // accumulators in flight: what the R columns leave of 512, at most 4
+constexpr int RADON_EXCHANGE_CTAS = 148;          // CTAs of a one-launch two-stage tabulation (one exchange slab each)
 constexpr int ROW_INVALID = -1;
 constexpr int ROW_VERT = 1 << 30;                 // flag: row of the extra ("vertical") class
 
@@ -887,6 +888,7 @@ cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (nph == 2 && sms > RADON_EXCHANGE_CTAS) sms = RADON_EXCHANGE_CTAS;  // one private exchange slab per CTA was sized for
   int64_t ctas = (int64_t)(sms / sh.parts) * sh.parts;
   const int64_t items = nph == 1 ? prm.slabs * sp[0].images * sh.parts : prm.slabs;
   if (items < ctas) ctas = items;
@@ -957,7 +959,7 @@ bool radon_two_stage_fits(int q, int transpose) {
   RadonShape sh;
   const int qq = q * q;
   if (!radon_shape(q, transpose, transpose ? 1 : 0, transpose ? qq : qq + q, &sh) || sh.parts != 1) return false;
-  return ((int64_t)qq * q + qq) * 256 * 148 <= (64LL << 20);
+  return ((int64_t)qq * q + qq) * 256 * RADON_EXCHANGE_CTAS <= (64LL << 20);
 }
 
 }  // namespace
@@ -968,7 +970,7 @@ int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems) {
   if (state_elems % 128) return 0;
   const int qq = geo.q * geo.q;
   RadonShape a, b;
-  return radon_encode_fn() && radon_shape(geo.q, 0, 0, qq + geo.q, &a) && radon_shape(geo.q, 1, 1, qq, &b) ? 1 : 0;
+  return radon_shape(geo.q, 0, 0, qq + geo.q, &a) && radon_shape(geo.q, 1, 1, qq, &b) ? 1 : 0;
 }
 
 // Rows (of state_elems bf16 each, per head) of the intermediate table the d = 4 stages exchange.
@@ -982,11 +984,8 @@ int64_t smat_tabulate_tc_scratch_elems(const SmatGeo& geo, int64_t state_elems, 
   const int64_t rows = smat_tabulate_tc_scratch_rows(geo);
   if (rows == 0) return 0;
   if (radon_two_stage_fits(geo.q, 0) && radon_two_stage_fits(geo.q, 1)) {
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     int64_t ctas = (int64_t)bh * (state_elems / 128);
-    if (ctas > sms) ctas = sms;
+    if (ctas > RADON_EXCHANGE_CTAS) ctas = RADON_EXCHANGE_CTAS;
     return ctas * rows * 128;
   }
   return (int64_t)bh * rows * state_elems;

@@ -71,3 +71,16 @@ extern "C" smat_status smat_forward_causal_static(const void* Q, const void* K, 
     return SMAT_ERR_LAUNCH;
   return SMAT_OK;
 }
+
+// Reads back the status word of the static scratch: a bounded wait that ran out inside one of the two kernels above
+// is reported here, since there is no caller-owned workspace that smat_check_status could look at.
+extern "C" smat_status smat_static_check_status(void* cuda_stream) {
+  void* scratch = nullptr;
+  if (!smat_tc_available()) { cudaGetLastError(); return SMAT_ERR_ARCH; }
+  if (scratch_for_current_device(&scratch) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, scratch, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  return word == 0 ? SMAT_OK : SMAT_ERR_DEVICE_TIMEOUT;
+}

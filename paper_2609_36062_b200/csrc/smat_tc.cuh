@@ -42,6 +42,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 struct WaitCtx {
   volatile int* cta_abort;  // shared memory flag
   int* status;              // global status word
+  long long limit = 4000000000LL;  // SM clock cycles before a wait gives up
 };
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -50,7 +51,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 255u) {
       if (*w.cta_abort) return false;
-      if (clock64() - start > 4000000000LL) break;
+      if (clock64() - start > w.limit) break;
     }
   }
   *w.cta_abort = 1;

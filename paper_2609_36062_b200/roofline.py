@@ -16,7 +16,8 @@ r = d_k, p = d_v, e = bytes per input element, fp32 tables:
 
 Chunk-state traffic (T/c states written and read) depends on the implementation and is not counted.
 Peaks come from MEASURED_PEAKS.json when present (HBM copy GB/s, dense bf16 TFLOP/s, both measured on
-this machine's B200s), else from the stated fallback.  The fp32 add peak is nominal:
+this machine's B200s), else from the stated fallback.  The fp32 add peak is the rate the library's add
+microbenchmark measures on the device (bench.py puts it into the peaks), else nominal:
 148 SMs x 128 lanes x the maximum SM clock.
 """
 from __future__ import annotations
@@ -85,13 +86,15 @@ def roofline_times(work: Work, peaks: dict, sustained: bool = True) -> dict:
     at the tensor peak against the HBM term; 3-term: table additions charged at the fp32 add peak)."""
     tflops = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"] * 1e12
     hbm = peaks["hbm_gbs"] * 1e9
-    alu = 148 * 128 * peaks.get("sm_max_mhz", 1965.0) * 1e6
+    # fp32 add peak: measured on the device when the caller put it into `peaks` (bench.py does), else nominal
+    alu = peaks.get("fadd_adds_per_s") or 148 * 128 * peaks.get("sm_max_mhz", 1965.0) * 1e6
     t_tensor = work.flops / tflops
     t_alu = work.adds / alu
     t_hbm = work.bytes / hbm
     t2 = max((work.flops + work.adds) / tflops, t_hbm)
     t3 = max(t_tensor, t_alu, t_hbm)
-    return {"t_tensor": t_tensor, "t_alu": t_alu, "t_hbm": t_hbm, "t_2term": t2, "t_3term": t3, "alu_peak_adds": alu}
+    return {"t_tensor": t_tensor, "t_alu": t_alu, "t_hbm": t_hbm, "t_2term": t2, "t_3term": t3, "alu_peak_adds": alu,
+            "alu_peak_source": "measured" if peaks.get("fadd_adds_per_s") else "nominal"}
 
 
 # Per-kernel algorithmic traffic (bytes), adds and flop, keyed by the stage names the library reports.

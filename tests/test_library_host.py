@@ -95,3 +95,42 @@ def test_non_default_geometry_flags():
     assert not g.vc_conditions_met
     g = binding.SmatPlan(1, 1, 256, 64, 64, 4, 16, "f32", q_override=2).geometry()
     assert g.vc_conditions_met and (g.P, g.B) == (8, 14)
+
+
+def test_workspace_regions_follow_the_stored_element_types():
+    """The bf16 tables and per-tile states of a tensor-core plan take half the bytes of their fp32 forms, and such a
+    plan reserves no score-tile buffers; the plan is a function of the shape alone (no device is needed to size it)."""
+    w = synth.WORKLOADS["t64k_d4"]
+    plan = binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype)
+    assert plan.uses_tensor_cores() and plan.profile_table_element_bytes() == 2 and plan.type_table_element_bytes() == 2
+    g = plan.geometry()
+    state = w.d_k * w.d_v
+    tables = w.bh * (g.P + g.B) * state * 2                      # F and U in bf16
+    exchange = w.bh * (g.q ** 3 + g.q ** 2) * state * 2          # intermediate of the two d = 4 tabulation stages
+    causal = w.bh * (w.T // 128) * state * 2
+    rows = w.bh * w.T * 128 * 4                                  # long-range rows
+    need = tables + exchange + causal + rows
+    got = plan.workspace_bytes(False)
+    assert need <= got <= need + 64 * 1024, (got, need)
+    assert got < 9.0e9                                           # 15 GB with every region at 4 bytes per entry
+    simt = binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype, flags=binding.FLAG_SIMT_ONLY)
+    assert simt.workspace_bytes(False) > got
+    # backward: adjoint tables in bf16 too, per-tile adjoint states
+    back = plan.workspace_bytes(True)
+    assert got + tables + causal <= back <= got + tables + causal + 64 * 1024
+
+
+def test_launching_calls_report_a_missing_sm100_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present: the calls below would launch")
+    lib = binding.load_library()
+    h = ctypes.c_void_p()
+    assert lib.smat_plan_create(ctypes.byref(h), 1, 1, 512, 64, 64, 2, 64, 0, 0, 0) == 0
+    # all arguments are acceptable; what is missing is a compute capability 10.x device
+    assert lib.smat_forward(h, 256, 256, 256, 256, 256, 1 << 40, None) == 7
+    assert lib.smat_backward(h, 256, 256, 256, 256, 256, 256, 256, 256, 1 << 40, None) == 7
+    assert lib.smat_forward_causal_static(256, 256, 256, 256, 1, 1, 128, None) == 7
+    assert lib.smat_debug_timeout_probe(256, 1000, None) == 7
+    assert "sm_100" in binding.status_string(7)
+    lib.smat_plan_destroy(h)

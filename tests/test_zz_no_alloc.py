@@ -1,4 +1,5 @@
-"""The allocation-free causal forward (smat_forward_causal_static) against the workspace-based smat_forward.
+"""The allocation-free causal forward (smat_forward_causal_static) against the fp64 oracle and against the
+workspace-based smat_forward.
 
 Runs last in the suite on purpose: if it fails, a run that stops at the first failure has already
 exercised everything else.  It must also pass alone in a fresh process, where its first call is the one
@@ -6,8 +7,9 @@ that looks up the static scratch array."""
 import pytest
 import torch
 
+from oracle import smat_oracle as so
 from paper_2609_36062_b200 import binding, synth
-from tests.helpers import TOL, device_inputs, rel_err, to_numpy64
+from tests.helpers import TOL, device_inputs, rel_err, sample_tokens, to_numpy64
 
 pytestmark = pytest.mark.gpu
 
@@ -27,10 +29,17 @@ def test_static_scratch_forward_matches_workspace_forward_twice_in_a_row():
         before = count()
         got = binding.forward_causal_static(dev["q"], dev["k"], dev["v"], out)
         assert count() == before                                 # nothing was allocated through torch either
-        torch.cuda.synchronize()
+        binding.static_check_status()                            # syncs; no bounded wait ran out on the static path
+        assert count() == before
         err = rel_err(to_numpy64(got), to_numpy64(ref))
         assert err <= TOL["bf16"], err
         outs.append(err)
+        # and against the oracle itself (d = 1: the causal mask), on sampled rows of the last head
+        geo = so.geometry(T, 128, 1)
+        rows = sample_tokens(geo, 48, seed=seed)
+        Q64, K64, V64 = (synth.as_float64(w, host[x][heads - 1]) for x in ("q", "k", "v"))
+        oracle_rows = so.forward_rows(Q64, K64, V64, geo, rows)
+        assert rel_err(to_numpy64(got[0, heads - 1][rows]), oracle_rows) <= TOL["bf16"]
     assert max(outs) <= TOL["bf16"]
 
 
