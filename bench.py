@@ -476,7 +476,6 @@ def run_native(args):
     secs_e2e = runner.time_e2e(max(4, steps // 2), 2, barrier)
     secs, secs_e2e = replicas.max_over_ranks([secs, secs_e2e], device="cuda")
     per_step = secs / steps
-    sustained = runner.time_sustained(runner.step, per_step, local) if rank == 0 else None
     value = world * w.tokens / per_step
     h2d, d2h = runner.bytes_e2e()
 
@@ -484,6 +483,7 @@ def run_native(args):
     if rank == 0:
         ub, fb = runner.plan.type_table_element_bytes(), runner.plan.profile_table_element_bytes()
         stages = runner.stage_profile(min(steps, 10))
+        sustained = runner.time_sustained(runner.step, per_step, local)   # last: it heats the board
         line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warm,
             "ms_per_step": 1e3 * per_step, "ms_per_step_median": 1e3 * float(np.median(each)),

@@ -68,6 +68,10 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
                                         with staged sums on the fp32 ALUs instead of the Radon stages on the tensor cores
                                         (which keep F, U and the stage intermediate in bf16) */
 
+#define SMAT_FLAG_D3_SHARED_SUMS 32u /* d = 3 with a prime beyond the tensor-core tabulation: form every q-term sum
+                                        straight from the shared-memory slab (one output row per thread) instead of
+                                        the register-resident form (K slopes x q offsets per thread) */
+
 /* Sizes of the construction (Sec. 3, "construction of G" and "Scaling with sequence length"). */
 typedef struct {
   int64_t T, c, n, m;  /* sequence length, chunk width, distant = c*floor(T/2c), recent = T - n */

@@ -21,6 +21,7 @@ FLAG_ALG2_TABULATION = 2
 FLAG_PER_TILE_STATES = 4
 FLAG_KEEP_FORWARD_TABLES = 8
 FLAG_ALU_TABULATION = 16
+FLAG_D3_SHARED_SUMS = 32
 
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",

@@ -28,6 +28,7 @@ struct smat_plan {
   bool f_bf16;         // the profile table is kept in bf16 (d = 2: it is the type table; tab_tc: it is an MMA operand)
   bool tab_tc;         // d = 3, 4: tabulation and its transpose on the tensor cores (bf16 tables, resident Radon matrix)
   bool tab_d3_bf16;    // d = 3 with a prime too large for that kernel: bf16 profile table, sums on the fp32 ALUs
+  bool tab_d3_regs;    // ... with the sums held in registers; the profile table is then stored slab-major
   bool ubar_tc;        // backward pools the per-type adjoint states on the tensor cores
   bool ubar_bf16;      // ... and keeps them in bf16
   bool fbar_bf16;      // the per-profile adjoint states (transposed tabulation) are kept in bf16
@@ -285,11 +286,14 @@ size_t build_type_table(Ctx& cx, const void* K, const void* V) {
     if (pl->pool_tc)
       SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, group(pl, SMAT_GM_PROFILE),
                                                   pl->geo.P, max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh,
-                                                  status, cx.st));
+                                                  status, cx.st, pl->tab_d3_regs ? 1 : 0));
     else
       outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
     if (pl->tab_tc)
       tabulate_tc(cx, "tabulate_tc", cx.ws + pl->off_F, cx.ws + pl->off_U, 0);
+    else if (pl->tab_d3_regs)
+      SMAT_TRY(cx, "tabulate_regs", smat_launch_tabulate_d3_regs(cx.ws + pl->off_F, cx.ws + pl->off_U, pl->geo, pl->rp,
+                                                                  pl->bh, status, cx.st));
     else if (pl->tab_d3_bf16)
       SMAT_TRY(cx, "tabulate_bf16", smat_launch_tabulate_d3_bf16(cx.ws + pl->off_F, cx.ws + pl->off_U, pl->geo, pl->rp,
                                                                   pl->bh, cx.st));
@@ -340,6 +344,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->tab_d3_bf16 = pl->tc && g.D == 2 && !pl->tab_tc &&
                     !(flags & (SMAT_FLAG_ALG2_TABULATION | SMAT_FLAG_ALU_TABULATION)) &&
                     smat_tabulate_d3_bf16_slab(g, pl->rp) > 0;
+  pl->tab_d3_regs = pl->tab_d3_bf16 && smat_tabulate_d3_regs_supported(g, pl->rp) && !(flags & SMAT_FLAG_D3_SHARED_SUMS);
   pl->pool_tc = pl->tc && !g.dense_G && (g.n / g.P >= 12 || pl->tab_tc || pl->tab_d3_bf16);
   pl->f_bf16 = pl->pool_tc && ((g.D == 1 && !(flags & SMAT_FLAG_ALG2_TABULATION)) || pl->tab_tc || pl->tab_d3_bf16);
   pl->u_bf16 = pl->f_bf16 || (pl->tc && g.D >= 2 && !(flags & SMAT_FLAG_ALG2_TABULATION) &&
@@ -666,7 +671,9 @@ smat_status smat_debug_tables(const smat_plan* pl, const void* workspace, float*
     }
   } else {
     if (F && err == cudaSuccess) {
-      if (pl->f_bf16)
+      if (pl->tab_d3_regs)
+        err = smat_launch_widen_bf16_slabs(ws + pl->off_F, F, pl->bh, pl->geo.P, pl->rp, st);
+      else if (pl->f_bf16)
         err = smat_launch_widen_bf16(ws + pl->off_F, F, (int64_t)pl->bh * pl->geo.P * pl->rp, st);
       else
         err = cudaMemcpyAsync(F, ws + pl->off_F, (size_t)pl->bh * pl->geo.P * state, cudaMemcpyDeviceToDevice, st);

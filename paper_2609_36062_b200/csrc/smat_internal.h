@@ -118,6 +118,11 @@ cudaError_t smat_launch_decode_step(const void* q, const void* k, const void* v,
 int smat_tabulate_d3_bf16_slab(const SmatGeo& geo, int64_t state_elems);
 cudaError_t smat_launch_tabulate_d3_bf16(const void* in, void* out, const SmatGeo& geo, int64_t state_elems, int bh,
                                          cudaStream_t st);
+// The same tabulation with the sums held in registers (K slopes x q offsets per thread, every column value loaded
+// once per K slopes); covers the primes it was instantiated for.
+int smat_tabulate_d3_regs_supported(const SmatGeo& geo, int64_t state_elems);
+cudaError_t smat_launch_tabulate_d3_regs(const void* in, void* out, const SmatGeo& geo, int64_t state_elems, int bh,
+                                         int* status, cudaStream_t st);
 // bf16 -> fp32 copy of a table (debug export).
 // Tabulation on the tensor cores (bf16 tables; d = 3, 4 with a prime small enough for a resident Radon matrix).
 int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems);
@@ -127,8 +132,13 @@ cudaError_t smat_launch_tabulate_tc(const void* in, void* out, void* scratch, co
                                     int bh, int transpose, int* status, cudaStream_t st, int* launches);
 cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st);
 // Pooling on tensor cores: F[bh][x] = Σ_{t ≡ x (mod P), t < n} k_t v_tᵀ, stored as fp32 or bf16.
+// slab_major = 1 (bf16 only): F is stored as [bh][rp / 32][groups][32], 32 consecutive entries of every state together.
 cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, const SmatGroupSpec& grp,
-                                int64_t groups, int64_t max_tokens, int64_t T, int bh, int* status, cudaStream_t st);
+                                int64_t groups, int64_t max_tokens, int64_t T, int bh, int* status, cudaStream_t st,
+                                int slab_major = 0);
+// bf16 table kept slab-major [bh][rp / 32][rows][32] -> fp32 [bh][rows][rp] (debug export).
+cudaError_t smat_launch_widen_bf16_slabs(const void* src_bf16, float* dst, int64_t heads, int64_t rows, int64_t rp,
+                                         cudaStream_t st);
 // Two-level causal branch: segment totals, then (after an exclusive scan of the totals) per-segment fused output.
 int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh);
 void smat_segment_counts(int64_t tiles0, int64_t tiles1, int bh, int L, int* nseg0, int* nseg1);

@@ -473,6 +473,22 @@ cudaError_t smat_launch_tabulate_d3_bf16(const void* in, void* out, const SmatGe
   return cudaGetLastError();
 }
 
+__global__ void widen_bf16_slabs_kernel(const __nv_bfloat16* __restrict__ src, float* __restrict__ dst, int64_t rows,
+                                        int64_t rp, int64_t count) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // index into dst [heads][rows][rp]
+  if (idx >= count) return;
+  const int64_t e = idx % rp, row = (idx / rp) % rows, head = idx / (rp * rows);
+  dst[idx] = __bfloat162float(src[((head * (rp / 32) + e / 32) * rows + row) * 32 + e % 32]);
+}
+
+cudaError_t smat_launch_widen_bf16_slabs(const void* src_bf16, float* dst, int64_t heads, int64_t rows, int64_t rp,
+                                         cudaStream_t st) {
+  const int64_t count = heads * rows * rp;
+  widen_bf16_slabs_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src_bf16), dst,
+                                                                           rows, rp, count);
+  return cudaGetLastError();
+}
+
 cudaError_t smat_launch_widen_bf16(const void* src_bf16, float* dst, int64_t count, cudaStream_t st) {
   widen_bf16_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src_bf16), dst,
                                                                      count);

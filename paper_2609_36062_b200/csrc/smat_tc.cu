@@ -915,6 +915,8 @@ struct PoolParams {
   const __nv_bfloat16* K;  // rows giving the first state index
   const __nv_bfloat16* V;  // rows giving the second state index
   void* F;                 // [bh][groups][128][128] fp32 or bf16
+  int slab_major;          // bf16 only: store as [bh][512 slabs of 32 entries][groups][32] instead (a slab of entries of
+                           // every state contiguous, the order the register-resident d = 3 tabulation reads)
   int* status;
 };
 
@@ -1022,6 +1024,10 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
           }
           if (OUT_BF16) {
             __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(prm.F) + (item * TILE + i) * TILE + cb * 32;
+            if (prm.slab_major) {   // entries 32 (4 i + cb) .. + 31 of this state are slab 4 i + cb of its head
+              const int64_t head = item / prm.groups, g = item - head * prm.groups;
+              dst = static_cast<__nv_bfloat16*>(prm.F) + ((head * (TILE * TILE / 32) + (4 * i + cb)) * prm.groups + g) * 32;
+            }
 #pragma unroll
             for (int h8 = 0; h8 < 2; ++h8) {  // whole 32-byte sectors
               uint32_t w[8];
@@ -1117,6 +1123,20 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t rows, int box_rows = 
 }
 
 }  // namespace
+
+// bf16 matrix [rows, inner] row-major; box = box_inner x box_rows; optional 128-byte swizzle (box_inner = 64 then).
+bool smat_make_map_2d_bf16(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint32_t box_inner,
+                           uint32_t box_rows, int swizzle128) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)inner * 2};
+  const cuuint32_t box[2] = {box_inner, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 // The library holds sm_100a code only: the current device must be compute capability 10.x, and the driver must
 // export the tensor-map encoder the TMA kernels need.
@@ -1233,8 +1253,11 @@ static cudaError_t launch_pool_tc(const PoolParams& prm, cudaStream_t st) {
 }
 
 cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_bf16, const SmatGroupSpec& grp,
-                                int64_t groups, int64_t max_tokens, int64_t T, int bh, int* status, cudaStream_t st) {
+                                int64_t groups, int64_t max_tokens, int64_t T, int bh, int* status, cudaStream_t st,
+                                int slab_major) {
   PoolParams prm;
+  if (slab_major && !out_bf16) return cudaErrorInvalidValue;
+  prm.slab_major = slab_major;
   prm.T = T; prm.grp = grp; prm.groups = groups; prm.items = (int64_t)bh * groups;
   prm.K = static_cast<const __nv_bfloat16*>(K);
   prm.V = static_cast<const __nv_bfloat16*>(V);
