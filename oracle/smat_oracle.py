@@ -193,6 +193,106 @@ def mask_col(s: int, geo: Geometry) -> np.ndarray:
     return col
 
 
+# --------------------------------------------------------------------------- user-supplied routing
+def routed_mask_row(t: int, geo: Geometry, prof_cells, types) -> np.ndarray:
+    """Row t of the mask when the assignment is given explicitly (Sec. 3, "construction of G": any maps prof, type give
+    G_ij = 1{prof(j) ∈ H_type(i)}, Eq. Gdef).  prof_cells[s] is the packed cell (little-endian base-q integer) of
+    distant token s, types[i] the type of recent token n + i; an entry outside its range belongs to no cell / no type
+    and contributes no long-range edge.  The two causal blocks do not depend on the assignment."""
+    row = np.zeros(geo.T, dtype=np.uint8)
+    if t < geo.n:
+        row[: t + 1] = 1
+        return row
+    row[geo.n : t + 1] = 1
+    if geo.dense_G:
+        row[: geo.n] = 1
+        return row
+    h = int(types[t - geo.n])
+    if not 0 <= h < geo.B:
+        return row
+    a, b = type_pair(h, geo)
+    cells = np.asarray(prof_cells, dtype=np.int64)
+    v = cells.copy()
+    acc = np.zeros(geo.n, dtype=np.int64)
+    for ell in range(geo.D):
+        acc += a[ell] * (v % geo.q)
+        v //= geo.q
+    row[: geo.n] = ((acc % geo.q) == b) & (cells >= 0) & (cells < geo.P)
+    return row
+
+
+def routed_mask_col(s: int, geo: Geometry, prof_cells, types) -> np.ndarray:
+    """Column s of the mask under an explicit assignment."""
+    col = np.zeros(geo.T, dtype=np.uint8)
+    if s >= geo.n:
+        col[s:] = 1
+        return col
+    col[s : geo.n] = 1
+    if geo.dense_G:
+        col[geo.n :] = 1
+        return col
+    cell = int(prof_cells[s])
+    if not 0 <= cell < geo.P:
+        return col
+    x = prof(cell, geo)                     # digits of the cell itself (prof() reduces its argument mod P)
+    dirs = directions(geo.q, geo.D)
+    dots = np.array([sum(ai * xi for ai, xi in zip(a, x)) % geo.q for a in dirs], dtype=np.int64)
+    h = np.asarray(types, dtype=np.int64)
+    ok = (h >= 0) & (h < geo.B)
+    hh = np.where(ok, h, 0)
+    col[geo.n :] = ok & (dots[hh // geo.q] == (hh % geo.q))
+    return col
+
+
+def routed_dense_mask(geo: Geometry, prof_cells, types) -> np.ndarray:
+    return np.stack([routed_mask_row(t, geo, prof_cells, types) for t in range(geo.T)])
+
+
+def positional_assignment(geo: Geometry):
+    """The paper's positional prof / type as explicit arrays (packed cells, types)."""
+    if geo.dense_G:
+        return np.zeros(geo.n, dtype=np.int32), np.zeros(geo.m, dtype=np.int32)
+    cells = (np.arange(geo.n, dtype=np.int64) % geo.P).astype(np.int32)
+    types = np.array([type_index(t, geo) for t in range(geo.n, geo.T)], dtype=np.int32)
+    return cells, types
+
+
+def type_through_cell(geo: Geometry, direction_index: int, cell: int) -> int:
+    """The content-based type of Sec. 3: the hyperplane with direction number `direction_index` that passes through
+    `cell`, i.e. H_{a, aᵀu} for u the digits of the cell."""
+    a = directions(geo.q, geo.D)[direction_index]
+    u = prof(cell, geo)
+    return direction_index * geo.q + sum(ai * ui for ai, ui in zip(a, u)) % geo.q
+
+
+def routed_forward_rows(Q, K, V, geo: Geometry, prof_cells, types, rows):
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64); V = np.asarray(V, dtype=np.float64)
+    out = np.empty((len(rows), V.shape[1]), dtype=np.float64)
+    for k, t in enumerate(rows):
+        out[k] = (routed_mask_row(int(t), geo, prof_cells, types) * (K @ Q[int(t)])) @ V
+    return out
+
+
+def routed_dq_rows(Q, K, V, dO, geo: Geometry, prof_cells, types, rows):
+    K = np.asarray(K, dtype=np.float64); V = np.asarray(V, dtype=np.float64); dO = np.asarray(dO, dtype=np.float64)
+    out = np.empty((len(rows), K.shape[1]), dtype=np.float64)
+    for k, t in enumerate(rows):
+        out[k] = (routed_mask_row(int(t), geo, prof_cells, types) * (V @ dO[int(t)])) @ K
+    return out
+
+
+def routed_dkdv_cols(Q, K, V, dO, geo: Geometry, prof_cells, types, cols):
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64); dO = np.asarray(dO, dtype=np.float64)
+    dK = np.empty((len(cols), K.shape[1]), dtype=np.float64)
+    dV = np.empty((len(cols), V.shape[1]), dtype=np.float64)
+    for k, s in enumerate(cols):
+        mc = routed_mask_col(int(s), geo, prof_cells, types).astype(np.float64)
+        dK[k] = (mc * (dO @ V[int(s)])) @ Q
+        dV[k] = (mc * (Q @ K[int(s)])) @ dO
+    return dK, dV
+
+
 def dense_mask(T: int, c: int, d: int, q: int | None = None) -> np.ndarray:
     """The whole mask as a uint8 [T, T] array, one row at a time."""
     geo = geometry(T, c, d, q)

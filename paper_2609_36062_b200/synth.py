@@ -121,3 +121,23 @@ def as_float64(w: Workload, stored_head: np.ndarray) -> np.ndarray:
 def full_tensor(w: Workload, tensor: str) -> np.ndarray:
     """All heads: shape [batch*heads, T, dim] in storage form."""
     return np.stack([stored(w, tensor, h) for h in range(w.bh)])
+
+
+def hashed_cells(w: Workload, head: int, n: int, P: int, skew: float = 0.0) -> np.ndarray:
+    """A fixed random hash of the distant tokens of one head into P cells (int32 [n]): uniform, or, with skew > 0,
+    drawn from a power law so that a few cells are heavy and many are empty."""
+    g = np.random.Generator(np.random.Philox(key=(int(w.seed) << 40) ^ (7 << 32) ^ int(head)))
+    if skew <= 0:
+        return g.integers(0, P, size=n, dtype=np.int64).astype(np.int32)
+    weights = 1.0 / np.arange(1, P + 1, dtype=np.float64) ** skew
+    perm = g.permutation(P)
+    return perm[g.choice(P, size=n, p=weights / weights.sum())].astype(np.int32)
+
+
+def hashed_query_draws(w: Workload, head: int, m: int, P: int, A: int) -> tuple[np.ndarray, np.ndarray]:
+    """Per recent token of one head: a hashed cell in [0, P) and a direction number in [0, A) (both int32 [m]); the
+    type that goes with them (the hyperplane of that direction through that cell) is the method's arithmetic and is
+    computed by whoever uses the draws."""
+    g = np.random.Generator(np.random.Philox(key=(int(w.seed) << 40) ^ (8 << 32) ^ int(head)))
+    return (g.integers(0, P, size=m, dtype=np.int64).astype(np.int32),
+            g.integers(0, A, size=m, dtype=np.int64).astype(np.int32))
