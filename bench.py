@@ -33,7 +33,7 @@ import numpy as np  # noqa: E402
 from paper_2609_36062_b200 import replicas, roofline, synth  # noqa: E402
 
 DEFAULT_WORKLOAD = "t16k_d4"
-SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd"]
+SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd", "t16k_d4_hashed"]
 METRIC = "SMat prefill tokens/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant stage per step — the tabulation, one
 # launch of radon_tc_kernel — from an ncu capture of the 8-head copy of the workload (351.3 MB read + 530.1 MB
@@ -123,7 +123,7 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------ helpers
 def workload_config(w: synth.Workload, n_gpus: int):
     return {"workload": w.name, "d": w.d, "batch": w.batch, "heads": w.heads, "T": w.T, "d_k": w.d_k, "d_v": w.d_v,
-            "chunk": w.chunk, "pass": "fwd+bwd (backward reuses the forward's profile/type tables left in the shared workspace)"
+            "chunk": w.chunk, "routing": w.routing, "pass": "fwd+bwd (backward reuses the forward's profile/type tables left in the shared workspace)"
             if w.backward else "fwd", "input_dtype": w.dtype,
             "replicas": n_gpus, "l2": "inputs and tables exceed the 126 MB L2; no flush"}
 
@@ -210,6 +210,12 @@ class Runner:
         self.ws = self.plan.workspace(for_backward=w.backward)
         if w.backward:
             self.dQ, self.dK, self.dV = (torch.empty_like(self.dev[x]) for x in ("q", "k", "v"))
+        self.routing = {}
+        if w.routing == "hashed":   # user-supplied routing: int32 cell / type of every token, resident on the device
+            g = self.plan.geometry()
+            prof = np.stack([synth.hashed_cells(w, h, g.n, g.P) for h in range(w.bh)])
+            typ = np.stack([synth.hashed_types(w, h, g.m, g.B) for h in range(w.bh)])
+            self.routing = {"prof": torch.from_numpy(prof).cuda(), "type": torch.from_numpy(typ).cuda()}
         self.host_out = {"o": torch.empty_like(self.host["v"]).pin_memory()}
         if w.backward:
             for nm, src in (("dq", "q"), ("dk", "k"), ("dv", "v")):
@@ -218,10 +224,10 @@ class Runner:
 
     def step(self):
         d = self.dev
-        self.plan.forward(d["q"], d["k"], d["v"], self.O, self.ws)
+        self.plan.forward(d["q"], d["k"], d["v"], self.O, self.ws, **self.routing)
         n = self.plan.last_launch_count()
         if self.w.backward:
-            self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws)
+            self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws, **self.routing)
             n += self.plan.last_launch_count()
         return n
 
@@ -256,9 +262,10 @@ class Runner:
                 if i >= 2:
                     s_cmp.wait_event(ev_out[b])     # the results of step i-2 have left these buffers
                 d, o = dev[b], outs[b]
-                self.plan.forward(d["q"], d["k"], d["v"], o["o"], self.ws, stream=s_cmp)
+                self.plan.forward(d["q"], d["k"], d["v"], o["o"], self.ws, stream=s_cmp, **self.routing)
                 if w.backward:
-                    self.plan.backward(d["q"], d["k"], d["v"], d["do"], o["dq"], o["dk"], o["dv"], self.ws, stream=s_cmp)
+                    self.plan.backward(d["q"], d["k"], d["v"], d["do"], o["dq"], o["dk"], o["dv"], self.ws, stream=s_cmp,
+                                       **self.routing)
                 ev_cmp[b].record(s_cmp)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_cmp[b])
@@ -336,10 +343,10 @@ class Runner:
         acc, order = {}, []
         for _ in range(steps):
             d = self.dev
-            self.plan.forward(d["q"], d["k"], d["v"], self.O, self.ws)
+            self.plan.forward(d["q"], d["k"], d["v"], self.O, self.ws, **self.routing)
             recs = self.plan.profile_read()
             if self.w.backward:
-                self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws)
+                self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws, **self.routing)
                 recs += [(n if n.startswith("bwd_") else "bwd_" + n, t) for n, t in self.plan.profile_read()]
             for n, t in recs:
                 if n not in acc:
@@ -483,7 +490,6 @@ def run_native(args):
     if rank == 0:
         ub, fb = runner.plan.type_table_element_bytes(), runner.plan.profile_table_element_bytes()
         stages = runner.stage_profile(min(steps, 10))
-        sustained = runner.time_sustained(runner.step, per_step, local)   # last: it heats the board
         line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warm,
             "ms_per_step": 1e3 * per_step, "ms_per_step_median": 1e3 * float(np.median(each)),
@@ -497,8 +503,6 @@ def run_native(args):
             "roofline": dominant_kernel_report(w, g, stages, peaks, ub, fb),
             "path_roofline": path_report(w, g, per_step, peaks, ub, fb),
             "tables": {"profile_states_P": g.P, "cached_subset_states_B": g.B, "nnzC": g.nnzC, "q": g.q},
-            "sustained": dict(sustained, value=world * w.tokens * sustained["steps"] / sustained["seconds"],
-                              unit="tokens/s"),
             "fadd_rates_adds_per_s": peaks.get("fadd_rates"),
         }
     del runner
@@ -528,6 +532,12 @@ def run_native(args):
             torch.cuda.empty_cache()
         line["sweep"] = sweep
         line["decode"] = decode_report(torch, binding, peaks)
+        # last, because it heats the board: the headline workload back to back for more than a second
+        r = Runner(w, torch, binding, args.flags)
+        sus = r.time_sustained(r.step, per_step, local)
+        line["sustained"] = dict(sus, value=w.tokens * sus["steps"] / sus["seconds"], unit="tokens/s")
+        del r
+        torch.cuda.empty_cache()
 
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:

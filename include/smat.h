@@ -144,6 +144,27 @@ smat_status smat_backward(const smat_plan* plan, const void* Q, const void* K, c
                           void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The same two passes under USER-SUPPLIED ROUTING (Sec. 3, "construction of G", the content-based assignment: any map
+ * of distant tokens to profile cells and of recent tokens to types gives G_ij = C[type(i), prof(j)], Eq. "Gdef" with
+ * the incidence matrix of Eq. "C"; the positional assignment is the special case smat_routing_indices returns).
+ *   prof [batch*heads, n]  DEVICE int32: the packed cell index in [0, P) of distant token t of every (batch, head)
+ *                          (little-endian base-q digits, as smat_routing_indices packs them)
+ *   type [batch*heads, m]  DEVICE int32: the type h = dir*q + b in [0, B) of recent token n + i
+ * Both are read once per call: a stable counting sort turns them into per-cell and per-type token lists in the
+ * workspace, and pooling (step 2), the typed read (step 4) and their adjoints walk those lists — a data-dependent
+ * gather — instead of the positional strides; tabulation and the causal branch are unchanged.  An entry outside its
+ * range puts the token in no group (it writes to, or reads from, no cached state).  Group sizes may be arbitrarily
+ * skewed, including empty groups.  d = 1 ignores both arrays (one cell, one type).  Everything else — workspace
+ * size, dtypes, errors — is as for smat_forward / smat_backward; SMAT_ERR_UNSUPPORTED if P or B exceeds 56000.
+ */
+smat_status smat_forward_routed(const smat_plan* plan, const void* Q, const void* K, const void* V, void* O,
+                                const int32_t* prof, const int32_t* type, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream);
+smat_status smat_backward_routed(const smat_plan* plan, const void* Q, const void* K, const void* V, const void* dO,
+                                 void* dQ, void* dK, void* dV, const int32_t* prof, const int32_t* type,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Routing as the library's index code sees it (HOST output buffers, caller-allocated):
  *   prof    [n * (d-1)]  base-q digits of (t mod P), least significant first      (Sec. 3, positional assignment)
  *   type    [m]          (t - n + 1) mod B for t = n .. T-1

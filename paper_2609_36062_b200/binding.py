@@ -29,6 +29,7 @@ EXPORTS = [
     "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
     "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step",
     "smat_static_check_status", "smat_debug_timeout_probe", "smat_measure_fadd_rate",
+    "smat_forward_routed", "smat_backward_routed",
 ]
 
 
@@ -83,6 +84,10 @@ def load_library() -> ctypes.CDLL:
     lib.smat_forward.restype = i
     lib.smat_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.smat_backward.restype = i
+    lib.smat_forward_routed.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.smat_forward_routed.restype = i
+    lib.smat_backward_routed.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.smat_backward_routed.restype = i
     lib.smat_routing_indices.argtypes = [vp, vp, vp, vp]
     lib.smat_routing_indices.restype = i
     lib.smat_debug_mask.argtypes = [vp, vp, vp]
@@ -252,18 +257,31 @@ class SmatPlan:
             raise ValueError(f"{name}: expected contiguous {self.torch_dtype} of shape {(b, h, T, last)}, "
                              f"got {t.dtype} {tuple(t.shape)}")
 
-    def forward(self, Q, K, V, O=None, workspace=None, stream=None):
+    def _check_routing(self, prof, typ):
+        b, h, _, _, _ = self.shape
+        g = self.geometry()
+        for name, t, count in (("prof", prof, g.n), ("type", typ, g.m)):
+            if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous() and tuple(t.shape) == (b * h, count)):
+                raise ValueError(f"{name}: expected a contiguous CUDA int32 tensor of shape {(b * h, count)}")
+
+    def forward(self, Q, K, V, O=None, workspace=None, stream=None, prof=None, type=None):
+        """smat_forward, or smat_forward_routed when prof [batch*heads, n] and type [batch*heads, m] are given."""
         _, _, _, dk, dv = self.shape
         self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
         if O is None:
             O = torch.empty_like(V)
         self._check_tensor(O, dv, "O")
         ws = self.workspace(False, Q.device) if workspace is None else workspace
+        if prof is not None or type is not None:
+            self._check_routing(prof, type)
+            _check(self.lib.smat_forward_routed(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(prof), _ptr(type),
+                                                _ptr(ws), ws.numel(), _stream(stream)), "smat_forward_routed")
+            return O
         _check(self.lib.smat_forward(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(ws), ws.numel(),
                                      _stream(stream)), "smat_forward")
         return O
 
-    def backward(self, Q, K, V, dO, dQ=None, dK=None, dV=None, workspace=None, stream=None):
+    def backward(self, Q, K, V, dO, dQ=None, dK=None, dV=None, workspace=None, stream=None, prof=None, type=None):
         _, _, _, dk, dv = self.shape
         self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
         self._check_tensor(dO, dv, "dO")
@@ -271,6 +289,12 @@ class SmatPlan:
         dK = torch.empty_like(K) if dK is None else dK
         dV = torch.empty_like(V) if dV is None else dV
         ws = self.workspace(True, Q.device) if workspace is None else workspace
+        if prof is not None or type is not None:
+            self._check_routing(prof, type)
+            _check(self.lib.smat_backward_routed(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(dQ), _ptr(dK),
+                                                 _ptr(dV), _ptr(prof), _ptr(type), _ptr(ws), ws.numel(), _stream(stream)),
+                   "smat_backward_routed")
+            return dQ, dK, dV
         _check(self.lib.smat_backward(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(dQ), _ptr(dK), _ptr(dV),
                                       _ptr(ws), ws.numel(), _stream(stream)), "smat_backward")
         return dQ, dK, dV

@@ -22,6 +22,7 @@ struct smat_plan {
   // workspace layout (byte offsets, 256-byte aligned)
   size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_W, off_fwd_end;
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
+  size_t off_plist, off_poffs, off_tlist, off_toffs;   // token lists of user-supplied routing (int32)
   bool tc;             // tensor-core kernels for the causal branch
   bool u_bf16;         // forward keeps the type table U in bf16 and reads it with the tensor-core typed read
   bool pool_tc;        // forward pools the profile table on the tensor cores (enough tokens per profile)
@@ -113,8 +114,12 @@ SmatOperand operand(const void* ptr, int bf16, int64_t s_bh, int64_t s_g, int64_
 SmatGroupSpec group(const smat_plan* pl, int mode) {
   SmatGroupSpec s; s.mode = mode; s.n = pl->geo.n; s.T = pl->T; s.c = pl->c;
   s.period = mode == SMAT_GM_PROFILE ? pl->geo.P : pl->geo.B;
+  s.list = nullptr; s.offs = nullptr; s.list_stride = 0; s.offs_stride = 0;
   return s;
 }
+
+struct Ctx;
+SmatGroupSpec group(const Ctx& cx, int mode);
 
 struct Ctx {
   const smat_plan* pl;
@@ -122,8 +127,24 @@ struct Ctx {
   char* ws;
   cudaError_t err;
   int launches;
+  bool routed = false;   // profile / type groups come from the token lists in the workspace, not from positions
+  const int32_t* prof = nullptr;   // the caller's arrays of a routed call
+  const int32_t* type = nullptr;
   float* f(size_t off) const { return reinterpret_cast<float*>(ws + off); }
 };
+
+SmatGroupSpec group(const Ctx& cx, int mode) {
+  const smat_plan* pl = cx.pl;
+  SmatGroupSpec s = group(pl, mode);
+  if (cx.routed && mode != SMAT_GM_CHUNK) {
+    const bool prof = mode == SMAT_GM_PROFILE;
+    s.list = reinterpret_cast<const int32_t*>(cx.ws + (prof ? pl->off_plist : pl->off_tlist));
+    s.offs = reinterpret_cast<const int32_t*>(cx.ws + (prof ? pl->off_poffs : pl->off_toffs));
+    s.list_stride = prof ? pl->geo.n : pl->geo.m;
+    s.offs_stride = (prof ? pl->geo.P : pl->geo.B) + 1;
+  }
+  return s;
+}
 
 void mark_stage(const smat_plan* pl, cudaStream_t st, const char* name) {
   if (!pl->profiling || pl->stages >= SMAT_MAX_STAGES) return;
@@ -146,8 +167,9 @@ void end_stage(const smat_plan* pl, cudaStream_t st) {
     }                                               \
   } while (0)
 
-int64_t max_group_tokens(const smat_plan* pl, int mode) {
+int64_t max_group_tokens(const smat_plan* pl, int mode, bool routed = false) {
   const SmatGeo& g = pl->geo;
+  if (routed && mode != SMAT_GM_CHUNK) return mode == SMAT_GM_PROFILE ? g.n : g.m;  // data-dependent: any size
   if (mode == SMAT_GM_CHUNK) return pl->c;
   if (mode == SMAT_GM_PROFILE) return (g.n + g.P - 1) / g.P;
   return (g.m + g.B - 1) / g.B;
@@ -162,7 +184,7 @@ void outer_sum(Ctx& cx, const char* name, int mode, const void* a, const void* b
   const smat_plan* pl = cx.pl;
   const int bf = pl->dtype == SMAT_BF16;
   const int64_t G = group_count(pl, mode);
-  SMAT_TRY(cx, name, smat_launch_pool(a, b, bf, state, group(pl, mode), pl->T, G, pl->bh, pl->r, pl->p, cx.st));
+  SMAT_TRY(cx, name, smat_launch_pool(a, b, bf, state, group(cx, mode), pl->T, G, pl->bh, pl->r, pl->p, cx.st));
 }
 
 // out[bh][t] (+)= x_t · state_g(t)  (transposed = 0: x: [T, r] contracts the first state index, out: [T, p];
@@ -175,7 +197,7 @@ void state_read(Ctx& cx, const char* name, int mode, const void* x, const float*
   const int64_t G = group_count(pl, mode);
   const int kdim = transposed ? pl->p : pl->r, odim = transposed ? pl->r : pl->p;
   if (mode != SMAT_GM_CHUNK && !out_final) {  // a handful of tokens per state: stream the state once
-    SMAT_TRY(cx, name, smat_launch_state_read(x, bf, state, transposed, acc_in, acc_out, group(pl, mode), pl->T, G,
+    SMAT_TRY(cx, name, smat_launch_state_read(x, bf, state, transposed, acc_in, acc_out, group(cx, mode), pl->T, G,
                                               pl->bh, pl->r, pl->p, reinterpret_cast<int*>(cx.ws + pl->off_status),
                                               cx.st));
     return;
@@ -186,7 +208,7 @@ void state_read(Ctx& cx, const char* name, int mode, const void* x, const float*
   g.Cin = operand(acc_in, 0, pl->T * odim, 0, odim, 1, 1, 0);
   g.C = out_final ? operand(out_final, bf, pl->T * odim, 0, odim, 1, 1, 0)
                   : operand(acc_out, 0, pl->T * odim, 0, odim, 1, 1, 0);
-  g.K = kdim; g.N = odim; g.tokM = 1; g.grp = group(pl, mode);
+  g.K = kdim; g.N = odim; g.tokM = 1; g.grp = group(cx, mode);
   SMAT_TRY(cx, name, smat_launch_gemm(g, (int)max_group_tokens(pl, mode), odim, G, pl->bh, cx.st));
 }
 
@@ -284,8 +306,8 @@ size_t build_type_table(Ctx& cx, const void* K, const void* V) {
   if (pl->tc) {
     int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
     if (pl->pool_tc)
-      SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, group(pl, SMAT_GM_PROFILE),
-                                                  pl->geo.P, max_group_tokens(pl, SMAT_GM_PROFILE), pl->T, pl->bh,
+      SMAT_TRY(cx, "pool_tc", smat_launch_pool_tc(K, V, cx.ws + pl->off_F, pl->f_bf16, group(cx, SMAT_GM_PROFILE),
+                                                  pl->geo.P, max_group_tokens(pl, SMAT_GM_PROFILE, cx.routed), pl->T, pl->bh,
                                                   status, cx.st, pl->tab_d3_regs ? 1 : 0));
     else
       outer_sum(cx, "pool", SMAT_GM_PROFILE, K, V, cx.f(pl->off_F));
@@ -373,6 +395,11 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->off_acc = off;    off = align_up(off + (size_t)pl->bh * T * wide * sizeof(float));
   pl->off_tileA = off;  off = align_up(off + tiles);
   pl->off_W = off;      off = align_up(off + (pl->tab_tc ? (size_t)smat_tabulate_tc_scratch_elems(g, pl->rp, pl->bh) * 2 : 0));
+  const bool lists = !g.dense_G;
+  pl->off_plist = off;  off = align_up(off + (lists ? (size_t)pl->bh * g.n * 4 : 0));
+  pl->off_poffs = off;  off = align_up(off + (lists ? (size_t)pl->bh * (g.P + 1) * 4 : 0));
+  pl->off_tlist = off;  off = align_up(off + (lists ? (size_t)pl->bh * g.m * 4 : 0));
+  pl->off_toffs = off;  off = align_up(off + (lists ? (size_t)pl->bh * (g.B + 1) * 4 : 0));
   pl->off_fwd_end = off;
   pl->off_dbar = off;   off = align_up(off + causal);
   pl->off_ubar = off;   off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.B * entries * (pl->ubar_bf16 ? 2 : 4)));
@@ -436,8 +463,40 @@ size_t smat_workspace_bytes(const smat_plan* pl, int for_backward) {
   return for_backward ? pl->off_bwd_end : pl->off_fwd_end;
 }
 
-smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, const void* V, void* O, void* workspace,
-                         size_t workspace_bytes, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+// Builds the token lists of a routed call in the workspace (or does nothing for a positional call).
+smat_status begin_routing(Ctx& cx, const int32_t* prof, const int32_t* type) {
+  const smat_plan* pl = cx.pl;
+  if (!prof && !type) return SMAT_OK;
+  if (!prof || !type) return SMAT_ERR_NULL;
+  if (pl->geo.dense_G) return SMAT_OK;   // d = 1: one cell, one type; there is nothing to route
+  if ((reinterpret_cast<uintptr_t>(prof) | reinterpret_cast<uintptr_t>(type)) & 3) return SMAT_ERR_ALIGN;
+  const int64_t gmax = pl->geo.P > pl->geo.B ? pl->geo.P : pl->geo.B;
+  if (gmax > smat_routing_max_groups()) return SMAT_ERR_UNSUPPORTED;
+  auto i32 = [&](size_t off) { return reinterpret_cast<int32_t*>(cx.ws + off); };
+  SMAT_TRY(cx, "routing_lists", smat_launch_routing_lists(prof, type, i32(pl->off_plist), i32(pl->off_poffs),
+                                                          i32(pl->off_tlist), i32(pl->off_toffs), pl->geo, pl->bh, cx.st));
+  cx.routed = true;
+  cx.prof = prof; cx.type = type;
+  return SMAT_OK;
+}
+
+// Routed calls on the tensor-core path: the rows a routed read does not visit (tokens of no group) must read as zero
+// for the kernel that adds them.
+void zero_unrouted(Ctx& cx, int mode, void* rows, int row_bytes) {
+  if (!cx.routed) return;
+  const smat_plan* pl = cx.pl;
+  const bool prof = mode == SMAT_GM_PROFILE;
+  SMAT_TRY(cx, "zero_unrouted", smat_launch_zero_unrouted(prof ? cx.prof : cx.type, prof ? pl->geo.n : pl->geo.m,
+                                                           prof ? pl->geo.P : pl->geo.B, prof ? 0 : pl->geo.n, rows, pl->T,
+                                                           row_bytes, pl->bh, cx.st));
+}
+
+smat_status forward_impl(const smat_plan* pl, const void* Q, const void* K, const void* V, void* O, const int32_t* prof,
+                         const int32_t* type, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!Q || !K || !V || !O) return SMAT_ERR_NULL;
   smat_status s = check_common(pl, workspace, workspace_bytes, 0);
   if (s != SMAT_OK) return s;
@@ -446,6 +505,8 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  s = begin_routing(cx, prof, type);
+  if (s != SMAT_OK) return s;
   if (pl->tc) {
     int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
     float* ylr = cx.f(pl->off_acc);
@@ -456,9 +517,10 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
     const int64_t tiles0 = lr ? pl->geo.n / 128 : pl->T / 128, tiles1 = lr ? pl->geo.m / 128 : 0;
     const int L = ((pl->flags & SMAT_FLAG_PER_TILE_STATES) || (lr && !pl->u_bf16)) ? 1 : smat_segment_tiles(tiles0, tiles1, pl->bh);
     if (lr) {                                                                                // step 4
+      zero_unrouted(cx, SMAT_GM_TYPE, ylr, L >= 2 && pl->u_bf16 ? 256 : 512);
       if (pl->u_bf16)
         SMAT_TRY(cx, "read_type_tc", smat_launch_state_read_tc(Q, cx.ws + pl->off_U, ylr, L >= 2 ? ylr : nullptr, 0,
-                                                               group(pl, SMAT_GM_TYPE), pl->geo.B, pl->T, pl->bh, status,
+                                                               group(cx, SMAT_GM_TYPE), pl->geo.B, pl->T, pl->bh, status,
                                                                cx.st));
       else
         state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);
@@ -495,8 +557,9 @@ smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, cons
   return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
 }
 
-smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, const void* V, const void* dO, void* dQ,
-                          void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+smat_status backward_impl(const smat_plan* pl, const void* Q, const void* K, const void* V, const void* dO, void* dQ,
+                          void* dK, void* dV, const int32_t* prof, const int32_t* type, void* workspace,
+                          size_t workspace_bytes, void* cuda_stream) {
   if (!Q || !K || !V || !dO || !dQ || !dK || !dV) return SMAT_ERR_NULL;
   smat_status s = check_common(pl, workspace, workspace_bytes, 1);
   if (s != SMAT_OK) return s;
@@ -507,6 +570,8 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
   cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  s = begin_routing(cx, prof, type);
+  if (s != SMAT_OK) return s;
   const bool lr = !pl->geo.dense_G;
   if (pl->tc) {
     // Tensor-core backward.  Forward tables are rebuilt as in smat_forward (U in bf16 where the plan keeps it so);
@@ -515,7 +580,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
     int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
     float* lrbuf = cx.f(pl->off_acc);
     pl->tile_states = true;
-    const SmatGroupSpec types = group(pl, SMAT_GM_TYPE), profs = group(pl, SMAT_GM_PROFILE);
+    const SmatGroupSpec types = group(cx, SMAT_GM_TYPE), profs = group(cx, SMAT_GM_PROFILE);
     const int64_t n = pl->geo.n;
     if (lr) {
       if (!(pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES)) build_type_table(cx, K, V);
@@ -523,7 +588,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
       const bool ubar_tc = pl->ubar_tc, ubar_bf16 = pl->ubar_bf16;
       if (ubar_tc)
         SMAT_TRY(cx, "bwd_pool_type_tc", smat_launch_pool_tc(Q, dO, cx.ws + pl->off_ubar, ubar_bf16, types, pl->geo.B,
-                                                             max_group_tokens(pl, SMAT_GM_TYPE), pl->T, pl->bh,
+                                                             max_group_tokens(pl, SMAT_GM_TYPE, cx.routed), pl->T, pl->bh,
                                                              status, cx.st));
       else
         outer_sum(cx, "bwd_pool_type", SMAT_GM_TYPE, Q, dO, cx.f(pl->off_ubar));
@@ -536,6 +601,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
       SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 0, 0, status, cx.st));
       SMAT_TRY(cx, "bwd_suffix_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 0, 1, status, cx.st));
       // dQ: recent rows add U_type dO
+      zero_unrouted(cx, SMAT_GM_TYPE, lrbuf, 512);
       if (pl->u_bf16)
         SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, lrbuf, nullptr, 1, types, pl->geo.B,
                                                                  pl->T, pl->bh, status, cx.st));
@@ -544,6 +610,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
       SMAT_TRY(cx, "bwd_dq_tile_tc", smat_launch_chunk_adjoint_tc(0, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
                                                                   lrbuf, n, pl->T, dQ, pl->T, pl->bh, status, cx.st));
       // dK: distant rows add F̄_prof v
+      zero_unrouted(cx, SMAT_GM_PROFILE, lrbuf, 512);
       if (fbar_is_bf16)
         SMAT_TRY(cx, "bwd_dk_profile_tc", smat_launch_state_read_tc(V, cx.ws + pl->off_fbar, lrbuf, nullptr, 1, profs, pl->geo.P,
                                                                     pl->T, pl->bh, status, cx.st));
@@ -552,6 +619,7 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
       SMAT_TRY(cx, "bwd_dk_tile_tc", smat_launch_chunk_adjoint_tc(1, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
                                                                   lrbuf, 0, n, dK, pl->T, pl->bh, status, cx.st));
       // dV: distant rows add F̄_profᵀ k
+      zero_unrouted(cx, SMAT_GM_PROFILE, lrbuf, 512);
       if (fbar_is_bf16)
         SMAT_TRY(cx, "bwd_dv_profile_tc", smat_launch_state_read_tc(K, cx.ws + pl->off_fbar, lrbuf, nullptr, 0, profs, pl->geo.P,
                                                                     pl->T, pl->bh, status, cx.st));
@@ -600,6 +668,34 @@ smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, con
   state_read(cx, "bwd_dv_chunk", SMAT_GM_CHUNK, K, dbar, 0, acc, nullptr, dV);
   pl->launches = cx.launches;
   return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
+}  // namespace
+
+extern "C" {
+
+smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, const void* V, void* O, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  return forward_impl(pl, Q, K, V, O, nullptr, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+smat_status smat_backward(const smat_plan* pl, const void* Q, const void* K, const void* V, const void* dO, void* dQ,
+                          void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return backward_impl(pl, Q, K, V, dO, dQ, dK, dV, nullptr, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+smat_status smat_forward_routed(const smat_plan* pl, const void* Q, const void* K, const void* V, void* O,
+                                const int32_t* prof, const int32_t* type, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream) {
+  if (!prof || !type) return SMAT_ERR_NULL;
+  return forward_impl(pl, Q, K, V, O, prof, type, workspace, workspace_bytes, cuda_stream);
+}
+
+smat_status smat_backward_routed(const smat_plan* pl, const void* Q, const void* K, const void* V, const void* dO,
+                                 void* dQ, void* dK, void* dV, const int32_t* prof, const int32_t* type, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+  if (!prof || !type) return SMAT_ERR_NULL;
+  return backward_impl(pl, Q, K, V, dO, dQ, dK, dV, prof, type, workspace, workspace_bytes, cuda_stream);
 }
 
 smat_status smat_routing_indices(const smat_plan* pl, int32_t* prof, int32_t* type, int32_t* type_ab) {

@@ -16,25 +16,47 @@ enum SmatGroupMode { SMAT_GM_NONE = 0, SMAT_GM_CHUNK = 1, SMAT_GM_PROFILE = 2, S
 struct SmatGroupSpec {
   int mode;
   int64_t n, T, c, period;  // period = P (PROFILE) or B (TYPE)
+  // User-supplied routing (content-based assignment, Sec. 3): when `list` is non-null the tokens of PROFILE / TYPE
+  // group g of head bh are list[bh * list_stride + offs[bh * offs_stride + g] ...  offs[... + g + 1]) (token positions
+  // in [0, T), ascending inside a group) instead of the positional strides.
+  const int32_t* list;
+  const int32_t* offs;
+  int64_t list_stride, offs_stride;
 };
 
-SMAT_HD void smat_group_tokens(const SmatGroupSpec& s, int64_t g, int64_t* t0, int64_t* ts, int64_t* cnt) {
+// The tokens of one group: position of the k-th one is at(k).
+struct SmatTokens {
+  int64_t t0, ts, cnt;
+  const int32_t* lst;
+  SMAT_HD int64_t at(int64_t k) const { return lst ? (int64_t)lst[k] : t0 + k * ts; }
+};
+
+SMAT_HD SmatTokens smat_group_tokens(const SmatGroupSpec& s, int64_t bh, int64_t g) {
+  SmatTokens r;
+  r.lst = nullptr; r.t0 = 0; r.ts = 1; r.cnt = 0;
+  if (s.mode != SMAT_GM_CHUNK && s.list) {
+    const int32_t* o = s.offs + bh * s.offs_stride + g;
+    r.lst = s.list + bh * s.list_stride + o[0];
+    r.cnt = o[1] - o[0];
+    return r;
+  }
   switch (s.mode) {
     case SMAT_GM_CHUNK:
-      *t0 = g * s.c; *ts = 1; *cnt = s.c;
+      r.t0 = g * s.c; r.ts = 1; r.cnt = s.c;
       break;
     case SMAT_GM_PROFILE:
-      *t0 = g; *ts = s.period; *cnt = g < s.n ? (s.n - g + s.period - 1) / s.period : 0;
+      r.t0 = g; r.ts = s.period; r.cnt = g < s.n ? (s.n - g + s.period - 1) / s.period : 0;
       break;
     case SMAT_GM_TYPE: {
       int64_t i0 = g ? g : s.period;  // paper's 1-based recent index of the first token of this type
       int64_t m = s.T - s.n;
-      *t0 = s.n + i0 - 1; *ts = s.period; *cnt = i0 <= m ? (m - i0) / s.period + 1 : 0;
+      r.t0 = s.n + i0 - 1; r.ts = s.period; r.cnt = i0 <= m ? (m - i0) / s.period + 1 : 0;
       break;
     }
     default:
-      *t0 = 0; *ts = 1; *cnt = 0;
+      break;
   }
+  return r;
 }
 
 // ---- generic batched small GEMM on the fp32 ALUs ---------------------------------------------------
@@ -139,6 +161,15 @@ cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_b
 // bf16 table kept slab-major [bh][rp / 32][rows][32] -> fp32 [bh][rows][rp] (debug export).
 cudaError_t smat_launch_widen_bf16_slabs(const void* src_bf16, float* dst, int64_t heads, int64_t rows, int64_t rp,
                                          cudaStream_t st);
+// Token lists of user-supplied routing: prof [bh][n] (cells in [0, P)) and type [bh][m] (types in [0, B)) -> CSR lists
+// (offsets [bh][G + 1], token positions [bh][count], ascending inside a group).  Keys out of range are dropped.
+int64_t smat_routing_max_groups();
+cudaError_t smat_launch_routing_lists(const int32_t* prof, const int32_t* type, int32_t* prof_list, int32_t* prof_offs,
+                                      int32_t* type_list, int32_t* type_offs, const SmatGeo& geo, int bh,
+                                      cudaStream_t st);
+// Zeroes the row (row_bytes bytes at rows + (bh*T + first + i) * row_bytes) of every token i whose key lies outside [0, G).
+cudaError_t smat_launch_zero_unrouted(const int32_t* key, int64_t count, int64_t G, int64_t first, void* rows, int64_t T,
+                                      int row_bytes, int bh, cudaStream_t st);
 // Two-level causal branch: segment totals, then (after an exclusive scan of the totals) per-segment fused output.
 int smat_segment_tiles(int64_t tiles_block0, int64_t tiles_block1, int bh);
 void smat_segment_counts(int64_t tiles0, int64_t tiles1, int bh, int L, int* nseg0, int* nseg1);

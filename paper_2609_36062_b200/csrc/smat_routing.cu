@@ -1,0 +1,130 @@
+// User-supplied routing (Sec. 3, "construction of G": the content-based assignment): the caller gives every distant
+// token its profile cell and every recent token its type as integer arrays; this file turns them into the per-group
+// token lists (CSR: offsets + token positions, ascending inside a group) that the pooling and routed-read kernels
+// walk instead of the positional strides.  Integer work only: a counting sort per (head, kind), stable so that the
+// order of the floating-point sums downstream does not depend on thread timing.
+#include <cuda_runtime.h>
+
+#include "smat_internal.h"
+
+namespace {
+
+constexpr int ROUTE_THREADS = 256;
+
+// One CTA per (head, kind); kind 0: profiles of the n distant tokens, kind 1: types of the m recent tokens.
+//   1. histogram of the keys in shared memory (keys outside [0, G) are dropped: such a token belongs to no group)
+//   2. exclusive scan -> offs[0 .. G]
+//   3. stable placement by ONE warp walking the tokens in order, 32 at a time: lanes with equal keys find each other
+//      with match.any, the lowest such lane advances the group's cursor, every lane writes its token's position
+struct RouteParams {
+  const int32_t* key[2];   // [bh][count]
+  int32_t* list[2];        // [bh][count]
+  int32_t* offs[2];        // [bh][G + 1]
+  int64_t count[2], G[2], first[2];   // tokens per head, groups, position of the first token of the kind
+};
+
+__global__ void __launch_bounds__(ROUTE_THREADS) routing_lists_kernel(const RouteParams prm) {
+  extern __shared__ int32_t cursor[];   // [G + 1]
+  const int kind = blockIdx.y;
+  const int64_t bh = blockIdx.x, n = prm.count[kind], G = prm.G[kind];
+  const int32_t* key = prm.key[kind] + bh * n;
+  int32_t* list = prm.list[kind] + bh * n;
+  int32_t* offs = prm.offs[kind] + bh * (G + 1);
+  const int tid = threadIdx.x;
+  for (int64_t g = tid; g <= G; g += ROUTE_THREADS) cursor[g] = 0;
+  __syncthreads();
+  for (int64_t t = tid; t < n; t += ROUTE_THREADS) {
+    const int32_t k = key[t];
+    if (k >= 0 && k < G) atomicAdd(&cursor[k + 1], 1);
+  }
+  __syncthreads();
+  // exclusive scan of cursor[1 .. G] in place (cursor[g] = first slot of group g), chunk by chunk with a carry
+  __shared__ int32_t warp_sum[ROUTE_THREADS / 32];
+  __shared__ int32_t carry;
+  if (tid == 0) carry = 0;
+  __syncthreads();
+  for (int64_t base = 1; base <= G; base += ROUTE_THREADS) {
+    const int64_t g = base + tid;
+    const int32_t v = g <= G ? cursor[g] : 0;
+    int32_t x = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int32_t y = __shfl_up_sync(0xffffffffu, x, d);
+      if ((tid & 31) >= d) x += y;
+    }
+    if ((tid & 31) == 31) warp_sum[tid >> 5] = x;
+    __syncthreads();
+    int32_t before = carry;
+    for (int w = 0; w < (tid >> 5); ++w) before += warp_sum[w];
+    if (g <= G) cursor[g] = before + x;   // inclusive: end of group g - 1 ... stored at index g
+    __syncthreads();
+    if (tid == ROUTE_THREADS - 1) carry = before + x;
+    __syncthreads();
+  }
+  // cursor[g] (g >= 1) now holds the number of tokens in groups < g; cursor[0] = 0
+  for (int64_t g = tid; g <= G; g += ROUTE_THREADS) offs[g] = cursor[g];
+  __syncthreads();
+  if (tid < 32) {
+    const int64_t first = prm.first[kind];
+    for (int64_t t0 = 0; t0 < n; t0 += 32) {
+      const int64_t t = t0 + tid;
+      const int32_t k = t < n ? key[t] : -1;
+      const bool valid = k >= 0 && k < G;
+      const unsigned peers = __match_any_sync(0xffffffffu, valid ? k : -1 - tid);
+      int32_t slot = 0;
+      if (valid) {
+        const int leader = __ffs(peers) - 1;
+        if (tid == leader) {
+          slot = cursor[k];
+          cursor[k] = slot + __popc(peers);
+        }
+        slot = __shfl_sync(peers, slot, leader) + __popc(peers & ((1u << tid) - 1));
+        list[slot] = (int32_t)(first + t);
+      }
+      __syncwarp();
+    }
+  }
+}
+
+// Rows of tokens that belong to no group are never written by a routed read; whoever adds those rows afterwards must
+// find zeros there.  One warp per token: zero the row when the token's key is out of range.
+__global__ void zero_unrouted_rows_kernel(const int32_t* __restrict__ key, int64_t count, int64_t G, int64_t first,
+                                          uint8_t* __restrict__ rows, int64_t T, int row_bytes, int64_t total) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (w >= total) return;
+  const int32_t k = key[w];
+  if (k >= 0 && k < G) return;
+  const int64_t bh = w / count, t = first + (w - bh * count);
+  uint4* dst = reinterpret_cast<uint4*>(rows + (bh * T + t) * row_bytes);
+  for (int i = threadIdx.x & 31; i < row_bytes / 16; i += 32) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+}  // namespace
+
+cudaError_t smat_launch_zero_unrouted(const int32_t* key, int64_t count, int64_t G, int64_t first, void* rows, int64_t T,
+                                      int row_bytes, int bh, cudaStream_t st) {
+  const int64_t total = (int64_t)bh * count;
+  const int64_t threads = total * 32;
+  zero_unrouted_rows_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(key, count, G, first,
+                                                                               static_cast<uint8_t*>(rows), T, row_bytes, total);
+  return cudaGetLastError();
+}
+
+// Largest group count the list builder handles (its cursors live in shared memory).
+int64_t smat_routing_max_groups() { return 56000; }
+
+cudaError_t smat_launch_routing_lists(const int32_t* prof, const int32_t* type, int32_t* prof_list, int32_t* prof_offs,
+                                      int32_t* type_list, int32_t* type_offs, const SmatGeo& geo, int bh,
+                                      cudaStream_t st) {
+  RouteParams prm;
+  prm.key[0] = prof; prm.list[0] = prof_list; prm.offs[0] = prof_offs; prm.count[0] = geo.n; prm.G[0] = geo.P; prm.first[0] = 0;
+  prm.key[1] = type; prm.list[1] = type_list; prm.offs[1] = type_offs; prm.count[1] = geo.m; prm.G[1] = geo.B; prm.first[1] = geo.n;
+  const int64_t gmax = geo.P > geo.B ? geo.P : geo.B;
+  if (gmax > smat_routing_max_groups()) return cudaErrorInvalidConfiguration;
+  const size_t smem = (size_t)(gmax + 1) * sizeof(int32_t);
+  cudaError_t err = cudaFuncSetAttribute(routing_lists_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  dim3 grid((unsigned)bh, 2);
+  routing_lists_kernel<<<grid, ROUTE_THREADS, smem, st>>>(prm);
+  return cudaGetLastError();
+}

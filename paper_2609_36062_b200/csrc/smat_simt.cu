@@ -19,8 +19,8 @@ __device__ __forceinline__ float load_elem(const SmatOperand& o, int64_t off) {
 __global__ void __launch_bounds__(256) gemm_grouped_kernel(const SmatGemmArgs a) {
   const int64_t g = blockIdx.y;
   const int64_t bh = blockIdx.z;
-  int64_t t0 = 0, ts = 1, cnt = 0;
-  smat_group_tokens(a.grp, g, &t0, &ts, &cnt);
+  const SmatTokens tk = smat_group_tokens(a.grp, bh, g);
+  const int64_t cnt = tk.cnt;
   const int M = a.tokM ? (int)cnt : a.M;
   const int N = a.tokN ? (int)cnt : a.N;
   const int K = a.tokK ? (int)cnt : a.K;
@@ -53,8 +53,8 @@ __global__ void __launch_bounds__(256) gemm_grouped_kernel(const SmatGemmArgs a)
       if (a_k_contig) { kk = e & (KSTEP - 1); mm = e >> 4; } else { mm = e & (TILE - 1); kk = e >> 6; }
       float v = 0.f;
       if (m0 + mm < M && k0 + kk < K) {
-        const int64_t x0 = a.A.tok0 ? t0 + (int64_t)(m0 + mm) * ts : (int64_t)(m0 + mm);
-        const int64_t x1 = a.A.tok1 ? t0 + (int64_t)(k0 + kk) * ts : (int64_t)(k0 + kk);
+        const int64_t x0 = a.A.tok0 ? tk.at(m0 + mm) : (int64_t)(m0 + mm);
+        const int64_t x1 = a.A.tok1 ? tk.at(k0 + kk) : (int64_t)(k0 + kk);
         v = load_elem(a.A, baseA + x0 * a.A.s0 + x1 * a.A.s1);
       }
       As[kk][mm] = v;
@@ -66,8 +66,8 @@ __global__ void __launch_bounds__(256) gemm_grouped_kernel(const SmatGemmArgs a)
       if (b_n_contig) { nn = e & (TILE - 1); kk = e >> 6; } else { kk = e & (KSTEP - 1); nn = e >> 4; }
       float v = 0.f;
       if (n0 + nn < N && k0 + kk < K) {
-        const int64_t x0 = a.B.tok0 ? t0 + (int64_t)(k0 + kk) * ts : (int64_t)(k0 + kk);
-        const int64_t x1 = a.B.tok1 ? t0 + (int64_t)(n0 + nn) * ts : (int64_t)(n0 + nn);
+        const int64_t x0 = a.B.tok0 ? tk.at(k0 + kk) : (int64_t)(k0 + kk);
+        const int64_t x1 = a.B.tok1 ? tk.at(n0 + nn) : (int64_t)(n0 + nn);
         v = load_elem(a.B, baseB + x0 * a.B.s0 + x1 * a.B.s1);
       }
       Bs[kk][nn] = v;
@@ -93,12 +93,12 @@ __global__ void __launch_bounds__(256) gemm_grouped_kernel(const SmatGemmArgs a)
   for (int i = 0; i < 4; ++i) {
     const int m = m0 + ty * 4 + i;
     if (m >= M) continue;
-    const int64_t x0 = a.C.tok0 ? t0 + (int64_t)m * ts : (int64_t)m;
+    const int64_t x0 = a.C.tok0 ? tk.at(m) : (int64_t)m;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tx * 4 + j;
       if (n >= N) continue;
-      const int64_t x1 = a.C.tok1 ? t0 + (int64_t)n * ts : (int64_t)n;
+      const int64_t x1 = a.C.tok1 ? tk.at(n) : (int64_t)n;
       float v = (a.tril && n > m) ? 0.f : acc[i][j];
       if (a.Cin.ptr) v += reinterpret_cast<const float*>(a.Cin.ptr)[baseI + x0 * a.Cin.s0 + x1 * a.Cin.s1];
       const int64_t off = baseC + x0 * a.C.s0 + x1 * a.C.s1;

@@ -74,20 +74,20 @@ __global__ void __launch_bounds__(256) pool_stream_kernel(const T* __restrict__ 
   auto prefetch = [&](int64_t item, int buf) {  // first tile of tokens of an item, raw, through cp.async
     if (item < items) {
       const int64_t bh = item / groups, g = item - bh * groups;
-      int64_t t0, ts, cnt;
-      smat_group_tokens(grp, g, &t0, &ts, &cnt);
+      const SmatTokens tk = smat_group_tokens(grp, bh, g);
+      const int64_t cnt = tk.cnt;
       const int kn = (int)(cnt < TK ? cnt : TK);
       const T* Ab = A + bh * Tlen * R;
       const T* Bb = Bm + bh * Tlen * PD;
       for (int idx = tid; idx < kn * RC; idx += 256) {
         const int k = idx / RC, c = idx - k * RC;
         cp_async16(reinterpret_cast<uint8_t*>(a_raw + (buf * TK + k) * R) + c * 16,
-                   reinterpret_cast<const uint8_t*>(Ab + (t0 + k * ts) * R) + c * 16);
+                   reinterpret_cast<const uint8_t*>(Ab + tk.at(k) * R) + c * 16);
       }
       for (int idx = tid; idx < kn * PC; idx += 256) {
         const int k = idx / PC, c = idx - k * PC;
         cp_async16(reinterpret_cast<uint8_t*>(b_raw + (buf * TK + k) * PD) + c * 16,
-                   reinterpret_cast<const uint8_t*>(Bb + (t0 + k * ts) * PD) + c * 16);
+                   reinterpret_cast<const uint8_t*>(Bb + tk.at(k) * PD) + c * 16);
       }
     }
     cp_async_commit();
@@ -101,8 +101,8 @@ __global__ void __launch_bounds__(256) pool_stream_kernel(const T* __restrict__ 
     cp_async_wait<1>();
     __syncthreads();
     const int64_t bh = item / groups, g = item - bh * groups;
-    int64_t t0, ts, cnt;
-    smat_group_tokens(grp, g, &t0, &ts, &cnt);
+    const SmatTokens tk = smat_group_tokens(grp, bh, g);
+    const int64_t cnt = tk.cnt;
     float4 acc[NS];
 #pragma unroll
     for (int s = 0; s < NS; ++s) acc[s] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -115,12 +115,12 @@ __global__ void __launch_bounds__(256) pool_stream_kernel(const T* __restrict__ 
         for (int idx = tid; idx < kn * RC; idx += 256) {
           const int k = idx / RC, c = idx - k * RC;
           cp_async16(reinterpret_cast<uint8_t*>(a_raw + (buf * TK + k) * R) + c * 16,
-                     reinterpret_cast<const uint8_t*>(Ab + (t0 + (k0 + k) * ts) * R) + c * 16);
+                     reinterpret_cast<const uint8_t*>(Ab + tk.at(k0 + k) * R) + c * 16);
         }
         for (int idx = tid; idx < kn * PC; idx += 256) {
           const int k = idx / PC, c = idx - k * PC;
           cp_async16(reinterpret_cast<uint8_t*>(b_raw + (buf * TK + k) * PD) + c * 16,
-                     reinterpret_cast<const uint8_t*>(Bb + (t0 + (k0 + k) * ts) * PD) + c * 16);
+                     reinterpret_cast<const uint8_t*>(Bb + tk.at(k0 + k) * PD) + c * 16);
         }
         cp_async_commit();
         cp_async_wait<0>();
@@ -180,14 +180,14 @@ __global__ void __launch_bounds__(256, 2) state_read_stream_kernel(const T* __re
   auto prefetch_x = [&](int64_t item, int buf) {
     if (item < items) {
       const int64_t bh = item / groups, g = item - bh * groups;
-      int64_t t0, ts, cnt;
-      smat_group_tokens(grp, g, &t0, &ts, &cnt);
+      const SmatTokens tk = smat_group_tokens(grp, bh, g);
+      const int64_t cnt = tk.cnt;
       const int kn = (int)(cnt < KT ? cnt : KT);
       const T* Xb = X + bh * Tlen * XD;
       for (int idx = tid; idx < kn * XC; idx += 256) {
         const int k = idx / XC, c = idx - k * XC;
         cp_async16(reinterpret_cast<uint8_t*>(Xraw + (buf * KT + k) * XD) + c * 16,
-                   reinterpret_cast<const uint8_t*>(Xb + (t0 + k * ts) * XD) + c * 16);
+                   reinterpret_cast<const uint8_t*>(Xb + tk.at(k) * XD) + c * 16);
       }
     }
     cp_async_commit();
@@ -208,8 +208,8 @@ __global__ void __launch_bounds__(256, 2) state_read_stream_kernel(const T* __re
   for (int64_t item = blockIdx.x; item < items; item += gridDim.x, ++n) {
     const int buf = n & 1;
     const int64_t bh = item / groups, g = item - bh * groups;
-    int64_t t0, ts, cnt;
-    smat_group_tokens(grp, g, &t0, &ts, &cnt);
+    const SmatTokens tk = smat_group_tokens(grp, bh, g);
+    const int64_t cnt = tk.cnt;
     const T* Xb = X + bh * Tlen * XD;
     const float4* S4 = reinterpret_cast<const float4*>(Sb);
     prefetch_x(item + gridDim.x, buf ^ 1);
@@ -221,7 +221,7 @@ __global__ void __launch_bounds__(256, 2) state_read_stream_kernel(const T* __re
       for (int idx = tid; idx < KT * XD; idx += 256) {
         const int k = idx / XD, i = idx % XD;
         float v = 0.f;
-        if (k < kn) v = k0 == 0 ? to_float(Xraw[(buf * KT + k) * XD + i]) : to_float(Xb[(t0 + (k0 + k) * ts) * XD + i]);
+        if (k < kn) v = k0 == 0 ? to_float(Xraw[(buf * KT + k) * XD + i]) : to_float(Xb[tk.at(k0 + k) * XD + i]);
         Xs[idx] = v;
       }
       __syncthreads();
@@ -244,7 +244,7 @@ __global__ void __launch_bounds__(256, 2) state_read_stream_kernel(const T* __re
           float v = 0.f;
 #pragma unroll
           for (int w = 0; w < NG; ++w) v += red[(w * KT + k) * PD + j];
-          const int64_t off = (bh * Tlen + t0 + (k0 + k) * ts) * OD + j;
+          const int64_t off = (bh * Tlen + tk.at(k0 + k)) * OD + j;
           acc_out[off] = v + (acc_in ? acc_in[off] : 0.f);
         }
       } else {
@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(256, 2) state_read_stream_kernel(const T* __re
         __syncthreads();
         for (int idx = tid; idx < kn * R; idx += 256) {
           const int k = idx / R, i = idx % R;
-          const int64_t off = (bh * Tlen + t0 + (k0 + k) * ts) * OD + i;
+          const int64_t off = (bh * Tlen + tk.at(k0 + k)) * OD + i;
           acc_out[off] = red[k * R + i] + (acc_in ? acc_in[off] : 0.f);
         }
       }

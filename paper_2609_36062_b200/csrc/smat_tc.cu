@@ -745,16 +745,19 @@ __device__ __forceinline__ void cp_async16_tc(uint32_t smem_addr, const void* gm
 struct ReadPass {
   const ReadParams* pp;
   int64_t item, stride;
-  int64_t bh, t_first, t_stride, cnt, k0;
+  int64_t bh, cnt, k0;
+  SmatTokens tk;
   __device__ ReadPass(const ReadParams& p, int64_t first, int64_t stride_) : pp(&p), item(first), stride(stride_) { load(); }
   __device__ void load() {
     k0 = 0;
     for (; item < pp->items; item += stride) {
       bh = item / pp->groups;
-      smat_group_tokens(pp->grp, item - bh * pp->groups, &t_first, &t_stride, &cnt);
+      tk = smat_group_tokens(pp->grp, bh, item - bh * pp->groups);
+      cnt = tk.cnt;
       if (cnt > 0) break;
     }
   }
+  __device__ int64_t token(int m) const { return tk.at(k0 + m); }   // position of row m of this pass
   __device__ bool valid() const { return item < pp->items; }
   __device__ bool first() const { return k0 == 0; }
   __device__ bool last() const { return k0 + TILE >= cnt; }
@@ -801,7 +804,7 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
       const int kn = ps.tokens();
       for (int idx = tid; idx < kn * 16; idx += 128) {
         const int m = idx >> 4, gc = idx & 15;
-        const __nv_bfloat16* src = prm.X + ((ps.bh * prm.T + ps.t_first + (ps.k0 + m) * ps.t_stride) * TILE + gc * 8);
+        const __nv_bfloat16* src = prm.X + ((ps.bh * prm.T + ps.token(m)) * TILE + gc * 8);
         cp_async16_tc(a_base + (gc >> 3) * BOX_BYTES + m * 128 + (((gc & 7) ^ (m & 7)) << 4), src);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
@@ -821,7 +824,7 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
       if (nxt.valid()) gather(nxt);                          // the next queries travel while this product is written out
       fence_after_sync();
       const int m = warp * 32 + lane, kn = cur.tokens();
-      const int64_t row = (cur.bh * prm.T + cur.t_first + (cur.k0 + m) * cur.t_stride) * TILE;
+      const int64_t row = (cur.bh * prm.T + (m < kn ? cur.token(m) : 0)) * TILE;
       float4* dst = reinterpret_cast<float4*>(prm.out + row);
       __nv_bfloat16* dst16 = prm.out_bf16 + row;
 #pragma unroll
@@ -925,15 +928,18 @@ template <int TOK>
 struct PoolPass {
   const PoolParams* pp;
   int64_t item, stride;          // current item; items advance by the grid size
-  int64_t bh, t_first, t_stride, cnt, k0;
+  int64_t bh, cnt, k0;
+  SmatTokens tk;
   __device__ PoolPass(const PoolParams& p, int64_t first, int64_t stride_) : pp(&p), item(first), stride(stride_) { load(); }
   __device__ void load() {
     k0 = 0;
     if (item < pp->items) {
       bh = item / pp->groups;
-      smat_group_tokens(pp->grp, item - bh * pp->groups, &t_first, &t_stride, &cnt);
+      tk = smat_group_tokens(pp->grp, bh, item - bh * pp->groups);
+      cnt = tk.cnt;
     }
   }
+  __device__ int64_t token(int k) const { return tk.at(k0 + k); }   // position of row k of this pass
   __device__ bool valid() const { return item < pp->items; }
   __device__ bool first() const { return k0 == 0; }
   __device__ bool last() const { return k0 + TOK >= cnt; }
@@ -988,7 +994,7 @@ __global__ void __launch_bounds__(160) pool_tc_kernel(const PoolParams prm) {
         const int k = idx >> 5, w = idx & 31, gc = w & 15;
         const uint32_t dst = (w < 16 ? a_base : b_base) + (gc >> 3) * (TOK * 128) + k * 128 + (((gc & 7) ^ (k & 7)) << 4);
         if (k < kn) {
-          const __nv_bfloat16* src = (w < 16 ? prm.K : prm.V) + ((ps.bh * prm.T + ps.t_first + (ps.k0 + k) * ps.t_stride) * TILE + gc * 8);
+          const __nv_bfloat16* src = (w < 16 ? prm.K : prm.V) + ((ps.bh * prm.T + ps.token(k)) * TILE + gc * 8);
           cp_async16_tc(dst, src);
         } else {
           asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");

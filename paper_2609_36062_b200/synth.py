@@ -37,6 +37,7 @@ class Workload:
     recipe: str       # "scaled" or "normalised"
     seed: int
     backward: bool = False
+    routing: str = "positional"   # or "hashed": prof / type arrays drawn by a fixed random hash (user-supplied routing)
 
     @property
     def bh(self) -> int:
@@ -66,6 +67,8 @@ WORKLOADS = {
     "t64k_d1_h4":    Workload("t64k_d1_h4", 1, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t64k_d2_h4":    Workload("t64k_d2_h4", 2, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t8k_d3_fwdbwd": Workload("t8k_d3_fwdbwd", 3, 8, 16, 8192, 128, 128, 64, "bf16", "normalised", 4, True),
+    # the 16 K configuration under user-supplied routing: every token hashed to a uniformly random cell / type
+    "t16k_d4_hashed": Workload("t16k_d4_hashed", 4, 2, 16, 16384, 128, 128, 128, "bf16", "normalised", 2, False, "hashed"),
     # cached decoding: 128 sequences of 16 heads, 2 K horizon (132 type states + one running state per head; the
     # running states alone, 134 MB, exceed L2)
     "decode_t2k_d3": Workload("decode_t2k_d3", 3, 128, 16, 2048, 128, 128, 64, "bf16", "normalised", 5),
@@ -141,3 +144,9 @@ def hashed_query_draws(w: Workload, head: int, m: int, P: int, A: int) -> tuple[
     g = np.random.Generator(np.random.Philox(key=(int(w.seed) << 40) ^ (8 << 32) ^ int(head)))
     return (g.integers(0, P, size=m, dtype=np.int64).astype(np.int32),
             g.integers(0, A, size=m, dtype=np.int64).astype(np.int32))
+
+
+def hashed_types(w: Workload, head: int, m: int, B: int) -> np.ndarray:
+    """A fixed random hash of the recent tokens of one head into B types (int32 [m]), uniform."""
+    g = np.random.Generator(np.random.Philox(key=(int(w.seed) << 40) ^ (9 << 32) ^ int(head)))
+    return g.integers(0, B, size=m, dtype=np.int64).astype(np.int32)

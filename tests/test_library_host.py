@@ -109,7 +109,8 @@ def test_workspace_regions_follow_the_stored_element_types():
     exchange = w.bh * (g.q ** 3 + g.q ** 2) * state * 2          # intermediate of the two d = 4 tabulation stages
     causal = w.bh * (w.T // 128) * state * 2
     rows = w.bh * w.T * 128 * 4                                  # long-range rows
-    need = tables + exchange + causal + rows
+    lists = w.bh * (w.T + g.P + g.B + 2) * 4                     # token lists of user-supplied routing (int32)
+    need = tables + exchange + causal + rows + lists
     got = plan.workspace_bytes(False)
     assert need <= got <= need + 64 * 1024, (got, need)
     assert got < 9.0e9                                           # 15 GB with every region at 4 bytes per entry
