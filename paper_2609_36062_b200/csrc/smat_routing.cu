@@ -66,9 +66,16 @@ __global__ void __launch_bounds__(ROUTE_THREADS) routing_lists_kernel(const Rout
   __syncthreads();
   if (tid < 32) {
     const int64_t first = prm.first[kind];
+    constexpr int AHEAD = 8;   // keys are fetched this many steps ahead: the loop is a chain of shared-memory updates
+    int32_t kq[AHEAD];
+#pragma unroll
+    for (int a = 0; a < AHEAD; ++a) kq[a] = (int64_t)a * 32 + tid < n ? key[(int64_t)a * 32 + tid] : -1;
     for (int64_t t0 = 0; t0 < n; t0 += 32) {
       const int64_t t = t0 + tid;
-      const int32_t k = t < n ? key[t] : -1;
+      const int32_t k = kq[0];
+#pragma unroll
+      for (int a = 0; a + 1 < AHEAD; ++a) kq[a] = kq[a + 1];
+      kq[AHEAD - 1] = t + (int64_t)AHEAD * 32 < n ? key[t + (int64_t)AHEAD * 32] : -1;
       const bool valid = k >= 0 && k < G;
       const unsigned peers = __match_any_sync(0xffffffffu, valid ? k : -1 - tid);
       int32_t slot = 0;
