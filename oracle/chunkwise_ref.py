@@ -172,3 +172,57 @@ def streaming_rows(Q, K, V, geo, rows):
         if t in want:
             out[t] = Q[t] @ (U[_type(t, geo)] + S)
     return out
+
+
+def gated_forward(Q, K, V, log_a, geo):
+    """Lemma "Gated SMat": the chunkwise forward under scalar per-token gates.  λ is one prefix sum; every factor is
+    exp of a difference λ_i - λ_j with j <= i.  Causal branch: tile entries times exp(λ_i - λ_j), chunk summaries with
+    every Z_j scaled to the chunk's last index, the carried state decayed by the chunk's total gate and read with
+    exp(λ_i - λ_{e(b-1)}).  Long-range branch: the factor splits at the boundary into a key-side scalar folded into Z_j
+    and a query-side scalar on the read; the tables are the ungated ones of rescaled inputs."""
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64); V = np.asarray(V, dtype=np.float64)
+    lam = np.cumsum(np.asarray(log_a, dtype=np.float64))
+    T, r = Q.shape
+    p = V.shape[1]
+    n = geo.n
+    lam_b = lam[n - 1] if n > 0 else 0.0
+    F = np.zeros((geo.P, r, p))
+    for t in range(n):
+        F[_profile(t, geo)] += np.exp(lam_b - lam[t]) * np.outer(K[t], V[t])
+    U = tabulate(F, geo)
+    O = np.zeros((T, p))
+    for t in range(n, T):
+        O[t] += np.exp(lam[t] - lam_b) * (Q[t] @ U[_type(t, geo)])
+    S = np.zeros((r, p))
+    for s, e, lo in _chunks(geo):
+        if s == lo:
+            S = np.zeros((r, p))                            # the state restarts at the head of each block
+        ref = lam[s - 1] if s > 0 else 0.0                  # λ at the last index of the previous chunk
+        idx = np.arange(s, e)
+        decay = np.exp(np.minimum(lam[idx][:, None] - lam[idx][None, :], 0.0))
+        A = np.tril(Q[s:e] @ K[s:e].T) * decay
+        O[s:e] += np.exp(lam[idx] - ref)[:, None] * (Q[s:e] @ S) + A @ V[s:e]
+        D = (np.exp(lam[e - 1] - lam[idx])[:, None] * K[s:e]).T @ V[s:e]
+        S = np.exp(lam[e - 1] - ref) * S + D
+    return O
+
+
+def gated_streaming_rows(Q, K, V, log_a, geo, rows):
+    """Gated streaming decode of the recent block: cached U^(n) of keys rescaled to the boundary, S_t = a_t S_{t-1} + Z_t,
+    g_t = a_t g_{t-1}, ȳ_t = φ_tᵀ(g_t U_type + S_t)."""
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64); V = np.asarray(V, dtype=np.float64)
+    a = np.exp(np.asarray(log_a, dtype=np.float64))
+    lam = np.cumsum(np.asarray(log_a, dtype=np.float64))
+    r, p = Q.shape[1], V.shape[1]
+    F = np.zeros((geo.P, r, p))
+    for t in range(geo.n):
+        F[_profile(t, geo)] += np.exp(lam[geo.n - 1] - lam[t]) * np.outer(K[t], V[t])
+    U = tabulate(F, geo)
+    want = set(int(t) for t in rows)
+    out, S, g = {}, np.zeros((r, p)), 1.0
+    for t in range(geo.n, geo.T):
+        S = a[t] * S + np.outer(K[t], V[t])
+        g = a[t] * g
+        if t in want:
+            out[t] = Q[t] @ (g * U[_type(t, geo)] + S)
+    return out

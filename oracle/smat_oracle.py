@@ -372,6 +372,45 @@ def dkdv_cols(Q, K, V, dO, geo: Geometry, cols):
     return dK, dV
 
 
+# --------------------------------------------------------------------------- gated mask (Sec. 3.2)
+def decay_matrix(log_a) -> np.ndarray:
+    """exp(λ_t - λ_s) for s <= t (0 elsewhere), λ_t = Σ_{k<=t} log a_k, from per-token log-gates log a_k <= 0
+    (Eq. gated).  Every factor is formed as the exponential of a difference, so nothing overflows."""
+    lam = np.cumsum(np.asarray(log_a, dtype=np.float64))
+    diff = lam[:, None] - lam[None, :]
+    return np.where(np.tril(np.ones_like(diff, dtype=bool)), np.exp(np.minimum(diff, 0.0)), 0.0)
+
+
+def gated_forward_dense(Q, K, V, M, log_a):
+    """O = ((M ⊙ decay) ⊙ QKᵀ) V: the binary mask replaced by the continuous mask of Eq. gated."""
+    return forward_dense(Q, K, V, np.asarray(M, dtype=np.float64) * decay_matrix(log_a))
+
+
+def gated_backward_dense(Q, K, V, dO, M, log_a):
+    """Gradients of <dO, O> with respect to Q, K, V and the log-gates.  With W = M ⊙ decay ⊙ (dO Vᵀ) ⊙ (QKᵀ) (the
+    contribution of every edge), ∂/∂λ_t is the sum of W over row t minus the sum over column t, and log a_k enters
+    every λ_t with t >= k."""
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64); dO = np.asarray(dO, dtype=np.float64)
+    Mt = np.asarray(M, dtype=np.float64) * decay_matrix(log_a)
+    dQ, dK, dV = backward_dense(Q, K, V, dO, Mt)
+    W = Mt * (dO @ V.T) * (Q @ K.T)
+    dlam = W.sum(axis=1) - W.sum(axis=0)
+    dlog_a = np.cumsum(dlam[::-1])[::-1]
+    return dQ, dK, dV, dlog_a
+
+
+def gated_forward_rows(Q, K, V, geo: Geometry, log_a, rows):
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64); V = np.asarray(V, dtype=np.float64)
+    lam = np.cumsum(np.asarray(log_a, dtype=np.float64))
+    out = np.empty((len(rows), V.shape[1]), dtype=np.float64)
+    for k, t in enumerate(rows):
+        t = int(t)
+        w = mask_row(t, geo) * np.exp(np.minimum(lam[t] - lam, 0.0)) * (K @ Q[t])
+        out[k] = w @ V
+    return out
+
+
 # --------------------------------------------------------------------------- VC dimension
 def vc_dimension(M: np.ndarray, limit: int | None = None) -> int:
     """Brute-force VC dimension of the row supports of a 0/1 matrix (Sec. 2, "VC dimension of a mask").
