@@ -72,6 +72,9 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
                                         straight from the shared-memory slab (one output row per thread) instead of
                                         the register-resident form (K slopes x q offsets per thread) */
 
+#define SMAT_FLAG_GATED 64u          /* the plan serves smat_forward_gated / smat_backward_gated: it runs on the fp32-ALU
+                                        kernels and its workspace holds λ and the rescaled copies of Q, K, V, dO */
+
 /* Sizes of the construction (Sec. 3, "construction of G" and "Scaling with sequence length"). */
 typedef struct {
   int64_t T, c, n, m;  /* sequence length, chunk width, distant = c*floor(T/2c), recent = T - n */
@@ -163,6 +166,25 @@ smat_status smat_forward_routed(const smat_plan* plan, const void* Q, const void
 smat_status smat_backward_routed(const smat_plan* plan, const void* Q, const void* K, const void* V, const void* dO,
                                  void* dQ, void* dK, void* dV, const int32_t* prof, const int32_t* type,
                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * SCALAR-GATED SMat (Sec. 3.2, Eq. "gated"; Lemma "Gated SMat"): the binary mask is replaced by
+ *        M~_ij = M_ij exp(λ_i - λ_j),   λ_i = Σ_{k <= i} log a_k,   j <= i,
+ * for per-token decay gates a_k in (0, 1].  log_a is a DEVICE fp32 array [batch*heads, T] of log-gates (<= 0).
+ * The chunkwise form of the lemma is used: λ by one prefix sum; within-chunk tiles times exp(λ_i - λ_j); chunk
+ * summaries of keys scaled to the chunk's last index; the carried state decayed by every chunk it passes and read with
+ * exp(λ_i - λ_{e(b-1)}); in the long-range branch the factor splits at the block boundary into a key-side scalar folded
+ * into k_j before pooling and a query-side scalar on the typed read, so tables and tabulation are the ungated ones of
+ * rescaled inputs.  Every factor is the exponential of a non-positive difference: nothing overflows however strong
+ * the decay.  smat_backward_gated also returns dlog_a [batch*heads, T] (DEVICE fp32), the gradient with respect to the
+ * log-gates.  The plan must carry SMAT_FLAG_GATED (else SMAT_ERR_UNSUPPORTED); this variant runs on the fp32-ALU
+ * kernels for every shape.  Otherwise as smat_forward / smat_backward.
+ */
+smat_status smat_forward_gated(const smat_plan* plan, const void* Q, const void* K, const void* V, const float* log_a,
+                               void* O, void* workspace, size_t workspace_bytes, void* cuda_stream);
+smat_status smat_backward_gated(const smat_plan* plan, const void* Q, const void* K, const void* V, const float* log_a,
+                                const void* dO, void* dQ, void* dK, void* dV, float* dlog_a, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream);
 
 /*
  * Routing as the library's index code sees it (HOST output buffers, caller-allocated):

@@ -22,6 +22,7 @@ FLAG_PER_TILE_STATES = 4
 FLAG_KEEP_FORWARD_TABLES = 8
 FLAG_ALU_TABULATION = 16
 FLAG_D3_SHARED_SUMS = 32
+FLAG_GATED = 64
 
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
@@ -29,7 +30,7 @@ EXPORTS = [
     "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
     "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step",
     "smat_static_check_status", "smat_debug_timeout_probe", "smat_measure_fadd_rate",
-    "smat_forward_routed", "smat_backward_routed",
+    "smat_forward_routed", "smat_backward_routed", "smat_forward_gated", "smat_backward_gated",
 ]
 
 
@@ -88,6 +89,10 @@ def load_library() -> ctypes.CDLL:
     lib.smat_forward_routed.restype = i
     lib.smat_backward_routed.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.smat_backward_routed.restype = i
+    lib.smat_forward_gated.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.smat_forward_gated.restype = i
+    lib.smat_backward_gated.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.smat_backward_gated.restype = i
     lib.smat_routing_indices.argtypes = [vp, vp, vp, vp]
     lib.smat_routing_indices.restype = i
     lib.smat_debug_mask.argtypes = [vp, vp, vp]
@@ -298,6 +303,34 @@ class SmatPlan:
         _check(self.lib.smat_backward(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), _ptr(dQ), _ptr(dK), _ptr(dV),
                                       _ptr(ws), ws.numel(), _stream(stream)), "smat_backward")
         return dQ, dK, dV
+
+    # -- scalar-gated variant ---------------------------------------------------------------------
+    def _check_gates(self, log_a):
+        b, h, T, _, _ = self.shape
+        if not (log_a.is_cuda and log_a.dtype == torch.float32 and log_a.is_contiguous() and tuple(log_a.shape) == (b * h, T)):
+            raise ValueError(f"log_a: expected a contiguous CUDA float32 tensor of shape {(b * h, T)}")
+
+    def forward_gated(self, Q, K, V, log_a, O=None, workspace=None, stream=None):
+        _, _, _, dk, dv = self.shape
+        self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
+        self._check_gates(log_a)
+        O = torch.empty_like(V) if O is None else O
+        ws = self.workspace(False, Q.device) if workspace is None else workspace
+        _check(self.lib.smat_forward_gated(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(log_a), _ptr(O), _ptr(ws),
+                                           ws.numel(), _stream(stream)), "smat_forward_gated")
+        return O
+
+    def backward_gated(self, Q, K, V, log_a, dO, workspace=None, stream=None):
+        _, _, _, dk, dv = self.shape
+        self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
+        self._check_tensor(dO, dv, "dO")
+        self._check_gates(log_a)
+        dQ, dK, dV, dla = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V), torch.empty_like(log_a)
+        ws = self.workspace(True, Q.device) if workspace is None else workspace
+        _check(self.lib.smat_backward_gated(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(log_a), _ptr(dO), _ptr(dQ),
+                                            _ptr(dK), _ptr(dV), _ptr(dla), _ptr(ws), ws.numel(), _stream(stream)),
+               "smat_backward_gated")
+        return dQ, dK, dV, dla
 
     # -- cached decoding -----------------------------------------------------------------------
     def decode_cache(self, device="cuda") -> torch.Tensor:

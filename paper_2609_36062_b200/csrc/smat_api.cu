@@ -23,6 +23,7 @@ struct smat_plan {
   size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_W, off_fwd_end;
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
   size_t off_plist, off_poffs, off_tlist, off_toffs;   // token lists of user-supplied routing (int32)
+  size_t off_lam, off_dlam, off_gq, off_gk, off_glr, off_gdo, off_gv, off_gvlr;   // gated variant (SMAT_FLAG_GATED)
   bool tc;             // tensor-core kernels for the causal branch
   bool u_bf16;         // forward keeps the type table U in bf16 and reads it with the tensor-core typed read
   bool pool_tc;        // forward pools the profile table on the tensor cores (enough tokens per profile)
@@ -213,14 +214,14 @@ void state_read(Ctx& cx, const char* name, int mode, const void* x, const float*
 }
 
 // tile[bh][chunk] (c x c, fp32) = tril(X_b Y_bᵀ), X, Y: [T, dim]
-void tril_scores(Ctx& cx, const char* name, const void* x, const void* y, int dim, float* tile) {
+void tril_scores(Ctx& cx, const char* name, const void* x, const void* y, int dim, float* tile, const float* lam = nullptr) {
   const smat_plan* pl = cx.pl;
   const int bf = pl->dtype == SMAT_BF16;
   SmatGemmArgs g{};
   g.A = operand(x, bf, pl->T * dim, 0, dim, 1, 1, 0);
   g.B = operand(y, bf, pl->T * dim, 0, 1, dim, 0, 1);
   g.C = operand(tile, 0, pl->NC * pl->c * pl->c, pl->c * pl->c, pl->c, 1);
-  g.K = dim; g.tokM = 1; g.tokN = 1; g.tril = 1; g.grp = group(pl, SMAT_GM_CHUNK);
+  g.K = dim; g.tokM = 1; g.tokN = 1; g.tril = 1; g.grp = group(pl, SMAT_GM_CHUNK); g.lam = lam;
   SMAT_TRY(cx, name, smat_launch_gemm(g, (int)pl->c, (int)pl->c, pl->NC, pl->bh, cx.st));
 }
 
@@ -357,7 +358,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   const SmatGeo& g = pl->geo;
   // Which kernels a plan uses depends on the shape alone (no device work here); whether the current device can run
   // them is checked by the calls that launch.
-  pl->tc = dtype == SMAT_BF16 && d_k == 128 && d_v == 128 && !(flags & SMAT_FLAG_SIMT_ONLY) && g.n % 128 == 0 &&
+  pl->tc = dtype == SMAT_BF16 && d_k == 128 && d_v == 128 && !(flags & (SMAT_FLAG_SIMT_ONLY | SMAT_FLAG_GATED)) && g.n % 128 == 0 &&
            g.m % 128 == 0 && g.n >= 128;
   if (!g.dense_G && (smat_tabulate_alg2_slab(g.B, pl->rp) < 1)) { delete pl; return SMAT_ERR_UNSUPPORTED; }
   // d >= 3 on the tensor-core path: U is only ever a bf16 MMA operand, so it is stored as bf16 (half the bytes)
@@ -400,7 +401,18 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->off_poffs = off;  off = align_up(off + (lists ? (size_t)pl->bh * (g.P + 1) * 4 : 0));
   pl->off_tlist = off;  off = align_up(off + (lists ? (size_t)pl->bh * g.m * 4 : 0));
   pl->off_toffs = off;  off = align_up(off + (lists ? (size_t)pl->bh * (g.B + 1) * 4 : 0));
+  // gated variant: λ and the rescaled copies of Q, K (forward) and dO, V (backward), in the plan's dtype
+  const size_t esz = dtype == SMAT_BF16 ? 2 : 4;
+  const size_t gated = (flags & SMAT_FLAG_GATED) ? 1 : 0;
+  pl->off_lam = off;    off = align_up(off + gated * (size_t)pl->bh * T * 4);
+  pl->off_gq = off;     off = align_up(off + gated * (size_t)pl->bh * T * d_k * esz);
+  pl->off_gk = off;     off = align_up(off + gated * (size_t)pl->bh * T * d_k * esz);
+  pl->off_glr = off;    off = align_up(off + gated * (size_t)pl->bh * T * d_k * esz);
   pl->off_fwd_end = off;
+  pl->off_dlam = off;   off = align_up(off + gated * (size_t)pl->bh * T * 4);
+  pl->off_gdo = off;    off = align_up(off + gated * (size_t)pl->bh * T * d_v * esz);
+  pl->off_gv = off;     off = align_up(off + gated * (size_t)pl->bh * T * d_v * esz);
+  pl->off_gvlr = off;   off = align_up(off + gated * (size_t)pl->bh * T * d_v * esz);
   pl->off_dbar = off;   off = align_up(off + causal);
   pl->off_ubar = off;   off = align_up(off + (g.dense_G || alias ? 0 : (size_t)pl->bh * g.B * entries * (pl->ubar_bf16 ? 2 : 4)));
   pl->off_fbar = off;   off = align_up(off + (g.dense_G ? 0 : (size_t)pl->bh * g.P * entries * (pl->fbar_bf16 ? 2 : 4)));
@@ -670,9 +682,137 @@ smat_status backward_impl(const smat_plan* pl, const void* Q, const void* K, con
   return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
 }
 
+// ---- scalar-gated variant (Sec. 3.2, Eq. "gated"; Lemma "Gated SMat") on the fp32-ALU kernels ------------------------
+struct Gated {
+  float* lam;
+  void *qc, *kc, *lr, *doc, *vc, *vlr;
+};
+
+Gated gated_buffers(const Ctx& cx) {
+  const smat_plan* pl = cx.pl;
+  return Gated{cx.f(pl->off_lam), cx.ws + pl->off_gq, cx.ws + pl->off_gk, cx.ws + pl->off_glr,
+               cx.ws + pl->off_gdo, cx.ws + pl->off_gv, cx.ws + pl->off_gvlr};
+}
+
+void gate_scale(Ctx& cx, const char* name, const void* a, const void* b, void* out, const float* lam, int mode, int dim) {
+  const smat_plan* pl = cx.pl;
+  SMAT_TRY(cx, name, smat_launch_gate_scale(a, b, out, lam, mode, pl->dtype == SMAT_BF16, pl->geo.n, pl->c, pl->T, dim,
+                                            pl->bh, cx.st));
+}
+
+void gated_scan(Ctx& cx, const char* name, float* S, const float* lam, int reverse) {
+  const smat_plan* pl = cx.pl;
+  const int64_t ncd = pl->geo.n / pl->c;
+  if (pl->geo.dense_G)   // d = 1: one causal block; the carried state crosses the boundary (it is U_0 decayed)
+    SMAT_TRY(cx, name, smat_launch_gated_scan(S, lam, pl->rp, pl->NC, pl->c, pl->bh, 0, pl->NC, 0, 0, reverse, cx.st));
+  else
+    SMAT_TRY(cx, name, smat_launch_gated_scan(S, lam, pl->rp, pl->NC, pl->c, pl->bh, 0, ncd, ncd, pl->NC, reverse, cx.st));
+}
+
+// λ, the rescaled inputs and the forward tables (S_in, F, U) of the gated pass.
+void gated_forward_tables(Ctx& cx, const Gated& gt, const void* Q, const void* K, const void* V, const float* log_a) {
+  const smat_plan* pl = cx.pl;
+  SMAT_TRY(cx, "gate_prefix", smat_launch_head_scan(log_a, gt.lam, pl->T, pl->bh, 0, cx.st));
+  gate_scale(cx, "gate_scale_q", Q, nullptr, gt.qc, gt.lam, 0, pl->r);       // exp(λ_i - λ_{e(b-1)}) q_i
+  gate_scale(cx, "gate_scale_k", K, nullptr, gt.kc, gt.lam, 1, pl->r);       // exp(λ_{e(b)} - λ_j) k_j
+  if (!pl->geo.dense_G) {
+    gate_scale(cx, "gate_scale_lr", K, Q, gt.lr, gt.lam, 2, pl->r);          // keys and queries split at the boundary
+    outer_sum(cx, "pool", SMAT_GM_PROFILE, gt.lr, V, cx.f(pl->off_F));
+    tabulate(cx, "tabulate", cx.f(pl->off_F), cx.f(pl->off_U), 0);
+  }
+  outer_sum(cx, "chunk_state", SMAT_GM_CHUNK, gt.kc, V, cx.f(pl->off_sin));
+  gated_scan(cx, "gated_scan", cx.f(pl->off_sin), gt.lam, 0);
+}
+
+smat_status gated_check(const smat_plan* pl, const void* log_a, void* ws, size_t ws_bytes, int for_backward) {
+  if (!log_a) return SMAT_ERR_NULL;
+  smat_status s = check_common(pl, ws, ws_bytes, for_backward);
+  if (s != SMAT_OK) return s;
+  if (!(pl->flags & SMAT_FLAG_GATED)) return SMAT_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(log_a) & 3) return SMAT_ERR_ALIGN;
+  return SMAT_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+smat_status smat_forward_gated(const smat_plan* pl, const void* Q, const void* K, const void* V, const float* log_a,
+                               void* O, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!Q || !K || !V || !O) return SMAT_ERR_NULL;
+  smat_status s = gated_check(pl, log_a, workspace, workspace_bytes, 0);
+  if (s != SMAT_OK) return s;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
+  Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
+  pl->stages = 0;
+  pl->tile_states = false;
+  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  const Gated gt = gated_buffers(cx);
+  gated_forward_tables(cx, gt, Q, K, V, log_a);
+  float* acc = cx.f(pl->off_acc);
+  float* tileA = cx.f(pl->off_tileA);
+  tril_scores(cx, "scores", Q, K, pl->r, tileA, gt.lam);                         // tril(QKᵀ) ⊙ exp(λ_i - λ_j)
+  state_read(cx, "read_chunk", SMAT_GM_CHUNK, gt.qc, cx.f(pl->off_sin), 0, nullptr, acc, nullptr);
+  if (!pl->geo.dense_G) state_read(cx, "read_type", SMAT_GM_TYPE, gt.lr, cx.f(pl->off_U), 0, acc, acc, nullptr);
+  tile_apply(cx, "output", tileA, 0, V, pl->p, acc, nullptr, O);
+  pl->launches = cx.launches;
+  return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
+smat_status smat_backward_gated(const smat_plan* pl, const void* Q, const void* K, const void* V, const float* log_a,
+                                const void* dO, void* dQ, void* dK, void* dV, float* dlog_a, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream) {
+  if (!Q || !K || !V || !dO || !dQ || !dK || !dV || !dlog_a) return SMAT_ERR_NULL;
+  smat_status s = gated_check(pl, log_a, workspace, workspace_bytes, 1);
+  if (s != SMAT_OK) return s;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(dO) || misaligned(dQ) || misaligned(dK) ||
+      misaligned(dV) || (reinterpret_cast<uintptr_t>(dlog_a) & 3))
+    return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
+  Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
+  pl->stages = 0;
+  pl->tile_states = false;
+  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  const bool lr = !pl->geo.dense_G;
+  const Gated gt = gated_buffers(cx);
+  gated_forward_tables(cx, gt, Q, K, V, log_a);
+  gate_scale(cx, "bwd_gate_scale_do", dO, nullptr, gt.doc, gt.lam, 0, pl->p);    // exp(λ_i - λ_{e(b-1)}) dO_i
+  gate_scale(cx, "bwd_gate_scale_v", V, nullptr, gt.vc, gt.lam, 1, pl->p);       // exp(λ_{e(b)} - λ_j) v_j
+  if (lr) gate_scale(cx, "bwd_gate_scale_lr", V, dO, gt.vlr, gt.lam, 2, pl->p);  // values / upstream rows at the boundary
+  float* sin = cx.f(pl->off_sin);
+  float* dbar = cx.f(pl->off_dbar);
+  float* acc = cx.f(pl->off_acc);
+  float* tileA = cx.f(pl->off_tileA);
+  float* tileG = cx.f(pl->off_tileG);
+  // adjoint of the carried state: S̄_in_b = Σ_i (scaled q_i) dO_iᵀ, then the decayed suffix recursion
+  outer_sum(cx, "bwd_chunk_state", SMAT_GM_CHUNK, gt.qc, dO, dbar);
+  gated_scan(cx, "bwd_gated_scan", dbar, gt.lam, 1);
+  if (lr) {
+    outer_sum(cx, "bwd_pool_type", SMAT_GM_TYPE, gt.lr, dO, cx.f(pl->off_ubar));
+    tabulate(cx, "bwd_tabulate_t", cx.f(pl->off_ubar), cx.f(pl->off_fbar), 1);
+  }
+  tril_scores(cx, "bwd_scores_qk", Q, K, pl->r, tileA, gt.lam);
+  tril_scores(cx, "bwd_scores_gv", dO, V, pl->p, tileG, gt.lam);
+  // dQ_i = S_in (scaled dO_i) + U_type (boundary-scaled dO_i) + Σ_j G_ij k_j
+  state_read(cx, "bwd_dq_chunk", SMAT_GM_CHUNK, gt.doc, sin, 1, nullptr, acc, nullptr);
+  if (lr) state_read(cx, "bwd_dq_type", SMAT_GM_TYPE, gt.vlr, cx.f(pl->off_U), 1, acc, acc, nullptr);
+  tile_apply(cx, "bwd_dq_tile", tileG, 0, K, pl->r, acc, nullptr, dQ);
+  // dK_j = Σ_i G_ij q_i + F̄_prof (boundary-scaled v_j) + D̄ (chunk-scaled v_j)
+  tile_apply(cx, "bwd_dk_tile", tileG, 1, Q, pl->r, nullptr, acc, nullptr);
+  if (lr) state_read(cx, "bwd_dk_profile", SMAT_GM_PROFILE, gt.vlr, cx.f(pl->off_fbar), 1, acc, acc, nullptr);
+  state_read(cx, "bwd_dk_chunk", SMAT_GM_CHUNK, gt.vc, dbar, 1, acc, nullptr, dK);
+  // dV_j = Σ_i A_ij dO_i + F̄_profᵀ (boundary-scaled k_j) + D̄ᵀ (chunk-scaled k_j)
+  tile_apply(cx, "bwd_dv_tile", tileA, 1, dO, pl->p, nullptr, acc, nullptr);
+  if (lr) state_read(cx, "bwd_dv_profile", SMAT_GM_PROFILE, gt.lr, cx.f(pl->off_fbar), 0, acc, acc, nullptr);
+  state_read(cx, "bwd_dv_chunk", SMAT_GM_CHUNK, gt.kc, dbar, 0, acc, nullptr, dV);
+  // gates: dλ_t = q_t·dQ_t - k_t·dK_t, and log a_k enters every λ_t with t >= k
+  float* dlam = cx.f(pl->off_dlam);
+  SMAT_TRY(cx, "bwd_gate_dlam", smat_launch_gate_dlam(Q, dQ, K, dK, dlam, pl->dtype == SMAT_BF16, pl->r, pl->T, pl->bh, cx.st));
+  SMAT_TRY(cx, "bwd_gate_suffix", smat_launch_head_scan(dlam, dlog_a, pl->T, pl->bh, 1, cx.st));
+  pl->launches = cx.launches;
+  return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
 
 smat_status smat_forward(const smat_plan* pl, const void* Q, const void* K, const void* V, void* O, void* workspace,
                          size_t workspace_bytes, void* cuda_stream) {

@@ -1,0 +1,156 @@
+// Small kernels of the scalar-gated variant (Sec. 3.2, Eq. "gated"; Lemma "Gated SMat"): the prefix sum λ of the
+// log-gates, the rescaled copies of Q, K, V, dO that carry the query-side and key-side factors, the decayed scan of the
+// chunk states and the gate gradient.  Every factor is the exponential of a difference λ_i - λ_j with j <= i, so it lies
+// in (0, 1] and nothing can overflow.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "smat_internal.h"
+
+namespace {
+
+// Inclusive prefix (reverse = 0) or suffix (reverse = 1) sum of one row of `len` floats per head; one CTA per head.
+__global__ void __launch_bounds__(1024) head_scan_kernel(const float* __restrict__ in, float* __restrict__ out, int64_t len,
+                                                         int reverse) {
+  __shared__ float warp_sum[32];
+  __shared__ float carry;
+  const int tid = threadIdx.x;
+  const float* src = in + (int64_t)blockIdx.x * len;
+  float* dst = out + (int64_t)blockIdx.x * len;
+  if (tid == 0) carry = 0.f;
+  __syncthreads();
+  for (int64_t base = 0; base < len; base += 1024) {
+    const int64_t k = base + tid;
+    const int64_t idx = reverse ? len - 1 - k : k;
+    const float v = k < len ? src[idx] : 0.f;
+    float x = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const float y = __shfl_up_sync(0xffffffffu, x, d);
+      if ((tid & 31) >= d) x += y;
+    }
+    if ((tid & 31) == 31) warp_sum[tid >> 5] = x;
+    __syncthreads();
+    float before = carry;
+    for (int w = 0; w < (tid >> 5); ++w) before += warp_sum[w];
+    if (k < len) dst[idx] = before + x;
+    __syncthreads();
+    if (tid == 1023) carry = before + x;
+    __syncthreads();
+  }
+}
+
+// Rescaled copy of token rows: out[t] = src[t] * f(t), dim values per row, in the plan's dtype.
+//   mode 0 (query side of a chunk)   : f = exp(λ_t - λ_{s(t)-1}),  s(t) = first token of t's chunk (λ_{-1} = 0)
+//   mode 1 (key side of a chunk)     : f = exp(λ_{e(t)} - λ_t),    e(t) = last token of t's chunk
+//   mode 2 (the block boundary)      : t <  n: src = A, f = exp(λ_{n-1} - λ_t)   (key side, folded into Z_j)
+//                                      t >= n: src = B, f = exp(λ_t - λ_{n-1})   (query side, on the read)
+template <typename T>
+__global__ void gate_scale_kernel(const T* __restrict__ A, const T* __restrict__ B, T* __restrict__ out,
+                                  const float* __restrict__ lam, int mode, int64_t n, int64_t c, int64_t Tlen, int dim,
+                                  int64_t rows) {
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
+  if (row >= rows) return;
+  const int lane = threadIdx.x & 31;
+  const int64_t bh = row / Tlen, t = row - bh * Tlen;
+  const float* l = lam + bh * Tlen;
+  float f;
+  const T* src = A;
+  if (mode == 0) {
+    const int64_t s = t - t % c;
+    f = __expf(l[t] - (s > 0 ? l[s - 1] : 0.f));
+  } else if (mode == 1) {
+    const int64_t e = t - t % c + c - 1;
+    f = __expf(l[e] - l[t]);
+  } else if (t < n) {
+    f = __expf(l[n - 1] - l[t]);
+  } else {
+    f = __expf(l[t] - l[n - 1]);
+    src = B;
+  }
+  for (int i = lane; i < dim; i += 32) out[row * dim + i] = (T)((float)src[row * dim + i] * f);
+}
+
+// Decayed exclusive scan of per-chunk states in place: walking the chunks of a range in order (or in reverse),
+//   out[b] = running;  running = γ_b running + in[b],   γ_b = exp(λ_{e(b)} - λ_{s(b)-1}) = the product of chunk b's gates.
+// Forward this is S_in (Lemma "Gated SMat": the carried state is decayed by every chunk it passes); in reverse it is the
+// adjoint recursion of the same scan.
+__global__ void __launch_bounds__(256) gated_scan_kernel(float* S, const float* __restrict__ lam, int64_t state_elems,
+                                                         int64_t NC, int64_t c, int64_t lo0, int64_t hi0, int64_t lo1,
+                                                         int64_t hi1, int reverse) {
+  const int64_t e4 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e4 * 4 >= state_elems) return;
+  const int64_t bh = blockIdx.y;
+  const int64_t lo = blockIdx.z ? lo1 : lo0, hi = blockIdx.z ? hi1 : hi0;
+  float4* base = reinterpret_cast<float4*>(S + bh * NC * state_elems) + e4;
+  const float* l = lam + bh * NC * c;
+  const int64_t stride4 = state_elems / 4;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int64_t k = 0; k < hi - lo; ++k) {
+    const int64_t b = reverse ? hi - 1 - k : lo + k;
+    const float4 v = base[b * stride4];
+    base[b * stride4] = acc;
+    const float g = __expf(l[b * c + c - 1] - (b > 0 ? l[b * c - 1] : 0.f));
+    acc.x = g * acc.x + v.x; acc.y = g * acc.y + v.y; acc.z = g * acc.z + v.z; acc.w = g * acc.w + v.w;
+  }
+}
+
+// dλ_t = q_t·dQ_t - k_t·dK_t (every edge's contribution enters once as a query and once as a key); one warp per token.
+template <typename T>
+__global__ void gate_dlam_kernel(const T* __restrict__ Q, const T* __restrict__ dQ, const T* __restrict__ K,
+                                 const T* __restrict__ dK, float* __restrict__ dlam, int dim, int64_t rows) {
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
+  if (row >= rows) return;
+  const int lane = threadIdx.x & 31;
+  float s = 0.f;
+  for (int i = lane; i < dim; i += 32)
+    s += (float)Q[row * dim + i] * (float)dQ[row * dim + i] - (float)K[row * dim + i] * (float)dK[row * dim + i];
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+  if (lane == 0) dlam[row] = s;
+}
+
+}  // namespace
+
+cudaError_t smat_launch_head_scan(const float* in, float* out, int64_t len, int bh, int reverse, cudaStream_t st) {
+  head_scan_kernel<<<(unsigned)bh, 1024, 0, st>>>(in, out, len, reverse);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_gate_scale(const void* A, const void* B, void* out, const float* lam, int mode, int bf16,
+                                   int64_t n, int64_t c, int64_t T, int dim, int bh, cudaStream_t st) {
+  const int64_t rows = (int64_t)bh * T;
+  const unsigned blocks = (unsigned)((rows * 32 + 255) / 256);
+  if (bf16)
+    gate_scale_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(A),
+                                                             static_cast<const __nv_bfloat16*>(B),
+                                                             static_cast<__nv_bfloat16*>(out), lam, mode, n, c, T, dim, rows);
+  else
+    gate_scale_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(A), static_cast<const float*>(B),
+                                                     static_cast<float*>(out), lam, mode, n, c, T, dim, rows);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_gated_scan(float* S, const float* lam, int64_t state_elems, int64_t NC, int64_t c, int bh,
+                                   int64_t lo0, int64_t hi0, int64_t lo1, int64_t hi1, int reverse, cudaStream_t st) {
+  const int ranges = (hi1 > lo1) ? 2 : 1;
+  dim3 grid((unsigned)((state_elems / 4 + 255) / 256), (unsigned)bh, (unsigned)ranges);
+  gated_scan_kernel<<<grid, 256, 0, st>>>(S, lam, state_elems, NC, c, lo0, hi0, lo1, hi1, reverse);
+  return cudaGetLastError();
+}
+
+cudaError_t smat_launch_gate_dlam(const void* Q, const void* dQ, const void* K, const void* dK, float* dlam, int bf16,
+                                  int dim, int64_t T, int bh, cudaStream_t st) {
+  const int64_t rows = (int64_t)bh * T;
+  const unsigned blocks = (unsigned)((rows * 32 + 255) / 256);
+  if (bf16)
+    gate_dlam_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(Q),
+                                                            static_cast<const __nv_bfloat16*>(dQ),
+                                                            static_cast<const __nv_bfloat16*>(K),
+                                                            static_cast<const __nv_bfloat16*>(dK), dlam, dim, rows);
+  else
+    gate_dlam_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(Q), static_cast<const float*>(dQ),
+                                                    static_cast<const float*>(K), static_cast<const float*>(dK), dlam, dim,
+                                                    rows);
+  return cudaGetLastError();
+}

@@ -77,6 +77,8 @@ struct SmatGemmArgs {
   int tril;
   int tilesN;                // number of 64-wide column tiles launched
   SmatGroupSpec grp;
+  const float* lam;          // gated variant: prefix sums of the log-gates [bh][T]; a tril tile over the tokens of a chunk
+                             // is multiplied entrywise by exp(λ_m - λ_n) (null: no decay)
 };
 
 cudaError_t smat_launch_gemm(const SmatGemmArgs& a, int max_M, int max_N, int64_t groups, int bh, cudaStream_t st);
@@ -161,6 +163,14 @@ cudaError_t smat_launch_pool_tc(const void* K, const void* V, void* F, int out_b
 // bf16 table kept slab-major [bh][rp / 32][rows][32] -> fp32 [bh][rows][rp] (debug export).
 cudaError_t smat_launch_widen_bf16_slabs(const void* src_bf16, float* dst, int64_t heads, int64_t rows, int64_t rp,
                                          cudaStream_t st);
+// Gated variant (Sec. 3.2): prefix / suffix sums per head, rescaled copies, decayed chunk scan, gate gradient.
+cudaError_t smat_launch_head_scan(const float* in, float* out, int64_t len, int bh, int reverse, cudaStream_t st);
+cudaError_t smat_launch_gate_scale(const void* A, const void* B, void* out, const float* lam, int mode, int bf16,
+                                   int64_t n, int64_t c, int64_t T, int dim, int bh, cudaStream_t st);
+cudaError_t smat_launch_gated_scan(float* S, const float* lam, int64_t state_elems, int64_t NC, int64_t c, int bh,
+                                   int64_t lo0, int64_t hi0, int64_t lo1, int64_t hi1, int reverse, cudaStream_t st);
+cudaError_t smat_launch_gate_dlam(const void* Q, const void* dQ, const void* K, const void* dK, float* dlam, int bf16,
+                                  int dim, int64_t T, int bh, cudaStream_t st);
 // Token lists of user-supplied routing: prof [bh][n] (cells in [0, P)) and type [bh][m] (types in [0, B)) -> CSR lists
 // (offsets [bh][G + 1], token positions [bh][count], ascending inside a group).  Keys out of range are dropped.
 int64_t smat_routing_max_groups();

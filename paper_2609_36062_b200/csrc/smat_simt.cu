@@ -100,6 +100,10 @@ __global__ void __launch_bounds__(256) gemm_grouped_kernel(const SmatGemmArgs a)
       if (n >= N) continue;
       const int64_t x1 = a.C.tok1 ? tk.at(n) : (int64_t)n;
       float v = (a.tril && n > m) ? 0.f : acc[i][j];
+      if (a.lam && a.tril && n <= m) {   // gated: decay between the key's and the query's position
+        const float* l = a.lam + bh * a.grp.T;
+        v *= __expf(l[tk.at(m)] - l[tk.at(n)]);
+      }
       if (a.Cin.ptr) v += reinterpret_cast<const float*>(a.Cin.ptr)[baseI + x0 * a.Cin.s0 + x1 * a.Cin.s1];
       const int64_t off = baseC + x0 * a.C.s0 + x1 * a.C.s1;
       if (a.C.bf16)

@@ -1,0 +1,96 @@
+"""Scalar-gated SMat on the GPU (smat_forward_gated / smat_backward_gated) against the fp64 oracle of Eq. "gated"."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import smat_oracle as so
+from paper_2609_36062_b200 import binding, synth
+from tests.helpers import TOL, device_inputs, rel_err, sample_tokens, to_numpy64
+
+pytestmark = pytest.mark.gpu
+
+
+def _gates(w, lo, seed):
+    g = np.random.default_rng(seed)
+    return np.log(g.uniform(lo, 1.0, (w.bh, w.T))).astype(np.float32)
+
+
+CASES = [
+    # d, T, dk, dv, c, dtype, q, smallest gate
+    (1, 256, 64, 64, 32, "f32", 0, 0.8), (2, 512, 64, 64, 64, "f32", 0, 0.9), (3, 512, 128, 64, 32, "f32", 0, 0.7),
+    (4, 1024, 64, 64, 16, "f32", 3, 0.9), (3, 768, 64, 64, 64, "bf16", 0, 0.9), (2, 384, 64, 128, 16, "f32", 0, 0.5),
+    (3, 1024, 128, 128, 128, "bf16", 0, 0.95), (1, 512, 128, 128, 128, "bf16", 0, 0.9),
+]
+
+
+@pytest.mark.parametrize("d,T,dk,dv,c,dtype,q,lo", CASES)
+def test_gated_forward_and_gradients_match_the_dense_oracle(d, T, dk, dv, c, dtype, q, lo):
+    w = synth.Workload("g", d, 1, 2, T, dk, dv, c, dtype, "scaled", 21)
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    la = _gates(w, lo, 3)
+    la_dev = torch.from_numpy(la).cuda()
+    plan = binding.SmatPlan(1, 2, T, dk, dv, d, c, dtype, q_override=q, flags=binding.FLAG_GATED)
+    assert not plan.uses_tensor_cores()
+    O = plan.forward_gated(dev["q"], dev["k"], dev["v"], la_dev)
+    dQ, dK, dV, dla = plan.backward_gated(dev["q"], dev["k"], dev["v"], la_dev, dev["do"])
+    plan.check_status()
+    M = so.dense_mask(T, c, d, q or None)
+    tol = TOL[dtype]
+    for h in range(w.bh):
+        Q64, K64, V64, G64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v", "do"))
+        lah = la[h].astype(np.float64)
+        assert rel_err(to_numpy64(O[0, h]), so.gated_forward_dense(Q64, K64, V64, M, lah)) <= tol
+        rq, rk, rv, rl = so.gated_backward_dense(Q64, K64, V64, G64, M, lah)
+        for name, got, ref in (("dQ", dQ, rq), ("dK", dK, rk), ("dV", dV, rv)):
+            e = rel_err(to_numpy64(got[0, h]), ref)
+            assert e <= tol, (name, h, e)
+        # the gate gradient is a difference of two row sums followed by a suffix sum over the whole sequence
+        e = rel_err(dla[h].double().cpu().numpy(), rl)
+        assert e <= (1e-3 if dtype == "f32" else 5e-2), ("dlog_a", h, e)
+
+
+def test_unit_gates_reproduce_the_ungated_pass():
+    w = synth.Workload("g1", 3, 1, 2, 512, 64, 64, 32, "f32", "scaled", 5)
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    zeros = torch.zeros(w.bh, w.T, device="cuda")
+    gated = binding.SmatPlan(1, 2, w.T, 64, 64, 3, 32, "f32", flags=binding.FLAG_GATED)
+    plain = binding.SmatPlan(1, 2, w.T, 64, 64, 3, 32, "f32")
+    a = gated.forward_gated(dev["q"], dev["k"], dev["v"], zeros)
+    b = plain.forward(dev["q"], dev["k"], dev["v"])
+    assert rel_err(to_numpy64(a), to_numpy64(b)) <= 1e-6
+    ga = gated.backward_gated(dev["q"], dev["k"], dev["v"], zeros, dev["do"])
+    gb = plain.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+    for x, y in zip(ga[:3], gb):
+        assert rel_err(to_numpy64(x), to_numpy64(y)) <= 1e-6
+
+
+def test_strong_decay_stays_finite_and_matches_the_oracle():
+    # λ reaches about -2000 at the end of the sequence: exp(-λ_j) alone would overflow fp32 after 13 tokens
+    w = synth.Workload("g2", 3, 1, 1, 512, 64, 64, 32, "f32", "scaled", 6)
+    host, dev = device_inputs(w)
+    la = np.full((1, w.T), np.log(0.02), dtype=np.float32)
+    plan = binding.SmatPlan(1, 1, w.T, 64, 64, 3, 32, "f32", flags=binding.FLAG_GATED)
+    O = plan.forward_gated(dev["q"], dev["k"], dev["v"], torch.from_numpy(la).cuda())
+    assert torch.isfinite(O).all()
+    Q64, K64, V64 = (synth.as_float64(w, host[x][0]) for x in ("q", "k", "v"))
+    ref = so.gated_forward_dense(Q64, K64, V64, so.dense_mask(w.T, 32, 3), la[0].astype(np.float64))
+    assert rel_err(to_numpy64(O[0, 0]), ref) <= 1e-4
+
+
+def test_gated_rows_at_a_longer_sequence_and_argument_errors():
+    w = synth.Workload("g3", 3, 1, 2, 4096, 128, 128, 64, "bf16", "normalised", 9)
+    host, dev = device_inputs(w)
+    la = _gates(w, 0.97, 4)
+    plan = binding.SmatPlan(1, 2, w.T, 128, 128, 3, 64, "bf16", flags=binding.FLAG_GATED)
+    O = plan.forward_gated(dev["q"], dev["k"], dev["v"], torch.from_numpy(la).cuda())
+    plan.check_status()
+    geo = so.geometry(w.T, 64, 3)
+    rows = sample_tokens(geo, 48, seed=2)
+    Q64, K64, V64 = (synth.as_float64(w, host[x][1]) for x in ("q", "k", "v"))
+    ref = so.gated_forward_rows(Q64, K64, V64, geo, la[1].astype(np.float64), rows)
+    assert rel_err(to_numpy64(O[0, 1][rows]), ref) <= TOL["bf16"]
+    # a plan without the flag has no room for λ and the rescaled copies
+    plain = binding.SmatPlan(1, 2, w.T, 128, 128, 3, 64, "bf16")
+    with pytest.raises(binding.SmatError) as err:
+        plain.forward_gated(dev["q"], dev["k"], dev["v"], torch.from_numpy(la).cuda())
+    assert err.value.code == 10
