@@ -411,6 +411,41 @@ def gated_forward_rows(Q, K, V, geo: Geometry, log_a, rows):
     return out
 
 
+# --------------------------------------------------------------------------- normalised output (Sec. 2)
+def normalized_forward_dense(Q, K, V, M):
+    """o_i = ȳ_{1:d_v} / ȳ_p with the augmented value v̄_j = [v_j; 1] (Eq. augmented-kv-state,
+    Eq. augmented-attention-output): numerator (M ⊙ QKᵀ)V, normaliser (M ⊙ QKᵀ)1.  Returns (O, normaliser).
+    Requires positive normalisers (non-negative features)."""
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64); V = np.asarray(V, dtype=np.float64)
+    W = np.asarray(M, dtype=np.float64) * (Q @ K.T)
+    den = W.sum(axis=1)
+    return (W @ V) / den[:, None], den
+
+
+def normalized_backward_dense(Q, K, V, dO, M):
+    """Gradients of <dO, O> for the normalised output, through the final division: with Y = W V and z = W 1,
+    dY = dO / z and dz = -Σ_c dO_c O_c / z; then the linear part with the augmented upstream [dY, dz]."""
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64); dO = np.asarray(dO, dtype=np.float64)
+    O, den = normalized_forward_dense(Q, K, V, M)
+    dY = dO / den[:, None]
+    dz = -np.sum(dO * O, axis=1) / den
+    Vbar = np.concatenate([V, np.ones((V.shape[0], 1))], axis=1)
+    dQ, dK, dVbar = backward_dense(Q, K, Vbar, np.concatenate([dY, dz[:, None]], axis=1), M)
+    return dQ, dK, dVbar[:, :-1]
+
+
+def normalized_forward_rows(Q, K, V, geo: Geometry, rows):
+    Q = np.asarray(Q, dtype=np.float64); K = np.asarray(K, dtype=np.float64); V = np.asarray(V, dtype=np.float64)
+    out = np.empty((len(rows), V.shape[1]), dtype=np.float64)
+    den = np.empty(len(rows), dtype=np.float64)
+    for k, t in enumerate(rows):
+        w = mask_row(int(t), geo) * (K @ Q[int(t)])
+        den[k] = w.sum()
+        out[k] = (w @ V) / den[k]
+    return out, den
+
+
 # --------------------------------------------------------------------------- VC dimension
 def vc_dimension(M: np.ndarray, limit: int | None = None) -> int:
     """Brute-force VC dimension of the row supports of a 0/1 matrix (Sec. 2, "VC dimension of a mask").
