@@ -33,7 +33,8 @@ import numpy as np  # noqa: E402
 from paper_2609_36062_b200 import replicas, roofline, synth  # noqa: E402
 
 DEFAULT_WORKLOAD = "t16k_d4"
-SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd", "t16k_d4_hashed"]
+SWEEP = ["t4k_d3", "t64k_d1", "t64k_d2", "t64k_d3", "t64k_d4", "t8k_d3_fwdbwd", "t16k_d4_hashed", "t16k_d4_normalized",
+         "t4k_d3_gated", "t4k_d3_gated_fwdbwd"]
 METRIC = "SMat prefill tokens/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant stage per step — the tabulation, one
 # launch of radon_tc_kernel — from an ncu capture of the 8-head copy of the workload (351.3 MB read + 530.1 MB
@@ -123,7 +124,7 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------ helpers
 def workload_config(w: synth.Workload, n_gpus: int):
     return {"workload": w.name, "d": w.d, "batch": w.batch, "heads": w.heads, "T": w.T, "d_k": w.d_k, "d_v": w.d_v,
-            "chunk": w.chunk, "routing": w.routing, "pass": "fwd+bwd (backward reuses the forward's profile/type tables left in the shared workspace)"
+            "chunk": w.chunk, "routing": w.routing, "variant": w.variant, "pass": "fwd+bwd (backward reuses the forward's profile/type tables left in the shared workspace)"
             if w.backward else "fwd", "input_dtype": w.dtype,
             "replicas": n_gpus, "l2": "inputs and tables exceed the 126 MB L2; no flush"}
 
@@ -201,8 +202,9 @@ def make_inputs(w: synth.Workload, torch):
 class Runner:
     def __init__(self, w: synth.Workload, torch, binding, flags=0):
         self.w, self.torch = w, torch
-        if w.backward:  # forward and backward of one step share the workspace: the backward reuses the forward's F, U
+        if w.backward and w.variant == "plain":  # one workspace per step: the backward reuses the forward's F, U
             flags |= binding.FLAG_KEEP_FORWARD_TABLES
+        flags |= {"gated": binding.FLAG_GATED, "normalized": binding.FLAG_NORMALIZED}.get(w.variant, 0)
         self.plan = binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype, flags=flags)
         self.host = make_inputs(w, torch)
         self.dev = {k: v.cuda(non_blocking=True) for k, v in self.host.items()}
@@ -210,6 +212,9 @@ class Runner:
         self.ws = self.plan.workspace(for_backward=w.backward)
         if w.backward:
             self.dQ, self.dK, self.dV = (torch.empty_like(self.dev[x]) for x in ("q", "k", "v"))
+        self.log_a = None
+        if w.variant == "gated":
+            self.log_a = torch.from_numpy(np.stack([synth.log_gates(w, h) for h in range(w.bh)])).cuda()
         self.routing = {}
         if w.routing == "hashed":   # user-supplied routing: int32 cell / type of every token, resident on the device
             g = self.plan.geometry()
@@ -222,12 +227,28 @@ class Runner:
                 self.host_out[nm] = torch.empty_like(self.host[src]).pin_memory()
         torch.cuda.synchronize()
 
+    def run_forward(self, d, O, stream=None):
+        if self.w.variant == "gated":
+            return self.plan.forward_gated(d["q"], d["k"], d["v"], self.log_a, O, self.ws, stream=stream)
+        if self.w.variant == "normalized":
+            return self.plan.forward_normalized(d["q"], d["k"], d["v"], O, self.ws, stream=stream)
+        return self.plan.forward(d["q"], d["k"], d["v"], O, self.ws, stream=stream, **self.routing)
+
+    def run_backward(self, d, outs, stream=None):
+        if self.w.variant == "gated":
+            if getattr(self, "dlog_a", None) is None:
+                self.dlog_a = self.torch.empty_like(self.log_a)
+            return self.plan.backward_gated(d["q"], d["k"], d["v"], self.log_a, d["do"], outs[0], outs[1], outs[2],
+                                            self.dlog_a, self.ws, stream=stream)
+        return self.plan.backward(d["q"], d["k"], d["v"], d["do"], outs[0], outs[1], outs[2], self.ws, stream=stream,
+                                  **self.routing)
+
     def step(self):
         d = self.dev
-        self.plan.forward(d["q"], d["k"], d["v"], self.O, self.ws, **self.routing)
+        self.run_forward(d, self.O)
         n = self.plan.last_launch_count()
         if self.w.backward:
-            self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws, **self.routing)
+            self.run_backward(d, (self.dQ, self.dK, self.dV))
             n += self.plan.last_launch_count()
         return n
 
@@ -262,10 +283,9 @@ class Runner:
                 if i >= 2:
                     s_cmp.wait_event(ev_out[b])     # the results of step i-2 have left these buffers
                 d, o = dev[b], outs[b]
-                self.plan.forward(d["q"], d["k"], d["v"], o["o"], self.ws, stream=s_cmp, **self.routing)
+                self.run_forward(d, o["o"], stream=s_cmp)
                 if w.backward:
-                    self.plan.backward(d["q"], d["k"], d["v"], d["do"], o["dq"], o["dk"], o["dv"], self.ws, stream=s_cmp,
-                                       **self.routing)
+                    self.run_backward(d, (o["dq"], o["dk"], o["dv"]), stream=s_cmp)
                 ev_cmp[b].record(s_cmp)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_cmp[b])
@@ -343,10 +363,10 @@ class Runner:
         acc, order = {}, []
         for _ in range(steps):
             d = self.dev
-            self.plan.forward(d["q"], d["k"], d["v"], self.O, self.ws, **self.routing)
+            self.run_forward(d, self.O)
             recs = self.plan.profile_read()
             if self.w.backward:
-                self.plan.backward(d["q"], d["k"], d["v"], d["do"], self.dQ, self.dK, self.dV, self.ws, **self.routing)
+                self.run_backward(d, (self.dQ, self.dK, self.dV))
                 recs += [(n if n.startswith("bwd_") else "bwd_" + n, t) for n, t in self.plan.profile_read()]
             for n, t in recs:
                 if n not in acc:

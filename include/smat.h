@@ -75,6 +75,9 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
 #define SMAT_FLAG_GATED 64u          /* the plan serves smat_forward_gated / smat_backward_gated: it runs on the fp32-ALU
                                         kernels and its workspace holds λ and the rescaled copies of Q, K, V, dO */
 
+#define SMAT_FLAG_NORMALIZED 128u    /* the plan serves smat_forward_normalized / smat_backward_normalized: its workspace
+                                        also holds the augmented values, the unnormalised rows and their upstream */
+
 /* Sizes of the construction (Sec. 3, "construction of G" and "Scaling with sequence length"). */
 typedef struct {
   int64_t T, c, n, m;  /* sequence length, chunk width, distant = c*floor(T/2c), recent = T - n */
@@ -166,6 +169,24 @@ smat_status smat_forward_routed(const smat_plan* plan, const void* Q, const void
 smat_status smat_backward_routed(const smat_plan* plan, const void* Q, const void* K, const void* V, const void* dO,
                                  void* dQ, void* dK, void* dV, const int32_t* prof, const int32_t* type,
                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * NORMALISED OUTPUT (Sec. 2, Eq. "augmented-kv-state", Eq. "augmented-attention-output"; "backward of the final
+ * division" in the chunking proof).  The value is augmented with a ones column, v̄_j = [v_j; 1], the linear pass runs
+ * once on it, and one division at the end gives o_i = ȳ_{1:p-1} / ȳ_p.  Here the augmented width is the plan's
+ * d_v = p: V carries p - 1 value columns and its LAST column is the normaliser column — the library replaces whatever
+ * the caller left there by one.  O [batch, heads, T, p] receives the normalised values in columns 0 .. p-2 and the
+ * normaliser ȳ_p itself in column p-1.  The caller supplies the (non-negative) features φ = Q, ψ = K; the normalisers
+ * must be positive, as Theorem 2 assumes.
+ * smat_backward_normalized takes the O that the forward returned (it holds the normaliser) and dO of the same shape
+ * (its last column is the upstream of the normaliser output; pass zeros if unused); dV's last column is returned as
+ * zero.  The plan must carry SMAT_FLAG_NORMALIZED.  Otherwise as smat_forward / smat_backward.
+ */
+smat_status smat_forward_normalized(const smat_plan* plan, const void* Q, const void* K, const void* V, void* O,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+smat_status smat_backward_normalized(const smat_plan* plan, const void* Q, const void* K, const void* V, const void* O,
+                                     const void* dO, void* dQ, void* dK, void* dV, void* workspace,
+                                     size_t workspace_bytes, void* cuda_stream);
 
 /*
  * SCALAR-GATED SMat (Sec. 3.2, Eq. "gated"; Lemma "Gated SMat"): the binary mask is replaced by

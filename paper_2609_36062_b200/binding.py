@@ -23,6 +23,7 @@ FLAG_KEEP_FORWARD_TABLES = 8
 FLAG_ALU_TABULATION = 16
 FLAG_D3_SHARED_SUMS = 32
 FLAG_GATED = 64
+FLAG_NORMALIZED = 128
 
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
@@ -31,6 +32,7 @@ EXPORTS = [
     "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step",
     "smat_static_check_status", "smat_debug_timeout_probe", "smat_measure_fadd_rate",
     "smat_forward_routed", "smat_backward_routed", "smat_forward_gated", "smat_backward_gated",
+    "smat_forward_normalized", "smat_backward_normalized",
 ]
 
 
@@ -93,6 +95,10 @@ def load_library() -> ctypes.CDLL:
     lib.smat_forward_gated.restype = i
     lib.smat_backward_gated.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.smat_backward_gated.restype = i
+    lib.smat_forward_normalized.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.smat_forward_normalized.restype = i
+    lib.smat_backward_normalized.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.smat_backward_normalized.restype = i
     lib.smat_routing_indices.argtypes = [vp, vp, vp, vp]
     lib.smat_routing_indices.restype = i
     lib.smat_debug_mask.argtypes = [vp, vp, vp]
@@ -304,6 +310,28 @@ class SmatPlan:
                                       _ptr(ws), ws.numel(), _stream(stream)), "smat_backward")
         return dQ, dK, dV
 
+    # -- normalised output ------------------------------------------------------------------------
+    def forward_normalized(self, Q, K, V, O=None, workspace=None, stream=None):
+        """V: p - 1 value columns and the normaliser column last; O: normalised values and the normaliser last."""
+        _, _, _, dk, dv = self.shape
+        self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
+        O = torch.empty_like(V) if O is None else O
+        ws = self.workspace(False, Q.device) if workspace is None else workspace
+        _check(self.lib.smat_forward_normalized(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(ws), ws.numel(),
+                                                _stream(stream)), "smat_forward_normalized")
+        return O
+
+    def backward_normalized(self, Q, K, V, O, dO, workspace=None, stream=None):
+        _, _, _, dk, dv = self.shape
+        self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
+        self._check_tensor(O, dv, "O"); self._check_tensor(dO, dv, "dO")
+        dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+        ws = self.workspace(True, Q.device) if workspace is None else workspace
+        _check(self.lib.smat_backward_normalized(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(dQ),
+                                                 _ptr(dK), _ptr(dV), _ptr(ws), ws.numel(), _stream(stream)),
+               "smat_backward_normalized")
+        return dQ, dK, dV
+
     # -- scalar-gated variant ---------------------------------------------------------------------
     def _check_gates(self, log_a):
         b, h, T, _, _ = self.shape
@@ -320,12 +348,15 @@ class SmatPlan:
                                            ws.numel(), _stream(stream)), "smat_forward_gated")
         return O
 
-    def backward_gated(self, Q, K, V, log_a, dO, workspace=None, stream=None):
+    def backward_gated(self, Q, K, V, log_a, dO, dQ=None, dK=None, dV=None, dlog_a=None, workspace=None, stream=None):
         _, _, _, dk, dv = self.shape
         self._check_tensor(Q, dk, "Q"); self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
         self._check_tensor(dO, dv, "dO")
         self._check_gates(log_a)
-        dQ, dK, dV, dla = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V), torch.empty_like(log_a)
+        dQ = torch.empty_like(Q) if dQ is None else dQ
+        dK = torch.empty_like(K) if dK is None else dK
+        dV = torch.empty_like(V) if dV is None else dV
+        dla = torch.empty_like(log_a) if dlog_a is None else dlog_a
         ws = self.workspace(True, Q.device) if workspace is None else workspace
         _check(self.lib.smat_backward_gated(self.handle, _ptr(Q), _ptr(K), _ptr(V), _ptr(log_a), _ptr(dO), _ptr(dQ),
                                             _ptr(dK), _ptr(dV), _ptr(dla), _ptr(ws), ws.numel(), _stream(stream)),

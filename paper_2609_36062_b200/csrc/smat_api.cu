@@ -24,6 +24,7 @@ struct smat_plan {
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
   size_t off_plist, off_poffs, off_tlist, off_toffs;   // token lists of user-supplied routing (int32)
   size_t off_lam, off_dlam, off_gq, off_gk, off_glr, off_gdo, off_gv, off_gvlr;   // gated variant (SMAT_FLAG_GATED)
+  size_t off_nv, off_ny, off_ndy;   // normalised output (SMAT_FLAG_NORMALIZED): V̄, ȳ and the upstream of the linear pass
   bool tc;             // tensor-core kernels for the causal branch
   bool u_bf16;         // forward keeps the type table U in bf16 and reads it with the tensor-core typed read
   bool pool_tc;        // forward pools the profile table on the tensor cores (enough tokens per profile)
@@ -408,7 +409,11 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->off_gq = off;     off = align_up(off + gated * (size_t)pl->bh * T * d_k * esz);
   pl->off_gk = off;     off = align_up(off + gated * (size_t)pl->bh * T * d_k * esz);
   pl->off_glr = off;    off = align_up(off + gated * (size_t)pl->bh * T * d_k * esz);
+  const size_t normd = (flags & SMAT_FLAG_NORMALIZED) ? 1 : 0;
+  pl->off_nv = off;     off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
+  pl->off_ny = off;     off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
   pl->off_fwd_end = off;
+  pl->off_ndy = off;    off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
   pl->off_dlam = off;   off = align_up(off + gated * (size_t)pl->bh * T * 4);
   pl->off_gdo = off;    off = align_up(off + gated * (size_t)pl->bh * T * d_v * esz);
   pl->off_gv = off;     off = align_up(off + gated * (size_t)pl->bh * T * d_v * esz);
@@ -736,6 +741,54 @@ smat_status gated_check(const smat_plan* pl, const void* log_a, void* ws, size_t
 }  // namespace
 
 extern "C" {
+
+smat_status smat_forward_normalized(const smat_plan* pl, const void* Q, const void* K, const void* V, void* O,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!pl) return SMAT_ERR_NULL;
+  if (!(pl->flags & SMAT_FLAG_NORMALIZED)) return SMAT_ERR_UNSUPPORTED;
+  if (!Q || !K || !V || !O || !workspace) return SMAT_ERR_NULL;
+  char* ws = static_cast<char*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (workspace_bytes < smat_workspace_bytes(pl, 0)) return SMAT_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255) || misaligned(V) || misaligned(O)) return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
+  const int bf = pl->dtype == SMAT_BF16;
+  const int64_t rows = (int64_t)pl->bh * pl->T;
+  // v̄ = [v; 1]: the last value column is the normaliser column (Eq. "augmented-kv-state")
+  if (smat_launch_normalize_step(0, V, nullptr, ws + pl->off_nv, bf, pl->p, rows, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  smat_status s = forward_impl(pl, Q, K, ws + pl->off_nv, ws + pl->off_ny, nullptr, nullptr, workspace, workspace_bytes,
+                               cuda_stream);
+  if (s != SMAT_OK) return s;
+  // the single final division (Eq. "augmented-attention-output")
+  if (smat_launch_normalize_step(1, ws + pl->off_ny, nullptr, O, bf, pl->p, rows, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  pl->launches += 2;
+  return SMAT_OK;
+}
+
+smat_status smat_backward_normalized(const smat_plan* pl, const void* Q, const void* K, const void* V, const void* O,
+                                     const void* dO, void* dQ, void* dK, void* dV, void* workspace,
+                                     size_t workspace_bytes, void* cuda_stream) {
+  if (!pl) return SMAT_ERR_NULL;
+  if (!(pl->flags & SMAT_FLAG_NORMALIZED)) return SMAT_ERR_UNSUPPORTED;
+  if (!Q || !K || !V || !O || !dO || !dQ || !dK || !dV || !workspace) return SMAT_ERR_NULL;
+  char* ws = static_cast<char*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (workspace_bytes < smat_workspace_bytes(pl, 1)) return SMAT_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255) || misaligned(V) || misaligned(O) || misaligned(dO) || misaligned(dV))
+    return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
+  const int bf = pl->dtype == SMAT_BF16;
+  const int64_t rows = (int64_t)pl->bh * pl->T;
+  if (smat_launch_normalize_step(0, V, nullptr, ws + pl->off_nv, bf, pl->p, rows, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  // backward of the final division, then the linear pass with the augmented upstream
+  if (smat_launch_normalize_step(2, O, dO, ws + pl->off_ndy, bf, pl->p, rows, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  smat_status s = backward_impl(pl, Q, K, ws + pl->off_nv, ws + pl->off_ndy, dQ, dK, dV, nullptr, nullptr, workspace,
+                                workspace_bytes, cuda_stream);
+  if (s != SMAT_OK) return s;
+  if (smat_launch_normalize_step(3, nullptr, nullptr, dV, bf, pl->p, rows, st) != cudaSuccess) return SMAT_ERR_LAUNCH;
+  pl->launches += 3;
+  return SMAT_OK;
+}
 
 smat_status smat_forward_gated(const smat_plan* pl, const void* Q, const void* K, const void* V, const float* log_a,
                                void* O, void* workspace, size_t workspace_bytes, void* cuda_stream) {

@@ -154,3 +154,75 @@ cudaError_t smat_launch_gate_dlam(const void* Q, const void* dQ, const void* K, 
                                                     rows);
   return cudaGetLastError();
 }
+
+// ---- normalised output (Sec. 2: augmented value v̄ = [v; 1], one final division) ------------------------------------
+namespace {
+
+// V̄ = V with its last column set to one.
+template <typename T>
+__global__ void augment_value_kernel(const T* __restrict__ V, T* __restrict__ Vbar, int p, int64_t rows) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * p) return;
+  Vbar[idx] = (int)(idx % p) == p - 1 ? (T)1.0f : V[idx];
+}
+
+// O = ȳ_{1:p-1} / ȳ_p, and the normaliser ȳ_p itself in the last column.  One warp per row.
+template <typename T>
+__global__ void normalize_rows_kernel(const T* __restrict__ Y, T* __restrict__ O, int p, int64_t rows) {
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
+  if (row >= rows) return;
+  const int lane = threadIdx.x & 31;
+  const float den = (float)Y[row * p + p - 1];
+  const float inv = 1.0f / den;
+  for (int i = lane; i < p; i += 32) O[row * p + i] = i == p - 1 ? (T)den : (T)((float)Y[row * p + i] * inv);
+}
+
+// Upstream of the linear pass from the upstream of the normalised output (the backward of the final division):
+//   dȳ_c = dO_c / z (c < p-1),   dȳ_p = dO_p - Σ_{c<p-1} dO_c O_c / z,   z = the normaliser kept in O's last column.
+template <typename T>
+__global__ void normalize_adjoint_kernel(const T* __restrict__ O, const T* __restrict__ dO, T* __restrict__ dY, int p,
+                                         int64_t rows) {
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
+  if (row >= rows) return;
+  const int lane = threadIdx.x & 31;
+  const float inv = 1.0f / (float)O[row * p + p - 1];
+  float dot = 0.f;
+  for (int i = lane; i < p - 1; i += 32) {
+    const float g = (float)dO[row * p + i];
+    dot += g * (float)O[row * p + i];
+    dY[row * p + i] = (T)(g * inv);
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, d);
+  if (lane == 0) dY[row * p + p - 1] = (T)((float)dO[row * p + p - 1] - dot * inv);
+}
+
+// The ones column of V̄ is a constant: its gradient is dropped.
+template <typename T>
+__global__ void clear_last_column_kernel(T* __restrict__ dV, int p, int64_t rows) {
+  const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (row < rows) dV[row * p + p - 1] = (T)0.0f;
+}
+
+template <typename T>
+cudaError_t normalize_step(int step, const void* a, const void* b, void* out, int p, int64_t rows, cudaStream_t st) {
+  const unsigned warp_blocks = (unsigned)((rows * 32 + 255) / 256);
+  if (step == 0)
+    augment_value_kernel<T><<<(unsigned)((rows * p + 255) / 256), 256, 0, st>>>(static_cast<const T*>(a), static_cast<T*>(out), p, rows);
+  else if (step == 1)
+    normalize_rows_kernel<T><<<warp_blocks, 256, 0, st>>>(static_cast<const T*>(a), static_cast<T*>(out), p, rows);
+  else if (step == 2)
+    normalize_adjoint_kernel<T><<<warp_blocks, 256, 0, st>>>(static_cast<const T*>(a), static_cast<const T*>(b),
+                                                             static_cast<T*>(out), p, rows);
+  else
+    clear_last_column_kernel<T><<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(static_cast<T*>(out), p, rows);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// step 0: out = V̄ from a = V;  1: out = O from a = ȳ;  2: out = dȳ from a = O, b = dO;  3: out (dV) last column := 0
+cudaError_t smat_launch_normalize_step(int step, const void* a, const void* b, void* out, int bf16, int p, int64_t rows,
+                                       cudaStream_t st) {
+  return bf16 ? normalize_step<__nv_bfloat16>(step, a, b, out, p, rows, st) : normalize_step<float>(step, a, b, out, p, rows, st);
+}

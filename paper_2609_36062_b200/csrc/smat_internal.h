@@ -171,6 +171,9 @@ cudaError_t smat_launch_gated_scan(float* S, const float* lam, int64_t state_ele
                                    int64_t lo0, int64_t hi0, int64_t lo1, int64_t hi1, int reverse, cudaStream_t st);
 cudaError_t smat_launch_gate_dlam(const void* Q, const void* dQ, const void* K, const void* dK, float* dlam, int bf16,
                                   int dim, int64_t T, int bh, cudaStream_t st);
+// Normalised output (Sec. 2): elementwise steps around the linear pass (see smat_gated.cu).
+cudaError_t smat_launch_normalize_step(int step, const void* a, const void* b, void* out, int bf16, int p, int64_t rows,
+                                       cudaStream_t st);
 // Token lists of user-supplied routing: prof [bh][n] (cells in [0, P)) and type [bh][m] (types in [0, B)) -> CSR lists
 // (offsets [bh][G + 1], token positions [bh][count], ascending inside a group).  Keys out of range are dropped.
 int64_t smat_routing_max_groups();

@@ -10,6 +10,7 @@ Recipe.  Every (tensor, batch·head) pair owns its own Philox stream keyed by
   * "scaled":     Q, K, V iid N(0,1)/sqrt(d)                         (fp32 small case)
   * "normalised": Q, K iid N(0,1)/sqrt(d_k), then every row L2-normalised in fp32;
                   V iid N(0,1)
+  * "positive":   Q, K iid |N(0,1)|/sqrt(d_k) (non-negative features for the normalised output); V iid N(0,1)
   * dO iid N(0,1)
 bf16 storage rounds the fp32 values once, to nearest even; the oracle widens exactly
 those rounded values to fp64.
@@ -38,6 +39,7 @@ class Workload:
     seed: int
     backward: bool = False
     routing: str = "positional"   # or "hashed": prof / type arrays drawn by a fixed random hash (user-supplied routing)
+    variant: str = "plain"        # "gated": scalar per-token gates; "normalized": augmented ones column and division
 
     @property
     def bh(self) -> int:
@@ -69,6 +71,12 @@ WORKLOADS = {
     "t8k_d3_fwdbwd": Workload("t8k_d3_fwdbwd", 3, 8, 16, 8192, 128, 128, 64, "bf16", "normalised", 4, True),
     # the 16 K configuration under user-supplied routing: every token hashed to a uniformly random cell / type
     "t16k_d4_hashed": Workload("t16k_d4_hashed", 4, 2, 16, 16384, 128, 128, 128, "bf16", "normalised", 2, False, "hashed"),
+    # the variants of the "next" list on benchmark-shaped inputs
+    "t4k_d3_gated":  Workload("t4k_d3_gated", 3, 4, 8, 4096, 128, 128, 64, "bf16", "normalised", 1, False, "positional", "gated"),
+    "t4k_d3_gated_fwdbwd": Workload("t4k_d3_gated_fwdbwd", 3, 4, 8, 4096, 128, 128, 64, "bf16", "normalised", 1, True,
+                                    "positional", "gated"),
+    "t16k_d4_normalized": Workload("t16k_d4_normalized", 4, 2, 16, 16384, 128, 128, 128, "bf16", "positive", 2, False,
+                                   "positional", "normalized"),
     # cached decoding: 128 sequences of 16 heads, 2 K horizon (132 type states + one running state per head; the
     # running states alone, 134 MB, exceed L2)
     "decode_t2k_d3": Workload("decode_t2k_d3", 3, 128, 16, 2048, 128, 128, 64, "bf16", "normalised", 5),
@@ -101,6 +109,8 @@ def head_tensor(w: Workload, tensor: str, head: int, T: int | None = None) -> np
         return x
     if w.recipe == "scaled":
         return x * np.float32(1.0 / np.sqrt(dim))
+    if w.recipe == "positive":      # non-negative features (normalised output): half-normal Q, K; V iid N(0,1)
+        return (np.abs(x) * np.float32(1.0 / np.sqrt(dim))).astype(np.float32) if tensor in ("q", "k") else x
     if tensor in ("q", "k"):
         x = x * np.float32(1.0 / np.sqrt(dim))
         norm = np.sqrt(np.sum(x * x, axis=1, keepdims=True, dtype=np.float32))
@@ -150,3 +160,9 @@ def hashed_types(w: Workload, head: int, m: int, B: int) -> np.ndarray:
     """A fixed random hash of the recent tokens of one head into B types (int32 [m]), uniform."""
     g = np.random.Generator(np.random.Philox(key=(int(w.seed) << 40) ^ (9 << 32) ^ int(head)))
     return g.integers(0, B, size=m, dtype=np.int64).astype(np.int32)
+
+
+def log_gates(w: Workload, head: int, lo: float = 0.9) -> np.ndarray:
+    """Per-token log-gates of one head (fp32 [T]): gates uniform in [lo, 1)."""
+    g = np.random.Generator(np.random.Philox(key=(int(w.seed) << 40) ^ (10 << 32) ^ int(head)))
+    return np.log(g.uniform(lo, 1.0, size=w.T)).astype(np.float32)
