@@ -333,6 +333,12 @@ smat_status smat_decode_begin(const smat_plan* plan, const void* K, const void* 
 smat_status smat_decode_step(const smat_plan* plan, const void* q, const void* k, const void* v, int64_t t, void* o,
                              void* cache, size_t cache_bytes, void* cuda_stream);
 
+/* Host-only self-check (the paper has no counterpart): 1 when, for field size q, the shared-memory map of every launch
+ * shape of the tensor-core tabulation kernel (ring slots, extra-class rows, output-row table, barrier words) is
+ * disjoint and inside the allocation, and no load box or staged tile can leave its slot; 0 otherwise.  The launcher
+ * makes the same check before every launch. */
+int smat_debug_tabulation_layout_ok(int q);
+
 /* Number of kernels the last smat_forward / smat_backward on this plan launched (host counter). */
 int smat_last_launch_count(const smat_plan* plan);
 

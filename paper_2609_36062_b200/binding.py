@@ -32,7 +32,7 @@ EXPORTS = [
     "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step",
     "smat_static_check_status", "smat_debug_timeout_probe", "smat_measure_fadd_rate",
     "smat_forward_routed", "smat_backward_routed", "smat_forward_gated", "smat_backward_gated",
-    "smat_forward_normalized", "smat_backward_normalized",
+    "smat_forward_normalized", "smat_backward_normalized", "smat_debug_tabulation_layout_ok",
 ]
 
 
@@ -99,6 +99,8 @@ def load_library() -> ctypes.CDLL:
     lib.smat_forward_normalized.restype = i
     lib.smat_backward_normalized.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.smat_backward_normalized.restype = i
+    lib.smat_debug_tabulation_layout_ok.argtypes = [i]
+    lib.smat_debug_tabulation_layout_ok.restype = i
     lib.smat_routing_indices.argtypes = [vp, vp, vp, vp]
     lib.smat_routing_indices.restype = i
     lib.smat_debug_mask.argtypes = [vp, vp, vp]

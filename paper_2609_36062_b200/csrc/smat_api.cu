@@ -990,6 +990,8 @@ smat_status smat_check_status(const smat_plan* pl, const void* workspace, void* 
 
 int smat_last_launch_count(const smat_plan* pl) { return pl ? pl->launches : 0; }
 
+int smat_debug_tabulation_layout_ok(int q) { return smat_tabulate_tc_layout_ok(q); }
+
 size_t smat_decode_cache_bytes(const smat_plan* pl) {
   if (!pl) return 0;
   return decode_table_bytes(pl) + (size_t)pl->bh * pl->rp * sizeof(float);

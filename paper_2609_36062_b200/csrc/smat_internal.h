@@ -150,6 +150,7 @@ cudaError_t smat_launch_tabulate_d3_regs(const void* in, void* out, const SmatGe
 // bf16 -> fp32 copy of a table (debug export).
 // Tabulation on the tensor cores (bf16 tables; d = 3, 4 with a prime small enough for a resident Radon matrix).
 int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems);
+int smat_tabulate_tc_layout_ok(int q);   // host-only self-check of the kernel's shared-memory map for prime q
 int64_t smat_tabulate_tc_scratch_rows(const SmatGeo& geo);
 int64_t smat_tabulate_tc_scratch_elems(const SmatGeo& geo, int64_t state_elems, int bh);
 cudaError_t smat_launch_tabulate_tc(const void* in, void* out, void* scratch, const SmatGeo& geo, int64_t state_elems,

@@ -792,6 +792,29 @@ bool radon_shape(int q, int transpose, int in_has_extra, int count_out, RadonSha
   return true;
 }
 
+// The shared-memory map of radon_tc_kernel for a shape, checked on the host before every launch: ring slots, the
+// per-slot extra-class rows (tile stores only), the output-row table and the barrier words must be disjoint and inside
+// the allocation; nothing the copy engine or a thread writes for a slot may leave the slot.
+//   [0, ring * slot)                      ring slots, slot = 2 halves of sr rows x 128 bytes (1024-byte aligned: sr % 16 == 0)
+//   [.., + ring * mini)                   extra-class rows per slot (two halves of mini / 2)
+//   [.., + 2 * 128 * 4)                   output-row table
+//   [.., + (4 ring + 2 MAX_ACC + 1) * 8 + 8)   barriers, the tensor-memory slot word, the abort flag
+bool radon_layout_ok(int q, const RadonShape& sh, int ring, int mini_bytes, int tma_out, int in_has_extra, int smem) {
+  const int slot = sh.sr * 256, half = sh.sr * 128;
+  const int bars = (4 * ring + 2 * MAX_ACC + 1) * 8 + 8;
+  bool ok = sh.sr % 16 == 0 && sh.sr <= TILE_ROWS && ring >= sh.nslots;           // the scratch copy of R: 128 rows x kt bf16
+  ok = ok && sh.nslots == sh.nreg + (in_has_extra ? 1 : 0) && sh.nreg * sh.sps >= q;
+  ok = ok && q * sh.sps * 128 <= half && q * 128 <= half;                         // a load box (lines or extra class) per half
+  ok = ok && ((sh.nslots * sh.sr / 2 + 31) & ~31) + 2 * 128 <= 512;               // R columns and two accumulators
+  ok = ok && sh.rows_pp <= TILE_ROWS && sh.parts * sh.rows_pp + sh.alu_rows >= 0;
+  if (tma_out) {   // the tile is written into the item's first slot: one 128-byte row per output index of the part
+    ok = ok && sh.rows_pp <= sh.sr;
+    ok = ok && (mini_bytes == 0 || (mini_bytes % 2048 == 0 && mini_bytes / 2 >= q * 128));
+  }
+  ok = ok && 1023 + ring * (slot + mini_bytes) + 2 * TILE_ROWS * 4 + bars <= smem && smem <= 227 * 1024;
+  return ok;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -885,6 +908,7 @@ cudaError_t launch_radon(int q, int transpose, int nph, const StageSpec* sp, int
       smem = ring * (slot + mini) + TILE_ROWS * 8 + 512 + 1024;
     }
   }
+  if (!radon_layout_ok(q, sh, prm.ring, prm.mini_bytes, prm.tma_out, in_has_extra, smem)) return cudaErrorInvalidConfiguration;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -971,6 +995,29 @@ int smat_tabulate_tc_supported(const SmatGeo& geo, int64_t state_elems) {
   const int qq = geo.q * geo.q;
   RadonShape a, b;
   return radon_shape(geo.q, 0, 0, qq + geo.q, &a) && radon_shape(geo.q, 1, 1, qq, &b) ? 1 : 0;
+}
+
+// Host-only: 1 when the shared-memory map of every launch shape this prime can take (both directions, with and without
+// the extra class on the input, with the tile-store variant where the launcher would pick it) passes radon_layout_ok.
+int smat_tabulate_tc_layout_ok(int q) {
+  const int qq = q * q;
+  for (int transpose = 0; transpose < 2; ++transpose)
+    for (int extra = 0; extra < 2; ++extra) {
+      RadonShape sh;
+      const int count_out = (transpose ? !extra : extra) ? qq + q : qq;   // forward stages grow, transposed ones shrink
+      for (int co : {count_out, qq, qq + q}) {
+        if (!radon_shape(q, transpose, extra, co, &sh)) continue;
+        if (!radon_layout_ok(q, sh, sh.ring, 0, 0, extra, sh.smem)) return 0;
+        if (!transpose && sh.nslots == 1 && sh.sr == TILE_ROWS && sh.parts == 1) {
+          const int mini = 2 * ((q + 7) & ~7) * 128, slot = sh.sr * 256;
+          int ring = (227 * 1024 - 1024 - 512 - TILE_ROWS * 8) / (slot + mini);
+          if (ring > sh.ring) ring = sh.ring;
+          if (ring >= 4 && !radon_layout_ok(q, sh, ring, mini, 1, extra, ring * (slot + mini) + TILE_ROWS * 8 + 512 + 1024))
+            return 0;
+        }
+      }
+    }
+  return 1;
 }
 
 // Rows (of state_elems bf16 each, per head) of the intermediate table the d = 4 stages exchange.

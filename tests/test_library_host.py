@@ -135,3 +135,10 @@ def test_launching_calls_report_a_missing_sm100_device():
     assert lib.smat_debug_timeout_probe(256, 1000, None) == 7
     assert "sm_100" in binding.status_string(7)
     lib.smat_plan_destroy(h)
+
+
+@pytest.mark.parametrize("q", [2, 3, 5, 7, 11, 13, 17, 19, 23])
+def test_tabulation_kernel_shared_memory_map_is_disjoint(q):
+    """Ring slots, per-slot extra rows, the output-row table and the barrier words of the tensor-core tabulation kernel
+    never overlap and no load box or staged tile leaves its slot, for every launch shape of every prime it accepts."""
+    assert binding.load_library().smat_debug_tabulation_layout_ok(q) == 1
