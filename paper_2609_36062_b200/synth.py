@@ -65,6 +65,7 @@ WORKLOADS = {
     "t16k_d4_h8":    Workload("t16k_d4_h8", 4, 1, 8, 16384, 128, 128, 128, "bf16", "normalised", 2),
     "t64k_d4_h1":    Workload("t64k_d4_h1", 4, 1, 1, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t64k_d3_h2":    Workload("t64k_d3_h2", 3, 1, 2, 65536, 128, 128, 128, "bf16", "normalised", 3),
+    "t64k_d3_h4":    Workload("t64k_d3_h4", 3, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t8k_d3_h8":     Workload("t8k_d3_h8", 3, 1, 8, 8192, 128, 128, 64, "bf16", "normalised", 4),
     "t64k_d1_h4":    Workload("t64k_d1_h4", 1, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t64k_d2_h4":    Workload("t64k_d2_h4", 2, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
