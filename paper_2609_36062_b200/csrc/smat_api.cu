@@ -23,6 +23,7 @@ struct smat_plan {
   size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_W, off_fwd_end;
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
   size_t off_plist, off_poffs, off_tlist, off_toffs;   // token lists of user-supplied routing (int32)
+  size_t off_sin_tiles;   // KEEP_FORWARD_TABLES on tensor-core plans: the bf16 state entering every tile, left by the forward
   size_t off_lam, off_dlam, off_gq, off_gk, off_glr, off_gdo, off_gv, off_gvlr;   // gated variant (SMAT_FLAG_GATED)
   size_t off_nv, off_ny, off_ndy;   // normalised output (SMAT_FLAG_NORMALIZED): V̄, ȳ and the upstream of the linear pass
   bool tc;             // tensor-core kernels for the causal branch
@@ -37,6 +38,7 @@ struct smat_plan {
   bool fbar_bf16;      // the per-profile adjoint states (transposed tabulation) are kept in bf16
   mutable int launches;
   mutable bool tile_states;       // the last call left one bf16 incoming state per 128-token tile at off_sin
+  mutable bool kept_tile_states;  // the last forward left them at off_sin_tiles for the backward (KEEP_FORWARD_TABLES)
   // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
   mutable bool profiling;
   mutable cudaEvent_t events[SMAT_MAX_STAGES + 1];
@@ -353,7 +355,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->batch = batch; pl->heads = heads; pl->bh = batch * heads;
   pl->r = d_k; pl->p = d_v; pl->T = T; pl->c = chunk; pl->NC = T / chunk;
   pl->dtype = dtype; pl->flags = flags; pl->rp = (int64_t)d_k * d_v; pl->launches = 0;
-  pl->profiling = false; pl->stages = 0; pl->tile_states = false;
+  pl->profiling = false; pl->stages = 0; pl->tile_states = false; pl->kept_tile_states = false;
   smat_status s = build_geometry(&pl->geo, T, chunk, d, q_override);
   if (s != SMAT_OK) { delete pl; return s; }
   const SmatGeo& g = pl->geo;
@@ -397,6 +399,8 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->off_acc = off;    off = align_up(off + (size_t)pl->bh * T * wide * sizeof(float));
   pl->off_tileA = off;  off = align_up(off + tiles);
   pl->off_W = off;      off = align_up(off + (pl->tab_tc ? (size_t)smat_tabulate_tc_scratch_elems(g, pl->rp, pl->bh) * 2 : 0));
+  pl->off_sin_tiles = off;
+  off = align_up(off + (pl->tc && (flags & SMAT_FLAG_KEEP_FORWARD_TABLES) ? (size_t)pl->bh * (T / 128) * entries * 2 : 0));
   const bool lists = !g.dense_G;
   pl->off_plist = off;  off = align_up(off + (lists ? (size_t)pl->bh * g.n * 4 : 0));
   pl->off_poffs = off;  off = align_up(off + (lists ? (size_t)pl->bh * (g.P + 1) * 4 : 0));
@@ -543,6 +547,7 @@ smat_status forward_impl(const smat_plan* pl, const void* Q, const void* K, cons
         state_read(cx, "read_type", SMAT_GM_TYPE, Q, cx.f(pl->off_U), 0, nullptr, ylr, nullptr);
     }
     pl->tile_states = L < 2;
+    pl->kept_tile_states = false;
     if (L >= 2) {  // steps 5-7, two-level: segment totals, scan of the totals, fused per-segment output
       float* seg = cx.f(pl->off_sin);
       int nseg0 = 0, nseg1 = 0;
@@ -550,8 +555,11 @@ smat_status forward_impl(const smat_plan* pl, const void* Q, const void* K, cons
       const int64_t nseg = nseg0 + nseg1;
       SMAT_TRY(cx, "segment_state_tc", smat_launch_segment_state_tc(K, V, seg, tiles0, tiles1, nseg0, nseg1, pl->bh, status, cx.st));
       SMAT_TRY(cx, "segment_scan", smat_launch_scan(seg, pl->rp, nseg, pl->bh, 0, nseg0, nseg0, nseg, 0, cx.st));
+      const bool keep = (pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES) != 0;   // a backward will want the per-tile states
       SMAT_TRY(cx, "segment_output_tc", smat_launch_segment_output_tc(Q, K, V, seg, ylr, lr ? pl->geo.n : pl->T, O,
-                                                                       tiles0, tiles1, nseg0, nseg1, pl->bh, status, cx.st));
+                                                                       tiles0, tiles1, nseg0, nseg1, pl->bh, status, cx.st,
+                                                                       keep ? cx.ws + pl->off_sin_tiles : nullptr));
+      pl->kept_tile_states = keep;
     } else {
       SMAT_TRY(cx, "chunk_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, pl->geo.n,
                                                                lr ? 0 : 1, 0, status, cx.st));   // steps 5-6
@@ -596,7 +604,10 @@ smat_status backward_impl(const smat_plan* pl, const void* Q, const void* K, con
     // that each within-chunk adjoint adds to its rows.
     int* status = reinterpret_cast<int*>(cx.ws + pl->off_status);
     float* lrbuf = cx.f(pl->off_acc);
-    pl->tile_states = true;
+    // With KEEP_FORWARD_TABLES the preceding forward has left the state entering every tile: no second scan of K, V
+    const bool kept = (pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES) && pl->kept_tile_states;
+    void* sin_tiles = cx.ws + (kept ? pl->off_sin_tiles : pl->off_sin);
+    pl->tile_states = !kept;
     const SmatGroupSpec types = group(cx, SMAT_GM_TYPE), profs = group(cx, SMAT_GM_PROFILE);
     const int64_t n = pl->geo.n;
     if (lr) {
@@ -615,41 +626,47 @@ smat_status backward_impl(const smat_plan* pl, const void* Q, const void* K, con
       else
         tabulate(cx, "bwd_tabulate_t", cx.f(pl->off_ubar), cx.f(pl->off_fbar), 1, pl->geo.D == 2 && pl->fbar_bf16);
       // per-tile states
-      SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 0, 0, status, cx.st));
+      if (!kept)
+        SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, sin_tiles, pl->T, pl->bh, n, 0, 0, status, cx.st));
       SMAT_TRY(cx, "bwd_suffix_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 0, 1, status, cx.st));
       // dQ: recent rows add U_type dO
-      zero_unrouted(cx, SMAT_GM_TYPE, lrbuf, 512);
+      // (the rows travel as bf16 where the tensor-core read writes them: rounded once, added in fp32 by the tile kernel)
+      zero_unrouted(cx, SMAT_GM_TYPE, lrbuf, pl->u_bf16 ? 256 : 512);
       if (pl->u_bf16)
-        SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, lrbuf, nullptr, 1, types, pl->geo.B,
+        SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, lrbuf, lrbuf, 1, types, pl->geo.B,
                                                                  pl->T, pl->bh, status, cx.st));
       else
         state_read(cx, "bwd_dq_type", SMAT_GM_TYPE, dO, cx.f(pl->off_U), 1, nullptr, lrbuf, nullptr);
-      SMAT_TRY(cx, "bwd_dq_tile_tc", smat_launch_chunk_adjoint_tc(0, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
-                                                                  lrbuf, n, pl->T, dQ, pl->T, pl->bh, status, cx.st));
+      SMAT_TRY(cx, "bwd_dq_tile_tc", smat_launch_chunk_adjoint_tc(0, Q, K, V, dO, sin_tiles, cx.ws + pl->off_dbar,
+                                                                  lrbuf, n, pl->T, dQ, pl->T, pl->bh, status, cx.st,
+                                                                  pl->u_bf16 ? 1 : 0));
       // dK: distant rows add F̄_prof v
-      zero_unrouted(cx, SMAT_GM_PROFILE, lrbuf, 512);
+      zero_unrouted(cx, SMAT_GM_PROFILE, lrbuf, fbar_is_bf16 ? 256 : 512);
       if (fbar_is_bf16)
-        SMAT_TRY(cx, "bwd_dk_profile_tc", smat_launch_state_read_tc(V, cx.ws + pl->off_fbar, lrbuf, nullptr, 1, profs, pl->geo.P,
+        SMAT_TRY(cx, "bwd_dk_profile_tc", smat_launch_state_read_tc(V, cx.ws + pl->off_fbar, lrbuf, lrbuf, 1, profs, pl->geo.P,
                                                                     pl->T, pl->bh, status, cx.st));
       else
         state_read(cx, "bwd_dk_profile", SMAT_GM_PROFILE, V, cx.f(pl->off_fbar), 1, nullptr, lrbuf, nullptr);
-      SMAT_TRY(cx, "bwd_dk_tile_tc", smat_launch_chunk_adjoint_tc(1, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
-                                                                  lrbuf, 0, n, dK, pl->T, pl->bh, status, cx.st));
+      SMAT_TRY(cx, "bwd_dk_tile_tc", smat_launch_chunk_adjoint_tc(1, Q, K, V, dO, sin_tiles, cx.ws + pl->off_dbar,
+                                                                  lrbuf, 0, n, dK, pl->T, pl->bh, status, cx.st,
+                                                                  fbar_is_bf16 ? 1 : 0));
       // dV: distant rows add F̄_profᵀ k
-      zero_unrouted(cx, SMAT_GM_PROFILE, lrbuf, 512);
+      zero_unrouted(cx, SMAT_GM_PROFILE, lrbuf, fbar_is_bf16 ? 256 : 512);
       if (fbar_is_bf16)
-        SMAT_TRY(cx, "bwd_dv_profile_tc", smat_launch_state_read_tc(K, cx.ws + pl->off_fbar, lrbuf, nullptr, 0, profs, pl->geo.P,
+        SMAT_TRY(cx, "bwd_dv_profile_tc", smat_launch_state_read_tc(K, cx.ws + pl->off_fbar, lrbuf, lrbuf, 0, profs, pl->geo.P,
                                                                     pl->T, pl->bh, status, cx.st));
       else
         state_read(cx, "bwd_dv_profile", SMAT_GM_PROFILE, K, cx.f(pl->off_fbar), 0, nullptr, lrbuf, nullptr);
-      SMAT_TRY(cx, "bwd_dv_tile_tc", smat_launch_chunk_adjoint_tc(2, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar,
-                                                                  lrbuf, 0, n, dV, pl->T, pl->bh, status, cx.st));
+      SMAT_TRY(cx, "bwd_dv_tile_tc", smat_launch_chunk_adjoint_tc(2, Q, K, V, dO, sin_tiles, cx.ws + pl->off_dbar,
+                                                                  lrbuf, 0, n, dV, pl->T, pl->bh, status, cx.st,
+                                                                  fbar_is_bf16 ? 1 : 0));
     } else {
-      SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, cx.ws + pl->off_sin, pl->T, pl->bh, n, 1, 0, status, cx.st));
+      if (!kept)
+        SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, sin_tiles, pl->T, pl->bh, n, 1, 0, status, cx.st));
       SMAT_TRY(cx, "bwd_suffix_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 1, 1, status, cx.st));
       for (int which = 0; which < 3; ++which)
         SMAT_TRY(cx, which == 0 ? "bwd_dq_tile_tc" : (which == 1 ? "bwd_dk_tile_tc" : "bwd_dv_tile_tc"),
-                 smat_launch_chunk_adjoint_tc(which, Q, K, V, dO, cx.ws + pl->off_sin, cx.ws + pl->off_dbar, lrbuf, 0, 0,
+                 smat_launch_chunk_adjoint_tc(which, Q, K, V, dO, sin_tiles, cx.ws + pl->off_dbar, lrbuf, 0, 0,
                                               which == 0 ? dQ : (which == 1 ? dK : dV), pl->T, pl->bh, status, cx.st));
     }
     pl->launches = cx.launches;

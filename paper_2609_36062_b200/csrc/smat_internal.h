@@ -123,7 +123,7 @@ cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf
 cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K, const void* V, const void* dO,
                                          const void* Sin_bf16, const void* Dbar_bf16, const float* addend,
                                          int64_t add_lo, int64_t add_hi, void* Out, int64_t T, int bh, int* status,
-                                         cudaStream_t st);
+                                         cudaStream_t st, int addend_bf16 = 0);
 // O_b = Q_b S_in[b] + tril(Q_b K_bᵀ) V_b (+ ylr rows for tokens >= n_lr).
 cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
                                         const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,
@@ -191,4 +191,5 @@ cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* to
                                          int nseg0, int nseg1, int bh, int* status, cudaStream_t st);
 cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const void* V, const float* seg_in,
                                           const void* ylr_bf16, int64_t n_lr, void* O, int64_t tiles0, int64_t tiles1,
-                                          int nseg0, int nseg1, int bh, int* status, cudaStream_t st);
+                                          int nseg0, int nseg1, int bh, int* status, cudaStream_t st,
+                                          void* sin_tiles = nullptr);

@@ -173,7 +173,8 @@ struct TileParams {
   int64_t T;
   int NC;
   int64_t add_lo, add_hi;  // rows add_lo <= t < add_hi of every head add `addend`
-  const float* addend;     // [bh][T][128] fp32
+  const float* addend;     // [bh][T][128] fp32, or
+  const __nv_bfloat16* addend16;   // the same rows in bf16 (when non-null)
   __nv_bfloat16* Out;      // [bh][T][128]
   int* status;
 };
@@ -308,6 +309,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
         const int64_t t = (int64_t)b * TILE + m;
         const bool add_lr = t >= prm.add_lo && t < prm.add_hi;
         const float4* y4 = reinterpret_cast<const float4*>(prm.addend + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
+        const uint4* y16 = reinterpret_cast<const uint4*>(prm.addend16 + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
         uint4* dst = reinterpret_cast<uint4*>(prm.Out + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
 #pragma unroll
         for (int cb = 0; cb < 2; ++cb) {
@@ -320,7 +322,15 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
             float f[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i * 8 + e]);
-            if (add_lr) {
+            if (add_lr && prm.addend16) {
+              const uint4 a = __ldg(y16 + cb * 4 + i);   // 8 bf16 values
+              const uint32_t yy[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                f[2 * e] += __uint_as_float(yy[e] << 16);
+                f[2 * e + 1] += __uint_as_float(yy[e] & 0xffff0000u);
+              }
+            } else if (add_lr) {
               const float4 a = __ldg(y4 + cb * 8 + i * 2), c = __ldg(y4 + cb * 8 + i * 2 + 1);
               f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
               f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
@@ -479,6 +489,7 @@ struct SegOutParams {
   int64_t n_lr;
   const __nv_bfloat16* ylr;   // [bh][T][128] long-range rows, bf16 (rows t >= n_lr are added)
   __nv_bfloat16* O;
+  __nv_bfloat16* sin_tiles;   // optional [bh][T/128][128][128]: the bf16 state entering every tile, for a later backward
   int* status;
 };
 
@@ -604,8 +615,9 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
 #pragma unroll
       for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(my_tile + (((ch0 + c) ^ (m & 7)) << 4)) = pk[c];
     };
-    // bf16 copy of this thread's 32 state columns into the shared tile
-    auto publish_state = [&](const uint32_t (&v)[32]) {
+    // bf16 copy of this thread's 32 state columns into the shared tile (and, when a backward will want the state
+    // entering tile `tile`, into the per-tile table as well: 64 bytes of row m)
+    auto publish_state = [&](const uint32_t (&v)[32], int64_t tile) {
       uint4 pk[4];
 #pragma unroll
       for (int c = 0; c < 4; ++c)
@@ -614,6 +626,11 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
                            pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
                            pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
       store_row(pk);
+      if (prm.sin_tiles) {
+        __nv_bfloat16* dst = prm.sin_tiles + (((int64_t)bh * (prm.T / TILE) + tile) * TILE + m) * TILE + col0;
+        st_global_v8(dst, pk[0].x, pk[0].y, pk[0].z, pk[0].w, pk[1].x, pk[1].y, pk[1].z, pk[1].w);
+        st_global_v8(dst + 16, pk[2].x, pk[2].y, pk[2].z, pk[2].w, pk[3].x, pk[3].y, pk[3].z, pk[3].w);
+      }
       fence_proxy_async();
       fence_before_sync();
       __syncwarp();
@@ -629,7 +646,7 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
       }
       tmem_st32(tmem_s + lane_base + col0, v);
       tmem_st_wait();
-      publish_state(v);
+      publish_state(v, tile0);
     }
     for (int it = 0; it < Lc; ++it) {
       // --- scores of this tile -> masked bf16 P (registers), stored once O = Q S has consumed the shared tile ---
@@ -674,7 +691,7 @@ __global__ void __launch_bounds__(SEG_OUT_THREADS) segment_output_tc_kernel(cons
         uint32_t v[32];
         tmem_ld32(tmem_s + lane_base + col0, v);
         tmem_ld_wait();
-        publish_state(v);
+        publish_state(v, tile0 + it + 1);
       }
       __nv_bfloat16* dst = prm.O + ((int64_t)bh * prm.T + t) * TILE + col0;
       const uint32_t tmem_o = tmem_o0 + (it & 1) * TILE;
@@ -1178,7 +1195,7 @@ cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf
 template <bool P4_IS_P1, bool XT, bool ST_KMAJOR>
 static cudaError_t launch_tile_product(const void* P1, const void* P2, const void* P3, const void* St_bf16,
                                        const float* addend, int64_t add_lo, int64_t add_hi, void* Out, int64_t T,
-                                       int bh, int* status, cudaStream_t st) {
+                                       int bh, int* status, cudaStream_t st, int addend_bf16 = 0) {
   CUtensorMap tm1, tm2, tm3, tmS;
   const int NC = (int)(T / TILE);
   if (!make_map(&tm1, P1, (uint64_t)bh * T) || !make_map(&tm2, P2, (uint64_t)bh * T) ||
@@ -1186,6 +1203,7 @@ static cudaError_t launch_tile_product(const void* P1, const void* P2, const voi
     return cudaErrorInvalidValue;
   TileParams prm;
   prm.T = T; prm.NC = NC; prm.add_lo = add_lo; prm.add_hi = add_hi; prm.addend = addend;
+  prm.addend16 = addend_bf16 ? reinterpret_cast<const __nv_bfloat16*>(addend) : nullptr;
   prm.Out = static_cast<__nv_bfloat16*>(Out);
   prm.status = status;
   cudaError_t err = cudaFuncSetAttribute(tile_product_tc_kernel<P4_IS_P1, XT, ST_KMAJOR>,
@@ -1207,12 +1225,12 @@ cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void
 cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K, const void* V, const void* dO,
                                          const void* Sin_bf16, const void* Dbar_bf16, const float* addend,
                                          int64_t add_lo, int64_t add_hi, void* Out, int64_t T, int bh, int* status,
-                                         cudaStream_t st) {
+                                         cudaStream_t st, int addend_bf16) {
   if (which == 0)
-    return launch_tile_product<true, false, true>(dO, V, K, Sin_bf16, addend, add_lo, add_hi, Out, T, bh, status, st);
+    return launch_tile_product<true, false, true>(dO, V, K, Sin_bf16, addend, add_lo, add_hi, Out, T, bh, status, st, addend_bf16);
   if (which == 1)
-    return launch_tile_product<false, true, true>(dO, V, Q, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st);
-  return launch_tile_product<false, true, false>(Q, K, dO, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st);
+    return launch_tile_product<false, true, true>(dO, V, Q, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st, addend_bf16);
+  return launch_tile_product<false, true, false>(Q, K, dO, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st, addend_bf16);
 }
 
 cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, void* out_bf16, int transposed,
@@ -1335,7 +1353,7 @@ cudaError_t smat_launch_segment_state_tc(const void* K, const void* V, float* to
 
 cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const void* V, const float* seg_in,
                                           const void* ylr_bf16, int64_t n_lr, void* O, int64_t tiles0, int64_t tiles1,
-                                          int nseg0, int nseg1, int bh, int* status, cudaStream_t st) {
+                                          int nseg0, int nseg1, int bh, int* status, cudaStream_t st, void* sin_tiles) {
   const int64_t T = (tiles0 + tiles1) * TILE;
   CUtensorMap tmQ, tmK, tmV;
   if (!make_map(&tmQ, Q, (uint64_t)bh * T) || !make_map(&tmK, K, (uint64_t)bh * T) ||
@@ -1345,6 +1363,7 @@ cudaError_t smat_launch_segment_output_tc(const void* Q, const void* K, const vo
   prm.T = T; prm.nseg = nseg0 + nseg1; prm.seg_in = seg_in; prm.n_lr = n_lr; prm.ylr = static_cast<const __nv_bfloat16*>(ylr_bf16);
   prm.cut.nseg0 = nseg0; prm.cut.nseg = nseg0 + nseg1; prm.cut.tiles0 = tiles0; prm.cut.tiles1 = tiles1;
   prm.O = static_cast<__nv_bfloat16*>(O);
+  prm.sin_tiles = static_cast<__nv_bfloat16*>(sin_tiles);
   prm.status = status;
   cudaError_t err =
       cudaFuncSetAttribute(segment_output_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_OUT_SMEM);

@@ -221,8 +221,18 @@ def test_backward_with_kept_forward_tables_matches_rebuilding_them():
     keep.check_status(ws)
     b = rebuild.backward(dev["q"], dev["k"], dev["v"], dev["do"])
     assert keep.last_launch_count() < rebuild.last_launch_count()
+    # The kept pass takes the per-tile incoming states the forward's segment kernel published (segment state + the
+    # tiles of the segment, summed in tensor memory) instead of re-scanning K, V tile by tile: the same fp32 sums in a
+    # different order, rounded to bf16 once either way.
     for x, y in zip(a, b):
-        assert torch.equal(x, y)
+        assert rel_err(to_numpy64(x), to_numpy64(y)) <= 4e-3
+    geo = so.geometry(w.T, w.chunk, w.d)
+    rows = sample_tokens(geo, 40, seed=4)
+    Q64, K64, V64, G64 = (synth.as_float64(w, host[x][1]) for x in ("q", "k", "v", "do"))
+    rq = so.dq_rows(Q64, K64, V64, G64, geo, rows)
+    rk, rv = so.dkdv_cols(Q64, K64, V64, G64, geo, rows)
+    for g, r in zip(a, (rq, rk, rv)):
+        assert rel_err(to_numpy64(g[0, 1][rows]), r) <= TOL["bf16"]
 
 
 def test_chunk_size_invariance_on_device():
