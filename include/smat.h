@@ -161,7 +161,7 @@ smat_status smat_backward(const smat_plan* plan, const void* Q, const void* K, c
  * gather — instead of the positional strides; tabulation and the causal branch are unchanged.  An entry outside its
  * range puts the token in no group (it writes to, or reads from, no cached state).  Group sizes may be arbitrarily
  * skewed, including empty groups.  d = 1 ignores both arrays (one cell, one type).  Everything else — workspace
- * size, dtypes, errors — is as for smat_forward / smat_backward; SMAT_ERR_UNSUPPORTED if P or B exceeds 56000.
+ * size, dtypes, errors — is as for smat_forward / smat_backward; SMAT_ERR_UNSUPPORTED if P or B exceeds 27000.
  */
 smat_status smat_forward_routed(const smat_plan* plan, const void* Q, const void* K, const void* V, void* O,
                                 const int32_t* prof, const int32_t* type, void* workspace, size_t workspace_bytes,

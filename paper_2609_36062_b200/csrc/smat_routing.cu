@@ -12,80 +12,99 @@ namespace {
 constexpr int ROUTE_THREADS = 256;
 
 // One CTA per (head, kind); kind 0: profiles of the n distant tokens, kind 1: types of the m recent tokens.
-//   1. histogram of the keys in shared memory (keys outside [0, G) are dropped: such a token belongs to no group)
-//   2. exclusive scan -> offs[0 .. G]
-//   3. stable placement by ONE warp walking the tokens in order, 32 at a time: lanes with equal keys find each other
-//      with match.any, the lowest such lane advances the group's cursor, every lane writes its token's position
+// The tokens are cut into W contiguous ranges, one per warp (W as large as shared memory allows, at most 8):
+//   1. every warp histograms the keys of its range in its own row of counters (keys outside [0, G) are dropped:
+//      such a token belongs to no group)
+//   2. totals per group, exclusive scan -> offs[0 .. G]; row w then becomes the first slot of group g for warp w's
+//      tokens: offs[g] + the counts of the warps before it
+//   3. stable placement: every warp walks ITS range in order, 32 tokens at a time; lanes with equal keys find each other
+//      with match.any, the lowest such lane advances the warp's cursor of the group, every lane writes its token's
+//      position.  Ranges are in token order and each warp's slots follow those of the warps before it, so the list of
+//      a group is ascending.
 struct RouteParams {
   const int32_t* key[2];   // [bh][count]
   int32_t* list[2];        // [bh][count]
   int32_t* offs[2];        // [bh][G + 1]
   int64_t count[2], G[2], first[2];   // tokens per head, groups, position of the first token of the kind
+  int warps;               // W: rows of per-warp counters in shared memory
 };
 
 __global__ void __launch_bounds__(ROUTE_THREADS) routing_lists_kernel(const RouteParams prm) {
-  extern __shared__ int32_t cursor[];   // [G + 1]
+  extern __shared__ int32_t rows[];     // [1 + W][G + 1]: row 0 totals / offsets, row 1 + w the counters of warp w
   const int kind = blockIdx.y;
-  const int64_t bh = blockIdx.x, n = prm.count[kind], G = prm.G[kind];
+  const int64_t bh = blockIdx.x, n = prm.count[kind], G = prm.G[kind], pitch = G + 1;
+  const int W = prm.warps;
   const int32_t* key = prm.key[kind] + bh * n;
   int32_t* list = prm.list[kind] + bh * n;
-  int32_t* offs = prm.offs[kind] + bh * (G + 1);
-  const int tid = threadIdx.x;
-  for (int64_t g = tid; g <= G; g += ROUTE_THREADS) cursor[g] = 0;
+  int32_t* offs = prm.offs[kind] + bh * pitch;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int32_t* total = rows;
+  for (int64_t i = tid; i < (1 + W) * pitch; i += ROUTE_THREADS) rows[i] = 0;
   __syncthreads();
-  for (int64_t t = tid; t < n; t += ROUTE_THREADS) {
-    const int32_t k = key[t];
-    if (k >= 0 && k < G) atomicAdd(&cursor[k + 1], 1);
+  const int64_t per = ((n + W - 1) / W + 31) & ~(int64_t)31;   // tokens per warp range, a multiple of 32
+  const int64_t lo = (int64_t)warp * per, hi = lo + per < n ? lo + per : n;
+  if (warp < W) {
+    int32_t* mine = rows + (1 + warp) * pitch;
+    for (int64_t t = lo + lane; t < hi; t += 32) {
+      const int32_t k = key[t];
+      if (k >= 0 && k < G) atomicAdd(&mine[k], 1);
+    }
   }
   __syncthreads();
-  // exclusive scan of cursor[1 .. G] in place (cursor[g] = first slot of group g), chunk by chunk with a carry
+  for (int64_t g = tid; g < G; g += ROUTE_THREADS) {
+    int32_t sum = 0;
+    for (int w = 0; w < W; ++w) sum += rows[(1 + w) * pitch + g];
+    total[g + 1] = sum;          // shifted by one: the inclusive scan below leaves the first slot of group g at index g
+  }
+  __syncthreads();
   __shared__ int32_t warp_sum[ROUTE_THREADS / 32];
   __shared__ int32_t carry;
   if (tid == 0) carry = 0;
   __syncthreads();
   for (int64_t base = 1; base <= G; base += ROUTE_THREADS) {
     const int64_t g = base + tid;
-    const int32_t v = g <= G ? cursor[g] : 0;
-    int32_t x = v;
+    int32_t x = g <= G ? total[g] : 0;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
       const int32_t y = __shfl_up_sync(0xffffffffu, x, d);
-      if ((tid & 31) >= d) x += y;
+      if (lane >= d) x += y;
     }
-    if ((tid & 31) == 31) warp_sum[tid >> 5] = x;
+    if (lane == 31) warp_sum[warp] = x;
     __syncthreads();
     int32_t before = carry;
-    for (int w = 0; w < (tid >> 5); ++w) before += warp_sum[w];
-    if (g <= G) cursor[g] = before + x;   // inclusive: end of group g - 1 ... stored at index g
+    for (int w = 0; w < warp; ++w) before += warp_sum[w];
+    if (g <= G) total[g] = before + x;
     __syncthreads();
     if (tid == ROUTE_THREADS - 1) carry = before + x;
     __syncthreads();
   }
-  // cursor[g] (g >= 1) now holds the number of tokens in groups < g; cursor[0] = 0
-  for (int64_t g = tid; g <= G; g += ROUTE_THREADS) offs[g] = cursor[g];
+  // total[g] = tokens in groups < g (total[0] = 0): the offsets; then the per-warp first slots
+  for (int64_t g = tid; g <= G; g += ROUTE_THREADS) offs[g] = total[g];
+  for (int64_t g = tid; g < G; g += ROUTE_THREADS) {
+    int32_t slot = total[g];
+    for (int w = 0; w < W; ++w) {
+      const int32_t c = rows[(1 + w) * pitch + g];
+      rows[(1 + w) * pitch + g] = slot;
+      slot += c;
+    }
+  }
   __syncthreads();
-  if (tid < 32) {
+  if (warp < W) {
+    int32_t* cursor = rows + (1 + warp) * pitch;
     const int64_t first = prm.first[kind];
-    constexpr int AHEAD = 8;   // keys are fetched this many steps ahead: the loop is a chain of shared-memory updates
-    int32_t kq[AHEAD];
-#pragma unroll
-    for (int a = 0; a < AHEAD; ++a) kq[a] = (int64_t)a * 32 + tid < n ? key[(int64_t)a * 32 + tid] : -1;
-    for (int64_t t0 = 0; t0 < n; t0 += 32) {
-      const int64_t t = t0 + tid;
-      const int32_t k = kq[0];
-#pragma unroll
-      for (int a = 0; a + 1 < AHEAD; ++a) kq[a] = kq[a + 1];
-      kq[AHEAD - 1] = t + (int64_t)AHEAD * 32 < n ? key[t + (int64_t)AHEAD * 32] : -1;
+    for (int64_t t0 = lo; t0 < hi; t0 += 32) {
+      const int64_t t = t0 + lane;
+      const int32_t k = t < hi ? key[t] : -1;
       const bool valid = k >= 0 && k < G;
-      const unsigned peers = __match_any_sync(0xffffffffu, valid ? k : -1 - tid);
-      int32_t slot = 0;
+      const unsigned peers = __match_any_sync(0xffffffffu, valid ? k : -1 - lane);
       if (valid) {
         const int leader = __ffs(peers) - 1;
-        if (tid == leader) {
+        int32_t slot = 0;
+        if (lane == leader) {
           slot = cursor[k];
           cursor[k] = slot + __popc(peers);
         }
-        slot = __shfl_sync(peers, slot, leader) + __popc(peers & ((1u << tid) - 1));
+        slot = __shfl_sync(peers, slot, leader) + __popc(peers & ((1u << lane) - 1));
         list[slot] = (int32_t)(first + t);
       }
       __syncwarp();
@@ -118,7 +137,7 @@ cudaError_t smat_launch_zero_unrouted(const int32_t* key, int64_t count, int64_t
 }
 
 // Largest group count the list builder handles (its cursors live in shared memory).
-int64_t smat_routing_max_groups() { return 56000; }
+int64_t smat_routing_max_groups() { return 27000; }
 
 cudaError_t smat_launch_routing_lists(const int32_t* prof, const int32_t* type, int32_t* prof_list, int32_t* prof_offs,
                                       int32_t* type_list, int32_t* type_offs, const SmatGeo& geo, int bh,
@@ -128,7 +147,11 @@ cudaError_t smat_launch_routing_lists(const int32_t* prof, const int32_t* type, 
   prm.key[1] = type; prm.list[1] = type_list; prm.offs[1] = type_offs; prm.count[1] = geo.m; prm.G[1] = geo.B; prm.first[1] = geo.n;
   const int64_t gmax = geo.P > geo.B ? geo.P : geo.B;
   if (gmax > smat_routing_max_groups()) return cudaErrorInvalidConfiguration;
-  const size_t smem = (size_t)(gmax + 1) * sizeof(int32_t);
+  int64_t warps = (int64_t)(220 * 1024 / sizeof(int32_t)) / (gmax + 1) - 1;
+  if (warps > ROUTE_THREADS / 32) warps = ROUTE_THREADS / 32;
+  if (warps < 1) warps = 1;
+  prm.warps = (int)warps;
+  const size_t smem = (size_t)(1 + warps) * (gmax + 1) * sizeof(int32_t);
   cudaError_t err = cudaFuncSetAttribute(routing_lists_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
   dim3 grid((unsigned)bh, 2);
