@@ -72,6 +72,8 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
                                         straight from the shared-memory slab (one output row per thread) instead of
                                         the register-resident form (K slopes x q offsets per thread) */
 
+#define SMAT_FLAG_SEPARATE_TILE_ADJOINTS 256u /* tensor-core backward: dQ, dK, dV of a tile by three launches of the general
+                                                 tile-product kernel instead of the one fused kernel (for comparison) */
 #define SMAT_FLAG_GATED 64u          /* the plan serves smat_forward_gated / smat_backward_gated: it runs on the fp32-ALU
                                         kernels and its workspace holds λ and the rescaled copies of Q, K, V, dO */
 

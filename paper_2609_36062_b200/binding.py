@@ -24,6 +24,7 @@ FLAG_ALU_TABULATION = 16
 FLAG_D3_SHARED_SUMS = 32
 FLAG_GATED = 64
 FLAG_NORMALIZED = 128
+FLAG_SEPARATE_TILE_ADJOINTS = 256
 
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",

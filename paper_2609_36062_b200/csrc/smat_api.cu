@@ -23,6 +23,7 @@ struct smat_plan {
   size_t off_status, off_sin, off_F, off_U, off_acc, off_tileA, off_W, off_fwd_end;
   size_t off_dbar, off_ubar, off_fbar, off_tileG, off_bwd_end;
   size_t off_plist, off_poffs, off_tlist, off_toffs;   // token lists of user-supplied routing (int32)
+  size_t off_lr3;         // tensor-core backward: third buffer of bf16 long-range rows (the first two share off_acc)
   size_t off_sin_tiles;   // KEEP_FORWARD_TABLES on tensor-core plans: the bf16 state entering every tile, left by the forward
   size_t off_lam, off_dlam, off_gq, off_gk, off_glr, off_gdo, off_gv, off_gvlr;   // gated variant (SMAT_FLAG_GATED)
   size_t off_nv, off_ny, off_ndy;   // normalised output (SMAT_FLAG_NORMALIZED): V̄, ȳ and the upstream of the linear pass
@@ -417,6 +418,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->off_nv = off;     off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
   pl->off_ny = off;     off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
   pl->off_fwd_end = off;
+  pl->off_lr3 = off;    off = align_up(off + (pl->tc ? (size_t)pl->bh * T * 128 * 2 : 0));
   pl->off_ndy = off;    off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
   pl->off_dlam = off;   off = align_up(off + gated * (size_t)pl->bh * T * 4);
   pl->off_gdo = off;    off = align_up(off + gated * (size_t)pl->bh * T * d_v * esz);
@@ -629,6 +631,27 @@ smat_status backward_impl(const smat_plan* pl, const void* Q, const void* K, con
       if (!kept)
         SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, sin_tiles, pl->T, pl->bh, n, 0, 0, status, cx.st));
       SMAT_TRY(cx, "bwd_suffix_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 0, 1, status, cx.st));
+      if (pl->u_bf16 && fbar_is_bf16 && !(pl->flags & SMAT_FLAG_SEPARATE_TILE_ADJOINTS)) {
+        // All three long-range terms come from the tensor-core read as bf16 rows: one buffer each, then ONE kernel for
+        // the three within-chunk adjoints (every operand of a tile loaded once, both score tiles formed once).
+        char* lr_q = cx.ws + pl->off_acc;
+        char* lr_k = lr_q + (size_t)pl->bh * pl->T * 128 * 2;
+        char* lr_v = cx.ws + pl->off_lr3;
+        zero_unrouted(cx, SMAT_GM_TYPE, lr_q, 256);
+        SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, nullptr, lr_q, 1, types, pl->geo.B,
+                                                                 pl->T, pl->bh, status, cx.st));
+        zero_unrouted(cx, SMAT_GM_PROFILE, lr_k, 256);
+        SMAT_TRY(cx, "bwd_dk_profile_tc", smat_launch_state_read_tc(V, cx.ws + pl->off_fbar, nullptr, lr_k, 1, profs, pl->geo.P,
+                                                                    pl->T, pl->bh, status, cx.st));
+        zero_unrouted(cx, SMAT_GM_PROFILE, lr_v, 256);
+        SMAT_TRY(cx, "bwd_dv_profile_tc", smat_launch_state_read_tc(K, cx.ws + pl->off_fbar, nullptr, lr_v, 0, profs, pl->geo.P,
+                                                                    pl->T, pl->bh, status, cx.st));
+        SMAT_TRY(cx, "bwd_tiles_fused_tc", smat_launch_bwd_tiles_fused_tc(Q, K, V, dO, sin_tiles, cx.ws + pl->off_dbar, lr_q,
+                                                                           lr_k, lr_v, n, dQ, dK, dV, pl->T, pl->bh, status,
+                                                                           cx.st));
+        pl->launches = cx.launches;
+        return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+      }
       // dQ: recent rows add U_type dO
       // (the rows travel as bf16 where the tensor-core read writes them: rounded once, added in fp32 by the tile kernel)
       zero_unrouted(cx, SMAT_GM_TYPE, lrbuf, pl->u_bf16 ? 256 : 512);
@@ -664,6 +687,13 @@ smat_status backward_impl(const smat_plan* pl, const void* Q, const void* K, con
       if (!kept)
         SMAT_TRY(cx, "bwd_state_scan_tc", smat_launch_chunk_scan_tc(K, V, sin_tiles, pl->T, pl->bh, n, 1, 0, status, cx.st));
       SMAT_TRY(cx, "bwd_suffix_scan_tc", smat_launch_chunk_scan_tc(Q, dO, cx.ws + pl->off_dbar, pl->T, pl->bh, n, 1, 1, status, cx.st));
+      if (!(pl->flags & SMAT_FLAG_SEPARATE_TILE_ADJOINTS)) {
+        SMAT_TRY(cx, "bwd_tiles_fused_tc", smat_launch_bwd_tiles_fused_tc(Q, K, V, dO, sin_tiles, cx.ws + pl->off_dbar, nullptr,
+                                                                           nullptr, nullptr, pl->T, dQ, dK, dV, pl->T, pl->bh,
+                                                                           status, cx.st));
+        pl->launches = cx.launches;
+        return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+      }
       for (int which = 0; which < 3; ++which)
         SMAT_TRY(cx, which == 0 ? "bwd_dq_tile_tc" : (which == 1 ? "bwd_dk_tile_tc" : "bwd_dv_tile_tc"),
                  smat_launch_chunk_adjoint_tc(which, Q, K, V, dO, sin_tiles, cx.ws + pl->off_dbar, lrbuf, 0, 0,

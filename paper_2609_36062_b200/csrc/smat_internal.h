@@ -124,6 +124,11 @@ cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K
                                          const void* Sin_bf16, const void* Dbar_bf16, const float* addend,
                                          int64_t add_lo, int64_t add_hi, void* Out, int64_t T, int bh, int* status,
                                          cudaStream_t st, int addend_bf16 = 0);
+// The three adjoints of every tile in one launch (all operands of a tile loaded once, both score tiles formed once).
+cudaError_t smat_launch_bwd_tiles_fused_tc(const void* Q, const void* K, const void* V, const void* dO,
+                                           const void* Sin_bf16, const void* Dbar_bf16, const void* lr_q, const void* lr_k,
+                                           const void* lr_v, int64_t n, void* dQ, void* dK, void* dV, int64_t T, int bh,
+                                           int* status, cudaStream_t st);
 // O_b = Q_b S_in[b] + tril(Q_b K_bᵀ) V_b (+ ylr rows for tokens >= n_lr).
 cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
                                         const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,

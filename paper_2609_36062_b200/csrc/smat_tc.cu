@@ -355,6 +355,220 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
 }
 
 // ---------------------------------------------------------------------------------------------------------------
+// bwd_tile_fused_tc_kernel: the three within-chunk adjoints of one 128-token tile in ONE CTA (Eq. "local-adjoint"
+// with the broadcast of the scanned state adjoint), all 128 output columns:
+//        G = tril(dO Vᵀ),  A = tril(Q Kᵀ)
+//        dQ = dO S_inᵀ + G K,      dK = V D̄ᵀ + Gᵀ Q,      dV = K D̄ + Aᵀ dO      (+ the long-range rows of each)
+// Q, K, V, dO, S_in and D̄ of the tile are loaded once (the three separate tile kernels load 2.7 times as much) and
+// the two score tiles are formed once.  Shared memory: seven 32 KB tiles (Q, K, V, dO, S_in, D̄, X); tensor memory:
+// scores [0,128), dQ [128,256), dK [256,384), dV [384,512).
+//   warp 4 lane 0 : TMA loads (dO, V first: the G scores need nothing else), then every MMA in order
+//   warps 0-3     : one tile row per thread: mask and round G, later A, into the swizzled X tile; read the three
+//                   accumulators, add the long-range rows and store
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int FUSED_SMEM = 14 * BOX_BYTES + 1024 + 256;
+
+struct FusedParams {
+  int64_t T;
+  int NC;
+  int64_t n;                         // rows t >= n add lr_q to dQ; rows t < n add lr_k, lr_v to dK, dV (when non-null)
+  const __nv_bfloat16 *lr_q, *lr_k, *lr_v;   // [bh][T][128] bf16
+  __nv_bfloat16 *dQ, *dK, *dV;       // [bh][T][128]
+  int* status;
+};
+
+__global__ void __launch_bounds__(160) bwd_tile_fused_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+                                                                const __grid_constant__ CUtensorMap tmK,
+                                                                const __grid_constant__ CUtensorMap tmV,
+                                                                const __grid_constant__ CUtensorMap tmG,
+                                                                const __grid_constant__ CUtensorMap tmSin,
+                                                                const __grid_constant__ CUtensorMap tmDb,
+                                                                const FusedParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + 2 * BOX_BYTES;
+  uint8_t* sV = smem + 4 * BOX_BYTES;
+  uint8_t* sG = smem + 6 * BOX_BYTES;      // dO
+  uint8_t* sS = smem + 8 * BOX_BYTES;      // S_in of the tile
+  uint8_t* sD = smem + 10 * BOX_BYTES;     // D̄ of the tile
+  uint8_t* sX = smem + 12 * BOX_BYTES;     // masked, rounded score tile (G, then A)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 14 * BOX_BYTES);
+  uint64_t* bar_in0 = bars + 0;   // dO, V landed
+  uint64_t* bar_in1 = bars + 1;   // Q, K, S_in, D̄ landed
+  uint64_t* bar_sc = bars + 2;    // a score tile is in tensor memory (two phases: G, then A)
+  uint64_t* bar_p = bars + 3;     // X written (one arrival per warp; two phases)
+  uint64_t* bar_x = bars + 4;     // the MMAs that read X = G have finished: dQ, dK complete, X may be overwritten
+  uint64_t* bar_o = bars + 5;     // dV complete
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x, bh = blockIdx.y;
+  const int64_t row0 = (int64_t)bh * prm.T + (int64_t)b * TILE;
+  const WaitCtx wc{cta_abort, prm.status};
+  if (threadIdx.x == 0) {
+    *cta_abort = 0;
+    mbar_init(bar_in0, 1); mbar_init(bar_in1, 1); mbar_init(bar_sc, 1); mbar_init(bar_p, 4); mbar_init(bar_x, 1);
+    mbar_init(bar_o, 1);
+    fence_barrier_init();
+  }
+  if (warp == 4) tmem_alloc(tmem_slot, 512);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tm_sc = tmem_base, tm_dq = tmem_base + TILE, tm_dk = tmem_base + 2 * TILE, tm_dv = tmem_base + 3 * TILE;
+
+  if (warp == 4 && lane == 0) {
+    auto load_tile = [&](uint8_t* dst, const CUtensorMap* map, int row, uint64_t* bar) {
+      tma_load_2d(dst, map, 0, row, bar);
+      tma_load_2d(dst + BOX_BYTES, map, HALF, row, bar);
+    };
+    mbar_expect_tx(bar_in0, 4 * BOX_BYTES);
+    load_tile(sG, &tmG, (int)row0, bar_in0);
+    load_tile(sV, &tmV, (int)row0, bar_in0);
+    mbar_expect_tx(bar_in1, 8 * BOX_BYTES);
+    load_tile(sQ, &tmQ, (int)row0, bar_in1);
+    load_tile(sK, &tmK, (int)row0, bar_in1);
+    const int srow = (int)(((int64_t)bh * prm.NC + b) * TILE);
+    load_tile(sS, &tmSin, srow, bar_in1);
+    load_tile(sD, &tmDb, srow, bar_in1);
+
+    constexpr uint32_t id_kk = make_idesc(TILE, TILE, 0, 0);   // A K-major, B K-major
+    constexpr uint32_t id_km = make_idesc(TILE, TILE, 0, 1);   // A K-major, B MN-major
+    constexpr uint32_t id_mm = make_idesc(TILE, TILE, 1, 1);   // A MN-major, B MN-major
+    // K-major view of a [128 rows][128 k] tile (two 64-wide k blocks 16 KB apart), K-step kk; MN-major view of a
+    // [128 k rows][128 n] tile (16 rows = 2048 bytes per K-step, the two 64-wide n blocks 16 KB apart)
+    auto kmaj = [](const uint8_t* t, int kk) { return make_desc(smem_u32(t) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024); };
+    auto mnmaj = [](const uint8_t* t, int kk) { return make_desc(smem_u32(t) + kk * 2048, BOX_BYTES, 1024); };
+    bool ok = mbar_wait(bar_in0, 0, wc);
+    if (ok) {
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_sc, kmaj(sG, kk), kmaj(sV, kk), id_kk, kk != 0);   // dO Vᵀ
+      mma_commit(bar_sc);
+      ok = mbar_wait(bar_in1, 0, wc);
+    }
+    if (ok) {
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_dq, kmaj(sG, kk), kmaj(sS, kk), id_kk, kk != 0);   // dO S_inᵀ
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_dk, kmaj(sV, kk), kmaj(sD, kk), id_kk, kk != 0);   // V D̄ᵀ
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_dv, kmaj(sK, kk), mnmaj(sD, kk), id_km, kk != 0);  // K D̄
+      ok = mbar_wait(bar_p, 0, wc);          // X = G in shared memory; the G scores have left tensor memory
+    }
+    if (ok) {
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_dq, kmaj(sX, kk), mnmaj(sK, kk), id_km, 1);        // G K
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_dk, mnmaj(sX, kk), mnmaj(sQ, kk), id_mm, 1);       // Gᵀ Q
+      mma_commit(bar_x);
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_sc, kmaj(sQ, kk), kmaj(sK, kk), id_kk, kk != 0);   // Q Kᵀ
+      mma_commit(bar_sc);
+      ok = mbar_wait(bar_p, 1, wc);          // X = A
+    }
+    if (ok) {
+      fence_after_sync();
+#pragma unroll
+      for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_dv, mnmaj(sX, kk), mnmaj(sG, kk), id_mm, 1);       // Aᵀ dO
+      mma_commit(bar_o);
+    }
+  } else if (warp < 4) {
+    const int m = warp * 32 + lane;  // row inside the tile = TMEM lane
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    // masked (column <= row), rounded copy of the score tile into X, swizzled as a K-major operand
+    auto stage_scores = [&]() {
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tm_sc + lane_base + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int h2 = 0; h2 < 4; ++h2) {
+            const int k0 = cb * 32 + i * 8 + h2 * 2;
+            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
+            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            pk[h2] = pack_bf16(lo, hi);
+          }
+          const int j8 = cb * 4 + i;
+          uint8_t* dst = sX + (j8 >> 3) * BOX_BYTES + m * 128 + (((j8 & 7) ^ (m & 7)) << 4);
+          *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
+      fence_proxy_async();
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p);
+    };
+    // one accumulator row (128 columns) plus its long-range row, rounded and stored
+    const int64_t t = (int64_t)b * TILE + m;
+    auto store_row = [&](uint32_t tm_acc, const __nv_bfloat16* lr, bool add, __nv_bfloat16* out) {
+      const uint4* y16 = reinterpret_cast<const uint4*>(lr + ((int64_t)bh * prm.T + t) * TILE);
+      __nv_bfloat16* dst = out + ((int64_t)bh * prm.T + t) * TILE;
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tm_acc + lane_base + cb * 32, v);
+        tmem_ld_wait();
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float f[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[i * 8 + e]);
+          if (add) {
+            const uint4 a = __ldg(y16 + cb * 4 + i);
+            const uint32_t yy[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              f[2 * e] += __uint_as_float(yy[e] << 16);
+              f[2 * e + 1] += __uint_as_float(yy[e] & 0xffff0000u);
+            }
+          }
+          w[4 * i] = pack_bf16(f[0], f[1]); w[4 * i + 1] = pack_bf16(f[2], f[3]);
+          w[4 * i + 2] = pack_bf16(f[4], f[5]); w[4 * i + 3] = pack_bf16(f[6], f[7]);
+        }
+#pragma unroll
+        for (int h8 = 0; h8 < 2; ++h8)
+          st_global_v8(dst + cb * 32 + 16 * h8, w[8 * h8], w[8 * h8 + 1], w[8 * h8 + 2], w[8 * h8 + 3], w[8 * h8 + 4],
+                       w[8 * h8 + 5], w[8 * h8 + 6], w[8 * h8 + 7]);
+      }
+    };
+    bool ok = mbar_wait(bar_sc, 0, wc);
+    if (ok) {
+      fence_after_sync();
+      stage_scores();                              // X = G
+      ok = mbar_wait(bar_sc, 1, wc);               // the A scores are in (the MMAs on G were issued before them)
+    }
+    if (ok) ok = mbar_wait(bar_x, 0, wc);          // ... and those MMAs have finished with X: dQ, dK are complete
+    if (ok) {
+      fence_after_sync();
+      stage_scores();                              // X = A
+      store_row(tm_dq, prm.lr_q, prm.lr_q != nullptr && t >= prm.n, prm.dQ);
+      store_row(tm_dk, prm.lr_k, prm.lr_k != nullptr && t < prm.n, prm.dK);
+      ok = mbar_wait(bar_o, 0, wc);
+    }
+    if (ok) {
+      fence_after_sync();
+      store_row(tm_dv, prm.lr_v, prm.lr_v != nullptr && t < prm.n, prm.dV);
+    }
+  }
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
 // Two-level form of the causal branch.  Each block of the sequence is cut into segments of L tiles.
 //   segment_state_tc_kernel  : total[seg] = Σ_{tiles of the segment} K_bᵀ V_b, accumulated in TMEM (fp32), written once
 //   (scan_kernel turns the totals into the state entering each segment: exclusive prefix sum per block, fp32)
@@ -1231,6 +1445,32 @@ cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K
   if (which == 1)
     return launch_tile_product<false, true, true>(dO, V, Q, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st, addend_bf16);
   return launch_tile_product<false, true, false>(Q, K, dO, Dbar_bf16, addend, add_lo, add_hi, Out, T, bh, status, st, addend_bf16);
+}
+
+// The three within-chunk adjoints in one launch: Sin / Dbar are the per-tile bf16 states, lr_q / lr_k / lr_v the bf16
+// long-range rows (null: none; lr_q is added to rows t >= n of dQ, lr_k and lr_v to rows t < n of dK and dV).
+cudaError_t smat_launch_bwd_tiles_fused_tc(const void* Q, const void* K, const void* V, const void* dO,
+                                           const void* Sin_bf16, const void* Dbar_bf16, const void* lr_q, const void* lr_k,
+                                           const void* lr_v, int64_t n, void* dQ, void* dK, void* dV, int64_t T, int bh,
+                                           int* status, cudaStream_t st) {
+  CUtensorMap tmQ, tmK, tmV, tmG, tmS, tmD;
+  const int NC = (int)(T / TILE);
+  if (!make_map(&tmQ, Q, (uint64_t)bh * T) || !make_map(&tmK, K, (uint64_t)bh * T) || !make_map(&tmV, V, (uint64_t)bh * T) ||
+      !make_map(&tmG, dO, (uint64_t)bh * T) || !make_map(&tmS, Sin_bf16, (uint64_t)bh * NC * TILE) ||
+      !make_map(&tmD, Dbar_bf16, (uint64_t)bh * NC * TILE))
+    return cudaErrorInvalidValue;
+  FusedParams prm;
+  prm.T = T; prm.NC = NC; prm.n = n;
+  prm.lr_q = static_cast<const __nv_bfloat16*>(lr_q);
+  prm.lr_k = static_cast<const __nv_bfloat16*>(lr_k);
+  prm.lr_v = static_cast<const __nv_bfloat16*>(lr_v);
+  prm.dQ = static_cast<__nv_bfloat16*>(dQ); prm.dK = static_cast<__nv_bfloat16*>(dK); prm.dV = static_cast<__nv_bfloat16*>(dV);
+  prm.status = status;
+  cudaError_t err = cudaFuncSetAttribute(bwd_tile_fused_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FUSED_SMEM);
+  if (err != cudaSuccess) return err;
+  dim3 grid((unsigned)NC, (unsigned)bh);
+  bwd_tile_fused_tc_kernel<<<grid, 160, FUSED_SMEM, st>>>(tmQ, tmK, tmV, tmG, tmS, tmD, prm);
+  return cudaGetLastError();
 }
 
 cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, void* out_bf16, int transposed,

@@ -327,3 +327,18 @@ def test_config4_t64k(name):
 def test_config5_t8k_d3_forward_backward():
     w = synth.WORKLOADS["t8k_d3_fwdbwd"]
     _check_sampled(w, heads_to_check=[0, 77, w.bh - 1], nrows=64, backward=True)
+
+
+@pytest.mark.parametrize("d,T", [(1, 2048), (2, 4096), (3, 4096), (4, 4096)])
+def test_fused_and_separate_tile_adjoints_agree(d, T):
+    """The one-kernel form of the three within-chunk adjoints against three launches of the general tile kernel."""
+    w = _small("fused", d, T, 128, 128, 128, "bf16", heads=3, seed=91, recipe="normalised")
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    fused, separate = _plan(w), _plan(w, flags=binding.FLAG_SEPARATE_TILE_ADJOINTS)
+    a = fused.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+    fused.check_status()
+    b = separate.backward(dev["q"], dev["k"], dev["v"], dev["do"])
+    separate.check_status()
+    assert fused.last_launch_count() == separate.last_launch_count() - 2
+    for x, y in zip(a, b):
+        assert rel_err(to_numpy64(x), to_numpy64(y)) <= 2e-3

@@ -118,7 +118,8 @@ def test_workspace_regions_follow_the_stored_element_types():
     assert simt.workspace_bytes(False) > got
     # backward: adjoint tables in bf16 too, per-tile adjoint states
     back = plan.workspace_bytes(True)
-    assert got + tables + causal <= back <= got + tables + causal + 64 * 1024
+    lr3 = w.bh * w.T * 128 * 2                                   # third buffer of bf16 long-range rows
+    assert got + tables + causal + lr3 <= back <= got + tables + causal + lr3 + 64 * 1024
 
 
 def test_launching_calls_report_a_missing_sm100_device():
