@@ -367,7 +367,9 @@ class Runner:
             recs = self.plan.profile_read()
             if self.w.backward:
                 self.run_backward(d, (self.dQ, self.dK, self.dV))
-                recs += [(n if n.startswith("bwd_") else "bwd_" + n, t) for n, t in self.plan.profile_read()]
+                # stages the backward shares with the forward (the rebuilt forward tables) get their own prefix, so that
+                # they cannot merge with an adjoint stage of the same base name
+                recs += [(n if n.startswith("bwd_") else "bwd_fwd_" + n, t) for n, t in self.plan.profile_read()]
             for n, t in recs:
                 if n not in acc:
                     acc[n] = 0.0; order.append(n)
@@ -406,17 +408,20 @@ def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4):
 
 def dominant_kernel_report(w, geo, stages, peaks, u_bytes=4, f_bytes=4):
     """Roofline of the stage that takes the longest.  Its bound is the slower of its bytes at the HBM peak and its
-    operations (contraction flop plus Algorithm 2's additions, one flop each) at the tensor peak."""
+    operations (contraction flop plus Algorithm 2's additions, one flop each) at the tensor peak; a tabulation that
+    adds on the fp32 ALUs is held against the measured fp32-add rate instead when that is the slower term."""
     e = 4 if w.dtype == "f32" else 2
     total = sum(t for _, t in stages)
     name, ms = max(stages, key=lambda s: s[1])
-    base = name
+    base = name[len("bwd_fwd_"):] if name.startswith("bwd_fwd_") else name   # a forward stage re-run by the backward
     work = roofline.stage_work(base, w.T, w.chunk, w.d_k, w.d_v, e, geo, u_bytes, f_bytes).scaled(w.bh)
     t = roofline.roofline_times(work, peaks, sustained=True)
     ops = work.flops + work.adds
     t_ops = ops / (peaks["bf16_tflops_sustained"] * 1e12)
     sec = ms / 1e3
-    if t["t_hbm"] >= t_ops:
+    if base in roofline.ALU_STAGES and t["t_alu"] > t["t_hbm"]:   # sums formed on the fp32 pipes: measured add rate
+        bound, achieved, peak, unit = "alu", work.adds / sec / 1e9, t["alu_peak_adds"] / 1e9, "Gadd/s"
+    elif t["t_hbm"] >= t_ops:
         bound, achieved, peak, unit = "hbm", work.bytes / sec / 1e9, peaks["hbm_gbs"], "GB/s"
     else:
         bound, achieved, peak, unit = "tensor", ops / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
@@ -540,7 +545,10 @@ def run_native(args):
             s = float(np.median(each_))
             rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes(), r.plan.profile_table_element_bytes())
             st_ = r.stage_profile(3)
-            sweep.append({"workload": name, "value": ws_.tokens / s, "unit": "tokens/s", "ms_per_step": 1e3 * s,
+            dom = dominant_kernel_report(ws_, gg, st_, peaks, r.plan.type_table_element_bytes(),
+                                         r.plan.profile_table_element_bytes())
+            sweep.append({"workload": name, "dominant": {k: dom[k] for k in ("kernel", "bound", "achieved", "peak", "unit",
+                                                                              "frac", "ms", "share")}, "value": ws_.tokens / s, "unit": "tokens/s", "ms_per_step": 1e3 * s,
                           "timing": "median of 15 steps after 5 warm-ups, one CUDA event pair per step",
                           "ms_min": 1e3 * min(each_), "ms_max": 1e3 * max(each_),
                           "frac_2term": rep["frac_2term"], "frac_3term": rep["frac_3term"],

@@ -112,6 +112,19 @@ def stage_work(name: str, T, c, r, p, e, geo, u_bytes=4, f_bytes=4) -> Work:
         "pool_tc":     Work(2 * n * rp, 0, n * (r + p) * e + P * sf),
         "tabulate":    Work(0, geo.nnzC * rp, P * st + B * su),
         "tabulate_tc": Work(0, geo.nnzC * rp, P * sf + B * su),
+        "tabulate_regs": Work(0, geo.nnzC * rp, P * sf + B * su),      # the same sums on the fp32 ALUs (bf16 tables)
+        "tabulate_bf16": Work(0, geo.nnzC * rp, P * sf + B * su),
+        "bwd_tabulate_t_tc": Work(0, geo.nnzC * rp, B * su + P * sf),
+        "bwd_pool_type_tc": Work(2 * m * rp, 0, m * (r + p) * e + B * su),
+        "bwd_dq_type_tc": Work(2 * m * rp, 0, m * p * e + B * su + m * r * 2),
+        "bwd_dk_profile_tc": Work(2 * n * rp, 0, n * p * e + P * sf + n * r * 2),
+        "bwd_dv_profile_tc": Work(2 * n * rp, 0, n * r * e + P * sf + n * p * 2),
+        "bwd_suffix_scan_tc": Work(2 * T * rp, tc_tiles * rp, T * (r + p) * e + tc_tiles * rp * 2),
+        # dQ, dK, dV of every 128-token tile: eight 128 x 128 x 128 products per tile; reads Q, K, V, dO, the two
+        # per-tile states and the three long-range buffers (bf16), writes the three gradients
+        "bwd_tiles_fused_tc": Work(tc_tiles * 8 * 2 * 128 * 128 * 128, 0,
+                                   T * (2 * r + 2 * p) * e + T * (2 * r + p) * e + 2 * tc_tiles * rp * 2 +
+                                   (m * r + n * r + n * p) * 2),
         "segment_state_tc": Work(2 * T * rp, 0, T * (r + p) * e),
         "segment_scan": Work(0, 0, 0),
         "segment_output_tc": Work(T * 129 * (r + p) + 4 * T * rp, 0, T * (2 * r + 2 * p) * e + m * p * 2),
@@ -126,3 +139,7 @@ def stage_work(name: str, T, c, r, p, e, geo, u_bytes=4, f_bytes=4) -> Work:
         "output":      Work(T * (c + 1) * p, 0, T * c * 4 + T * p * e + T * p * 4 + T * p * e),
     }
     return table.get(name, Work(0, 0, 0))
+
+
+# Stages whose additions run on the fp32 ALUs (the other tabulations form the same sums on the tensor cores).
+ALU_STAGES = ("tabulate", "tabulate_regs", "tabulate_bf16", "bwd_tabulate_t")
