@@ -378,12 +378,19 @@ class Runner:
         return [(n, acc[n] / steps) for n in order]
 
 
-def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4):
+def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4, gated_tc_forward=False):
     """Fractions against the path roofline.  The bytes are those of the design that ran: where a table is kept as
     bf16 its round trip is charged at 2 bytes per entry, and the fraction against the roofline with fp32 tables is
-    given beside it."""
+    given beside it.  A gated plan whose forward runs on the tensor cores keeps bf16 tables there, while its backward
+    rebuilds fp32 tables on the ALU kernels: each pass is charged with its own."""
     e = 4 if w.dtype == "f32" else 2
     def total(ub, fb):
+        if gated_tc_forward and (ub, fb) != (4, 4):
+            wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, 2, 2)
+            if w.backward:
+                wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, 4, 4, keep_forward_tables=False,
+                                                 f_bytes=4, ubar_bytes=4)
+            return wk.scaled(w.bh)
         wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub, fb)
         if w.backward:  # bench.py's fwd+bwd step keeps the forward's tables; the adjoint tables follow the forward's
             fbar = 2 if (fb == 2 or (ub == 2 and geo.d <= 3)) else 4
@@ -391,13 +398,14 @@ def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4):
             wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub, fbar, keep_forward_tables=True,
                                              f_bytes=fb, ubar_bytes=ubar)
         return wk.scaled(w.bh)
-    work = total(u_bytes, f_bytes)
+    work = total(2, 2) if gated_tc_forward else total(u_bytes, f_bytes)
     t = roofline.roofline_times(work, peaks)
     t32 = roofline.roofline_times(total(4, 4), peaks)
     return {
         "frac_2term": t["t_2term"] / seconds_per_step, "frac_3term": t["t_3term"] / seconds_per_step,
-        "frac_2term_fp32_tables": t32["t_2term"] / seconds_per_step, "type_table_bytes_per_entry": u_bytes,
-        "profile_table_bytes_per_entry": f_bytes,
+        "frac_2term_fp32_tables": t32["t_2term"] / seconds_per_step,
+        "type_table_bytes_per_entry": 2 if gated_tc_forward else u_bytes,
+        "profile_table_bytes_per_entry": 2 if gated_tc_forward else f_bytes,
         "roofline_ms_2term": 1e3 * t["t_2term"], "roofline_ms_3term": 1e3 * t["t_3term"],
         "t_tensor_ms": 1e3 * t["t_tensor"], "t_alu_ms": 1e3 * t["t_alu"], "t_hbm_ms": 1e3 * t["t_hbm"],
         "alu_peak_adds_per_s": t["alu_peak_adds"], "alu_peak_source": t["alu_peak_source"],
@@ -526,7 +534,7 @@ def run_native(args):
             "gpu_launches": launches * steps,
             "clocks": clocks,
             "roofline": dominant_kernel_report(w, g, stages, peaks, ub, fb),
-            "path_roofline": path_report(w, g, per_step, peaks, ub, fb),
+            "path_roofline": path_report(w, g, per_step, peaks, ub, fb, runner.plan.gated_forward_uses_tensor_cores()),
             "tables": {"profile_states_P": g.P, "cached_subset_states_B": g.B, "nnzC": g.nnzC, "q": g.q},
             "fadd_rates_adds_per_s": peaks.get("fadd_rates"),
         }
@@ -543,7 +551,8 @@ def run_native(args):
             gg = r.plan.geometry()
             each_ = r.time_each(r.step, 15, 5)
             s = float(np.median(each_))
-            rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes(), r.plan.profile_table_element_bytes())
+            rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes(), r.plan.profile_table_element_bytes(),
+                              r.plan.gated_forward_uses_tensor_cores())
             st_ = r.stage_profile(3)
             dom = dominant_kernel_report(ws_, gg, st_, peaks, r.plan.type_table_element_bytes(),
                                          r.plan.profile_table_element_bytes())

@@ -27,6 +27,10 @@ struct smat_plan {
   size_t off_sin_tiles;   // KEEP_FORWARD_TABLES on tensor-core plans: the bf16 state entering every tile, left by the forward
   size_t off_lam, off_dlam, off_gq, off_gk, off_glr, off_gdo, off_gv, off_gvlr;   // gated variant (SMAT_FLAG_GATED)
   size_t off_nv, off_ny, off_ndy;   // normalised output (SMAT_FLAG_NORMALIZED): V̄, ȳ and the upstream of the linear pass
+  // Gated plans on tensor-core shapes run their FORWARD through a plan of its own (ungated flags, one state per tile)
+  // whose workspace is the region at off_inner; the backward and every other shape use the fp32-ALU kernels.
+  smat_plan* inner;
+  size_t off_inner;
   bool tc;             // tensor-core kernels for the causal branch
   bool u_bf16;         // forward keeps the type table U in bf16 and reads it with the tensor-core typed read
   bool pool_tc;        // forward pools the profile table on the tensor cores (enough tokens per profile)
@@ -132,6 +136,7 @@ struct Ctx {
   char* ws;
   cudaError_t err;
   int launches;
+  const smat_plan* rec = nullptr;   // plan whose stage timer records the launches (default: pl)
   bool routed = false;   // profile / type groups come from the token lists in the workspace, not from positions
   const int32_t* prof = nullptr;   // the caller's arrays of a routed call
   const int32_t* type = nullptr;
@@ -151,6 +156,16 @@ SmatGroupSpec group(const Ctx& cx, int mode) {
   return s;
 }
 
+// Every pass starts from clean device status words: the plan's own and, on gated plans whose forward runs through an
+// inner plan, that plan's (smat_check_status reads both).
+cudaError_t clear_status(const Ctx& cx) {
+  const smat_plan* pl = cx.pl;
+  cudaError_t err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  if (err == cudaSuccess && pl->inner)
+    err = cudaMemsetAsync(cx.ws + pl->off_inner + pl->inner->off_status, 0, 256, cx.st);
+  return err;
+}
+
 void mark_stage(const smat_plan* pl, cudaStream_t st, const char* name) {
   if (!pl->profiling || pl->stages >= SMAT_MAX_STAGES) return;
   if (pl->stages == 0) cudaEventRecord(pl->events[0], st);
@@ -165,9 +180,9 @@ void end_stage(const smat_plan* pl, cudaStream_t st) {
 #define SMAT_TRY(ctx, name, call)                   \
   do {                                              \
     if ((ctx).err == cudaSuccess) {                 \
-      mark_stage((ctx).pl, (ctx).st, name);         \
+      mark_stage((ctx).rec ? (ctx).rec : (ctx).pl, (ctx).st, name);   \
       (ctx).err = (call);                           \
-      end_stage((ctx).pl, (ctx).st);                \
+      end_stage((ctx).rec ? (ctx).rec : (ctx).pl, (ctx).st);          \
       ++(ctx).launches;                             \
     }                                               \
   } while (0)
@@ -417,6 +432,19 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   const size_t normd = (flags & SMAT_FLAG_NORMALIZED) ? 1 : 0;
   pl->off_nv = off;     off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
   pl->off_ny = off;     off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
+  pl->inner = nullptr;
+  pl->off_inner = off;
+  if ((flags & SMAT_FLAG_GATED) && !(flags & SMAT_FLAG_SIMT_ONLY) && dtype == SMAT_BF16 && d_k == 128 && d_v == 128) {
+    smat_plan* in = nullptr;
+    const unsigned keep = SMAT_FLAG_ALG2_TABULATION | SMAT_FLAG_ALU_TABULATION | SMAT_FLAG_D3_SHARED_SUMS;
+    if (smat_plan_create(&in, batch, heads, T, d_k, d_v, d, chunk, q_override, dtype,
+                         (flags & keep) | SMAT_FLAG_PER_TILE_STATES) == SMAT_OK && in->tc) {
+      pl->inner = in;
+      off = align_up(off + in->off_fwd_end);
+    } else if (in) {
+      smat_plan_destroy(in);
+    }
+  }
   pl->off_fwd_end = off;
   pl->off_lr3 = off;    off = align_up(off + (pl->tc ? (size_t)pl->bh * T * 128 * 2 : 0));
   pl->off_ndy = off;    off = align_up(off + normd * (size_t)pl->bh * T * d_v * esz);
@@ -435,6 +463,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
 
 void smat_plan_destroy(smat_plan* plan) {
   if (plan && plan->profiling) smat_profile_enable(plan, 0);
+  if (plan && plan->inner) smat_plan_destroy(plan->inner);
   delete plan;
 }
 
@@ -476,6 +505,8 @@ smat_status smat_get_geometry(const smat_plan* pl, smat_geometry* out) {
 }
 
 int smat_uses_tensor_cores(const smat_plan* pl) { return pl && pl->tc ? 1 : 0; }
+
+int smat_gated_forward_uses_tensor_cores(const smat_plan* pl) { return pl && pl->inner ? 1 : 0; }
 
 int smat_type_table_element_bytes(const smat_plan* pl) { return pl && pl->u_bf16 ? 2 : 4; }
 
@@ -527,7 +558,7 @@ smat_status forward_impl(const smat_plan* pl, const void* Q, const void* K, cons
   if (!device_ok()) return SMAT_ERR_ARCH;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
-  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  cx.err = clear_status(cx);
   s = begin_routing(cx, prof, type);
   if (s != SMAT_OK) return s;
   if (pl->tc) {
@@ -596,7 +627,7 @@ smat_status backward_impl(const smat_plan* pl, const void* Q, const void* K, con
   if (!device_ok()) return SMAT_ERR_ARCH;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
-  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  cx.err = clear_status(cx);
   s = begin_routing(cx, prof, type);
   if (s != SMAT_OK) return s;
   const bool lr = !pl->geo.dense_G;
@@ -776,6 +807,42 @@ void gated_forward_tables(Ctx& cx, const Gated& gt, const void* Q, const void* K
   gated_scan(cx, "gated_scan", cx.f(pl->off_sin), gt.lam, 0);
 }
 
+// Gated forward on the tensor cores (bf16, d_k = d_v = 128, blocks of whole 128-token tiles).  The long-range part is
+// the ungated pipeline on the boundary-rescaled keys and queries; the causal part carries one state per tile: the scan
+// adds the sums of keys rescaled to the end of their tile and decays the running state by the tile's total gate; the
+// tile kernel multiplies the masked scores by exp(λ_i - λ_j) and the state product of row i by exp(λ_i - λ_{tile start - 1}).
+// Every exponent is a non-positive difference.
+smat_status forward_gated_tc(Ctx& cx, const Gated& gt, const void* Q, const void* K, const void* V, const float* log_a,
+                             void* O) {
+  const smat_plan* pl = cx.pl;
+  const smat_plan* in = pl->inner;
+  const bool lr = !pl->geo.dense_G;
+  Ctx ci{in, cx.st, cx.ws + pl->off_inner, cudaSuccess, 0};
+  ci.rec = pl;
+  int* status = reinterpret_cast<int*>(ci.ws + in->off_status);
+  SMAT_TRY(cx, "gate_prefix", smat_launch_head_scan(log_a, gt.lam, pl->T, pl->bh, 0, cx.st));
+  SMAT_TRY(cx, "gate_scale_k", smat_launch_gate_scale(K, nullptr, gt.kc, gt.lam, 1, 1, pl->geo.n, 128, pl->T, pl->r, pl->bh,
+                                                      cx.st));                                // exp(λ_{tile end} - λ_j) k_j
+  if (lr) gate_scale(cx, "gate_scale_lr", K, Q, gt.lr, gt.lam, 2, pl->r);                    // split at the boundary
+  ci.err = cx.err;
+  float* ylr = ci.f(in->off_acc);
+  if (lr) {
+    build_type_table(ci, gt.lr, V);                                                          // steps 2-3 on the rescaled keys
+    if (in->u_bf16)
+      SMAT_TRY(ci, "read_type_tc", smat_launch_state_read_tc(gt.lr, ci.ws + in->off_U, ylr, nullptr, 0,
+                                                             group(ci, SMAT_GM_TYPE), in->geo.B, in->T, in->bh, status,
+                                                             ci.st));                        // step 4 on the rescaled queries
+    else
+      state_read(ci, "read_type", SMAT_GM_TYPE, gt.lr, ci.f(in->off_U), 0, nullptr, ylr, nullptr);
+  }
+  SMAT_TRY(ci, "gated_chunk_scan_tc", smat_launch_chunk_scan_tc(gt.kc, V, ci.ws + in->off_sin, in->T, in->bh, in->geo.n,
+                                                                 lr ? 0 : 1, 0, status, ci.st, gt.lam));
+  SMAT_TRY(ci, "gated_chunk_output_tc", smat_launch_chunk_output_tc(Q, K, V, ci.ws + in->off_sin, ylr, lr ? in->geo.n : in->T,
+                                                                     O, in->T, in->bh, status, ci.st, gt.lam));
+  pl->launches = cx.launches + ci.launches;
+  return ci.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
 smat_status gated_check(const smat_plan* pl, const void* log_a, void* ws, size_t ws_bytes, int for_backward) {
   if (!log_a) return SMAT_ERR_NULL;
   smat_status s = check_common(pl, ws, ws_bytes, for_backward);
@@ -847,8 +914,9 @@ smat_status smat_forward_gated(const smat_plan* pl, const void* Q, const void* K
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
   pl->tile_states = false;
-  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  cx.err = clear_status(cx);
   const Gated gt = gated_buffers(cx);
+  if (pl->inner) return forward_gated_tc(cx, gt, Q, K, V, log_a, O);
   gated_forward_tables(cx, gt, Q, K, V, log_a);
   float* acc = cx.f(pl->off_acc);
   float* tileA = cx.f(pl->off_tileA);
@@ -873,7 +941,7 @@ smat_status smat_backward_gated(const smat_plan* pl, const void* Q, const void* 
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
   pl->tile_states = false;
-  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  cx.err = clear_status(cx);
   const bool lr = !pl->geo.dense_G;
   const Gated gt = gated_buffers(cx);
   gated_forward_tables(cx, gt, Q, K, V, log_a);
@@ -1027,12 +1095,16 @@ smat_status smat_debug_tables(const smat_plan* pl, const void* workspace, float*
 smat_status smat_check_status(const smat_plan* pl, const void* workspace, void* cuda_stream) {
   if (!pl || !workspace) return SMAT_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  int word = 0;
+  int word = 0, word2 = 0;
   if (cudaMemcpyAsync(&word, static_cast<const char*>(workspace) + pl->off_status, sizeof(int), cudaMemcpyDeviceToHost,
                       st) != cudaSuccess)
     return SMAT_ERR_LAUNCH;
+  if (pl->inner &&   // the tensor-core forward of a gated plan reports into the status word of its own region
+      cudaMemcpyAsync(&word2, static_cast<const char*>(workspace) + pl->off_inner + pl->inner->off_status, sizeof(int),
+                      cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return SMAT_ERR_LAUNCH;
   if (cudaStreamSynchronize(st) != cudaSuccess) return SMAT_ERR_LAUNCH;
-  return word == 0 ? SMAT_OK : SMAT_ERR_DEVICE_TIMEOUT;
+  return (word | word2) == 0 ? SMAT_OK : SMAT_ERR_DEVICE_TIMEOUT;
 }
 
 int smat_last_launch_count(const smat_plan* pl) { return pl ? pl->launches : 0; }
@@ -1054,7 +1126,7 @@ smat_status smat_decode_begin(const smat_plan* pl, const void* K, const void* V,
   if (!device_ok()) return SMAT_ERR_ARCH;
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
-  cx.err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
+  cx.err = clear_status(cx);
   const size_t off = build_type_table(cx, K, V);
   const size_t tbytes = (size_t)pl->bh * pl->geo.B * pl->rp * (pl->u_bf16 ? 2 : 4);
   if (cx.err == cudaSuccess)

@@ -68,6 +68,18 @@ __global__ void gate_scale_kernel(const T* __restrict__ A, const T* __restrict__
     f = __expf(l[t] - l[n - 1]);
     src = B;
   }
+  if (dim % 128 == 0) {   // four consecutive elements per lane: 8-byte (bf16) or 16-byte (fp32) accesses
+    for (int i = lane * 4; i < dim; i += 128) {
+      __align__(16) T v[4];
+      if (sizeof(T) == 2) *reinterpret_cast<uint2*>(v) = *reinterpret_cast<const uint2*>(src + row * dim + i);
+      else *reinterpret_cast<uint4*>(v) = *reinterpret_cast<const uint4*>(src + row * dim + i);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) v[k] = (T)((float)v[k] * f);
+      if (sizeof(T) == 2) *reinterpret_cast<uint2*>(out + row * dim + i) = *reinterpret_cast<const uint2*>(v);
+      else *reinterpret_cast<uint4*>(out + row * dim + i) = *reinterpret_cast<const uint4*>(v);
+    }
+    return;
+  }
   for (int i = lane; i < dim; i += 32) out[row * dim + i] = (T)((float)src[row * dim + i] * f);
 }
 

@@ -41,6 +41,8 @@ struct ScanParams {
   int NC;           // tiles per head
   int lo[2], hi[2]; // tile ranges of the (up to two) blocks
   int reverse;      // 0: exclusive prefix sums (S_in); 1: exclusive suffix sums (the scan adjoint D̄)
+  const float* lam; // gated variant (forward order only): inclusive prefix sums of the log-gates, [bh][T]; the running
+                    // state is multiplied by the tile's total gate before the tile's (key-rescaled) sum is added
   __nv_bfloat16* Sin;  // [bh][NC][128][128]
   int* status;
 };
@@ -133,10 +135,16 @@ __global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constan
       fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(dempty + db);
+      float decay = 1.f;
+      if (prm.lam) {   // exp(λ_{last token of tile b} - λ_{last token before it})
+        const float* lh = prm.lam + (int64_t)bh * prm.T;
+        const int64_t t0 = (int64_t)b * TILE;
+        decay = __expf(lh[t0 + TILE - 1] - (t0 > 0 ? lh[t0 - 1] : 0.f));
+      }
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
-        acc[j] += __uint_as_float(v0[j]);
-        acc[32 + j] += __uint_as_float(v1[j]);
+        acc[j] = fmaf(acc[j], decay, __uint_as_float(v0[j]));
+        acc[32 + j] = fmaf(acc[32 + j], decay, __uint_as_float(v1[j]));
       }
     }
   }
@@ -167,7 +175,7 @@ __global__ void __launch_bounds__(192) chunk_scan_tc_kernel(const __grid_constan
 //   warps 0-3     : one tile row per thread: mask and round the scores into the swizzled layout, later read Oh,
 //                   add the long-range rows and store
 // ---------------------------------------------------------------------------------------------------------------
-constexpr int OUT_SMEM = 6 * BOX_BYTES + 1024 + 256;
+constexpr int OUT_SMEM = 6 * BOX_BYTES + 1024 + 256 + TILE * 4;   // operands, alignment, barriers, the tile's λ (gated)
 
 struct TileParams {
   int64_t T;
@@ -175,11 +183,15 @@ struct TileParams {
   int64_t add_lo, add_hi;  // rows add_lo <= t < add_hi of every head add `addend`
   const float* addend;     // [bh][T][128] fp32, or
   const __nv_bfloat16* addend16;   // the same rows in bf16 (when non-null)
+  const float* lam;        // GATED: inclusive prefix sums of the log-gates [bh][T]
   __nv_bfloat16* Out;      // [bh][T][128]
   int* status;
 };
 
-template <bool P4_IS_P1, bool XT, bool ST_KMAJOR>
+// GATED (forward tile only, Lemma "Gated SMat"): the masked scores are multiplied by exp(λ_i - λ_j) before they are
+// rounded, and the state product keeps an accumulator of its own so that row i can be scaled by
+// exp(λ_i - λ_{last token before the tile}) when the two are added.
+template <bool P4_IS_P1, bool XT, bool ST_KMAJOR, bool GATED = false>
 __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_constant__ CUtensorMap tm1,
                                                               const __grid_constant__ CUtensorMap tm2,
                                                               const __grid_constant__ CUtensorMap tm3,
@@ -201,12 +213,14 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
   uint64_t* bar_o = bars + 4;    // output in TMEM
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* sLam = reinterpret_cast<float*>(smem + 6 * BOX_BYTES + 256);   // [128] λ of the tile's tokens (GATED)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int half = blockIdx.x & 1, b = blockIdx.x >> 1;
   const int bh = blockIdx.y;
   const int64_t row0 = (int64_t)bh * prm.T + (int64_t)b * TILE;
   const WaitCtx wc{cta_abort, prm.status};
+  if (GATED && threadIdx.x < TILE) sLam[threadIdx.x] = prm.lam[row0 + threadIdx.x];
 
   if (threadIdx.x == 0) {
     *cta_abort = 0;
@@ -219,6 +233,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_sc = tmem_base, tmem_o = tmem_base + TILE;
+  const uint32_t tmem_st = GATED ? tmem_base + TILE + HALF : tmem_o;   // accumulator of the state product
 
   if (warp == 4 && lane == 0) {
     mbar_expect_tx(bar_qk, 4 * BOX_BYTES);
@@ -258,7 +273,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
         const uint64_t dA = make_desc(smem_u32(s4) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
         const uint64_t dB = ST_KMAJOR ? make_desc(smem_u32(sS) + (kk >> 2) * (BOX_BYTES / 2) + (kk & 3) * 32, 16, 1024)
                                       : make_desc(smem_u32(sS) + kk * 2048, BOX_BYTES, 1024);
-        mma_bf16(tmem_o, dA, dB, idesc_st, kk != 0);
+        mma_bf16(tmem_st, dA, dB, idesc_st, kk != 0);
       }
       ok = mbar_wait(bar_p, 0, wc);
     }
@@ -271,7 +286,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
         const uint64_t dA = XT ? make_desc(smem_u32(sX) + kk * 2048, BOX_BYTES, 1024)
                                : make_desc(smem_u32(sX) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
         const uint64_t dB = make_desc(smem_u32(s3) + kk * 2048, BOX_BYTES, 1024);
-        mma_bf16(tmem_o, dA, dB, idesc_x, 1);
+        mma_bf16(tmem_o, dA, dB, idesc_x, GATED ? (kk != 0) : 1);
       }
       mma_commit(bar_o);
     }
@@ -280,6 +295,7 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     if (mbar_wait(bar_sc, 0, wc)) {
       fence_after_sync();
+      const float lam_m = GATED ? sLam[m] : 0.f;
 #pragma unroll
       for (int cb = 0; cb < 4; ++cb) {
         uint32_t v[32];
@@ -291,8 +307,12 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
 #pragma unroll
           for (int h2 = 0; h2 < 4; ++h2) {
             const int k0 = cb * 32 + i * 8 + h2 * 2;
-            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
-            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
+            float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            if (GATED) {   // exponents of non-positive differences only: the rows above the diagonal stay zero
+              if (k0 <= m) lo *= __expf(lam_m - sLam[k0]);
+              if (k0 + 1 <= m) hi *= __expf(lam_m - sLam[k0 + 1]);
+            }
             pk[h2] = pack_bf16(lo, hi);
           }
           const int j8 = cb * 4 + i;  // chunk index along the key dimension, 0..15
@@ -308,6 +328,8 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
         fence_after_sync();
         const int64_t t = (int64_t)b * TILE + m;
         const bool add_lr = t >= prm.add_lo && t < prm.add_hi;
+        float row_scale = 1.f;   // GATED: exp(λ_i - λ of the last token before the tile)
+        if (GATED) row_scale = __expf(lam_m - (b > 0 ? prm.lam[row0 - 1] : 0.f));
         const float4* y4 = reinterpret_cast<const float4*>(prm.addend + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
         const uint4* y16 = reinterpret_cast<const uint4*>(prm.addend16 + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
         uint4* dst = reinterpret_cast<uint4*>(prm.Out + ((int64_t)bh * prm.T + t) * TILE + half * HALF);
@@ -316,6 +338,13 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
           uint32_t v[32];
           tmem_ld32(tmem_o + lane_base + cb * 32, v);
           tmem_ld_wait();
+          if (GATED) {
+            uint32_t vs[32];
+            tmem_ld32(tmem_st + lane_base + cb * 32, vs);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(fmaf(row_scale, __uint_as_float(vs[e]), __uint_as_float(v[e])));
+          }
           uint32_t w[16];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -1385,10 +1414,12 @@ bool smat_tc_available() {
 }
 
 cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf16, int64_t T, int bh, int64_t n,
-                                      int through, int reverse, int* status, cudaStream_t st) {
+                                      int through, int reverse, int* status, cudaStream_t st, const float* lam) {
   CUtensorMap tmK, tmV;
+  if (lam && reverse) return cudaErrorInvalidValue;   // the decayed recursion is built for the forward order only
   if (!make_map(&tmK, K, (uint64_t)bh * T) || !make_map(&tmV, V, (uint64_t)bh * T)) return cudaErrorInvalidValue;
   ScanParams prm;
+  prm.lam = lam;
   prm.T = T; prm.NC = (int)(T / TILE);
   prm.Sin = static_cast<__nv_bfloat16*>(Sin_bf16);
   prm.status = status;
@@ -1406,10 +1437,11 @@ cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf
   return cudaGetLastError();
 }
 
-template <bool P4_IS_P1, bool XT, bool ST_KMAJOR>
+template <bool P4_IS_P1, bool XT, bool ST_KMAJOR, bool GATED = false>
 static cudaError_t launch_tile_product(const void* P1, const void* P2, const void* P3, const void* St_bf16,
                                        const float* addend, int64_t add_lo, int64_t add_hi, void* Out, int64_t T,
-                                       int bh, int* status, cudaStream_t st, int addend_bf16 = 0) {
+                                       int bh, int* status, cudaStream_t st, int addend_bf16 = 0,
+                                       const float* lam = nullptr) {
   CUtensorMap tm1, tm2, tm3, tmS;
   const int NC = (int)(T / TILE);
   if (!make_map(&tm1, P1, (uint64_t)bh * T) || !make_map(&tm2, P2, (uint64_t)bh * T) ||
@@ -1418,19 +1450,22 @@ static cudaError_t launch_tile_product(const void* P1, const void* P2, const voi
   TileParams prm;
   prm.T = T; prm.NC = NC; prm.add_lo = add_lo; prm.add_hi = add_hi; prm.addend = addend;
   prm.addend16 = addend_bf16 ? reinterpret_cast<const __nv_bfloat16*>(addend) : nullptr;
+  prm.lam = lam;
   prm.Out = static_cast<__nv_bfloat16*>(Out);
   prm.status = status;
-  cudaError_t err = cudaFuncSetAttribute(tile_product_tc_kernel<P4_IS_P1, XT, ST_KMAJOR>,
+  cudaError_t err = cudaFuncSetAttribute(tile_product_tc_kernel<P4_IS_P1, XT, ST_KMAJOR, GATED>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, OUT_SMEM);
   if (err != cudaSuccess) return err;
   dim3 grid((unsigned)(NC * 2), (unsigned)bh);
-  tile_product_tc_kernel<P4_IS_P1, XT, ST_KMAJOR><<<grid, 160, OUT_SMEM, st>>>(tm1, tm2, tm3, tmS, prm);
+  tile_product_tc_kernel<P4_IS_P1, XT, ST_KMAJOR, GATED><<<grid, 160, OUT_SMEM, st>>>(tm1, tm2, tm3, tmS, prm);
   return cudaGetLastError();
 }
 
 cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
                                         const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,
-                                        cudaStream_t st) {
+                                        cudaStream_t st, const float* lam) {
+  if (lam)
+    return launch_tile_product<true, false, false, true>(Q, K, V, Sin_bf16, ylr, n_lr, T, O, T, bh, status, st, 0, lam);
   return launch_tile_product<true, false, false>(Q, K, V, Sin_bf16, ylr, n_lr, T, O, T, bh, status, st);
 }
 

@@ -31,6 +31,8 @@ def test_gated_forward_and_gradients_match_the_dense_oracle(d, T, dk, dv, c, dty
     la_dev = torch.from_numpy(la).cuda()
     plan = binding.SmatPlan(1, 2, T, dk, dv, d, c, dtype, q_override=q, flags=binding.FLAG_GATED)
     assert not plan.uses_tensor_cores()
+    # bf16 with 128-wide heads and blocks of whole 128-token tiles: the forward runs on the tensor-core kernels
+    assert plan.gated_forward_uses_tensor_cores() == (dtype == "bf16" and dk == 128 and dv == 128 and (T // 2) % 128 == 0)
     O = plan.forward_gated(dev["q"], dev["k"], dev["v"], la_dev)
     dQ, dK, dV, dla = plan.backward_gated(dev["q"], dev["k"], dev["v"], la_dev, dev["do"])
     plan.check_status()
@@ -94,3 +96,61 @@ def test_gated_rows_at_a_longer_sequence_and_argument_errors():
     with pytest.raises(binding.SmatError) as err:
         plain.forward_gated(dev["q"], dev["k"], dev["v"], torch.from_numpy(la).cuda())
     assert err.value.code == 10
+
+
+@pytest.mark.parametrize("d,T,c,q,lo", [(1, 2048, 128, 0, 0.97), (2, 4096, 128, 0, 0.95), (3, 4096, 64, 0, 0.9),
+                                        (4, 2048, 128, 5, 0.98), (3, 8192, 128, 0, 0.999)])
+def test_tensor_core_gated_forward_against_oracle_rows_and_the_alu_path(d, T, c, q, lo):
+    w = synth.Workload("gtc", d, 1, 3, T, 128, 128, c, "bf16", "normalised", 31)
+    host, dev = device_inputs(w)
+    la = _gates(w, lo, 8)
+    la_dev = torch.from_numpy(la).cuda()
+    plan = binding.SmatPlan(1, 3, T, 128, 128, d, c, "bf16", q_override=q, flags=binding.FLAG_GATED)
+    assert plan.gated_forward_uses_tensor_cores()
+    O = plan.forward_gated(dev["q"], dev["k"], dev["v"], la_dev)
+    plan.check_status()
+    alu = binding.SmatPlan(1, 3, T, 128, 128, d, c, "bf16", q_override=q,
+                           flags=binding.FLAG_GATED | binding.FLAG_SIMT_ONLY)
+    assert not alu.gated_forward_uses_tensor_cores()
+    O_alu = alu.forward_gated(dev["q"], dev["k"], dev["v"], la_dev)
+    assert rel_err(to_numpy64(O), to_numpy64(O_alu)) <= 8e-3
+    geo = so.geometry(T, c, d, q or None)
+    rows = sample_tokens(geo, 64, seed=5)
+    rows = np.unique(np.concatenate([rows, [0, 127, 128, geo.n - 1, geo.n, geo.n + 127, geo.n + 128, T - 1]]))
+    for h in (0, 2):
+        Q64, K64, V64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v"))
+        ref = so.gated_forward_rows(Q64, K64, V64, geo, la[h].astype(np.float64), rows)
+        assert rel_err(to_numpy64(O[0, h][rows]), ref) <= TOL["bf16"], (h,)
+    # the pass is repeatable bit for bit
+    O2 = plan.forward_gated(dev["q"], dev["k"], dev["v"], la_dev)
+    assert torch.equal(O, O2)
+
+
+def test_tensor_core_gated_forward_under_strong_decay():
+    # λ falls by about 4 per token: exp(-λ_j) overflows after two dozen tokens; every exponent taken is a difference <= 0
+    w = synth.Workload("gtc2", 3, 1, 2, 2048, 128, 128, 128, "bf16", "normalised", 32)
+    host, dev = device_inputs(w)
+    la = np.full((w.bh, w.T), np.log(0.02), dtype=np.float32)
+    la[:, ::7] = np.log(0.9)
+    plan = binding.SmatPlan(1, 2, w.T, 128, 128, 3, 128, "bf16", flags=binding.FLAG_GATED)
+    assert plan.gated_forward_uses_tensor_cores()
+    O = plan.forward_gated(dev["q"], dev["k"], dev["v"], torch.from_numpy(la).cuda())
+    plan.check_status()
+    assert torch.isfinite(O).all()
+    geo = so.geometry(w.T, 128, 3)
+    rows = sample_tokens(geo, 48, seed=6)
+    Q64, K64, V64 = (synth.as_float64(w, host[x][1]) for x in ("q", "k", "v"))
+    ref = so.gated_forward_rows(Q64, K64, V64, geo, la[1].astype(np.float64), rows)
+    assert rel_err(to_numpy64(O[0, 1][rows]), ref) <= TOL["bf16"]
+
+
+def test_unit_gates_on_the_tensor_core_path_reproduce_the_ungated_forward():
+    w = synth.Workload("gtc3", 3, 1, 2, 4096, 128, 128, 128, "bf16", "normalised", 33)
+    host, dev = device_inputs(w)
+    zeros = torch.zeros(w.bh, w.T, device="cuda")
+    gated = binding.SmatPlan(1, 2, w.T, 128, 128, 3, 128, "bf16", flags=binding.FLAG_GATED)
+    plain = binding.SmatPlan(1, 2, w.T, 128, 128, 3, 128, "bf16", flags=binding.FLAG_PER_TILE_STATES)
+    a = gated.forward_gated(dev["q"], dev["k"], dev["v"], zeros)
+    b = plain.forward(dev["q"], dev["k"], dev["v"])
+    # the gated tile adds its two accumulators in the epilogue: same sums, another order, so not the same bits
+    assert rel_err(to_numpy64(a), to_numpy64(b)) <= 4e-3
