@@ -672,11 +672,10 @@ smat_status backward_impl(const smat_plan* pl, const void* Q, const void* K, con
         SMAT_TRY(cx, "bwd_dq_type_tc", smat_launch_state_read_tc(dO, cx.ws + pl->off_U, nullptr, lr_q, 1, types, pl->geo.B,
                                                                  pl->T, pl->bh, status, cx.st));
         zero_unrouted(cx, SMAT_GM_PROFILE, lr_k, 256);
-        SMAT_TRY(cx, "bwd_dk_profile_tc", smat_launch_state_read_tc(V, cx.ws + pl->off_fbar, nullptr, lr_k, 1, profs, pl->geo.P,
-                                                                    pl->T, pl->bh, status, cx.st));
         zero_unrouted(cx, SMAT_GM_PROFILE, lr_v, 256);
-        SMAT_TRY(cx, "bwd_dv_profile_tc", smat_launch_state_read_tc(K, cx.ws + pl->off_fbar, nullptr, lr_v, 0, profs, pl->geo.P,
-                                                                    pl->T, pl->bh, status, cx.st));
+        // dK's and dV's long-range rows read the same state F̄_x: one launch, every state loaded once
+        SMAT_TRY(cx, "bwd_dkdv_profile_tc", smat_launch_state_read_dual_tc(V, K, cx.ws + pl->off_fbar, lr_k, lr_v, profs,
+                                                                            pl->geo.P, pl->T, pl->bh, status, cx.st));
         SMAT_TRY(cx, "bwd_tiles_fused_tc", smat_launch_bwd_tiles_fused_tc(Q, K, V, dO, sin_tiles, cx.ws + pl->off_dbar, lr_q,
                                                                            lr_k, lr_v, n, dQ, dK, dV, pl->T, pl->bh, status,
                                                                            cx.st));

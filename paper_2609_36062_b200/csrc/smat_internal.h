@@ -141,6 +141,11 @@ cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void
 cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, void* out_bf16, int transposed,
                                       const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh, int* status,
                                       cudaStream_t st);
+// Both reads of the per-profile adjoint states in one launch (every state loaded once): out_t[t] = St x_t for rows Xt,
+// out_n[t] = Stᵀ x_t for rows Xn; bf16 results.
+cudaError_t smat_launch_state_read_dual_tc(const void* Xt, const void* Xn, const void* state_bf16, void* out_t_bf16,
+                                           void* out_n_bf16, const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh,
+                                           int* status, cudaStream_t st);
 // One step of cached decoding: S += k vᵀ, o = qᵀ (U_type + S) for every head (fp32 running state).
 cudaError_t smat_launch_decode_step(const void* q, const void* k, const void* v, void* o, float* S, const void* U,
                                     int u_bf16, int in_bf16, int64_t type, int64_t types, int r, int p, int bh,

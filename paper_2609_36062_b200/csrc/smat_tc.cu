@@ -991,6 +991,8 @@ struct ReadParams {
   const __nv_bfloat16* X;  // [bh][T][128] rows contracted against the state
   float* out;            // [bh][T][128] fp32 rows, or
   __nv_bfloat16* out_bf16;  // bf16 rows (when non-null)
+  const __nv_bfloat16* X2;  // DUAL: second set of rows, contracted against the FIRST state index of the same state,
+  __nv_bfloat16* out2_bf16; // and their bf16 result rows
   int* status;
 };
 
@@ -1027,14 +1029,18 @@ struct ReadPass {
   }
 };
 
-template <int TRANS>
+// DUAL (with TRANS = 1): both adjoint reads of a profile's tokens from one load of the state F̄_x —
+// out[t] = F̄_x x_t (rows X, e.g. dK from v) and out2[t] = F̄_xᵀ x2_t (rows X2, e.g. dV from k) — two operand tiles, two
+// accumulators, bf16 results.
+template <int TRANS, int DUAL = 0>
 __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constant__ CUtensorMap tmU,
                                                             const ReadParams prm) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sA = smem;                    // queries, K-major, two 64-column blocks
   uint8_t* sB = smem + 2 * BOX_BYTES;    // state, MN-major, two 64-column blocks
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 4 * BOX_BYTES);
+  uint8_t* sA2 = smem + 4 * BOX_BYTES;   // DUAL: the second rows
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (DUAL ? 6 : 4) * BOX_BYTES);
   uint64_t* bar_u = bars + 0;   // state landed (TMA)
   uint64_t* bar_a = bars + 1;   // queries landed (one arrival per warp)
   uint64_t* bar_d = bars + 2;   // product in TMEM
@@ -1049,23 +1055,26 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
     mbar_init(bar_u, 1); mbar_init(bar_a, 4); mbar_init(bar_d, 1); mbar_init(bar_e, 4);
     fence_barrier_init();
   }
-  if (warp == 4) tmem_alloc(tmem_slot, TILE);
+  if (warp == 4) tmem_alloc(tmem_slot, DUAL ? 2 * TILE : TILE);
   fence_before_sync();
   __syncthreads();
   fence_after_sync();
   const uint32_t tmem_d = *tmem_slot;
   constexpr uint32_t idesc = make_idesc(TILE, TILE, 0, TRANS ? 0 : 1);
+  constexpr uint32_t idesc2 = make_idesc(TILE, TILE, 0, 1);
   ReadPass cur(prm, blockIdx.x, gridDim.x);
 
   if (warp < 4) {
     const int tid = threadIdx.x;
-    const uint32_t a_base = smem_u32(sA);
+    const uint32_t a_base = smem_u32(sA), a2_base = smem_u32(sA2);
     auto gather = [&](const ReadPass& ps) {
       const int kn = ps.tokens();
       for (int idx = tid; idx < kn * 16; idx += 128) {
         const int m = idx >> 4, gc = idx & 15;
-        const __nv_bfloat16* src = prm.X + ((ps.bh * prm.T + ps.token(m)) * TILE + gc * 8);
-        cp_async16_tc(a_base + (gc >> 3) * BOX_BYTES + m * 128 + (((gc & 7) ^ (m & 7)) << 4), src);
+        const int64_t row = (ps.bh * prm.T + ps.token(m)) * TILE + gc * 8;
+        const uint32_t off = (gc >> 3) * BOX_BYTES + m * 128 + (((gc & 7) ^ (m & 7)) << 4);
+        cp_async16_tc(a_base + off, prm.X + row);
+        if (DUAL) cp_async16_tc(a2_base + off, prm.X2 + row);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -1086,14 +1095,15 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
       const int m = warp * 32 + lane, kn = cur.tokens();
       const int64_t row = (cur.bh * prm.T + (m < kn ? cur.token(m) : 0)) * TILE;
       float4* dst = reinterpret_cast<float4*>(prm.out + row);
-      __nv_bfloat16* dst16 = prm.out_bf16 + row;
 #pragma unroll
-      for (int cb = 0; cb < 4; ++cb) {
+      for (int cbo = 0; cbo < (DUAL ? 8 : 4); ++cbo) {
+        const int cb = cbo & 3;
+        __nv_bfloat16* dst16 = (cbo < 4 ? prm.out_bf16 : prm.out2_bf16) + row;
         uint32_t v[32];
-        tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cb * 32, v);
+        tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + cbo * 32, v);
         tmem_ld_wait();
         if (m < kn) {
-          if (prm.out_bf16) {
+          if (DUAL || prm.out_bf16) {
 #pragma unroll
             for (int h8 = 0; h8 < 2; ++h8) {
               uint32_t w[8];
@@ -1118,6 +1128,7 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
   } else if (lane == 0) {
+    (void)idesc2;
     auto load_state = [&](int64_t item) {
       mbar_expect_tx(bar_u, 2 * BOX_BYTES);
       const int row = (int)(item * TILE);
@@ -1140,6 +1151,14 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
                                   : make_desc(smem_u32(sB) + kk * 2048, BOX_BYTES, 1024);
         mma_bf16(tmem_d, dA, dB, idesc, kk != 0);
       }
+      if (DUAL) {
+#pragma unroll
+        for (int kk = 0; kk < TILE / 16; ++kk) {   // the second rows against the state as it lies (MN-major B)
+          const uint64_t dA = make_desc(smem_u32(sA2) + (kk >> 2) * BOX_BYTES + (kk & 3) * 32, 16, 1024);
+          const uint64_t dB = make_desc(smem_u32(sB) + kk * 2048, BOX_BYTES, 1024);
+          mma_bf16(tmem_d + TILE, dA, dB, idesc2, kk != 0);
+        }
+      }
       mma_commit(bar_d);
       // the state tile may be overwritten (next item) only after the MMAs have read it
       ok = mbar_wait(bar_d, n_pass & 1, wc);
@@ -1156,7 +1175,7 @@ __global__ void __launch_bounds__(160) state_read_tc_kernel(const __grid_constan
   __syncthreads();
   if (warp == 4) {
     fence_after_sync();
-    tmem_dealloc(tmem_d, TILE);
+    tmem_dealloc(tmem_d, DUAL ? 2 * TILE : TILE);
   }
 }
 
@@ -1508,6 +1527,32 @@ cudaError_t smat_launch_bwd_tiles_fused_tc(const void* Q, const void* K, const v
   return cudaGetLastError();
 }
 
+// Both adjoint reads of the profile states in one launch: out_t[t] = St x_t (rows Xt, the second state index
+// contracted) and out_n[t] = Stᵀ x_t (rows Xn, the first one), bf16 rows; every state is loaded once.
+cudaError_t smat_launch_state_read_dual_tc(const void* Xt, const void* Xn, const void* state_bf16, void* out_t_bf16,
+                                           void* out_n_bf16, const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh,
+                                           int* status, cudaStream_t st) {
+  CUtensorMap tmU;
+  if (!make_map(&tmU, state_bf16, (uint64_t)bh * groups * TILE)) return cudaErrorInvalidValue;
+  ReadParams prm;
+  prm.T = T; prm.grp = grp; prm.groups = groups; prm.items = (int64_t)bh * groups;
+  prm.X = static_cast<const __nv_bfloat16*>(Xt);
+  prm.X2 = static_cast<const __nv_bfloat16*>(Xn);
+  prm.out = nullptr;
+  prm.out_bf16 = static_cast<__nv_bfloat16*>(out_t_bf16);
+  prm.out2_bf16 = static_cast<__nv_bfloat16*>(out_n_bf16);
+  prm.status = status;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int smem = READ_SMEM + 2 * BOX_BYTES;
+  const int64_t grid = prm.items < 2LL * sms ? prm.items : 2LL * sms;   // 256 columns of tensor memory and 97 KB each
+  cudaError_t err = cudaFuncSetAttribute(state_read_tc_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (err != cudaSuccess) return err;
+  state_read_tc_kernel<1, 1><<<(unsigned)grid, 160, smem, st>>>(tmU, prm);
+  return cudaGetLastError();
+}
+
 cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, float* out, void* out_bf16, int transposed,
                                       const SmatGroupSpec& grp, int64_t groups, int64_t T, int bh, int* status,
                                       cudaStream_t st) {
@@ -1516,6 +1561,7 @@ cudaError_t smat_launch_state_read_tc(const void* X, const void* state_bf16, flo
   ReadParams prm;
   prm.T = T; prm.grp = grp; prm.groups = groups; prm.items = (int64_t)bh * groups;
   prm.X = static_cast<const __nv_bfloat16*>(X);
+  prm.X2 = nullptr; prm.out2_bf16 = nullptr;
   prm.out = out;
   prm.out_bf16 = static_cast<__nv_bfloat16*>(out_bf16);
   prm.status = status;

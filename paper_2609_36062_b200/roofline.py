@@ -119,6 +119,7 @@ def stage_work(name: str, T, c, r, p, e, geo, u_bytes=4, f_bytes=4) -> Work:
         "bwd_dq_type_tc": Work(2 * m * rp, 0, m * p * e + B * su + m * r * 2),
         "bwd_dk_profile_tc": Work(2 * n * rp, 0, n * p * e + P * sf + n * r * 2),
         "bwd_dv_profile_tc": Work(2 * n * rp, 0, n * r * e + P * sf + n * p * 2),
+        "bwd_dkdv_profile_tc": Work(4 * n * rp, 0, n * (r + p) * e + P * sf + n * (r + p) * 2),
         "bwd_suffix_scan_tc": Work(2 * T * rp, tc_tiles * rp, T * (r + p) * e + tc_tiles * rp * 2),
         # dQ, dK, dV of every 128-token tile: eight 128 x 128 x 128 products per tile; reads Q, K, V, dO, the two
         # per-tile states and the three long-range buffers (bf16), writes the three gradients

@@ -339,6 +339,7 @@ def test_fused_and_separate_tile_adjoints_agree(d, T):
     fused.check_status()
     b = separate.backward(dev["q"], dev["k"], dev["v"], dev["do"])
     separate.check_status()
-    assert fused.last_launch_count() == separate.last_launch_count() - 2
+    # one tile kernel instead of three, and (d >= 2) one read of the per-profile adjoint states instead of two
+    assert fused.last_launch_count() == separate.last_launch_count() - (2 if d == 1 else 3)
     for x, y in zip(a, b):
         assert rel_err(to_numpy64(x), to_numpy64(y)) <= 2e-3
