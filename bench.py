@@ -378,18 +378,27 @@ class Runner:
         return [(n, acc[n] / steps) for n in order]
 
 
-def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4, gated_tc_forward=False):
+def gated_tc_mode(plan) -> int:
+    """0: not a gated plan on the tensor cores; 1: its forward only; 2: forward and backward."""
+    if not plan.gated_forward_uses_tensor_cores():
+        return 0
+    return 2 if plan.gated_backward_uses_tensor_cores() else 1
+
+
+def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4, gated_tc_forward=0):
     """Fractions against the path roofline.  The bytes are those of the design that ran: where a table is kept as
     bf16 its round trip is charged at 2 bytes per entry, and the fraction against the roofline with fp32 tables is
-    given beside it.  A gated plan whose forward runs on the tensor cores keeps bf16 tables there, while its backward
-    rebuilds fp32 tables on the ALU kernels: each pass is charged with its own."""
+    given beside it.  gated_tc_forward: 0 = not a gated tensor-core pass; 1 = a gated plan whose forward runs on the
+    tensor cores (bf16 tables) while its backward rebuilds fp32 tables on the ALU kernels; 2 = both passes on the
+    tensor cores.  Each pass is charged with the tables it keeps."""
     e = 4 if w.dtype == "f32" else 2
     def total(ub, fb):
         if gated_tc_forward and (ub, fb) != (4, 4):
             wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, 2, 2)
-            if w.backward:
-                wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, 4, 4, keep_forward_tables=False,
-                                                 f_bytes=4, ubar_bytes=4)
+            if w.backward:   # the gated backward rebuilds the forward tables; fp32 tables where it runs on the ALU kernels
+                tb = 2 if gated_tc_forward == 2 else 4
+                wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, tb, tb, keep_forward_tables=False,
+                                                 f_bytes=tb, ubar_bytes=tb)
             return wk.scaled(w.bh)
         wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub, fb)
         if w.backward:  # bench.py's fwd+bwd step keeps the forward's tables; the adjoint tables follow the forward's
@@ -534,7 +543,7 @@ def run_native(args):
             "gpu_launches": launches * steps,
             "clocks": clocks,
             "roofline": dominant_kernel_report(w, g, stages, peaks, ub, fb),
-            "path_roofline": path_report(w, g, per_step, peaks, ub, fb, runner.plan.gated_forward_uses_tensor_cores()),
+            "path_roofline": path_report(w, g, per_step, peaks, ub, fb, gated_tc_mode(runner.plan)),
             "tables": {"profile_states_P": g.P, "cached_subset_states_B": g.B, "nnzC": g.nnzC, "q": g.q},
             "fadd_rates_adds_per_s": peaks.get("fadd_rates"),
         }
@@ -552,7 +561,7 @@ def run_native(args):
             each_ = r.time_each(r.step, 15, 5)
             s = float(np.median(each_))
             rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes(), r.plan.profile_table_element_bytes(),
-                              r.plan.gated_forward_uses_tensor_cores())
+                              gated_tc_mode(r.plan))
             st_ = r.stage_profile(3)
             dom = dominant_kernel_report(ws_, gg, st_, peaks, r.plan.type_table_element_bytes(),
                                          r.plan.profile_table_element_bytes())

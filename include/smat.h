@@ -75,8 +75,8 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
 #define SMAT_FLAG_SEPARATE_TILE_ADJOINTS 256u /* tensor-core backward: dQ, dK, dV of a tile by three launches of the general
                                                  tile-product kernel instead of the one fused kernel (for comparison) */
 #define SMAT_FLAG_GATED 64u          /* the plan serves smat_forward_gated / smat_backward_gated: its workspace holds λ and the
-                                        rescaled copies of Q, K, V, dO.  The backward runs on the fp32-ALU kernels; the
-                                        forward on the tensor cores where the shape allows (with SMAT_FLAG_SIMT_ONLY: never) */
+                                        rescaled copies of Q, K, V, dO.  Both passes run on the tensor cores where the
+                                        shape allows (with SMAT_FLAG_SIMT_ONLY: never), else on the fp32-ALU kernels */
 
 #define SMAT_FLAG_NORMALIZED 128u    /* the plan serves smat_forward_normalized / smat_backward_normalized: its workspace
                                         also holds the augmented values, the unnormalised rows and their upstream */
@@ -114,10 +114,12 @@ smat_status smat_get_geometry(const smat_plan* plan, smat_geometry* out);
  * A property of the shape, not of the device. */
 int smat_uses_tensor_cores(const smat_plan* plan);
 
-/* 1 when smat_forward_gated of this plan (SMAT_FLAG_GATED) runs on the tensor-core kernels: the same shape rule as
- * above.  The gated backward, and the gated forward of every other shape, run on the fp32 ALUs; smat_uses_tensor_cores
- * of a gated plan is therefore 0. */
+/* 1 when smat_forward_gated / smat_backward_gated of this plan (SMAT_FLAG_GATED) run on the tensor-core kernels: the
+ * same shape rule as above (the backward also needs the plan to keep its tables in bf16, which the tabulation flags
+ * can prevent).  Every other shape runs on the fp32 ALUs.  The gated passes go through a plan of their own inside the
+ * gated plan; smat_uses_tensor_cores of a gated plan itself is 0. */
 int smat_gated_forward_uses_tensor_cores(const smat_plan* plan);
+int smat_gated_backward_uses_tensor_cores(const smat_plan* plan);
 
 /* Bytes per element of the type table U as smat_forward keeps it: 4 (fp32), or 2 when the plan runs the typed read on
  * the tensor cores (bf16 inputs; d >= 3, or d = 2 with at least 12 tokens per profile): there U is only ever a bf16
@@ -206,8 +208,9 @@ smat_status smat_backward_normalized(const smat_plan* plan, const void* Q, const
  * into k_j before pooling and a query-side scalar on the typed read, so tables and tabulation are the ungated ones of
  * rescaled inputs.  Every factor is the exponential of a non-positive difference: nothing overflows however strong
  * the decay.  smat_backward_gated also returns dlog_a [batch*heads, T] (DEVICE fp32), the gradient with respect to the
- * log-gates.  The plan must carry SMAT_FLAG_GATED (else SMAT_ERR_UNSUPPORTED).  The forward runs on the tensor
- * cores where smat_gated_forward_uses_tensor_cores says so, everything else of this variant on the fp32-ALU kernels.
+ * log-gates.  The plan must carry SMAT_FLAG_GATED (else SMAT_ERR_UNSUPPORTED).  The passes run on the tensor
+ * cores where smat_gated_forward_uses_tensor_cores / smat_gated_backward_uses_tensor_cores say so, else on the fp32-ALU
+ * kernels.
  * Otherwise as smat_forward / smat_backward.
  */
 smat_status smat_forward_gated(const smat_plan* plan, const void* Q, const void* K, const void* V, const float* log_a,

@@ -29,7 +29,7 @@ FLAG_SEPARATE_TILE_ADJOINTS = 256
 EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
-    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_gated_forward_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
+    "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_gated_forward_uses_tensor_cores", "smat_gated_backward_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
     "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step",
     "smat_static_check_status", "smat_debug_timeout_probe", "smat_measure_fadd_rate",
     "smat_forward_routed", "smat_backward_routed", "smat_forward_gated", "smat_backward_gated",
@@ -126,6 +126,8 @@ def load_library() -> ctypes.CDLL:
     lib.smat_uses_tensor_cores.restype = i
     lib.smat_gated_forward_uses_tensor_cores.argtypes = [vp]
     lib.smat_gated_forward_uses_tensor_cores.restype = i
+    lib.smat_gated_backward_uses_tensor_cores.argtypes = [vp]
+    lib.smat_gated_backward_uses_tensor_cores.restype = i
     lib.smat_forward_causal_static.argtypes = [vp, vp, vp, vp, i, i, i64, vp]
     lib.smat_forward_causal_static.restype = i
     lib.smat_static_check_status.argtypes = [vp]
@@ -238,6 +240,9 @@ class SmatPlan:
 
     def gated_forward_uses_tensor_cores(self) -> bool:
         return bool(self.lib.smat_gated_forward_uses_tensor_cores(self.handle))
+
+    def gated_backward_uses_tensor_cores(self) -> bool:
+        return bool(self.lib.smat_gated_backward_uses_tensor_cores(self.handle))
 
     def type_table_element_bytes(self) -> int:
         return int(self.lib.smat_type_table_element_bytes(self.handle))

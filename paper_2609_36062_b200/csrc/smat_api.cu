@@ -440,7 +440,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
     if (smat_plan_create(&in, batch, heads, T, d_k, d_v, d, chunk, q_override, dtype,
                          (flags & keep) | SMAT_FLAG_PER_TILE_STATES) == SMAT_OK && in->tc) {
       pl->inner = in;
-      off = align_up(off + in->off_fwd_end);
+      off = align_up(off + in->off_bwd_end);   // the gated backward runs through the same inner plan
     } else if (in) {
       smat_plan_destroy(in);
     }
@@ -507,6 +507,10 @@ smat_status smat_get_geometry(const smat_plan* pl, smat_geometry* out) {
 int smat_uses_tensor_cores(const smat_plan* pl) { return pl && pl->tc ? 1 : 0; }
 
 int smat_gated_forward_uses_tensor_cores(const smat_plan* pl) { return pl && pl->inner ? 1 : 0; }
+
+int smat_gated_backward_uses_tensor_cores(const smat_plan* pl) {
+  return pl && pl->inner && (pl->geo.dense_G || (pl->inner->u_bf16 && pl->inner->fbar_bf16)) ? 1 : 0;
+}
 
 int smat_type_table_element_bytes(const smat_plan* pl) { return pl && pl->u_bf16 ? 2 : 4; }
 
@@ -842,6 +846,73 @@ smat_status forward_gated_tc(Ctx& cx, const Gated& gt, const void* Q, const void
   return ci.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
 }
 
+// The gated backward runs on the tensor cores when the forward does and the inner plan keeps bf16 tables (the fused
+// tile kernel takes its long-range rows as bf16); d = 1 has no tables.
+bool gated_backward_on_tc(const smat_plan* pl) {
+  const smat_plan* in = pl->inner;
+  return in && (pl->geo.dense_G || (in->u_bf16 && in->fbar_bf16));
+}
+
+// Gated backward on the tensor cores: the ungated adjoint pipeline on rescaled copies (Ū from the boundary-scaled
+// queries, the reads of U and F̄ on the boundary-scaled dO, V and K), the decayed scans for S_in (keys rescaled to the
+// end of their tile) and D̄ (queries rescaled to the start of theirs, reverse order), and the fused tile kernel with
+// the decays on both score tiles and the row factors on the three state products.  dλ_t = q_t·dQ_t - k_t·dK_t.
+smat_status backward_gated_tc(Ctx& cx, const Gated& gt, const void* Q, const void* K, const void* V, const float* log_a,
+                              const void* dO, void* dQ, void* dK, void* dV, float* dlog_a) {
+  const smat_plan* pl = cx.pl;
+  const smat_plan* in = pl->inner;
+  const bool lr = !pl->geo.dense_G;
+  Ctx ci{in, cx.st, cx.ws + pl->off_inner, cudaSuccess, 0};
+  ci.rec = pl;
+  int* status = reinterpret_cast<int*>(ci.ws + in->off_status);
+  const int64_t n = in->geo.n;
+  SMAT_TRY(cx, "gate_prefix", smat_launch_head_scan(log_a, gt.lam, pl->T, pl->bh, 0, cx.st));
+  SMAT_TRY(cx, "gate_scale_k", smat_launch_gate_scale(K, nullptr, gt.kc, gt.lam, 1, 1, n, 128, pl->T, pl->r, pl->bh, cx.st));
+  SMAT_TRY(cx, "bwd_gate_scale_q", smat_launch_gate_scale(Q, nullptr, gt.qc, gt.lam, 0, 1, n, 128, pl->T, pl->r, pl->bh, cx.st));
+  if (lr) {
+    gate_scale(cx, "gate_scale_lr", K, Q, gt.lr, gt.lam, 2, pl->r);
+    gate_scale(cx, "bwd_gate_scale_lr", V, dO, gt.vlr, gt.lam, 2, pl->p);
+  }
+  ci.err = cx.err;
+  char* sin = ci.ws + in->off_sin;
+  char* dbar = ci.ws + in->off_dbar;
+  char *lr_q = nullptr, *lr_k = nullptr, *lr_v = nullptr;
+  if (lr) {
+    const SmatGroupSpec types = group(ci, SMAT_GM_TYPE), profs = group(ci, SMAT_GM_PROFILE);
+    build_type_table(ci, gt.lr, V);
+    if (in->ubar_tc)
+      SMAT_TRY(ci, "bwd_pool_type_tc", smat_launch_pool_tc(gt.lr, dO, ci.ws + in->off_ubar, in->ubar_bf16, types, in->geo.B,
+                                                           max_group_tokens(in, SMAT_GM_TYPE), in->T, in->bh, status, ci.st));
+    else
+      outer_sum(ci, "bwd_pool_type", SMAT_GM_TYPE, gt.lr, dO, ci.f(in->off_ubar));
+    if (in->tab_tc)
+      tabulate_tc(ci, "bwd_tabulate_t_tc", ci.ws + in->off_ubar, ci.ws + in->off_fbar, 1);
+    else
+      tabulate(ci, "bwd_tabulate_t", ci.f(in->off_ubar), ci.f(in->off_fbar), 1, in->geo.D == 2 && in->fbar_bf16);
+    lr_q = ci.ws + in->off_acc;
+    lr_k = lr_q + (size_t)in->bh * in->T * 128 * 2;
+    lr_v = ci.ws + in->off_lr3;
+    SMAT_TRY(ci, "bwd_dq_type_tc", smat_launch_state_read_tc(gt.vlr, ci.ws + in->off_U, nullptr, lr_q, 1, types, in->geo.B,
+                                                             in->T, in->bh, status, ci.st));
+    SMAT_TRY(ci, "bwd_dkdv_profile_tc", smat_launch_state_read_dual_tc(gt.vlr, gt.lr, ci.ws + in->off_fbar, lr_k, lr_v, profs,
+                                                                        in->geo.P, in->T, in->bh, status, ci.st));
+  }
+  SMAT_TRY(ci, "gated_chunk_scan_tc", smat_launch_chunk_scan_tc(gt.kc, V, sin, in->T, in->bh, n, lr ? 0 : 1, 0, status, ci.st,
+                                                                 gt.lam));
+  SMAT_TRY(ci, "bwd_gated_suffix_scan_tc", smat_launch_chunk_scan_tc(gt.qc, dO, dbar, in->T, in->bh, n, lr ? 0 : 1, 1, status,
+                                                                      ci.st, gt.lam));
+  SMAT_TRY(ci, "bwd_gated_tiles_fused_tc", smat_launch_bwd_tiles_fused_tc(Q, K, V, dO, sin, dbar, lr_q, lr_k, lr_v,
+                                                                           lr ? n : in->T, dQ, dK, dV, in->T, in->bh, status,
+                                                                           ci.st, gt.lam));
+  cx.err = ci.err;
+  cx.launches += ci.launches;
+  float* dlam = cx.f(pl->off_dlam);
+  SMAT_TRY(cx, "bwd_gate_dlam", smat_launch_gate_dlam(Q, dQ, K, dK, dlam, 1, pl->r, pl->T, pl->bh, cx.st));
+  SMAT_TRY(cx, "bwd_gate_suffix", smat_launch_head_scan(dlam, dlog_a, pl->T, pl->bh, 1, cx.st));
+  pl->launches = cx.launches;
+  return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
 smat_status gated_check(const smat_plan* pl, const void* log_a, void* ws, size_t ws_bytes, int for_backward) {
   if (!log_a) return SMAT_ERR_NULL;
   smat_status s = check_common(pl, ws, ws_bytes, for_backward);
@@ -943,6 +1014,7 @@ smat_status smat_backward_gated(const smat_plan* pl, const void* Q, const void* 
   cx.err = clear_status(cx);
   const bool lr = !pl->geo.dense_G;
   const Gated gt = gated_buffers(cx);
+  if (gated_backward_on_tc(pl)) return backward_gated_tc(cx, gt, Q, K, V, log_a, dO, dQ, dK, dV, dlog_a);
   gated_forward_tables(cx, gt, Q, K, V, log_a);
   gate_scale(cx, "bwd_gate_scale_do", dO, nullptr, gt.doc, gt.lam, 0, pl->p);    // exp(λ_i - λ_{e(b-1)}) dO_i
   gate_scale(cx, "bwd_gate_scale_v", V, nullptr, gt.vc, gt.lam, 1, pl->p);       // exp(λ_{e(b)} - λ_j) v_j

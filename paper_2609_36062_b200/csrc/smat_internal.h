@@ -117,8 +117,8 @@ bool smat_tc_available();
 // S_in[bh][tile] (bf16 [128][128]) = exclusive prefix sum of K_bᵀ V_b over the tiles of each block;
 // through = 1 runs one scan over the whole sequence (d = 1), else the scan restarts at token n.
 // reverse = 1 gives exclusive suffix sums instead (the scan adjoint, with K, V replaced by Q, dO).
-// lam (gated variant, forward order): inclusive prefix sums of the log-gates [bh][T]; K then holds the keys rescaled to
-// the end of their tile, and the running state decays by the tile's total gate.
+// lam (gated variant): inclusive prefix sums of the log-gates [bh][T]; K then holds the rows rescaled to the end of
+// their tile (forward order) or to its start (reverse order), and the running state decays by the tile's total gate.
 cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf16, int64_t T, int bh, int64_t n,
                                       int through, int reverse, int* status, cudaStream_t st, const float* lam = nullptr);
 // Within-chunk adjoints on tensor cores (which = 0: dQ, 1: dK, 2: dV), see tile_product_tc_kernel.
@@ -130,7 +130,7 @@ cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K
 cudaError_t smat_launch_bwd_tiles_fused_tc(const void* Q, const void* K, const void* V, const void* dO,
                                            const void* Sin_bf16, const void* Dbar_bf16, const void* lr_q, const void* lr_k,
                                            const void* lr_v, int64_t n, void* dQ, void* dK, void* dV, int64_t T, int bh,
-                                           int* status, cudaStream_t st);
+                                           int* status, cudaStream_t st, const float* lam = nullptr);
 // O_b = Q_b S_in[b] + tril(Q_b K_bᵀ) V_b (+ ylr rows for tokens >= n_lr).
 cudaError_t smat_launch_chunk_output_tc(const void* Q, const void* K, const void* V, const void* Sin_bf16,
                                         const float* ylr, int64_t n_lr, void* O, int64_t T, int bh, int* status,

@@ -41,8 +41,9 @@ struct ScanParams {
   int NC;           // tiles per head
   int lo[2], hi[2]; // tile ranges of the (up to two) blocks
   int reverse;      // 0: exclusive prefix sums (S_in); 1: exclusive suffix sums (the scan adjoint D̄)
-  const float* lam; // gated variant (forward order only): inclusive prefix sums of the log-gates, [bh][T]; the running
-                    // state is multiplied by the tile's total gate before the tile's (key-rescaled) sum is added
+  const float* lam; // gated variant: inclusive prefix sums of the log-gates, [bh][T]; the running state is multiplied by
+                    // the tile's total gate before the tile's sum (of rows rescaled to the tile's end, or in reverse
+                    // order to its start) is added — the same recursion in both directions
   __nv_bfloat16* Sin;  // [bh][NC][128][128]
   int* status;
 };
@@ -395,17 +396,23 @@ __global__ void __launch_bounds__(160) tile_product_tc_kernel(const __grid_const
 //   warps 0-3     : one tile row per thread: mask and round G, later A, into the swizzled X tile; read the three
 //                   accumulators, add the long-range rows and store
 // ---------------------------------------------------------------------------------------------------------------
-constexpr int FUSED_SMEM = 14 * BOX_BYTES + 1024 + 256;
+constexpr int FUSED_SMEM = 14 * BOX_BYTES + 1024 + 256 + TILE * 4;   // tiles, alignment, barriers, the tile's λ (gated)
 
 struct FusedParams {
   int64_t T;
   int NC;
   int64_t n;                         // rows t >= n add lr_q to dQ; rows t < n add lr_k, lr_v to dK, dV (when non-null)
   const __nv_bfloat16 *lr_q, *lr_k, *lr_v;   // [bh][T][128] bf16
+  const float* lam;                  // GATED: inclusive prefix sums of the log-gates [bh][T]
   __nv_bfloat16 *dQ, *dK, *dV;       // [bh][T][128]
   int* status;
 };
 
+// GATED (Lemma "Gated SMat", adjoint side): both score tiles are multiplied by exp(λ_i - λ_j) as they are rounded, and
+// the three state products are scaled row by row in tensor memory before the score products are added to them — row i
+// of dO S_inᵀ by exp(λ_i - λ_{last token before the tile}), row j of V D̄ᵀ and of K D̄ by exp(λ_{last token of the
+// tile} - λ_j).  S_in and D̄ are the decayed per-tile states.
+template <bool GATED>
 __global__ void __launch_bounds__(160) bwd_tile_fused_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                 const __grid_constant__ CUtensorMap tmK,
                                                                 const __grid_constant__ CUtensorMap tmV,
@@ -429,16 +436,20 @@ __global__ void __launch_bounds__(160) bwd_tile_fused_tc_kernel(const __grid_con
   uint64_t* bar_p = bars + 3;     // X written (one arrival per warp; two phases)
   uint64_t* bar_x = bars + 4;     // the MMAs that read X = G have finished: dQ, dK complete, X may be overwritten
   uint64_t* bar_o = bars + 5;     // dV complete
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6);
+  uint64_t* bar_st = bars + 6;    // GATED: the three state products are in tensor memory
+  uint64_t* bar_sl = bars + 7;    // GATED: ... and scaled (one arrival per warp)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* sLam = reinterpret_cast<float*>(smem + 14 * BOX_BYTES + 256);   // [128] λ of the tile's tokens (GATED)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.x, bh = blockIdx.y;
   const int64_t row0 = (int64_t)bh * prm.T + (int64_t)b * TILE;
   const WaitCtx wc{cta_abort, prm.status};
+  if (GATED && threadIdx.x < TILE) sLam[threadIdx.x] = prm.lam[row0 + threadIdx.x];
   if (threadIdx.x == 0) {
     *cta_abort = 0;
     mbar_init(bar_in0, 1); mbar_init(bar_in1, 1); mbar_init(bar_sc, 1); mbar_init(bar_p, 4); mbar_init(bar_x, 1);
-    mbar_init(bar_o, 1);
+    mbar_init(bar_o, 1); mbar_init(bar_st, 1); mbar_init(bar_sl, 4);
     fence_barrier_init();
   }
   if (warp == 4) tmem_alloc(tmem_slot, 512);
@@ -486,7 +497,9 @@ __global__ void __launch_bounds__(160) bwd_tile_fused_tc_kernel(const __grid_con
       for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_dk, kmaj(sV, kk), kmaj(sD, kk), id_kk, kk != 0);   // V D̄ᵀ
 #pragma unroll
       for (int kk = 0; kk < TILE / 16; ++kk) mma_bf16(tm_dv, kmaj(sK, kk), mnmaj(sD, kk), id_km, kk != 0);  // K D̄
+      if (GATED) mma_commit(bar_st);
       ok = mbar_wait(bar_p, 0, wc);          // X = G in shared memory; the G scores have left tensor memory
+      if (GATED && ok) ok = mbar_wait(bar_sl, 0, wc);   // the state products carry their row factors
     }
     if (ok) {
       fence_after_sync();
@@ -509,6 +522,7 @@ __global__ void __launch_bounds__(160) bwd_tile_fused_tc_kernel(const __grid_con
   } else if (warp < 4) {
     const int m = warp * 32 + lane;  // row inside the tile = TMEM lane
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const float lam_m = GATED ? sLam[m] : 0.f;
     // masked (column <= row), rounded copy of the score tile into X, swizzled as a K-major operand
     auto stage_scores = [&]() {
 #pragma unroll
@@ -522,8 +536,12 @@ __global__ void __launch_bounds__(160) bwd_tile_fused_tc_kernel(const __grid_con
 #pragma unroll
           for (int h2 = 0; h2 < 4; ++h2) {
             const int k0 = cb * 32 + i * 8 + h2 * 2;
-            const float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
-            const float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            float lo = (k0 <= m) ? __uint_as_float(v[i * 8 + h2 * 2]) : 0.f;
+            float hi = (k0 + 1 <= m) ? __uint_as_float(v[i * 8 + h2 * 2 + 1]) : 0.f;
+            if (GATED) {   // exponents of non-positive differences only
+              if (k0 <= m) lo *= __expf(lam_m - sLam[k0]);
+              if (k0 + 1 <= m) hi *= __expf(lam_m - sLam[k0 + 1]);
+            }
             pk[h2] = pack_bf16(lo, hi);
           }
           const int j8 = cb * 4 + i;
@@ -570,11 +588,38 @@ __global__ void __launch_bounds__(160) bwd_tile_fused_tc_kernel(const __grid_con
                        w[8 * h8 + 5], w[8 * h8 + 6], w[8 * h8 + 7]);
       }
     };
+    // GATED: one accumulator's rows times this row's factor, in place
+    auto scale_rows = [&](uint32_t tm_acc, float f) {
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tm_acc + lane_base + cb * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
+        tmem_st32(tm_acc + lane_base + cb * 32, v);
+      }
+    };
     bool ok = mbar_wait(bar_sc, 0, wc);
     if (ok) {
       fence_after_sync();
       stage_scores();                              // X = G
-      ok = mbar_wait(bar_sc, 1, wc);               // the A scores are in (the MMAs on G were issued before them)
+      if (GATED) {
+        ok = mbar_wait(bar_st, 0, wc);
+        if (ok) {
+          fence_after_sync();
+          const float row_in = __expf(lam_m - (b > 0 ? prm.lam[row0 - 1] : 0.f));   // queries' side: from the tile's start
+          const float row_out = __expf(sLam[TILE - 1] - lam_m);                       // keys' side: to the tile's end
+          scale_rows(tm_dq, row_in);
+          scale_rows(tm_dk, row_out);
+          scale_rows(tm_dv, row_out);
+          tmem_st_wait();
+          fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_sl);
+        }
+      }
+      if (ok) ok = mbar_wait(bar_sc, 1, wc);       // the A scores are in (the MMAs on G were issued before them)
     }
     if (ok) ok = mbar_wait(bar_x, 0, wc);          // ... and those MMAs have finished with X: dQ, dK are complete
     if (ok) {
@@ -1435,7 +1480,6 @@ bool smat_tc_available() {
 cudaError_t smat_launch_chunk_scan_tc(const void* K, const void* V, void* Sin_bf16, int64_t T, int bh, int64_t n,
                                       int through, int reverse, int* status, cudaStream_t st, const float* lam) {
   CUtensorMap tmK, tmV;
-  if (lam && reverse) return cudaErrorInvalidValue;   // the decayed recursion is built for the forward order only
   if (!make_map(&tmK, K, (uint64_t)bh * T) || !make_map(&tmV, V, (uint64_t)bh * T)) return cudaErrorInvalidValue;
   ScanParams prm;
   prm.lam = lam;
@@ -1506,7 +1550,7 @@ cudaError_t smat_launch_chunk_adjoint_tc(int which, const void* Q, const void* K
 cudaError_t smat_launch_bwd_tiles_fused_tc(const void* Q, const void* K, const void* V, const void* dO,
                                            const void* Sin_bf16, const void* Dbar_bf16, const void* lr_q, const void* lr_k,
                                            const void* lr_v, int64_t n, void* dQ, void* dK, void* dV, int64_t T, int bh,
-                                           int* status, cudaStream_t st) {
+                                           int* status, cudaStream_t st, const float* lam) {
   CUtensorMap tmQ, tmK, tmV, tmG, tmS, tmD;
   const int NC = (int)(T / TILE);
   if (!make_map(&tmQ, Q, (uint64_t)bh * T) || !make_map(&tmK, K, (uint64_t)bh * T) || !make_map(&tmV, V, (uint64_t)bh * T) ||
@@ -1520,10 +1564,12 @@ cudaError_t smat_launch_bwd_tiles_fused_tc(const void* Q, const void* K, const v
   prm.lr_v = static_cast<const __nv_bfloat16*>(lr_v);
   prm.dQ = static_cast<__nv_bfloat16*>(dQ); prm.dK = static_cast<__nv_bfloat16*>(dK); prm.dV = static_cast<__nv_bfloat16*>(dV);
   prm.status = status;
-  cudaError_t err = cudaFuncSetAttribute(bwd_tile_fused_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FUSED_SMEM);
+  prm.lam = lam;
+  auto kernel = lam ? bwd_tile_fused_tc_kernel<true> : bwd_tile_fused_tc_kernel<false>;
+  cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FUSED_SMEM);
   if (err != cudaSuccess) return err;
   dim3 grid((unsigned)NC, (unsigned)bh);
-  bwd_tile_fused_tc_kernel<<<grid, 160, FUSED_SMEM, st>>>(tmQ, tmK, tmV, tmG, tmS, tmD, prm);
+  kernel<<<grid, 160, FUSED_SMEM, st>>>(tmQ, tmK, tmV, tmG, tmS, tmD, prm);
   return cudaGetLastError();
 }
 

@@ -124,6 +124,24 @@ def test_tensor_core_gated_forward_against_oracle_rows_and_the_alu_path(d, T, c,
     # the pass is repeatable bit for bit
     O2 = plan.forward_gated(dev["q"], dev["k"], dev["v"], la_dev)
     assert torch.equal(O, O2)
+    # gradients: the tensor-core backward against the fp32-ALU one (itself held to the dense oracle on small shapes)
+    assert plan.gated_backward_uses_tensor_cores() and not alu.gated_backward_uses_tensor_cores()
+    host2, dev2 = device_inputs(w, ("q", "k", "v", "do"))
+    got = plan.backward_gated(dev2["q"], dev2["k"], dev2["v"], la_dev, dev2["do"])
+    plan.check_status()
+    ref = alu.backward_gated(dev2["q"], dev2["k"], dev2["v"], la_dev, dev2["do"])
+    for name, x, y in zip(("dQ", "dK", "dV"), got[:3], ref[:3]):
+        e = rel_err(to_numpy64(x), to_numpy64(y))
+        assert e <= 8e-3, (name, e)
+    e = rel_err(got[3].double().cpu().numpy(), ref[3].double().cpu().numpy())
+    assert e <= 5e-2, ("dlog_a", e)
+    if T <= 2048:   # and against the dense fp64 oracle where the T x T mask is small enough
+        M = so.dense_mask(T, c, d, q or None)
+        Q64, K64, V64, G64 = (synth.as_float64(w, host2[x][1]) for x in ("q", "k", "v", "do"))
+        rq, rk, rv, rl = so.gated_backward_dense(Q64, K64, V64, G64, M, la[1].astype(np.float64))
+        for name, x, r in (("dQ", got[0], rq), ("dK", got[1], rk), ("dV", got[2], rv)):
+            assert rel_err(to_numpy64(x[0, 1]), r) <= TOL["bf16"], (name,)
+        assert rel_err(got[3][1].double().cpu().numpy(), rl) <= 5e-2
 
 
 def test_tensor_core_gated_forward_under_strong_decay():
