@@ -170,12 +170,39 @@ cudaError_t smat_launch_gate_dlam(const void* Q, const void* dQ, const void* K, 
 // ---- normalised output (Sec. 2: augmented value v̄ = [v; 1], one final division) ------------------------------------
 namespace {
 
+// Four consecutive elements of a row, as one 8-byte (bf16) or 16-byte (fp32) access.
+template <typename T>
+struct Quad {
+  __align__(16) T v[4];
+  __device__ __forceinline__ void load(const T* src) {
+    if (sizeof(T) == 2) *reinterpret_cast<uint2*>(v) = *reinterpret_cast<const uint2*>(src);
+    else *reinterpret_cast<uint4*>(v) = *reinterpret_cast<const uint4*>(src);
+  }
+  __device__ __forceinline__ void store(T* dst) const {
+    if (sizeof(T) == 2) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(v);
+    else *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(v);
+  }
+};
+
+// The three row kernels below take one warp per row; rows whose length is a multiple of 128 move four elements per lane
+// and access (the elementwise form was bound by its 2-byte accesses and per-element index arithmetic).
+
 // V̄ = V with its last column set to one.
 template <typename T>
 __global__ void augment_value_kernel(const T* __restrict__ V, T* __restrict__ Vbar, int p, int64_t rows) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= rows * p) return;
-  Vbar[idx] = (int)(idx % p) == p - 1 ? (T)1.0f : V[idx];
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
+  if (row >= rows) return;
+  const int lane = threadIdx.x & 31;
+  if (p % 128 == 0) {
+    for (int i = lane * 4; i < p; i += 128) {
+      Quad<T> q;
+      q.load(V + row * p + i);
+      if (i + 4 == p) q.v[3] = (T)1.0f;
+      q.store(Vbar + row * p + i);
+    }
+    return;
+  }
+  for (int i = lane; i < p; i += 32) Vbar[row * p + i] = i == p - 1 ? (T)1.0f : V[row * p + i];
 }
 
 // O = ȳ_{1:p-1} / ȳ_p, and the normaliser ȳ_p itself in the last column.  One warp per row.
@@ -186,6 +213,16 @@ __global__ void normalize_rows_kernel(const T* __restrict__ Y, T* __restrict__ O
   const int lane = threadIdx.x & 31;
   const float den = (float)Y[row * p + p - 1];
   const float inv = 1.0f / den;
+  if (p % 128 == 0) {
+    for (int i = lane * 4; i < p; i += 128) {
+      Quad<T> q;
+      q.load(Y + row * p + i);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) q.v[k] = i + k == p - 1 ? (T)den : (T)((float)q.v[k] * inv);
+      q.store(O + row * p + i);
+    }
+    return;
+  }
   for (int i = lane; i < p; i += 32) O[row * p + i] = i == p - 1 ? (T)den : (T)((float)Y[row * p + i] * inv);
 }
 
@@ -199,6 +236,29 @@ __global__ void normalize_adjoint_kernel(const T* __restrict__ O, const T* __res
   const int lane = threadIdx.x & 31;
   const float inv = 1.0f / (float)O[row * p + p - 1];
   float dot = 0.f;
+  if (p % 128 == 0) {
+    float last = 0.f;   // dO of the normaliser column (held by the lane that owns the row's last quad)
+    for (int i = lane * 4; i < p; i += 128) {
+      Quad<T> g, o;
+      g.load(dO + row * p + i);
+      o.load(O + row * p + i);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (i + k == p - 1) { last = (float)g.v[k]; continue; }
+        dot += (float)g.v[k] * (float)o.v[k];
+        g.v[k] = (T)((float)g.v[k] * inv);
+      }
+      if (i + 4 != p) g.store(dY + row * p + i);
+      else {   // the last quad waits for the row's dot product
+#pragma unroll
+        for (int k = 0; k < 3; ++k) dY[row * p + i + k] = g.v[k];
+      }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, d);
+    if (lane == ((p - 4) % 128) / 4) dY[row * p + p - 1] = (T)(last - dot * inv);
+    return;
+  }
   for (int i = lane; i < p - 1; i += 32) {
     const float g = (float)dO[row * p + i];
     dot += g * (float)O[row * p + i];
@@ -220,7 +280,7 @@ template <typename T>
 cudaError_t normalize_step(int step, const void* a, const void* b, void* out, int p, int64_t rows, cudaStream_t st) {
   const unsigned warp_blocks = (unsigned)((rows * 32 + 255) / 256);
   if (step == 0)
-    augment_value_kernel<T><<<(unsigned)((rows * p + 255) / 256), 256, 0, st>>>(static_cast<const T*>(a), static_cast<T*>(out), p, rows);
+    augment_value_kernel<T><<<warp_blocks, 256, 0, st>>>(static_cast<const T*>(a), static_cast<T*>(out), p, rows);
   else if (step == 1)
     normalize_rows_kernel<T><<<warp_blocks, 256, 0, st>>>(static_cast<const T*>(a), static_cast<T*>(out), p, rows);
   else if (step == 2)
