@@ -343,3 +343,73 @@ def test_fused_and_separate_tile_adjoints_agree(d, T):
     assert fused.last_launch_count() == separate.last_launch_count() - (2 if d == 1 else 3)
     for x, y in zip(a, b):
         assert rel_err(to_numpy64(x), to_numpy64(y)) <= 2e-3
+
+
+# ---- the "next" rows at the sizes and in the launch configuration bench.py times ---------------------------------
+def _bench_plan(w):
+    flags = {"gated": binding.FLAG_GATED, "normalized": binding.FLAG_NORMALIZED}.get(w.variant, 0)
+    return binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype, flags=flags)
+
+
+def test_bench_workload_hashed_routing_sampled_rows():
+    w = synth.WORKLOADS["t16k_d4_hashed"]
+    host, dev = device_inputs(w)
+    plan = _bench_plan(w)
+    geo = so.geometry(w.T, w.chunk, w.d)
+    prof = np.stack([synth.hashed_cells(w, h, geo.n, geo.P) for h in range(w.bh)])
+    typ = np.stack([synth.hashed_types(w, h, geo.m, geo.B) for h in range(w.bh)])
+    O = plan.forward(dev["q"], dev["k"], dev["v"], prof=torch.from_numpy(prof).cuda(), type=torch.from_numpy(typ).cuda())
+    plan.check_status()
+    O = O.reshape(w.bh, w.T, w.d_v)
+    for h in (0, w.bh - 1):
+        Q64, K64, V64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v"))
+        rows = sample_tokens(geo, 64, seed=300 + h)
+        ref = so.routed_forward_rows(Q64, K64, V64, geo, prof[h], typ[h], rows)
+        assert rel_err(to_numpy64(O[h][rows]), ref) <= TOL[w.dtype], (h,)
+
+
+def test_bench_workload_normalized_sampled_rows():
+    w = synth.WORKLOADS["t16k_d4_normalized"]
+    host, dev = device_inputs(w)
+    plan = _bench_plan(w)
+    geo = so.geometry(w.T, w.chunk, w.d)
+    O = plan.forward_normalized(dev["q"], dev["k"], dev["v"])
+    plan.check_status()
+    O = O.reshape(w.bh, w.T, w.d_v)
+    for h in (0, w.bh - 1):
+        Q64, K64, V64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v"))
+        rows = sample_tokens(geo, 64, seed=400 + h)
+        ref, den = so.normalized_forward_rows(Q64, K64, V64[:, :-1], geo, rows)
+        got = to_numpy64(O[h][rows])
+        assert rel_err(got[:, :-1], ref) <= TOL[w.dtype], (h,)
+        assert rel_err(got[:, -1], den) <= TOL[w.dtype], (h,)            # the last column carries the normaliser
+
+
+@pytest.mark.parametrize("name", ["t4k_d3_gated", "t4k_d3_gated_fwdbwd"])
+def test_bench_workload_gated(name):
+    w = synth.WORKLOADS[name]
+    tensors = ("q", "k", "v", "do") if w.backward else ("q", "k", "v")
+    host, dev = device_inputs(w, tensors)
+    plan = _bench_plan(w)
+    assert plan.gated_forward_uses_tensor_cores()
+    geo = so.geometry(w.T, w.chunk, w.d)
+    la = np.stack([synth.log_gates(w, h) for h in range(w.bh)])
+    la_dev = torch.from_numpy(la).cuda()
+    O = plan.forward_gated(dev["q"], dev["k"], dev["v"], la_dev)
+    grads = plan.backward_gated(dev["q"], dev["k"], dev["v"], la_dev, dev["do"]) if w.backward else None
+    plan.check_status()
+    O = O.reshape(w.bh, w.T, w.d_v)
+    for h in (0, w.bh - 1):
+        Q64, K64, V64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v"))
+        rows = sample_tokens(geo, 64, seed=500 + h)
+        ref = so.gated_forward_rows(Q64, K64, V64, geo, la[h].astype(np.float64), rows)
+        assert rel_err(to_numpy64(O[h][rows]), ref) <= TOL[w.dtype], (h,)
+    if w.backward:   # one head against the dense fp64 adjoint (T = 4096: the mask is 16 M entries)
+        h = w.bh - 1
+        Q64, K64, V64, G64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v", "do"))
+        M = so.dense_mask(w.T, w.chunk, w.d)
+        rq, rk, rv, rl = so.gated_backward_dense(Q64, K64, V64, G64, M, la[h].astype(np.float64))
+        dQ, dK, dV = (g.reshape(w.bh, w.T, -1)[h] for g in grads[:3])
+        for nm, g, r in (("dQ", dQ, rq), ("dK", dK, rk), ("dV", dV, rv)):
+            assert rel_err(to_numpy64(g), r) <= TOL[w.dtype], (nm,)
+        assert rel_err(grads[3].reshape(w.bh, w.T)[h].double().cpu().numpy(), rl) <= 5e-2
