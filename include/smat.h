@@ -345,6 +345,19 @@ smat_status smat_decode_begin(const smat_plan* plan, const void* K, const void* 
 smat_status smat_decode_step(const smat_plan* plan, const void* q, const void* k, const void* v, int64_t t, void* o,
                              void* cache, size_t cache_bytes, void* cuda_stream);
 
+/* The same for the scalar-gated variant (Sec. 3.2, the streaming form of Lemma "Gated SMat"); the plan must carry
+ * SMAT_FLAG_GATED (the ungated pair of calls then returns SMAT_ERR_UNSUPPORTED, and these on an ungated plan):
+ *     S_t = a_t S_{t-1} + k_t v_t^T,   g_t = a_t g_{t-1}  (g_{n-1} = 1),   o_t = q_t^T (g_t U_type(t) + S_t),
+ * where the cached type table is built from the keys rescaled to the block boundary, exp(λ_{n-1} - λ_j) k_j.
+ * o_t equals row t of smat_forward_gated's O.  The cache holds, after the type table (bf16 where the plan's gated
+ * forward runs on the tensor cores, else fp32) and S, one fp32 word per (batch, head): log g.
+ * smat_decode_begin_gated : log_a DEVICE fp32 [B*H, T] as for smat_forward_gated (entries 0 .. n-1 of every head are used).
+ * smat_decode_step_gated  : log_a_t DEVICE fp32 [B*H], the log-gates of token t. */
+smat_status smat_decode_begin_gated(const smat_plan* plan, const void* K, const void* V, const float* log_a, void* cache,
+                                    size_t cache_bytes, void* workspace, size_t workspace_bytes, void* cuda_stream);
+smat_status smat_decode_step_gated(const smat_plan* plan, const void* q, const void* k, const void* v, const float* log_a_t,
+                                   int64_t t, void* o, void* cache, size_t cache_bytes, void* cuda_stream);
+
 /* Host-only self-check (the paper has no counterpart): 1 when, for field size q, the shared-memory map of every launch
  * shape of the tensor-core tabulation kernel (ring slots, extra-class rows, output-row table, barrier words) is
  * disjoint and inside the allocation, and no load box or staged tile can leave its slot; 0 otherwise.  The launcher

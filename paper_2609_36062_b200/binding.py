@@ -30,7 +30,7 @@ EXPORTS = [
     "smat_plan_create", "smat_plan_destroy", "smat_get_geometry", "smat_workspace_bytes", "smat_forward",
     "smat_backward", "smat_routing_indices", "smat_debug_mask", "smat_debug_tables", "smat_check_status",
     "smat_last_launch_count", "smat_status_string", "smat_profile_enable", "smat_profile_read", "smat_uses_tensor_cores", "smat_gated_forward_uses_tensor_cores", "smat_gated_backward_uses_tensor_cores", "smat_forward_causal_static", "smat_type_table_element_bytes",
-    "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step",
+    "smat_profile_table_element_bytes", "smat_decode_cache_bytes", "smat_decode_begin", "smat_decode_step", "smat_decode_begin_gated", "smat_decode_step_gated",
     "smat_static_check_status", "smat_debug_timeout_probe", "smat_measure_fadd_rate",
     "smat_forward_routed", "smat_backward_routed", "smat_forward_gated", "smat_backward_gated",
     "smat_forward_normalized", "smat_backward_normalized", "smat_debug_tabulation_layout_ok",
@@ -120,6 +120,10 @@ def load_library() -> ctypes.CDLL:
     lib.smat_decode_begin.restype = i
     lib.smat_decode_step.argtypes = [vp, vp, vp, vp, i64, vp, vp, ctypes.c_size_t, vp]
     lib.smat_decode_step.restype = i
+    lib.smat_decode_begin_gated.argtypes = [vp, vp, vp, vp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
+    lib.smat_decode_begin_gated.restype = i
+    lib.smat_decode_step_gated.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, ctypes.c_size_t, vp]
+    lib.smat_decode_step_gated.restype = i
     lib.smat_profile_table_element_bytes.argtypes = [vp]
     lib.smat_profile_table_element_bytes.restype = i
     lib.smat_uses_tensor_cores.argtypes = [vp]
@@ -396,6 +400,27 @@ class SmatPlan:
         o = torch.empty_like(v) if o is None else o
         _check(self.lib.smat_decode_step(self.handle, _ptr(q), _ptr(k), _ptr(v), int(t), _ptr(o), _ptr(cache), cache.numel(),
                                          _stream(stream)), "smat_decode_step")
+        return o
+
+    def decode_begin_gated(self, K, V, log_a, cache, workspace=None, stream=None) -> None:
+        _, _, _, dk, dv = self.shape
+        self._check_tensor(K, dk, "K"); self._check_tensor(V, dv, "V")
+        self._check_gates(log_a)
+        ws = self.workspace(False, K.device) if workspace is None else workspace
+        self._ws = ws
+        _check(self.lib.smat_decode_begin_gated(self.handle, _ptr(K), _ptr(V), _ptr(log_a), _ptr(cache), cache.numel(),
+                                                _ptr(ws), ws.numel(), _stream(stream)), "smat_decode_begin_gated")
+
+    def decode_step_gated(self, q, k, v, log_a_t, t: int, cache, o=None, stream=None):
+        b, h, _, dk, dv = self.shape
+        for name, x, dim in (("q", q, dk), ("k", k, dk), ("v", v, dv)):
+            if not (x.is_cuda and x.is_contiguous() and x.dtype == self.torch_dtype and tuple(x.shape) == (b, h, dim)):
+                raise ValueError(f"{name}: expected a contiguous CUDA tensor [{b}, {h}, {dim}] of the plan's dtype")
+        if not (log_a_t.is_cuda and log_a_t.is_contiguous() and log_a_t.dtype == torch.float32 and log_a_t.numel() == b * h):
+            raise ValueError(f"log_a_t: expected a contiguous CUDA fp32 tensor of {b * h} log-gates")
+        o = torch.empty_like(v) if o is None else o
+        _check(self.lib.smat_decode_step_gated(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(log_a_t), int(t), _ptr(o),
+                                               _ptr(cache), cache.numel(), _stream(stream)), "smat_decode_step_gated")
         return o
 
     # -- verification exports ------------------------------------------------------------------

@@ -348,9 +348,15 @@ size_t build_type_table(Ctx& cx, const void* K, const void* V) {
   return pl->off_U;
 }
 
-size_t decode_table_bytes(const smat_plan* pl) {
-  return align_up((size_t)pl->bh * pl->geo.B * pl->rp * (pl->u_bf16 ? 2 : 4));
+// The plan whose kernels build (and whose element type stores) the type table of the decode cache: a gated plan with
+// a tensor-core inner plan tabulates through that one.
+const smat_plan* decode_table_plan(const smat_plan* pl) {
+  return (pl->flags & SMAT_FLAG_GATED) && pl->inner ? pl->inner : pl;
 }
+size_t decode_table_bytes(const smat_plan* pl) {
+  return align_up((size_t)pl->bh * pl->geo.B * pl->rp * (decode_table_plan(pl)->u_bf16 ? 2 : 4));
+}
+size_t decode_state_bytes(const smat_plan* pl) { return align_up((size_t)pl->bh * pl->rp * sizeof(float)); }
 
 }  // namespace
 
@@ -1183,13 +1189,14 @@ int smat_last_launch_count(const smat_plan* pl) { return pl ? pl->launches : 0; 
 int smat_debug_tabulation_layout_ok(int q) { return smat_tabulate_tc_layout_ok(q); }
 
 size_t smat_decode_cache_bytes(const smat_plan* pl) {
-  if (!pl) return 0;
-  return decode_table_bytes(pl) + (size_t)pl->bh * pl->rp * sizeof(float);
+  if (!pl) return 0;   // type table, running state, and on gated plans the running log-gate of every head
+  return decode_table_bytes(pl) + decode_state_bytes(pl) + ((pl->flags & SMAT_FLAG_GATED) ? align_up((size_t)pl->bh * 4) : 0);
 }
 
 smat_status smat_decode_begin(const smat_plan* pl, const void* K, const void* V, void* cache, size_t cache_bytes,
                               void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!K || !V || !cache) return SMAT_ERR_NULL;
+  if (pl && (pl->flags & SMAT_FLAG_GATED)) return SMAT_ERR_UNSUPPORTED;   // gated plans decode with the gated pair of calls
   smat_status s = check_common(pl, workspace, workspace_bytes, 0);
   if (s != SMAT_OK) return s;
   if (cache_bytes < smat_decode_cache_bytes(pl)) return SMAT_ERR_WORKSPACE;
@@ -1212,6 +1219,7 @@ smat_status smat_decode_begin(const smat_plan* pl, const void* K, const void* V,
 smat_status smat_decode_step(const smat_plan* pl, const void* q, const void* k, const void* v, int64_t t, void* o,
                              void* cache, size_t cache_bytes, void* cuda_stream) {
   if (!pl || !q || !k || !v || !o || !cache) return SMAT_ERR_NULL;
+  if (pl->flags & SMAT_FLAG_GATED) return SMAT_ERR_UNSUPPORTED;
   if (cache_bytes < smat_decode_cache_bytes(pl)) return SMAT_ERR_WORKSPACE;
   if (t < pl->geo.n || t >= pl->T) return SMAT_ERR_SHAPE;
   if (reinterpret_cast<uintptr_t>(cache) & 255) return SMAT_ERR_ALIGN;
@@ -1220,6 +1228,53 @@ smat_status smat_decode_step(const smat_plan* pl, const void* q, const void* k, 
   const cudaError_t err = smat_launch_decode_step(q, k, v, o, S, cache, pl->u_bf16 ? 1 : 0, pl->dtype == SMAT_BF16 ? 1 : 0,
                                                   smat_type_of(pl->geo, t), pl->geo.B, pl->r, pl->p, pl->bh,
                                                   static_cast<cudaStream_t>(cuda_stream));
+  pl->launches = 1;
+  return err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
+smat_status smat_decode_begin_gated(const smat_plan* pl, const void* K, const void* V, const float* log_a, void* cache,
+                                    size_t cache_bytes, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!K || !V || !cache) return SMAT_ERR_NULL;
+  smat_status s = gated_check(pl, log_a, workspace, workspace_bytes, 0);
+  if (s != SMAT_OK) return s;
+  if (cache_bytes < smat_decode_cache_bytes(pl)) return SMAT_ERR_WORKSPACE;
+  if (misaligned(K) || misaligned(V) || (reinterpret_cast<uintptr_t>(cache) & 255)) return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
+  Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
+  pl->stages = 0;
+  cx.err = clear_status(cx);
+  const Gated gt = gated_buffers(cx);
+  // λ, the keys rescaled to the block boundary (rows t < n of the split copy), then steps 2-3 of Algorithm 1 on them
+  SMAT_TRY(cx, "gate_prefix", smat_launch_head_scan(log_a, gt.lam, pl->T, pl->bh, 0, cx.st));
+  gate_scale(cx, "gate_scale_lr", K, K, gt.lr, gt.lam, 2, pl->r);
+  const smat_plan* tp = decode_table_plan(pl);
+  Ctx ct{tp, cx.st, cx.ws + (tp == pl ? 0 : pl->off_inner), cx.err, 0};
+  ct.rec = pl;
+  const size_t off = build_type_table(ct, gt.lr, V);
+  cx.err = ct.err;
+  const size_t tbytes = (size_t)pl->bh * pl->geo.B * pl->rp * (tp->u_bf16 ? 2 : 4);
+  if (cx.err == cudaSuccess) cx.err = cudaMemcpyAsync(cache, ct.ws + off, tbytes, cudaMemcpyDeviceToDevice, cx.st);
+  if (cx.err == cudaSuccess)   // S = 0 and log g = 0 (they follow the table)
+    cx.err = cudaMemsetAsync(static_cast<char*>(cache) + decode_table_bytes(pl), 0,
+                             smat_decode_cache_bytes(pl) - decode_table_bytes(pl), cx.st);
+  pl->launches = cx.launches + ct.launches;
+  return cx.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
+}
+
+smat_status smat_decode_step_gated(const smat_plan* pl, const void* q, const void* k, const void* v, const float* log_a_t,
+                                   int64_t t, void* o, void* cache, size_t cache_bytes, void* cuda_stream) {
+  if (!pl || !q || !k || !v || !o || !cache || !log_a_t) return SMAT_ERR_NULL;
+  if (!(pl->flags & SMAT_FLAG_GATED)) return SMAT_ERR_UNSUPPORTED;
+  if (cache_bytes < smat_decode_cache_bytes(pl)) return SMAT_ERR_WORKSPACE;
+  if (t < pl->geo.n || t >= pl->T) return SMAT_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(cache) & 255) || (reinterpret_cast<uintptr_t>(log_a_t) & 3)) return SMAT_ERR_ALIGN;
+  if (!device_ok()) return SMAT_ERR_ARCH;
+  char* base = static_cast<char*>(cache);
+  float* S = reinterpret_cast<float*>(base + decode_table_bytes(pl));
+  float* log_g = reinterpret_cast<float*>(base + decode_table_bytes(pl) + decode_state_bytes(pl));
+  const cudaError_t err = smat_launch_decode_step(q, k, v, o, S, cache, decode_table_plan(pl)->u_bf16 ? 1 : 0,
+                                                  pl->dtype == SMAT_BF16 ? 1 : 0, smat_type_of(pl->geo, t), pl->geo.B, pl->r,
+                                                  pl->p, pl->bh, static_cast<cudaStream_t>(cuda_stream), log_a_t, log_g);
   pl->launches = 1;
   return err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
 }

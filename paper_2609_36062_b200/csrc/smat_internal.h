@@ -149,7 +149,7 @@ cudaError_t smat_launch_state_read_dual_tc(const void* Xt, const void* Xn, const
 // One step of cached decoding: S += k vᵀ, o = qᵀ (U_type + S) for every head (fp32 running state).
 cudaError_t smat_launch_decode_step(const void* q, const void* k, const void* v, void* o, float* S, const void* U,
                                     int u_bf16, int in_bf16, int64_t type, int64_t types, int r, int p, int bh,
-                                    cudaStream_t st);
+                                    cudaStream_t st, const float* log_a = nullptr, float* log_g = nullptr);
 // d = 3 tabulation from a bf16 profile table on the fp32 ALUs (primes too large for the resident-matrix kernel).
 int smat_tabulate_d3_bf16_slab(const SmatGeo& geo, int64_t state_elems);
 cudaError_t smat_launch_tabulate_d3_bf16(const void* in, void* out, const SmatGeo& geo, int64_t state_elems, int bh,
