@@ -202,7 +202,7 @@ def make_inputs(w: synth.Workload, torch):
 class Runner:
     def __init__(self, w: synth.Workload, torch, binding, flags=0):
         self.w, self.torch = w, torch
-        if w.backward and w.variant == "plain":  # one workspace per step: the backward reuses the forward's F, U
+        if w.backward and w.variant in ("plain", "gated"):  # one workspace per step: the backward reuses the forward's F, U
             flags |= binding.FLAG_KEEP_FORWARD_TABLES
         flags |= {"gated": binding.FLAG_GATED, "normalized": binding.FLAG_NORMALIZED}.get(w.variant, 0)
         self.plan = binding.SmatPlan(w.batch, w.heads, w.T, w.d_k, w.d_v, w.d, w.chunk, w.dtype, flags=flags)
@@ -396,9 +396,9 @@ def path_report(w, geo, seconds_per_step, peaks, u_bytes=4, f_bytes=4, gated_tc_
         if gated_tc_forward and (ub, fb) != (4, 4):
             wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, 2, 2)
             if w.backward:   # the gated backward rebuilds the forward tables; fp32 tables where it runs on the ALU kernels
-                tb = 2 if gated_tc_forward == 2 else 4
-                wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, tb, tb, keep_forward_tables=False,
-                                                 f_bytes=tb, ubar_bytes=tb)
+                tb = 2 if gated_tc_forward == 2 else 4   # the tensor-core backward reuses the forward's tables
+                wk = wk + roofline.backward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, tb, tb,
+                                                 keep_forward_tables=gated_tc_forward == 2, f_bytes=tb, ubar_bytes=tb)
             return wk.scaled(w.bh)
         wk = roofline.forward_work(w.T, w.chunk, w.d_k, w.d_v, e, geo, ub, fb)
         if w.backward:  # bench.py's fwd+bwd step keeps the forward's tables; the adjoint tables follow the forward's

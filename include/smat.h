@@ -60,7 +60,10 @@ typedef enum { SMAT_F32 = 0, SMAT_BF16 = 1 } smat_dtype;
 #define SMAT_FLAG_ALG2_TABULATION 2u /* tabulate with the direct double loop of Algorithm 2 instead of the staged sums */
 #define SMAT_FLAG_KEEP_FORWARD_TABLES 8u /* smat_backward does not rebuild the profile and type tables F, U: the caller
                                             promises that `workspace` still holds what smat_forward wrote for the same
-                                            K, V with this plan (no other call on that workspace in between) */
+                                            K, V with this plan (no other call on that workspace in between).  With
+                                            SMAT_FLAG_GATED: smat_backward_gated right after smat_forward_gated of the
+                                            same inputs and gates (tensor-core shapes) reuses its tables likewise; after
+                                            any other call it rebuilds them */
 #define SMAT_FLAG_PER_TILE_STATES 4u /* tensor-core causal branch: store one incoming state per 128-token tile (scan, then
                                         independent tiles) instead of one per segment of tiles (two-level form) */
 

@@ -44,6 +44,8 @@ struct smat_plan {
   mutable int launches;
   mutable bool tile_states;       // the last call left one bf16 incoming state per 128-token tile at off_sin
   mutable bool kept_tile_states;  // the last forward left them at off_sin_tiles for the backward (KEEP_FORWARD_TABLES)
+  mutable bool kept_gated_forward;  // the last call was the tensor-core gated forward: λ, the rescaled K copies, U and the
+                                    // per-tile states are still in the workspace (used under KEEP_FORWARD_TABLES)
   // optional per-launch timing (smat_profile_enable): event k is recorded before launch k
   mutable bool profiling;
   mutable cudaEvent_t events[SMAT_MAX_STAGES + 1];
@@ -160,6 +162,7 @@ SmatGroupSpec group(const Ctx& cx, int mode) {
 // inner plan, that plan's (smat_check_status reads both).
 cudaError_t clear_status(const Ctx& cx) {
   const smat_plan* pl = cx.pl;
+  pl->kept_gated_forward = false;   // whatever pass starts here may overwrite what a gated forward left behind
   cudaError_t err = cudaMemsetAsync(cx.ws + pl->off_status, 0, 256, cx.st);
   if (err == cudaSuccess && pl->inner)
     err = cudaMemsetAsync(cx.ws + pl->off_inner + pl->inner->off_status, 0, 256, cx.st);
@@ -378,6 +381,7 @@ smat_status smat_plan_create(smat_plan** out, int batch, int heads, int64_t T, i
   pl->r = d_k; pl->p = d_v; pl->T = T; pl->c = chunk; pl->NC = T / chunk;
   pl->dtype = dtype; pl->flags = flags; pl->rp = (int64_t)d_k * d_v; pl->launches = 0;
   pl->profiling = false; pl->stages = 0; pl->tile_states = false; pl->kept_tile_states = false;
+  pl->kept_gated_forward = false;
   smat_status s = build_geometry(&pl->geo, T, chunk, d, q_override);
   if (s != SMAT_OK) { delete pl; return s; }
   const SmatGeo& g = pl->geo;
@@ -849,6 +853,7 @@ smat_status forward_gated_tc(Ctx& cx, const Gated& gt, const void* Q, const void
   SMAT_TRY(ci, "gated_chunk_output_tc", smat_launch_chunk_output_tc(Q, K, V, ci.ws + in->off_sin, ylr, lr ? in->geo.n : in->T,
                                                                      O, in->T, in->bh, status, ci.st, gt.lam));
   pl->launches = cx.launches + ci.launches;
+  pl->kept_gated_forward = ci.err == cudaSuccess;
   return ci.err == cudaSuccess ? SMAT_OK : SMAT_ERR_LAUNCH;
 }
 
@@ -864,7 +869,7 @@ bool gated_backward_on_tc(const smat_plan* pl) {
 // end of their tile) and D̄ (queries rescaled to the start of theirs, reverse order), and the fused tile kernel with
 // the decays on both score tiles and the row factors on the three state products.  dλ_t = q_t·dQ_t - k_t·dK_t.
 smat_status backward_gated_tc(Ctx& cx, const Gated& gt, const void* Q, const void* K, const void* V, const float* log_a,
-                              const void* dO, void* dQ, void* dK, void* dV, float* dlog_a) {
+                              const void* dO, void* dQ, void* dK, void* dV, float* dlog_a, bool after_gated_forward) {
   const smat_plan* pl = cx.pl;
   const smat_plan* in = pl->inner;
   const bool lr = !pl->geo.dense_G;
@@ -872,20 +877,23 @@ smat_status backward_gated_tc(Ctx& cx, const Gated& gt, const void* Q, const voi
   ci.rec = pl;
   int* status = reinterpret_cast<int*>(ci.ws + in->off_status);
   const int64_t n = in->geo.n;
-  SMAT_TRY(cx, "gate_prefix", smat_launch_head_scan(log_a, gt.lam, pl->T, pl->bh, 0, cx.st));
-  SMAT_TRY(cx, "gate_scale_k", smat_launch_gate_scale(K, nullptr, gt.kc, gt.lam, 1, 1, n, 128, pl->T, pl->r, pl->bh, cx.st));
-  SMAT_TRY(cx, "bwd_gate_scale_q", smat_launch_gate_scale(Q, nullptr, gt.qc, gt.lam, 0, 1, n, 128, pl->T, pl->r, pl->bh, cx.st));
-  if (lr) {
-    gate_scale(cx, "gate_scale_lr", K, Q, gt.lr, gt.lam, 2, pl->r);
-    gate_scale(cx, "bwd_gate_scale_lr", V, dO, gt.vlr, gt.lam, 2, pl->p);
+  // With KEEP_FORWARD_TABLES, right after the gated forward of the same inputs on this workspace: λ, the rescaled keys
+  // and the boundary-split copy, U and the per-tile incoming states are all still there.
+  const bool kept = (pl->flags & SMAT_FLAG_KEEP_FORWARD_TABLES) && after_gated_forward;
+  if (!kept) {
+    SMAT_TRY(cx, "gate_prefix", smat_launch_head_scan(log_a, gt.lam, pl->T, pl->bh, 0, cx.st));
+    SMAT_TRY(cx, "gate_scale_k", smat_launch_gate_scale(K, nullptr, gt.kc, gt.lam, 1, 1, n, 128, pl->T, pl->r, pl->bh, cx.st));
+    if (lr) gate_scale(cx, "gate_scale_lr", K, Q, gt.lr, gt.lam, 2, pl->r);
   }
+  SMAT_TRY(cx, "bwd_gate_scale_q", smat_launch_gate_scale(Q, nullptr, gt.qc, gt.lam, 0, 1, n, 128, pl->T, pl->r, pl->bh, cx.st));
+  if (lr) gate_scale(cx, "bwd_gate_scale_lr", V, dO, gt.vlr, gt.lam, 2, pl->p);
   ci.err = cx.err;
   char* sin = ci.ws + in->off_sin;
   char* dbar = ci.ws + in->off_dbar;
   char *lr_q = nullptr, *lr_k = nullptr, *lr_v = nullptr;
   if (lr) {
     const SmatGroupSpec types = group(ci, SMAT_GM_TYPE), profs = group(ci, SMAT_GM_PROFILE);
-    build_type_table(ci, gt.lr, V);
+    if (!kept) build_type_table(ci, gt.lr, V);
     if (in->ubar_tc)
       SMAT_TRY(ci, "bwd_pool_type_tc", smat_launch_pool_tc(gt.lr, dO, ci.ws + in->off_ubar, in->ubar_bf16, types, in->geo.B,
                                                            max_group_tokens(in, SMAT_GM_TYPE), in->T, in->bh, status, ci.st));
@@ -903,8 +911,9 @@ smat_status backward_gated_tc(Ctx& cx, const Gated& gt, const void* Q, const voi
     SMAT_TRY(ci, "bwd_dkdv_profile_tc", smat_launch_state_read_dual_tc(gt.vlr, gt.lr, ci.ws + in->off_fbar, lr_k, lr_v, profs,
                                                                         in->geo.P, in->T, in->bh, status, ci.st));
   }
-  SMAT_TRY(ci, "gated_chunk_scan_tc", smat_launch_chunk_scan_tc(gt.kc, V, sin, in->T, in->bh, n, lr ? 0 : 1, 0, status, ci.st,
-                                                                 gt.lam));
+  if (!kept)
+    SMAT_TRY(ci, "gated_chunk_scan_tc", smat_launch_chunk_scan_tc(gt.kc, V, sin, in->T, in->bh, n, lr ? 0 : 1, 0, status, ci.st,
+                                                                   gt.lam));
   SMAT_TRY(ci, "bwd_gated_suffix_scan_tc", smat_launch_chunk_scan_tc(gt.qc, dO, dbar, in->T, in->bh, n, lr ? 0 : 1, 1, status,
                                                                       ci.st, gt.lam));
   SMAT_TRY(ci, "bwd_gated_tiles_fused_tc", smat_launch_bwd_tiles_fused_tc(Q, K, V, dO, sin, dbar, lr_q, lr_k, lr_v,
@@ -1017,10 +1026,11 @@ smat_status smat_backward_gated(const smat_plan* pl, const void* Q, const void* 
   Ctx cx{pl, static_cast<cudaStream_t>(cuda_stream), static_cast<char*>(workspace), cudaSuccess, 0};
   pl->stages = 0;
   pl->tile_states = false;
+  const bool after_gated_forward = pl->kept_gated_forward;   // read before the pass resets it
   cx.err = clear_status(cx);
   const bool lr = !pl->geo.dense_G;
   const Gated gt = gated_buffers(cx);
-  if (gated_backward_on_tc(pl)) return backward_gated_tc(cx, gt, Q, K, V, log_a, dO, dQ, dK, dV, dlog_a);
+  if (gated_backward_on_tc(pl)) return backward_gated_tc(cx, gt, Q, K, V, log_a, dO, dQ, dK, dV, dlog_a, after_gated_forward);
   gated_forward_tables(cx, gt, Q, K, V, log_a);
   gate_scale(cx, "bwd_gate_scale_do", dO, nullptr, gt.doc, gt.lam, 0, pl->p);    // exp(λ_i - λ_{e(b-1)}) dO_i
   gate_scale(cx, "bwd_gate_scale_v", V, nullptr, gt.vc, gt.lam, 1, pl->p);       // exp(λ_{e(b)} - λ_j) v_j

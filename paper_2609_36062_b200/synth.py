@@ -70,6 +70,7 @@ WORKLOADS = {
     "t64k_d1_h4":    Workload("t64k_d1_h4", 1, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t64k_d2_h4":    Workload("t64k_d2_h4", 2, 1, 4, 65536, 128, 128, 128, "bf16", "normalised", 3),
     "t8k_d3_fwdbwd": Workload("t8k_d3_fwdbwd", 3, 8, 16, 8192, 128, 128, 64, "bf16", "normalised", 4, True),
+    "t8k_d3_h16_fwdbwd": Workload("t8k_d3_h16_fwdbwd", 3, 1, 16, 8192, 128, 128, 64, "bf16", "normalised", 4, True),
     # the 16 K configuration under user-supplied routing: every token hashed to a uniformly random cell / type
     "t16k_d4_hashed": Workload("t16k_d4_hashed", 4, 2, 16, 16384, 128, 128, 128, "bf16", "normalised", 2, False, "hashed"),
     # the variants of the "next" list on benchmark-shaped inputs

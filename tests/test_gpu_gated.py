@@ -172,3 +172,25 @@ def test_unit_gates_on_the_tensor_core_path_reproduce_the_ungated_forward():
     b = plain.forward(dev["q"], dev["k"], dev["v"])
     # the gated tile adds its two accumulators in the epilogue: same sums, another order, so not the same bits
     assert rel_err(to_numpy64(a), to_numpy64(b)) <= 4e-3
+
+
+def test_gated_backward_reuses_the_forward_tables_when_asked():
+    w = synth.Workload("gkeep", 3, 1, 2, 4096, 128, 128, 128, "bf16", "normalised", 35)
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    la = torch.from_numpy(_gates(w, 0.95, 5)).cuda()
+    keep = binding.SmatPlan(1, 2, w.T, 128, 128, 3, 128, "bf16", flags=binding.FLAG_GATED | binding.FLAG_KEEP_FORWARD_TABLES)
+    full = binding.SmatPlan(1, 2, w.T, 128, 128, 3, 128, "bf16", flags=binding.FLAG_GATED)
+    ws = keep.workspace(for_backward=True)
+    keep.forward_gated(dev["q"], dev["k"], dev["v"], la, workspace=ws)
+    a = keep.backward_gated(dev["q"], dev["k"], dev["v"], la, dev["do"], workspace=ws)
+    n_kept = keep.last_launch_count()
+    keep.check_status(ws)
+    b = full.backward_gated(dev["q"], dev["k"], dev["v"], la, dev["do"])
+    assert n_kept < full.last_launch_count()                 # no λ, no rescaled keys, no pooling, tabulation or state scan
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    # without a gated forward right before it, the same plan rebuilds everything
+    c = keep.backward_gated(dev["q"], dev["k"], dev["v"], la, dev["do"], workspace=ws)
+    assert keep.last_launch_count() == full.last_launch_count()
+    for x, y in zip(c, b):
+        assert torch.equal(x, y)
