@@ -378,6 +378,14 @@ class Runner:
         return [(n, acc[n] / steps) for n in order]
 
 
+def table_bytes(plan):
+    """Bytes per entry of the type and profile tables as the kernels that ran keep them (a gated plan whose passes run
+    on the tensor cores keeps bf16 tables in its inner plan)."""
+    if plan.gated_forward_uses_tensor_cores():
+        return 2, 2
+    return plan.type_table_element_bytes(), plan.profile_table_element_bytes()
+
+
 def gated_tc_mode(plan) -> int:
     """0: not a gated plan on the tensor cores; 1: its forward only; 2: forward and backward."""
     if not plan.gated_forward_uses_tensor_cores():
@@ -530,7 +538,7 @@ def run_native(args):
 
     line = None
     if rank == 0:
-        ub, fb = runner.plan.type_table_element_bytes(), runner.plan.profile_table_element_bytes()
+        ub, fb = table_bytes(runner.plan)
         stages = runner.stage_profile(min(steps, 10))
         line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps, "warmup": warm,
@@ -563,8 +571,7 @@ def run_native(args):
             rep = path_report(ws_, gg, s, peaks, r.plan.type_table_element_bytes(), r.plan.profile_table_element_bytes(),
                               gated_tc_mode(r.plan))
             st_ = r.stage_profile(3)
-            dom = dominant_kernel_report(ws_, gg, st_, peaks, r.plan.type_table_element_bytes(),
-                                         r.plan.profile_table_element_bytes())
+            dom = dominant_kernel_report(ws_, gg, st_, peaks, *table_bytes(r.plan))
             sweep.append({"workload": name, "dominant": {k: dom[k] for k in ("kernel", "bound", "achieved", "peak", "unit",
                                                                               "frac", "ms", "share")}, "value": ws_.tokens / s, "unit": "tokens/s", "ms_per_step": 1e3 * s,
                           "timing": "median of 15 steps after 5 warm-ups, one CUDA event pair per step",

@@ -139,7 +139,9 @@ def stage_work(name: str, T, c, r, p, e, geo, u_bytes=4, f_bytes=4) -> Work:
         "chunk_output_tc": Work(T * 129 * (r + p) + 2 * T * rp, 0, T * (2 * r + 2 * p) * e + tc_tiles * rp * 2 + m * p * 4),
         "output":      Work(T * (c + 1) * p, 0, T * c * 4 + T * p * e + T * p * 4 + T * p * e),
     }
-    return table.get(name, Work(0, 0, 0))
+    aliases = {"gated_chunk_scan_tc": "chunk_scan_tc", "gated_chunk_output_tc": "chunk_output_tc",
+               "bwd_gated_suffix_scan_tc": "bwd_suffix_scan_tc", "bwd_gated_tiles_fused_tc": "bwd_tiles_fused_tc"}
+    return table.get(aliases.get(name, name), Work(0, 0, 0))
 
 
 # Stages whose additions run on the fp32 ALUs (the other tabulations form the same sums on the tensor cores).
