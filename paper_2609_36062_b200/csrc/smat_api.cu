@@ -192,7 +192,13 @@ void end_stage(const smat_plan* pl, cudaStream_t st) {
 
 int64_t max_group_tokens(const smat_plan* pl, int mode, bool routed = false) {
   const SmatGeo& g = pl->geo;
-  if (routed && mode != SMAT_GM_CHUNK) return mode == SMAT_GM_PROFILE ? g.n : g.m;  // data-dependent: any size
+  if (routed && mode != SMAT_GM_CHUNK) {
+    // Data-dependent: any size.  The kernels loop over passes of their tile height, so this is only a hint for which
+    // height to instantiate: groups that hold few tokens on average get the small one (more CTAs per SM), and a heavy
+    // group simply takes more passes.
+    const int64_t tokens = mode == SMAT_GM_PROFILE ? g.n : g.m, groups = mode == SMAT_GM_PROFILE ? g.P : g.B;
+    return 2 * tokens <= 32 * groups ? 32 : tokens;
+  }
   if (mode == SMAT_GM_CHUNK) return pl->c;
   if (mode == SMAT_GM_PROFILE) return (g.n + g.P - 1) / g.P;
   return (g.m + g.B - 1) / g.B;

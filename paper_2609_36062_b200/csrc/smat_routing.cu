@@ -113,16 +113,16 @@ __global__ void __launch_bounds__(ROUTE_THREADS) routing_lists_kernel(const Rout
 }
 
 // Rows of tokens that belong to no group are never written by a routed read; whoever adds those rows afterwards must
-// find zeros there.  One warp per token: zero the row when the token's key is out of range.
+// find zeros there.  One thread per token reads its key; the (rare) token whose key is out of range zeroes its row.
 __global__ void zero_unrouted_rows_kernel(const int32_t* __restrict__ key, int64_t count, int64_t G, int64_t first,
                                           uint8_t* __restrict__ rows, int64_t T, int row_bytes, int64_t total) {
-  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t w = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (w >= total) return;
   const int32_t k = key[w];
   if (k >= 0 && k < G) return;
   const int64_t bh = w / count, t = first + (w - bh * count);
   uint4* dst = reinterpret_cast<uint4*>(rows + (bh * T + t) * row_bytes);
-  for (int i = threadIdx.x & 31; i < row_bytes / 16; i += 32) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = 0; i < row_bytes / 16; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 }  // namespace
@@ -130,8 +130,7 @@ __global__ void zero_unrouted_rows_kernel(const int32_t* __restrict__ key, int64
 cudaError_t smat_launch_zero_unrouted(const int32_t* key, int64_t count, int64_t G, int64_t first, void* rows, int64_t T,
                                       int row_bytes, int bh, cudaStream_t st) {
   const int64_t total = (int64_t)bh * count;
-  const int64_t threads = total * 32;
-  zero_unrouted_rows_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(key, count, G, first,
+  zero_unrouted_rows_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(key, count, G, first,
                                                                                static_cast<uint8_t*>(rows), T, row_bytes, total);
   return cudaGetLastError();
 }
