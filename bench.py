@@ -71,27 +71,29 @@ def oracle_sample(w: synth.Workload, budget_s: float, backward: bool):
         threads = os.cpu_count() or 1
     geo = so.geometry(w.T, w.chunk, w.d)
     names = ("q", "k", "v", "do") if backward else ("q", "k", "v")
-    host = {x: synth.as_float64(w, synth.stored(w, x, 0)) for x in names}
     rng = np.random.default_rng(0)
-    order = rng.permutation(w.T)
-    done, t0 = 0, time.perf_counter()
+    done, heads_touched, t0 = 0, 0, time.perf_counter()
     batch = 8
-    while True:
-        rows = order[done:done + batch]
-        if len(rows) == 0:
-            break
-        so.forward_rows(host["q"], host["k"], host["v"], geo, rows)
-        if backward:
-            so.dq_rows(host["q"], host["k"], host["v"], host["do"], geo, rows)
-            so.dkdv_cols(host["q"], host["k"], host["v"], host["do"], geo, rows)
-        done += len(rows)
+    for head in range(w.bh):            # head after head, rows in random order, until the time budget is used up
+        host = {x: synth.as_float64(w, synth.stored(w, x, head)) for x in names}
+        order = rng.permutation(w.T)
+        heads_touched += 1
+        pos = 0
+        while pos < w.T and time.perf_counter() - t0 <= budget_s:
+            rows = order[pos:pos + batch]
+            so.forward_rows(host["q"], host["k"], host["v"], geo, rows)
+            if backward:
+                so.dq_rows(host["q"], host["k"], host["v"], host["do"], geo, rows)
+                so.dkdv_cols(host["q"], host["k"], host["v"], host["do"], geo, rows)
+            pos += len(rows)
+            done += len(rows)
         if time.perf_counter() - t0 > budget_s:
             break
     dt = time.perf_counter() - t0
     # a token is done when its row is done in every head of its batch element
     tokens_per_s = done / dt / w.heads
     what = (f"{done} uniformly sampled rows of O" + (" and of dQ, dK, dV" if backward else "") +
-            f" of head 0 ({dt:.1f} s), scaled by 1/heads to whole tokens")
+            f" of the first {heads_touched} head(s) ({dt:.1f} s), scaled by 1/heads to whole tokens")
     return tokens_per_s, threads, what, done, dt
 
 
