@@ -194,3 +194,27 @@ def test_gated_backward_reuses_the_forward_tables_when_asked():
     assert keep.last_launch_count() == full.last_launch_count()
     for x, y in zip(c, b):
         assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("flag", [binding.FLAG_ALU_TABULATION, binding.FLAG_ALG2_TABULATION])
+def test_gated_passes_with_the_other_tabulations_of_the_inner_plan(flag):
+    """The tabulation flags reach the plan that the gated passes run through: fp32 tables there send the typed read
+    (and, for the literal Algorithm 2, the whole backward) to the fp32-ALU kernels; the results must not change."""
+    w = synth.Workload("gflag", 3, 1, 2, 1024, 128, 128, 128, "bf16", "normalised", 36)
+    host, dev = device_inputs(w, ("q", "k", "v", "do"))
+    la = _gates(w, 0.93, 6)
+    la_dev = torch.from_numpy(la).cuda()
+    plan = binding.SmatPlan(1, 2, w.T, 128, 128, 3, 128, "bf16", flags=binding.FLAG_GATED | flag)
+    assert plan.gated_forward_uses_tensor_cores()
+    O = plan.forward_gated(dev["q"], dev["k"], dev["v"], la_dev)
+    dQ, dK, dV, dla = plan.backward_gated(dev["q"], dev["k"], dev["v"], la_dev, dev["do"])
+    plan.check_status()
+    M = so.dense_mask(w.T, 128, 3)
+    for h in range(w.bh):
+        Q64, K64, V64, G64 = (synth.as_float64(w, host[x][h]) for x in ("q", "k", "v", "do"))
+        lah = la[h].astype(np.float64)
+        assert rel_err(to_numpy64(O[0, h]), so.gated_forward_dense(Q64, K64, V64, M, lah)) <= TOL["bf16"]
+        rq, rk, rv, rl = so.gated_backward_dense(Q64, K64, V64, G64, M, lah)
+        for name, got, ref in (("dQ", dQ, rq), ("dK", dK, rk), ("dV", dV, rv)):
+            assert rel_err(to_numpy64(got[0, h]), ref) <= TOL["bf16"], (name, h)
+        assert rel_err(dla[h].double().cpu().numpy(), rl) <= 5e-2

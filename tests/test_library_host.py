@@ -143,3 +143,32 @@ def test_tabulation_kernel_shared_memory_map_is_disjoint(q):
     """Ring slots, per-slot extra rows, the output-row table and the barrier words of the tensor-core tabulation kernel
     never overlap and no load box or staged tile leaves its slot, for every launch shape of every prime it accepts."""
     assert binding.load_library().smat_debug_tabulation_layout_ok(q) == 1
+
+
+def test_gated_plans_size_their_inner_plan_and_decode_cache():
+    """A gated plan on a tensor-core shape carries an ungated plan of its own for both passes: its workspace holds that
+    plan's backward workspace as a region, its decode cache the bf16 type table, the running state and one word per
+    head; other shapes, and SIMT_ONLY, have no inner plan and keep fp32 tables."""
+    shape = (2, 4, 4096, 128, 128, 3, 64, "bf16")
+    gated = binding.SmatPlan(*shape, flags=binding.FLAG_GATED)
+    plain = binding.SmatPlan(*shape, flags=binding.FLAG_PER_TILE_STATES)
+    alu = binding.SmatPlan(*shape, flags=binding.FLAG_GATED | binding.FLAG_SIMT_ONLY)
+    assert not gated.uses_tensor_cores()                        # the gated plan itself keeps the fp32-ALU layout
+    assert gated.gated_forward_uses_tensor_cores() and gated.gated_backward_uses_tensor_cores()
+    assert not alu.gated_forward_uses_tensor_cores() and not alu.gated_backward_uses_tensor_cores()
+    assert not plain.gated_forward_uses_tensor_cores()
+    inner = plain.workspace_bytes(True)
+    assert alu.workspace_bytes(False) + inner <= gated.workspace_bytes(False) <= alu.workspace_bytes(False) + inner + 4096
+    assert gated.workspace_bytes(True) - gated.workspace_bytes(False) == alu.workspace_bytes(True) - alu.workspace_bytes(False)
+    g = gated.geometry()
+    bh, state = 8, 128 * 128
+    lib = binding.load_library()
+    assert lib.smat_decode_cache_bytes(gated.handle) == bh * g.B * state * 2 + bh * state * 4 + 256
+    assert lib.smat_decode_cache_bytes(alu.handle) == bh * g.B * state * 4 + bh * state * 4 + 256
+    assert lib.smat_decode_cache_bytes(plain.handle) == bh * g.B * state * 2 + bh * state * 4
+    # the tabulation flags reach the inner plan: fp32 tables there (the literal Algorithm 2) mean an fp32-ALU gated backward
+    odd = binding.SmatPlan(*shape, flags=binding.FLAG_GATED | binding.FLAG_ALG2_TABULATION)
+    assert odd.gated_forward_uses_tensor_cores() and not odd.gated_backward_uses_tensor_cores()
+    # a block boundary that is not a whole tile: no inner plan
+    ragged = binding.SmatPlan(1, 2, 640, 128, 128, 3, 32, "bf16", flags=binding.FLAG_GATED)
+    assert not ragged.gated_forward_uses_tensor_cores()
